@@ -1,0 +1,181 @@
+/*
+ * libdisco -- batched, trace-driven evaluation of DiSCo's cost-aware dispatch
+ * and token-level migration policy (arXiv 2502.11417) on one NVIDIA B200.
+ *
+ * For every (request, policy) pair the library derives the dispatch decision
+ * (server only, device only, wait-then-race; Sec. 4.2, Algorithms 1-3), plays
+ * the decode stream out token by token with per-token jitter, paced delivery
+ * and buffer-based migration (Sec. 4.3, Eq. 4-6), prices it (Appendix E,
+ * Eq. 8), reduces the pairs to per-policy QoE statistics (Sec. 5.1: mean and
+ * tail TTFT, P99 TBT, cost) and picks a policy under a cost cap.
+ *
+ * Conventions
+ *  - Plain C ABI.  Every function returns 0 on success or a negative status:
+ *    DISCO_EINVAL (bad argument or input value), DISCO_ENOMEM, DISCO_ECUDA
+ *    (a CUDA call failed), DISCO_EINFEASIBLE (selection only).  Nothing aborts
+ *    or throws across the boundary; disco_last_error() describes the last
+ *    failure of the calling thread.
+ *  - "host" / "device" on a pointer says where the memory must live.  Inputs
+ *    are never modified.  The context owns every byte it allocates; per-pair
+ *    output arrays are allocated and owned by the caller.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *  - Time is kept internally in integer microsecond ticks, so that results do
+ *    not depend on the order of the parallel reductions.
+ *  - There is no CPU fallback: without a CUDA device every call fails.
+ */
+#ifndef DISCO_H
+#define DISCO_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DISCO_NBINS 864          /* histogram bins: 32 per octave of ticks */
+#define DISCO_MAX_PROMPT 4096
+#define DISCO_MAX_OUTPUT 8192
+
+#define DISCO_EINVAL (-1)
+#define DISCO_ENOMEM (-2)
+#define DISCO_ECUDA (-3)
+#define DISCO_EINFEASIBLE (-4)
+
+/* dispatch decisions (per-pair output `decision`) */
+#define DISCO_SERVER_ONLY 0      /* device never started: the server answered within the wait */
+#define DISCO_DEVICE_ONLY 1      /* Algorithm 3: prompt shorter than l_th */
+#define DISCO_RACE 2             /* both endpoints ran; the first token won */
+
+/* policy flags */
+#define DISCO_FLAG_MIGRATION 1u  /* token-level migration on (Sec. 4.3) */
+#define DISCO_FLAG_PACING 2u     /* delivery buffer: tokens handed over no faster than r_c */
+#define DISCO_MODE_AUTO (0u << 2)               /* Algorithm 1 decides from the costs */
+#define DISCO_MODE_DEVICE_CONSTRAINED (1u << 2) /* force Algorithm 2 */
+#define DISCO_MODE_SERVER_CONSTRAINED (2u << 2) /* force Algorithm 3 */
+
+/* Server endpoint (Sec. 4.1 cost model; Sec. 3 decode characteristics). */
+typedef struct {
+    float tbt_s;       /* mean time between decode tokens, seconds, > 0 */
+    float jitter;      /* per-token TBT varies uniformly by +- this fraction, in [0,1] */
+    float c_prefill;   /* c^p_s, cost per prompt token */
+    float c_decode;    /* c^d_s, cost per generated token */
+} disco_server_profile_t;
+
+/* Device endpoint: TTFT is linear in the prompt length, T_d(l) = l / prefill_tps + intercept (Sec. 4.2). */
+typedef struct {
+    float prefill_tps;        /* prompt tokens per second, > 0 */
+    float ttft_intercept_s;   /* c of T_d = k l + c, >= 0 */
+    float decode_tps;         /* generated tokens per second, > 0 */
+    float jitter;             /* as for the server */
+    float c_prefill;          /* c^p_d, energy cost per prompt token */
+    float c_decode;           /* c^d_d */
+    float lambda;             /* exchange rate energy -> money (Eq. 8) */
+} disco_device_profile_t;
+
+/* A request trace.  A request belongs to group (server_profile, device_profile);
+ * each group has its own prompt-length distribution p(l) and server-TTFT
+ * distribution F (Algorithm 1 inputs), both taken from the group's own rows. */
+typedef struct {
+    uint64_t n;                       /* requests, may be 0, < 2^31 */
+    const int32_t* prompt_len;        /* [n], 1..DISCO_MAX_PROMPT */
+    const int32_t* output_len;        /* [n], 1..DISCO_MAX_OUTPUT */
+    const float*   server_ttft_s;     /* [n], finite, > 0, <= 2000 */
+    const uint8_t* server_profile;    /* [n] or NULL (all 0) */
+    const uint8_t* device_profile;    /* [n] or NULL (all 0) */
+    const disco_server_profile_t* servers;  /* host, [n_servers] */
+    uint32_t n_servers;               /* >= 1; n_servers * n_devices <= 64 */
+    const disco_device_profile_t* devices;  /* host, [n_devices] */
+    uint32_t n_devices;
+    uint32_t arrays_on_device;        /* 0: the five [n] arrays are host memory; 1: device memory */
+} disco_trace_desc_t;
+
+/* One policy setting (Algorithm 1 inputs b, alpha; Eq. 4 overhead; Eq. 6 t_m, r_c). */
+typedef struct {
+    float budget;          /* b in [0,1] */
+    float alpha;           /* tail ratio in (0,1) */
+    float mig_threshold;   /* Overhead_migration of Eq. 4, cost units, >= 0; +INF = never migrate */
+    float t_m_s;           /* estimated migration time, seconds; buffer B = ceil(r_c t_m) tokens */
+    float r_c;             /* consumption rate, tokens/s, > 0 */
+    uint32_t flags;        /* DISCO_FLAG_* | DISCO_MODE_* */
+} disco_policy_t;
+
+/* Optional per-pair outputs, device memory, each [P][n] with requests
+ * contiguous (index p * n + i, i = position in the caller's trace); any
+ * member may be NULL. */
+typedef struct {
+    float *ttft_s, *tbt_mean_s, *tbt_max_s, *cost;
+    uint32_t *tok_server, *tok_device;   /* generated tokens per endpoint; they sum to output_len */
+    uint32_t *mig_at;                    /* hand-off index m (source generated tokens 1..m), 0 = no migration */
+    uint16_t *delayed;                   /* tokens generated after their delivery slot during a migration */
+    uint8_t *decision;                   /* DISCO_SERVER_ONLY / DEVICE_ONLY / RACE */
+} disco_pair_out_t;
+
+typedef struct {
+    double mean_ttft_s, total_cost;
+    float p50_ttft_s, p95_ttft_s, p99_ttft_s;   /* lower edge of the histogram bin holding the nearest rank */
+    float p99_tbt_s;                            /* pooled over every inter-token interval of every request */
+    int32_t bin_p50_ttft, bin_p95_ttft, bin_p99_ttft, bin_p99_tbt;
+    uint64_t n_requests, n_intervals;
+    uint64_t n_server_only, n_device_only, n_race, n_device_started, n_device_won, n_migrations;
+    uint64_t tok_server, tok_device, prefill_tok_server, prefill_tok_device, delayed_tokens;
+} disco_policy_stats_t;
+
+/* What Algorithms 1-3 return for one (group, policy), for inspection. */
+typedef struct {
+    int32_t device_constrained;   /* Algorithm 1 */
+    int32_t l_th;                 /* Algorithm 3 / Eq. 3: prompts shorter than this run on the device only */
+    int32_t l_star;               /* Algorithm 2: shorter prompts wait 0, this length waits w_star, longer ones w_tail */
+    int32_t B;                    /* Eq. 6 buffer, tokens */
+    int64_t w_star, w_tail, tau;  /* ticks (microseconds) */
+} disco_prep_t;
+
+typedef struct disco_ctx disco_ctx_t;
+
+/* Loads a trace (Algorithm 1's inputs): copies the arrays to the device if
+ * they are host memory, converts times to ticks and builds, per group, the
+ * prompt-length histogram p(l) and the sorted server-TTFT sample F.
+ * *ctx must be NULL (a context is created) or a context from an earlier call
+ * (it is reloaded in place, reusing its memory).  Synchronises `stream`.
+ * DISCO_EINVAL if a value is out of the ranges above or a profile is invalid. */
+int disco_load_trace(disco_ctx_t** ctx, const disco_trace_desc_t* desc, void* stream);
+
+/* Evaluates every (request, policy) pair: dispatch (Sec. 4.2), play-out and
+ * migration (Sec. 4.3), cost (Eq. 8); accumulates the per-policy sums and
+ * histograms inside the context and, if `out` is not NULL, writes the per-pair
+ * arrays.  pol is host memory [P], P >= 1.  `seed` keys the per-token jitter
+ * hash.  Asynchronous on `stream`; results are read with disco_reduce_stats.
+ * DISCO_EINVAL for a bad policy, or when a stream could outlast 2^31 ticks. */
+int disco_eval_policies(disco_ctx_t* ctx, const disco_policy_t* pol, uint32_t P, uint64_t seed,
+                        const disco_pair_out_t* out, void* stream);
+
+/* Finishes the reductions of the last evaluation (Sec. 5.1 metrics) and copies
+ * P records to host memory `stats`.  Synchronises `stream`. */
+int disco_reduce_stats(disco_ctx_t* ctx, disco_policy_stats_t* stats, void* stream);
+
+/* Picks, among the policies of the last reduction whose total cost is within
+ * cost_cap and whose P99 TBT is within tbt_slo_s, the one with the smallest
+ * P99 TTFT (then mean TTFT, then cost, then index) -- the objectives of
+ * Sec. 4.1.  *best (host) receives its index.  If none is feasible, returns
+ * DISCO_EINFEASIBLE and *best is the cheapest policy.  Synchronises. */
+int disco_select_policy(disco_ctx_t* ctx, double cost_cap, float tbt_slo_s, int32_t* best, void* stream);
+
+/* Copies policy p's TTFT and pooled TBT histograms (host, DISCO_NBINS each; either may be NULL). */
+int disco_get_histograms(disco_ctx_t* ctx, uint32_t p, uint64_t* ttft_hist, uint64_t* tbt_hist, void* stream);
+
+/* Copies what Algorithms 1-3 produced for group g = server_profile * n_devices + device_profile, policy p. */
+int disco_get_prep(disco_ctx_t* ctx, uint32_t g, uint32_t p, disco_prep_t* out, void* stream);
+
+/* Copies group g's tables to host memory (any may be NULL): requests per prompt
+ * length cnt[DISCO_MAX_PROMPT+1], the 257 equally spaced order statistics of F,
+ * and up to `n_sorted` of the smallest sorted TTFT ticks.  Returns the group's
+ * request count, or a negative status. */
+int64_t disco_get_group_tables(disco_ctx_t* ctx, uint32_t g, int64_t* cnt, int32_t* knots,
+                               int32_t* sorted_ticks, uint64_t n_sorted, void* stream);
+
+void disco_free_trace(disco_ctx_t* ctx);
+const char* disco_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

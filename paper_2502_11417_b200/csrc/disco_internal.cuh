@@ -1,0 +1,133 @@
+// Internal declarations shared by the translation units of libdisco.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "disco.h"
+
+namespace disco {
+
+constexpr int kNBins = DISCO_NBINS;
+constexpr int kMaxPrompt = DISCO_MAX_PROMPT;
+constexpr int kMaxOutput = DISCO_MAX_OUTPUT;
+constexpr int kNKnots = 257;
+constexpr int kMaxGroups = 64;
+
+// ---- per-group constants, ticks and costs (one per (server, device) profile pair) ----
+struct GroupConst {
+    int32_t T_srv, J_srv;        // server decode interval and jitter amplitude, ticks
+    int32_t T_dev, J_dev;        // device decode interval and jitter amplitude
+    int32_t kappa, c0;           // device TTFT = kappa * l + c0
+    int32_t auto_device_constrained;   // Algorithm 1 evaluated on this group's costs
+    int32_t candidate;           // 0 none, 1 a winning server may migrate (it is the dearer decoder), 2 a winning device may
+    float delta_c;               // |c^d_s - lambda c^d_d|  (Eq. 5)
+    float cps, cds, lcpd, lcdd;  // fp32 cost rates, device ones already in money
+    double cps_d, cds_d, cpd_d, cdd_d, lambda_d;   // fp64 rates for the totals
+};
+
+// ---- per-policy constants derived on the host ----
+struct PolicyConst {
+    float budget, alpha, theta;
+    uint32_t flags;
+    int32_t tau, B;
+    int32_t cls;                 // timeline class (policies with equal tau, B, pacing share play-outs)
+    int32_t mode;                // 0 Algorithm 1 decides, 1 device-constrained, 2 server-constrained
+};
+
+// ---- what Algorithms 1-3 produce for one (group, policy) ----
+struct Prep {
+    int32_t device_constrained;
+    int32_t l_th;
+    int32_t l_star;
+    int32_t w_star, w_tail;
+    float theta;
+    int32_t mig_on;
+    int32_t pad;
+};
+
+// ---- a timeline class: the parameters a play-out depends on besides the request ----
+struct ClassConst {
+    int32_t tau_eff;             // tau when pacing is on, else 0 (then delivery = generation)
+    int32_t tau;                 // tau of the policies (for the "equals tau" fast count)
+    int32_t B;
+    int32_t pacing, mig_any;
+    // dense windows of histogram bins that regular inter-token intervals can fall in
+    int32_t W[3];                // bins per request for the server, device and migrated timelines
+    int32_t lo[kMaxGroups][3];   // first bin of each window, per group
+    int32_t ktau[kMaxGroups][3]; // index of bin(tau) inside the window, or -1
+};
+
+// Per-request summaries of the up to three distinct decode timelines of a class.
+struct TimelineRec {
+    uint32_t *sum[3], *max[3];   // d_n - d_1 and the largest TBT, ticks ([n] each)
+    uint32_t* stall;             // TBT of the first token after a hand-off
+    uint16_t *m, *delayed;       // hand-off index (0 = buffer never fills) and delayed tokens
+    uint16_t* win[3];            // [n][W[c]] counts per window bin
+};
+
+struct TraceDev {
+    uint32_t n;
+    int32_t n_groups;
+    const int32_t* S;            // server TTFT ticks, internal order (requests partitioned by group)
+    const uint16_t *l, *nout;
+    const uint32_t* orig;        // caller's index of each request
+    const uint32_t* grp_off;     // [G+1]
+};
+
+struct Chunk { uint32_t start, len; int32_t g; int32_t pad; };
+
+enum AccSlot { A_SERVER_ONLY = 0, A_DEVICE_ONLY, A_RACE, A_STARTED, A_DEVICE_WON, A_MIGR, A_TOK_DEVICE,
+               A_PRE_SERVER, A_PRE_DEVICE, A_DELAYED, A_TTFT_LO, A_TTFT_HI, kNAcc };
+
+// ---- device helpers -------------------------------------------------------------------------------------
+
+// Jitter hash: xorshift-multiply finaliser over a per-request key plus token counter.
+__host__ __device__ __forceinline__ uint32_t mix32(uint32_t x) {
+    x ^= x >> 16; x *= 0xA54FF53Bu;
+    x ^= x >> 15; x *= 0x510E527Fu;
+    x ^= x >> 16;
+    return x;
+}
+constexpr uint32_t kHashSeed = 0x6A09E667u, kHashReq = 0xBB67AE85u, kHashTok = 0x3C6EF373u;
+
+__host__ __device__ __forceinline__ uint32_t seed_key(uint64_t seed) {
+    return mix32((uint32_t)seed ^ kHashSeed) ^ (uint32_t)(seed >> 32);
+}
+
+#ifdef __CUDACC__
+// Histogram bin of a tick count: exact below 32, then 32 bins per octave.  The exponent and the five
+// leading mantissa bits come from the float representation (round-toward-zero keeps them exact).
+__device__ __forceinline__ int bin_of_ticks(uint32_t t) {
+    if (t < 32u) return (int)t;
+    int b = (int)(__float_as_uint(__uint2float_rz(t)) >> 18) - ((127 + 4) << 5);
+    return min(b, kNBins - 1);
+}
+#endif
+
+// Host-side bin (same partition of the axis, integer arithmetic).
+inline int host_bin_of_ticks(int64_t t) {
+    if (t < 0) t = 0;
+    if (t < 32) return (int)t;
+    int e = 63 - __builtin_clzll((unsigned long long)t);
+    int64_t b = 32 * (int64_t)(e - 4) + ((t >> (e - 5)) & 31);
+    return (int)(b < kNBins - 1 ? b : kNBins - 1);
+}
+
+// ---- launch wrappers (defined in the kernel translation units) -------------------------------------------
+cudaError_t launch_prep(const PolicyConst* pol, uint32_t P, int G, const GroupConst* gc, const int64_t* cum_mass,
+                        const uint32_t* cnt, const int32_t* sorted, const uint32_t* grp_off, Prep* prep,
+                        cudaStream_t st);
+cudaError_t launch_timeline(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const int32_t* knots,
+                            uint64_t seed, TimelineRec rec, int32_t* err, cudaStream_t st);
+cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const Prep* prep, uint32_t P,
+                         const uint32_t* pol_list, uint32_t n_list, const Chunk* chunks, uint32_t n_chunks,
+                         TimelineRec rec, disco_pair_out_t out, uint64_t* acc, uint64_t* hist_ttft,
+                         uint64_t* hist_tbt, cudaStream_t st);
+cudaError_t launch_finalize(uint32_t P, int G, const GroupConst* gc, const uint64_t* acc, const uint64_t* hist_ttft,
+                            const uint64_t* hist_tbt, const uint64_t* grp_sum_n, const uint32_t* grp_off,
+                            disco_policy_stats_t* stats, cudaStream_t st);
+cudaError_t launch_select(const disco_policy_stats_t* stats, uint32_t P, double cost_cap, float tbt_slo_s,
+                          int32_t* result /* [2]: status, index */, cudaStream_t st);
+
+}  // namespace disco

@@ -1,0 +1,238 @@
+// Trace ingestion on the device: tick conversion and validation, per-group prompt-length histogram,
+// stable partition of the requests by group, radix sort of the server-TTFT ticks (the empirical F of
+// Algorithm 1), cumulative input-token mass (Eq. 3) and the quantile knots of F.
+#include "load.cuh"
+
+namespace disco {
+
+namespace {
+
+constexpr int kIngestThreads = 256;
+
+__global__ void k_ingest(uint32_t n, const int32_t* __restrict__ prompt, const int32_t* __restrict__ outlen,
+                         const float* __restrict__ ttft, const uint8_t* __restrict__ sp,
+                         const uint8_t* __restrict__ dp, uint32_t ns, uint32_t nd, uint64_t* __restrict__ keys,
+                         uint32_t* __restrict__ cnt, unsigned long long* __restrict__ grp_sum_n,
+                         uint32_t* __restrict__ max_n, int32_t* __restrict__ err) {
+    __shared__ unsigned long long s_sum[kMaxGroups];
+    __shared__ uint32_t s_max;
+    const int G = (int)(ns * nd);
+    for (int g = threadIdx.x; g < G; g += blockDim.x) s_sum[g] = 0;
+    if (threadIdx.x == 0) s_max = 0;
+    __syncthreads();
+    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+        const int32_t l = prompt[i], o = outlen[i];
+        const float t = ttft[i];
+        const uint32_t s = sp ? sp[i] : 0u, d = dp ? dp[i] : 0u;
+        int bad = 0;
+        if (l < 1 || l > kMaxPrompt) bad = 1;
+        else if (o < 1 || o > kMaxOutput) bad = 2;
+        else if (!(t > 0.0f) || !(t <= 2000.0f)) bad = 3;      // NaN fails both comparisons
+        else if (s >= ns || d >= nd) bad = 4;
+        if (bad) {
+            if (atomicCAS(&err[0], 0, bad) == 0) err[1] = (int32_t)i;
+            keys[i] = 0;
+            continue;
+        }
+        // ticks = nearest integer (ties to even) of the fp64 product, as a host llrint would give
+        const long long S = __double2ll_rn(__dmul_rn((double)t, 1e6));
+        const uint32_t g = s * nd + d;
+        keys[i] = ((uint64_t)g << 32) | (uint32_t)S;
+        atomicAdd(&cnt[g * (kMaxPrompt + 1) + l], 1u);
+        atomicAdd(&s_sum[g], (unsigned long long)o);
+        atomicMax(&s_max, (uint32_t)o);
+    }
+    __syncthreads();
+    for (int g = threadIdx.x; g < G; g += blockDim.x)
+        if (s_sum[g]) atomicAdd(&grp_sum_n[g], s_sum[g]);
+    if (threadIdx.x == 0 && s_max) atomicMax(max_n, s_max);
+}
+
+// ---- one stable LSD radix pass over 64-bit keys (8-bit digit), optional 32-bit payload -------------------
+constexpr int kRadixThreads = 256;
+constexpr int kRadixWarps = kRadixThreads / 32;
+
+__global__ void k_radix_hist(const uint64_t* __restrict__ keys, uint32_t n, uint32_t per_block, int shift,
+                             uint32_t* __restrict__ counts /* [256][gridDim.x] */) {
+    __shared__ uint32_t h[256];
+    h[threadIdx.x] = 0;
+    __syncthreads();
+    const uint32_t lo = min(n, blockIdx.x * per_block), hi = min(n, lo + per_block);
+    for (uint32_t i = lo + threadIdx.x; i < hi; i += kRadixThreads)
+        atomicAdd(&h[(uint32_t)(keys[i] >> shift) & 255u], 1u);
+    __syncthreads();
+    counts[threadIdx.x * gridDim.x + blockIdx.x] = h[threadIdx.x];
+}
+
+// exclusive scan of `m` counters by one block of 1024 threads
+__global__ void k_scan_counts(uint32_t* __restrict__ counts, uint32_t m) {
+    __shared__ uint32_t part[1024];
+    const uint32_t per = (m + 1023u) / 1024u;
+    const uint32_t lo = min(m, threadIdx.x * per), hi = min(m, lo + per);
+    uint32_t s = 0;
+    for (uint32_t i = lo; i < hi; ++i) s += counts[i];
+    part[threadIdx.x] = s;
+    __syncthreads();
+    for (int off = 1; off < 1024; off <<= 1) {
+        uint32_t v = threadIdx.x >= (unsigned)off ? part[threadIdx.x - off] : 0u;
+        __syncthreads();
+        part[threadIdx.x] += v;
+        __syncthreads();
+    }
+    uint32_t run = part[threadIdx.x] - s;
+    for (uint32_t i = lo; i < hi; ++i) { const uint32_t c = counts[i]; counts[i] = run; run += c; }
+}
+
+__global__ void k_radix_scatter(const uint64_t* __restrict__ keys_in, uint64_t* __restrict__ keys_out,
+                                const uint32_t* __restrict__ pay_in, uint32_t* __restrict__ pay_out, uint32_t n,
+                                uint32_t per_block, int shift, const uint32_t* __restrict__ offsets) {
+    __shared__ uint32_t run[256];                 // next output slot of each digit for this block
+    __shared__ uint32_t wcnt[kRadixWarps][256];   // keys of each digit per warp in the current slab
+    const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    run[threadIdx.x] = offsets[threadIdx.x * gridDim.x + blockIdx.x];
+    const uint32_t lo = min(n, blockIdx.x * per_block), hi = min(n, lo + per_block);
+    for (uint32_t base = lo; base < hi; base += kRadixThreads) {
+        for (int k = 0; k < kRadixWarps; ++k) wcnt[k][threadIdx.x] = 0;
+        __syncthreads();
+        const uint32_t i = base + threadIdx.x;
+        const bool live = i < hi;
+        uint64_t key = 0;
+        uint32_t dig = 256u + (uint32_t)lane;     // dead lanes get digits of their own
+        if (live) { key = keys_in[i]; dig = (uint32_t)(key >> shift) & 255u; }
+        const uint32_t peers = __match_any_sync(0xFFFFFFFFu, dig);
+        const uint32_t rank = __popc(peers & ((1u << lane) - 1u));
+        if (live && rank == 0) wcnt[w][dig] = __popc(peers);
+        __syncthreads();
+        if (live) {
+            uint32_t before = 0;
+            for (int k = 0; k < w; ++k) before += wcnt[k][dig];
+            const uint32_t pos = run[dig] + before + rank;
+            keys_out[pos] = key;
+            if (pay_out) pay_out[pos] = pay_in ? pay_in[i] : i;
+        }
+        __syncthreads();
+        uint32_t tot = 0;
+        for (int k = 0; k < kRadixWarps; ++k) tot += wcnt[k][threadIdx.x];
+        run[threadIdx.x] += tot;
+        __syncthreads();
+    }
+}
+
+__global__ void k_gather(uint32_t n, const uint32_t* __restrict__ orig_in, const uint64_t* __restrict__ keys,
+                         const int32_t* __restrict__ prompt, const int32_t* __restrict__ outlen,
+                         int32_t* __restrict__ S, uint16_t* __restrict__ l, uint16_t* __restrict__ nout,
+                         uint32_t* __restrict__ orig) {
+    for (uint32_t k = blockIdx.x * blockDim.x + threadIdx.x; k < n; k += gridDim.x * blockDim.x) {
+        const uint32_t i = orig_in ? orig_in[k] : k;
+        S[k] = (int32_t)(uint32_t)keys[i];
+        l[k] = (uint16_t)prompt[i];
+        nout[k] = (uint16_t)outlen[i];
+        orig[k] = i;
+    }
+}
+
+__global__ void k_low_words(uint32_t n, const uint64_t* __restrict__ keys, int32_t* __restrict__ out) {
+    for (uint32_t k = blockIdx.x * blockDim.x + threadIdx.x; k < n; k += gridDim.x * blockDim.x)
+        out[k] = (int32_t)(uint32_t)keys[k];
+}
+
+// One block per group: cumulative input-token mass cum[L] = sum_{l<L} l*cnt[l], L = 0..4097, and N_g.
+__global__ void k_group_mass(const uint32_t* __restrict__ cnt, int64_t* __restrict__ cum, uint32_t* __restrict__ ng) {
+    constexpr int NT = 1024, L = kMaxPrompt + 1;      // 4097 lengths
+    __shared__ unsigned long long pm[NT];
+    __shared__ uint32_t pc[NT];
+    const int g = blockIdx.x;
+    const uint32_t* c = cnt + (size_t)g * L;
+    int64_t* out = cum + (size_t)g * (L + 1);
+    const int per = (L + NT - 1) / NT;                 // 5
+    const int lo = min(L, (int)threadIdx.x * per), hi = min(L, lo + per);
+    unsigned long long m = 0; uint32_t k = 0;
+    for (int l = lo; l < hi; ++l) { m += (unsigned long long)l * c[l]; k += c[l]; }
+    pm[threadIdx.x] = m; pc[threadIdx.x] = k;
+    __syncthreads();
+    for (int off = 1; off < NT; off <<= 1) {
+        unsigned long long vm = 0; uint32_t vc = 0;
+        if ((int)threadIdx.x >= off) { vm = pm[threadIdx.x - off]; vc = pc[threadIdx.x - off]; }
+        __syncthreads();
+        pm[threadIdx.x] += vm; pc[threadIdx.x] += vc;
+        __syncthreads();
+    }
+    unsigned long long run = pm[threadIdx.x] - m;
+    for (int l = lo; l < hi; ++l) { out[l] = (int64_t)run; run += (unsigned long long)l * c[l]; }
+    if (threadIdx.x == NT - 1) { out[L] = (int64_t)pm[NT - 1]; ng[g] = pc[NT - 1]; }
+}
+
+// Group offsets in the partitioned order and the 257 knots K_g[k] = sorted_g[(k (N_g - 1)) / 256].
+__global__ void k_group_knots(int G, const uint32_t* __restrict__ ng, const int32_t* __restrict__ sorted,
+                              uint32_t* __restrict__ grp_off, int32_t* __restrict__ knots) {
+    __shared__ uint32_t off[kMaxGroups + 1];
+    if (threadIdx.x == 0) {
+        uint32_t r = 0;
+        for (int g = 0; g < G; ++g) { off[g] = r; r += ng[g]; }
+        off[G] = r;
+        for (int g = 0; g <= G; ++g) grp_off[g] = off[g];
+    }
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < G * kNKnots; idx += blockDim.x) {
+        const int g = idx / kNKnots, k = idx % kNKnots;
+        const uint32_t N = off[g + 1] - off[g];
+        knots[idx] = N ? sorted[off[g] + (uint32_t)(((uint64_t)k * (N - 1)) / 256u)] : 0;
+    }
+}
+
+int grid_for(uint32_t n, int threads) {
+    long long b = ((long long)n + threads - 1) / threads;
+    if (b < 1) b = 1;
+    if (b > 148 * 16) b = 148 * 16;
+    return (int)b;
+}
+
+cudaError_t radix_pass(const uint64_t* kin, uint64_t* kout, const uint32_t* pin, uint32_t* pout, uint32_t n,
+                       int shift, uint32_t* counts, cudaStream_t st) {
+    uint32_t blocks = (n + 4095u) / 4096u;
+    if (blocks < 1) blocks = 1;
+    if (blocks > kRadixMaxBlocks) blocks = kRadixMaxBlocks;
+    uint32_t per_block = (n + blocks - 1) / blocks;
+    per_block = (per_block + kRadixThreads - 1) / kRadixThreads * kRadixThreads;
+    k_radix_hist<<<blocks, kRadixThreads, 0, st>>>(kin, n, per_block, shift, counts);
+    k_scan_counts<<<1, 1024, 0, st>>>(counts, 256u * blocks);
+    k_radix_scatter<<<blocks, kRadixThreads, 0, st>>>(kin, kout, pin, pout, n, per_block, shift, counts);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t run_load(const LoadArgs& a, cudaStream_t st) {
+    const uint32_t n = a.n;
+    const int G = (int)(a.ns * a.nd);
+    cudaError_t e;
+    if ((e = cudaMemsetAsync(a.cnt, 0, sizeof(uint32_t) * G * (kMaxPrompt + 1), st))) return e;
+    if ((e = cudaMemsetAsync(a.grp_sum_n, 0, sizeof(uint64_t) * kMaxGroups, st))) return e;
+    if ((e = cudaMemsetAsync(a.max_n, 0, sizeof(uint32_t), st))) return e;
+    if ((e = cudaMemsetAsync(a.err, 0, sizeof(int32_t) * 4, st))) return e;
+    if (n) {
+        k_ingest<<<grid_for(n, kIngestThreads), kIngestThreads, 0, st>>>(
+            n, a.prompt, a.outlen, a.ttft, a.sp, a.dp, a.ns, a.nd, a.keys_a, a.cnt,
+            (unsigned long long*)a.grp_sum_n, a.max_n, a.err);
+        // internal request order: stable partition by group (identity for a single group)
+        const uint32_t* orig_src = nullptr;
+        if (G > 1) {
+            if ((e = radix_pass(a.keys_a, a.keys_b, nullptr, a.tmp_idx, n, 32, a.radix_counts, st))) return e;
+            orig_src = a.tmp_idx;
+        }
+        k_gather<<<grid_for(n, 256), 256, 0, st>>>(n, orig_src, a.keys_a, a.prompt, a.outlen, a.S, a.l, a.nout, a.orig);
+        // sort (group, ticks): four byte passes over the ticks, one over the group id
+        uint64_t *src = a.keys_a, *dst = a.keys_b;
+        const int passes = G > 1 ? 5 : 4;
+        for (int p = 0; p < passes; ++p) {
+            if ((e = radix_pass(src, dst, nullptr, nullptr, n, 8 * p, a.radix_counts, st))) return e;
+            uint64_t* t = src; src = dst; dst = t;
+        }
+        k_low_words<<<grid_for(n, 256), 256, 0, st>>>(n, src, a.sorted);
+    }
+    k_group_mass<<<G, 1024, 0, st>>>(a.cnt, a.cum_mass, a.ng);
+    k_group_knots<<<1, 256, 0, st>>>(G, a.ng, a.sorted, a.grp_off, a.knots);
+    return cudaGetLastError();
+}
+
+}  // namespace disco

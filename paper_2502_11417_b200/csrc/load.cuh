@@ -1,0 +1,34 @@
+// Arguments of the device-side trace ingestion (all pointers are device memory).
+#pragma once
+
+#include "disco_internal.cuh"
+
+namespace disco {
+
+constexpr uint32_t kRadixMaxBlocks = 1024;
+
+struct LoadArgs {
+    uint32_t n, ns, nd;
+    // inputs in the caller's order
+    const int32_t *prompt, *outlen;
+    const float* ttft;
+    const uint8_t *sp, *dp;               // may be null
+    // scratch
+    uint64_t *keys_a, *keys_b;            // [n] (group << 32 | ticks)
+    uint32_t* tmp_idx;                    // [n]
+    uint32_t* radix_counts;               // [256 * kRadixMaxBlocks]
+    // outputs
+    int32_t* S; uint16_t *l, *nout; uint32_t* orig;   // internal (group-partitioned) order, [n]
+    int32_t* sorted;                      // [n] ticks ascending within each group
+    uint32_t* cnt;                        // [G][4097] requests per prompt length
+    int64_t* cum_mass;                    // [G][4098]
+    uint32_t *ng, *grp_off;               // [G], [G+1]
+    int32_t* knots;                       // [G][257]
+    uint64_t* grp_sum_n;                  // [kMaxGroups] output tokens per group
+    uint32_t* max_n;                      // longest output
+    int32_t* err;                         // [4]: code, request index, window flag
+};
+
+cudaError_t run_load(const LoadArgs& a, cudaStream_t st);
+
+}  // namespace disco
