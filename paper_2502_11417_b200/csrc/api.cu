@@ -1,0 +1,480 @@
+// Host side of the C ABI: argument checks, device memory, launch order.  No arithmetic of the method runs
+// here apart from turning the handful of profile and policy parameters into ticks.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "disco_internal.cuh"
+#include "load.cuh"
+
+using namespace disco;
+
+namespace {
+
+thread_local std::string g_err;
+
+int fail(int code, const std::string& msg) { g_err = msg; return code; }
+int fail_cuda(cudaError_t e, const char* what) {
+    g_err = std::string(what) + ": " + cudaGetErrorString(e);
+    return e == cudaErrorMemoryAllocation ? DISCO_ENOMEM : DISCO_ECUDA;
+}
+#define CU(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return fail_cuda(e_, #call); } while (0)
+
+// A growable device buffer.
+struct DevBuf {
+    void* p = nullptr;
+    size_t cap = 0;
+    cudaError_t reserve(size_t bytes) {
+        if (bytes <= cap && p) return cudaSuccess;
+        if (p) { cudaFree(p); p = nullptr; cap = 0; }
+        if (bytes < 16) bytes = 16;
+        cudaError_t e = cudaMalloc(&p, bytes);
+        if (e == cudaSuccess) cap = bytes;
+        return e;
+    }
+    void release() { if (p) cudaFree(p); p = nullptr; cap = 0; }
+    template <class T> T* as() const { return (T*)p; }
+};
+
+int64_t ticks_of_seconds(float s) { return llrint((double)s * 1e6); }
+int64_t ticks_of_rate(float per_s) { return llrint(1e6 / (double)per_s); }
+
+struct HostReadback {            // pinned; filled by the load call
+    int32_t err[4];
+    uint32_t max_n;
+    uint32_t ng[kMaxGroups];
+    uint32_t grp_off[kMaxGroups + 1];
+    int32_t knot_max[kMaxGroups];
+    uint64_t grp_sum_n[kMaxGroups];
+};
+
+__global__ void k_knot_max(int G, const int32_t* __restrict__ knots, int32_t* __restrict__ out) {
+    const int g = threadIdx.x;
+    if (g < G) out[g] = knots[g * kNKnots + kNKnots - 1];
+}
+
+}  // namespace
+
+struct disco_ctx {
+    uint32_t n = 0, ns = 0, nd = 0;
+    int G = 0;
+    bool loaded = false;
+    std::vector<GroupConst> gc;
+    // trace
+    DevBuf in_prompt, in_out, in_ttft, in_sp, in_dp;      // staging of host inputs
+    DevBuf keys_a, keys_b, tmp_idx, radix_counts;
+    DevBuf S, l, nout, orig, sorted;
+    DevBuf cnt, cum_mass, ng, grp_off, knots, grp_sum_n, max_n, err, d_gc;
+    HostReadback* rb = nullptr;
+    // evaluation
+    uint32_t P = 0;
+    bool evaluated = false, reduced = false;
+    std::vector<PolicyConst> pol;
+    DevBuf d_pol, d_prep, d_acc, d_hist_ttft, d_hist_tbt, d_stats, d_pol_list, d_classes, d_chunks, d_select;
+    DevBuf rec_u32[7], rec_u16[2], rec_win[3];
+    void* stage = nullptr;       // pinned staging for the small host->device tables
+    size_t stage_cap = 0;
+    cudaEvent_t stage_free = nullptr;
+    int32_t* sel_host = nullptr; // pinned [2]
+
+    ~disco_ctx() {
+        DevBuf* all[] = {&in_prompt, &in_out, &in_ttft, &in_sp, &in_dp, &keys_a, &keys_b, &tmp_idx, &radix_counts,
+                         &S, &l, &nout, &orig, &sorted, &cnt, &cum_mass, &ng, &grp_off, &knots, &grp_sum_n, &max_n,
+                         &err, &d_gc, &d_pol, &d_prep, &d_acc, &d_hist_ttft, &d_hist_tbt, &d_stats, &d_pol_list,
+                         &d_classes, &d_chunks, &d_select};
+        for (DevBuf* b : all) b->release();
+        for (auto& b : rec_u32) b.release();
+        for (auto& b : rec_u16) b.release();
+        for (auto& b : rec_win) b.release();
+        if (rb) cudaFreeHost(rb);
+        if (stage) cudaFreeHost(stage);
+        if (sel_host) cudaFreeHost(sel_host);
+        if (stage_free) cudaEventDestroy(stage_free);
+    }
+};
+
+namespace {
+
+int check_profiles(const disco_trace_desc_t* d, std::vector<GroupConst>* out) {
+    if (!d->servers || !d->devices || d->n_servers == 0 || d->n_devices == 0 ||
+        (uint64_t)d->n_servers * d->n_devices > kMaxGroups)
+        return fail(DISCO_EINVAL, "profile tables: need at least one server and one device and at most 64 groups");
+    out->clear();
+    for (uint32_t s = 0; s < d->n_servers; ++s) {
+        const disco_server_profile_t& sv = d->servers[s];
+        if (!(sv.tbt_s > 0.0f) || !std::isfinite(sv.tbt_s) || !(sv.jitter >= 0.0f && sv.jitter <= 1.0f) ||
+            !std::isfinite(sv.c_prefill) || !std::isfinite(sv.c_decode))
+            return fail(DISCO_EINVAL, "server profile " + std::to_string(s) + " is invalid");
+        for (uint32_t k = 0; k < d->n_devices; ++k) {
+            const disco_device_profile_t& dv = d->devices[k];
+            if (!(dv.prefill_tps > 0.0f) || !(dv.decode_tps > 0.0f) || !std::isfinite(dv.prefill_tps) ||
+                !std::isfinite(dv.decode_tps) || !(dv.jitter >= 0.0f && dv.jitter <= 1.0f) ||
+                !(dv.ttft_intercept_s >= 0.0f) || !std::isfinite(dv.ttft_intercept_s) ||
+                !std::isfinite(dv.c_prefill) || !std::isfinite(dv.c_decode) || !std::isfinite(dv.lambda))
+                return fail(DISCO_EINVAL, "device profile " + std::to_string(k) + " is invalid");
+            const int64_t Ts = ticks_of_seconds(sv.tbt_s), Tdv = ticks_of_rate(dv.decode_tps);
+            const int64_t Js = llrint((double)Ts * (double)sv.jitter), Jd = llrint((double)Tdv * (double)dv.jitter);
+            const int64_t kappa = ticks_of_rate(dv.prefill_tps), c0 = ticks_of_seconds(dv.ttft_intercept_s);
+            if (Ts + Js >= (1 << 30) || Tdv + Jd >= (1 << 30) || kappa * (kMaxPrompt + kMaxOutput) + c0 >= (1LL << 31))
+                return fail(DISCO_EINVAL, "profile too slow: a token interval or device TTFT exceeds the 32-bit tick range");
+            GroupConst g;
+            std::memset(&g, 0, sizeof g);
+            g.T_srv = (int32_t)Ts; g.J_srv = (int32_t)Js; g.T_dev = (int32_t)Tdv; g.J_dev = (int32_t)Jd;
+            g.kappa = (int32_t)kappa; g.c0 = (int32_t)c0;
+            const double cps = sv.c_prefill, cds = sv.c_decode, lam = dv.lambda;
+            const double dcp = lam * (double)dv.c_prefill, dcd = lam * (double)dv.c_decode;
+            g.auto_device_constrained = std::fmin(dcp, dcd) > std::fmax(cps, cds) ? 1 : 0;   // Algorithm 1
+            g.candidate = cds > dcd ? 1 : (dcd > cds ? 2 : 0);
+            g.delta_c = (float)std::fabs(cds - dcd);
+            g.cps = (float)cps; g.cds = (float)cds; g.lcpd = (float)dcp; g.lcdd = (float)dcd;
+            g.cps_d = cps; g.cds_d = cds; g.cpd_d = dv.c_prefill; g.cdd_d = dv.c_decode; g.lambda_d = lam;
+            out->push_back(g);
+        }
+    }
+    return 0;
+}
+
+cudaError_t reserve_trace(disco_ctx* c, uint32_t n, bool host_inputs, bool has_sp, bool has_dp) {
+    cudaError_t e;
+    const size_t N = n ? n : 1;
+    const int G = c->G;
+#define R(buf, bytes) if ((e = c->buf.reserve(bytes)) != cudaSuccess) return e
+    if (host_inputs) {
+        R(in_prompt, N * 4); R(in_out, N * 4); R(in_ttft, N * 4);
+        if (has_sp) R(in_sp, N);
+        if (has_dp) R(in_dp, N);
+    }
+    R(keys_a, N * 8); R(keys_b, N * 8); R(tmp_idx, std::max<size_t>(N, kMaxGroups) * 4);
+    R(radix_counts, 256 * kRadixMaxBlocks * 4);
+    R(S, N * 4); R(l, N * 2); R(nout, N * 2); R(orig, N * 4); R(sorted, N * 4);
+    R(cnt, (size_t)G * (kMaxPrompt + 1) * 4); R(cum_mass, (size_t)G * (kMaxPrompt + 2) * 8);
+    R(ng, kMaxGroups * 4); R(grp_off, (kMaxGroups + 1) * 4); R(knots, (size_t)G * kNKnots * 4);
+    R(grp_sum_n, kMaxGroups * 8); R(max_n, 4); R(err, 16); R(d_gc, (size_t)G * sizeof(GroupConst));
+#undef R
+    return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* disco_last_error(void) { return g_err.c_str(); }
+
+void disco_free_trace(disco_ctx_t* ctx) { delete ctx; }
+
+int disco_load_trace(disco_ctx_t** pctx, const disco_trace_desc_t* d, void* stream) {
+    if (!pctx || !d) return fail(DISCO_EINVAL, "null argument");
+    if (d->n >= (1ull << 31)) return fail(DISCO_EINVAL, "too many requests");
+    if (d->n && (!d->prompt_len || !d->output_len || !d->server_ttft_s)) return fail(DISCO_EINVAL, "null trace array");
+    if (d->arrays_on_device > 1) return fail(DISCO_EINVAL, "arrays_on_device must be 0 or 1");
+    std::vector<GroupConst> gc;
+    if (int rc = check_profiles(d, &gc)) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+
+    disco_ctx* c = *pctx;
+    const bool fresh = c == nullptr;
+    if (fresh) {
+        c = new (std::nothrow) disco_ctx;
+        if (!c) return fail(DISCO_ENOMEM, "out of host memory");
+    }
+    auto bail = [&](int rc) { if (fresh) delete c; else c->loaded = false; return rc; };
+    c->loaded = c->evaluated = c->reduced = false;
+    c->n = (uint32_t)d->n; c->ns = d->n_servers; c->nd = d->n_devices; c->G = (int)gc.size(); c->gc = gc;
+    const uint32_t n = c->n;
+    const bool host_in = d->arrays_on_device == 0;
+    cudaError_t e;
+    if (!c->rb && (e = cudaMallocHost((void**)&c->rb, sizeof(HostReadback))) != cudaSuccess)
+        return bail(fail_cuda(e, "cudaMallocHost"));
+    if ((e = reserve_trace(c, n, host_in, d->server_profile != nullptr, d->device_profile != nullptr)) != cudaSuccess)
+        return bail(fail_cuda(e, "device allocation for the trace"));
+
+    LoadArgs a;
+    std::memset(&a, 0, sizeof a);
+    a.n = n; a.ns = c->ns; a.nd = c->nd;
+    if (host_in && n) {
+#define H2D(dst, src, bytes) if ((e = cudaMemcpyAsync(c->dst.p, src, bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess) return bail(fail_cuda(e, "host to device copy"))
+        H2D(in_prompt, d->prompt_len, (size_t)n * 4); H2D(in_out, d->output_len, (size_t)n * 4);
+        H2D(in_ttft, d->server_ttft_s, (size_t)n * 4);
+        if (d->server_profile) H2D(in_sp, d->server_profile, (size_t)n);
+        if (d->device_profile) H2D(in_dp, d->device_profile, (size_t)n);
+#undef H2D
+        a.prompt = c->in_prompt.as<int32_t>(); a.outlen = c->in_out.as<int32_t>(); a.ttft = c->in_ttft.as<float>();
+        a.sp = d->server_profile ? c->in_sp.as<uint8_t>() : nullptr;
+        a.dp = d->device_profile ? c->in_dp.as<uint8_t>() : nullptr;
+    } else {
+        a.prompt = d->prompt_len; a.outlen = d->output_len; a.ttft = d->server_ttft_s;
+        a.sp = d->server_profile; a.dp = d->device_profile;
+    }
+    a.keys_a = c->keys_a.as<uint64_t>(); a.keys_b = c->keys_b.as<uint64_t>(); a.tmp_idx = c->tmp_idx.as<uint32_t>();
+    a.radix_counts = c->radix_counts.as<uint32_t>();
+    a.S = c->S.as<int32_t>(); a.l = c->l.as<uint16_t>(); a.nout = c->nout.as<uint16_t>(); a.orig = c->orig.as<uint32_t>();
+    a.sorted = c->sorted.as<int32_t>(); a.cnt = c->cnt.as<uint32_t>(); a.cum_mass = c->cum_mass.as<int64_t>();
+    a.ng = c->ng.as<uint32_t>(); a.grp_off = c->grp_off.as<uint32_t>(); a.knots = c->knots.as<int32_t>();
+    a.grp_sum_n = c->grp_sum_n.as<uint64_t>(); a.max_n = c->max_n.as<uint32_t>(); a.err = c->err.as<int32_t>();
+    // the profile table is read from pageable memory: this copy returns once it has been staged
+    if ((e = cudaMemcpyAsync(c->d_gc.p, c->gc.data(), c->gc.size() * sizeof(GroupConst), cudaMemcpyHostToDevice, st)) != cudaSuccess)
+        return bail(fail_cuda(e, "profile copy"));
+    if ((e = run_load(a, st)) != cudaSuccess) return bail(fail_cuda(e, "trace ingestion kernels"));
+    // read back the few numbers the host needs: error word, group sizes, longest output, largest TTFT per group
+    HostReadback* rb = c->rb;
+    k_knot_max<<<1, kMaxGroups, 0, st>>>(c->G, a.knots, (int32_t*)c->tmp_idx.p);
+    bool ok = true;
+    ok &= cudaMemcpyAsync(rb->err, a.err, 16, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(&rb->max_n, a.max_n, 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(rb->ng, a.ng, 4 * c->G, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(rb->grp_off, a.grp_off, 4 * (c->G + 1), cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(rb->knot_max, c->tmp_idx.p, 4 * c->G, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(rb->grp_sum_n, a.grp_sum_n, 8 * c->G, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (!ok) return bail(fail_cuda(cudaGetLastError(), "readback"));
+    if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return bail(fail_cuda(e, "trace ingestion"));
+    if (rb->err[0]) {
+        static const char* what[] = {"", "prompt length outside 1..4096", "output length outside 1..8192",
+                                     "server TTFT not finite, not positive or above 2000 s", "profile id out of range"};
+        return bail(fail(DISCO_EINVAL, std::string(what[rb->err[0]]) + " at request " + std::to_string(rb->err[1])));
+    }
+    c->loaded = true;
+    *pctx = c;
+    return 0;
+}
+
+int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, uint64_t seed,
+                        const disco_pair_out_t* out, void* stream) {
+    if (!c || !pol || P == 0) return fail(DISCO_EINVAL, "null context, null policies or P = 0");
+    if (!c->loaded) return fail(DISCO_EINVAL, "no trace loaded");
+    if (P > (1u << 19)) return fail(DISCO_EINVAL, "too many policies");
+    cudaStream_t st = (cudaStream_t)stream;
+    const int G = c->G;
+    const uint32_t n = c->n;
+    c->evaluated = c->reduced = false;
+
+    // ---- policy constants and timeline classes
+    std::vector<PolicyConst> pc(P);
+    std::vector<ClassConst> classes;
+    for (uint32_t p = 0; p < P; ++p) {
+        const disco_policy_t& q = pol[p];
+        const std::string at = " (policy " + std::to_string(p) + ")";
+        if (!(q.budget >= 0.0f && q.budget <= 1.0f)) return fail(DISCO_EINVAL, "budget outside [0,1]" + at);
+        if (!(q.alpha > 0.0f && q.alpha < 1.0f)) return fail(DISCO_EINVAL, "alpha outside (0,1)" + at);
+        if (!(q.mig_threshold >= 0.0f)) return fail(DISCO_EINVAL, "migration threshold negative or NaN" + at);
+        if (!(q.r_c > 0.0f) || !std::isfinite(q.r_c)) return fail(DISCO_EINVAL, "consumption rate must be positive" + at);
+        if (!(q.t_m_s >= 0.0f) || !std::isfinite(q.t_m_s)) return fail(DISCO_EINVAL, "migration time must be >= 0" + at);
+        const uint32_t mode = (q.flags >> 2) & 3u;
+        if (mode == 3 || (q.flags >> 4)) return fail(DISCO_EINVAL, "unknown flags" + at);
+        const int64_t tau = ticks_of_rate(q.r_c), t_m = ticks_of_seconds(q.t_m_s);
+        if (tau < 1 || tau >= (1 << 30)) return fail(DISCO_EINVAL, "consumption interval outside 1 .. 2^30 ticks" + at);
+        const bool pacing = (q.flags & DISCO_FLAG_PACING) != 0, mig = (q.flags & DISCO_FLAG_MIGRATION) != 0;
+        int64_t B = pacing ? (t_m + tau - 1) / tau : 0;               // Eq. 6, rounded up
+        if (B > kMaxOutput) B = kMaxOutput;                            // a buffer no stream can fill
+        PolicyConst& o = pc[p];
+        o.budget = q.budget; o.alpha = q.alpha; o.theta = q.mig_threshold; o.flags = q.flags;
+        o.tau = (int32_t)tau; o.B = (int32_t)B; o.mode = (int32_t)mode;
+        int cls = -1;
+        for (size_t k = 0; k < classes.size(); ++k)
+            if (classes[k].tau == o.tau && classes[k].B == o.B && classes[k].pacing == (int)pacing) { cls = (int)k; break; }
+        if (cls < 0) {
+            ClassConst cc;
+            std::memset(&cc, 0, sizeof cc);
+            cc.tau = o.tau; cc.tau_eff = pacing ? o.tau : 0; cc.B = o.B; cc.pacing = pacing;
+            classes.push_back(cc);
+            cls = (int)classes.size() - 1;
+        }
+        classes[cls].mig_any |= mig ? 1 : 0;
+        o.cls = cls;
+    }
+    // ---- per class: 32-bit range proof and histogram windows of the regular TBTs
+    const HostReadback& rb = *c->rb;
+    const int64_t n_max = rb.max_n;
+    for (ClassConst& cc : classes) {
+        int Wmax[3] = {1, 1, 1};
+        for (int g = 0; g < G; ++g) {
+            const GroupConst& gc = c->gc[g];
+            const int64_t xs = gc.T_srv + (int64_t)gc.J_srv, xd = gc.T_dev + (int64_t)gc.J_dev;
+            if (rb.ng[g]) {
+                const int64_t step = std::max<int64_t>(cc.tau_eff, std::max(xs, xd));
+                const int64_t Mmax = std::max<int64_t>(rb.knot_max[g], (int64_t)gc.kappa * (kMaxPrompt + n_max) + gc.c0);
+                if ((n_max - 1) * step + Mmax >= (1LL << 31))
+                    return fail(DISCO_EINVAL, "a decode stream could outlast 2^31 ticks (about 35 minutes)");
+            }
+            int64_t lo_v[3], hi_v[3];
+            lo_v[0] = cc.pacing ? cc.tau : gc.T_srv - (int64_t)gc.J_srv; hi_v[0] = cc.pacing ? std::max<int64_t>(cc.tau, xs) : xs;
+            lo_v[1] = cc.pacing ? cc.tau : gc.T_dev - (int64_t)gc.J_dev; hi_v[1] = cc.pacing ? std::max<int64_t>(cc.tau, xd) : xd;
+            lo_v[2] = std::min(lo_v[0], lo_v[1]); hi_v[2] = std::max(hi_v[0], hi_v[1]);
+            for (int k = 0; k < 3; ++k) {
+                const int lo = host_bin_of_ticks(lo_v[k]), hi = host_bin_of_ticks(hi_v[k]);
+                cc.lo[g][k] = lo;
+                cc.ktau[g][k] = cc.pacing ? host_bin_of_ticks(cc.tau) - lo : -1;
+                Wmax[k] = std::max(Wmax[k], hi - lo + 1);
+            }
+        }
+        for (int k = 0; k < 3; ++k) cc.W[k] = Wmax[k];
+        const size_t win_bytes = (size_t)n * (Wmax[0] + Wmax[1] + Wmax[2]) * 2;
+        if (win_bytes > (48ull << 30)) return fail(DISCO_ENOMEM, "per-request TBT windows would exceed 48 GB");
+    }
+
+    // ---- device buffers
+    cudaError_t e;
+    const size_t N1 = n ? n : 1;
+    size_t wmax[3] = {1, 1, 1};
+    for (const ClassConst& cc : classes) for (int k = 0; k < 3; ++k) wmax[k] = std::max<size_t>(wmax[k], cc.W[k]);
+#define R(buf, bytes) if ((e = c->buf.reserve(bytes)) != cudaSuccess) return fail_cuda(e, "device allocation for the evaluation")
+    R(d_pol, P * sizeof(PolicyConst)); R(d_prep, (size_t)G * P * sizeof(Prep));
+    R(d_acc, (size_t)P * G * kNAcc * 8); R(d_hist_ttft, (size_t)P * kNBins * 8); R(d_hist_tbt, (size_t)P * kNBins * 8);
+    R(d_stats, P * sizeof(disco_policy_stats_t)); R(d_pol_list, P * 4);
+    R(d_classes, classes.size() * sizeof(ClassConst)); R(d_select, 8);
+    for (int k = 0; k < 7; ++k) R(rec_u32[k], N1 * 4);
+    for (int k = 0; k < 2; ++k) R(rec_u16[k], N1 * 2);
+    for (int k = 0; k < 3; ++k) R(rec_win[k], N1 * wmax[k] * 2);
+
+    // ---- policies grouped by class; request chunks (one group each) sized so that chunks x policy tiles
+    //      fill the GPU about once
+    std::vector<uint32_t> pol_list;
+    std::vector<std::pair<uint32_t, uint32_t>> cls_range;       // [begin, end) in pol_list per class
+    for (size_t k = 0; k < classes.size(); ++k) {
+        const uint32_t b = (uint32_t)pol_list.size();
+        for (uint32_t p = 0; p < P; ++p) if (pc[p].cls == (int)k) pol_list.push_back(p);
+        cls_range.push_back({b, (uint32_t)pol_list.size()});
+    }
+    const uint32_t tiles = (P + 15) / 16;
+    const uint32_t want_chunks = std::max<uint32_t>(1, 296 / std::min<uint32_t>(tiles, 296));
+    uint32_t CH = (uint32_t)((N1 + want_chunks - 1) / want_chunks);
+    CH = (CH + 255) / 256 * 256;
+    CH = std::min<uint32_t>(std::max<uint32_t>(CH, 256), 8192);
+    std::vector<Chunk> chunks;
+    for (int g = 0; g < G; ++g)
+        for (uint32_t s = rb.grp_off[g]; s < rb.grp_off[g + 1]; s += CH)
+            chunks.push_back({s, std::min(CH, rb.grp_off[g + 1] - s), g, 0});
+    R(d_chunks, std::max<size_t>(1, chunks.size()) * sizeof(Chunk));
+#undef R
+
+    // ---- small tables to the device through pinned staging
+    const size_t need = P * sizeof(PolicyConst) + classes.size() * sizeof(ClassConst) + P * 4 +
+                        chunks.size() * sizeof(Chunk) + 64;
+    if (c->stage_free) CU(cudaEventSynchronize(c->stage_free));     // an earlier call's copies may still read it
+    else CU(cudaEventCreateWithFlags(&c->stage_free, cudaEventDisableTiming));
+    if (need > c->stage_cap) {
+        if (c->stage) cudaFreeHost(c->stage);
+        c->stage = nullptr; c->stage_cap = 0;
+        CU(cudaMallocHost(&c->stage, need));
+        c->stage_cap = need;
+    }
+    char* sp = (char*)c->stage;
+    auto push = [&](void* dst, const void* src, size_t bytes) -> cudaError_t {
+        if (!bytes) return cudaSuccess;
+        std::memcpy(sp, src, bytes);
+        cudaError_t r = cudaMemcpyAsync(dst, sp, bytes, cudaMemcpyHostToDevice, st);
+        sp += (bytes + 15) / 16 * 16;
+        return r;
+    };
+    CU(push(c->d_pol.p, pc.data(), P * sizeof(PolicyConst)));
+    CU(push(c->d_classes.p, classes.data(), classes.size() * sizeof(ClassConst)));
+    CU(push(c->d_pol_list.p, pol_list.data(), P * 4));
+    CU(push(c->d_chunks.p, chunks.data(), chunks.size() * sizeof(Chunk)));
+    CU(cudaEventRecord(c->stage_free, st));
+
+    CU(cudaMemsetAsync(c->d_acc.p, 0, (size_t)P * G * kNAcc * 8, st));
+    CU(cudaMemsetAsync(c->d_hist_ttft.p, 0, (size_t)P * kNBins * 8, st));
+    CU(cudaMemsetAsync(c->d_hist_tbt.p, 0, (size_t)P * kNBins * 8, st));
+
+    // ---- Algorithms 1-3 for every (group, policy)
+    CU(launch_prep(c->d_pol.as<PolicyConst>(), P, G, c->d_gc.as<GroupConst>(), c->cum_mass.as<int64_t>(),
+                   c->cnt.as<uint32_t>(), c->sorted.as<int32_t>(), c->grp_off.as<uint32_t>(), c->d_prep.as<Prep>(), st));
+
+    TraceDev tr;
+    tr.n = n; tr.n_groups = G; tr.S = c->S.as<int32_t>(); tr.l = c->l.as<uint16_t>(); tr.nout = c->nout.as<uint16_t>();
+    tr.orig = c->orig.as<uint32_t>(); tr.grp_off = c->grp_off.as<uint32_t>();
+    TimelineRec rec;
+    for (int k = 0; k < 3; ++k) {
+        rec.sum[k] = c->rec_u32[2 * k].as<uint32_t>(); rec.max[k] = c->rec_u32[2 * k + 1].as<uint32_t>();
+        rec.win[k] = c->rec_win[k].as<uint16_t>();
+    }
+    rec.stall = c->rec_u32[6].as<uint32_t>();
+    rec.m = c->rec_u16[0].as<uint16_t>(); rec.delayed = c->rec_u16[1].as<uint16_t>();
+    disco_pair_out_t po;
+    std::memset(&po, 0, sizeof po);
+    if (out) po = *out;
+
+    // ---- per timeline class: play every request out, then evaluate the class's policies on the summaries
+    for (size_t k = 0; k < classes.size(); ++k) {
+        const ClassConst* dcc = c->d_classes.as<ClassConst>() + k;
+        CU(launch_timeline(tr, c->d_gc.as<GroupConst>(), dcc, c->knots.as<int32_t>(), seed, rec, c->err.as<int32_t>(), st));
+        CU(launch_pairs(tr, c->d_gc.as<GroupConst>(), dcc, c->d_prep.as<Prep>(), P,
+                        c->d_pol_list.as<uint32_t>() + cls_range[k].first, cls_range[k].second - cls_range[k].first,
+                        c->d_chunks.as<Chunk>(), (uint32_t)chunks.size(), rec, po, c->d_acc.as<uint64_t>(),
+                        c->d_hist_ttft.as<uint64_t>(), c->d_hist_tbt.as<uint64_t>(), st));
+    }
+    c->P = P; c->pol = pc;
+    c->evaluated = true;
+    return 0;
+}
+
+int disco_reduce_stats(disco_ctx_t* c, disco_policy_stats_t* stats, void* stream) {
+    if (!c || !stats) return fail(DISCO_EINVAL, "null argument");
+    if (!c->evaluated) return fail(DISCO_EINVAL, "no evaluation to reduce");
+    cudaStream_t st = (cudaStream_t)stream;
+    CU(launch_finalize(c->P, c->G, c->d_gc.as<GroupConst>(), c->d_acc.as<uint64_t>(), c->d_hist_ttft.as<uint64_t>(),
+                       c->d_hist_tbt.as<uint64_t>(), c->grp_sum_n.as<uint64_t>(), c->grp_off.as<uint32_t>(),
+                       c->d_stats.as<disco_policy_stats_t>(), st));
+    CU(cudaMemcpyAsync(stats, c->d_stats.p, c->P * sizeof(disco_policy_stats_t), cudaMemcpyDeviceToHost, st));
+    CU(cudaMemcpyAsync(c->rb->err, c->err.p, 16, cudaMemcpyDeviceToHost, st));
+    CU(cudaStreamSynchronize(st));
+    if (c->rb->err[2]) return fail(DISCO_ECUDA, "internal error: an inter-token interval fell outside its histogram window");
+    c->reduced = true;
+    return 0;
+}
+
+int disco_select_policy(disco_ctx_t* c, double cost_cap, float tbt_slo_s, int32_t* best, void* stream) {
+    if (!c || !best) return fail(DISCO_EINVAL, "null argument");
+    if (!c->reduced) return fail(DISCO_EINVAL, "reduce the statistics before selecting");
+    cudaStream_t st = (cudaStream_t)stream;
+    if (!c->sel_host) CU(cudaMallocHost((void**)&c->sel_host, 8));
+    CU(launch_select(c->d_stats.as<disco_policy_stats_t>(), c->P, cost_cap, tbt_slo_s, c->d_select.as<int32_t>(), st));
+    CU(cudaMemcpyAsync(c->sel_host, c->d_select.p, 8, cudaMemcpyDeviceToHost, st));
+    CU(cudaStreamSynchronize(st));
+    *best = c->sel_host[1];
+    if (c->sel_host[0] != 0) return fail(DISCO_EINFEASIBLE, "no policy meets the cost cap and the TBT objective");
+    return 0;
+}
+
+int disco_get_histograms(disco_ctx_t* c, uint32_t p, uint64_t* ttft_hist, uint64_t* tbt_hist, void* stream) {
+    if (!c || !c->evaluated || p >= c->P) return fail(DISCO_EINVAL, "no evaluation or policy index out of range");
+    cudaStream_t st = (cudaStream_t)stream;
+    if (ttft_hist) CU(cudaMemcpyAsync(ttft_hist, c->d_hist_ttft.as<uint64_t>() + (size_t)p * kNBins, kNBins * 8, cudaMemcpyDeviceToHost, st));
+    if (tbt_hist) CU(cudaMemcpyAsync(tbt_hist, c->d_hist_tbt.as<uint64_t>() + (size_t)p * kNBins, kNBins * 8, cudaMemcpyDeviceToHost, st));
+    CU(cudaStreamSynchronize(st));
+    return 0;
+}
+
+int disco_get_prep(disco_ctx_t* c, uint32_t g, uint32_t p, disco_prep_t* out, void* stream) {
+    if (!c || !out || !c->evaluated || p >= c->P || g >= (uint32_t)c->G) return fail(DISCO_EINVAL, "bad argument");
+    cudaStream_t st = (cudaStream_t)stream;
+    Prep pr;
+    CU(cudaMemcpyAsync(&pr, c->d_prep.as<Prep>() + (size_t)g * c->P + p, sizeof pr, cudaMemcpyDeviceToHost, st));
+    CU(cudaStreamSynchronize(st));
+    out->device_constrained = pr.device_constrained; out->l_th = pr.l_th; out->l_star = pr.l_star;
+    out->B = c->pol[p].B; out->w_star = pr.w_star; out->w_tail = pr.w_tail; out->tau = c->pol[p].tau;
+    return 0;
+}
+
+int64_t disco_get_group_tables(disco_ctx_t* c, uint32_t g, int64_t* cnt, int32_t* knots, int32_t* sorted_ticks,
+                               uint64_t n_sorted, void* stream) {
+    if (!c || !c->loaded || g >= (uint32_t)c->G) return fail(DISCO_EINVAL, "bad argument");
+    cudaStream_t st = (cudaStream_t)stream;
+    const uint32_t ng = c->rb->ng[g], off = c->rb->grp_off[g];
+    if (cnt) {
+        std::vector<uint32_t> tmp(kMaxPrompt + 1);
+        CU(cudaMemcpyAsync(tmp.data(), c->cnt.as<uint32_t>() + (size_t)g * (kMaxPrompt + 1), tmp.size() * 4, cudaMemcpyDeviceToHost, st));
+        CU(cudaStreamSynchronize(st));
+        for (size_t i = 0; i < tmp.size(); ++i) cnt[i] = tmp[i];
+    }
+    if (knots) CU(cudaMemcpyAsync(knots, c->knots.as<int32_t>() + (size_t)g * kNKnots, kNKnots * 4, cudaMemcpyDeviceToHost, st));
+    const uint64_t k = std::min<uint64_t>(n_sorted, ng);
+    if (sorted_ticks && k) CU(cudaMemcpyAsync(sorted_ticks, c->sorted.as<int32_t>() + off, k * 4, cudaMemcpyDeviceToHost, st));
+    CU(cudaStreamSynchronize(st));
+    return (int64_t)ng;
+}
+
+}  // extern "C"

@@ -1,0 +1,135 @@
+// Final reductions per policy (Sec. 5.1 metrics: mean and tail TTFT, P99 TBT, cost) and policy selection.
+#include "disco_internal.cuh"
+
+namespace disco {
+
+namespace {
+
+__device__ __forceinline__ double bin_edge_seconds(int b) {
+    long long edge = b < 32 ? b : ((long long)(32 + (b & 31)) << ((b >> 5) - 1));
+    return __dmul_rn((double)edge, 1e-6);
+}
+
+// nearest-rank quantile: bin holding the ceil(q*M)-th smallest item
+__device__ int quantile_bin(const unsigned long long* hist, double q, unsigned long long M) {
+    if (M == 0) return 0;
+    unsigned long long rank = (unsigned long long)ceil(__dmul_rn(q, (double)M));
+    if (rank < 1) rank = 1;
+    unsigned long long acc = 0;
+    for (int b = 0; b < kNBins; ++b) { acc += hist[b]; if (acc >= rank) return b; }
+    return kNBins - 1;
+}
+
+// One block of 32 threads per policy.
+__global__ void k_finalize(uint32_t P, int G, const GroupConst* __restrict__ gc,
+                           const unsigned long long* __restrict__ acc, const unsigned long long* __restrict__ hist_ttft,
+                           const unsigned long long* __restrict__ hist_tbt,
+                           const unsigned long long* __restrict__ grp_sum_n, const uint32_t* __restrict__ grp_off,
+                           disco_policy_stats_t* __restrict__ stats) {
+    const uint32_t p = blockIdx.x;
+    __shared__ unsigned long long tot[kNAcc];
+    __shared__ int qb[4];
+    const unsigned long long N = grp_off[G];
+    if (threadIdx.x < kNAcc) {
+        unsigned long long s = 0;
+        for (int g = 0; g < G; ++g) s += acc[((size_t)p * G + g) * kNAcc + threadIdx.x];
+        tot[threadIdx.x] = s;
+    }
+    unsigned long long sum_n = 0;
+    for (int g = 0; g < G; ++g) sum_n += grp_sum_n[g];
+    if (threadIdx.x < 3) {
+        const double q = threadIdx.x == 0 ? 0.50 : threadIdx.x == 1 ? 0.95 : 0.99;
+        qb[threadIdx.x] = quantile_bin(hist_ttft + (size_t)p * kNBins, q, N);
+    } else if (threadIdx.x == 3) {
+        qb[3] = quantile_bin(hist_tbt + (size_t)p * kNBins, 0.99, sum_n - N);
+    }
+    __syncthreads();
+    if (threadIdx.x != 0) return;
+    // Eq. 8 on the exact integer token totals of each group
+    double cost = 0.0;
+    unsigned long long tok_dev = 0;
+    for (int g = 0; g < G; ++g) {
+        const unsigned long long* a = acc + ((size_t)p * G + g) * kNAcc;
+        const double dts = (double)(grp_sum_n[g] - a[A_TOK_DEVICE]), dtd = (double)a[A_TOK_DEVICE];
+        const double pts = (double)a[A_PRE_SERVER], ptd = (double)a[A_PRE_DEVICE];
+        const GroupConst& c = gc[g];
+        const double srv = __dadd_rn(__dmul_rn(c.cps_d, pts), __dmul_rn(c.cds_d, dts));
+        const double dev = __dadd_rn(__dmul_rn(c.cpd_d, ptd), __dmul_rn(c.cdd_d, dtd));
+        cost = __dadd_rn(cost, __dadd_rn(srv, __dmul_rn(c.lambda_d, dev)));
+        tok_dev += a[A_TOK_DEVICE];
+    }
+    disco_policy_stats_t s;
+    const unsigned long long ttft_ticks = tot[A_TTFT_LO] + (tot[A_TTFT_HI] << 16);
+    s.mean_ttft_s = N ? __ddiv_rn(__dmul_rn((double)ttft_ticks, 1e-6), (double)N) : 0.0;
+    s.total_cost = cost;
+    s.bin_p50_ttft = qb[0]; s.bin_p95_ttft = qb[1]; s.bin_p99_ttft = qb[2]; s.bin_p99_tbt = qb[3];
+    s.p50_ttft_s = (float)bin_edge_seconds(qb[0]); s.p95_ttft_s = (float)bin_edge_seconds(qb[1]);
+    s.p99_ttft_s = (float)bin_edge_seconds(qb[2]); s.p99_tbt_s = (float)bin_edge_seconds(qb[3]);
+    s.n_requests = N; s.n_intervals = sum_n - N;
+    s.n_server_only = tot[A_SERVER_ONLY]; s.n_device_only = tot[A_DEVICE_ONLY]; s.n_race = tot[A_RACE];
+    s.n_device_started = tot[A_STARTED]; s.n_device_won = tot[A_DEVICE_WON]; s.n_migrations = tot[A_MIGR];
+    s.tok_device = tok_dev; s.tok_server = sum_n - tok_dev;
+    s.prefill_tok_server = tot[A_PRE_SERVER]; s.prefill_tok_device = tot[A_PRE_DEVICE];
+    s.delayed_tokens = tot[A_DELAYED];
+    stats[p] = s;
+}
+
+// Lexicographic objective of the selection: (tail TTFT bin, mean TTFT, cost, index), feasible policies only.
+struct Pick { int feasible; int bin; double mean, cost; int idx; };
+
+__device__ __forceinline__ bool better(const Pick& a, const Pick& b) {
+    if (b.idx < 0) return a.idx >= 0;
+    if (a.idx < 0) return false;
+    if (a.feasible != b.feasible) return a.feasible > b.feasible;
+    if (a.feasible) {
+        if (a.bin != b.bin) return a.bin < b.bin;
+        if (a.mean != b.mean) return a.mean < b.mean;
+        if (a.cost != b.cost) return a.cost < b.cost;
+    } else {
+        if (a.cost != b.cost) return a.cost < b.cost;        // none feasible: cheapest
+    }
+    return a.idx < b.idx;
+}
+
+__global__ void k_select(const disco_policy_stats_t* __restrict__ stats, uint32_t P, double cost_cap, double tbt_slo,
+                         int32_t* __restrict__ result) {
+    __shared__ Pick best[256];
+    Pick mine = {0, 0, 0.0, 0.0, -1};
+    for (uint32_t p = threadIdx.x; p < P; p += blockDim.x) {
+        const disco_policy_stats_t& s = stats[p];
+        Pick c;
+        c.feasible = (s.total_cost <= cost_cap) && (bin_edge_seconds(s.bin_p99_tbt) <= tbt_slo);
+        c.bin = s.bin_p99_ttft; c.mean = s.mean_ttft_s; c.cost = s.total_cost; c.idx = (int)p;
+        if (better(c, mine)) mine = c;
+    }
+    best[threadIdx.x] = mine;
+    __syncthreads();
+    for (int off = 128; off > 0; off >>= 1) {
+        if ((int)threadIdx.x < off && better(best[threadIdx.x + off], best[threadIdx.x]))
+            best[threadIdx.x] = best[threadIdx.x + off];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        result[0] = best[0].feasible ? 0 : DISCO_EINFEASIBLE;
+        result[1] = best[0].idx;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_finalize(uint32_t P, int G, const GroupConst* gc, const uint64_t* acc, const uint64_t* hist_ttft,
+                            const uint64_t* hist_tbt, const uint64_t* grp_sum_n, const uint32_t* grp_off,
+                            disco_policy_stats_t* stats, cudaStream_t st) {
+    k_finalize<<<P, 32, 0, st>>>(P, G, gc, (const unsigned long long*)acc, (const unsigned long long*)hist_ttft,
+                                 (const unsigned long long*)hist_tbt, (const unsigned long long*)grp_sum_n, grp_off,
+                                 stats);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_select(const disco_policy_stats_t* stats, uint32_t P, double cost_cap, float tbt_slo_s,
+                          int32_t* result, cudaStream_t st) {
+    k_select<<<1, 256, 0, st>>>(stats, P, cost_cap, (double)tbt_slo_s, result);
+    return cudaGetLastError();
+}
+
+}  // namespace disco
