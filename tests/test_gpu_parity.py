@@ -1,0 +1,162 @@
+"""CUDA path against the oracle, through the C ABI (needs a GPU)."""
+import numpy as np
+import pytest
+
+from paper_2502_11417_b200 import synth, Trace, DiscoError
+from parity import full_parity, check_stats, check_pairs
+from helpers import constructed
+
+pytestmark = pytest.mark.gpu
+
+MIG, PACE = synth.FLAG_MIGRATION, synth.FLAG_PACING
+S_MODE, D_MODE = synth.MODE_SERVER_CONSTRAINED, synth.MODE_DEVICE_CONSTRAINED
+
+
+def test_config0_full():
+    full_parity(synth.make_workload(0), tag="config0")
+
+
+def test_config1_shape_ragged_tiles():
+    # several request chunks and policy tiles, none of them full
+    w = synth.make_workload(1, n=7013, n_budgets=21)
+    full_parity(w, tag="config1-small")
+
+
+def test_config2_shape_threshold_grid():
+    w = synth.make_workload(2, n=5000, n_budgets=9)
+    full_parity(w, tag="config2-small")
+
+
+def test_config3_shape_long_outputs():
+    w = synth.make_workload(3, n=1500, n_budgets=5)
+    assert w.output_len.max() > 2048
+    full_parity(w, tag="config3-small")
+
+
+def test_config4_shape_six_groups_two_modes():
+    w = synth.make_workload(4, n=9000, n_budgets=7)
+    gs, _ = full_parity(w, tag="config4-small")
+    assert any(s.n_migrations for s in gs)
+
+
+@pytest.mark.parametrize("flags", [0, PACE, MIG, MIG | PACE])
+@pytest.mark.parametrize("mode", [S_MODE, D_MODE])
+def test_flag_and_mode_matrix(flags, mode):
+    pols = [synth.policy(b, mig_threshold=th, t_m_s=tm, flags=flags | mode)
+            for b in (0.0, 0.04, 0.3, 1.0) for th in (0.0, 0.01) for tm in (0.0, 0.45, 1.0)]
+    for dear in (False, True):
+        w = synth.tiny_workload(17 + dear, 700, n_servers=2, n_devices=2, max_prompt=500, max_out=150,
+                                device_dearer=dear)
+        full_parity(w, pols, tag=f"matrix flags={flags} mode={mode} dear={dear}")
+
+
+def test_mixed_timeline_classes_in_one_call():
+    # policies differing in r_c, t_m and pacing need separate play-outs inside one evaluation
+    pols = [synth.policy(0.5, r_c=5.0), synth.policy(0.5, r_c=12.0, t_m_s=0.5), synth.policy(0.7, flags=MIG),
+            synth.policy(0.2, r_c=5.0, t_m_s=3.0), synth.policy(0.9, r_c=40.0), synth.policy(1.0, r_c=5.0)]
+    w = synth.tiny_workload(5, 900, max_prompt=800, max_out=200)
+    full_parity(w, pols, tag="classes")
+
+
+def test_generation_slower_than_consumption():
+    # r_c above the decode rates: the buffer drains, TBTs follow generation, hand-offs are rare
+    pols = [synth.policy(b, r_c=rc, t_m_s=0.2, flags=MIG | PACE | S_MODE) for b in (0.5, 1.0) for rc in (25.0, 60.0)]
+    w = synth.tiny_workload(9, 600, max_prompt=300, max_out=300)
+    full_parity(w, pols, tag="slow-gen")
+
+
+def test_edge_cases():
+    # single-token outputs, longest outputs, extreme prompts, ties at S = Td, one request
+    tr = constructed([1, 4096, 45, 45, 45, 7, 4096], [1, 8192, 2, 1, 8192, 3, 1],
+                     [1e-3, 1999.0, 0.1, 0.1, 0.100001, 0.05, 1.0],
+                     devices=[synth.device(500.0, 20.0, ttft_intercept_s=0.01, jitter=0.05)],
+                     servers=[synth.server(jitter=0.2)])
+    w = synth.Workload(name="edges", seed=3, materialise=True, policies=[], **tr)
+    pols = [synth.policy(b, flags=f | md) for b in (0.0, 0.5, 1.0) for f in (MIG | PACE, PACE) for md in (S_MODE, D_MODE)]
+    full_parity(w, pols, tag="edges")
+    one = synth.Workload(name="one", seed=1, materialise=True, policies=[],
+                         **constructed([100], [50], [0.2]))
+    full_parity(one, [synth.policy(1.0)], tag="one")
+
+
+def test_empty_trace_and_reload():
+    w = synth.tiny_workload(1, 300)
+    t = Trace.from_workload(w)
+    e = constructed([], [], [])
+    t.load_trace(e["prompt_len"], e["output_len"], e["server_ttft_s"], None, None, e["servers"], e["devices"])
+    t.eval_policies([synth.policy(0.5)], 0)
+    s = t.reduce_stats()[0]
+    assert s.n_requests == 0 and s.total_cost == 0.0 and s.tok_server == 0
+    # reload a larger trace into the same context
+    w2 = synth.tiny_workload(2, 2000)
+    t.load_trace(w2.prompt_len, w2.output_len, w2.server_ttft_s, w2.server_profile, w2.device_profile,
+                 w2.servers, w2.devices)
+    from oracle import Oracle
+    t.eval_policies(w2.policies, 7)
+    gs = t.reduce_stats()
+    os_, _ = Oracle.from_workload(w2).eval(w2.policies, 7)
+    check_stats(gs, os_, t.histograms, "reload")
+
+
+def test_device_resident_inputs_match_host_inputs():
+    import torch
+    w = synth.make_workload(4, n=4000, n_budgets=3)
+    a = Trace.from_workload(w)
+    a.eval_policies(w.policies, 4)
+    sa = a.reduce_stats()
+    dev = [torch.from_numpy(x).cuda() for x in (w.prompt_len, w.output_len, w.server_ttft_s, w.server_profile,
+                                                 w.device_profile)]
+    b = Trace().load_trace(*dev, w.servers, w.devices)
+    b.eval_policies(w.policies, 4)
+    sb = b.reduce_stats()
+    for p in range(len(w.policies)):
+        assert bytes(sa[p]) == bytes(sb[p])
+
+
+def test_non_default_stream_and_partial_outputs():
+    import torch
+    w = synth.make_workload(1, n=3000, n_budgets=4)
+    st = torch.cuda.Stream()
+    t = Trace.from_workload(w, stream=st)
+    out = t.alloc_pair_outputs(4, ["ttft_s", "decision"])
+    with torch.cuda.stream(st):
+        t.eval_policies(w.policies, 1, out)
+        gs = t.reduce_stats()
+    from oracle import Oracle
+    os_, oout = Oracle.from_workload(w).eval(w.policies, 1, pairs=True)
+    check_stats(gs, os_, t.histograms, "stream")
+    assert (out["decision"].cpu().numpy() == oout["decision"]).all()
+
+
+def test_invalid_inputs_are_rejected():
+    ok = constructed([10, 20], [5, 5], [0.3, 0.4])
+    def load(**kw):
+        d = dict(ok); d.update(kw)
+        return Trace().load_trace(d["prompt_len"], d["output_len"], d["server_ttft_s"], d["server_profile"],
+                                  d["device_profile"], d["servers"], d["devices"])
+    for bad in [dict(prompt_len=np.array([0, 5], np.int32)), dict(prompt_len=np.array([4097, 5], np.int32)),
+                dict(output_len=np.array([5, 8193], np.int32)), dict(output_len=np.array([0, 1], np.int32)),
+                dict(server_ttft_s=np.array([np.nan, 1.0], np.float32)),
+                dict(server_ttft_s=np.array([0.0, 1.0], np.float32)),
+                dict(server_ttft_s=np.array([np.inf, 1.0], np.float32)),
+                dict(server_profile=np.array([0, 1], np.uint8)),
+                dict(servers=[synth.server(tbt_s=0.0)]), dict(devices=[synth.device(0.0, 20.0)]),
+                dict(servers=[synth.server(jitter=1.5)])]:
+        with pytest.raises(DiscoError) as ei:
+            load(**bad)
+        assert ei.value.code == -1
+    t = load()
+    for badpol in [synth.policy(1.5), synth.policy(0.5, alpha=0.0), synth.policy(0.5, mig_threshold=-1.0),
+                   synth.policy(0.5, r_c=0.0), synth.policy(0.5, flags=3 << 2), synth.policy(float("nan"))]:
+        with pytest.raises(DiscoError) as ei:
+            t.eval_policies([badpol], 0)
+        assert ei.value.code == -1
+    with pytest.raises(DiscoError):
+        t.reduce_stats()                      # nothing evaluated
+    # a stream that could outlast the 32-bit tick range is refused, not wrapped
+    slow = constructed([10], [8192], [0.3])
+    t2 = Trace().load_trace(slow["prompt_len"], slow["output_len"], slow["server_ttft_s"], None, None,
+                            slow["servers"], slow["devices"])
+    with pytest.raises(DiscoError) as ei:
+        t2.eval_policies([synth.policy(0.5, r_c=2.0)], 0)
+    assert ei.value.code == -1
