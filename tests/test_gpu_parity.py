@@ -68,12 +68,17 @@ def test_generation_slower_than_consumption():
 def test_edge_cases():
     # single-token outputs, longest outputs, extreme prompts, ties at S = Td, one request
     tr = constructed([1, 4096, 45, 45, 45, 7, 4096], [1, 8192, 2, 1, 8192, 3, 1],
-                     [1e-3, 1999.0, 0.1, 0.1, 0.100001, 0.05, 1.0],
+                     [1e-3, 400.0, 0.1, 0.1, 0.100001, 0.05, 1.0],
                      devices=[synth.device(500.0, 20.0, ttft_intercept_s=0.01, jitter=0.05)],
                      servers=[synth.server(jitter=0.2)])
     w = synth.Workload(name="edges", seed=3, materialise=True, policies=[], **tr)
     pols = [synth.policy(b, flags=f | md) for b in (0.0, 0.5, 1.0) for f in (MIG | PACE, PACE) for md in (S_MODE, D_MODE)]
     full_parity(w, pols, tag="edges")
+    # the largest server TTFT the loader accepts, with outputs short enough for the 32-bit tick range
+    far = synth.Workload(name="far", seed=2, materialise=True, policies=[],
+                         **constructed([300, 20, 4096], [500, 40, 2], [2000.0, 1999.5, 0.2],
+                                       devices=[synth.device(500.0, 20.0, c_prefill=5e-3, c_decode=5e-3)]))
+    full_parity(far, [synth.policy(b) for b in (0.0, 0.5, 1.0)], tag="far")
     one = synth.Workload(name="one", seed=1, materialise=True, policies=[],
                          **constructed([100], [50], [0.2]))
     full_parity(one, [synth.policy(1.0)], tag="one")
