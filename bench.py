@@ -1,0 +1,304 @@
+#!/usr/bin/env python
+"""Throughput of the DiSCo policy-evaluation path on B200: request-policy evaluations per second.
+
+One step = one pass of the whole path over one synthetic workload: trace ingestion (ticks, p(l), sorted
+F), Algorithms 1-3 for every policy, token-by-token play-out, per-pair evaluation with the per-pair
+arrays written (workloads 0 and 1), per-policy reductions and policy selection.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference]
+
+`value` is measured with the trace arrays already resident in HBM; `e2e` goes through the same calls with
+pinned host arrays (host->device copies and the statistics read-back inside the timed region).  With
+N > 1 (torchrun) every rank evaluates an independent trace of the same shape (weak scaling, no
+collective on the data path).  `--impl reference` times the CPU oracle on the host cores instead.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "request-policy evaluations/s"
+UNIT = "pairs/s"
+PAIR_OUT_BYTES = 31          # four fp32, three u32, one u16, one u8 per pair
+TRACE_BYTES = 9              # packed request: ticks, prompt, output length, group
+# Lane-instructions a token-step needs for the three streams that share one hash draw:
+# hash 10, two range maps 4, three Lindley steps of 6 (subtract, max, subtract, add, max, compare-count).
+PLAYOUT_INSTR_PER_TOKEN = 32
+SM_COUNT, SCHEDULERS, LANES = 148, 4, 32
+# DRAM bytes per launch from the committed ncu capture of the dominant kernel (None until captured for
+# the current kernel; see profiles/).
+NCU_TRAFFIC_BYTES = {"pairs": None, "playout": None}
+
+
+def env_rank():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), float(d.get("sm_max_mhz", 1965.0)), "measured"
+    return 6650.0, 1965.0, "fallback"
+
+
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc = index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_sample_run(w, n_req, threads):
+    """Times the oracle, as it stands, on the first n_req requests under every policy of w, one thread per
+    contiguous request range.  Returns seconds."""
+    from concurrent.futures import ThreadPoolExecutor
+    from oracle import Oracle
+    orc = oracle_sample_run.cache.get(id(w))
+    if orc is None:
+        orc = Oracle.from_workload(w)
+        oracle_sample_run.cache[id(w)] = orc
+    threads = max(1, min(threads, n_req))
+    bounds = [n_req * k // threads for k in range(threads + 1)]
+    t0 = time.perf_counter()
+    if threads == 1:
+        orc.eval(w.policies, w.seed, 0, n_req, finish=False)
+    else:
+        with ThreadPoolExecutor(threads) as ex:
+            list(ex.map(lambda k: orc.eval(w.policies, w.seed, bounds[k], bounds[k + 1], finish=False),
+                        range(threads)))
+    return time.perf_counter() - t0
+
+
+oracle_sample_run.cache = {}
+
+
+def size_oracle_sample(w, threads, seconds):
+    probe = min(w.n, max(threads * 64, 2048))
+    t = oracle_sample_run(w, probe, threads)
+    return int(min(w.n, max(probe, probe * seconds / max(t, 1e-4))))
+
+
+def run_reference(args):
+    rank, _, world = env_rank()
+    if rank != 0:
+        return 0
+    from paper_2502_11417_b200 import synth
+    w = synth.make_workload(args.config)
+    cores = os.cpu_count() or 1
+    n_req = size_oracle_sample(w, cores, args.oracle_step_seconds)
+    for _ in range(args.warmup):
+        oracle_sample_run(w, n_req, cores)
+    times = [oracle_sample_run(w, n_req, cores) for _ in range(args.steps)]
+    pairs = n_req * w.n_policies
+    toks = int(w.output_len[:n_req].sum()) * w.n_policies
+    total = sum(times)
+    value = pairs * args.steps / total
+    sample = "first %d of %d requests x all %d policies per step" % (n_req, w.n, w.n_policies)
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "impl": "reference", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+            "sim_tokens_per_s": toks * args.steps / total,
+            "config": {"workload": w.name, "requests": w.n, "policies": w.n_policies, "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": min(cores, n_req), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+def run_ours(args):
+    import torch
+    rank, local_rank, world = env_rank()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    from paper_2502_11417_b200 import synth, Trace
+    from paper_2502_11417_b200.api import policy_array, kernel_launch_count, PolicyStats
+    import ctypes
+
+    w = synth.make_workload(args.config, replica=rank)
+    P, n = w.n_policies, w.n
+    pols = policy_array(w.policies)
+    host = [torch.from_numpy(x).pin_memory() for x in (w.prompt_len, w.output_len, w.server_ttft_s,
+                                                       w.server_profile, w.device_profile)]
+    dev = [x.cuda() for x in host]
+    h2d = sum(x.numel() * x.element_size() for x in host) + P * ctypes.sizeof(pols[0])
+    d2h = P * ctypes.sizeof(PolicyStats) + 8
+    tr = Trace()
+    tr.n = n
+    out = None
+    if w.materialise:
+        tr.load_trace(*dev, w.servers, w.devices)
+        out = tr.alloc_pair_outputs(P)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")       # larger than the 126 MB L2
+    stream = torch.cuda.current_stream()
+    tr.load_trace(*dev, w.servers, w.devices)
+    tr.set_timing(True)
+    cap_factor, slo = w.select["cost_cap_factor"], w.select["tbt_slo_s"]
+
+    def step(arrays):
+        tr.load_trace(*arrays, w.servers, w.devices)
+        tr.eval_policies(pols, w.seed, out)
+        st = tr.reduce_stats()
+        cap = cap_factor * min(st[p].total_cost for p in range(P))
+        return tr.select_policy(cap, slo)
+
+    def timed(arrays, steps, warmup, collect=None):
+        for _ in range(warmup):
+            step(arrays)
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        evs = []
+        for _ in range(steps):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            step(arrays)
+            e1.record(stream)
+            evs.append((e0, e1))
+            if collect is not None:
+                collect.append(tr.timing())
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        total_ms = sum(a.elapsed_time(b) for a, b in evs)
+        if dist is not None:
+            t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            total_ms = float(t.item())
+        return total_ms
+
+    sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else
+                           os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank])
+    ktimes = []
+    l0 = kernel_launch_count()
+    timed(dev, 0, args.warmup)
+    l_warm = kernel_launch_count()
+    sampler.start()
+    total_ms = timed(dev, args.steps, 0, ktimes)
+    clocks = sampler.stop()
+    launches = kernel_launch_count() - l_warm
+    e2e_ms = timed(host, args.steps, args.warmup)
+
+    pairs = n * P * world
+    toks = int(w.output_len.sum()) * P * world          # approximate for N > 1: replicas have like shapes
+    value = pairs * args.steps / (total_ms * 1e-3)
+    e2e_value = pairs * args.steps / (e2e_ms * 1e-3)
+
+    # ---- roofline of the dominant kernel of a step
+    hbm_gbs, sm_max_mhz, src = measured_peaks()
+    play_ms = statistics.mean(t[0] for t in ktimes)
+    pair_ms = statistics.mean(t[1] for t in ktimes)
+    token_steps = int((w.output_len - 1).sum())
+    if pair_ms >= play_ms:
+        bytes_alg = n * P * (PAIR_OUT_BYTES if w.materialise else 0) + n * TRACE_BYTES
+        ach = bytes_alg / (pair_ms * 1e-3) / 1e9
+        roof = {"kernel": "k_pairs", "bound": "hbm", "achieved": ach, "peak": hbm_gbs, "unit": "GB/s",
+                "frac": ach / hbm_gbs, "traffic": NCU_TRAFFIC_BYTES["pairs"], "peak_source": src,
+                "algorithmic_bytes": bytes_alg, "ms_per_launch": pair_ms}
+    else:
+        peak = SM_COUNT * SCHEDULERS * LANES * sm_max_mhz * 1e6 / 1e12     # T lane-instructions/s
+        ach = token_steps * PLAYOUT_INSTR_PER_TOKEN / (play_ms * 1e-3) / 1e12
+        roof = {"kernel": "k_timeline", "bound": "alu", "achieved": ach, "peak": peak, "unit": "Tinstr/s",
+                "frac": ach / peak, "traffic": NCU_TRAFFIC_BYTES["playout"],
+                "peak_source": "148 SMs x 4 schedulers x 32 lanes x %.0f MHz" % sm_max_mhz,
+                "token_steps": token_steps, "ms_per_launch": play_ms}
+    roof["other_kernels_ms"] = {"k_timeline": play_ms, "k_pairs": pair_ms}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return 0
+    cpu = None
+    if world == 1:
+        cores = os.cpu_count() or 1
+        n_req = size_oracle_sample(w, cores, args.oracle_seconds)
+        t = oracle_sample_run(w, n_req, cores)
+        cpu = {"value": n_req * P / t, "unit": UNIT, "cores": min(cores, n_req), "kind": "oracle",
+               "sample": "first %d of %d requests x all %d policies, %.1f s" % (n_req, n, P, t),
+               "sim_tokens_per_s": int(w.output_len[:n_req].sum()) * P / t}
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+            "sim_tokens_per_s": toks * args.steps / (total_ms * 1e-3),
+            "config": {"workload": w.name, "requests_per_gpu": n, "policies": P, "pairs_per_step": pairs,
+                       "per_pair_outputs": bool(w.materialise), "l2": "flushed between steps (512 MB write)",
+                       "seed": w.seed},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": e2e_ms / args.steps},
+            "gpu_launches": launches,
+            "roofline": roof, "cpu_baseline": cpu}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=1, help="workload 0..4 (default: workload 1)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--oracle-seconds", type=float, default=15.0, help="CPU time of the oracle baseline sample")
+    ap.add_argument("--oracle-step-seconds", type=float, default=3.0, help="--impl reference: CPU time per step")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    return run_reference(args) if args.impl == "reference" else run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

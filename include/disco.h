@@ -172,6 +172,14 @@ int disco_get_prep(disco_ctx_t* ctx, uint32_t g, uint32_t p, disco_prep_t* out, 
 int64_t disco_get_group_tables(disco_ctx_t* ctx, uint32_t g, int64_t* cnt, int32_t* knots,
                                int32_t* sorted_ticks, uint64_t n_sorted, void* stream);
 
+/* Measurement aids.  disco_set_timing(ctx, 1) makes each evaluation record CUDA events on its stream around
+ * the play-out kernel and the pair kernel; after disco_reduce_stats, disco_get_timing returns their device
+ * durations in milliseconds (only for evaluations whose policies share one pacing / buffer setting).
+ * disco_kernel_launch_count returns how many kernels this library has launched in this process. */
+int disco_set_timing(disco_ctx_t* ctx, int on);
+int disco_get_timing(disco_ctx_t* ctx, float* playout_ms, float* pairs_ms);
+uint64_t disco_kernel_launch_count(void);
+
 void disco_free_trace(disco_ctx_t* ctx);
 const char* disco_last_error(void);
 

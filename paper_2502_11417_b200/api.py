@@ -74,7 +74,7 @@ class Prep(C.Structure):
 
 EXPORTS = ["disco_load_trace", "disco_eval_policies", "disco_reduce_stats", "disco_select_policy",
            "disco_get_histograms", "disco_get_prep", "disco_get_group_tables", "disco_free_trace",
-           "disco_last_error"]
+           "disco_last_error", "disco_set_timing", "disco_get_timing", "disco_kernel_launch_count"]
 
 PAIR_FIELDS = [("ttft_s", "float32"), ("tbt_mean_s", "float32"), ("tbt_max_s", "float32"), ("cost", "float32"),
                ("tok_server", "uint32"), ("tok_device", "uint32"), ("mig_at", "uint32"), ("delayed", "uint16"),
@@ -105,8 +105,16 @@ def lib() -> C.CDLL:
         L.disco_get_group_tables.argtypes = [vp, u32, vp, vp, vp, u64, vp]
         L.disco_free_trace.restype = None; L.disco_free_trace.argtypes = [vp]
         L.disco_last_error.restype = C.c_char_p
+        L.disco_set_timing.restype = C.c_int; L.disco_set_timing.argtypes = [vp, C.c_int]
+        L.disco_get_timing.restype = C.c_int
+        L.disco_get_timing.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_float)]
+        L.disco_kernel_launch_count.restype = u64; L.disco_kernel_launch_count.argtypes = []
         _lib = L
     return _lib
+
+
+def kernel_launch_count() -> int:
+    return int(lib().disco_kernel_launch_count())
 
 
 def _check(rc: int, allow=()):
@@ -269,6 +277,15 @@ class Trace:
         if rc < 0:
             _check(int(rc))
         return cnt, kn, srt[:k]
+
+    def set_timing(self, on: bool = True):
+        _check(lib().disco_set_timing(self._h, int(on)))
+
+    def timing(self):
+        """(play-out ms, pair-kernel ms) of the last reduced evaluation."""
+        a, b = C.c_float(), C.c_float()
+        _check(lib().disco_get_timing(self._h, C.byref(a), C.byref(b)))
+        return a.value, b.value
 
     def close(self):
         if self._h:

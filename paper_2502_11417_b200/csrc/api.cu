@@ -1,6 +1,7 @@
 // Host side of the C ABI: argument checks, device memory, launch order.  No arithmetic of the method runs
 // here apart from turning the handful of profile and policy parameters into ticks.
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -16,6 +17,7 @@ using namespace disco;
 namespace {
 
 thread_local std::string g_err;
+std::atomic<uint64_t> g_launches{0};   // kernels launched by this library, all contexts
 
 int fail(int code, const std::string& msg) { g_err = msg; return code; }
 int fail_cuda(cudaError_t e, const char* what) {
@@ -80,6 +82,10 @@ struct disco_ctx {
     size_t stage_cap = 0;
     cudaEvent_t stage_free = nullptr;
     int32_t* sel_host = nullptr; // pinned [2]
+    bool timing = false;         // record events around the play-out and pair kernels
+    cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
+    float ms_timeline = 0.f, ms_pairs = 0.f;
+    bool timing_valid = false;
 
     ~disco_ctx() {
         DevBuf* all[] = {&in_prompt, &in_out, &in_ttft, &in_sp, &in_dp, &keys_a, &keys_b, &tmp_idx, &radix_counts,
@@ -94,6 +100,7 @@ struct disco_ctx {
         if (stage) cudaFreeHost(stage);
         if (sel_host) cudaFreeHost(sel_host);
         if (stage_free) cudaEventDestroy(stage_free);
+        for (auto& e : ev) if (e) cudaEventDestroy(e);
     }
 };
 
@@ -219,6 +226,7 @@ int disco_load_trace(disco_ctx_t** pctx, const disco_trace_desc_t* d, void* stre
     if ((e = cudaMemcpyAsync(c->d_gc.p, c->gc.data(), c->gc.size() * sizeof(GroupConst), cudaMemcpyHostToDevice, st)) != cudaSuccess)
         return bail(fail_cuda(e, "profile copy"));
     if ((e = run_load(a, st)) != cudaSuccess) return bail(fail_cuda(e, "trace ingestion kernels"));
+    g_launches += load_kernel_launches(n, c->G) + 1;
     // read back the few numbers the host needs: error word, group sizes, longest output, largest TTFT per group
     HostReadback* rb = c->rb;
     k_knot_max<<<1, kMaxGroups, 0, st>>>(c->G, a.knots, (int32_t*)c->tmp_idx.p);
@@ -398,14 +406,22 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
     if (out) po = *out;
 
     // ---- per timeline class: play every request out, then evaluate the class's policies on the summaries
+    g_launches += 1;
+    c->timing_valid = false;
+    const bool timed = c->timing && classes.size() == 1;
     for (size_t k = 0; k < classes.size(); ++k) {
         const ClassConst* dcc = c->d_classes.as<ClassConst>() + k;
+        if (timed) CU(cudaEventRecord(c->ev[0], st));
         CU(launch_timeline(tr, c->d_gc.as<GroupConst>(), dcc, c->knots.as<int32_t>(), seed, rec, c->err.as<int32_t>(), st));
+        if (timed) CU(cudaEventRecord(c->ev[1], st));
         CU(launch_pairs(tr, c->d_gc.as<GroupConst>(), dcc, c->d_prep.as<Prep>(), P,
                         c->d_pol_list.as<uint32_t>() + cls_range[k].first, cls_range[k].second - cls_range[k].first,
                         c->d_chunks.as<Chunk>(), (uint32_t)chunks.size(), rec, po, c->d_acc.as<uint64_t>(),
                         c->d_hist_ttft.as<uint64_t>(), c->d_hist_tbt.as<uint64_t>(), st));
+        if (timed) CU(cudaEventRecord(c->ev[2], st));
+        g_launches += (n ? 1 : 0) + ((n && !chunks.empty()) ? 1 : 0);
     }
+    c->timing_valid = timed && n != 0;
     c->P = P; c->pol = pc;
     c->evaluated = true;
     return 0;
@@ -421,6 +437,11 @@ int disco_reduce_stats(disco_ctx_t* c, disco_policy_stats_t* stats, void* stream
     CU(cudaMemcpyAsync(stats, c->d_stats.p, c->P * sizeof(disco_policy_stats_t), cudaMemcpyDeviceToHost, st));
     CU(cudaMemcpyAsync(c->rb->err, c->err.p, 16, cudaMemcpyDeviceToHost, st));
     CU(cudaStreamSynchronize(st));
+    g_launches += 1;
+    if (c->timing_valid) {
+        CU(cudaEventElapsedTime(&c->ms_timeline, c->ev[0], c->ev[1]));
+        CU(cudaEventElapsedTime(&c->ms_pairs, c->ev[1], c->ev[2]));
+    }
     if (c->rb->err[2]) return fail(DISCO_ECUDA, "internal error: an inter-token interval fell outside its histogram window");
     c->reduced = true;
     return 0;
@@ -431,11 +452,29 @@ int disco_select_policy(disco_ctx_t* c, double cost_cap, float tbt_slo_s, int32_
     if (!c->reduced) return fail(DISCO_EINVAL, "reduce the statistics before selecting");
     cudaStream_t st = (cudaStream_t)stream;
     if (!c->sel_host) CU(cudaMallocHost((void**)&c->sel_host, 8));
+    g_launches += 1;
     CU(launch_select(c->d_stats.as<disco_policy_stats_t>(), c->P, cost_cap, tbt_slo_s, c->d_select.as<int32_t>(), st));
     CU(cudaMemcpyAsync(c->sel_host, c->d_select.p, 8, cudaMemcpyDeviceToHost, st));
     CU(cudaStreamSynchronize(st));
     *best = c->sel_host[1];
     if (c->sel_host[0] != 0) return fail(DISCO_EINFEASIBLE, "no policy meets the cost cap and the TBT objective");
+    return 0;
+}
+
+uint64_t disco_kernel_launch_count(void) { return g_launches.load(); }
+
+int disco_set_timing(disco_ctx_t* c, int on) {
+    if (!c) return fail(DISCO_EINVAL, "null context");
+    if (on) for (auto& e : c->ev) if (!e) CU(cudaEventCreate(&e));
+    c->timing = on != 0;
+    c->timing_valid = false;
+    return 0;
+}
+
+int disco_get_timing(disco_ctx_t* c, float* playout_ms, float* pairs_ms) {
+    if (!c || !playout_ms || !pairs_ms) return fail(DISCO_EINVAL, "null argument");
+    if (!c->timing_valid || !c->reduced) return fail(DISCO_EINVAL, "no timed evaluation has been reduced");
+    *playout_ms = c->ms_timeline; *pairs_ms = c->ms_pairs;
     return 0;
 }
 

@@ -202,6 +202,12 @@ cudaError_t radix_pass(const uint64_t* kin, uint64_t* kout, const uint32_t* pin,
 
 }  // namespace
 
+uint32_t load_kernel_launches(uint32_t n, int G) {
+    if (n == 0) return 2;
+    const uint32_t passes = G > 1 ? 6 : 4;       // radix passes: partition + 5, or 4
+    return 1 + 1 + 3 * passes + 1 + 2;            // ingest, gather, passes, low words, group tables
+}
+
 cudaError_t run_load(const LoadArgs& a, cudaStream_t st) {
     const uint32_t n = a.n;
     const int G = (int)(a.ns * a.nd);

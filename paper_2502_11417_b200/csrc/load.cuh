@@ -30,5 +30,6 @@ struct LoadArgs {
 };
 
 cudaError_t run_load(const LoadArgs& a, cudaStream_t st);
+uint32_t load_kernel_launches(uint32_t n, int G);   // kernels run_load launches for such a trace
 
 }  // namespace disco

@@ -86,13 +86,16 @@ def budget_grid(k: int) -> List[float]:
 _SIZES = {0: 1_000, 1: 100_000, 2: 1_000_000, 3: 4_000_000, 4: 16_000_000}
 
 
-def make_workload(cfg: int, n: Optional[int] = None, n_budgets: Optional[int] = None) -> Workload:
+def make_workload(cfg: int, n: Optional[int] = None, n_budgets: Optional[int] = None,
+                  replica: int = 0) -> Workload:
     """Build workload ``cfg`` (0..4).  ``n`` / ``n_budgets`` shrink the request
-    count / the budget axis for parity tests; distributions stay the same."""
+    count / the budget axis for parity tests; distributions stay the same.
+    ``replica`` > 0 draws an independent trace of the same shape (one per GPU
+    in a multi-GPU run)."""
     if cfg not in _SIZES:
         raise ValueError("cfg must be 0..4")
     n = _SIZES[cfg] if n is None else int(n)
-    rng = np.random.Generator(np.random.PCG64(cfg))
+    rng = np.random.Generator(np.random.PCG64(cfg if replica == 0 else [cfg, replica]))
 
     prompt = _lengths(rng, n, 5.5, 1.0, 16, 4096)
     if cfg == 3:
