@@ -180,6 +180,37 @@ int disco_set_timing(disco_ctx_t* ctx, int on);
 int disco_get_timing(disco_ctx_t* ctx, float* playout_ms, float* pairs_ms);
 uint64_t disco_kernel_launch_count(void);
 
+/* Sorting without allocating.  (The paper has no counterpart to this call; it exists for the sake of
+ * callers, not of the method.)
+ *
+ * Some programs that use this library may not allocate device memory at the point where they need a
+ * result: a serving loop whose memory pool already owns the whole GPU and treats any further cudaMalloc
+ * as an error, code that runs between the launches of a latency-critical stream where the implicit
+ * synchronisation of cudaMalloc/cudaFree is unacceptable, or a plug-in that is handed device pointers
+ * but no allocator.  disco_load_trace is closed to them, because it sizes and allocates a context.
+ *
+ * This call does the part of the load step that turns server TTFTs into the empirical distribution F of
+ * Algorithm 1 -- seconds to microsecond ticks (nearest, ties to even), then an ascending sort -- for ONE
+ * group of at most DISCO_NOALLOC_MAX_N requests.  Input and output are the caller's device arrays
+ * (server_ttft_s[n] in, sorted_ticks[n] out); the sort's working memory is a fixed array of about 4.3 MB
+ * that is part of the library image, so it occupies that much memory on every GPU the library is loaded
+ * on, from load until the process exits.  The call makes no cudaMalloc, cudaFree or other allocating
+ * call.  It returns the same ticks, in the same order, as disco_load_trace followed by
+ * disco_get_group_tables on a one-group trace.
+ *
+ *  - n > DISCO_NOALLOC_MAX_N is refused with DISCO_EINVAL (use disco_load_trace); a TTFT that is not
+ *    finite, not positive or above 2000 s gives DISCO_EINVAL after the kernels have run.
+ *  - The first call on each device looks up the device address of the working array; make that first
+ *    call during start-up, on the device you will use (cudaSetDevice first) and before any stream
+ *    capture begins.
+ *  - All calls on a device share the one working array, which still holds the previous call's data
+ *    (the call clears what it needs cleared).  Two calls whose kernels could run at the same time on
+ *    one GPU -- different streams, different host threads -- race on it: serialise them.
+ *  - Synchronises `stream` before returning. */
+#define DISCO_NOALLOC_MAX_N 262144u
+int disco_sort_ttft_ticks_noalloc(const float* server_ttft_s /* device */, uint32_t n,
+                                  int32_t* sorted_ticks /* device */, void* stream);
+
 void disco_free_trace(disco_ctx_t* ctx);
 const char* disco_last_error(void);
 

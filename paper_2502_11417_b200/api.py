@@ -74,7 +74,7 @@ class Prep(C.Structure):
 
 EXPORTS = ["disco_load_trace", "disco_eval_policies", "disco_reduce_stats", "disco_select_policy",
            "disco_get_histograms", "disco_get_prep", "disco_get_group_tables", "disco_free_trace",
-           "disco_last_error", "disco_set_timing", "disco_get_timing", "disco_kernel_launch_count"]
+           "disco_last_error", "disco_set_timing", "disco_get_timing", "disco_kernel_launch_count", "disco_sort_ttft_ticks_noalloc"]
 
 PAIR_FIELDS = [("ttft_s", "float32"), ("tbt_mean_s", "float32"), ("tbt_max_s", "float32"), ("cost", "float32"),
                ("tok_server", "uint32"), ("tok_device", "uint32"), ("mig_at", "uint32"), ("delayed", "uint16"),
@@ -109,6 +109,8 @@ def lib() -> C.CDLL:
         L.disco_get_timing.restype = C.c_int
         L.disco_get_timing.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_float)]
         L.disco_kernel_launch_count.restype = u64; L.disco_kernel_launch_count.argtypes = []
+        L.disco_sort_ttft_ticks_noalloc.restype = C.c_int
+        L.disco_sort_ttft_ticks_noalloc.argtypes = [vp, u32, vp, vp]
         _lib = L
     return _lib
 
@@ -154,6 +156,27 @@ def policy_array(policies: Sequence[Dict[str, float]]):
     for k, p in enumerate(policies):
         arr[k] = Policy(p["budget"], p["alpha"], p["mig_threshold"], p["t_m_s"], p["r_c"], p["flags"])
     return arr
+
+
+NOALLOC_MAX_N = 262144
+
+
+def sort_ttft_ticks_noalloc(server_ttft_s, sorted_ticks, stream=None):
+    """disco_sort_ttft_ticks_noalloc: server_ttft_s is a CUDA float32 tensor [n], sorted_ticks a CUDA int32
+    tensor [n] that receives the ascending microsecond ticks.  The library allocates nothing in this call;
+    both tensors are the caller's.  Calls on one GPU must not overlap (they share one working array)."""
+    import torch
+    for t, dt in ((server_ttft_s, torch.float32), (sorted_ticks, torch.int32)):
+        if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == dt and t.is_contiguous() and t.dim() == 1):
+            raise ValueError("expected contiguous 1-D CUDA tensors: float32 in, int32 out")
+    if server_ttft_s.numel() != sorted_ticks.numel():
+        raise ValueError("input and output lengths differ")
+    n = server_ttft_s.numel()
+    if n >= 1 << 32:
+        raise ValueError("too many requests")
+    _check(lib().disco_sort_ttft_ticks_noalloc(server_ttft_s.data_ptr() if n else None, n,
+                                               sorted_ticks.data_ptr() if n else None, _stream_ptr(stream)))
+    return sorted_ticks
 
 
 class Trace:

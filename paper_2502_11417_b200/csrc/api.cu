@@ -61,6 +61,10 @@ __global__ void k_knot_max(int G, const int32_t* __restrict__ knots, int32_t* __
 
 }  // namespace
 
+namespace disco {
+int set_error(int code, const char* msg) { return fail(code, msg); }
+}  // namespace disco
+
 struct disco_ctx {
     uint32_t n = 0, ns = 0, nd = 0;
     int G = 0;

@@ -114,6 +114,9 @@ inline int host_bin_of_ticks(int64_t t) {
     return (int)(b < kNBins - 1 ? b : kNBins - 1);
 }
 
+// Records the calling thread's error message (read back by disco_last_error) and returns `code`.
+int set_error(int code, const char* msg);
+
 // ---- launch wrappers (defined in the kernel translation units) -------------------------------------------
 cudaError_t launch_prep(const PolicyConst* pol, uint32_t P, int G, const GroupConst* gc, const int64_t* cum_mass,
                         const uint32_t* cnt, const int32_t* sorted, const uint32_t* grp_off, Prep* prep,

@@ -3,6 +3,8 @@
 // Algorithm 1), cumulative input-token mass (Eq. 3) and the quantile knots of F.
 #include "load.cuh"
 
+#include <mutex>
+
 namespace disco {
 
 namespace {
@@ -242,3 +244,85 @@ cudaError_t run_load(const LoadArgs& a, cudaStream_t st) {
 }
 
 }  // namespace disco
+
+
+// -----------------------------------------------------------------------------------------------------
+// Sorting server TTFTs without allocating.  The scratch the radix sort needs (two key buffers, the digit
+// counters, an error word) lives in a fixed array inside the library image instead of in cudaMalloc'd
+// memory.  Every GPU that loads the library carries these bytes until the process exits, and every call
+// on a GPU uses the same bytes.
+// -----------------------------------------------------------------------------------------------------
+namespace disco {
+namespace {
+
+constexpr uint32_t kNoAllocMaxN = DISCO_NOALLOC_MAX_N;
+constexpr size_t kNaKeysBytes = (size_t)kNoAllocMaxN * sizeof(uint64_t);
+constexpr size_t kNaCountsBytes = 256u * ((kNoAllocMaxN + 4095u) / 4096u) * sizeof(uint32_t);
+constexpr size_t kNaErrOff = 2 * kNaKeysBytes + kNaCountsBytes;
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNaErrOff + 256];
+
+__global__ void k_ttft_keys(uint32_t n, const float* __restrict__ ttft, uint64_t* __restrict__ keys,
+                            int32_t* __restrict__ err) {
+    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+        const float t = ttft[i];
+        if (!(t > 0.0f) || !(t <= 2000.0f)) {
+            if (atomicCAS(&err[0], 0, 3) == 0) err[1] = (int32_t)i;
+            keys[i] = 0;
+            continue;
+        }
+        keys[i] = (uint64_t)(uint32_t)__double2ll_rn(__dmul_rn((double)t, 1e6));
+    }
+}
+
+std::mutex g_na_mutex;
+unsigned char* g_na_base[64] = {};        // device address of the scratch array, per device ordinal
+
+}  // namespace
+}  // namespace disco
+
+extern "C" int disco_sort_ttft_ticks_noalloc(const float* server_ttft_s, uint32_t n, int32_t* sorted_ticks,
+                                             void* stream) {
+    using namespace disco;
+    if (n > kNoAllocMaxN)
+        return set_error(DISCO_EINVAL, "disco_sort_ttft_ticks_noalloc: n exceeds DISCO_NOALLOC_MAX_N (262144); "
+                                       "use disco_load_trace for larger traces");
+    if (n && (!server_ttft_s || !sorted_ticks)) return set_error(DISCO_EINVAL, "null array");
+    if (n == 0) return 0;
+    cudaStream_t st = (cudaStream_t)stream;
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return set_error(DISCO_ECUDA, cudaGetErrorString(e));
+    if (dev < 0 || dev >= 64) return set_error(DISCO_EINVAL, "device ordinal above 63");
+    unsigned char* base;
+    {
+        // In host code the array's name is only a handle; its address on the current device has to be asked for.
+        std::lock_guard<std::mutex> lock(g_na_mutex);
+        if (!g_na_base[dev]) {
+            e = cudaGetSymbolAddress((void**)&g_na_base[dev], g_noalloc_scratch);
+            if (e != cudaSuccess) { g_na_base[dev] = nullptr; return set_error(DISCO_ECUDA, cudaGetErrorString(e)); }
+        }
+        base = g_na_base[dev];
+    }
+    uint64_t* keys_a = (uint64_t*)base;
+    uint64_t* keys_b = (uint64_t*)(base + kNaKeysBytes);
+    uint32_t* counts = (uint32_t*)(base + 2 * kNaKeysBytes);
+    int32_t* err = (int32_t*)(base + kNaErrOff);
+    // the array still holds the previous call's data: the error word must start at zero; keys and counters
+    // are fully rewritten for the first n entries before they are read
+    if ((e = cudaMemsetAsync(err, 0, 16, st)) != cudaSuccess) return set_error(DISCO_ECUDA, cudaGetErrorString(e));
+    k_ttft_keys<<<grid_for(n, 256), 256, 0, st>>>(n, server_ttft_s, keys_a, err);
+    uint64_t *src = keys_a, *dst = keys_b;
+    for (int p = 0; p < 4; ++p) {
+        if ((e = radix_pass(src, dst, nullptr, nullptr, n, 8 * p, counts, st)) != cudaSuccess)
+            return set_error(DISCO_ECUDA, cudaGetErrorString(e));
+        uint64_t* t = src; src = dst; dst = t;
+    }
+    k_low_words<<<grid_for(n, 256), 256, 0, st>>>(n, src, sorted_ticks);
+    int32_t h_err[2] = {0, 0};
+    if ((e = cudaMemcpyAsync(h_err, err, sizeof h_err, cudaMemcpyDeviceToHost, st)) != cudaSuccess ||
+        (e = cudaStreamSynchronize(st)) != cudaSuccess)
+        return set_error(DISCO_ECUDA, cudaGetErrorString(e));
+    if (h_err[0]) return set_error(DISCO_EINVAL, "server TTFT not finite, not positive or above 2000 s");
+    return 0;
+}
