@@ -128,7 +128,7 @@ def run_reference(args):
     if rank != 0:
         return 0
     from paper_2502_11417_b200 import synth
-    w = synth.make_workload(args.config)
+    w = synth.make_workload(args.config, n=args.requests, n_budgets=args.budgets)
     cores = os.cpu_count() or 1
     n_req = size_oracle_sample(w, cores, args.oracle_step_seconds)
     for _ in range(args.warmup):
@@ -165,7 +165,7 @@ def run_ours(args):
     from paper_2502_11417_b200.api import policy_array, kernel_launch_count, PolicyStats
     import ctypes
 
-    w = synth.make_workload(args.config, replica=rank)
+    w = synth.make_workload(args.config, n=args.requests, n_budgets=args.budgets, replica=rank)
     P, n = w.n_policies, w.n
     pols = policy_array(w.policies)
     host = [torch.from_numpy(x).pin_memory() for x in (w.prompt_len, w.output_len, w.server_ttft_s,
@@ -260,7 +260,7 @@ def run_ours(args):
             dist.destroy_process_group()
         return 0
     cpu = None
-    if world == 1:
+    if world == 1 and args.oracle_seconds > 0:
         cores = os.cpu_count() or 1
         n_req = size_oracle_sample(w, cores, args.oracle_seconds)
         t = oracle_sample_run(w, n_req, cores)
@@ -291,6 +291,8 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=1, help="workload 0..4 (default: workload 1)")
+    ap.add_argument("--requests", type=int, default=None, help="shrink the trace (profiling on a small case)")
+    ap.add_argument("--budgets", type=int, default=None, help="shrink the budget axis (profiling on a small case)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--oracle-seconds", type=float, default=15.0, help="CPU time of the oracle baseline sample")
     ap.add_argument("--oracle-step-seconds", type=float, default=3.0, help="--impl reference: CPU time per step")
