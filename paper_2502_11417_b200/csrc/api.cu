@@ -323,7 +323,7 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
             }
         }
         for (int k = 0; k < 3; ++k) cc.W[k] = Wmax[k];
-        const size_t win_bytes = (size_t)n * (Wmax[0] + Wmax[1] + Wmax[2]) * 2;
+        const size_t win_bytes = (size_t)n * (Wmax[0] + Wmax[1] + Wmax[2]) * 4;
         if (win_bytes > (48ull << 30)) return fail(DISCO_ENOMEM, "per-request TBT windows would exceed 48 GB");
     }
 
@@ -339,7 +339,7 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
     R(d_classes, classes.size() * sizeof(ClassConst)); R(d_select, 8);
     for (int k = 0; k < 7; ++k) R(rec_u32[k], N1 * 4);
     for (int k = 0; k < 2; ++k) R(rec_u16[k], N1 * 2);
-    for (int k = 0; k < 3; ++k) R(rec_win[k], N1 * wmax[k] * 2);
+    for (int k = 0; k < 3; ++k) R(rec_win[k], N1 * wmax[k] * 4);
 
     // ---- policies grouped by class; request chunks (one group each) sized so that chunks x policy tiles
     //      fill the GPU about once
@@ -401,7 +401,7 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
     TimelineRec rec;
     for (int k = 0; k < 3; ++k) {
         rec.sum[k] = c->rec_u32[2 * k].as<uint32_t>(); rec.max[k] = c->rec_u32[2 * k + 1].as<uint32_t>();
-        rec.win[k] = c->rec_win[k].as<uint16_t>();
+        rec.win[k] = c->rec_win[k].as<uint32_t>();
     }
     rec.stall = c->rec_u32[6].as<uint32_t>();
     rec.m = c->rec_u16[0].as<uint16_t>(); rec.delayed = c->rec_u16[1].as<uint16_t>();

@@ -63,7 +63,7 @@ struct TimelineRec {
     uint32_t *sum[3], *max[3];   // d_n - d_1 and the largest TBT, ticks ([n] each)
     uint32_t* stall;             // TBT of the first token after a hand-off
     uint16_t *m, *delayed;       // hand-off index (0 = buffer never fills) and delayed tokens
-    uint16_t* win[3];            // [n][W[c]] counts per window bin
+    uint32_t* win[3];            // [n][W[c]] counts per window bin
 };
 
 struct TraceDev {

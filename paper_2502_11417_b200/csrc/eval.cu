@@ -1,10 +1,11 @@
-// Policy preparation (Algorithms 1-3), decode play-out per request (Sec. 4.3) and per-pair evaluation.
+// Policy preparation (Algorithms 1-3) and per-pair evaluation.
 //
 // Relative to its first token, a request's decode stream depends on a policy only through the winning
 // endpoint, the pacing interval, the buffer size and whether a hand-off happens -- not on the budget.
 // So each request is played out token by token once per timeline class for its (at most) three distinct
-// streams: server decodes all, device decodes all, and the dearer winner hands off to the other endpoint.
-// The pair kernel then derives every policy's dispatch decision and picks the stream that applies.
+// streams (playout.cu): server decodes all, device decodes all, and the dearer winner hands off to the
+// other endpoint.  The pair kernel here derives every policy's dispatch decision and picks the stream
+// that applies.
 #include "disco_internal.cuh"
 
 namespace disco {
@@ -78,130 +79,6 @@ __global__ void k_prep(const PolicyConst* __restrict__ pol, uint32_t P, int G, c
         }
     }
     prep[(size_t)g * P + p] = r;
-}
-
-// ------------------------------------------------------------------------------------------------------
-// Play-out, one thread per request (sequential over tokens).
-// ------------------------------------------------------------------------------------------------------
-struct Stream {                 // one decode timeline: Lindley form of d_j = max(g_j, d_{j-1} + tau)
-    uint32_t e;                 // d_j - g_j: how far delivery lags generation
-    uint32_t sum, mx, ntau;     // sum and max of the TBTs, and how many equal tau exactly
-};
-
-__device__ __forceinline__ uint32_t step(Stream& s, uint32_t x, uint32_t tau_eff) {
-    const int32_t t = (int32_t)x - (int32_t)s.e;                      // g_j - d_{j-1}
-    const int32_t tbt = max(t, (int32_t)tau_eff);                     // d_j - d_{j-1}
-    s.e = (uint32_t)(tbt - t);
-    s.sum += (uint32_t)tbt;
-    s.mx = max(s.mx, (uint32_t)tbt);
-    return (uint32_t)tbt;
-}
-
-__device__ __forceinline__ void count_tbt(Stream& s, uint32_t tbt, int32_t tau_fast, uint16_t* win, int lo, int W,
-                                          int32_t* err) {
-    if ((int32_t)tbt == tau_fast) { ++s.ntau; return; }
-    const int b = bin_of_ticks(tbt) - lo;
-    if (b >= 0 && b < W) win[b] += 1; else atomicExch(&err[2], 1);
-}
-
-__global__ void __launch_bounds__(128)
-k_timeline_seq(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __restrict__ ccp,
-               const int32_t* __restrict__ knots, uint32_t k0, TimelineRec rec, int32_t* err) {
-    const uint32_t k = blockIdx.x * blockDim.x + threadIdx.x;
-    if (k >= tr.n) return;
-    int g = 0;
-    while (g + 1 < tr.n_groups && k >= tr.grp_off[g + 1]) ++g;
-    const GroupConst gc = gcs[g];
-    const ClassConst& cc = *ccp;
-    const uint32_t n = tr.nout[k], l = tr.l[k];
-    const uint32_t key = mix32(k0 + tr.orig[k] * kHashReq);
-    const uint32_t tau_eff = (uint32_t)cc.tau_eff;
-    const int32_t tau = cc.tau;
-    const int32_t tau_fast = cc.pacing ? cc.tau : -1;
-    const int W0 = cc.W[0], W1 = cc.W[1], W2 = cc.W[2];
-    const int lo0 = cc.lo[g][0], lo1 = cc.lo[g][1], lo2 = cc.lo[g][2];
-    uint16_t* win0 = rec.win[0] + (size_t)k * W0;
-    uint16_t* win1 = rec.win[1] + (size_t)k * W1;
-    uint16_t* win2 = rec.win[2] + (size_t)k * W2;
-    for (int i = 0; i < W0; ++i) win0[i] = 0;
-    for (int i = 0; i < W1; ++i) win1[i] = 0;
-    for (int i = 0; i < W2; ++i) win2[i] = 0;
-
-    const uint32_t mulS = 2u * (uint32_t)gc.J_srv + 1u, baseS = (uint32_t)(gc.T_srv - gc.J_srv);
-    const uint32_t mulD = 2u * (uint32_t)gc.J_dev + 1u, baseD = (uint32_t)(gc.T_dev - gc.J_dev);
-
-    Stream sS = {0, 0, 0, 0}, sD = {0, 0, 0, 0}, sX = {0, 0, 0, 0};
-    // The stream of the dearer winner (the candidate) is searched for the hand-off index m: the first
-    // token j in [B, n-1] generated while token j-B+1 is still undelivered (buffer holds B tokens).
-    const int cand = (cc.mig_any && n >= 2) ? gc.candidate : 0;         // 1: server stream, 2: device stream
-    const uint32_t B = (uint32_t)cc.B;
-    uint32_t m = 0, stall = 0, delayed = 0, M = 0;
-    uint32_t gC = 0;                          // candidate's generation time g_j
-    uint32_t g_lag = 0, e_lag = 0;            // candidate's g and d - g at token j - B + 1
-    uint32_t h_lag = key + kHashTok;
-    int32_t slot_lag = 0;                     // g_j - d_m - (j - m) tau on the migrated stream
-    auto handoff_latency = [&](uint32_t mm) -> uint32_t {
-        if (cand == 1)                        // target = device: re-prefill prompt + generated tokens
-            return (uint32_t)gc.kappa * (l + mm) + (uint32_t)gc.c0;
-        const uint32_t u = mix32(key);        // target = server: a TTFT drawn from the group's F by its knots
-        const int32_t* K = knots + g * kNKnots;
-        const uint32_t kk = u >> 24, fr = (u >> 8) & 0xFFFFu;
-        return (uint32_t)(K[kk] + (int32_t)(((int64_t)(K[kk + 1] - K[kk]) * (int64_t)fr) >> 16));
-    };
-    if (cand && B == 0) { m = 1; M = handoff_latency(1); }   // nothing to fill: hand off after the first token
-
-    uint32_t hin = key + kHashTok;            // key + j * C_TOK at j = 1
-    for (uint32_t j = 2; j <= n; ++j) {
-        hin += kHashTok;
-        const uint32_t h = mix32(hin);
-        const uint32_t xS = baseS + __umulhi(h, mulS);                  // T + jitter in [-J, J]
-        const uint32_t xD = baseD + __umulhi(h, mulD);
-        if (m) {                                                         // migrated stream, tokens after m
-            if (j == m + 1) {
-                const uint32_t e_m = sX.e;
-                stall = step(sX, M, tau_eff);
-                slot_lag = (int32_t)M - (int32_t)e_m - tau;
-            } else {
-                const uint32_t xT = cand == 1 ? xD : xS;
-                count_tbt(sX, step(sX, xT, tau_eff), tau_fast, win2, lo2, W2, err);
-                slot_lag += (int32_t)xT - tau;
-            }
-            if (cc.pacing && slot_lag > 0) ++delayed;
-        }
-        count_tbt(sS, step(sS, xS, tau_eff), tau_fast, win0, lo0, W0, err);
-        count_tbt(sD, step(sD, xD, tau_eff), tau_fast, win1, lo1, W1, err);
-        if (cand && !m) {
-            gC += cand == 1 ? xS : xD;
-            if (j >= B && j + 1 <= n) {
-                if (j > B) {                                             // advance the lagged copy to token j-B+1
-                    h_lag += kHashTok;
-                    const uint32_t hl = mix32(h_lag);
-                    const uint32_t xl = cand == 1 ? baseS + __umulhi(hl, mulS) : baseD + __umulhi(hl, mulD);
-                    const int32_t t = (int32_t)xl - (int32_t)e_lag;
-                    const int32_t tbt = max(t, (int32_t)tau_eff);
-                    e_lag = (uint32_t)(tbt - t);
-                    g_lag += xl;
-                }
-                if (g_lag + e_lag > gC) {                                // d_{j-B+1} > g_j
-                    m = j;
-                    M = handoff_latency(m);
-                    sX = cand == 1 ? sS : sD;
-                    const uint16_t* wc = cand == 1 ? win0 : win1;
-                    const int Wc = cand == 1 ? W0 : W1, shift = (cand == 1 ? lo0 : lo1) - lo2;
-                    for (int i = 0; i < Wc; ++i) if (wc[i]) win2[i + shift] = wc[i];
-                }
-            }
-        }
-    }
-    const int kt0 = cc.ktau[g][0], kt1 = cc.ktau[g][1], kt2 = cc.ktau[g][2];
-    if (kt0 >= 0) win0[kt0] += (uint16_t)sS.ntau;
-    if (kt1 >= 0) win1[kt1] += (uint16_t)sD.ntau;
-    if (kt2 >= 0 && m) win2[kt2] += (uint16_t)sX.ntau;
-    rec.sum[0][k] = sS.sum; rec.max[0][k] = sS.mx;
-    rec.sum[1][k] = sD.sum; rec.max[1][k] = sD.mx;
-    rec.sum[2][k] = m ? sX.sum : 0u; rec.max[2][k] = m ? sX.mx : 0u;
-    rec.stall[k] = stall;
-    rec.m[k] = (uint16_t)m; rec.delayed[k] = (uint16_t)delayed;
 }
 
 // ------------------------------------------------------------------------------------------------------
@@ -284,7 +161,7 @@ k_pairs(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __res
             // ---- reductions
             if (live) {
                 atomicAdd(&h_ttft[pi * kHStride + bin_of_ticks(ttft)], 1u);
-                const uint16_t* wp = rec.win[c] + (size_t)k * W[c];
+                const uint32_t* wp = rec.win[c] + (size_t)k * W[c];
                 for (int kk = 0; kk < W[c]; ++kk) {
                     if (kk == kt[c]) continue;
                     const uint32_t v = wp[kk];
@@ -357,13 +234,6 @@ cudaError_t launch_prep(const PolicyConst* pol, uint32_t P, int G, const GroupCo
                         cudaStream_t st) {
     const uint32_t total = P * (uint32_t)G;
     k_prep<<<(total + 127) / 128, 128, 0, st>>>(pol, P, G, gc, cum_mass, cnt, sorted, grp_off, prep);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_timeline(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const int32_t* knots,
-                            uint64_t seed, TimelineRec rec, int32_t* err, cudaStream_t st) {
-    if (tr.n == 0) return cudaSuccess;
-    k_timeline_seq<<<(tr.n + 127) / 128, 128, 0, st>>>(tr, gc, cc, knots, seed_key(seed), rec, err);
     return cudaGetLastError();
 }
 

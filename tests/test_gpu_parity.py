@@ -65,6 +65,25 @@ def test_generation_slower_than_consumption():
     full_parity(w, pols, tag="slow-gen")
 
 
+def test_buffer_search_paths():
+    # the hand-off search under clamping (generation sometimes slower than consumption), for shallow
+    # buffers, buffers deeper than a warp's delivery-time history, and buffers that never fill
+    srv, dev = [synth.server(tbt_s=0.050, jitter=0.3)], [synth.device(900.0, 22.0, jitter=0.3)]
+    for dear in (False, True):
+        if dear:
+            dev = [synth.device(900.0, 22.0, jitter=0.3, c_prefill=5e-3, c_decode=5e-3)]
+        rng = np.random.default_rng(77 + dear)
+        n = 500
+        tr = constructed(rng.integers(1, 600, size=n), rng.integers(1, 1500, size=n),
+                         rng.uniform(0.01, 1.5, size=n), servers=srv, devices=dev)
+        w = synth.Workload(name="search", seed=11, materialise=True, policies=[], **tr)
+        pols = [synth.policy(1.0, r_c=rc, t_m_s=tm, flags=MIG | PACE | md)
+                for md in (S_MODE, D_MODE) for rc, tm in ((18.0, 0.3), (18.0, 15.0), (21.0, 14.0), (25.0, 2.0),
+                                                          (16.0, 40.0), (30.0, 0.05))]
+        gs, _ = full_parity(w, pols, tag=f"search dear={dear}")
+        assert any(s.n_migrations for s in gs)
+
+
 def test_edge_cases():
     # single-token outputs, longest outputs, extreme prompts, ties at S = Td, one request
     tr = constructed([1, 4096, 45, 45, 45, 7, 4096], [1, 8192, 2, 1, 8192, 3, 1],
