@@ -1,4 +1,4 @@
-// Decode play-out (Sec. 4.3): one warp per request, every token of every stream.
+// Decode play-out (Sec. 4.3): warps play requests cooperatively, every token of every stream.
 //
 // A stream's delivery times follow d_1 = 0, d_j = max(g_j, d_{j-1} + tau) over generation times
 // g_j = g_{j-1} + x_j, x_j = T + jitter(hash(seed, request, j)).  With e_j = d_j - g_j (how far delivery lags
@@ -8,8 +8,14 @@
 // lanes' maps are combined by a shuffle scan, and each lane replays its tokens from its true state.  When
 // no c_j of a round is negative nothing clamps: every TBT equals tau and the round reduces to one sum.
 //
-// Streams per request: S (server decodes all), D (device decodes all) share the hash draws and run
-// together; X (the dearer winner hands off after token m) runs as a second pass once m is known.
+// Streams per request: S (server decodes all) and D (device decodes all) share the hash draws and run
+// together.  X (the dearer winner, the "candidate", hands off after token m) consists of the candidate's
+// tokens up to m, one token that waits for the hand-off latency, and the other endpoint's tokens after
+// it; while nothing clamps it follows from the two streams' prefix sums, otherwise it is played out in a
+// second pass.
+//
+// A warp takes 32 consecutive requests at a time: their inputs are loaded and their results stored one
+// request per lane, so the per-request memory traffic is coalesced and paid once per 32 requests.
 #include <climits>
 
 #include "disco_internal.cuh"
@@ -20,7 +26,7 @@ namespace {
 
 constexpr int kR = 8;                    // tokens per lane and round
 constexpr int kRing = 512;               // delivery times kept per warp for the buffer test
-constexpr int kWarps = 8;                // warps (requests) per block
+constexpr int kWarps = 8;                // warps per block
 constexpr uint32_t FULL = 0xFFFFFFFFu;
 constexpr uint32_t kNone = 0xFFFFFFFFu;
 
@@ -40,9 +46,27 @@ struct Round {                           // what a lane knows about the current 
     int32_t* err;
 };
 
+struct GroupClass {                      // constants of the request's group under the current class
+    uint32_t mulS, mulD;
+    int32_t cS_base, cD_base;            // tau_eff - (T - J): c = base - ((h * (2J+1)) >> 32)
+    int32_t kappa, c0;
+    int cand;                            // 0 none, 1 the server stream may hand off, 2 the device stream
+    int lo0, lo1, lo2, kt0, kt1, kt2;
+    const int32_t* K;
+};
+
 __device__ __forceinline__ void count_slow(uint32_t tbt, uint32_t* win, int lo, int W, int32_t* err) {
     const int b = bin_of_ticks(tbt) - lo;
     if (b >= 0 && b < W) atomicAdd(&win[b], 1u); else atomicExch(&err[2], 1);
+}
+
+__device__ __forceinline__ int32_t warp_inclusive_sum(int32_t v, int lane) {
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const int32_t p = __shfl_up_sync(FULL, v, off);
+        if (lane >= off) v += p;
+    }
+    return v;
 }
 
 // State (e, S) in front of each lane's first token: exclusive shuffle scan of the lanes' maps.
@@ -65,8 +89,8 @@ __device__ __forceinline__ void lane_state(const WS& st, const int32_t (&c)[kR],
 }
 
 // Sequential search of the hand-off index by one lane, for buffers deeper than the warp's history ring.
-__device__ uint32_t find_handoff_sequential(uint32_t key, int32_t c_base, uint32_t mul, int32_t tau, uint32_t B,
-                                            uint32_t n) {
+__device__ __noinline__ uint32_t find_handoff_sequential(uint32_t key, int32_t c_base, uint32_t mul, int32_t tau,
+                                                         uint32_t B, uint32_t n) {
     int32_t e = 0, e_lag = 0, S = 0, S_lag = 0;
     uint32_t h = key + kHashTok, h_lag = key + kHashTok;
     for (uint32_t j = 2; j + 1 <= n; ++j) {
@@ -85,38 +109,33 @@ __device__ uint32_t find_handoff_sequential(uint32_t key, int32_t c_base, uint32
     return 0;
 }
 
-// One round of streams S or D.  `search`: this is the candidate stream and the hand-off index is still
-// unknown; then m_out receives it when the buffer first holds B tokens (d_{j-B+1} > g_j) in this round.
-__device__ __forceinline__ void play_round(WS& st, uint32_t& mxl, uint32_t& ntl, const int32_t (&c)[kR],
-                                           const Round& rd, uint32_t* win, int lo, int W, bool search, uint32_t B,
-                                           int32_t thr, uint32_t& clean_until, uint32_t* ring, uint32_t& m_out) {
-    int32_t s = 0, mn = 0;
-#pragma unroll
-    for (int t = 0; t < kR; ++t)
-        if (t < rd.cper) { s += c[t]; mn = min(mn, c[t]); }
-    const bool fast = rd.pacing && __all_sync(FULL, mn >= 0) && !(search && !st.clean);
-    if (fast) {                                         // no clamp: every TBT of the round equals tau
+// One round of stream S or D.  s = the lane's sum of c, nonneg = no c of the round is negative.
+// `search`: this is the candidate stream and the hand-off index is still unknown; then m_out receives it
+// when the buffer first holds B tokens (d_{j-B+1} > g_j) in this round, and, if the stream never clamped
+// before, em_out its delivery lag e_m.
+__device__ __forceinline__ void play_round(WS& st, uint32_t& mxl, uint32_t& ntl, const int32_t (&c)[kR], int32_t s,
+                                           bool nonneg, const Round& rd, uint32_t* win, int lo, int W, bool search,
+                                           uint32_t B, int32_t thr, uint32_t& clean_until, uint32_t* ring,
+                                           uint32_t& m_out, int32_t& em_out) {
+    if (rd.pacing && nonneg && !(search && !st.clean)) {   // no clamp: every TBT of the round equals tau
         const int32_t tot = __reduce_add_sync(FULL, s);
         if (search) {
             // clean stream: d_q = (q-1) tau, so d_{j-B+1} > g_j  <=>  S_j > (B-1) tau, and S is non-decreasing
             if (st.S + tot > thr) {
-                int32_t si = s;
-#pragma unroll
-                for (int off = 1; off < 32; off <<= 1) {
-                    const int32_t sp = __shfl_up_sync(FULL, si, off);
-                    if (rd.lane >= off) si += sp;
-                }
-                int32_t run = st.S + si - s;
+                int32_t run = st.S + warp_inclusive_sum(s, rd.lane) - s, run_first = 0;
                 uint32_t first = kNone;
 #pragma unroll
                 for (int t = 0; t < kR; ++t)
                     if (t < rd.cnt) {
                         run += c[t];
                         const uint32_t j = rd.j0 + t;
-                        if (first == kNone && run > thr && j + 1 <= rd.n) first = j;
+                        if (first == kNone && run > thr && j + 1 <= rd.n) { first = j; run_first = run; }
                     }
                 const uint32_t found = __reduce_min_sync(FULL, first);
-                if (found != kNone) m_out = found;
+                if (found != kNone) {
+                    m_out = found;
+                    em_out = __shfl_sync(FULL, run_first, __ffs(__ballot_sync(FULL, first == found)) - 1);
+                }
             }
             clean_until = rd.last_j;
         }
@@ -164,207 +183,296 @@ __device__ __forceinline__ void play_round(WS& st, uint32_t& mxl, uint32_t& ntl,
     st.clean = false;
 }
 
-__global__ void __launch_bounds__(kWarps * 32)
-k_playout(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __restrict__ ccp,
-          const int32_t* __restrict__ knots, uint32_t k0, TimelineRec rec, int32_t* err) {
-    __shared__ uint32_t ring_s[kWarps][kRing];
-    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
-    const uint32_t k = blockIdx.x * kWarps + wib;
-    if (k >= tr.n) return;
-    uint32_t* ring = ring_s[wib];
-    int g = 0;
-    while (g + 1 < tr.n_groups && k >= tr.grp_off[g + 1]) ++g;
-    const GroupConst gc = gcs[g];
-    const ClassConst& cc = *ccp;
-    const uint32_t n = tr.nout[k], l = tr.l[k];
-    const uint32_t nI = n - 1;                                        // inter-token intervals, tokens 2..n
-    const uint32_t key = mix32(k0 + tr.orig[k] * kHashReq);
-    const int32_t tau_eff = cc.tau_eff, tau = cc.tau;
-    const bool pacing = cc.pacing != 0;
-    const int W0 = cc.W[0], W1 = cc.W[1], W2 = cc.W[2];
-    const int lo0 = cc.lo[g][0], lo1 = cc.lo[g][1], lo2 = cc.lo[g][2];
-    uint32_t* win0 = rec.win[0] + (size_t)k * W0;
-    uint32_t* win1 = rec.win[1] + (size_t)k * W1;
-    uint32_t* win2 = rec.win[2] + (size_t)k * W2;
-    for (int i = lane; i < W0; i += 32) win0[i] = 0;
-    for (int i = lane; i < W1; i += 32) win1[i] = 0;
-    for (int i = lane; i < W2; i += 32) win2[i] = 0;
-    __syncwarp();
+struct XResult { uint32_t sum, mx, stall, delayed, nt; };
 
-    const uint32_t mulS = 2u * (uint32_t)gc.J_srv + 1u, mulD = 2u * (uint32_t)gc.J_dev + 1u;
-    const int32_t cS_base = tau_eff - (gc.T_srv - gc.J_srv), cD_base = tau_eff - (gc.T_dev - gc.J_dev);
-    const int cand = (cc.mig_any && n >= 2) ? gc.candidate : 0;      // 1: server stream may hand off, 2: device stream
-    const uint32_t B = (uint32_t)cc.B;
-    const long long thr64 = (long long)(B ? B - 1 : 0) * tau;
-    const int32_t thr = thr64 > INT_MAX ? INT_MAX : (int32_t)thr64;
+__device__ __forceinline__ uint32_t handoff_latency(const GroupClass& G, uint32_t key, uint32_t l, uint32_t m) {
+    if (G.cand == 1) return (uint32_t)G.kappa * (l + m) + (uint32_t)G.c0;   // device re-prefills prompt + m tokens
+    const uint32_t u = mix32(key);                                          // a server TTFT drawn from F by its knots
+    const uint32_t kk = u >> 24, fr = (u >> 8) & 0xFFFFu;
+    return (uint32_t)(G.K[kk] + (int32_t)(((int64_t)(G.K[kk + 1] - G.K[kk]) * (int64_t)fr) >> 16));
+}
 
-    Round rd;
-    rd.lane = lane; rd.n = n; rd.tau_eff = tau_eff; rd.pacing = pacing; rd.err = err;
-    rd.cper = (int)min((uint32_t)kR, (nI + 31u) / 32u);
+// Stream X played out token by token: the candidate's tokens up to m, the hand-off latency, then the target.
+__device__ __noinline__ void play_x(const GroupClass& G, Round rd, uint32_t key, uint32_t nI, uint32_t m, uint32_t M,
+                                    uint32_t* win2, int W2, XResult* out) {
+    const int32_t tau_eff = rd.tau_eff;
+    const bool pacing = rd.pacing;
     const uint32_t span = 32u * (uint32_t)rd.cper;
-
-    WS sS = {0, 0, 0, true}, sD = {0, 0, 0, true};
-    uint32_t mxS = 0, ntS = 0, mxD = 0, ntD = 0;
-    uint32_t m = (cand && B == 0) ? 1u : 0u;                           // nothing to fill: hand off after token 1
-    uint32_t clean_until = 1;
-
+    const int32_t cM = tau_eff - (int32_t)M;
+    const uint32_t mulC = G.cand == 1 ? G.mulS : G.mulD, mulT = G.cand == 1 ? G.mulD : G.mulS;
+    const int32_t cC_base = G.cand == 1 ? G.cS_base : G.cD_base, cT_base = G.cand == 1 ? G.cD_base : G.cS_base;
+    WS sX = {0, 0, 0, true};
+    uint32_t mxX = 0, ntX = 0, dl = 0, stall = 0;
+    int32_t D0 = 0;                                                // e_m - S_m: slot lag of token j is -(D0 + S_j)
+    bool D0_known = false;
     for (uint32_t base = 0; base < nI; base += span) {
-        const uint32_t idx0 = base + (uint32_t)lane * rd.cper;
+        const uint32_t idx0 = base + (uint32_t)rd.lane * rd.cper;
         rd.cnt = idx0 >= nI ? 0 : (int)min((uint32_t)rd.cper, nI - idx0);
         rd.j0 = idx0 + 2;
         rd.round_valid = min(span, nI - base);
         rd.last_j = base + rd.round_valid + 1;
-        int32_t cs[kR], cd[kR];
+        int32_t cx[kR];
         uint32_t hin = key + rd.j0 * kHashTok;
+        int32_t s = 0, neg = 0;
 #pragma unroll
         for (int t = 0; t < kR; ++t) {
-            cs[t] = 0; cd[t] = 0;
+            cx[t] = 0;
             if (t < rd.cper) {
                 const uint32_t h = mix32(hin);
                 hin += kHashTok;
                 if (t < rd.cnt) {
-                    cs[t] = cS_base - (int32_t)__umulhi(h, mulS);     // tau - (T + jitter), jitter in [-J, J]
-                    cd[t] = cD_base - (int32_t)__umulhi(h, mulD);
+                    const uint32_t j = rd.j0 + t;
+                    const bool src = j <= m;
+                    const int32_t v = (src ? cC_base : cT_base) - (int32_t)__umulhi(h, src ? mulC : mulT);
+                    cx[t] = j == m + 1 ? cM : v;
                 }
+                s += cx[t]; neg |= cx[t];
             }
         }
-        bool searchS = cand == 1 && m == 0, searchD = cand == 2 && m == 0;
-        // buffers deeper than the ring: once the candidate stream clamps, one lane searches sequentially
-        if ((searchS || searchD) && B > kRing / 2) {
-            const int32_t(&cc_)[kR] = searchS ? cs : cd;
-            int32_t mn = 0;
+        const bool special = base + 2 <= m + 1 && rd.last_j >= m;        // round holds token m or m+1
+        const bool late = pacing && D0_known && D0 + sX.S < 0;           // tokens may still miss their slots
+        const bool nonneg = !__any_sync(FULL, neg < 0);
+        if (pacing && !special && !late && nonneg) {
+            const int32_t tot = __reduce_add_sync(FULL, s);
+            sX.e += tot; sX.S += tot; sX.nt += rd.round_valid;
+            continue;
+        }
+        int32_t e, S_in, tot;
+        lane_state(sX, cx, rd, e, S_in, tot);
+        int32_t run = S_in, em_minus_Sm = 0;
 #pragma unroll
-            for (int t = 0; t < kR; ++t) mn = min(mn, cc_[t]);
-            if (!__all_sync(FULL, mn >= 0)) {
-                uint32_t mm = 0;
-                if (lane == 0)
-                    mm = find_handoff_sequential(key, searchS ? cS_base : cD_base, searchS ? mulS : mulD, tau, B, n);
-                mm = __shfl_sync(FULL, mm, 0);
-                m = mm ? mm : kNone;                                   // kNone: searched, never fills
-                searchS = searchD = false;
+        for (int t = 0; t < kR; ++t)
+            if (t < rd.cnt) {
+                const uint32_t j = rd.j0 + t;
+                const int32_t v = e + cx[t];
+                e = max(v, 0);
+                const uint32_t ex = (uint32_t)(e - v);
+                mxX = max(mxX, ex);
+                run += cx[t];
+                if (j == m + 1) stall = (uint32_t)tau_eff + ex;          // kept apart from the regular TBTs
+                else if (pacing && ex == 0) ++ntX;
+                else count_slow((uint32_t)tau_eff + ex, win2, G.lo2, W2, rd.err);
+                if (j == m) em_minus_Sm = e - run;
+            }
+        sX.e = __shfl_sync(FULL, e, 31);
+        if (m >= base + 2 && m <= rd.last_j) {                           // token m is in this round (m >= 2)
+            D0 = __shfl_sync(FULL, em_minus_Sm, (int)((m - 2 - base) / rd.cper));
+            D0_known = true;
+        } else if (m == 1 && base == 0) {
+            D0 = 0; D0_known = true;                                     // e_1 = S_1 = 0
+        }
+        if (pacing && D0_known) {                                        // generated after d_m + (j-m) tau ?
+            run = S_in;
+#pragma unroll
+            for (int t = 0; t < kR; ++t)
+                if (t < rd.cnt) {
+                    run += cx[t];
+                    if (rd.j0 + t > m && D0 + run < 0) ++dl;
+                }
+        }
+        sX.S += tot;
+    }
+    out->nt = sX.nt + __reduce_add_sync(FULL, ntX);
+    out->mx = (uint32_t)tau_eff + __reduce_max_sync(FULL, mxX);
+    out->stall = __reduce_max_sync(FULL, stall);
+    out->delayed = __reduce_add_sync(FULL, dl);
+    out->sum = (uint32_t)((int32_t)nI * tau_eff - sX.S + sX.e);
+}
+
+// Tokens after the hand-off that are generated later than their delivery slots, when the target stream
+// never clamps: token m+1 misses its slot by `need` ticks and each later token gains c on the pace.
+__device__ __forceinline__ uint32_t count_delayed_clean(const GroupClass& G, Round rd, uint32_t key, uint32_t nI,
+                                                        uint32_t m, int32_t need) {
+    const uint32_t span = 32u * (uint32_t)rd.cper;
+    const uint32_t mulT = G.cand == 1 ? G.mulD : G.mulS;
+    const int32_t cT_base = G.cand == 1 ? G.cD_base : G.cS_base;
+    uint32_t dl = 1;                                                   // token m+1 itself
+    int32_t carry = 0;                                                 // sum of c over tokens m+2 .. before this round
+    for (uint32_t base = (m / span) * span; base < nI && carry < need; base += span) {   // round of token m+2
+        const uint32_t idx0 = base + (uint32_t)rd.lane * rd.cper;
+        const int cnt = idx0 >= nI ? 0 : (int)min((uint32_t)rd.cper, nI - idx0);
+        const uint32_t j0 = idx0 + 2;
+        int32_t c[kR], s = 0;
+        uint32_t hin = key + j0 * kHashTok;
+#pragma unroll
+        for (int t = 0; t < kR; ++t) {
+            c[t] = 0;
+            if (t < rd.cper) {
+                const uint32_t h = mix32(hin);
+                hin += kHashTok;
+                if (t < cnt && j0 + t >= m + 2) c[t] = cT_base - (int32_t)__umulhi(h, mulT);
+                s += c[t];
             }
         }
-        uint32_t m_new = 0;
-        play_round(sS, mxS, ntS, cs, rd, win0, lo0, W0, searchS, B, thr, clean_until, ring, m_new);
-        play_round(sD, mxD, ntD, cd, rd, win1, lo1, W1, searchD, B, thr, clean_until, ring, m_new);
-        if (m_new) m = m_new;
+        const int32_t incl = warp_inclusive_sum(s, rd.lane);
+        int32_t run = carry + incl - s;
+        uint32_t here = 0;
+#pragma unroll
+        for (int t = 0; t < kR; ++t)
+            if (t < cnt && j0 + t >= m + 2) { run += c[t]; here += run < need; }
+        dl += __reduce_add_sync(FULL, here);
+        carry += __shfl_sync(FULL, incl, 31);
     }
-    if (m == kNone) m = 0;
+    return dl;
+}
 
-    // ---- summaries of S and D
-    {
-        const uint32_t tS = sS.nt + __reduce_add_sync(FULL, ntS), tD = sD.nt + __reduce_add_sync(FULL, ntD);
-        const uint32_t xS = __reduce_max_sync(FULL, mxS), xD = __reduce_max_sync(FULL, mxD);
-        __syncwarp();
-        if (lane == 0) {
-            const int ktS = cc.ktau[g][0], ktD = cc.ktau[g][1];
-            if (ktS >= 0 && tS) atomicAdd(&win0[ktS], tS);
-            if (ktD >= 0 && tD) atomicAdd(&win1[ktD], tD);
-            rec.sum[0][k] = (uint32_t)((int32_t)nI * tau_eff - sS.S + sS.e);       // d_n - d_1 = g_n + e_n
-            rec.sum[1][k] = (uint32_t)((int32_t)nI * tau_eff - sD.S + sD.e);
-            rec.max[0][k] = nI ? (uint32_t)tau_eff + xS : 0u;
-            rec.max[1][k] = nI ? (uint32_t)tau_eff + xD : 0u;
-        }
+__global__ void __launch_bounds__(kWarps * 32)
+k_playout(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __restrict__ ccp,
+          const int32_t* __restrict__ knots, uint32_t k0, TimelineRec rec, int32_t* err) {
+    __shared__ uint32_t ring_s[kWarps][kRing];
+    __shared__ XResult xres_s[kWarps];
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    const uint32_t batch0 = (blockIdx.x * kWarps + wib) * 32u;
+    if (batch0 >= tr.n) return;
+    uint32_t* ring = ring_s[wib];
+    const ClassConst& cc = *ccp;
+    const int32_t tau_eff = cc.tau_eff, tau = cc.tau;
+    const bool pacing = cc.pacing != 0;
+    const int W0 = cc.W[0], W1 = cc.W[1], W2 = cc.W[2];
+    const uint32_t B = (uint32_t)cc.B;
+    const long long thr64 = (long long)(B ? B - 1 : 0) * tau;
+    const int32_t thr = thr64 > INT_MAX ? INT_MAX : (int32_t)thr64;
+
+    // ---- one request per lane: inputs
+    const uint32_t kk = batch0 + lane;
+    const bool live = kk < tr.n;
+    uint32_t n_l = 1, l_l = 1, key_l = 0;
+    int g_l = 0;
+    if (live) {
+        n_l = tr.nout[kk]; l_l = tr.l[kk];
+        key_l = mix32(k0 + tr.orig[kk] * kHashReq);
+        while (g_l + 1 < tr.n_groups && kk >= tr.grp_off[g_l + 1]) ++g_l;
+        for (int i = 0; i < W0; ++i) rec.win[0][(size_t)kk * W0 + i] = 0;
+        for (int i = 0; i < W1; ++i) rec.win[1][(size_t)kk * W1 + i] = 0;
+        for (int i = 0; i < W2; ++i) rec.win[2][(size_t)kk * W2 + i] = 0;
     }
+    __syncwarp();
+    // ---- one request per lane: results
+    uint32_t o_sumS = 0, o_maxS = 0, o_sumD = 0, o_maxD = 0, o_sumX = 0, o_maxX = 0, o_stall = 0, o_m = 0, o_dl = 0;
+    uint32_t o_ntS = 0, o_ntD = 0, o_ntX = 0;
 
-    // ---- stream X: the candidate's tokens up to m, then the target after the hand-off latency M
-    uint32_t stall = 0, delayed = 0, sumX = 0, maxX = 0;
-    if (m) {
-        uint32_t M;
-        if (cand == 1) {
-            M = (uint32_t)gc.kappa * (l + m) + (uint32_t)gc.c0;        // device re-prefills prompt + generated tokens
-        } else {
-            const uint32_t u = mix32(key);                             // a server TTFT drawn from F by its knots
-            const int32_t* K = knots + g * kNKnots;
-            const uint32_t kk = u >> 24, fr = (u >> 8) & 0xFFFFu;
-            M = (uint32_t)(K[kk] + (int32_t)(((int64_t)(K[kk + 1] - K[kk]) * (int64_t)fr) >> 16));
+    GroupClass G;
+    int cur_g = -1;
+    Round rd;
+    rd.lane = lane; rd.tau_eff = tau_eff; rd.pacing = pacing; rd.err = err;
+    const int n_here = (int)min(32u, tr.n - batch0);
+
+    for (int r = 0; r < n_here; ++r) {
+        const uint32_t n = __shfl_sync(FULL, n_l, r), l = __shfl_sync(FULL, l_l, r);
+        const uint32_t key = __shfl_sync(FULL, key_l, r);
+        const int g = __shfl_sync(FULL, g_l, r);
+        const uint32_t k = batch0 + r;
+        if (g != cur_g) {
+            cur_g = g;
+            const GroupConst& gc = gcs[g];
+            G.mulS = 2u * (uint32_t)gc.J_srv + 1u; G.mulD = 2u * (uint32_t)gc.J_dev + 1u;
+            G.cS_base = tau_eff - (gc.T_srv - gc.J_srv); G.cD_base = tau_eff - (gc.T_dev - gc.J_dev);
+            G.kappa = gc.kappa; G.c0 = gc.c0;
+            G.cand = cc.mig_any ? gc.candidate : 0;
+            G.lo0 = cc.lo[g][0]; G.lo1 = cc.lo[g][1]; G.lo2 = cc.lo[g][2];
+            G.kt0 = cc.ktau[g][0]; G.kt1 = cc.ktau[g][1]; G.kt2 = cc.ktau[g][2];
+            G.K = knots + g * kNKnots;
         }
-        const int32_t cM = tau_eff - (int32_t)M;
-        const uint32_t mulC = cand == 1 ? mulS : mulD, mulT = cand == 1 ? mulD : mulS;
-        const int32_t cC_base = cand == 1 ? cS_base : cD_base, cT_base = cand == 1 ? cD_base : cS_base;
-        WS sX = {0, 0, 0, true};
-        uint32_t mxX = 0, ntX = 0, dl = 0;
-        int32_t D0 = 0;                                                // e_m - S_m: slot lag of token j is -(D0 + S_j)
-        bool D0_known = false;
+        const uint32_t nI = n - 1;                                     // inter-token intervals, tokens 2..n
+        if (nI == 0) continue;                                         // a single token: all results stay 0
+        uint32_t* win0 = rec.win[0] + (size_t)k * W0;
+        uint32_t* win1 = rec.win[1] + (size_t)k * W1;
+        uint32_t* win2 = rec.win[2] + (size_t)k * W2;
+        const int cand = G.cand;
+        rd.n = n;
+        rd.cper = (int)min((uint32_t)kR, (nI + 31u) / 32u);
+        const uint32_t span = 32u * (uint32_t)rd.cper;
+
+        WS sS = {0, 0, 0, true}, sD = {0, 0, 0, true};
+        uint32_t mxS = 0, ntS = 0, mxD = 0, ntD = 0;
+        uint32_t m = (cand && B == 0) ? 1u : 0u;                       // nothing to fill: hand off after token 1
+        int32_t e_m = 0;                                               // candidate's delivery lag at m
+        bool m_clean = m != 0;                                         // candidate never clamped up to m
+        uint32_t clean_until = 1;
+
         for (uint32_t base = 0; base < nI; base += span) {
             const uint32_t idx0 = base + (uint32_t)lane * rd.cper;
             rd.cnt = idx0 >= nI ? 0 : (int)min((uint32_t)rd.cper, nI - idx0);
             rd.j0 = idx0 + 2;
             rd.round_valid = min(span, nI - base);
             rd.last_j = base + rd.round_valid + 1;
-            int32_t cx[kR];
+            int32_t cs[kR], cd[kR], s_S = 0, s_D = 0, negS = 0, negD = 0;
             uint32_t hin = key + rd.j0 * kHashTok;
-            int32_t s = 0, mn = 0;
 #pragma unroll
             for (int t = 0; t < kR; ++t) {
-                cx[t] = 0;
+                cs[t] = 0; cd[t] = 0;
                 if (t < rd.cper) {
                     const uint32_t h = mix32(hin);
                     hin += kHashTok;
-                    if (t < rd.cnt) {
-                        const uint32_t j = rd.j0 + t;
-                        const bool src = j <= m;
-                        const int32_t v = (src ? cC_base : cT_base) - (int32_t)__umulhi(h, src ? mulC : mulT);
-                        cx[t] = j == m + 1 ? cM : v;
-                    }
-                    s += cx[t]; mn = min(mn, cx[t]);
+                    const bool valid = t < rd.cnt;
+                    cs[t] = valid ? G.cS_base - (int32_t)__umulhi(h, G.mulS) : 0;   // tau - (T + jitter in [-J, J])
+                    cd[t] = valid ? G.cD_base - (int32_t)__umulhi(h, G.mulD) : 0;
+                    s_S += cs[t]; s_D += cd[t]; negS |= cs[t]; negD |= cd[t];
                 }
             }
-            const bool special = base + 2 <= m + 1 && rd.last_j >= m;        // round holds token m or m+1
-            const bool late = pacing && D0_known && D0 + sX.S < 0;           // tokens may still miss their slots
-            const bool fast = pacing && !special && !late && __all_sync(FULL, mn >= 0);
-            if (fast) {
-                const int32_t tot = __reduce_add_sync(FULL, s);
-                sX.e += tot; sX.S += tot; sX.nt += rd.round_valid;
-                continue;
+            const bool posS = !__any_sync(FULL, negS < 0), posD = !__any_sync(FULL, negD < 0);
+            bool searchS = cand == 1 && m == 0, searchD = cand == 2 && m == 0;
+            // buffers deeper than the ring: once the candidate stream clamps, one lane searches sequentially
+            if ((searchS || searchD) && B > kRing / 2 && !(searchS ? posS : posD)) {
+                uint32_t mm = 0;
+                if (lane == 0)
+                    mm = find_handoff_sequential(key, searchS ? G.cS_base : G.cD_base, searchS ? G.mulS : G.mulD, tau,
+                                                 B, n);
+                mm = __shfl_sync(FULL, mm, 0);
+                m = mm ? mm : kNone;                                   // kNone: searched, the buffer never fills
+                searchS = searchD = false;
             }
-            int32_t e, S_in, tot;
-            lane_state(sX, cx, rd, e, S_in, tot);
-            int32_t run = S_in, em_minus_Sm = 0;
-#pragma unroll
-            for (int t = 0; t < kR; ++t)
-                if (t < rd.cnt) {
-                    const uint32_t j = rd.j0 + t;
-                    const int32_t v = e + cx[t];
-                    e = max(v, 0);
-                    const uint32_t ex = (uint32_t)(e - v);
-                    mxX = max(mxX, ex);
-                    run += cx[t];
-                    if (j == m + 1) stall = (uint32_t)tau_eff + ex;          // kept apart from the regular TBTs
-                    else if (pacing && ex == 0) ++ntX;
-                    else count_slow((uint32_t)tau_eff + ex, win2, lo2, W2, err);
-                    if (j == m) em_minus_Sm = e - run;
-                }
-            sX.e = __shfl_sync(FULL, e, 31);
-            if (m >= base + 2 && m <= rd.last_j) {                           // token m is in this round (m >= 2)
-                D0 = __shfl_sync(FULL, em_minus_Sm, (int)((m - 2 - base) / rd.cper));
-                D0_known = true;
-            } else if (m == 1 && base == 0) {
-                D0 = 0; D0_known = true;                                     // e_1 = S_1 = 0
-            }
-            if (pacing && D0_known) {                                        // generated after d_m + (j-m) tau ?
-                run = S_in;
-#pragma unroll
-                for (int t = 0; t < kR; ++t)
-                    if (t < rd.cnt) {
-                        run += cx[t];
-                        if (rd.j0 + t > m && D0 + run < 0) ++dl;
-                    }
-            }
-            sX.S += tot;
+            uint32_t m_new = 0;
+            const bool was_clean = cand == 1 ? sS.clean : sD.clean;
+            play_round(sS, mxS, ntS, cs, s_S, posS, rd, win0, G.lo0, W0, searchS, B, thr, clean_until, ring, m_new, e_m);
+            play_round(sD, mxD, ntD, cd, s_D, posD, rd, win1, G.lo1, W1, searchD, B, thr, clean_until, ring, m_new, e_m);
+            if (m_new) { m = m_new; m_clean = was_clean && (cand == 1 ? sS.clean : sD.clean); }
         }
-        const uint32_t tX = sX.nt + __reduce_add_sync(FULL, ntX);
-        maxX = (uint32_t)tau_eff + __reduce_max_sync(FULL, mxX);
-        stall = __reduce_max_sync(FULL, stall);
-        delayed = __reduce_add_sync(FULL, dl);
-        sumX = (uint32_t)((int32_t)nI * tau_eff - sX.S + sX.e);
-        __syncwarp();
-        const int ktX = cc.ktau[g][2];
-        if (lane == 0 && ktX >= 0 && tX) atomicAdd(&win2[ktX], tX);
+        if (m == kNone) m = 0;
+
+        // ---- summaries of S and D
+        const uint32_t tS = sS.nt + __reduce_add_sync(FULL, ntS), tD = sD.nt + __reduce_add_sync(FULL, ntD);
+        const uint32_t r_sumS = (uint32_t)((int32_t)nI * tau_eff - sS.S + sS.e);       // d_n - d_1 = g_n + e_n
+        const uint32_t r_sumD = (uint32_t)((int32_t)nI * tau_eff - sD.S + sD.e);
+        const uint32_t r_maxS = (uint32_t)tau_eff + __reduce_max_sync(FULL, mxS);
+        const uint32_t r_maxD = (uint32_t)tau_eff + __reduce_max_sync(FULL, mxD);
+
+        // ---- stream X
+        XResult xr = {0, 0, 0, 0, 0};
+        if (m) {
+            const uint32_t M = handoff_latency(G, key, l, m);
+            const bool target_clean = cand == 1 ? sD.clean : sS.clean;
+            if (pacing && m_clean && target_clean) {
+                // nothing clamps but the hand-off itself: tokens up to m and after m+1 are delivered tau apart
+                const int32_t v = e_m + (tau_eff - (int32_t)M);               // lag of token m+1 behind its slot, negated
+                xr.stall = (uint32_t)tau_eff + (uint32_t)max(-v, 0);
+                xr.nt = nI - 1;
+                xr.sum = (nI - 1) * (uint32_t)tau_eff + xr.stall;
+                xr.mx = xr.stall;
+                xr.delayed = v < 0 ? count_delayed_clean(G, rd, key, nI, m, -v) : 0u;
+            } else {
+                play_x(G, rd, key, nI, m, M, win2, W2, &xres_s[wib]);
+                __syncwarp();
+                xr = xres_s[wib];
+                __syncwarp();
+            }
+        }
+        if (lane == r) {
+            o_sumS = r_sumS; o_maxS = r_maxS; o_sumD = r_sumD; o_maxD = r_maxD; o_ntS = tS; o_ntD = tD;
+            o_sumX = xr.sum; o_maxX = xr.mx; o_stall = xr.stall; o_m = m; o_dl = xr.delayed; o_ntX = xr.nt;
+        }
     }
-    if (lane == 0) {
-        rec.sum[2][k] = sumX; rec.max[2][k] = maxX; rec.stall[k] = stall;
-        rec.m[k] = (uint16_t)m; rec.delayed[k] = (uint16_t)delayed;
+    __syncwarp();
+    // ---- one request per lane: results out
+    if (live) {
+        rec.sum[0][kk] = o_sumS; rec.max[0][kk] = o_maxS;
+        rec.sum[1][kk] = o_sumD; rec.max[1][kk] = o_maxD;
+        rec.sum[2][kk] = o_sumX; rec.max[2][kk] = o_maxX;
+        rec.stall[kk] = o_stall; rec.m[kk] = (uint16_t)o_m; rec.delayed[kk] = (uint16_t)o_dl;
+        const int kt0 = cc.ktau[g_l][0], kt1 = cc.ktau[g_l][1], kt2 = cc.ktau[g_l][2];
+        if (kt0 >= 0 && o_ntS) rec.win[0][(size_t)kk * W0 + kt0] += o_ntS;
+        if (kt1 >= 0 && o_ntD) rec.win[1][(size_t)kk * W1 + kt1] += o_ntD;
+        if (kt2 >= 0 && o_ntX) rec.win[2][(size_t)kk * W2 + kt2] += o_ntX;
     }
 }
 
@@ -373,7 +481,8 @@ k_playout(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __r
 cudaError_t launch_timeline(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const int32_t* knots,
                             uint64_t seed, TimelineRec rec, int32_t* err, cudaStream_t st) {
     if (tr.n == 0) return cudaSuccess;
-    k_playout<<<(tr.n + kWarps - 1) / kWarps, kWarps * 32, 0, st>>>(tr, gc, cc, knots, seed_key(seed), rec, err);
+    const uint32_t per_block = kWarps * 32;
+    k_playout<<<(tr.n + per_block - 1) / per_block, kWarps * 32, 0, st>>>(tr, gc, cc, knots, seed_key(seed), rec, err);
     return cudaGetLastError();
 }
 
