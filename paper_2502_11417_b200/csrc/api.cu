@@ -350,11 +350,11 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
         for (uint32_t p = 0; p < P; ++p) if (pc[p].cls == (int)k) pol_list.push_back(p);
         cls_range.push_back({b, (uint32_t)pol_list.size()});
     }
-    const uint32_t tiles = (P + 15) / 16;
-    const uint32_t want_chunks = std::max<uint32_t>(1, 296 / std::min<uint32_t>(tiles, 296));
+    const uint32_t tiles = (P + 31) / 32;
+    const uint32_t want_chunks = std::max<uint32_t>(1, 592 / std::min<uint32_t>(tiles, 592));
     uint32_t CH = (uint32_t)((N1 + want_chunks - 1) / want_chunks);
     CH = (CH + 255) / 256 * 256;
-    CH = std::min<uint32_t>(std::max<uint32_t>(CH, 256), 8192);
+    CH = std::min<uint32_t>(std::max<uint32_t>(CH, 256), 65280);     // 16-bit histogram counters per block
     std::vector<Chunk> chunks;
     for (int g = 0; g < G; ++g)
         for (uint32_t s = rb.grp_off[g]; s < rb.grp_off[g + 1]; s += CH)
@@ -423,7 +423,7 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
                         c->d_chunks.as<Chunk>(), (uint32_t)chunks.size(), rec, po, c->d_acc.as<uint64_t>(),
                         c->d_hist_ttft.as<uint64_t>(), c->d_hist_tbt.as<uint64_t>(), st));
         if (timed) CU(cudaEventRecord(c->ev[2], st));
-        g_launches += (n ? 1 : 0) + ((n && !chunks.empty()) ? 1 : 0);
+        g_launches += (n ? 1 : 0) + ((n && !chunks.empty()) ? (out ? 2 : 1) : 0);
     }
     c->timing_valid = timed && n != 0;
     c->P = P; c->pol = pc;

@@ -78,7 +78,7 @@ struct TraceDev {
 struct Chunk { uint32_t start, len; int32_t g; int32_t pad; };
 
 enum AccSlot { A_SERVER_ONLY = 0, A_DEVICE_ONLY, A_RACE, A_STARTED, A_DEVICE_WON, A_MIGR, A_TOK_DEVICE,
-               A_PRE_SERVER, A_PRE_DEVICE, A_DELAYED, A_TTFT_LO, A_TTFT_HI, kNAcc };
+               A_PRE_SERVER, A_PRE_DEVICE, A_DELAYED, A_TTFT_SUM, A_TAU_CNT, kNAcc };
 
 // ---- device helpers -------------------------------------------------------------------------------------
 

@@ -1,0 +1,262 @@
+// Per-pair evaluation: dispatch decision (Algorithms 2-3, wait-then-race), TTFT, which decode stream
+// applies (migration trigger, Eq. 4), tokens per endpoint and cost (Eq. 8), for every (request, policy).
+//
+// Two kernels share the decision logic:
+//  * k_pairs_acc  -- reductions.  A lane owns a policy and walks the requests, so every per-policy sum
+//    lives in registers and needs no cross-lane traffic; the TTFT histogram and the histogram of hand-off
+//    stalls are block-private in shared memory (16-bit counters, two per word).
+//  * k_pairs_rows -- the optional per-pair arrays.  A lane owns a request and walks the policies, so each
+//    store instruction writes 32 consecutive requests of one policy row.
+#include "disco_internal.cuh"
+
+namespace disco {
+
+namespace {
+
+constexpr uint32_t FULL = 0xFFFFFFFFu;
+
+struct PairIn {                 // one request and its play-out summaries
+    uint32_t l, n, S, m;
+    float saving;               // delta_c * (n - m): Eq. 4's projected saving
+};
+
+struct PairOut {
+    bool dev_only, started, dev_wins, race, migr;
+    uint32_t ttft;
+};
+
+// Dispatch and race for one (request, policy); candidate = which winner may migrate in this group.
+__device__ __forceinline__ PairOut decide(const PairIn& q, const Prep& pr, uint32_t Td, int candidate) {
+    PairOut o;
+    o.dev_only = !pr.device_constrained && (int32_t)q.l < pr.l_th;                 // Algorithm 3
+    uint32_t w = 0;                                                                // Algorithm 2's wait map
+    if (pr.device_constrained)
+        w = (int32_t)q.l < pr.l_star ? 0u : ((int32_t)q.l == pr.l_star ? (uint32_t)pr.w_star : (uint32_t)pr.w_tail);
+    o.started = o.dev_only || q.S > w;                                             // the device starts after the wait
+    const uint32_t wTd = w + Td;
+    o.dev_wins = o.dev_only || (o.started && q.S > wTd);                           // a tie goes to the server
+    o.ttft = o.dev_only ? Td : min(q.S, wTd);
+    o.race = o.started && !o.dev_only;
+    o.migr = pr.mig_on && o.race && q.m != 0 && candidate == (o.dev_wins ? 2 : 1) && q.saving > pr.theta;
+    return o;
+}
+
+// ------------------------------------------------------------------------------------------------------
+// Reductions: lane = policy.
+// ------------------------------------------------------------------------------------------------------
+constexpr int kAccThreads = 256;
+constexpr int kAccWarps = kAccThreads / 32;
+constexpr int kHWords = 433;            // 866 sixteen-bit counters per policy row; odd word stride
+
+__device__ __forceinline__ void hist16_add(uint32_t* row, int bin) {
+    atomicAdd(&row[bin >> 1], 1u << ((bin & 1) * 16));
+}
+
+__global__ void __launch_bounds__(kAccThreads)
+k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __restrict__ ccp,
+            const Prep* __restrict__ prep, uint32_t P, const uint32_t* __restrict__ pol_list, uint32_t n_list,
+            int PL, const Chunk* __restrict__ chunks, TimelineRec rec, unsigned long long* __restrict__ acc,
+            unsigned long long* __restrict__ hist_ttft, unsigned long long* __restrict__ hist_tbt) {
+    extern __shared__ uint32_t smem[];
+    uint32_t* h_ttft = smem;                                  // [PL][kHWords]
+    uint32_t* h_stall = smem + PL * kHWords;                  // [PL][kHWords]
+    unsigned long long* s_acc = (unsigned long long*)(smem + 2 * PL * kHWords);   // [PL][kNAcc]; 866 words per policy keep it 8-byte aligned
+
+    const Chunk ch = chunks[blockIdx.x];
+    const int g = ch.g;
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    const int pol_in_tile = lane % PL, slot = lane / PL, slots = 32 / PL;
+    const uint32_t pol_idx = blockIdx.y * PL + pol_in_tile;
+    const bool act = pol_idx < n_list;
+    const uint32_t p = pol_list[act ? pol_idx : 0];
+    const Prep pr = prep[(size_t)g * P + p];
+    const GroupConst& gc = gcs[g];
+    const ClassConst& cc = *ccp;
+    const uint32_t kappa = (uint32_t)gc.kappa, c0 = (uint32_t)gc.c0;
+    const int candidate = gc.candidate;
+    const float delta_c = gc.delta_c;
+    const int W0 = cc.W[0], W1 = cc.W[1], W2 = cc.W[2];
+    const int kt0 = cc.ktau[g][0], kt1 = cc.ktau[g][1], kt2 = cc.ktau[g][2];
+    const bool wide = W0 > 1 || W1 > 1 || W2 > 1;             // some stream's regular TBTs span several bins
+    const uint32_t tau = (uint32_t)cc.tau;
+
+    for (int i = threadIdx.x; i < 2 * PL * kHWords + 2 * PL * kNAcc; i += kAccThreads) smem[i] = 0;
+    __syncthreads();
+    uint32_t* my_ttft = h_ttft + pol_in_tile * kHWords;
+    uint32_t* my_stall = h_stall + pol_in_tile * kHWords;
+
+    uint32_t c_do = 0, c_rc = 0, c_dw = 0, c_mg = 0, a_td = 0, a_ps = 0, a_pd = 0, a_dl = 0, a_tau = 0;
+    unsigned long long a_tt = 0;
+
+    for (uint32_t b0 = wib * 32u; b0 < ch.len; b0 += kAccWarps * 32u) {
+        // ---- 32 requests, one per lane
+        const uint32_t kk = ch.start + min(b0 + lane, ch.len - 1);
+        const uint32_t ln = (uint32_t)tr.l[kk] | ((uint32_t)tr.nout[kk] << 16);
+        const uint32_t S_l = (uint32_t)tr.S[kk];
+        const uint32_t md = (uint32_t)rec.m[kk] | ((uint32_t)rec.delayed[kk] << 16);
+        const uint32_t stall_l = rec.stall[kk];
+        const uint32_t nt0 = kt0 >= 0 ? rec.win[0][(size_t)kk * W0 + kt0] : 0u;
+        const uint32_t nt1 = kt1 >= 0 ? rec.win[1][(size_t)kk * W1 + kt1] : 0u;
+        const uint32_t nt2 = kt2 >= 0 ? rec.win[2][(size_t)kk * W2 + kt2] : 0u;
+        const uint32_t nt01 = nt0 | (nt1 << 16);
+        const int n_here = (int)min(32u, ch.len - b0);
+        for (int r0 = 0; r0 < n_here; r0 += slots) {
+            const int r = r0 + slot;
+            const uint32_t ln_r = __shfl_sync(FULL, ln, r), S = __shfl_sync(FULL, S_l, r);
+            const uint32_t md_r = __shfl_sync(FULL, md, r), stall = __shfl_sync(FULL, stall_l, r);
+            const uint32_t nt01_r = __shfl_sync(FULL, nt01, r), nt2_r = __shfl_sync(FULL, nt2, r);
+            if (!act || r >= n_here) continue;
+            PairIn q;
+            q.l = ln_r & 0xFFFFu; q.n = ln_r >> 16; q.S = S; q.m = md_r & 0xFFFFu;
+            q.saving = delta_c * (float)(q.n - q.m);
+            const PairOut o = decide(q, pr, kappa * q.l + c0, candidate);
+            const uint32_t lm = q.l + q.m;
+            const uint32_t tok_src = o.migr ? q.m : q.n;
+            c_do += o.dev_only; c_rc += o.race; c_dw += o.race && o.dev_wins; c_mg += o.migr;
+            a_td += o.dev_wins ? tok_src : q.n - tok_src;
+            a_ps += (o.dev_only ? 0u : q.l) + ((o.migr && o.dev_wins) ? lm : 0u);
+            a_pd += (o.started ? q.l : 0u) + ((o.migr && !o.dev_wins) ? lm : 0u);
+            a_dl += o.migr ? md_r >> 16 : 0u;
+            a_tt += o.ttft;
+            uint32_t ntau = o.migr ? nt2_r : (o.dev_wins ? nt01_r >> 16 : nt01_r & 0xFFFFu);
+            hist16_add(my_ttft, bin_of_ticks(o.ttft));
+            if (o.migr) {                                      // the token after the hand-off
+                if (stall == tau) ++ntau; else hist16_add(my_stall, bin_of_ticks(stall));
+            }
+            a_tau += ntau;
+            if (wide) {                                        // regular TBTs outside the bin of tau
+                const int c = o.migr ? 2 : (o.dev_wins ? 1 : 0);
+                const int W = c == 2 ? W2 : (c == 1 ? W1 : W0), kt = c == 2 ? kt2 : (c == 1 ? kt1 : kt0);
+                const uint32_t* wp = rec.win[c] + (size_t)(ch.start + b0 + r) * W;
+                unsigned long long* hp = hist_tbt + (size_t)p * kNBins + cc.lo[g][c];
+                for (int j = 0; j < W; ++j) {
+                    const uint32_t v = j == kt ? 0u : wp[j];
+                    if (v) atomicAdd(&hp[j], (unsigned long long)v);
+                }
+            }
+        }
+    }
+    // ---- block totals, then one flush per block
+    if (act) {
+        unsigned long long* a = s_acc + pol_in_tile * kNAcc;
+        atomicAdd(&a[A_DEVICE_ONLY], (unsigned long long)c_do); atomicAdd(&a[A_RACE], (unsigned long long)c_rc);
+        atomicAdd(&a[A_DEVICE_WON], (unsigned long long)c_dw); atomicAdd(&a[A_MIGR], (unsigned long long)c_mg);
+        atomicAdd(&a[A_TOK_DEVICE], (unsigned long long)a_td); atomicAdd(&a[A_PRE_SERVER], (unsigned long long)a_ps);
+        atomicAdd(&a[A_PRE_DEVICE], (unsigned long long)a_pd); atomicAdd(&a[A_DELAYED], (unsigned long long)a_dl);
+        atomicAdd(&a[A_TTFT_SUM], a_tt); atomicAdd(&a[A_TAU_CNT], (unsigned long long)a_tau);
+    }
+    __syncthreads();
+    const int pols_here = (int)min((uint32_t)PL, n_list - blockIdx.y * PL);
+    const int bin_tau = bin_of_ticks(tau);
+    for (int i = threadIdx.x; i < pols_here * kHWords; i += kAccThreads) {
+        const int pi = i / kHWords, wd = i - pi * kHWords;
+        const size_t o = (size_t)pol_list[blockIdx.y * PL + pi] * kNBins + 2 * wd;
+        const uint32_t a = h_ttft[pi * kHWords + wd], b = h_stall[pi * kHWords + wd];
+        if (a & 0xFFFFu) atomicAdd(&hist_ttft[o], (unsigned long long)(a & 0xFFFFu));
+        if (a >> 16) atomicAdd(&hist_ttft[o + 1], (unsigned long long)(a >> 16));
+        if (b & 0xFFFFu) atomicAdd(&hist_tbt[o], (unsigned long long)(b & 0xFFFFu));
+        if (b >> 16) atomicAdd(&hist_tbt[o + 1], (unsigned long long)(b >> 16));
+    }
+    for (int i = threadIdx.x; i < pols_here * kNAcc; i += kAccThreads) {
+        const int pi = i / kNAcc, s = i - pi * kNAcc;
+        const unsigned long long v = s_acc[pi * kNAcc + s];
+        if (!v) continue;
+        const uint32_t pp = pol_list[blockIdx.y * PL + pi];
+        if (s == A_TAU_CNT) atomicAdd(&hist_tbt[(size_t)pp * kNBins + bin_tau], v);   // TBTs equal to tau
+        else atomicAdd(&acc[((size_t)pp * tr.n_groups + g) * kNAcc + s], v);
+    }
+}
+
+size_t acc_smem_bytes(int PL) { return sizeof(uint32_t) * (2 * PL * kHWords + 2 * PL * kNAcc); }
+
+// ------------------------------------------------------------------------------------------------------
+// Per-pair arrays: lane = request, eight policies per block column.
+// ------------------------------------------------------------------------------------------------------
+constexpr int kRowThreads = 256;
+constexpr int kRowPols = 8;
+
+__global__ void __launch_bounds__(kRowThreads)
+k_pairs_rows(TraceDev tr, const GroupConst* __restrict__ gcs, const Prep* __restrict__ prep, uint32_t P,
+             const uint32_t* __restrict__ pol_list, uint32_t n_list, const Chunk* __restrict__ chunks,
+             TimelineRec rec, disco_pair_out_t out) {
+    __shared__ Prep s_prep[kRowPols];
+    __shared__ uint32_t s_pol[kRowPols];
+    const Chunk ch = chunks[blockIdx.x];
+    const int g = ch.g;
+    const uint32_t first = blockIdx.y * kRowPols;
+    const int npol = (int)min((uint32_t)kRowPols, n_list - first);
+    if ((int)threadIdx.x < npol) {
+        const uint32_t p = pol_list[first + threadIdx.x];
+        s_pol[threadIdx.x] = p;
+        s_prep[threadIdx.x] = prep[(size_t)g * P + p];
+    }
+    __syncthreads();
+    const GroupConst& gc = gcs[g];
+    const uint32_t kappa = (uint32_t)gc.kappa, c0 = (uint32_t)gc.c0;
+    const int candidate = gc.candidate;
+    const float delta_c = gc.delta_c, cps = gc.cps, cds = gc.cds, lcpd = gc.lcpd, lcdd = gc.lcdd;
+    const size_t N = tr.n;
+
+    for (uint32_t r = threadIdx.x; r < ch.len; r += kRowThreads) {
+        const uint32_t k = ch.start + r;
+        PairIn q;
+        q.l = tr.l[k]; q.n = tr.nout[k]; q.S = (uint32_t)tr.S[k]; q.m = rec.m[k];
+        q.saving = delta_c * (float)(q.n - q.m);
+        const uint32_t orig = tr.orig[k], Td = kappa * q.l + c0, dly = rec.delayed[k];
+        const uint32_t sum0 = rec.sum[0][k], sum1 = rec.sum[1][k], sum2 = rec.sum[2][k];
+        const uint32_t max0 = rec.max[0][k], max1 = rec.max[1][k], max2 = rec.max[2][k];
+        const float inv_cnt = q.n > 1 ? 1e-6f / (float)(q.n - 1) : 0.0f;
+        for (int pi = 0; pi < npol; ++pi) {
+            const PairOut o = decide(q, s_prep[pi], Td, candidate);
+            const uint32_t sum = o.migr ? sum2 : (o.dev_wins ? sum1 : sum0);
+            const uint32_t mx = o.migr ? max2 : (o.dev_wins ? max1 : max0);
+            const uint32_t lm = q.l + q.m;
+            const uint32_t tok_src = o.migr ? q.m : q.n;
+            const uint32_t tok_dev = o.dev_wins ? tok_src : q.n - tok_src, tok_srv = q.n - tok_dev;
+            const uint32_t pre_srv = (o.dev_only ? 0u : q.l) + ((o.migr && o.dev_wins) ? lm : 0u);
+            const uint32_t pre_dev = (o.started ? q.l : 0u) + ((o.migr && !o.dev_wins) ? lm : 0u);
+            const size_t at = (size_t)s_pol[pi] * N + orig;
+            if (out.ttft_s) out.ttft_s[at] = (float)o.ttft * 1e-6f;
+            if (out.tbt_mean_s) out.tbt_mean_s[at] = (float)sum * inv_cnt;
+            if (out.tbt_max_s) out.tbt_max_s[at] = (float)mx * 1e-6f;
+            if (out.cost) out.cost[at] = cps * (float)pre_srv + cds * (float)tok_srv + lcpd * (float)pre_dev +
+                                         lcdd * (float)tok_dev;                        // Eq. 8
+            if (out.tok_server) out.tok_server[at] = tok_srv;
+            if (out.tok_device) out.tok_device[at] = tok_dev;
+            if (out.mig_at) out.mig_at[at] = o.migr ? q.m : 0u;
+            if (out.delayed) out.delayed[at] = (uint16_t)(o.migr ? dly : 0u);
+            if (out.decision) out.decision[at] = (uint8_t)(o.dev_only ? DISCO_DEVICE_ONLY
+                                                                     : (o.started ? DISCO_RACE : DISCO_SERVER_ONLY));
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const Prep* prep, uint32_t P,
+                         const uint32_t* pol_list, uint32_t n_list, const Chunk* chunks, uint32_t n_chunks,
+                         TimelineRec rec, disco_pair_out_t out, uint64_t* acc, uint64_t* hist_ttft,
+                         uint64_t* hist_tbt, cudaStream_t st) {
+    if (n_chunks == 0 || n_list == 0) return cudaSuccess;
+    int PL = 1;
+    while (PL < 32 && (uint32_t)PL < n_list) PL <<= 1;
+    cudaError_t e = cudaFuncSetAttribute(k_pairs_acc, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)acc_smem_bytes(32));
+    if (e) return e;
+    dim3 grid(n_chunks, (n_list + PL - 1) / PL);
+    k_pairs_acc<<<grid, kAccThreads, acc_smem_bytes(PL), st>>>(tr, gc, cc, prep, P, pol_list, n_list, PL, chunks, rec,
+                                                               (unsigned long long*)acc,
+                                                               (unsigned long long*)hist_ttft,
+                                                               (unsigned long long*)hist_tbt);
+    if ((e = cudaGetLastError())) return e;
+    const bool rows = out.ttft_s || out.tbt_mean_s || out.tbt_max_s || out.cost || out.tok_server || out.tok_device ||
+                      out.mig_at || out.delayed || out.decision;
+    if (rows) {
+        dim3 grid_r(n_chunks, (n_list + kRowPols - 1) / kRowPols);
+        k_pairs_rows<<<grid_r, kRowThreads, 0, st>>>(tr, gc, prep, P, pol_list, n_list, chunks, rec, out);
+        e = cudaGetLastError();
+    }
+    return e;
+}
+
+}  // namespace disco

@@ -197,7 +197,6 @@ __device__ __noinline__ void play_x(const GroupClass& G, Round rd, uint32_t key,
                                     uint32_t* win2, int W2, XResult* out) {
     const int32_t tau_eff = rd.tau_eff;
     const bool pacing = rd.pacing;
-    const uint32_t span = 32u * (uint32_t)rd.cper;
     const int32_t cM = tau_eff - (int32_t)M;
     const uint32_t mulC = G.cand == 1 ? G.mulS : G.mulD, mulT = G.cand == 1 ? G.mulD : G.mulS;
     const int32_t cC_base = G.cand == 1 ? G.cS_base : G.cD_base, cT_base = G.cand == 1 ? G.cD_base : G.cS_base;
@@ -205,7 +204,10 @@ __device__ __noinline__ void play_x(const GroupClass& G, Round rd, uint32_t key,
     uint32_t mxX = 0, ntX = 0, dl = 0, stall = 0;
     int32_t D0 = 0;                                                // e_m - S_m: slot lag of token j is -(D0 + S_j)
     bool D0_known = false;
+    uint32_t span = 0;
     for (uint32_t base = 0; base < nI; base += span) {
+        rd.cper = (int)min((uint32_t)kR, (nI - base + 31u) / 32u);
+        span = 32u * (uint32_t)rd.cper;
         const uint32_t idx0 = base + (uint32_t)rd.lane * rd.cper;
         rd.cnt = idx0 >= nI ? 0 : (int)min((uint32_t)rd.cper, nI - idx0);
         rd.j0 = idx0 + 2;
@@ -279,43 +281,6 @@ __device__ __noinline__ void play_x(const GroupClass& G, Round rd, uint32_t key,
     out->sum = (uint32_t)((int32_t)nI * tau_eff - sX.S + sX.e);
 }
 
-// Tokens after the hand-off that are generated later than their delivery slots, when the target stream
-// never clamps: token m+1 misses its slot by `need` ticks and each later token gains c on the pace.
-__device__ __forceinline__ uint32_t count_delayed_clean(const GroupClass& G, Round rd, uint32_t key, uint32_t nI,
-                                                        uint32_t m, int32_t need) {
-    const uint32_t span = 32u * (uint32_t)rd.cper;
-    const uint32_t mulT = G.cand == 1 ? G.mulD : G.mulS;
-    const int32_t cT_base = G.cand == 1 ? G.cD_base : G.cS_base;
-    uint32_t dl = 1;                                                   // token m+1 itself
-    int32_t carry = 0;                                                 // sum of c over tokens m+2 .. before this round
-    for (uint32_t base = (m / span) * span; base < nI && carry < need; base += span) {   // round of token m+2
-        const uint32_t idx0 = base + (uint32_t)rd.lane * rd.cper;
-        const int cnt = idx0 >= nI ? 0 : (int)min((uint32_t)rd.cper, nI - idx0);
-        const uint32_t j0 = idx0 + 2;
-        int32_t c[kR], s = 0;
-        uint32_t hin = key + j0 * kHashTok;
-#pragma unroll
-        for (int t = 0; t < kR; ++t) {
-            c[t] = 0;
-            if (t < rd.cper) {
-                const uint32_t h = mix32(hin);
-                hin += kHashTok;
-                if (t < cnt && j0 + t >= m + 2) c[t] = cT_base - (int32_t)__umulhi(h, mulT);
-                s += c[t];
-            }
-        }
-        const int32_t incl = warp_inclusive_sum(s, rd.lane);
-        int32_t run = carry + incl - s;
-        uint32_t here = 0;
-#pragma unroll
-        for (int t = 0; t < kR; ++t)
-            if (t < cnt && j0 + t >= m + 2) { run += c[t]; here += run < need; }
-        dl += __reduce_add_sync(FULL, here);
-        carry += __shfl_sync(FULL, incl, 31);
-    }
-    return dl;
-}
-
 __global__ void __launch_bounds__(kWarps * 32)
 k_playout(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __restrict__ ccp,
           const int32_t* __restrict__ knots, uint32_t k0, TimelineRec rec, int32_t* err) {
@@ -380,37 +345,73 @@ k_playout(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __r
         uint32_t* win2 = rec.win[2] + (size_t)k * W2;
         const int cand = G.cand;
         rd.n = n;
-        rd.cper = (int)min((uint32_t)kR, (nI + 31u) / 32u);
-        const uint32_t span = 32u * (uint32_t)rd.cper;
-
         WS sS = {0, 0, 0, true}, sD = {0, 0, 0, true};
         uint32_t mxS = 0, ntS = 0, mxD = 0, ntD = 0;
         uint32_t m = (cand && B == 0) ? 1u : 0u;                       // nothing to fill: hand off after token 1
         int32_t e_m = 0;                                               // candidate's delivery lag at m
         bool m_clean = m != 0;                                         // candidate never clamped up to m
         uint32_t clean_until = 1;
+        // Hand-off stream while nothing clamps: token m+1 is generated `need` ticks after its slot and every
+        // later token of the target gains its c on the pace; dl_clean counts the tokens still late.
+        uint32_t M = 0, dl_clean = 0;
+        int32_t v_m1 = 0, need = 0, carry = 0;
+        bool counting = false;
+        if (m && pacing) {
+            M = handoff_latency(G, key, l, m);
+            v_m1 = tau_eff - (int32_t)M;
+            if (v_m1 < 0) { counting = true; need = -v_m1; dl_clean = 1; }
+        }
 
+        uint32_t span = 0;
         for (uint32_t base = 0; base < nI; base += span) {
+            rd.cper = (int)min((uint32_t)kR, (nI - base + 31u) / 32u);
+            span = 32u * (uint32_t)rd.cper;
             const uint32_t idx0 = base + (uint32_t)lane * rd.cper;
             rd.cnt = idx0 >= nI ? 0 : (int)min((uint32_t)rd.cper, nI - idx0);
             rd.j0 = idx0 + 2;
             rd.round_valid = min(span, nI - base);
             rd.last_j = base + rd.round_valid + 1;
-            int32_t cs[kR], cd[kR], s_S = 0, s_D = 0, negS = 0, negD = 0;
+            // every token's hash draw and both endpoints' jitter: sums and maxima of ((h * (2J+1)) >> 32)
+            uint32_t hS = 0, hD = 0, xS = 0, xD = 0;
             uint32_t hin = key + rd.j0 * kHashTok;
+#pragma unroll
+            for (int t = 0; t < kR; ++t)
+                if (t < rd.cper) {
+                    uint32_t h = mix32(hin);
+                    hin += kHashTok;
+                    h = t < rd.cnt ? h : 0u;
+                    const uint32_t a = __umulhi(h, G.mulS), b = __umulhi(h, G.mulD);
+                    hS += a; hD += b; xS = max(xS, a); xD = max(xD, b);
+                }
+            const int32_t s_S = rd.cnt * G.cS_base - (int32_t)hS, s_D = rd.cnt * G.cD_base - (int32_t)hD;
+            const bool posS = __all_sync(FULL, rd.cnt == 0 || (int32_t)xS <= G.cS_base);    // c = tau - x >= 0
+            const bool posD = __all_sync(FULL, rd.cnt == 0 || (int32_t)xD <= G.cD_base);
+            const int32_t totS = __reduce_add_sync(FULL, s_S), totD = __reduce_add_sync(FULL, s_D);
+            const bool searching = cand != 0 && m == 0;
+            const bool cand_clean = cand == 1 ? sS.clean : sD.clean;
+            const int32_t cand_after = cand == 1 ? sS.S + totS : sD.S + totD;
+            if (pacing && posS && posD && !counting && !(searching && (!cand_clean || cand_after > thr))) {
+                // nothing clamps, the buffer does not fill in this round: every TBT equals tau
+                sS.e += totS; sS.S += totS; sS.nt += rd.round_valid;
+                sD.e += totD; sD.S += totD; sD.nt += rd.round_valid;
+                if (searching) clean_until = rd.last_j;
+                continue;
+            }
+            // ---- the round needs its tokens one by one
+            int32_t cs[kR], cd[kR];
+            hin = key + rd.j0 * kHashTok;
 #pragma unroll
             for (int t = 0; t < kR; ++t) {
                 cs[t] = 0; cd[t] = 0;
                 if (t < rd.cper) {
                     const uint32_t h = mix32(hin);
                     hin += kHashTok;
-                    const bool valid = t < rd.cnt;
-                    cs[t] = valid ? G.cS_base - (int32_t)__umulhi(h, G.mulS) : 0;   // tau - (T + jitter in [-J, J])
-                    cd[t] = valid ? G.cD_base - (int32_t)__umulhi(h, G.mulD) : 0;
-                    s_S += cs[t]; s_D += cd[t]; negS |= cs[t]; negD |= cd[t];
+                    if (t < rd.cnt) {
+                        cs[t] = G.cS_base - (int32_t)__umulhi(h, G.mulS);     // tau - (T + jitter in [-J, J])
+                        cd[t] = G.cD_base - (int32_t)__umulhi(h, G.mulD);
+                    }
                 }
             }
-            const bool posS = !__any_sync(FULL, negS < 0), posD = !__any_sync(FULL, negD < 0);
             bool searchS = cand == 1 && m == 0, searchD = cand == 2 && m == 0;
             // buffers deeper than the ring: once the candidate stream clamps, one lane searches sequentially
             if ((searchS || searchD) && B > kRing / 2 && !(searchS ? posS : posD)) {
@@ -423,10 +424,34 @@ k_playout(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __r
                 searchS = searchD = false;
             }
             uint32_t m_new = 0;
-            const bool was_clean = cand == 1 ? sS.clean : sD.clean;
             play_round(sS, mxS, ntS, cs, s_S, posS, rd, win0, G.lo0, W0, searchS, B, thr, clean_until, ring, m_new, e_m);
             play_round(sD, mxD, ntD, cd, s_D, posD, rd, win1, G.lo1, W1, searchD, B, thr, clean_until, ring, m_new, e_m);
-            if (m_new) { m = m_new; m_clean = was_clean && (cand == 1 ? sS.clean : sD.clean); }
+            if (m_new) {
+                m = m_new;
+                m_clean = cand_clean && (cand == 1 ? sS.clean : sD.clean);
+                if (m_clean) {
+                    M = handoff_latency(G, key, l, m);
+                    v_m1 = e_m + (tau_eff - (int32_t)M);
+                    if (v_m1 < 0) { counting = true; need = -v_m1; dl_clean = 1; }
+                }
+            }
+            if (counting) {                                            // tokens m+2.. of this round on the target stream
+                int32_t ct[kR], sc = 0;
+#pragma unroll
+                for (int t = 0; t < kR; ++t) {
+                    ct[t] = (t < rd.cnt && rd.j0 + t >= m + 2) ? (cand == 1 ? cd[t] : cs[t]) : 0;
+                    sc += ct[t];
+                }
+                const int32_t incl = warp_inclusive_sum(sc, lane);
+                int32_t run = carry + incl - sc;
+                uint32_t here = 0;
+#pragma unroll
+                for (int t = 0; t < kR; ++t)
+                    if (t < rd.cnt && rd.j0 + t >= m + 2) { run += ct[t]; here += run < need; }
+                dl_clean += __reduce_add_sync(FULL, here);
+                carry += __shfl_sync(FULL, incl, 31);
+                if (carry >= need) counting = false;
+            }
         }
         if (m == kNone) m = 0;
 
@@ -440,17 +465,16 @@ k_playout(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __r
         // ---- stream X
         XResult xr = {0, 0, 0, 0, 0};
         if (m) {
-            const uint32_t M = handoff_latency(G, key, l, m);
             const bool target_clean = cand == 1 ? sD.clean : sS.clean;
             if (pacing && m_clean && target_clean) {
                 // nothing clamps but the hand-off itself: tokens up to m and after m+1 are delivered tau apart
-                const int32_t v = e_m + (tau_eff - (int32_t)M);               // lag of token m+1 behind its slot, negated
-                xr.stall = (uint32_t)tau_eff + (uint32_t)max(-v, 0);
+                xr.stall = (uint32_t)tau_eff + (uint32_t)max(-v_m1, 0);
                 xr.nt = nI - 1;
                 xr.sum = (nI - 1) * (uint32_t)tau_eff + xr.stall;
                 xr.mx = xr.stall;
-                xr.delayed = v < 0 ? count_delayed_clean(G, rd, key, nI, m, -v) : 0u;
+                xr.delayed = v_m1 < 0 ? dl_clean : 0u;
             } else {
+                if (!(pacing && m_clean)) M = handoff_latency(G, key, l, m);
                 play_x(G, rd, key, nI, m, M, win2, W2, &xres_s[wib]);
                 __syncwarp();
                 xr = xres_s[wib];

@@ -59,15 +59,17 @@ __global__ void k_finalize(uint32_t P, int G, const GroupConst* __restrict__ gc,
         tok_dev += a[A_TOK_DEVICE];
     }
     disco_policy_stats_t s;
-    const unsigned long long ttft_ticks = tot[A_TTFT_LO] + (tot[A_TTFT_HI] << 16);
+    const unsigned long long ttft_ticks = tot[A_TTFT_SUM];
     s.mean_ttft_s = N ? __ddiv_rn(__dmul_rn((double)ttft_ticks, 1e-6), (double)N) : 0.0;
     s.total_cost = cost;
     s.bin_p50_ttft = qb[0]; s.bin_p95_ttft = qb[1]; s.bin_p99_ttft = qb[2]; s.bin_p99_tbt = qb[3];
     s.p50_ttft_s = (float)bin_edge_seconds(qb[0]); s.p95_ttft_s = (float)bin_edge_seconds(qb[1]);
     s.p99_ttft_s = (float)bin_edge_seconds(qb[2]); s.p99_tbt_s = (float)bin_edge_seconds(qb[3]);
     s.n_requests = N; s.n_intervals = sum_n - N;
-    s.n_server_only = tot[A_SERVER_ONLY]; s.n_device_only = tot[A_DEVICE_ONLY]; s.n_race = tot[A_RACE];
-    s.n_device_started = tot[A_STARTED]; s.n_device_won = tot[A_DEVICE_WON]; s.n_migrations = tot[A_MIGR];
+    s.n_device_only = tot[A_DEVICE_ONLY]; s.n_race = tot[A_RACE];
+    s.n_server_only = N - s.n_device_only - s.n_race;          // every request takes exactly one decision
+    s.n_device_started = s.n_device_only + s.n_race;           // the device ran in both of these
+     s.n_device_won = tot[A_DEVICE_WON]; s.n_migrations = tot[A_MIGR];
     s.tok_device = tok_dev; s.tok_server = sum_n - tok_dev;
     s.prefill_tok_server = tot[A_PRE_SERVER]; s.prefill_tok_device = tot[A_PRE_DEVICE];
     s.delayed_tokens = tot[A_DELAYED];
