@@ -42,22 +42,12 @@ struct DevBuf {
     template <class T> T* as() const { return (T*)p; }
 };
 
+struct DevBufView { size_t off = 0; };
+
 int64_t ticks_of_seconds(float s) { return llrint((double)s * 1e6); }
 int64_t ticks_of_rate(float per_s) { return llrint(1e6 / (double)per_s); }
 
-struct HostReadback {            // pinned; filled by the load call
-    int32_t err[4];
-    uint32_t max_n;
-    uint32_t ng[kMaxGroups];
-    uint32_t grp_off[kMaxGroups + 1];
-    int32_t knot_max[kMaxGroups];
-    uint64_t grp_sum_n[kMaxGroups];
-};
-
-__global__ void k_knot_max(int G, const int32_t* __restrict__ knots, int32_t* __restrict__ out) {
-    const int g = threadIdx.x;
-    if (g < G) out[g] = knots[g * kNKnots + kNKnots - 1];
-}
+using HostReadback = LoadReadback;   // pinned host mirror of the load's read-back block
 
 }  // namespace
 
@@ -72,30 +62,37 @@ struct disco_ctx {
     std::vector<GroupConst> gc;
     // trace
     DevBuf in_prompt, in_out, in_ttft, in_sp, in_dp;      // staging of host inputs
-    DevBuf keys_a, keys_b, tmp_idx, radix_counts;
+    DevBuf keys_a, keys_b, tmp_idx;
     DevBuf S, l, nout, orig, sorted;
-    DevBuf cnt, cum_mass, ng, grp_off, knots, grp_sum_n, max_n, err, d_gc;
+    DevBuf zero, cum_mass, ng_exact, grp_off, knots, d_rb, d_gc;   // `zero`: every table a load must clear, contiguous
+    uint32_t *cnt = nullptr, *ng = nullptr, *max_n = nullptr, *radix_counts = nullptr;
+    uint64_t* grp_sum_n = nullptr;
+    int32_t* err = nullptr;
+    size_t zero_bytes = 0;
     HostReadback* rb = nullptr;
     // evaluation
     uint32_t P = 0;
     bool evaluated = false, reduced = false;
     std::vector<PolicyConst> pol;
-    DevBuf d_pol, d_prep, d_acc, d_hist_ttft, d_hist_tbt, d_stats, d_pol_list, d_classes, d_chunks, d_select;
+    DevBuf d_prep, d_accum, d_stats, d_tables, d_select;
+    struct View { void* p = nullptr; template <class T> T* as() const { return (T*)p; } };
+    View d_acc, d_hist_ttft, d_hist_tbt;               // three regions of d_accum (cleared by one memset)
+    View d_pol, d_classes, d_pol_list, d_chunks;       // four regions of d_tables (filled by one copy)
     DevBuf rec_u32[7], rec_u16[2], rec_win[3];
     void* stage = nullptr;       // pinned staging for the small host->device tables
     size_t stage_cap = 0;
     cudaEvent_t stage_free = nullptr;
     int32_t* sel_host = nullptr; // pinned [2]
+    void* stats_host = nullptr;  // pinned mirror of the statistics
+    size_t stats_host_cap = 0;
     bool timing = false;         // record events around the play-out and pair kernels
     cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
     float ms_timeline = 0.f, ms_pairs = 0.f;
     bool timing_valid = false;
 
     ~disco_ctx() {
-        DevBuf* all[] = {&in_prompt, &in_out, &in_ttft, &in_sp, &in_dp, &keys_a, &keys_b, &tmp_idx, &radix_counts,
-                         &S, &l, &nout, &orig, &sorted, &cnt, &cum_mass, &ng, &grp_off, &knots, &grp_sum_n, &max_n,
-                         &err, &d_gc, &d_pol, &d_prep, &d_acc, &d_hist_ttft, &d_hist_tbt, &d_stats, &d_pol_list,
-                         &d_classes, &d_chunks, &d_select};
+        DevBuf* all[] = {&in_prompt, &in_out, &in_ttft, &in_sp, &in_dp, &keys_a, &keys_b, &tmp_idx,
+                         &S, &l, &nout, &orig, &sorted, &zero, &cum_mass, &ng_exact, &grp_off, &knots, &d_rb, &d_gc, &d_prep, &d_accum, &d_stats, &d_tables, &d_select};
         for (DevBuf* b : all) b->release();
         for (auto& b : rec_u32) b.release();
         for (auto& b : rec_u16) b.release();
@@ -103,6 +100,7 @@ struct disco_ctx {
         if (rb) cudaFreeHost(rb);
         if (stage) cudaFreeHost(stage);
         if (sel_host) cudaFreeHost(sel_host);
+        if (stats_host) cudaFreeHost(stats_host);
         if (stage_free) cudaEventDestroy(stage_free);
         for (auto& e : ev) if (e) cudaEventDestroy(e);
     }
@@ -159,12 +157,22 @@ cudaError_t reserve_trace(disco_ctx* c, uint32_t n, bool host_inputs, bool has_s
         if (has_sp) R(in_sp, N);
         if (has_dp) R(in_dp, N);
     }
-    R(keys_a, N * 8); R(keys_b, N * 8); R(tmp_idx, std::max<size_t>(N, kMaxGroups) * 4);
-    R(radix_counts, 256 * kRadixMaxBlocks * 4);
+    R(keys_a, N * 8); R(keys_b, N * 8); R(tmp_idx, N * 4);
     R(S, N * 4); R(l, N * 2); R(nout, N * 2); R(orig, N * 4); R(sorted, N * 4);
-    R(cnt, (size_t)G * (kMaxPrompt + 1) * 4); R(cum_mass, (size_t)G * (kMaxPrompt + 2) * 8);
-    R(ng, kMaxGroups * 4); R(grp_off, (kMaxGroups + 1) * 4); R(knots, (size_t)G * kNKnots * 4);
-    R(grp_sum_n, kMaxGroups * 8); R(max_n, 4); R(err, 16); R(d_gc, (size_t)G * sizeof(GroupConst));
+    // one block for everything a load clears: cnt | grp_sum_n | ng | max_n | err | first radix counter buffer,
+    // followed by the second counter buffer
+    const size_t cnt_bytes = ((size_t)G * (kMaxPrompt + 1) * 4 + 15) / 16 * 16;
+    const size_t counts_bytes = (size_t)256 * kRadixMaxBlocks * 4;
+    const size_t head = cnt_bytes + kMaxGroups * 8 + kMaxGroups * 4 + 16 + 16;
+    R(zero, head + 2 * counts_bytes);
+    char* z = (char*)c->zero.p;
+    c->cnt = (uint32_t*)z; c->grp_sum_n = (uint64_t*)(z + cnt_bytes); c->ng = (uint32_t*)(z + cnt_bytes + kMaxGroups * 8);
+    c->max_n = (uint32_t*)(z + cnt_bytes + kMaxGroups * 12); c->err = (int32_t*)(z + cnt_bytes + kMaxGroups * 12 + 16);
+    c->radix_counts = (uint32_t*)(z + head);
+    c->zero_bytes = head + counts_bytes;
+    R(cum_mass, (size_t)G * (kMaxPrompt + 2) * 8); R(ng_exact, kMaxGroups * 4);
+    R(grp_off, (kMaxGroups + 1) * 4); R(knots, (size_t)G * kNKnots * 4);
+    R(d_rb, sizeof(LoadReadback)); R(d_gc, (size_t)G * sizeof(GroupConst));
 #undef R
     return cudaSuccess;
 }
@@ -221,27 +229,21 @@ int disco_load_trace(disco_ctx_t** pctx, const disco_trace_desc_t* d, void* stre
         a.sp = d->server_profile; a.dp = d->device_profile;
     }
     a.keys_a = c->keys_a.as<uint64_t>(); a.keys_b = c->keys_b.as<uint64_t>(); a.tmp_idx = c->tmp_idx.as<uint32_t>();
-    a.radix_counts = c->radix_counts.as<uint32_t>();
+    a.radix_counts = c->radix_counts; a.zero_block = c->zero.p; a.zero_bytes = c->zero_bytes;
+    a.ng_exact = c->ng_exact.as<uint32_t>(); a.readback = c->d_rb.as<LoadReadback>();
     a.S = c->S.as<int32_t>(); a.l = c->l.as<uint16_t>(); a.nout = c->nout.as<uint16_t>(); a.orig = c->orig.as<uint32_t>();
-    a.sorted = c->sorted.as<int32_t>(); a.cnt = c->cnt.as<uint32_t>(); a.cum_mass = c->cum_mass.as<int64_t>();
-    a.ng = c->ng.as<uint32_t>(); a.grp_off = c->grp_off.as<uint32_t>(); a.knots = c->knots.as<int32_t>();
-    a.grp_sum_n = c->grp_sum_n.as<uint64_t>(); a.max_n = c->max_n.as<uint32_t>(); a.err = c->err.as<int32_t>();
+    a.sorted = c->sorted.as<int32_t>(); a.cnt = c->cnt; a.cum_mass = c->cum_mass.as<int64_t>();
+    a.ng = c->ng; a.grp_off = c->grp_off.as<uint32_t>(); a.knots = c->knots.as<int32_t>();
+    a.grp_sum_n = c->grp_sum_n; a.max_n = c->max_n; a.err = c->err;
     // the profile table is read from pageable memory: this copy returns once it has been staged
     if ((e = cudaMemcpyAsync(c->d_gc.p, c->gc.data(), c->gc.size() * sizeof(GroupConst), cudaMemcpyHostToDevice, st)) != cudaSuccess)
         return bail(fail_cuda(e, "profile copy"));
     if ((e = run_load(a, st)) != cudaSuccess) return bail(fail_cuda(e, "trace ingestion kernels"));
-    g_launches += load_kernel_launches(n, c->G) + 1;
+    g_launches += load_kernel_launches(n, c->G);
     // read back the few numbers the host needs: error word, group sizes, longest output, largest TTFT per group
     HostReadback* rb = c->rb;
-    k_knot_max<<<1, kMaxGroups, 0, st>>>(c->G, a.knots, (int32_t*)c->tmp_idx.p);
-    bool ok = true;
-    ok &= cudaMemcpyAsync(rb->err, a.err, 16, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-    ok &= cudaMemcpyAsync(&rb->max_n, a.max_n, 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-    ok &= cudaMemcpyAsync(rb->ng, a.ng, 4 * c->G, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-    ok &= cudaMemcpyAsync(rb->grp_off, a.grp_off, 4 * (c->G + 1), cudaMemcpyDeviceToHost, st) == cudaSuccess;
-    ok &= cudaMemcpyAsync(rb->knot_max, c->tmp_idx.p, 4 * c->G, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-    ok &= cudaMemcpyAsync(rb->grp_sum_n, a.grp_sum_n, 8 * c->G, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-    if (!ok) return bail(fail_cuda(cudaGetLastError(), "readback"));
+    if ((e = cudaMemcpyAsync(rb, c->d_rb.p, sizeof(LoadReadback), cudaMemcpyDeviceToHost, st)) != cudaSuccess)
+        return bail(fail_cuda(e, "readback"));
     if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return bail(fail_cuda(e, "trace ingestion"));
     if (rb->err[0]) {
         static const char* what[] = {"", "prompt length outside 1..4096", "output length outside 1..8192",
@@ -333,10 +335,12 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
     size_t wmax[3] = {1, 1, 1};
     for (const ClassConst& cc : classes) for (int k = 0; k < 3; ++k) wmax[k] = std::max<size_t>(wmax[k], cc.W[k]);
 #define R(buf, bytes) if ((e = c->buf.reserve(bytes)) != cudaSuccess) return fail_cuda(e, "device allocation for the evaluation")
-    R(d_pol, P * sizeof(PolicyConst)); R(d_prep, (size_t)G * P * sizeof(Prep));
-    R(d_acc, (size_t)P * G * kNAcc * 8); R(d_hist_ttft, (size_t)P * kNBins * 8); R(d_hist_tbt, (size_t)P * kNBins * 8);
-    R(d_stats, P * sizeof(disco_policy_stats_t)); R(d_pol_list, P * 4);
-    R(d_classes, classes.size() * sizeof(ClassConst)); R(d_select, 8);
+    R(d_prep, (size_t)G * P * sizeof(Prep));
+    const size_t acc_bytes = (size_t)P * G * kNAcc * 8, hist_bytes = (size_t)P * kNBins * 8;
+    R(d_accum, acc_bytes + 2 * hist_bytes);
+    c->d_acc.p = c->d_accum.p; c->d_hist_ttft.p = (char*)c->d_accum.p + acc_bytes;
+    c->d_hist_tbt.p = (char*)c->d_accum.p + acc_bytes + hist_bytes;
+    R(d_stats, P * sizeof(disco_policy_stats_t) + 16); R(d_select, 8);
     for (int k = 0; k < 7; ++k) R(rec_u32[k], N1 * 4);
     for (int k = 0; k < 2; ++k) R(rec_u16[k], N1 * 2);
     for (int k = 0; k < 3; ++k) R(rec_win[k], N1 * wmax[k] * 4);
@@ -351,7 +355,7 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
         cls_range.push_back({b, (uint32_t)pol_list.size()});
     }
     const uint32_t tiles = (P + 31) / 32;
-    const uint32_t want_chunks = std::max<uint32_t>(1, 592 / std::min<uint32_t>(tiles, 592));
+    const uint32_t want_chunks = std::max<uint32_t>(1, 296 / std::min<uint32_t>(tiles, 296));
     uint32_t CH = (uint32_t)((N1 + want_chunks - 1) / want_chunks);
     CH = (CH + 255) / 256 * 256;
     CH = std::min<uint32_t>(std::max<uint32_t>(CH, 256), 65280);     // 16-bit histogram counters per block
@@ -359,7 +363,6 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
     for (int g = 0; g < G; ++g)
         for (uint32_t s = rb.grp_off[g]; s < rb.grp_off[g + 1]; s += CH)
             chunks.push_back({s, std::min(CH, rb.grp_off[g + 1] - s), g, 0});
-    R(d_chunks, std::max<size_t>(1, chunks.size()) * sizeof(Chunk));
 #undef R
 
     // ---- small tables to the device through pinned staging
@@ -373,27 +376,31 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
         CU(cudaMallocHost(&c->stage, need));
         c->stage_cap = need;
     }
+    // one staging block, one copy: policies | classes | policy list | chunks (16-byte aligned regions)
     char* sp = (char*)c->stage;
-    auto push = [&](void* dst, const void* src, size_t bytes) -> cudaError_t {
-        if (!bytes) return cudaSuccess;
-        std::memcpy(sp, src, bytes);
-        cudaError_t r = cudaMemcpyAsync(dst, sp, bytes, cudaMemcpyHostToDevice, st);
-        sp += (bytes + 15) / 16 * 16;
-        return r;
+    size_t off = 0;
+    auto put = [&](DevBufView& v, const void* src, size_t bytes) {
+        std::memcpy(sp + off, src, bytes);
+        v.off = off;
+        off += (bytes + 15) / 16 * 16;
     };
-    CU(push(c->d_pol.p, pc.data(), P * sizeof(PolicyConst)));
-    CU(push(c->d_classes.p, classes.data(), classes.size() * sizeof(ClassConst)));
-    CU(push(c->d_pol_list.p, pol_list.data(), P * 4));
-    CU(push(c->d_chunks.p, chunks.data(), chunks.size() * sizeof(Chunk)));
+    DevBufView v_pol, v_cls, v_list, v_chunks;
+    put(v_pol, pc.data(), P * sizeof(PolicyConst));
+    put(v_cls, classes.data(), classes.size() * sizeof(ClassConst));
+    put(v_list, pol_list.data(), P * 4);
+    put(v_chunks, chunks.data(), chunks.size() * sizeof(Chunk));
+    if ((e = c->d_tables.reserve(off + 16)) != cudaSuccess) return fail_cuda(e, "device allocation for the evaluation");
+    char* dt = (char*)c->d_tables.p;
+    c->d_pol.p = dt + v_pol.off; c->d_classes.p = dt + v_cls.off; c->d_pol_list.p = dt + v_list.off;
+    c->d_chunks.p = dt + v_chunks.off;
+    CU(cudaMemcpyAsync(dt, sp, off, cudaMemcpyHostToDevice, st));
     CU(cudaEventRecord(c->stage_free, st));
 
-    CU(cudaMemsetAsync(c->d_acc.p, 0, (size_t)P * G * kNAcc * 8, st));
-    CU(cudaMemsetAsync(c->d_hist_ttft.p, 0, (size_t)P * kNBins * 8, st));
-    CU(cudaMemsetAsync(c->d_hist_tbt.p, 0, (size_t)P * kNBins * 8, st));
+    CU(cudaMemsetAsync(c->d_accum.p, 0, acc_bytes + 2 * hist_bytes, st));
 
     // ---- Algorithms 1-3 for every (group, policy)
     CU(launch_prep(c->d_pol.as<PolicyConst>(), P, G, c->d_gc.as<GroupConst>(), c->cum_mass.as<int64_t>(),
-                   c->cnt.as<uint32_t>(), c->sorted.as<int32_t>(), c->grp_off.as<uint32_t>(), c->d_prep.as<Prep>(), st));
+                   c->cnt, c->sorted.as<int32_t>(), c->grp_off.as<uint32_t>(), c->d_prep.as<Prep>(), st));
 
     TraceDev tr;
     tr.n = n; tr.n_groups = G; tr.S = c->S.as<int32_t>(); tr.l = c->l.as<uint16_t>(); tr.nout = c->nout.as<uint16_t>();
@@ -416,7 +423,7 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
     for (size_t k = 0; k < classes.size(); ++k) {
         const ClassConst* dcc = c->d_classes.as<ClassConst>() + k;
         if (timed) CU(cudaEventRecord(c->ev[0], st));
-        CU(launch_timeline(tr, c->d_gc.as<GroupConst>(), dcc, c->knots.as<int32_t>(), seed, rec, c->err.as<int32_t>(), st));
+        CU(launch_timeline(tr, c->d_gc.as<GroupConst>(), dcc, c->knots.as<int32_t>(), seed, rec, c->err, st));
         if (timed) CU(cudaEventRecord(c->ev[1], st));
         CU(launch_pairs(tr, c->d_gc.as<GroupConst>(), dcc, c->d_prep.as<Prep>(), P,
                         c->d_pol_list.as<uint32_t>() + cls_range[k].first, cls_range[k].second - cls_range[k].first,
@@ -436,11 +443,20 @@ int disco_reduce_stats(disco_ctx_t* c, disco_policy_stats_t* stats, void* stream
     if (!c->evaluated) return fail(DISCO_EINVAL, "no evaluation to reduce");
     cudaStream_t st = (cudaStream_t)stream;
     CU(launch_finalize(c->P, c->G, c->d_gc.as<GroupConst>(), c->d_acc.as<uint64_t>(), c->d_hist_ttft.as<uint64_t>(),
-                       c->d_hist_tbt.as<uint64_t>(), c->grp_sum_n.as<uint64_t>(), c->grp_off.as<uint32_t>(),
-                       c->d_stats.as<disco_policy_stats_t>(), st));
-    CU(cudaMemcpyAsync(stats, c->d_stats.p, c->P * sizeof(disco_policy_stats_t), cudaMemcpyDeviceToHost, st));
-    CU(cudaMemcpyAsync(c->rb->err, c->err.p, 16, cudaMemcpyDeviceToHost, st));
+                       c->d_hist_tbt.as<uint64_t>(), c->grp_sum_n, c->grp_off.as<uint32_t>(),
+                       c->d_stats.as<disco_policy_stats_t>(), c->err, st));
+    // statistics and the error word come back in one copy through pinned memory
+    const size_t bytes = c->P * sizeof(disco_policy_stats_t) + 16;
+    if (bytes > c->stats_host_cap) {
+        if (c->stats_host) cudaFreeHost(c->stats_host);
+        c->stats_host = nullptr; c->stats_host_cap = 0;
+        CU(cudaMallocHost(&c->stats_host, bytes));
+        c->stats_host_cap = bytes;
+    }
+    CU(cudaMemcpyAsync(c->stats_host, c->d_stats.p, bytes, cudaMemcpyDeviceToHost, st));
     CU(cudaStreamSynchronize(st));
+    std::memcpy(stats, c->stats_host, c->P * sizeof(disco_policy_stats_t));
+    std::memcpy(c->rb->err, (char*)c->stats_host + c->P * sizeof(disco_policy_stats_t), 16);
     g_launches += 1;
     if (c->timing_valid) {
         CU(cudaEventElapsedTime(&c->ms_timeline, c->ev[0], c->ev[1]));
@@ -509,7 +525,7 @@ int64_t disco_get_group_tables(disco_ctx_t* c, uint32_t g, int64_t* cnt, int32_t
     const uint32_t ng = c->rb->ng[g], off = c->rb->grp_off[g];
     if (cnt) {
         std::vector<uint32_t> tmp(kMaxPrompt + 1);
-        CU(cudaMemcpyAsync(tmp.data(), c->cnt.as<uint32_t>() + (size_t)g * (kMaxPrompt + 1), tmp.size() * 4, cudaMemcpyDeviceToHost, st));
+        CU(cudaMemcpyAsync(tmp.data(), c->cnt + (size_t)g * (kMaxPrompt + 1), tmp.size() * 4, cudaMemcpyDeviceToHost, st));
         CU(cudaStreamSynchronize(st));
         for (size_t i = 0; i < tmp.size(); ++i) cnt[i] = tmp[i];
     }

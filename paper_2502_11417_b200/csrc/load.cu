@@ -15,11 +15,17 @@ __global__ void k_ingest(uint32_t n, const int32_t* __restrict__ prompt, const i
                          const float* __restrict__ ttft, const uint8_t* __restrict__ sp,
                          const uint8_t* __restrict__ dp, uint32_t ns, uint32_t nd, uint64_t* __restrict__ keys,
                          uint32_t* __restrict__ cnt, unsigned long long* __restrict__ grp_sum_n,
-                         uint32_t* __restrict__ max_n, int32_t* __restrict__ err) {
+                         uint32_t* __restrict__ grp_n, uint32_t* __restrict__ max_n, int32_t* __restrict__ err,
+                         int32_t* __restrict__ S_out, uint16_t* __restrict__ l_out, uint16_t* __restrict__ n_out,
+                         uint32_t* __restrict__ orig_out, uint32_t* __restrict__ counts0, uint32_t per_block0,
+                         uint32_t blocks0) {
+    // S_out..orig_out: single-group traces keep the caller's order, so the internal arrays are written here;
+    // counts0: first radix digit counted per sort block (small traces; large ones use the histogram kernel)
     __shared__ unsigned long long s_sum[kMaxGroups];
+    __shared__ uint32_t s_cnt[kMaxGroups];
     __shared__ uint32_t s_max;
     const int G = (int)(ns * nd);
-    for (int g = threadIdx.x; g < G; g += blockDim.x) s_sum[g] = 0;
+    for (int g = threadIdx.x; g < G; g += blockDim.x) { s_sum[g] = 0; s_cnt[g] = 0; }
     if (threadIdx.x == 0) s_max = 0;
     __syncthreads();
     for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
@@ -42,11 +48,14 @@ __global__ void k_ingest(uint32_t n, const int32_t* __restrict__ prompt, const i
         keys[i] = ((uint64_t)g << 32) | (uint32_t)S;
         atomicAdd(&cnt[g * (kMaxPrompt + 1) + l], 1u);
         atomicAdd(&s_sum[g], (unsigned long long)o);
+        atomicAdd(&s_cnt[g], 1u);
         atomicMax(&s_max, (uint32_t)o);
+        if (S_out) { S_out[i] = (int32_t)S; l_out[i] = (uint16_t)l; n_out[i] = (uint16_t)o; orig_out[i] = i; }
+        if (counts0) atomicAdd(&counts0[((uint32_t)S & 255u) * blocks0 + i / per_block0], 1u);
     }
     __syncthreads();
     for (int g = threadIdx.x; g < G; g += blockDim.x)
-        if (s_sum[g]) atomicAdd(&grp_sum_n[g], s_sum[g]);
+        if (s_cnt[g]) { atomicAdd(&grp_sum_n[g], s_sum[g]); atomicAdd(&grp_n[g], s_cnt[g]); }
     if (threadIdx.x == 0 && s_max) atomicMax(max_n, s_max);
 }
 
@@ -67,8 +76,9 @@ __global__ void k_radix_hist(const uint64_t* __restrict__ keys, uint32_t n, uint
 }
 
 // exclusive scan of `m` counters by one block of 1024 threads
-__global__ void k_scan_counts(uint32_t* __restrict__ counts, uint32_t m) {
+__global__ void k_scan_counts(uint32_t* __restrict__ counts, uint32_t m, uint32_t* __restrict__ clear = nullptr) {
     __shared__ uint32_t part[1024];
+    if (clear) for (uint32_t i = threadIdx.x; i < m; i += 1024) clear[i] = 0;
     const uint32_t per = (m + 1023u) / 1024u;
     const uint32_t lo = min(m, threadIdx.x * per), hi = min(m, lo + per);
     uint32_t s = 0;
@@ -87,7 +97,8 @@ __global__ void k_scan_counts(uint32_t* __restrict__ counts, uint32_t m) {
 
 __global__ void k_radix_scatter(const uint64_t* __restrict__ keys_in, uint64_t* __restrict__ keys_out,
                                 const uint32_t* __restrict__ pay_in, uint32_t* __restrict__ pay_out, uint32_t n,
-                                uint32_t per_block, int shift, const uint32_t* __restrict__ offsets) {
+                                uint32_t per_block, int shift, const uint32_t* __restrict__ offsets,
+                                uint32_t* __restrict__ counts_next = nullptr, int32_t* __restrict__ low_out = nullptr) {
     __shared__ uint32_t run[256];                 // next output slot of each digit for this block
     __shared__ uint32_t wcnt[kRadixWarps][256];   // keys of each digit per warp in the current slab
     const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -109,8 +120,10 @@ __global__ void k_radix_scatter(const uint64_t* __restrict__ keys_in, uint64_t* 
             uint32_t before = 0;
             for (int k = 0; k < w; ++k) before += wcnt[k][dig];
             const uint32_t pos = run[dig] + before + rank;
-            keys_out[pos] = key;
+            if (low_out) low_out[pos] = (int32_t)(uint32_t)key; else keys_out[pos] = key;
             if (pay_out) pay_out[pos] = pay_in ? pay_in[i] : i;
+            if (counts_next)
+                atomicAdd(&counts_next[((uint32_t)(key >> (shift + 8)) & 255u) * gridDim.x + pos / per_block], 1u);
         }
         __syncthreads();
         uint32_t tot = 0;
@@ -164,21 +177,31 @@ __global__ void k_group_mass(const uint32_t* __restrict__ cnt, int64_t* __restri
     if (threadIdx.x == NT - 1) { out[L] = (int64_t)pm[NT - 1]; ng[g] = pc[NT - 1]; }
 }
 
-// Group offsets in the partitioned order and the 257 knots K_g[k] = sorted_g[(k (N_g - 1)) / 256].
+// Group offsets in the partitioned order, the 257 knots K_g[k] = sorted_g[(k (N_g - 1)) / 256] and the few
+// numbers the host reads back.  One block per group (after k_group_mass has produced the group sizes).
 __global__ void k_group_knots(int G, const uint32_t* __restrict__ ng, const int32_t* __restrict__ sorted,
-                              uint32_t* __restrict__ grp_off, int32_t* __restrict__ knots) {
+                              uint32_t* __restrict__ grp_off, int32_t* __restrict__ knots,
+                              const int32_t* __restrict__ err, const uint32_t* __restrict__ max_n,
+                              const unsigned long long* __restrict__ grp_sum_n, LoadReadback* __restrict__ rb) {
     __shared__ uint32_t off[kMaxGroups + 1];
+    const int g = blockIdx.x;
     if (threadIdx.x == 0) {
         uint32_t r = 0;
-        for (int g = 0; g < G; ++g) { off[g] = r; r += ng[g]; }
+        for (int k = 0; k < G; ++k) { off[k] = r; r += ng[k]; }
         off[G] = r;
-        for (int g = 0; g <= G; ++g) grp_off[g] = off[g];
     }
     __syncthreads();
-    for (int idx = threadIdx.x; idx < G * kNKnots; idx += blockDim.x) {
-        const int g = idx / kNKnots, k = idx % kNKnots;
-        const uint32_t N = off[g + 1] - off[g];
-        knots[idx] = N ? sorted[off[g] + (uint32_t)(((uint64_t)k * (N - 1)) / 256u)] : 0;
+    const uint32_t N = off[g + 1] - off[g];
+    for (int k = threadIdx.x; k < kNKnots; k += blockDim.x)
+        knots[g * kNKnots + k] = N ? sorted[off[g] + (uint32_t)(((uint64_t)k * (N - 1)) / 256u)] : 0;
+    if (threadIdx.x == 0) {
+        rb->knot_max[g] = N ? sorted[off[g] + N - 1] : 0;
+        rb->ng[g] = N; rb->grp_sum_n[g] = grp_sum_n[g];
+        if (g == 0) {
+            for (int k = 0; k <= G; ++k) { grp_off[k] = off[k]; rb->grp_off[k] = off[k]; }
+            for (int k = 0; k < 4; ++k) rb->err[k] = err[k];
+            rb->max_n = *max_n;
+        }
     }
 }
 
@@ -206,40 +229,60 @@ cudaError_t radix_pass(const uint64_t* kin, uint64_t* kout, const uint32_t* pin,
 
 uint32_t load_kernel_launches(uint32_t n, int G) {
     if (n == 0) return 2;
-    const uint32_t passes = G > 1 ? 6 : 4;       // radix passes: partition + 5, or 4
-    return 1 + 1 + 3 * passes + 1 + 2;            // ingest, gather, passes, low words, group tables
+    if (G == 1 && n <= (1u << 20)) return 1 + 2 * 4 + 2;     // ingest, (scan, scatter) x 4, group tables
+    const uint32_t passes = G > 1 ? 6 : 4;                  // radix passes: partition + 5, or 4
+    return 1 + (G > 1 ? 1 : 0) + 3 * passes + 1 + 2;         // ingest, gather, passes, low words, group tables
 }
 
 cudaError_t run_load(const LoadArgs& a, cudaStream_t st) {
     const uint32_t n = a.n;
     const int G = (int)(a.ns * a.nd);
     cudaError_t e;
-    if ((e = cudaMemsetAsync(a.cnt, 0, sizeof(uint32_t) * G * (kMaxPrompt + 1), st))) return e;
-    if ((e = cudaMemsetAsync(a.grp_sum_n, 0, sizeof(uint64_t) * kMaxGroups, st))) return e;
-    if ((e = cudaMemsetAsync(a.max_n, 0, sizeof(uint32_t), st))) return e;
-    if ((e = cudaMemsetAsync(a.err, 0, sizeof(int32_t) * 4, st))) return e;
+    // radix geometry (as in radix_pass)
+    uint32_t blocks = (n + 4095u) / 4096u;
+    if (blocks < 1) blocks = 1;
+    if (blocks > kRadixMaxBlocks) blocks = kRadixMaxBlocks;
+    uint32_t per_block = (n + blocks - 1) / blocks;
+    per_block = (per_block + kRadixThreads - 1) / kRadixThreads * kRadixThreads;
+    const bool small = G == 1 && n <= (1u << 20);      // fused histograms pay off while launches dominate
+    // everything that must start at zero lies in one block: cnt, grp_sum_n, grp_n, max_n, err, counts A
+    if ((e = cudaMemsetAsync(a.zero_block, 0, a.zero_bytes, st))) return e;
     if (n) {
+        uint32_t* counts_a = a.radix_counts;
+        uint32_t* counts_b = a.radix_counts + 256u * kRadixMaxBlocks;
         k_ingest<<<grid_for(n, kIngestThreads), kIngestThreads, 0, st>>>(
             n, a.prompt, a.outlen, a.ttft, a.sp, a.dp, a.ns, a.nd, a.keys_a, a.cnt,
-            (unsigned long long*)a.grp_sum_n, a.max_n, a.err);
-        // internal request order: stable partition by group (identity for a single group)
-        const uint32_t* orig_src = nullptr;
+            (unsigned long long*)a.grp_sum_n, a.ng, a.max_n, a.err,
+            G == 1 ? a.S : nullptr, a.l, a.nout, a.orig, small ? counts_a : nullptr, per_block, blocks);
         if (G > 1) {
-            if ((e = radix_pass(a.keys_a, a.keys_b, nullptr, a.tmp_idx, n, 32, a.radix_counts, st))) return e;
-            orig_src = a.tmp_idx;
+            // internal request order: stable partition by group
+            if ((e = radix_pass(a.keys_a, a.keys_b, nullptr, a.tmp_idx, n, 32, counts_b, st))) return e;
+            k_gather<<<grid_for(n, 256), 256, 0, st>>>(n, a.tmp_idx, a.keys_a, a.prompt, a.outlen, a.S, a.l, a.nout, a.orig);
         }
-        k_gather<<<grid_for(n, 256), 256, 0, st>>>(n, orig_src, a.keys_a, a.prompt, a.outlen, a.S, a.l, a.nout, a.orig);
         // sort (group, ticks): four byte passes over the ticks, one over the group id
         uint64_t *src = a.keys_a, *dst = a.keys_b;
         const int passes = G > 1 ? 5 : 4;
-        for (int p = 0; p < passes; ++p) {
-            if ((e = radix_pass(src, dst, nullptr, nullptr, n, 8 * p, a.radix_counts, st))) return e;
-            uint64_t* t = src; src = dst; dst = t;
+        if (small) {
+            uint32_t *cur = counts_a, *nxt = counts_b;
+            for (int p = 0; p < passes; ++p) {
+                const bool last = p == passes - 1;
+                k_scan_counts<<<1, 1024, 0, st>>>(cur, 256u * blocks, last ? nullptr : nxt);
+                k_radix_scatter<<<blocks, kRadixThreads, 0, st>>>(src, dst, nullptr, nullptr, n, per_block, 8 * p, cur,
+                                                                  last ? nullptr : nxt, last ? a.sorted : nullptr);
+                uint64_t* t = src; src = dst; dst = t;
+                uint32_t* c = cur; cur = nxt; nxt = c;
+            }
+        } else {
+            for (int p = 0; p < passes; ++p) {
+                if ((e = radix_pass(src, dst, nullptr, nullptr, n, 8 * p, counts_b, st))) return e;
+                uint64_t* t = src; src = dst; dst = t;
+            }
+            k_low_words<<<grid_for(n, 256), 256, 0, st>>>(n, src, a.sorted);
         }
-        k_low_words<<<grid_for(n, 256), 256, 0, st>>>(n, src, a.sorted);
     }
-    k_group_mass<<<G, 1024, 0, st>>>(a.cnt, a.cum_mass, a.ng);
-    k_group_knots<<<1, 256, 0, st>>>(G, a.ng, a.sorted, a.grp_off, a.knots);
+    k_group_mass<<<G, 1024, 0, st>>>(a.cnt, a.cum_mass, a.ng_exact);
+    k_group_knots<<<G, 256, 0, st>>>(G, a.ng, a.sorted, a.grp_off, a.knots, a.err, a.max_n,
+                                     (const unsigned long long*)a.grp_sum_n, a.readback);
     return cudaGetLastError();
 }
 

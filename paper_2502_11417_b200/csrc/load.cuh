@@ -7,6 +7,15 @@ namespace disco {
 
 constexpr uint32_t kRadixMaxBlocks = 1024;
 
+struct LoadReadback {            // what the host needs after a load, gathered for one copy
+    int32_t err[4];
+    uint32_t max_n;
+    uint32_t ng[kMaxGroups];
+    uint32_t grp_off[kMaxGroups + 1];
+    int32_t knot_max[kMaxGroups];
+    uint64_t grp_sum_n[kMaxGroups];
+};
+
 struct LoadArgs {
     uint32_t n, ns, nd;
     // inputs in the caller's order
@@ -16,7 +25,10 @@ struct LoadArgs {
     // scratch
     uint64_t *keys_a, *keys_b;            // [n] (group << 32 | ticks)
     uint32_t* tmp_idx;                    // [n]
-    uint32_t* radix_counts;               // [256 * kRadixMaxBlocks]
+    uint32_t* radix_counts;               // [2][256 * kRadixMaxBlocks]; the first half lies in zero_block
+    void* zero_block; size_t zero_bytes;  // cnt, grp_sum_n, ng, max_n, err and the first counter buffer, contiguous
+    uint32_t* ng_exact;                   // [G] group sizes recounted from the length histogram
+    LoadReadback* readback;               // device copy of what the host reads back
     // outputs
     int32_t* S; uint16_t *l, *nout; uint32_t* orig;   // internal (group-partitioned) order, [n]
     int32_t* sorted;                      // [n] ticks ascending within each group

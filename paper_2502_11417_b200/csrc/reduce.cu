@@ -10,14 +10,43 @@ __device__ __forceinline__ double bin_edge_seconds(int b) {
     return __dmul_rn((double)edge, 1e-6);
 }
 
-// nearest-rank quantile: bin holding the ceil(q*M)-th smallest item
-__device__ int quantile_bin(const unsigned long long* hist, double q, unsigned long long M) {
-    if (M == 0) return 0;
-    unsigned long long rank = (unsigned long long)ceil(__dmul_rn(q, (double)M));
-    if (rank < 1) rank = 1;
-    unsigned long long acc = 0;
-    for (int b = 0; b < kNBins; ++b) { acc += hist[b]; if (acc >= rank) return b; }
-    return kNBins - 1;
+// Nearest-rank quantiles of one 864-bin histogram by a warp: lane i owns bins [27 i, 27 i + 27); the bin
+// holding the ceil(q*M)-th smallest item is found from the lanes' prefix counts.  All lanes return the bins.
+constexpr int kBinsPerLane = kNBins / 32;
+static_assert(kBinsPerLane * 32 == kNBins, "864 bins split evenly over a warp");
+
+__device__ void warp_quantile_bins(const unsigned long long* hist, unsigned long long M, const double* qs, int nq,
+                                   int* out) {
+    const int lane = threadIdx.x & 31;
+    unsigned long long mine[kBinsPerLane], sum = 0;
+#pragma unroll
+    for (int i = 0; i < kBinsPerLane; ++i) { mine[i] = hist[lane * kBinsPerLane + i]; sum += mine[i]; }
+    unsigned long long incl = sum;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const unsigned long long v = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+        if (lane >= off) incl += v;
+    }
+    const unsigned long long excl = incl - sum;
+    for (int k = 0; k < nq; ++k) {
+        int bin = 0;
+        if (M) {
+            unsigned long long rank = (unsigned long long)ceil(__dmul_rn(qs[k], (double)M));
+            if (rank < 1) rank = 1;
+            int found = -1;
+            if (rank > excl && rank <= incl) {
+                unsigned long long acc = excl;
+#pragma unroll
+                for (int i = 0; i < kBinsPerLane; ++i) {
+                    acc += mine[i];
+                    if (found < 0 && acc >= rank) found = lane * kBinsPerLane + i;
+                }
+            }
+            const unsigned owner = __ballot_sync(0xFFFFFFFFu, found >= 0);
+            bin = owner ? __shfl_sync(0xFFFFFFFFu, found, __ffs(owner) - 1) : kNBins - 1;
+        }
+        out[k] = bin;
+    }
 }
 
 // One block of 32 threads per policy.
@@ -25,8 +54,9 @@ __global__ void k_finalize(uint32_t P, int G, const GroupConst* __restrict__ gc,
                            const unsigned long long* __restrict__ acc, const unsigned long long* __restrict__ hist_ttft,
                            const unsigned long long* __restrict__ hist_tbt,
                            const unsigned long long* __restrict__ grp_sum_n, const uint32_t* __restrict__ grp_off,
-                           disco_policy_stats_t* __restrict__ stats) {
+                           disco_policy_stats_t* __restrict__ stats, const int32_t* __restrict__ err) {
     const uint32_t p = blockIdx.x;
+    if (p == 0 && threadIdx.x < 4) ((int32_t*)(stats + P))[threadIdx.x] = err[threadIdx.x];   // error word rides along
     __shared__ unsigned long long tot[kNAcc];
     __shared__ int qb[4];
     const unsigned long long N = grp_off[G];
@@ -37,11 +67,12 @@ __global__ void k_finalize(uint32_t P, int G, const GroupConst* __restrict__ gc,
     }
     unsigned long long sum_n = 0;
     for (int g = 0; g < G; ++g) sum_n += grp_sum_n[g];
-    if (threadIdx.x < 3) {
-        const double q = threadIdx.x == 0 ? 0.50 : threadIdx.x == 1 ? 0.95 : 0.99;
-        qb[threadIdx.x] = quantile_bin(hist_ttft + (size_t)p * kNBins, q, N);
-    } else if (threadIdx.x == 3) {
-        qb[3] = quantile_bin(hist_tbt + (size_t)p * kNBins, 0.99, sum_n - N);
+    {
+        const double q_ttft[3] = {0.50, 0.95, 0.99}, q_tbt[1] = {0.99};
+        int b3[3], b1[1];
+        warp_quantile_bins(hist_ttft + (size_t)p * kNBins, N, q_ttft, 3, b3);
+        warp_quantile_bins(hist_tbt + (size_t)p * kNBins, sum_n - N, q_tbt, 1, b1);
+        if (threadIdx.x == 0) { qb[0] = b3[0]; qb[1] = b3[1]; qb[2] = b3[2]; qb[3] = b1[0]; }
     }
     __syncthreads();
     if (threadIdx.x != 0) return;
@@ -69,7 +100,7 @@ __global__ void k_finalize(uint32_t P, int G, const GroupConst* __restrict__ gc,
     s.n_device_only = tot[A_DEVICE_ONLY]; s.n_race = tot[A_RACE];
     s.n_server_only = N - s.n_device_only - s.n_race;          // every request takes exactly one decision
     s.n_device_started = s.n_device_only + s.n_race;           // the device ran in both of these
-     s.n_device_won = tot[A_DEVICE_WON]; s.n_migrations = tot[A_MIGR];
+    s.n_device_won = tot[A_DEVICE_WON]; s.n_migrations = tot[A_MIGR];
     s.tok_device = tok_dev; s.tok_server = sum_n - tok_dev;
     s.prefill_tok_server = tot[A_PRE_SERVER]; s.prefill_tok_device = tot[A_PRE_DEVICE];
     s.delayed_tokens = tot[A_DELAYED];
@@ -121,10 +152,10 @@ __global__ void k_select(const disco_policy_stats_t* __restrict__ stats, uint32_
 
 cudaError_t launch_finalize(uint32_t P, int G, const GroupConst* gc, const uint64_t* acc, const uint64_t* hist_ttft,
                             const uint64_t* hist_tbt, const uint64_t* grp_sum_n, const uint32_t* grp_off,
-                            disco_policy_stats_t* stats, cudaStream_t st) {
+                            disco_policy_stats_t* stats, const int32_t* err, cudaStream_t st) {
     k_finalize<<<P, 32, 0, st>>>(P, G, gc, (const unsigned long long*)acc, (const unsigned long long*)hist_ttft,
                                  (const unsigned long long*)hist_tbt, (const unsigned long long*)grp_sum_n, grp_off,
-                                 stats);
+                                 stats, err);
     return cudaGetLastError();
 }
 
