@@ -192,7 +192,7 @@ uint64_t disco_kernel_launch_count(void);
  * This call does the part of the load step that turns server TTFTs into the empirical distribution F of
  * Algorithm 1 -- seconds to microsecond ticks (nearest, ties to even), then an ascending sort -- for ONE
  * group of at most DISCO_NOALLOC_MAX_N requests.  Input and output are the caller's device arrays
- * (server_ttft_s[n] in, sorted_ticks[n] out); the sort's working memory is a fixed array of about 4.3 MB
+ * (server_ttft_s[n] in, sorted_ticks[n] out); the sort's working memory is a fixed array of about 4.5 MB
  * that is part of the library image, so it occupies that much memory on every GPU the library is loaded
  * on, from load until the process exits.  The call makes no cudaMalloc, cudaFree or other allocating
  * call.  It returns the same ticks, in the same order, as disco_load_trace followed by

@@ -164,12 +164,12 @@ cudaError_t reserve_trace(disco_ctx* c, uint32_t n, bool host_inputs, bool has_s
     const size_t cnt_bytes = ((size_t)G * (kMaxPrompt + 1) * 4 + 15) / 16 * 16;
     const size_t counts_bytes = (size_t)256 * kRadixMaxBlocks * 4;
     const size_t head = cnt_bytes + kMaxGroups * 8 + kMaxGroups * 4 + 16 + 16;
-    R(zero, head + 2 * counts_bytes);
+    R(zero, head + 5 * counts_bytes);
     char* z = (char*)c->zero.p;
     c->cnt = (uint32_t*)z; c->grp_sum_n = (uint64_t*)(z + cnt_bytes); c->ng = (uint32_t*)(z + cnt_bytes + kMaxGroups * 8);
     c->max_n = (uint32_t*)(z + cnt_bytes + kMaxGroups * 12); c->err = (int32_t*)(z + cnt_bytes + kMaxGroups * 12 + 16);
     c->radix_counts = (uint32_t*)(z + head);
-    c->zero_bytes = head + counts_bytes;
+    c->zero_bytes = head;
     R(cum_mass, (size_t)G * (kMaxPrompt + 2) * 8); R(ng_exact, kMaxGroups * 4);
     R(grp_off, (kMaxGroups + 1) * 4); R(knots, (size_t)G * kNKnots * 4);
     R(d_rb, sizeof(LoadReadback)); R(d_gc, (size_t)G * sizeof(GroupConst));

@@ -3,6 +3,7 @@
 // Algorithm 1), cumulative input-token mass (Eq. 3) and the quantile knots of F.
 #include "load.cuh"
 
+#include <algorithm>
 #include <mutex>
 
 namespace disco {
@@ -24,38 +25,54 @@ __global__ void k_ingest(uint32_t n, const int32_t* __restrict__ prompt, const i
     __shared__ unsigned long long s_sum[kMaxGroups];
     __shared__ uint32_t s_cnt[kMaxGroups];
     __shared__ uint32_t s_max;
+    __shared__ uint32_t s_len[kMaxPrompt + 1];       // length histogram of this block (single-group traces)
     const int G = (int)(ns * nd);
+    const bool one = G == 1;
     for (int g = threadIdx.x; g < G; g += blockDim.x) { s_sum[g] = 0; s_cnt[g] = 0; }
+    if (one) for (int i = threadIdx.x; i <= kMaxPrompt; i += blockDim.x) s_len[i] = 0;
     if (threadIdx.x == 0) s_max = 0;
     __syncthreads();
-    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
-        const int32_t l = prompt[i], o = outlen[i];
-        const float t = ttft[i];
-        const uint32_t s = sp ? sp[i] : 0u, d = dp ? dp[i] : 0u;
+    const uint32_t stride = gridDim.x * blockDim.x;
+    for (uint32_t i0 = blockIdx.x * blockDim.x; i0 < n; i0 += stride) {       // whole warps iterate together
+        const uint32_t i = i0 + threadIdx.x;
+        const bool in = i < n;
+        const int32_t l = in ? prompt[i] : 1, o = in ? outlen[i] : 1;
+        const float t = in ? ttft[i] : 1.0f;
+        const uint32_t s = (in && sp) ? sp[i] : 0u, d = (in && dp) ? dp[i] : 0u;
         int bad = 0;
         if (l < 1 || l > kMaxPrompt) bad = 1;
         else if (o < 1 || o > kMaxOutput) bad = 2;
         else if (!(t > 0.0f) || !(t <= 2000.0f)) bad = 3;      // NaN fails both comparisons
         else if (s >= ns || d >= nd) bad = 4;
-        if (bad) {
+        const bool ok = in && !bad;
+        if (in && bad) {
             if (atomicCAS(&err[0], 0, bad) == 0) err[1] = (int32_t)i;
             keys[i] = 0;
-            continue;
         }
         // ticks = nearest integer (ties to even) of the fp64 product, as a host llrint would give
         const long long S = __double2ll_rn(__dmul_rn((double)t, 1e6));
-        const uint32_t g = s * nd + d;
-        keys[i] = ((uint64_t)g << 32) | (uint32_t)S;
-        atomicAdd(&cnt[g * (kMaxPrompt + 1) + l], 1u);
-        atomicAdd(&s_sum[g], (unsigned long long)o);
-        atomicAdd(&s_cnt[g], 1u);
-        atomicMax(&s_max, (uint32_t)o);
-        if (S_out) { S_out[i] = (int32_t)S; l_out[i] = (uint16_t)l; n_out[i] = (uint16_t)o; orig_out[i] = i; }
-        if (counts0) atomicAdd(&counts0[((uint32_t)S & 255u) * blocks0 + i / per_block0], 1u);
+        const uint32_t g = ok ? s * nd + d : 0u;
+        if (ok) {
+            keys[i] = ((uint64_t)g << 32) | (uint32_t)S;
+            if (one) atomicAdd(&s_len[l], 1u); else atomicAdd(&cnt[g * (kMaxPrompt + 1) + l], 1u);
+            if (S_out) { S_out[i] = (int32_t)S; l_out[i] = (uint16_t)l; n_out[i] = (uint16_t)o; orig_out[i] = i; }
+            if (counts0) atomicAdd(&counts0[((uint32_t)S & 255u) * blocks0 + i / per_block0], 1u);
+        }
+        if (one) {                                             // one group: sums by warp reduction
+            const uint32_t so = __reduce_add_sync(0xFFFFFFFFu, ok ? (uint32_t)o : 0u);
+            const uint32_t mo = __reduce_max_sync(0xFFFFFFFFu, ok ? (uint32_t)o : 0u);
+            const uint32_t co = __popc(__ballot_sync(0xFFFFFFFFu, ok));
+            if ((threadIdx.x & 31) == 0 && co) {
+                atomicAdd(&s_sum[0], (unsigned long long)so); atomicAdd(&s_cnt[0], co); atomicMax(&s_max, mo);
+            }
+        } else if (ok) {
+            atomicAdd(&s_sum[g], (unsigned long long)o); atomicAdd(&s_cnt[g], 1u); atomicMax(&s_max, (uint32_t)o);
+        }
     }
     __syncthreads();
     for (int g = threadIdx.x; g < G; g += blockDim.x)
         if (s_cnt[g]) { atomicAdd(&grp_sum_n[g], s_sum[g]); atomicAdd(&grp_n[g], s_cnt[g]); }
+    if (one) for (int i = threadIdx.x; i <= kMaxPrompt; i += blockDim.x) if (s_len[i]) atomicAdd(&cnt[i], s_len[i]);
     if (threadIdx.x == 0 && s_max) atomicMax(max_n, s_max);
 }
 
@@ -98,11 +115,31 @@ __global__ void k_scan_counts(uint32_t* __restrict__ counts, uint32_t m, uint32_
 __global__ void k_radix_scatter(const uint64_t* __restrict__ keys_in, uint64_t* __restrict__ keys_out,
                                 const uint32_t* __restrict__ pay_in, uint32_t* __restrict__ pay_out, uint32_t n,
                                 uint32_t per_block, int shift, const uint32_t* __restrict__ offsets,
-                                uint32_t* __restrict__ counts_next = nullptr, int32_t* __restrict__ low_out = nullptr) {
+                                uint32_t* __restrict__ counts_next = nullptr, int32_t* __restrict__ low_out = nullptr,
+                                bool raw = false) {
     __shared__ uint32_t run[256];                 // next output slot of each digit for this block
     __shared__ uint32_t wcnt[kRadixWarps][256];   // keys of each digit per warp in the current slab
     const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    run[threadIdx.x] = offsets[threadIdx.x * gridDim.x + blockIdx.x];
+    if (!raw) {
+        run[threadIdx.x] = offsets[threadIdx.x * gridDim.x + blockIdx.x];
+    } else {
+        // `offsets` holds plain counts [digit][block]: this block's slots start after every key of a smaller
+        // digit and after the keys of the same digit in earlier blocks
+        const uint32_t* row = offsets + threadIdx.x * gridDim.x;
+        uint32_t total = 0, before = 0;
+        for (uint32_t b = 0; b < gridDim.x; ++b) { const uint32_t c = row[b]; total += c; before += b < blockIdx.x ? c : 0u; }
+        uint32_t* tot = wcnt[0];
+        tot[threadIdx.x] = total;
+        __syncthreads();
+        for (int off = 1; off < 256; off <<= 1) {
+            const uint32_t v = (int)threadIdx.x >= off ? tot[threadIdx.x - off] : 0u;
+            __syncthreads();
+            tot[threadIdx.x] += v;
+            __syncthreads();
+        }
+        run[threadIdx.x] = tot[threadIdx.x] - total + before;
+        __syncthreads();
+    }
     const uint32_t lo = min(n, blockIdx.x * per_block), hi = min(n, lo + per_block);
     for (uint32_t base = lo; base < hi; base += kRadixThreads) {
         for (int k = 0; k < kRadixWarps; ++k) wcnt[k][threadIdx.x] = 0;
@@ -214,7 +251,7 @@ int grid_for(uint32_t n, int threads) {
 
 cudaError_t radix_pass(const uint64_t* kin, uint64_t* kout, const uint32_t* pin, uint32_t* pout, uint32_t n,
                        int shift, uint32_t* counts, cudaStream_t st) {
-    uint32_t blocks = (n + 4095u) / 4096u;
+    uint32_t blocks = (n + 1023u) / 1024u;
     if (blocks < 1) blocks = 1;
     if (blocks > kRadixMaxBlocks) blocks = kRadixMaxBlocks;
     uint32_t per_block = (n + blocks - 1) / blocks;
@@ -229,7 +266,7 @@ cudaError_t radix_pass(const uint64_t* kin, uint64_t* kout, const uint32_t* pin,
 
 uint32_t load_kernel_launches(uint32_t n, int G) {
     if (n == 0) return 2;
-    if (G == 1 && n <= (1u << 20)) return 1 + 2 * 4 + 2;     // ingest, (scan, scatter) x 4, group tables
+    if (G == 1 && n <= (1u << 20)) return 1 + 4 + 2;         // ingest, four scatter passes, group tables
     const uint32_t passes = G > 1 ? 6 : 4;                  // radix passes: partition + 5, or 4
     return 1 + (G > 1 ? 1 : 0) + 3 * passes + 1 + 2;         // ingest, gather, passes, low words, group tables
 }
@@ -239,18 +276,19 @@ cudaError_t run_load(const LoadArgs& a, cudaStream_t st) {
     const int G = (int)(a.ns * a.nd);
     cudaError_t e;
     // radix geometry (as in radix_pass)
-    uint32_t blocks = (n + 4095u) / 4096u;
+    uint32_t blocks = (n + 1023u) / 1024u;
     if (blocks < 1) blocks = 1;
     if (blocks > kRadixMaxBlocks) blocks = kRadixMaxBlocks;
     uint32_t per_block = (n + blocks - 1) / blocks;
     per_block = (per_block + kRadixThreads - 1) / kRadixThreads * kRadixThreads;
     const bool small = G == 1 && n <= (1u << 20);      // fused histograms pay off while launches dominate
     // everything that must start at zero lies in one block: cnt, grp_sum_n, grp_n, max_n, err, counts A
-    if ((e = cudaMemsetAsync(a.zero_block, 0, a.zero_bytes, st))) return e;
+    // (zero_bytes covers the tables; the per-pass digit counters of the small path follow them)
+    if ((e = cudaMemsetAsync(a.zero_block, 0, a.zero_bytes + (small ? (size_t)5 * 256u * blocks * 4u : 0u), st))) return e;
     if (n) {
-        uint32_t* counts_a = a.radix_counts;
-        uint32_t* counts_b = a.radix_counts + 256u * kRadixMaxBlocks;
-        k_ingest<<<grid_for(n, kIngestThreads), kIngestThreads, 0, st>>>(
+        uint32_t* counts_a = a.radix_counts;                                   // small path: pass p uses slice p
+        uint32_t* counts_b = a.radix_counts + (size_t)4 * 256u * kRadixMaxBlocks;  // large path: one scanned buffer
+        k_ingest<<<std::min(grid_for(n, 4 * kIngestThreads), 296), kIngestThreads, 0, st>>>(
             n, a.prompt, a.outlen, a.ttft, a.sp, a.dp, a.ns, a.nd, a.keys_a, a.cnt,
             (unsigned long long*)a.grp_sum_n, a.ng, a.max_n, a.err,
             G == 1 ? a.S : nullptr, a.l, a.nout, a.orig, small ? counts_a : nullptr, per_block, blocks);
@@ -263,14 +301,13 @@ cudaError_t run_load(const LoadArgs& a, cudaStream_t st) {
         uint64_t *src = a.keys_a, *dst = a.keys_b;
         const int passes = G > 1 ? 5 : 4;
         if (small) {
-            uint32_t *cur = counts_a, *nxt = counts_b;
-            for (int p = 0; p < passes; ++p) {
+            for (int p = 0; p < passes; ++p) {                  // one launch per pass: no separate scan
                 const bool last = p == passes - 1;
-                k_scan_counts<<<1, 1024, 0, st>>>(cur, 256u * blocks, last ? nullptr : nxt);
+                uint32_t* cur = a.radix_counts + (size_t)p * 256u * blocks;
                 k_radix_scatter<<<blocks, kRadixThreads, 0, st>>>(src, dst, nullptr, nullptr, n, per_block, 8 * p, cur,
-                                                                  last ? nullptr : nxt, last ? a.sorted : nullptr);
+                                                                  last ? nullptr : cur + 256u * blocks,
+                                                                  last ? a.sorted : nullptr, true);
                 uint64_t* t = src; src = dst; dst = t;
-                uint32_t* c = cur; cur = nxt; nxt = c;
             }
         } else {
             for (int p = 0; p < passes; ++p) {
@@ -300,7 +337,7 @@ namespace {
 
 constexpr uint32_t kNoAllocMaxN = DISCO_NOALLOC_MAX_N;
 constexpr size_t kNaKeysBytes = (size_t)kNoAllocMaxN * sizeof(uint64_t);
-constexpr size_t kNaCountsBytes = 256u * ((kNoAllocMaxN + 4095u) / 4096u) * sizeof(uint32_t);
+constexpr size_t kNaCountsBytes = 256u * ((kNoAllocMaxN + 1023u) / 1024u) * sizeof(uint32_t);   // as radix_pass sizes its grid
 constexpr size_t kNaErrOff = 2 * kNaKeysBytes + kNaCountsBytes;
 
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNaErrOff + 256];

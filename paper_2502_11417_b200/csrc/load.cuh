@@ -25,8 +25,8 @@ struct LoadArgs {
     // scratch
     uint64_t *keys_a, *keys_b;            // [n] (group << 32 | ticks)
     uint32_t* tmp_idx;                    // [n]
-    uint32_t* radix_counts;               // [2][256 * kRadixMaxBlocks]; the first half lies in zero_block
-    void* zero_block; size_t zero_bytes;  // cnt, grp_sum_n, ng, max_n, err and the first counter buffer, contiguous
+    uint32_t* radix_counts;               // [5][256 * kRadixMaxBlocks], directly after zero_block's tables
+    void* zero_block; size_t zero_bytes;  // cnt, grp_sum_n, ng, max_n, err, contiguous
     uint32_t* ng_exact;                   // [G] group sizes recounted from the length histogram
     LoadReadback* readback;               // device copy of what the host reads back
     // outputs
