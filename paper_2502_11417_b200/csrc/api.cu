@@ -74,7 +74,7 @@ struct disco_ctx {
     uint32_t P = 0;
     bool evaluated = false, reduced = false;
     std::vector<PolicyConst> pol;
-    DevBuf d_prep, d_accum, d_stats, d_tables, d_select;
+    DevBuf d_prep, d_accum, d_stats, d_tables, d_select, d_todo;
     struct View { void* p = nullptr; template <class T> T* as() const { return (T*)p; } };
     View d_acc, d_hist_ttft, d_hist_tbt;               // three regions of d_accum (cleared by one memset)
     View d_pol, d_classes, d_pol_list, d_chunks;       // four regions of d_tables (filled by one copy)
@@ -92,7 +92,7 @@ struct disco_ctx {
 
     ~disco_ctx() {
         DevBuf* all[] = {&in_prompt, &in_out, &in_ttft, &in_sp, &in_dp, &keys_a, &keys_b, &tmp_idx,
-                         &S, &l, &nout, &orig, &sorted, &zero, &cum_mass, &ng_exact, &grp_off, &knots, &d_rb, &d_gc, &d_prep, &d_accum, &d_stats, &d_tables, &d_select};
+                         &S, &l, &nout, &orig, &sorted, &zero, &cum_mass, &ng_exact, &grp_off, &knots, &d_rb, &d_gc, &d_prep, &d_accum, &d_stats, &d_tables, &d_select, &d_todo};
         for (DevBuf* b : all) b->release();
         for (auto& b : rec_u32) b.release();
         for (auto& b : rec_u16) b.release();
@@ -337,7 +337,9 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
 #define R(buf, bytes) if ((e = c->buf.reserve(bytes)) != cudaSuccess) return fail_cuda(e, "device allocation for the evaluation")
     R(d_prep, (size_t)G * P * sizeof(Prep));
     const size_t acc_bytes = (size_t)P * G * kNAcc * 8, hist_bytes = (size_t)P * kNBins * 8;
-    R(d_accum, acc_bytes + 2 * hist_bytes);
+    const size_t cnt_bytes = (classes.size() * 4 + 15) / 16 * 16;        // one to-do counter per class
+    R(d_accum, acc_bytes + 2 * hist_bytes + cnt_bytes);
+    R(d_todo, N1 * 4);
     c->d_acc.p = c->d_accum.p; c->d_hist_ttft.p = (char*)c->d_accum.p + acc_bytes;
     c->d_hist_tbt.p = (char*)c->d_accum.p + acc_bytes + hist_bytes;
     R(d_stats, P * sizeof(disco_policy_stats_t) + 16); R(d_select, 8);
@@ -396,7 +398,8 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
     CU(cudaMemcpyAsync(dt, sp, off, cudaMemcpyHostToDevice, st));
     CU(cudaEventRecord(c->stage_free, st));
 
-    CU(cudaMemsetAsync(c->d_accum.p, 0, acc_bytes + 2 * hist_bytes, st));
+    CU(cudaMemsetAsync(c->d_accum.p, 0, acc_bytes + 2 * hist_bytes + cnt_bytes, st));
+    uint32_t* todo_counts = (uint32_t*)((char*)c->d_accum.p + acc_bytes + 2 * hist_bytes);
 
     // ---- Algorithms 1-3 for every (group, policy)
     CU(launch_prep(c->d_pol.as<PolicyConst>(), P, G, c->d_gc.as<GroupConst>(), c->cum_mass.as<int64_t>(),
@@ -423,14 +426,15 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
     for (size_t k = 0; k < classes.size(); ++k) {
         const ClassConst* dcc = c->d_classes.as<ClassConst>() + k;
         if (timed) CU(cudaEventRecord(c->ev[0], st));
-        CU(launch_timeline(tr, c->d_gc.as<GroupConst>(), dcc, c->knots.as<int32_t>(), seed, rec, c->err, st));
+        CU(launch_timeline(tr, c->d_gc.as<GroupConst>(), dcc, classes[k].pacing != 0, c->knots.as<int32_t>(), seed, rec,
+                           c->err, c->d_todo.as<uint32_t>(), todo_counts + k, st));
         if (timed) CU(cudaEventRecord(c->ev[1], st));
         CU(launch_pairs(tr, c->d_gc.as<GroupConst>(), dcc, c->d_prep.as<Prep>(), P,
                         c->d_pol_list.as<uint32_t>() + cls_range[k].first, cls_range[k].second - cls_range[k].first,
                         c->d_chunks.as<Chunk>(), (uint32_t)chunks.size(), rec, po, c->d_acc.as<uint64_t>(),
                         c->d_hist_ttft.as<uint64_t>(), c->d_hist_tbt.as<uint64_t>(), st));
         if (timed) CU(cudaEventRecord(c->ev[2], st));
-        g_launches += (n ? 1 : 0) + ((n && !chunks.empty()) ? (out ? 2 : 1) : 0);
+        g_launches += (n ? (classes[k].pacing ? 2 : 1) : 0) + ((n && !chunks.empty()) ? (out ? 2 : 1) : 0);
     }
     c->timing_valid = timed && n != 0;
     c->P = P; c->pol = pc;

@@ -121,8 +121,9 @@ int set_error(int code, const char* msg);
 cudaError_t launch_prep(const PolicyConst* pol, uint32_t P, int G, const GroupConst* gc, const int64_t* cum_mass,
                         const uint32_t* cnt, const int32_t* sorted, const uint32_t* grp_off, Prep* prep,
                         cudaStream_t st);
-cudaError_t launch_timeline(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const int32_t* knots,
-                            uint64_t seed, TimelineRec rec, int32_t* err, cudaStream_t st);
+cudaError_t launch_timeline(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, bool pacing,
+                            const int32_t* knots, uint64_t seed, TimelineRec rec, int32_t* err, uint32_t* todo,
+                            uint32_t* todo_count /* zero on entry */, cudaStream_t st);
 cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const Prep* prep, uint32_t P,
                          const uint32_t* pol_list, uint32_t n_list, const Chunk* chunks, uint32_t n_chunks,
                          TimelineRec rec, disco_pair_out_t out, uint64_t* acc, uint64_t* hist_ttft,

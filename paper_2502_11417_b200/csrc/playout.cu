@@ -16,6 +16,7 @@
 //
 // A warp takes 32 consecutive requests at a time: their inputs are loaded and their results stored one
 // request per lane, so the per-request memory traffic is coalesced and paid once per 32 requests.
+#include <algorithm>
 #include <climits>
 
 #include "disco_internal.cuh"
@@ -283,12 +284,14 @@ __device__ __noinline__ void play_x(const GroupClass& G, Round rd, uint32_t key,
 
 __global__ void __launch_bounds__(kWarps * 32)
 k_playout(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __restrict__ ccp,
-          const int32_t* __restrict__ knots, uint32_t k0, TimelineRec rec, int32_t* err) {
+          const int32_t* __restrict__ knots, uint32_t k0, TimelineRec rec, int32_t* err,
+          const uint32_t* __restrict__ todo, const uint32_t* __restrict__ todo_count, uint32_t count_imm) {
+    // Requests to play: todo[0 .. *todo_count), or 0 .. count_imm when there is no list.
     __shared__ uint32_t ring_s[kWarps][kRing];
     __shared__ XResult xres_s[kWarps];
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
-    const uint32_t batch0 = (blockIdx.x * kWarps + wib) * 32u;
-    if (batch0 >= tr.n) return;
+    const uint32_t count = todo_count ? *todo_count : count_imm;
+    for (uint32_t batch0 = (blockIdx.x * kWarps + wib) * 32u; batch0 < count; batch0 += gridDim.x * kWarps * 32u) {
     uint32_t* ring = ring_s[wib];
     const ClassConst& cc = *ccp;
     const int32_t tau_eff = cc.tau_eff, tau = cc.tau;
@@ -299,8 +302,8 @@ k_playout(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __r
     const int32_t thr = thr64 > INT_MAX ? INT_MAX : (int32_t)thr64;
 
     // ---- one request per lane: inputs
-    const uint32_t kk = batch0 + lane;
-    const bool live = kk < tr.n;
+    const bool live = batch0 + lane < count;
+    const uint32_t kk = !live ? 0u : (todo ? todo[batch0 + lane] : batch0 + lane);
     uint32_t n_l = 1, l_l = 1, key_l = 0;
     int g_l = 0;
     if (live) {
@@ -320,13 +323,13 @@ k_playout(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __r
     int cur_g = -1;
     Round rd;
     rd.lane = lane; rd.tau_eff = tau_eff; rd.pacing = pacing; rd.err = err;
-    const int n_here = (int)min(32u, tr.n - batch0);
+    const int n_here = (int)min(32u, count - batch0);
 
     for (int r = 0; r < n_here; ++r) {
         const uint32_t n = __shfl_sync(FULL, n_l, r), l = __shfl_sync(FULL, l_l, r);
         const uint32_t key = __shfl_sync(FULL, key_l, r);
         const int g = __shfl_sync(FULL, g_l, r);
-        const uint32_t k = batch0 + r;
+        const uint32_t k = __shfl_sync(FULL, kk, r);
         if (g != cur_g) {
             cur_g = g;
             const GroupConst& gc = gcs[g];
@@ -498,15 +501,31 @@ k_playout(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __r
         if (kt1 >= 0 && o_ntD) rec.win[1][(size_t)kk * W1 + kt1] += o_ntD;
         if (kt2 >= 0 && o_ntX) rec.win[2][(size_t)kk * W2 + kt2] += o_ntX;
     }
+    __syncwarp();
+    }   // next batch
 }
 
 }  // namespace
 
-cudaError_t launch_timeline(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const int32_t* knots,
-                            uint64_t seed, TimelineRec rec, int32_t* err, cudaStream_t st) {
+cudaError_t launch_playout_fast(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const int32_t* knots,
+                                uint64_t seed, TimelineRec rec, uint32_t* todo, uint32_t* todo_count, cudaStream_t st);
+
+// pacing: with the delivery buffer on, the clamp-free kernel plays every request it can and lists the rest
+// in todo[0 .. *todo_count) (todo_count must be zero on entry); the general kernel then plays the list.
+cudaError_t launch_timeline(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, bool pacing,
+                            const int32_t* knots, uint64_t seed, TimelineRec rec, int32_t* err, uint32_t* todo,
+                            uint32_t* todo_count, cudaStream_t st) {
     if (tr.n == 0) return cudaSuccess;
     const uint32_t per_block = kWarps * 32;
-    k_playout<<<(tr.n + per_block - 1) / per_block, kWarps * 32, 0, st>>>(tr, gc, cc, knots, seed_key(seed), rec, err);
+    if (!pacing) {
+        const uint32_t blocks = std::min<uint32_t>((tr.n + per_block - 1) / per_block, 148u * 16u);
+        k_playout<<<blocks, kWarps * 32, 0, st>>>(tr, gc, cc, knots, seed_key(seed), rec, err, nullptr, nullptr, tr.n);
+        return cudaGetLastError();
+    }
+    cudaError_t e = launch_playout_fast(tr, gc, cc, knots, seed, rec, todo, todo_count, st);
+    if (e) return e;
+    const uint32_t blocks = std::min<uint32_t>((tr.n + per_block - 1) / per_block, 148u * 2u);
+    k_playout<<<blocks, kWarps * 32, 0, st>>>(tr, gc, cc, knots, seed_key(seed), rec, err, todo, todo_count, 0u);
     return cudaGetLastError();
 }
 
