@@ -29,13 +29,17 @@ METRIC = "request-policy evaluations/s"
 UNIT = "pairs/s"
 PAIR_OUT_BYTES = 31          # four fp32, three u32, one u16, one u8 per pair
 TRACE_BYTES = 9              # packed request: ticks, prompt, output length, group
-# Lane-instructions a token-step needs for the three streams that share one hash draw:
-# hash 10, two range maps 4, three Lindley steps of 6 (subtract, max, subtract, add, max, compare-count).
-PLAYOUT_INSTR_PER_TOKEN = 32
+# Lane-instructions one token-step of the play-out needs (both endpoints' streams share the hash draw):
+# counter add 1, hash finaliser 8, two range maps (multiply-high) 2, tail mask 1, two sums and two maxima 4,
+# loop 1.
+PLAYOUT_INSTR_PER_TOKEN = 17
+# Lane-instructions one (request, policy) pair needs in the reduction kernel: wait map and race 12,
+# trigger 4, tokens and prefill 10, ten running sums 10, TTFT bin and histogram update 6.
+PAIR_INSTR = 42
 SM_COUNT, SCHEDULERS, LANES = 148, 4, 32
 # DRAM bytes per launch from the committed ncu capture of the dominant kernel (None until captured for
 # the current kernel; see profiles/).
-NCU_TRAFFIC_BYTES = {"pairs": None, "playout": None}
+NCU_TRAFFIC_BYTES = {"k_pairs_rows": None, "k_pairs_acc": None, "k_playout_fast": None, "k_playout": None}
 
 
 def env_rank():
@@ -62,7 +66,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
-                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -237,23 +241,30 @@ def run_ours(args):
 
     # ---- roofline of the dominant kernel of a step
     hbm_gbs, sm_max_mhz, src = measured_peaks()
-    play_ms = statistics.mean(t[0] for t in ktimes)
-    pair_ms = statistics.mean(t[1] for t in ktimes)
+    names = ["k_playout_fast", "k_playout", "k_pairs_acc", "k_pairs_rows"]
+    kms = {nm: statistics.mean(t[i] for t in ktimes) for i, nm in enumerate(names)}
     token_steps = int((w.output_len - 1).sum())
-    if pair_ms >= play_ms:
-        bytes_alg = n * P * (PAIR_OUT_BYTES if w.materialise else 0) + n * TRACE_BYTES
-        ach = bytes_alg / (pair_ms * 1e-3) / 1e9
-        roof = {"kernel": "k_pairs", "bound": "hbm", "achieved": ach, "peak": hbm_gbs, "unit": "GB/s",
-                "frac": ach / hbm_gbs, "traffic": NCU_TRAFFIC_BYTES["pairs"], "peak_source": src,
-                "algorithmic_bytes": bytes_alg, "ms_per_launch": pair_ms}
+    top = max(kms, key=kms.get)
+    alu_peak = SM_COUNT * SCHEDULERS * LANES * sm_max_mhz * 1e6 / 1e12         # T lane-instructions/s
+    alu_src = "148 SMs x 4 schedulers x 32 lanes x %.0f MHz (issue slots)" % sm_max_mhz
+    if top == "k_pairs_rows":
+        bytes_alg = n * P * PAIR_OUT_BYTES + n * TRACE_BYTES
+        ach = bytes_alg / (kms[top] * 1e-3) / 1e9
+        roof = {"kernel": top, "bound": "hbm", "achieved": ach, "peak": hbm_gbs, "unit": "GB/s",
+                "frac": ach / hbm_gbs, "traffic": NCU_TRAFFIC_BYTES[top], "peak_source": src,
+                "algorithmic_bytes": bytes_alg}
+    elif top == "k_pairs_acc":
+        ach = n * P * PAIR_INSTR / (kms[top] * 1e-3) / 1e12
+        roof = {"kernel": top, "bound": "alu", "achieved": ach, "peak": alu_peak, "unit": "Tinstr/s",
+                "frac": ach / alu_peak, "traffic": NCU_TRAFFIC_BYTES[top], "peak_source": alu_src,
+                "instr_per_pair": PAIR_INSTR}
     else:
-        peak = SM_COUNT * SCHEDULERS * LANES * sm_max_mhz * 1e6 / 1e12     # T lane-instructions/s
-        ach = token_steps * PLAYOUT_INSTR_PER_TOKEN / (play_ms * 1e-3) / 1e12
-        roof = {"kernel": "k_timeline", "bound": "alu", "achieved": ach, "peak": peak, "unit": "Tinstr/s",
-                "frac": ach / peak, "traffic": NCU_TRAFFIC_BYTES["playout"],
-                "peak_source": "148 SMs x 4 schedulers x 32 lanes x %.0f MHz" % sm_max_mhz,
-                "token_steps": token_steps, "ms_per_launch": play_ms}
-    roof["other_kernels_ms"] = {"k_timeline": play_ms, "k_pairs": pair_ms}
+        ach = token_steps * PLAYOUT_INSTR_PER_TOKEN / (kms[top] * 1e-3) / 1e12
+        roof = {"kernel": top, "bound": "alu", "achieved": ach, "peak": alu_peak, "unit": "Tinstr/s",
+                "frac": ach / alu_peak, "traffic": NCU_TRAFFIC_BYTES[top], "peak_source": alu_src,
+                "token_steps": token_steps, "instr_per_token_step": PLAYOUT_INSTR_PER_TOKEN}
+    roof["ms_per_launch"] = kms[top]
+    roof["kernels_ms"] = kms
 
     if rank != 0:
         if dist is not None:
@@ -288,7 +299,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=1, help="workload 0..4 (default: workload 1)")
     ap.add_argument("--requests", type=int, default=None, help="shrink the trace (profiling on a small case)")

@@ -173,11 +173,12 @@ int64_t disco_get_group_tables(disco_ctx_t* ctx, uint32_t g, int64_t* cnt, int32
                                int32_t* sorted_ticks, uint64_t n_sorted, void* stream);
 
 /* Measurement aids.  disco_set_timing(ctx, 1) makes each evaluation record CUDA events on its stream around
- * the play-out kernel and the pair kernel; after disco_reduce_stats, disco_get_timing returns their device
- * durations in milliseconds (only for evaluations whose policies share one pacing / buffer setting).
- * disco_kernel_launch_count returns how many kernels this library has launched in this process. */
+ * its four main kernels; after disco_reduce_stats, disco_get_timing fills ms4[0..3] with the device
+ * durations in milliseconds of: the play-out of clamp-free requests, the general play-out, the pair
+ * reductions, the per-pair row writer (only for evaluations whose policies share one pacing / buffer
+ * setting).  disco_kernel_launch_count returns how many kernels this library has launched in this process. */
 int disco_set_timing(disco_ctx_t* ctx, int on);
-int disco_get_timing(disco_ctx_t* ctx, float* playout_ms, float* pairs_ms);
+int disco_get_timing(disco_ctx_t* ctx, float* ms4);
 uint64_t disco_kernel_launch_count(void);
 
 /* Sorting without allocating.  (The paper has no counterpart to this call; it exists for the sake of

@@ -107,7 +107,7 @@ def lib() -> C.CDLL:
         L.disco_last_error.restype = C.c_char_p
         L.disco_set_timing.restype = C.c_int; L.disco_set_timing.argtypes = [vp, C.c_int]
         L.disco_get_timing.restype = C.c_int
-        L.disco_get_timing.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_float)]
+        L.disco_get_timing.argtypes = [vp, C.POINTER(C.c_float)]
         L.disco_kernel_launch_count.restype = u64; L.disco_kernel_launch_count.argtypes = []
         L.disco_sort_ttft_ticks_noalloc.restype = C.c_int
         L.disco_sort_ttft_ticks_noalloc.argtypes = [vp, u32, vp, vp]
@@ -305,10 +305,11 @@ class Trace:
         _check(lib().disco_set_timing(self._h, int(on)))
 
     def timing(self):
-        """(play-out ms, pair-kernel ms) of the last reduced evaluation."""
-        a, b = C.c_float(), C.c_float()
-        _check(lib().disco_get_timing(self._h, C.byref(a), C.byref(b)))
-        return a.value, b.value
+        """Device milliseconds of the last reduced evaluation's kernels:
+        (clamp-free play-out, general play-out, pair reductions, per-pair rows)."""
+        ms = (C.c_float * 4)()
+        _check(lib().disco_get_timing(self._h, ms))
+        return tuple(ms)
 
     def close(self):
         if self._h:

@@ -86,8 +86,8 @@ struct disco_ctx {
     void* stats_host = nullptr;  // pinned mirror of the statistics
     size_t stats_host_cap = 0;
     bool timing = false;         // record events around the play-out and pair kernels
-    cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
-    float ms_timeline = 0.f, ms_pairs = 0.f;
+    cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+    float ms[4] = {0.f, 0.f, 0.f, 0.f};   // clamp-free play-out, general play-out, pair reductions, pair rows
     bool timing_valid = false;
 
     ~disco_ctx() {
@@ -427,13 +427,13 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
         const ClassConst* dcc = c->d_classes.as<ClassConst>() + k;
         if (timed) CU(cudaEventRecord(c->ev[0], st));
         CU(launch_timeline(tr, c->d_gc.as<GroupConst>(), dcc, classes[k].pacing != 0, c->knots.as<int32_t>(), seed, rec,
-                           c->err, c->d_todo.as<uint32_t>(), todo_counts + k, st));
-        if (timed) CU(cudaEventRecord(c->ev[1], st));
+                           c->err, c->d_todo.as<uint32_t>(), todo_counts + k, timed ? c->ev[1] : nullptr, st));
+        if (timed) CU(cudaEventRecord(c->ev[2], st));
         CU(launch_pairs(tr, c->d_gc.as<GroupConst>(), dcc, c->d_prep.as<Prep>(), P,
                         c->d_pol_list.as<uint32_t>() + cls_range[k].first, cls_range[k].second - cls_range[k].first,
                         c->d_chunks.as<Chunk>(), (uint32_t)chunks.size(), rec, po, c->d_acc.as<uint64_t>(),
-                        c->d_hist_ttft.as<uint64_t>(), c->d_hist_tbt.as<uint64_t>(), st));
-        if (timed) CU(cudaEventRecord(c->ev[2], st));
+                        c->d_hist_ttft.as<uint64_t>(), c->d_hist_tbt.as<uint64_t>(), timed ? c->ev[3] : nullptr, st));
+        if (timed) CU(cudaEventRecord(c->ev[4], st));
         g_launches += (n ? (classes[k].pacing ? 2 : 1) : 0) + ((n && !chunks.empty()) ? (out ? 2 : 1) : 0);
     }
     c->timing_valid = timed && n != 0;
@@ -463,8 +463,7 @@ int disco_reduce_stats(disco_ctx_t* c, disco_policy_stats_t* stats, void* stream
     std::memcpy(c->rb->err, (char*)c->stats_host + c->P * sizeof(disco_policy_stats_t), 16);
     g_launches += 1;
     if (c->timing_valid) {
-        CU(cudaEventElapsedTime(&c->ms_timeline, c->ev[0], c->ev[1]));
-        CU(cudaEventElapsedTime(&c->ms_pairs, c->ev[1], c->ev[2]));
+        for (int k = 0; k < 4; ++k) CU(cudaEventElapsedTime(&c->ms[k], c->ev[k], c->ev[k + 1]));
     }
     if (c->rb->err[2]) return fail(DISCO_ECUDA, "internal error: an inter-token interval fell outside its histogram window");
     c->reduced = true;
@@ -495,10 +494,10 @@ int disco_set_timing(disco_ctx_t* c, int on) {
     return 0;
 }
 
-int disco_get_timing(disco_ctx_t* c, float* playout_ms, float* pairs_ms) {
-    if (!c || !playout_ms || !pairs_ms) return fail(DISCO_EINVAL, "null argument");
+int disco_get_timing(disco_ctx_t* c, float* ms4) {
+    if (!c || !ms4) return fail(DISCO_EINVAL, "null argument");
     if (!c->timing_valid || !c->reduced) return fail(DISCO_EINVAL, "no timed evaluation has been reduced");
-    *playout_ms = c->ms_timeline; *pairs_ms = c->ms_pairs;
+    for (int k = 0; k < 4; ++k) ms4[k] = c->ms[k];
     return 0;
 }
 

@@ -123,11 +123,13 @@ cudaError_t launch_prep(const PolicyConst* pol, uint32_t P, int G, const GroupCo
                         cudaStream_t st);
 cudaError_t launch_timeline(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, bool pacing,
                             const int32_t* knots, uint64_t seed, TimelineRec rec, int32_t* err, uint32_t* todo,
-                            uint32_t* todo_count /* zero on entry */, cudaStream_t st);
+                            uint32_t* todo_count /* zero on entry */, cudaEvent_t mid /* recorded between its two kernels, or null */,
+                            cudaStream_t st);
 cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const Prep* prep, uint32_t P,
                          const uint32_t* pol_list, uint32_t n_list, const Chunk* chunks, uint32_t n_chunks,
                          TimelineRec rec, disco_pair_out_t out, uint64_t* acc, uint64_t* hist_ttft,
-                         uint64_t* hist_tbt, cudaStream_t st);
+                         uint64_t* hist_tbt, cudaEvent_t mid /* recorded between its two kernels, or null */,
+                         cudaStream_t st);
 cudaError_t launch_finalize(uint32_t P, int G, const GroupConst* gc, const uint64_t* acc, const uint64_t* hist_ttft,
                             const uint64_t* hist_tbt, const uint64_t* grp_sum_n, const uint32_t* grp_off,
                             disco_policy_stats_t* stats /* [P] + 16 bytes */, const int32_t* err, cudaStream_t st);

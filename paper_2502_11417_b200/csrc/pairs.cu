@@ -236,8 +236,8 @@ k_pairs_rows(TraceDev tr, const GroupConst* __restrict__ gcs, const Prep* __rest
 cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const Prep* prep, uint32_t P,
                          const uint32_t* pol_list, uint32_t n_list, const Chunk* chunks, uint32_t n_chunks,
                          TimelineRec rec, disco_pair_out_t out, uint64_t* acc, uint64_t* hist_ttft,
-                         uint64_t* hist_tbt, cudaStream_t st) {
-    if (n_chunks == 0 || n_list == 0) return cudaSuccess;
+                         uint64_t* hist_tbt, cudaEvent_t mid, cudaStream_t st) {
+    if (n_chunks == 0 || n_list == 0) return mid ? cudaEventRecord(mid, st) : cudaSuccess;
     int PL = 1;
     while (PL < 32 && (uint32_t)PL < n_list) PL <<= 1;
     cudaError_t e = cudaFuncSetAttribute(k_pairs_acc, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -249,6 +249,7 @@ cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassCo
                                                                (unsigned long long*)hist_ttft,
                                                                (unsigned long long*)hist_tbt);
     if ((e = cudaGetLastError())) return e;
+    if (mid && (e = cudaEventRecord(mid, st))) return e;
     const bool rows = out.ttft_s || out.tbt_mean_s || out.tbt_max_s || out.cost || out.tok_server || out.tok_device ||
                       out.mig_at || out.delayed || out.decision;
     if (rows) {

@@ -1,8 +1,8 @@
 // Decode play-out (Sec. 4.3) for requests whose streams never clamp: both endpoints generate every token
 // no slower than it is consumed (c_j = tau - x_j >= 0 for all j), so delivery is exactly tau-paced.
 //
-// Teams of eight lanes play one request each, four requests per warp at a time; a lane owns a contiguous
-// run of tokens.  Every token's hash is drawn and mapped to both endpoints' jitter; the lane keeps the sums
+// A warp plays four requests at a time and shares its 32 lanes among them in proportion to their token
+// counts (every lane then owns a contiguous run of about the same length, whatever the mix of lengths).  Every token's hash is drawn and mapped to both endpoints' jitter; the lane keeps the sums
 // and maxima.  If any c_j is negative the request is put on a list for the general kernel (playout.cu).
 // Otherwise:
 //  * streams S and D: every TBT equals tau;
@@ -17,7 +17,7 @@ namespace disco {
 namespace {
 
 constexpr uint32_t FULL = 0xFFFFFFFFu;
-constexpr int kTeam = 8;
+constexpr int kPerIter = 4;               // requests a warp plays at a time
 constexpr int kFastWarps = 8;
 
 struct LaneGroup {                       // constants of a lane's current request group
@@ -27,18 +27,13 @@ struct LaneGroup {                       // constants of a lane's current reques
     const int32_t* K;
 };
 
+// Inclusive prefix sum over the lanes of a team (q = lane's position in its team); all 32 lanes call it.
 __device__ __forceinline__ int32_t team_inclusive_sum(int32_t v, int q) {
 #pragma unroll
-    for (int off = 1; off < kTeam; off <<= 1) {
-        const int32_t p = __shfl_up_sync(FULL, v, off, kTeam);
+    for (int off = 1; off < 32; off <<= 1) {
+        const int32_t p = __shfl_up_sync(FULL, v, off);
         if (q >= off) v += p;
     }
-    return v;
-}
-
-__device__ __forceinline__ uint32_t team_sum(uint32_t v, uint32_t tmask) {
-#pragma unroll
-    for (int off = 1; off < kTeam; off <<= 1) v += __shfl_xor_sync(tmask, v, off, kTeam);
     return v;
 }
 
@@ -60,14 +55,14 @@ __device__ __forceinline__ uint32_t walk(uint32_t key, uint32_t j0, int t0, int 
     return passed;
 }
 
+
+// rpw = requests per warp (4, 8, 16 or 32): small traces use small batches so that enough warps are in flight.
 __global__ void __launch_bounds__(kFastWarps * 32)
 k_playout_fast(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __restrict__ ccp,
                const int32_t* __restrict__ knots, uint32_t k0, TimelineRec rec, uint32_t* __restrict__ todo,
-               uint32_t* __restrict__ todo_count) {
+               uint32_t* __restrict__ todo_count, int rpw) {
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
-    const int team = lane >> 3, q = lane & 7;
-    const uint32_t tmask = 0xFFu << (team * kTeam);               // the lanes of this team: teams may diverge
-    const uint32_t batch0 = (blockIdx.x * kFastWarps + wib) * 32u;
+    const uint32_t batch0 = (blockIdx.x * kFastWarps + wib) * (uint32_t)rpw;
     if (batch0 >= tr.n) return;
     const ClassConst& cc = *ccp;
     const int32_t tau = cc.tau;                                   // pacing is on for every launch of this kernel
@@ -79,7 +74,7 @@ k_playout_fast(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst
 
     // ---- one request per lane: inputs
     const uint32_t kk = batch0 + lane;
-    const bool live = kk < tr.n;
+    const bool live = lane < rpw && kk < tr.n;
     uint32_t n_l = 1, l_l = 1, key_l = 0;
     int g_l = 0;
     if (live) {
@@ -87,20 +82,39 @@ k_playout_fast(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst
         key_l = mix32(k0 + tr.orig[kk] * kHashReq);
         while (g_l + 1 < tr.n_groups && kk >= tr.grp_off[g_l + 1]) ++g_l;
     }
-    // ---- one request per lane: results (request team*8 + it is kept by lane q == it of its team)
-    uint32_t o_sumX = 0, o_stall = 0, o_m = 0, o_dl = 0;
-    bool o_done = false;
+    // ---- one request per lane: results (bit 31 of o_md: played here; bits 0-15 m, 16-30 late tokens)
+    uint32_t o_md = 0, o_stall = 0;
 
     LaneGroup G;
     int cur_g = -1;
-    const int n_here = (int)min(32u, tr.n - batch0);
 
-    for (int it = 0; it < kTeam; ++it) {
-        const int r = team * kTeam + it;
+    for (int it = 0; it < rpw / kPerIter; ++it) {
+        // ---- share the lanes among the four requests in proportion to their intervals (n - 1 each)
+        const int r0 = it * kPerIter;
+        const uint32_t nI0 = __shfl_sync(FULL, n_l, r0) - 1, nI1 = __shfl_sync(FULL, n_l, r0 + 1) - 1;
+        const uint32_t nI2 = __shfl_sync(FULL, n_l, r0 + 2) - 1, nI3 = __shfl_sync(FULL, n_l, r0 + 3) - 1;
+        const uint32_t tot = nI0 + nI1 + nI2 + nI3;
+        int b1 = 0, b2 = 0, b3 = 0;                                // team i owns lanes [b_i, b_{i+1}), b0 = 0, b4 = 32
+        if (tot) {
+            b1 = (int)((32u * nI0 + tot / 2) / tot);
+            b2 = (int)((32u * (nI0 + nI1) + tot / 2) / tot);
+            b3 = (int)((32u * (nI0 + nI1 + nI2) + tot / 2) / tot);
+            b1 = max(b1, (int)(nI0 != 0));                         // a request with tokens gets at least one lane
+            b2 = max(b2, b1 + (int)(nI1 != 0));
+            b3 = max(b3, b2 + (int)(nI2 != 0));
+            b3 = min(b3, 32 - (int)(nI3 != 0));
+            b2 = min(b2, b3 - (int)(nI2 != 0));
+            b1 = min(b1, b2 - (int)(nI1 != 0));
+        }
+        const int team = (lane >= b1) + (lane >= b2) + (lane >= b3);
+        const int a = team == 0 ? 0 : (team == 1 ? b1 : (team == 2 ? b2 : b3));
+        const int a_next = team == 0 ? b1 : (team == 1 ? b2 : (team == 2 ? b3 : 32));
+        const int lanes = a_next - a, q = lane - a;
+        const uint32_t tmask = lanes == 32 ? FULL : (((1u << lanes) - 1u) << a);   // this team's lanes: teams may diverge
+        const int r = r0 + team;
         const uint32_t n = __shfl_sync(FULL, n_l, r), l = __shfl_sync(FULL, l_l, r);
         const uint32_t key = __shfl_sync(FULL, key_l, r);
         const int g = __shfl_sync(FULL, g_l, r);
-        const bool active = r < n_here;
         if (g != cur_g) {
             cur_g = g;
             const GroupConst& gc = gcs[g];
@@ -110,8 +124,8 @@ k_playout_fast(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst
             G.cand = mig_any ? gc.candidate : 0;
             G.K = knots + g * kNKnots;
         }
-        const uint32_t nI = active ? n - 1 : 0u;                   // inter-token intervals, tokens 2..n
-        const uint32_t L = (nI + kTeam - 1) / kTeam;               // tokens per lane
+        const uint32_t nI = tot ? n - 1 : 0u;                      // inter-token intervals, tokens 2..n
+        const uint32_t L = (nI + (uint32_t)lanes - 1) / (uint32_t)lanes;   // tokens per lane (lanes >= 1 here)
         const uint32_t lo = (uint32_t)q * L;
         const int cnt = lo >= nI ? 0 : (int)min(L, nI - lo);
         const uint32_t j0 = lo + 2;
@@ -125,17 +139,14 @@ k_playout_fast(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst
             uint32_t h = mix32(hin);
             hin += kHashTok;
             h = t < cnt ? h : 0u;
-            const uint32_t a = __umulhi(h, G.mulS), b = __umulhi(h, G.mulD);
-            hS += a; hD += b; xS = max(xS, a); xD = max(xD, b);
+            const uint32_t x = __umulhi(h, G.mulS), y = __umulhi(h, G.mulD);
+            hS += x; hD += y; xS = max(xS, x); xD = max(xD, y);
         }
         const int32_t s_S = cnt * G.cS_base - (int32_t)hS, s_D = cnt * G.cD_base - (int32_t)hD;
         const bool neg = cnt != 0 && ((int32_t)xS > G.cS_base || (int32_t)xD > G.cD_base);   // some c_j < 0
-        const uint32_t team_neg = (__ballot_sync(FULL, neg) >> (team * kTeam)) & 0xFFu;
-        const bool clean = team_neg == 0;
-        if (active && !clean) {                                    // leave it to the general kernel
-            if (q == 0) todo[atomicAdd(todo_count, 1u)] = batch0 + r;
-        }
-        const bool go = active && clean && nI != 0;
+        const bool clean = (__ballot_sync(FULL, neg) & tmask) == 0;
+        if (nI != 0 && !clean && q == 0) todo[atomicAdd(todo_count, 1u)] = batch0 + r;   // for the general kernel
+        const bool go = clean && nI != 0;
         // ---- hand-off index on the candidate stream
         const int cand = go ? G.cand : 0;
         const int32_t sC = cand == 1 ? s_S : s_D, sT = cand == 1 ? s_D : s_S;
@@ -145,76 +156,78 @@ k_playout_fast(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst
         uint32_t m = 0;
         int32_t e_m = 0;
         if (cand && B == 0) m = 1;                                 // nothing to fill: hand off after token 1
-        const uint32_t crossers = (__ballot_sync(FULL, cand && B != 0 && inC > thr) >> (team * kTeam)) & 0xFFu;
-        if (crossers) {
-            const int owner = __ffs(crossers) - 1;
+        const uint32_t crossers = __ballot_sync(FULL, cand && B != 0 && inC > thr) & tmask;
+        if (crossers) {                                            // team-uniform from here on
+            const int owner = __ffs(crossers) - 1;                 // first lane whose run takes the sum past thr
             uint32_t j_found = 0;
             int32_t run = inC - sC;
-            if (q == owner) {
+            if (lane == owner) {
                 bool hit;
                 const uint32_t passed = walk(key, j0, 0, cnt, cC_base, mulC, thr, true, run, hit);
                 j_found = j0 + passed;                             // hit is certain: the run's total exceeds thr
             }
-            j_found = __shfl_sync(tmask, j_found, owner, kTeam);
-            e_m = __shfl_sync(tmask, run, owner, kTeam);            // clean stream: e_m = S_m
+            j_found = __shfl_sync(tmask, j_found, owner);
+            e_m = __shfl_sync(tmask, run, owner);                  // clean stream: e_m = S_m
             m = j_found + 1 <= n ? j_found : 0u;                   // the hand-off needs a token left to generate
         }
         // ---- stream X
         uint32_t stall = 0, delayed = 0;
-        {
-            const uint32_t has_m = (__ballot_sync(FULL, m != 0) >> (team * kTeam)) & 0xFFu;   // team-uniform
-            if (has_m) {
-                uint32_t M;
-                if (cand == 1) M = (uint32_t)G.kappa * (l + m) + (uint32_t)G.c0;   // device re-prefills prompt + m tokens
-                else {
-                    const uint32_t u = mix32(key);                 // a server TTFT drawn from F by its knots
-                    const uint32_t ki = u >> 24, fr = (u >> 8) & 0xFFFFu;
-                    M = (uint32_t)(G.K[ki] + (int32_t)(((int64_t)(G.K[ki + 1] - G.K[ki]) * (int64_t)fr) >> 16));
+        if (m) {                                                   // team-uniform
+            uint32_t M;
+            if (cand == 1) M = (uint32_t)G.kappa * (l + m) + (uint32_t)G.c0;       // device re-prefills prompt + m tokens
+            else {
+                const uint32_t u = mix32(key);                     // a server TTFT drawn from F by its knots
+                const uint32_t ki = u >> 24, fr = (u >> 8) & 0xFFFFu;
+                M = (uint32_t)(G.K[ki] + (int32_t)(((int64_t)(G.K[ki + 1] - G.K[ki]) * (int64_t)fr) >> 16));
+            }
+            const int32_t v = e_m + (tau - (int32_t)M);            // slot lag of token m+1, negated
+            stall = (uint32_t)tau + (uint32_t)max(-v, 0);
+            if (v < 0) {
+                // tokens m+2.. stay late while the target's prefix sum of c is below `need`
+                const int32_t need = -v;
+                const uint32_t first_idx = m;                      // run-global index (j - 2) of token m+2
+                const int qs = (int)min((uint32_t)(lanes - 1), first_idx / L);
+                int32_t runA = 0;
+                uint32_t contrib = 0;
+                bool hitA = false;
+                if (q == qs && first_idx < nI)
+                    contrib = walk(key, j0, (int)(first_idx - lo), cnt, cT_base, mulT, need, false, runA, hitA);
+                runA = __shfl_sync(tmask, runA, a + qs);
+                hitA = __shfl_sync(tmask, (int)hitA, a + qs) != 0;
+                const int32_t inT_qs = __shfl_sync(tmask, inT, a + qs);
+                if (!hitA && q > qs && cnt) {
+                    const int32_t through = runA + (inT - inT_qs);               // target's sum up to this run's end
+                    int32_t before = through - sT;
+                    if (through < need) contrib = (uint32_t)cnt;
+                    else if (before < need) { bool hit; contrib = walk(key, j0, 0, cnt, cT_base, mulT, need, false, before, hit); }
                 }
-                const int32_t v = e_m + (tau - (int32_t)M);        // slot lag of token m+1, negated
-                stall = (uint32_t)tau + (uint32_t)max(-v, 0);
-                const uint32_t late = __ballot_sync(tmask, v < 0);
-                if (late) {
-                    // tokens m+2.. stay late while the target's prefix sum of c is below `need`
-                    const int32_t need = -v;
-                    const uint32_t first_idx = m;                  // run-global index (j - 2) of token m+2
-                    const int qs = L ? (int)min((uint32_t)(kTeam - 1), first_idx / L) : 0;
-                    int32_t runA = 0;
-                    uint32_t contrib = 0;
-                    bool hitA = false;
-                    if (q == qs && first_idx < nI)
-                        contrib = walk(key, j0, (int)(first_idx - lo), cnt, cT_base, mulT, need, false, runA, hitA);
-                    runA = __shfl_sync(tmask, runA, qs, kTeam);
-                    hitA = __shfl_sync(tmask, (int)hitA, qs, kTeam) != 0;
-                    const int32_t inT_qs = __shfl_sync(tmask, inT, qs, kTeam);
-                    if (!hitA && q > qs && cnt) {
-                        const int32_t through = runA + (inT - inT_qs);           // target's sum up to this run's end
-                        int32_t before = through - sT;
-                        if (through < need) contrib = (uint32_t)cnt;
-                        else if (before < need) { bool hit; contrib = walk(key, j0, 0, cnt, cT_base, mulT, need, false, before, hit); }
-                    }
-                    delayed = 1u + team_sum(contrib, tmask);
-                }
+                delayed = 1u + __reduce_add_sync(tmask, contrib);
             }
         }
-        if (q == it) {
-            o_done = go || (active && nI == 0);
-            o_m = m; o_stall = m ? stall : 0u; o_dl = m ? delayed : 0u;
-            o_sumX = m ? (nI - 1) * (uint32_t)tau + stall : 0u;
+        // ---- hand the results to the lanes that own the four requests' slots
+        const uint32_t packed = (nI == 0 || go ? 0x80000000u : 0u) | m | (delayed << 16);
+        const int slot = lane & 3;                                 // which of the four requests this lane may own
+        const int src = slot == 0 ? 0 : (slot == 1 ? b1 : (slot == 2 ? b2 : b3));
+        const int src_next = slot == 0 ? b1 : (slot == 1 ? b2 : (slot == 2 ? b3 : 32));
+        const uint32_t got_md = __shfl_sync(FULL, packed, src & 31), got_stall = __shfl_sync(FULL, stall, src & 31);
+        if ((lane >> 2) == it) {
+            const bool has_lanes = tot != 0 && src_next > src;     // no lanes: a single-token request, all zeros
+            o_md = has_lanes ? got_md : 0x80000000u;
+            o_stall = has_lanes ? got_stall : 0u;
         }
     }
     __syncwarp();
     // ---- one request per lane: results out
-    if (live && o_done) {
-        const uint32_t nI = n_l - 1, ut = (uint32_t)tau;
+    if (live && (o_md >> 31)) {
+        const uint32_t nI = n_l - 1, ut = (uint32_t)tau, m = o_md & 0xFFFFu, dl = (o_md >> 16) & 0x7FFFu;
         rec.sum[0][kk] = nI * ut; rec.max[0][kk] = nI ? ut : 0u;
         rec.sum[1][kk] = nI * ut; rec.max[1][kk] = nI ? ut : 0u;
-        rec.sum[2][kk] = o_sumX; rec.max[2][kk] = o_stall;
-        rec.stall[kk] = o_stall; rec.m[kk] = (uint16_t)o_m; rec.delayed[kk] = (uint16_t)o_dl;
+        rec.sum[2][kk] = m ? (nI - 1) * ut + o_stall : 0u; rec.max[2][kk] = m ? o_stall : 0u;
+        rec.stall[kk] = m ? o_stall : 0u; rec.m[kk] = (uint16_t)m; rec.delayed[kk] = (uint16_t)(m ? dl : 0u);
         const int kt0 = cc.ktau[g_l][0], kt1 = cc.ktau[g_l][1], kt2 = cc.ktau[g_l][2];
         for (int i = 0; i < W0; ++i) rec.win[0][(size_t)kk * W0 + i] = i == kt0 ? nI : 0u;
         for (int i = 0; i < W1; ++i) rec.win[1][(size_t)kk * W1 + i] = i == kt1 ? nI : 0u;
-        for (int i = 0; i < W2; ++i) rec.win[2][(size_t)kk * W2 + i] = (i == kt2 && o_m) ? nI - 1 : 0u;
+        for (int i = 0; i < W2; ++i) rec.win[2][(size_t)kk * W2 + i] = (i == kt2 && m) ? nI - 1 : 0u;
     }
 }
 
@@ -224,9 +237,12 @@ cudaError_t launch_playout_fast(const TraceDev& tr, const GroupConst* gc, const 
                                 uint64_t seed, TimelineRec rec, uint32_t* todo, uint32_t* todo_count,
                                 cudaStream_t st) {
     if (tr.n == 0) return cudaSuccess;
-    const uint32_t per_block = kFastWarps * 32;
+    // requests per warp: enough warps to fill the GPU (about 48 per SM) before batches grow to 32
+    int rpw = 4;
+    while (rpw < 32 && (uint64_t)tr.n / (2 * rpw) >= 148u * 48u) rpw *= 2;
+    const uint32_t per_block = kFastWarps * (uint32_t)rpw;
     k_playout_fast<<<(tr.n + per_block - 1) / per_block, kFastWarps * 32, 0, st>>>(tr, gc, cc, knots, seed_key(seed), rec,
-                                                                                    todo, todo_count);
+                                                                                    todo, todo_count, rpw);
     return cudaGetLastError();
 }
 
