@@ -357,7 +357,7 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
         cls_range.push_back({b, (uint32_t)pol_list.size()});
     }
     const uint32_t tiles = (P + 31) / 32;
-    const uint32_t want_chunks = std::max<uint32_t>(1, 296 / std::min<uint32_t>(tiles, 296));
+    const uint32_t want_chunks = std::max<uint32_t>(1, 148 / std::min<uint32_t>(tiles, 148));   // one block per SM
     uint32_t CH = (uint32_t)((N1 + want_chunks - 1) / want_chunks);
     CH = (CH + 255) / 256 * 256;
     CH = std::min<uint32_t>(std::max<uint32_t>(CH, 256), 65280);     // 16-bit histogram counters per block

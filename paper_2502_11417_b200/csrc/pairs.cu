@@ -13,8 +13,6 @@ namespace disco {
 
 namespace {
 
-constexpr uint32_t FULL = 0xFFFFFFFFu;
-
 struct PairIn {                 // one request and its play-out summaries
     uint32_t l, n, S, m;
     float saving;               // delta_c * (n - m): Eq. 4's projected saving
@@ -44,9 +42,12 @@ __device__ __forceinline__ PairOut decide(const PairIn& q, const Prep& pr, uint3
 // ------------------------------------------------------------------------------------------------------
 // Reductions: lane = policy.
 // ------------------------------------------------------------------------------------------------------
-constexpr int kAccThreads = 256;
+constexpr int kAccThreads = 512;         // one block per SM: its histograms take about half the shared memory
 constexpr int kAccWarps = kAccThreads / 32;
 constexpr int kHWords = 433;            // 866 sixteen-bit counters per policy row; odd word stride
+
+// words in front of the staging area: two histograms and the sums, rounded up to 16 bytes
+__host__ __device__ constexpr int acc_stage_offset_words(int PL) { return (2 * PL * kHWords + 2 * PL * kNAcc + 3) / 4 * 4; }
 
 __device__ __forceinline__ void hist16_add(uint32_t* row, int bin) {
     atomicAdd(&row[bin >> 1], 1u << ((bin & 1) * 16));
@@ -80,7 +81,7 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
     const bool wide = W0 > 1 || W1 > 1 || W2 > 1;             // some stream's regular TBTs span several bins
     const uint32_t tau = (uint32_t)cc.tau;
 
-    for (int i = threadIdx.x; i < 2 * PL * kHWords + 2 * PL * kNAcc; i += kAccThreads) smem[i] = 0;
+    for (int i = threadIdx.x; i < 2 * PL * kHWords + 2 * PL * kNAcc; i += kAccThreads) smem[i] = 0;   // (staging needs no clearing)
     __syncthreads();
     uint32_t* my_ttft = h_ttft + pol_in_tile * kHWords;
     uint32_t* my_stall = h_stall + pol_in_tile * kHWords;
@@ -88,44 +89,62 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
     uint32_t c_do = 0, c_rc = 0, c_dw = 0, c_mg = 0, a_td = 0, a_ps = 0, a_pd = 0, a_dl = 0, a_tau = 0;
     unsigned long long a_tt = 0;
 
+    // Per-request values are worked out once per request by the lane that loaded it and staged in shared
+    // memory; the policy lanes then read them as broadcasts.
+    uint4* stage = (uint4*)(smem + acc_stage_offset_words(PL)) + wib * 32 * 3;     // [warp][32 requests][3 x uint4]
+    // The wait map without mode tests: Algorithm 3 has no waits (l_star beyond every length), Algorithm 2 no
+    // device-only prompts (l_th = 0, as the preparation kernel leaves it).
+    const int32_t l_th = pr.l_th, l_star = pr.device_constrained ? pr.l_star : 0x7FFFFFFF;
+    const uint32_t w_star = (uint32_t)pr.w_star, w_tail = (uint32_t)pr.w_tail;
+    const float theta = pr.theta;
+    const bool mig_on = pr.mig_on != 0;
+
     for (uint32_t b0 = wib * 32u; b0 < ch.len; b0 += kAccWarps * 32u) {
         // ---- 32 requests, one per lane
-        const uint32_t kk = ch.start + min(b0 + lane, ch.len - 1);
-        const uint32_t ln = (uint32_t)tr.l[kk] | ((uint32_t)tr.nout[kk] << 16);
-        const uint32_t S_l = (uint32_t)tr.S[kk];
-        const uint32_t md = (uint32_t)rec.m[kk] | ((uint32_t)rec.delayed[kk] << 16);
-        const uint32_t stall_l = rec.stall[kk];
-        const uint32_t nt0 = kt0 >= 0 ? rec.win[0][(size_t)kk * W0 + kt0] : 0u;
-        const uint32_t nt1 = kt1 >= 0 ? rec.win[1][(size_t)kk * W1 + kt1] : 0u;
-        const uint32_t nt2 = kt2 >= 0 ? rec.win[2][(size_t)kk * W2 + kt2] : 0u;
-        const uint32_t nt01 = nt0 | (nt1 << 16);
+        {
+            const uint32_t kk = ch.start + min(b0 + lane, ch.len - 1);
+            const uint32_t l = tr.l[kk], n = tr.nout[kk], S = (uint32_t)tr.S[kk], m = rec.m[kk];
+            const uint32_t stall = rec.stall[kk];
+            const uint32_t nt0 = kt0 >= 0 ? rec.win[0][(size_t)kk * W0 + kt0] : 0u;
+            const uint32_t nt1 = kt1 >= 0 ? rec.win[1][(size_t)kk * W1 + kt1] : 0u;
+            uint32_t nt2 = kt2 >= 0 ? rec.win[2][(size_t)kk * W2 + kt2] : 0u;
+            int stall_bin = -1;                                // the token after a hand-off: counted with tau's bin
+            if (stall == tau) ++nt2; else stall_bin = bin_of_ticks(stall);
+            // a request may only migrate if its buffer filled (m != 0); fold that into the saving (Eq. 4)
+            const float saving = m ? delta_c * (float)(n - m) : -1.0f;
+            __syncwarp();
+            stage[lane * 3 + 0] = make_uint4(l, n, S, kappa * l + c0);
+            stage[lane * 3 + 1] = make_uint4(m, l + m, __float_as_uint(saving), rec.delayed[kk]);
+            stage[lane * 3 + 2] = make_uint4(nt0, nt1, nt2, (uint32_t)stall_bin);
+            __syncwarp();
+        }
         const int n_here = (int)min(32u, ch.len - b0);
         for (int r0 = 0; r0 < n_here; r0 += slots) {
             const int r = r0 + slot;
-            const uint32_t ln_r = __shfl_sync(FULL, ln, r), S = __shfl_sync(FULL, S_l, r);
-            const uint32_t md_r = __shfl_sync(FULL, md, r), stall = __shfl_sync(FULL, stall_l, r);
-            const uint32_t nt01_r = __shfl_sync(FULL, nt01, r), nt2_r = __shfl_sync(FULL, nt2, r);
             if (!act || r >= n_here) continue;
-            PairIn q;
-            q.l = ln_r & 0xFFFFu; q.n = ln_r >> 16; q.S = S; q.m = md_r & 0xFFFFu;
-            q.saving = delta_c * (float)(q.n - q.m);
-            const PairOut o = decide(q, pr, kappa * q.l + c0, candidate);
-            const uint32_t lm = q.l + q.m;
-            const uint32_t tok_src = o.migr ? q.m : q.n;
-            c_do += o.dev_only; c_rc += o.race; c_dw += o.race && o.dev_wins; c_mg += o.migr;
-            a_td += o.dev_wins ? tok_src : q.n - tok_src;
-            a_ps += (o.dev_only ? 0u : q.l) + ((o.migr && o.dev_wins) ? lm : 0u);
-            a_pd += (o.started ? q.l : 0u) + ((o.migr && !o.dev_wins) ? lm : 0u);
-            a_dl += o.migr ? md_r >> 16 : 0u;
-            a_tt += o.ttft;
-            uint32_t ntau = o.migr ? nt2_r : (o.dev_wins ? nt01_r >> 16 : nt01_r & 0xFFFFu);
-            hist16_add(my_ttft, bin_of_ticks(o.ttft));
-            if (o.migr) {                                      // the token after the hand-off
-                if (stall == tau) ++ntau; else hist16_add(my_stall, bin_of_ticks(stall));
-            }
-            a_tau += ntau;
+            const uint4 A = stage[r * 3 + 0], Bq = stage[r * 3 + 1], Cq = stage[r * 3 + 2];
+            const uint32_t l = A.x, n = A.y, S = A.z, Td = A.w, m = Bq.x, lm = Bq.y;
+            // ---- dispatch (Algorithm 2's wait map / Algorithm 3's threshold) and the race
+            const bool dev_only = (int32_t)l < l_th;
+            const uint32_t w = (int32_t)l < l_star ? 0u : ((int32_t)l == l_star ? w_star : w_tail);
+            const bool started = dev_only || S > w;                // the device starts after the wait
+            const uint32_t wTd = w + Td;
+            const bool dev_wins = dev_only || (started && S > wTd);   // a tie goes to the server
+            const uint32_t ttft = dev_only ? Td : min(S, wTd);
+            const bool race = started && !dev_only;
+            const bool migr = mig_on && race && candidate == (dev_wins ? 2 : 1) && __uint_as_float(Bq.z) > theta;
+            const uint32_t tok_src = migr ? m : n;
+            c_do += dev_only; c_rc += race; c_dw += race && dev_wins; c_mg += migr;
+            a_td += dev_wins ? tok_src : n - tok_src;
+            a_ps += (dev_only ? 0u : l) + ((migr && dev_wins) ? lm : 0u);
+            a_pd += (started ? l : 0u) + ((migr && !dev_wins) ? lm : 0u);
+            a_dl += migr ? Bq.w : 0u;
+            a_tt += ttft;
+            a_tau += migr ? Cq.z : (dev_wins ? Cq.y : Cq.x);
+            hist16_add(my_ttft, bin_of_ticks(ttft));
+            if (migr && (int32_t)Cq.w >= 0) hist16_add(my_stall, (int)Cq.w);
             if (wide) {                                        // regular TBTs outside the bin of tau
-                const int c = o.migr ? 2 : (o.dev_wins ? 1 : 0);
+                const int c = migr ? 2 : (dev_wins ? 1 : 0);
                 const int W = c == 2 ? W2 : (c == 1 ? W1 : W0), kt = c == 2 ? kt2 : (c == 1 ? kt1 : kt0);
                 const uint32_t* wp = rec.win[c] + (size_t)(ch.start + b0 + r) * W;
                 unsigned long long* hp = hist_tbt + (size_t)p * kNBins + cc.lo[g][c];
@@ -167,7 +186,9 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
     }
 }
 
-size_t acc_smem_bytes(int PL) { return sizeof(uint32_t) * (2 * PL * kHWords + 2 * PL * kNAcc); }
+size_t acc_smem_bytes(int PL) {
+    return sizeof(uint32_t) * acc_stage_offset_words(PL) + (size_t)kAccWarps * 32 * 3 * sizeof(uint4);
+}
 
 // ------------------------------------------------------------------------------------------------------
 // Per-pair arrays: lane = request, eight policies per block column.
