@@ -164,7 +164,7 @@ cudaError_t reserve_trace(disco_ctx* c, uint32_t n, bool host_inputs, bool has_s
     const size_t cnt_bytes = ((size_t)G * (kMaxPrompt + 1) * 4 + 15) / 16 * 16;
     const size_t counts_bytes = (size_t)256 * kRadixMaxBlocks * 4;
     const size_t head = cnt_bytes + kMaxGroups * 8 + kMaxGroups * 4 + 16 + 16;
-    R(zero, head + 5 * counts_bytes);
+    R(zero, head + 5 * counts_bytes + 1024);                    // + the 256 digit totals
     char* z = (char*)c->zero.p;
     c->cnt = (uint32_t*)z; c->grp_sum_n = (uint64_t*)(z + cnt_bytes); c->ng = (uint32_t*)(z + cnt_bytes + kMaxGroups * 8);
     c->max_n = (uint32_t*)(z + cnt_bytes + kMaxGroups * 12); c->err = (int32_t*)(z + cnt_bytes + kMaxGroups * 12 + 16);

@@ -92,43 +92,41 @@ __global__ void k_radix_hist(const uint64_t* __restrict__ keys, uint32_t n, uint
     counts[threadIdx.x * gridDim.x + blockIdx.x] = h[threadIdx.x];
 }
 
-// exclusive scan of `m` counters by one block of 1024 threads
-__global__ void k_scan_counts(uint32_t* __restrict__ counts, uint32_t m, uint32_t* __restrict__ clear = nullptr) {
-    __shared__ uint32_t part[1024];
-    if (clear) for (uint32_t i = threadIdx.x; i < m; i += 1024) clear[i] = 0;
-    const uint32_t per = (m + 1023u) / 1024u;
-    const uint32_t lo = min(m, threadIdx.x * per), hi = min(m, lo + per);
+// One block per digit: exclusive scan of the digit's per-block counts, in place, and the digit's total.
+__global__ void k_radix_rowscan(uint32_t* __restrict__ counts /* [256][blocks] */, uint32_t blocks,
+                                uint32_t* __restrict__ totals /* [256] */) {
+    __shared__ uint32_t part[128];
+    uint32_t* row = counts + (size_t)blockIdx.x * blocks;
+    const uint32_t per = (blocks + 127u) / 128u;
+    const uint32_t lo = min(blocks, threadIdx.x * per), hi = min(blocks, lo + per);
     uint32_t s = 0;
-    for (uint32_t i = lo; i < hi; ++i) s += counts[i];
+    for (uint32_t i = lo; i < hi; ++i) s += row[i];
     part[threadIdx.x] = s;
     __syncthreads();
-    for (int off = 1; off < 1024; off <<= 1) {
-        uint32_t v = threadIdx.x >= (unsigned)off ? part[threadIdx.x - off] : 0u;
+    for (int off = 1; off < 128; off <<= 1) {
+        const uint32_t v = (int)threadIdx.x >= off ? part[threadIdx.x - off] : 0u;
         __syncthreads();
         part[threadIdx.x] += v;
         __syncthreads();
     }
     uint32_t run = part[threadIdx.x] - s;
-    for (uint32_t i = lo; i < hi; ++i) { const uint32_t c = counts[i]; counts[i] = run; run += c; }
+    for (uint32_t i = lo; i < hi; ++i) { const uint32_t c = row[i]; row[i] = run; run += c; }
+    if (threadIdx.x == 127) totals[blockIdx.x] = part[127];
 }
 
 __global__ void k_radix_scatter(const uint64_t* __restrict__ keys_in, uint64_t* __restrict__ keys_out,
                                 const uint32_t* __restrict__ pay_in, uint32_t* __restrict__ pay_out, uint32_t n,
                                 uint32_t per_block, int shift, const uint32_t* __restrict__ offsets,
-                                uint32_t* __restrict__ counts_next = nullptr, int32_t* __restrict__ low_out = nullptr,
-                                bool raw = false) {
+                                const uint32_t* __restrict__ totals, uint32_t* __restrict__ counts_next = nullptr,
+                                int32_t* __restrict__ low_out = nullptr) {
     __shared__ uint32_t run[256];                 // next output slot of each digit for this block
     __shared__ uint32_t wcnt[kRadixWarps][256];   // keys of each digit per warp in the current slab
     const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (!raw) {
-        run[threadIdx.x] = offsets[threadIdx.x * gridDim.x + blockIdx.x];
-    } else {
-        // `offsets` holds plain counts [digit][block]: this block's slots start after every key of a smaller
-        // digit and after the keys of the same digit in earlier blocks
-        const uint32_t* row = offsets + threadIdx.x * gridDim.x;
-        uint32_t total = 0, before = 0;
-        for (uint32_t b = 0; b < gridDim.x; ++b) { const uint32_t c = row[b]; total += c; before += b < blockIdx.x ? c : 0u; }
+    {
+        // offsets[d][b]: keys of digit d in earlier blocks (k_radix_rowscan); totals[d]: keys of digit d.
+        // This block's first slot for digit d = keys of smaller digits + keys of d in earlier blocks.
         uint32_t* tot = wcnt[0];
+        const uint32_t total = totals[threadIdx.x];
         tot[threadIdx.x] = total;
         __syncthreads();
         for (int off = 1; off < 256; off <<= 1) {
@@ -137,35 +135,63 @@ __global__ void k_radix_scatter(const uint64_t* __restrict__ keys_in, uint64_t* 
             tot[threadIdx.x] += v;
             __syncthreads();
         }
-        run[threadIdx.x] = tot[threadIdx.x] - total + before;
+        run[threadIdx.x] = tot[threadIdx.x] - total + offsets[threadIdx.x * gridDim.x + blockIdx.x];
         __syncthreads();
     }
     const uint32_t lo = min(n, blockIdx.x * per_block), hi = min(n, lo + per_block);
-    for (uint32_t base = lo; base < hi; base += kRadixThreads) {
+    constexpr int kPer = 4;                                   // keys per thread and tile
+    constexpr uint32_t kTile = kRadixThreads * kPer;          // a warp owns 128 consecutive keys of a tile
+    for (uint32_t base = lo; base < hi; base += kTile) {
         for (int k = 0; k < kRadixWarps; ++k) wcnt[k][threadIdx.x] = 0;
-        __syncthreads();
-        const uint32_t i = base + threadIdx.x;
-        const bool live = i < hi;
-        uint64_t key = 0;
-        uint32_t dig = 256u + (uint32_t)lane;     // dead lanes get digits of their own
-        if (live) { key = keys_in[i]; dig = (uint32_t)(key >> shift) & 255u; }
-        const uint32_t peers = __match_any_sync(0xFFFFFFFFu, dig);
-        const uint32_t rank = __popc(peers & ((1u << lane) - 1u));
-        if (live && rank == 0) wcnt[w][dig] = __popc(peers);
-        __syncthreads();
-        if (live) {
-            uint32_t before = 0;
-            for (int k = 0; k < w; ++k) before += wcnt[k][dig];
-            const uint32_t pos = run[dig] + before + rank;
-            if (low_out) low_out[pos] = (int32_t)(uint32_t)key; else keys_out[pos] = key;
-            if (pay_out) pay_out[pos] = pay_in ? pay_in[i] : i;
-            if (counts_next)
-                atomicAdd(&counts_next[((uint32_t)(key >> (shift + 8)) & 255u) * gridDim.x + pos / per_block], 1u);
+        uint64_t key[kPer];
+        uint32_t dig[kPer], peers[kPer];
+        bool live[kPer];
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) {
+            const uint32_t i = base + w * (32 * kPer) + j * 32 + lane;
+            live[j] = i < hi;
+            key[j] = live[j] ? keys_in[i] : 0;
+            dig[j] = (uint32_t)(key[j] >> shift) & 255u;
+            // lanes holding the same digit, from eight ballots over the digit's bits
+            uint32_t m = __ballot_sync(0xFFFFFFFFu, live[j]);
+#pragma unroll
+            for (int b = 0; b < 8; ++b) {
+                const uint32_t bal = __ballot_sync(0xFFFFFFFFu, (dig[j] >> b) & 1u);
+                m &= ((dig[j] >> b) & 1u) ? bal : ~bal;
+            }
+            peers[j] = m;
         }
         __syncthreads();
-        uint32_t tot = 0;
-        for (int k = 0; k < kRadixWarps; ++k) tot += wcnt[k][threadIdx.x];
-        run[threadIdx.x] += tot;
+        // keys of each digit in each warp (a warp's row is its own: plain adds, rounds in order)
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) {
+            if (live[j] && (peers[j] & ((1u << lane) - 1u)) == 0) wcnt[w][dig[j]] += __popc(peers[j]);
+            __syncwarp();
+        }
+        __syncthreads();
+        {   // turn the counts into each warp's first slot per digit; advance the block's running slots
+            uint32_t at = run[threadIdx.x];
+            for (int k = 0; k < kRadixWarps; ++k) { const uint32_t c = wcnt[k][threadIdx.x]; wcnt[k][threadIdx.x] = at; at += c; }
+            run[threadIdx.x] = at;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) {
+            if (live[j]) {
+                const uint32_t rank = __popc(peers[j] & ((1u << lane) - 1u));
+                const uint32_t pos = wcnt[w][dig[j]] + rank;
+                if (low_out) low_out[pos] = (int32_t)(uint32_t)key[j]; else keys_out[pos] = key[j];
+                if (pay_out) {
+                    const uint32_t i = base + w * (32 * kPer) + j * 32 + lane;
+                    pay_out[pos] = pay_in ? pay_in[i] : i;
+                }
+                if (counts_next)
+                    atomicAdd(&counts_next[((uint32_t)(key[j] >> (shift + 8)) & 255u) * gridDim.x + pos / per_block], 1u);
+            }
+            __syncwarp();
+            if (live[j] && (peers[j] & ((1u << lane) - 1u)) == 0) wcnt[w][dig[j]] += __popc(peers[j]);
+            __syncwarp();
+        }
         __syncthreads();
     }
 }
@@ -256,9 +282,10 @@ cudaError_t radix_pass(const uint64_t* kin, uint64_t* kout, const uint32_t* pin,
     if (blocks > kRadixMaxBlocks) blocks = kRadixMaxBlocks;
     uint32_t per_block = (n + blocks - 1) / blocks;
     per_block = (per_block + kRadixThreads - 1) / kRadixThreads * kRadixThreads;
+    uint32_t* totals = counts + (size_t)256u * blocks;       // the caller's buffer has room for these 256 words
     k_radix_hist<<<blocks, kRadixThreads, 0, st>>>(kin, n, per_block, shift, counts);
-    k_scan_counts<<<1, 1024, 0, st>>>(counts, 256u * blocks);
-    k_radix_scatter<<<blocks, kRadixThreads, 0, st>>>(kin, kout, pin, pout, n, per_block, shift, counts);
+    k_radix_rowscan<<<256, 128, 0, st>>>(counts, blocks, totals);
+    k_radix_scatter<<<blocks, kRadixThreads, 0, st>>>(kin, kout, pin, pout, n, per_block, shift, counts, totals);
     return cudaGetLastError();
 }
 
@@ -266,7 +293,7 @@ cudaError_t radix_pass(const uint64_t* kin, uint64_t* kout, const uint32_t* pin,
 
 uint32_t load_kernel_launches(uint32_t n, int G) {
     if (n == 0) return 2;
-    if (G == 1 && n <= (1u << 20)) return 1 + 4 + 2;         // ingest, four scatter passes, group tables
+    if (G == 1 && n <= (1u << 20)) return 1 + 2 * 4 + 2;     // ingest, (row scan, scatter) x 4, group tables
     const uint32_t passes = G > 1 ? 6 : 4;                  // radix passes: partition + 5, or 4
     return 1 + (G > 1 ? 1 : 0) + 3 * passes + 1 + 2;         // ingest, gather, passes, low words, group tables
 }
@@ -301,12 +328,14 @@ cudaError_t run_load(const LoadArgs& a, cudaStream_t st) {
         uint64_t *src = a.keys_a, *dst = a.keys_b;
         const int passes = G > 1 ? 5 : 4;
         if (small) {
-            for (int p = 0; p < passes; ++p) {                  // one launch per pass: no separate scan
+            uint32_t* totals = a.radix_counts + (size_t)5 * 256u * kRadixMaxBlocks;
+            for (int p = 0; p < passes; ++p) {                  // the scatter also counts the next digit
                 const bool last = p == passes - 1;
                 uint32_t* cur = a.radix_counts + (size_t)p * 256u * blocks;
+                k_radix_rowscan<<<256, 128, 0, st>>>(cur, blocks, totals);
                 k_radix_scatter<<<blocks, kRadixThreads, 0, st>>>(src, dst, nullptr, nullptr, n, per_block, 8 * p, cur,
-                                                                  last ? nullptr : cur + 256u * blocks,
-                                                                  last ? a.sorted : nullptr, true);
+                                                                  totals, last ? nullptr : cur + 256u * blocks,
+                                                                  last ? a.sorted : nullptr);
                 uint64_t* t = src; src = dst; dst = t;
             }
         } else {
@@ -337,7 +366,7 @@ namespace {
 
 constexpr uint32_t kNoAllocMaxN = DISCO_NOALLOC_MAX_N;
 constexpr size_t kNaKeysBytes = (size_t)kNoAllocMaxN * sizeof(uint64_t);
-constexpr size_t kNaCountsBytes = 256u * ((kNoAllocMaxN + 1023u) / 1024u) * sizeof(uint32_t);   // as radix_pass sizes its grid
+constexpr size_t kNaCountsBytes = (256u * ((kNoAllocMaxN + 1023u) / 1024u) + 256u) * sizeof(uint32_t);   // as radix_pass sizes its grid, plus the digit totals
 constexpr size_t kNaErrOff = 2 * kNaKeysBytes + kNaCountsBytes;
 
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNaErrOff + 256];
