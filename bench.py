@@ -39,7 +39,7 @@ PAIR_INSTR = 42
 SM_COUNT, SCHEDULERS, LANES = 148, 4, 32
 # DRAM bytes per launch from the committed ncu capture of the dominant kernel (None until captured for
 # the current kernel; see profiles/).
-NCU_TRAFFIC_BYTES = {"k_pairs_rows": None, "k_pairs_acc": None, "k_playout_fast": None, "k_playout": None}
+NCU_TRAFFIC_BYTES = {"k_pairs_rows": 145562368, "k_pairs_acc": None, "k_playout_fast": 823040, "k_playout": None}
 
 
 def env_rank():
@@ -56,45 +56,60 @@ def measured_peaks():
 
 
 class ClockSampler:
-    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
-              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """Samples SM clock and throttle reasons of one GPU every 20 ms through NVML while the timed region runs
+    (read-only queries)."""
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
 
     def __init__(self, index):
-        self.index, self.proc = index, None
+        import threading
+        self.index, self.samples, self.reasons, self.max_mhz = int(index), [], set(), None
+        self._stop = threading.Event()
+        self._thread = threading.Thread(target=self._run, daemon=True)
+        self.error = None
+
+    def _run(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+            while True:
+                self.samples.append(float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)))
+                mask = pynvml.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+                if self._stop.wait(0.02):
+                    break
+        except Exception as e:                      # no NVML: report that rather than invent numbers
+            self.error = repr(e)
 
     def start(self):
-        try:
-            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
-                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-        except OSError:
-            self.proc = None
+        self._thread.start()
 
     def stop(self):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            out, _ = self.proc.communicate(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
-            out, _ = self.proc.communicate()
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in out.splitlines():
-            f = [x.strip() for x in line.split(",")]
-            if len(f) < 9:
-                continue
-            try:
-                sm.append(float(f[1])); mx.append(float(f[2]))
-            except ValueError:
-                continue
-            for name, v in zip(names, f[5:9]):
-                if v.lower().startswith("active"):
-                    reasons.add(name)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+        self._stop.set()
+        self._thread.join(timeout=5)
+        if self.error or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "samples": 0,
+                    "reasons": ["clock sampling failed: %s" % self.error]}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz, "samples": len(self.samples),
+                "reasons": sorted(self.reasons)}
+
+
+def max_over_ranks(total_ms, dist, device):
+    """The slowest rank's time decides a multi-GPU step (all-reduce MAX); a single process returns its own."""
+    if dist is None:
+        return total_ms
+    import torch
+    t = torch.tensor([total_ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(units_per_rank, world, steps, total_ms):
+    """Whole-job throughput: units of all ranks over the slowest rank's time."""
+    return units_per_rank * world * steps / (total_ms * 1e-3)
 
 
 def oracle_sample_run(w, n_req, threads):
@@ -215,15 +230,14 @@ def run_ours(args):
         torch.cuda.synchronize()
         if dist is not None:
             dist.barrier()
-        total_ms = sum(a.elapsed_time(b) for a, b in evs)
-        if dist is not None:
-            t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            total_ms = float(t.item())
-        return total_ms
+        return max_over_ranks(sum(a.elapsed_time(b) for a, b in evs), dist, "cuda")
 
-    sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else
-                           os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank])
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+    try:
+        phys = int(vis.split(",")[local_rank]) if vis else local_rank
+    except ValueError:
+        phys = local_rank
+    sampler = ClockSampler(phys)
     ktimes = []
     l0 = kernel_launch_count()
     timed(dev, 0, args.warmup)
@@ -236,8 +250,8 @@ def run_ours(args):
 
     pairs = n * P * world
     toks = int(w.output_len.sum()) * P * world          # approximate for N > 1: replicas have like shapes
-    value = pairs * args.steps / (total_ms * 1e-3)
-    e2e_value = pairs * args.steps / (e2e_ms * 1e-3)
+    value = whole_job_rate(n * P, world, args.steps, total_ms)
+    e2e_value = whole_job_rate(n * P, world, args.steps, e2e_ms)
 
     # ---- roofline of the dominant kernel of a step
     hbm_gbs, sm_max_mhz, src = measured_peaks()
@@ -251,18 +265,18 @@ def run_ours(args):
         bytes_alg = n * P * PAIR_OUT_BYTES + n * TRACE_BYTES
         ach = bytes_alg / (kms[top] * 1e-3) / 1e9
         roof = {"kernel": top, "bound": "hbm", "achieved": ach, "peak": hbm_gbs, "unit": "GB/s",
-                "frac": ach / hbm_gbs, "traffic": NCU_TRAFFIC_BYTES[top], "peak_source": src,
+                "frac": ach / hbm_gbs, "traffic": NCU_TRAFFIC_BYTES[top] if args.config == 1 and not args.requests else None,
+                "peak_source": src,
                 "algorithmic_bytes": bytes_alg}
     elif top == "k_pairs_acc":
         ach = n * P * PAIR_INSTR / (kms[top] * 1e-3) / 1e12
         roof = {"kernel": top, "bound": "alu", "achieved": ach, "peak": alu_peak, "unit": "Tinstr/s",
-                "frac": ach / alu_peak, "traffic": NCU_TRAFFIC_BYTES[top], "peak_source": alu_src,
-                "instr_per_pair": PAIR_INSTR}
+                "frac": ach / alu_peak, "traffic": None, "peak_source": alu_src, "instr_per_pair": PAIR_INSTR}
     else:
         ach = token_steps * PLAYOUT_INSTR_PER_TOKEN / (kms[top] * 1e-3) / 1e12
         roof = {"kernel": top, "bound": "alu", "achieved": ach, "peak": alu_peak, "unit": "Tinstr/s",
-                "frac": ach / alu_peak, "traffic": NCU_TRAFFIC_BYTES[top], "peak_source": alu_src,
-                "token_steps": token_steps, "instr_per_token_step": PLAYOUT_INSTR_PER_TOKEN}
+                "frac": ach / alu_peak, "traffic": NCU_TRAFFIC_BYTES[top] if args.config == 1 and not args.requests else None,
+                "peak_source": alu_src, "token_steps": token_steps, "instr_per_token_step": PLAYOUT_INSTR_PER_TOKEN}
     roof["ms_per_launch"] = kms[top]
     roof["kernels_ms"] = kms
 
@@ -299,7 +313,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=1, help="workload 0..4 (default: workload 1)")
     ap.add_argument("--requests", type=int, default=None, help="shrink the trace (profiling on a small case)")
