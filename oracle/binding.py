@@ -40,7 +40,7 @@ class device_struct(C.Structure):
 
 class policy_struct(C.Structure):
     _fields_ = [("budget", C.c_float), ("alpha", C.c_float), ("mig_threshold", C.c_float),
-                ("t_m_s", C.c_float), ("r_c", C.c_float), ("flags", C.c_uint32)]
+                ("t_m_s", C.c_float), ("r_c", C.c_float), ("flags", C.c_uint32), ("expected_len", C.c_uint32)]
 
 
 class prep_struct(C.Structure):
@@ -134,7 +134,8 @@ def _devices(devices: Sequence[Dict[str, float]]):
 def _policies(policies: Sequence[Dict[str, float]]):
     arr = (policy_struct * len(policies))()
     for k, p in enumerate(policies):
-        arr[k] = policy_struct(p["budget"], p["alpha"], p["mig_threshold"], p["t_m_s"], p["r_c"], p["flags"])
+        arr[k] = policy_struct(p["budget"], p["alpha"], p["mig_threshold"], p["t_m_s"], p["r_c"], p["flags"],
+                               p.get("expected_len", 0))
     return arr
 
 

@@ -114,7 +114,7 @@ int policy_ticks(const orc_policy_t& p, PolicyTicks* o) {
     o->mig = (p.flags & ORC_FLAG_MIGRATION) != 0;
     o->pacing = (p.flags & ORC_FLAG_PACING) != 0;
     o->mode = (int)((p.flags >> 2) & 3);
-    if (o->mode == 3) return fail("unknown mode");
+    if (o->mode == 3 || (p.flags >> 5)) return fail("unknown flags");
     /* Eq. 6: B = r_c * t_m tokens, rounded up; nothing to fill without a buffer */
     o->B = o->pacing ? (int32_t)std::min<int64_t>((o->t_m + o->tau - 1) / o->tau, 1 << 30) : 0;
     return 0;
@@ -217,7 +217,16 @@ void play(const orc_trace& tr, const orc_policy_t& pol, const orc_prep_t& pr, ui
     R->server_dispatched = true;
     int64_t w = 0;
     bool device_only = false;
-    if (!pr.device_constrained) {
+    bool server_only = false;
+    if (pol.flags & ORC_FLAG_STOCHASTIC) {
+        /* Stoch-S / Stoch-D baselines (Sec. 5.1): each request goes to the constrained endpoint with
+         * probability b, otherwise to the other one; one endpoint only, no race, no migration. */
+        const uint32_t u = token_hash(key, 0xFFFFFFFFu);
+        const double b = (double)pol.budget;
+        const bool constrained = b >= 1.0 || (double)u < std::floor(b * 4294967296.0);
+        const bool to_device = pr.device_constrained ? constrained : !constrained;
+        device_only = to_device; server_only = !to_device;
+    } else if (!pr.device_constrained) {
         if (l < pr.l_th) device_only = true;           /* Algorithm 3: short prompts stay on the device */
     } else {
         w = (l < pr.l_star) ? 0 : (l == pr.l_star) ? pr.w_star : pr.w_tail;   /* Algorithm 2's map W */
@@ -225,6 +234,8 @@ void play(const orc_trace& tr, const orc_policy_t& pol, const orc_prep_t& pr, ui
     if (device_only) {
         R->decision = ORC_DEVICE_ONLY; R->server_dispatched = false; R->device_started = true;
         R->winner_device = true; R->ttft = Td;
+    } else if (server_only) {
+        R->decision = ORC_SERVER_ONLY; R->device_started = false; R->winner_device = false; R->ttft = S;
     } else {
         /* server first; the device starts after w if no server token has arrived; first token wins */
         R->device_started = S > w;
@@ -260,8 +271,10 @@ void play(const orc_trace& tr, const orc_policy_t& pol, const orc_prep_t& pr, ui
             }
         }
         if (m > 0) {
-            /* Eq. 4: projected saving on the true remainder against the overhead */
-            const float saving = pr.delta_c * (float)(n - m);
+            /* Eq. 4: projected saving on the remaining length against the overhead; the remainder is the
+             * trace's true one, or what is left of an expected total length when the policy gives one */
+            const int32_t remaining = pol.expected_len ? std::max<int32_t>((int32_t)pol.expected_len - m, 0) : n - m;
+            const float saving = pr.delta_c * (float)remaining;
             if (saving > pol.mig_threshold) {
                 int64_t M;
                 int64_t Tt, Jt;
