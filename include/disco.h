@@ -49,6 +49,8 @@ extern "C" {
 /* policy flags */
 #define DISCO_FLAG_MIGRATION 1u  /* token-level migration on (Sec. 4.3) */
 #define DISCO_FLAG_PACING 2u     /* delivery buffer: tokens handed over no faster than r_c */
+#define DISCO_FLAG_STOCHASTIC 16u /* Stoch-S / Stoch-D baseline (Sec. 5.1): each request goes to the constrained
+                                    endpoint with probability b, else to the other one; no race, no migration */
 #define DISCO_MODE_AUTO (0u << 2)               /* Algorithm 1 decides from the costs */
 #define DISCO_MODE_DEVICE_CONSTRAINED (1u << 2) /* force Algorithm 2 */
 #define DISCO_MODE_SERVER_CONSTRAINED (2u << 2) /* force Algorithm 3 */
@@ -97,6 +99,8 @@ typedef struct {
     float t_m_s;           /* estimated migration time, seconds; buffer B = ceil(r_c t_m) tokens */
     float r_c;             /* consumption rate, tokens/s, > 0 */
     uint32_t flags;        /* DISCO_FLAG_* | DISCO_MODE_* */
+    uint32_t expected_len; /* Eq. 4's remaining length: 0 = the trace's true remainder n - m; else what is left of
+                              this expected total output length, max(expected_len - m, 0) */
 } disco_policy_t;
 
 /* Optional per-pair outputs, device memory, each [P][n] with requests

@@ -44,7 +44,7 @@ class TraceDesc(C.Structure):
 
 class Policy(C.Structure):
     _fields_ = [("budget", C.c_float), ("alpha", C.c_float), ("mig_threshold", C.c_float), ("t_m_s", C.c_float),
-                ("r_c", C.c_float), ("flags", C.c_uint32)]
+                ("r_c", C.c_float), ("flags", C.c_uint32), ("expected_len", C.c_uint32)]
 
 
 class PairOut(C.Structure):
@@ -154,7 +154,8 @@ def device_array(devices: Sequence[Dict[str, float]]):
 def policy_array(policies: Sequence[Dict[str, float]]):
     arr = (Policy * len(policies))()
     for k, p in enumerate(policies):
-        arr[k] = Policy(p["budget"], p["alpha"], p["mig_threshold"], p["t_m_s"], p["r_c"], p["flags"])
+        arr[k] = Policy(p["budget"], p["alpha"], p["mig_threshold"], p["t_m_s"], p["r_c"], p["flags"],
+                        p.get("expected_len", 0))
     return arr
 
 

@@ -268,6 +268,7 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
     // ---- policy constants and timeline classes
     std::vector<PolicyConst> pc(P);
     std::vector<ClassConst> classes;
+    bool cls_extras_pending = false;      // some policy routes at random or triggers on an expected length
     for (uint32_t p = 0; p < P; ++p) {
         const disco_policy_t& q = pol[p];
         const std::string at = " (policy " + std::to_string(p) + ")";
@@ -277,7 +278,8 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
         if (!(q.r_c > 0.0f) || !std::isfinite(q.r_c)) return fail(DISCO_EINVAL, "consumption rate must be positive" + at);
         if (!(q.t_m_s >= 0.0f) || !std::isfinite(q.t_m_s)) return fail(DISCO_EINVAL, "migration time must be >= 0" + at);
         const uint32_t mode = (q.flags >> 2) & 3u;
-        if (mode == 3 || (q.flags >> 4)) return fail(DISCO_EINVAL, "unknown flags" + at);
+        if (mode == 3 || (q.flags >> 5)) return fail(DISCO_EINVAL, "unknown flags" + at);
+        if (q.expected_len > (1u << 20)) return fail(DISCO_EINVAL, "expected length too large" + at);
         const int64_t tau = ticks_of_rate(q.r_c), t_m = ticks_of_seconds(q.t_m_s);
         if (tau < 1 || tau >= (1 << 30)) return fail(DISCO_EINVAL, "consumption interval outside 1 .. 2^30 ticks" + at);
         const bool pacing = (q.flags & DISCO_FLAG_PACING) != 0, mig = (q.flags & DISCO_FLAG_MIGRATION) != 0;
@@ -286,6 +288,10 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
         PolicyConst& o = pc[p];
         o.budget = q.budget; o.alpha = q.alpha; o.theta = q.mig_threshold; o.flags = q.flags;
         o.tau = (int32_t)tau; o.B = (int32_t)B; o.mode = (int32_t)mode;
+        o.expected_len = q.expected_len; o.pad = 0;
+        o.route_all = q.budget >= 1.0f ? 1 : 0;
+        o.route_thr = o.route_all ? 0xFFFFFFFFu : (uint32_t)std::floor((double)q.budget * 4294967296.0);
+        if ((q.flags & DISCO_FLAG_STOCHASTIC) || q.expected_len) cls_extras_pending = true;
         int cls = -1;
         for (size_t k = 0; k < classes.size(); ++k)
             if (classes[k].tau == o.tau && classes[k].B == o.B && classes[k].pacing == (int)pacing) { cls = (int)k; break; }
@@ -432,7 +438,8 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
         CU(launch_pairs(tr, c->d_gc.as<GroupConst>(), dcc, c->d_prep.as<Prep>(), P,
                         c->d_pol_list.as<uint32_t>() + cls_range[k].first, cls_range[k].second - cls_range[k].first,
                         c->d_chunks.as<Chunk>(), (uint32_t)chunks.size(), rec, po, c->d_acc.as<uint64_t>(),
-                        c->d_hist_ttft.as<uint64_t>(), c->d_hist_tbt.as<uint64_t>(), timed ? c->ev[3] : nullptr, st));
+                        c->d_hist_ttft.as<uint64_t>(), c->d_hist_tbt.as<uint64_t>(), seed, cls_extras_pending,
+                        timed ? c->ev[3] : nullptr, st));
         if (timed) CU(cudaEventRecord(c->ev[4], st));
         g_launches += (n ? (classes[k].pacing ? 2 : 1) : 0) + ((n && !chunks.empty()) ? (out ? 2 : 1) : 0);
     }

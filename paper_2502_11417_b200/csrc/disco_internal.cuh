@@ -33,6 +33,10 @@ struct PolicyConst {
     int32_t tau, B;
     int32_t cls;                 // timeline class (policies with equal tau, B, pacing share play-outs)
     int32_t mode;                // 0 Algorithm 1 decides, 1 device-constrained, 2 server-constrained
+    uint32_t expected_len;       // 0 = true remainder in the migration trigger
+    uint32_t route_thr;          // stochastic routing: constrained endpoint iff hash < route_thr (or route_all)
+    int32_t route_all;
+    int32_t pad;
 };
 
 // ---- what Algorithms 1-3 produce for one (group, policy) ----
@@ -43,6 +47,9 @@ struct Prep {
     int32_t w_star, w_tail;
     float theta;
     int32_t mig_on;
+    int32_t stochastic;          // random routing instead of Algorithms 2-3
+    uint32_t expected_len, route_thr;
+    int32_t route_all;
     int32_t pad;
 };
 
@@ -128,7 +135,8 @@ cudaError_t launch_timeline(const TraceDev& tr, const GroupConst* gc, const Clas
 cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const Prep* prep, uint32_t P,
                          const uint32_t* pol_list, uint32_t n_list, const Chunk* chunks, uint32_t n_chunks,
                          TimelineRec rec, disco_pair_out_t out, uint64_t* acc, uint64_t* hist_ttft,
-                         uint64_t* hist_tbt, cudaEvent_t mid /* recorded between its two kernels, or null */,
+                         uint64_t* hist_tbt, uint64_t seed, bool extras /* some policy routes at random or uses an
+                         expected length */, cudaEvent_t mid /* recorded between its two kernels, or null */,
                          cudaStream_t st);
 cudaError_t launch_finalize(uint32_t P, int G, const GroupConst* gc, const uint64_t* acc, const uint64_t* hist_ttft,
                             const uint64_t* hist_tbt, const uint64_t* grp_sum_n, const uint32_t* grp_off,

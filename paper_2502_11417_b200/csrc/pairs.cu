@@ -15,7 +15,9 @@ namespace {
 
 struct PairIn {                 // one request and its play-out summaries
     uint32_t l, n, S, m;
-    float saving;               // delta_c * (n - m): Eq. 4's projected saving
+    float saving;               // delta_c * (n - m): Eq. 4's projected saving on the true remainder
+    uint32_t u;                 // the request's routing draw (stochastic baselines only)
+    float delta_c;
 };
 
 struct PairOut {
@@ -23,19 +25,35 @@ struct PairOut {
     uint32_t ttft;
 };
 
+// The request's draw for the stochastic baselines: the jitter hash at the reserved token index 2^32 - 1.
+__device__ __forceinline__ uint32_t routing_draw(uint32_t k0, uint32_t orig) {
+    return mix32(mix32(k0 + orig * kHashReq) + 0xFFFFFFFFu * kHashTok);
+}
+
 // Dispatch and race for one (request, policy); candidate = which winner may migrate in this group.
+// EXT: the policy may be a Stoch-S / Stoch-D baseline or trigger migration on an expected length.
+template <bool EXT>
 __device__ __forceinline__ PairOut decide(const PairIn& q, const Prep& pr, uint32_t Td, int candidate) {
     PairOut o;
     o.dev_only = !pr.device_constrained && (int32_t)q.l < pr.l_th;                 // Algorithm 3
     uint32_t w = 0;                                                                // Algorithm 2's wait map
     if (pr.device_constrained)
         w = (int32_t)q.l < pr.l_star ? 0u : ((int32_t)q.l == pr.l_star ? (uint32_t)pr.w_star : (uint32_t)pr.w_tail);
+    float saving = q.saving;
+    if (EXT) {
+        if (pr.stochastic) {                                                       // constrained endpoint with probability b
+            const bool constrained = pr.route_all || q.u < pr.route_thr;
+            o.dev_only = pr.device_constrained ? constrained : !constrained;
+            w = 0xFFFFFFFFu;                                                       // otherwise the device never starts
+        }
+        if (pr.expected_len) saving = q.delta_c * (float)max((int32_t)pr.expected_len - (int32_t)q.m, 0);
+    }
     o.started = o.dev_only || q.S > w;                                             // the device starts after the wait
     const uint32_t wTd = w + Td;
     o.dev_wins = o.dev_only || (o.started && q.S > wTd);                           // a tie goes to the server
-    o.ttft = o.dev_only ? Td : min(q.S, wTd);
+    o.ttft = o.dev_only ? Td : (EXT && !o.started ? q.S : min(q.S, wTd));
     o.race = o.started && !o.dev_only;
-    o.migr = pr.mig_on && o.race && q.m != 0 && candidate == (o.dev_wins ? 2 : 1) && q.saving > pr.theta;
+    o.migr = pr.mig_on && o.race && q.m != 0 && candidate == (o.dev_wins ? 2 : 1) && saving > pr.theta;
     return o;
 }
 
@@ -53,10 +71,11 @@ __device__ __forceinline__ void hist16_add(uint32_t* row, int bin) {
     atomicAdd(&row[bin >> 1], 1u << ((bin & 1) * 16));
 }
 
+template <bool EXT>
 __global__ void __launch_bounds__(kAccThreads)
 k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __restrict__ ccp,
             const Prep* __restrict__ prep, uint32_t P, const uint32_t* __restrict__ pol_list, uint32_t n_list,
-            int PL, const Chunk* __restrict__ chunks, TimelineRec rec, unsigned long long* __restrict__ acc,
+            int PL, const Chunk* __restrict__ chunks, TimelineRec rec, uint32_t k0, unsigned long long* __restrict__ acc,
             unsigned long long* __restrict__ hist_ttft, unsigned long long* __restrict__ hist_tbt) {
     extern __shared__ uint32_t smem[];
     uint32_t* h_ttft = smem;                                  // [PL][kHWords]
@@ -114,7 +133,8 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
             const float saving = m ? delta_c * (float)(n - m) : -1.0f;
             __syncwarp();
             stage[lane * 3 + 0] = make_uint4(l, n, S, kappa * l + c0);
-            stage[lane * 3 + 1] = make_uint4(m, l + m, __float_as_uint(saving), rec.delayed[kk]);
+            stage[lane * 3 + 1] = make_uint4(m, EXT ? routing_draw(k0, tr.orig[kk]) : l + m, __float_as_uint(saving),
+                                             rec.delayed[kk]);
             stage[lane * 3 + 2] = make_uint4(nt0, nt1, nt2, (uint32_t)stall_bin);
             __syncwarp();
         }
@@ -123,16 +143,25 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
             const int r = r0 + slot;
             if (!act || r >= n_here) continue;
             const uint4 A = stage[r * 3 + 0], Bq = stage[r * 3 + 1], Cq = stage[r * 3 + 2];
-            const uint32_t l = A.x, n = A.y, S = A.z, Td = A.w, m = Bq.x, lm = Bq.y;
-            // ---- dispatch (Algorithm 2's wait map / Algorithm 3's threshold) and the race
-            const bool dev_only = (int32_t)l < l_th;
-            const uint32_t w = (int32_t)l < l_star ? 0u : ((int32_t)l == l_star ? w_star : w_tail);
-            const bool started = dev_only || S > w;                // the device starts after the wait
-            const uint32_t wTd = w + Td;
-            const bool dev_wins = dev_only || (started && S > wTd);   // a tie goes to the server
-            const uint32_t ttft = dev_only ? Td : min(S, wTd);
-            const bool race = started && !dev_only;
-            const bool migr = mig_on && race && candidate == (dev_wins ? 2 : 1) && __uint_as_float(Bq.z) > theta;
+            const uint32_t l = A.x, n = A.y, S = A.z, Td = A.w, m = Bq.x, lm = l + m;
+            bool dev_only, started, dev_wins, race, migr;
+            uint32_t ttft;
+            if (EXT) {
+                PairIn q;
+                q.l = l; q.n = n; q.S = S; q.m = m; q.saving = __uint_as_float(Bq.z); q.u = Bq.y; q.delta_c = delta_c;
+                const PairOut o = decide<true>(q, pr, Td, candidate);
+                dev_only = o.dev_only; started = o.started; dev_wins = o.dev_wins; race = o.race; migr = o.migr; ttft = o.ttft;
+            } else {
+                // ---- dispatch (Algorithm 2's wait map / Algorithm 3's threshold) and the race
+                dev_only = (int32_t)l < l_th;
+                const uint32_t w = (int32_t)l < l_star ? 0u : ((int32_t)l == l_star ? w_star : w_tail);
+                started = dev_only || S > w;                       // the device starts after the wait
+                const uint32_t wTd = w + Td;
+                dev_wins = dev_only || (started && S > wTd);        // a tie goes to the server
+                ttft = dev_only ? Td : min(S, wTd);
+                race = started && !dev_only;
+                migr = mig_on && race && candidate == (dev_wins ? 2 : 1) && __uint_as_float(Bq.z) > theta;
+            }
             const uint32_t tok_src = migr ? m : n;
             c_do += dev_only; c_rc += race; c_dw += race && dev_wins; c_mg += migr;
             a_td += dev_wins ? tok_src : n - tok_src;
@@ -196,10 +225,11 @@ size_t acc_smem_bytes(int PL) {
 constexpr int kRowThreads = 256;
 constexpr int kRowPols = 8;
 
+template <bool EXT>
 __global__ void __launch_bounds__(kRowThreads)
 k_pairs_rows(TraceDev tr, const GroupConst* __restrict__ gcs, const Prep* __restrict__ prep, uint32_t P,
              const uint32_t* __restrict__ pol_list, uint32_t n_list, const Chunk* __restrict__ chunks,
-             TimelineRec rec, disco_pair_out_t out) {
+             TimelineRec rec, uint32_t k0, disco_pair_out_t out) {
     __shared__ Prep s_prep[kRowPols];
     __shared__ uint32_t s_pol[kRowPols];
     const Chunk ch = chunks[blockIdx.x];
@@ -223,12 +253,15 @@ k_pairs_rows(TraceDev tr, const GroupConst* __restrict__ gcs, const Prep* __rest
         PairIn q;
         q.l = tr.l[k]; q.n = tr.nout[k]; q.S = (uint32_t)tr.S[k]; q.m = rec.m[k];
         q.saving = delta_c * (float)(q.n - q.m);
-        const uint32_t orig = tr.orig[k], Td = kappa * q.l + c0, dly = rec.delayed[k];
+        q.delta_c = delta_c;
+        const uint32_t orig = tr.orig[k];
+        q.u = EXT ? routing_draw(k0, orig) : 0u;
+        const uint32_t Td = kappa * q.l + c0, dly = rec.delayed[k];
         const uint32_t sum0 = rec.sum[0][k], sum1 = rec.sum[1][k], sum2 = rec.sum[2][k];
         const uint32_t max0 = rec.max[0][k], max1 = rec.max[1][k], max2 = rec.max[2][k];
         const float inv_cnt = q.n > 1 ? 1e-6f / (float)(q.n - 1) : 0.0f;
         for (int pi = 0; pi < npol; ++pi) {
-            const PairOut o = decide(q, s_prep[pi], Td, candidate);
+            const PairOut o = decide<EXT>(q, s_prep[pi], Td, candidate);
             const uint32_t sum = o.migr ? sum2 : (o.dev_wins ? sum1 : sum0);
             const uint32_t mx = o.migr ? max2 : (o.dev_wins ? max1 : max0);
             const uint32_t lm = q.l + q.m;
@@ -257,15 +290,18 @@ k_pairs_rows(TraceDev tr, const GroupConst* __restrict__ gcs, const Prep* __rest
 cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const Prep* prep, uint32_t P,
                          const uint32_t* pol_list, uint32_t n_list, const Chunk* chunks, uint32_t n_chunks,
                          TimelineRec rec, disco_pair_out_t out, uint64_t* acc, uint64_t* hist_ttft,
-                         uint64_t* hist_tbt, cudaEvent_t mid, cudaStream_t st) {
+                         uint64_t* hist_tbt, uint64_t seed, bool extras, cudaEvent_t mid, cudaStream_t st) {
     if (n_chunks == 0 || n_list == 0) return mid ? cudaEventRecord(mid, st) : cudaSuccess;
     int PL = 1;
     while (PL < 32 && (uint32_t)PL < n_list) PL <<= 1;
-    cudaError_t e = cudaFuncSetAttribute(k_pairs_acc, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    auto* acc_kernel = extras ? k_pairs_acc<true> : k_pairs_acc<false>;
+    auto* row_kernel = extras ? k_pairs_rows<true> : k_pairs_rows<false>;
+    const uint32_t k0 = seed_key(seed);
+    cudaError_t e = cudaFuncSetAttribute(acc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)acc_smem_bytes(32));
     if (e) return e;
     dim3 grid(n_chunks, (n_list + PL - 1) / PL);
-    k_pairs_acc<<<grid, kAccThreads, acc_smem_bytes(PL), st>>>(tr, gc, cc, prep, P, pol_list, n_list, PL, chunks, rec,
+    acc_kernel<<<grid, kAccThreads, acc_smem_bytes(PL), st>>>(tr, gc, cc, prep, P, pol_list, n_list, PL, chunks, rec, k0,
                                                                (unsigned long long*)acc,
                                                                (unsigned long long*)hist_ttft,
                                                                (unsigned long long*)hist_tbt);
@@ -275,7 +311,7 @@ cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassCo
                       out.mig_at || out.delayed || out.decision;
     if (rows) {
         dim3 grid_r(n_chunks, (n_list + kRowPols - 1) / kRowPols);
-        k_pairs_rows<<<grid_r, kRowThreads, 0, st>>>(tr, gc, prep, P, pol_list, n_list, chunks, rec, out);
+        row_kernel<<<grid_r, kRowThreads, 0, st>>>(tr, gc, prep, P, pol_list, n_list, chunks, rec, k0, out);
         e = cudaGetLastError();
     }
     return e;

@@ -39,6 +39,8 @@ __global__ void k_prep(const PolicyConst* __restrict__ pol, uint32_t P, int G, c
     r.l_th = 0; r.l_star = 0; r.w_star = 0; r.w_tail = 0;
     r.theta = pc.theta;
     r.mig_on = (pc.flags & DISCO_FLAG_MIGRATION) ? 1 : 0;
+    r.stochastic = (pc.flags & DISCO_FLAG_STOCHASTIC) ? 1 : 0;
+    r.expected_len = pc.expected_len; r.route_thr = pc.route_thr; r.route_all = pc.route_all;
     r.pad = 0;
 
     if (!r.device_constrained) {

@@ -65,6 +65,20 @@ def test_generation_slower_than_consumption():
     full_parity(w, pols, tag="slow-gen")
 
 
+def test_stochastic_baselines_and_expected_length():
+    # Stoch-S / Stoch-D routing and the expected-length trigger, mixed with ordinary policies in one call
+    STOCH = synth.FLAG_STOCHASTIC
+    pols = [synth.policy(b, flags=STOCH | f | md) for b in (0.0, 0.3, 0.77, 1.0) for f in (PACE, MIG | PACE)
+            for md in (S_MODE, D_MODE, synth.MODE_AUTO)]
+    pols += [synth.policy(b, mig_threshold=th, expected_len=E) for b in (0.4, 1.0) for th in (0.0, 0.02)
+             for E in (0, 5, 64, 128, 4096)]
+    for dear in (False, True):
+        w = synth.tiny_workload(31 + dear, 3000, n_servers=2, n_devices=2, max_prompt=600, max_out=200,
+                                device_dearer=dear)
+        gs, _ = full_parity(w, pols, tag=f"next dear={dear}")
+        assert gs[0].n_race == 0 and gs[3].n_race == 0
+
+
 def test_buffer_search_paths():
     # the hand-off search under clamping (generation sometimes slower than consumption), for shallow
     # buffers, buffers deeper than a warp's delivery-time history, and buffers that never fill
@@ -171,7 +185,8 @@ def test_invalid_inputs_are_rejected():
         assert ei.value.code == -1
     t = load()
     for badpol in [synth.policy(1.5), synth.policy(0.5, alpha=0.0), synth.policy(0.5, mig_threshold=-1.0),
-                   synth.policy(0.5, r_c=0.0), synth.policy(0.5, flags=3 << 2), synth.policy(float("nan"))]:
+                   synth.policy(0.5, r_c=0.0), synth.policy(0.5, flags=3 << 2), synth.policy(0.5, flags=1 << 5),
+                   synth.policy(float("nan"))]:
         with pytest.raises(DiscoError) as ei:
             t.eval_policies([badpol], 0)
         assert ei.value.code == -1
