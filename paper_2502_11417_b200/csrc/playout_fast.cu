@@ -2,8 +2,8 @@
 // no slower than it is consumed (c_j = tau - x_j >= 0 for all j), so delivery is exactly tau-paced.
 //
 // A warp plays four requests at a time and shares its 32 lanes among them in proportion to their token
-// counts (every lane then owns a contiguous run of about the same length, whatever the mix of lengths).  Every token's hash is drawn and mapped to both endpoints' jitter; the lane keeps the sums
-// and maxima.  If any c_j is negative the request is put on a list for the general kernel (playout.cu).
+// counts (every lane then owns a contiguous run of about the same length, whatever the mix of lengths).
+// Every token's hash is drawn and mapped to both endpoints' jitter; the lane keeps the sums and maxima.  If any c_j is negative the request is put on a list for the general kernel (playout.cu).
 // Otherwise:
 //  * streams S and D: every TBT equals tau;
 //  * hand-off index m (buffer holds B tokens: d_{j-B+1} > g_j) is the first j whose prefix sum of c on the

@@ -84,7 +84,7 @@ def budget_grid(k: int) -> List[float]:
     return [float(np.float32(i) / np.float32(k - 1)) for i in range(k)]
 
 
-_SIZES = {0: 1_000, 1: 100_000, 2: 1_000_000, 3: 4_000_000, 4: 16_000_000}
+_SIZES = {0: 1_000, 1: 100_000, 2: 1_000_000, 3: 4_000_000, 4: 16_000_000, 5: 600_000}
 
 
 def make_workload(cfg: int, n: Optional[int] = None, n_budgets: Optional[int] = None,
@@ -94,10 +94,12 @@ def make_workload(cfg: int, n: Optional[int] = None, n_budgets: Optional[int] = 
     ``replica`` > 0 draws an independent trace of the same shape (one per GPU
     in a multi-GPU run)."""
     if cfg not in _SIZES:
-        raise ValueError("cfg must be 0..4")
+        raise ValueError("cfg must be 0..5")
     n = _SIZES[cfg] if n is None else int(n)
     rng = np.random.Generator(np.random.PCG64(cfg if replica == 0 else [cfg, replica]))
 
+    if cfg == 5:
+        return _paper_profiles_workload(rng, n, n_budgets)
     prompt = _lengths(rng, n, 5.5, 1.0, 16, 4096)
     if cfg == 3:
         out = _lengths(rng, n, 6.5, 0.7, 64, 8192)
@@ -149,6 +151,34 @@ def make_workload(cfg: int, n: Optional[int] = None, n_budgets: Optional[int] = 
                     server_ttft_s=ttft, server_profile=sprof, device_profile=dprof,
                     servers=servers, devices=devices, policies=policies, seed=cfg,
                     materialise=cfg in (0, 1), select=select)
+
+
+def _paper_profiles_workload(rng, n, n_budgets) -> Workload:
+    """Workload 5: the paper's own endpoint constants on a synthetic trace.  Devices: the three phone
+    profiles of Sec. 5.1 (prefill/decode tokens/s 31.32/13.93, 51.80/20.14, 79.90/21.47), device cost per
+    token = the model's GFLOPs per token (Table 6: prefill at L=64, decode) priced at two exchange rates so
+    that Algorithm 1 yields a server-constrained and a device-constrained variant of each (the paper's
+    0.3 vs 5 energy_to_money settings, Appendix E); server prices of GPT-4o-mini (Table 8, $ per token);
+    outputs capped at the paper's generation limit 128; short instruction-style prompts.  The server TTFT
+    column is synthetic (the commercial traces are not available)."""
+    prompt = _lengths(rng, n, 3.3, 0.8, 4, 512)
+    out = _lengths(rng, n, 5.0, 0.8, 8, 128)
+    z = rng.normal(0.0, 1.0, size=n)
+    u = rng.random(size=n)
+    mixv = rng.uniform(5.0, 15.0, size=n)
+    ttft = np.where(u < 0.02, mixv, np.exp(-0.5 + 0.9 * z))
+    sprof = np.zeros(n, dtype=np.uint8)
+    dprof = rng.integers(0, 6, size=n).astype(np.uint8)
+    ttft = np.clip(ttft, 1e-3, 600.0).astype(np.float32)
+    servers = [server(jitter=0.20, c_prefill=0.15e-6, c_decode=0.60e-6)]
+    phones = [(31.32, 13.93, 0.93, 0.82), (51.80, 20.14, 0.50, 0.42), (79.90, 21.47, 0.45, 0.37)]
+    devices = [device(pf, dc, jitter=0.05, c_prefill=cp, c_decode=cd, lam=lam)
+               for lam in (0.3e-6, 5.0e-6) for pf, dc, cp, cd in phones]
+    nb = 32 if n_budgets is None else int(n_budgets)
+    policies = [policy(b, mig_threshold=th, expected_len=128) for th in (0.0, INF) for b in budget_grid(nb)]
+    return Workload(name="config5", prompt_len=prompt, output_len=out, server_ttft_s=ttft, server_profile=sprof,
+                    device_profile=dprof, servers=servers, devices=devices, policies=policies, seed=5,
+                    materialise=False, select=dict(cost_cap_factor=1.25, tbt_slo_s=0.25))
 
 
 def tiny_workload(seed: int, n: int, *, n_servers=1, n_devices=1, max_prompt=64, max_out=40,

@@ -39,6 +39,12 @@ def test_config4_shape_six_groups_two_modes():
     assert any(s.n_migrations for s in gs)
 
 
+def test_config5_shape_paper_device_profiles():
+    w = synth.make_workload(5, n=8000, n_budgets=6)
+    gs, _ = full_parity(w, tag="config5-small")
+    assert any(s.n_migrations for s in gs) and any(s.n_device_won for s in gs)
+
+
 @pytest.mark.parametrize("flags", [0, PACE, MIG, MIG | PACE])
 @pytest.mark.parametrize("mode", [S_MODE, D_MODE])
 def test_flag_and_mode_matrix(flags, mode):
