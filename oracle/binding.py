@@ -40,14 +40,16 @@ class device_struct(C.Structure):
 
 class policy_struct(C.Structure):
     _fields_ = [("budget", C.c_float), ("alpha", C.c_float), ("mig_threshold", C.c_float),
-                ("t_m_s", C.c_float), ("r_c", C.c_float), ("flags", C.c_uint32), ("expected_len", C.c_uint32)]
+                ("t_m_s", C.c_float), ("r_c", C.c_float), ("flags", C.c_uint32), ("expected_len", C.c_uint32),
+                ("l_immediate", C.c_uint32)]
 
 
 class prep_struct(C.Structure):
     _fields_ = [("device_constrained", C.c_int32), ("l_th", C.c_int32), ("l_star", C.c_int32), ("B", C.c_int32),
                 ("w_star", C.c_int64), ("w_tail", C.c_int64), ("tau", C.c_int64), ("t_m", C.c_int64),
                 ("candidate_winner", C.c_int32), ("delta_c", C.c_float),
-                ("funded_fraction", C.c_double), ("budget_A", C.c_double)]
+                ("funded_fraction", C.c_double), ("budget_A", C.c_double),
+                ("beta_rule", C.c_int32), ("l_immediate", C.c_int32), ("beta", C.c_int64)]
 
 
 class pair_out_struct(C.Structure):
@@ -135,7 +137,7 @@ def _policies(policies: Sequence[Dict[str, float]]):
     arr = (policy_struct * len(policies))()
     for k, p in enumerate(policies):
         arr[k] = policy_struct(p["budget"], p["alpha"], p["mig_threshold"], p["t_m_s"], p["r_c"], p["flags"],
-                               p.get("expected_len", 0))
+                               p.get("expected_len", 0), p.get("l_immediate", 0))
     return arr
 
 

@@ -114,7 +114,8 @@ int policy_ticks(const orc_policy_t& p, PolicyTicks* o) {
     o->mig = (p.flags & ORC_FLAG_MIGRATION) != 0;
     o->pacing = (p.flags & ORC_FLAG_PACING) != 0;
     o->mode = (int)((p.flags >> 2) & 3);
-    if (o->mode == 3 || (p.flags >> 5)) return fail("unknown flags");
+    if (o->mode == 3 || (p.flags >> 6)) return fail("unknown flags");
+    if (p.l_immediate > ORC_MAX_PROMPT) return fail("l_immediate above the longest prompt");
     /* Eq. 6: B = r_c * t_m tokens, rounded up; nothing to fill without a buffer */
     o->B = o->pacing ? (int32_t)std::min<int64_t>((o->t_m + o->tau - 1) / o->tau, 1 << 30) : 0;
     return 0;
@@ -162,6 +163,36 @@ int prep_group(const orc_trace& tr, const orc_policy_t& p, uint32_t g, orc_prep_
     const double q_tail = 1.0 - std::min(alpha, b);
     out->w_tail = inverse_cdf(G, q_tail);
     out->l_th = 0;
+    if (p.flags & ORC_FLAG_BETA_RULE) {
+        /* Phase 2 as in the body text (Eq. 1-2): w(l) = 0 for l <= l_immediate, min(beta l, w_tail) above.
+         * beta (whole ticks per prompt token) is the smallest one under which the device's expected share
+         * of input tokens, sum_l l cnt[l] P(S > w(l)), stays within b Total.  Counts are kept exact:
+         * share * N = sum_l l cnt[l] #{S > w(l)}. */
+        out->beta_rule = 1;
+        out->l_star = 0; out->w_star = 0;
+        const int64_t beta_hi = out->w_tail + 1;             /* from here on every wait is w_tail */
+        if (b <= alpha) { out->l_immediate = 0; out->beta = beta_hi; return 0; }
+        out->l_immediate = (int32_t)p.l_immediate;
+        const double limit = (b * (double)G.Total) * (double)G.N;
+        auto started_tokens = [&](int64_t beta) {
+            int64_t acc = 0;
+            for (int32_t l = 1; l <= ORC_MAX_PROMPT; ++l) {
+                if (G.cnt[l] == 0) continue;
+                const int64_t w = l <= out->l_immediate ? 0 : std::min(beta * (int64_t)l, out->w_tail);
+                const int64_t later = G.N - (std::upper_bound(G.sorted.begin(), G.sorted.end(), w) - G.sorted.begin());
+                acc += (int64_t)l * G.cnt[l] * later;
+            }
+            return acc;
+        };
+        int64_t lo = 0, hi = beta_hi;                        /* smallest beta in [0, beta_hi] within the limit */
+        if ((double)started_tokens(hi) > limit) { out->beta = beta_hi; return 0; }   /* not even the longest waits fit */
+        while (lo < hi) {
+            const int64_t mid = lo + (hi - lo) / 2;
+            if ((double)started_tokens(mid) <= limit) hi = mid; else lo = mid + 1;
+        }
+        out->beta = lo;
+        return 0;
+    }
     if (b <= alpha) {                 /* every length keeps the maximum wait */
         out->l_star = 0;
         out->w_star = out->w_tail;
@@ -229,7 +260,8 @@ void play(const orc_trace& tr, const orc_policy_t& pol, const orc_prep_t& pr, ui
     } else if (!pr.device_constrained) {
         if (l < pr.l_th) device_only = true;           /* Algorithm 3: short prompts stay on the device */
     } else {
-        w = (l < pr.l_star) ? 0 : (l == pr.l_star) ? pr.w_star : pr.w_tail;   /* Algorithm 2's map W */
+        if (pr.beta_rule) w = l <= pr.l_immediate ? 0 : std::min(pr.beta * (int64_t)l, pr.w_tail);      /* Eq. 1 */
+        else w = (l < pr.l_star) ? 0 : (l == pr.l_star) ? pr.w_star : pr.w_tail;   /* Algorithm 2's map W */
     }
     if (device_only) {
         R->decision = ORC_DEVICE_ONLY; R->server_dispatched = false; R->device_started = true;

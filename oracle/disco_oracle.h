@@ -26,11 +26,11 @@ extern "C" {
 #define ORC_NKNOTS 257
 
 enum { ORC_SERVER_ONLY = 0, ORC_DEVICE_ONLY = 1, ORC_RACE = 2 };
-enum { ORC_FLAG_MIGRATION = 1, ORC_FLAG_PACING = 2, ORC_FLAG_STOCHASTIC = 16 };
+enum { ORC_FLAG_MIGRATION = 1, ORC_FLAG_PACING = 2, ORC_FLAG_STOCHASTIC = 16, ORC_FLAG_BETA_RULE = 32 };
 
 typedef struct { float tbt_s, jitter, c_prefill, c_decode; } orc_server_t;
 typedef struct { float prefill_tps, ttft_intercept_s, decode_tps, jitter, c_prefill, c_decode, lambda; } orc_device_t;
-typedef struct { float budget, alpha, mig_threshold, t_m_s, r_c; uint32_t flags; uint32_t expected_len; } orc_policy_t;
+typedef struct { float budget, alpha, mig_threshold, t_m_s, r_c; uint32_t flags; uint32_t expected_len; uint32_t l_immediate; } orc_policy_t;
 
 /* Dispatch rule of one (group, policy): what Algorithms 1-3 return, plus the
  * constants of the migration controller (Eq. 4-6). */
@@ -45,6 +45,9 @@ typedef struct {
     float   delta_c;             /* Eq. 5 */
     double  funded_fraction;     /* f of the class l_star (Algorithm 2), for tests */
     double  budget_A;            /* funded input tokens beyond the tail share, for tests */
+    int32_t beta_rule;           /* Eq. 1: w(l) = 0 for l <= l_immediate, else min(beta l, w_tail) */
+    int32_t l_immediate;
+    int64_t beta;                /* ticks per prompt token */
 } orc_prep_t;
 
 typedef struct {

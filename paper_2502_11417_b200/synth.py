@@ -26,6 +26,7 @@ FLAG_PACING = 2
 MODE_AUTO = 0 << 2
 MODE_DEVICE_CONSTRAINED = 1 << 2
 MODE_SERVER_CONSTRAINED = 2 << 2
+FLAG_BETA_RULE = 32         # device-constrained phase 2 as in the body text: w(l) = min(beta l, w_tail)
 FLAG_STOCHASTIC = 16        # Stoch-S / Stoch-D baseline: random routing to the constrained endpoint with probability b
 
 INF = float("inf")
@@ -72,9 +73,10 @@ def device(prefill_tps, decode_tps, jitter=0.0, c_prefill=0.2e-3, c_decode=0.2e-
 
 
 def policy(budget, alpha=0.05, mig_threshold=0.0, t_m_s=1.0, r_c=5.0,
-           flags=FLAG_MIGRATION | FLAG_PACING | MODE_AUTO, expected_len=0):
+           flags=FLAG_MIGRATION | FLAG_PACING | MODE_AUTO, expected_len=0, l_immediate=0):
     return dict(budget=float(np.float32(budget)), alpha=alpha,
-                mig_threshold=mig_threshold, t_m_s=t_m_s, r_c=r_c, flags=int(flags), expected_len=int(expected_len))
+                mig_threshold=mig_threshold, t_m_s=t_m_s, r_c=r_c, flags=int(flags), expected_len=int(expected_len),
+                l_immediate=int(l_immediate))
 
 
 def budget_grid(k: int) -> List[float]:

@@ -72,3 +72,60 @@ def test_expected_length_trigger():
             assert list(r["g"]) == list(base["g"]) and list(r["d"]) == list(base["d"])
     st, out = o.eval([synth.policy(1.0, flags=S_MODE | MIG | PACE, expected_len=128)], 0, pairs=True)
     assert out["tok_server"][0, 0] == 6 and out["tok_device"][0, 0] == n - 6
+
+
+def _started_tokens(lens, cnt, srt, l_imm, beta, w_tail):
+    """sum_l l cnt[l] #{S > w(l)} with w(l) = 0 for l <= l_imm, min(beta l, w_tail) above (exact integers)."""
+    acc = 0
+    for l in lens:
+        w = 0 if l <= l_imm else min(beta * int(l), w_tail)
+        acc += int(l) * int(cnt[l]) * int(len(srt) - np.searchsorted(srt, w, side="right"))
+    return acc
+
+
+@pytest.mark.parametrize("l_imm", [0, 40])
+def test_beta_rule_of_eq_1_2(l_imm):
+    BETA = synth.FLAG_BETA_RULE
+    w = synth.make_workload(1, n=3000)
+    tr = vars(w)
+    tr["devices"] = [synth.device(500.0, 20.0, jitter=0.05, c_prefill=5e-3, c_decode=5e-3)]     # device-constrained
+    o = oracle_of(tr)
+    cnt, srt, kn = o.group_tables(0)
+    lens = np.nonzero(cnt)[0]
+    total, N = int((np.arange(4097) * cnt).sum()), len(srt)
+    prev = None
+    for b in [0.0, 0.03, 0.05, 0.1, 0.3, 0.6, 0.9, 1.0]:
+        pol = synth.policy(b, flags=BETA | PACE | D_MODE, l_immediate=l_imm)
+        pr = o.prep(pol)
+        ref = o.prep(synth.policy(b, flags=PACE | D_MODE))
+        assert pr.beta_rule == 1 and pr.device_constrained == 1 and pr.w_tail == ref.w_tail     # phase 1 is shared
+        bf = float(np.float32(b))
+        if bf <= float(np.float32(0.05)):
+            assert pr.beta == pr.w_tail + 1 and pr.l_immediate == 0      # b <= alpha: every prompt waits w_tail
+        else:
+            limit = bf * total * N
+            got = _started_tokens(lens, cnt, srt, l_imm, pr.beta, pr.w_tail)
+            floor_share = _started_tokens(lens, cnt, srt, l_imm, pr.w_tail + 1, pr.w_tail)
+            if floor_share > limit:
+                assert pr.beta == pr.w_tail + 1                          # even the longest waits exceed the budget
+            else:
+                assert got <= limit                                      # the budget holds ...
+                assert pr.beta == 0 or _started_tokens(lens, cnt, srt, l_imm, pr.beta - 1, pr.w_tail) > limit   # ... tightly
+        if prev is not None:
+            assert pr.beta <= prev                                       # more budget, shorter waits
+        prev = pr.beta
+        # the rule as played: wait 0 up to l_immediate, min(beta l, w_tail) above; device starts iff S > w
+        st, out = o.eval([pol], 0, pairs=True)
+        S = np.rint(w.server_ttft_s.astype(np.float64) * 1e6).astype(np.int64)
+        l = w.prompt_len.astype(np.int64)
+        wait = np.where(l <= pr.l_immediate, 0, np.minimum(pr.beta * l, pr.w_tail))
+        assert ((out["decision"][0] == RACE) == (S > wait)).all()
+        assert st[0].prefill_tok_device == int(l[S > wait].sum())
+        if bf > 0.05:
+            # realised share tracks the expectation the rule budgets (S is independent of l in this trace)
+            assert abs(st[0].prefill_tok_device - _started_tokens(lens, cnt, srt, l_imm, pr.beta, pr.w_tail) / N) < 0.03 * total
+    assert o.prep(synth.policy(1.0, flags=BETA | PACE | D_MODE, l_immediate=l_imm)).beta == 0
+    # in the server-constrained mode the flag changes nothing
+    a = o.prep(synth.policy(0.4, flags=BETA | PACE | S_MODE))
+    b_ = o.prep(synth.policy(0.4, flags=PACE | S_MODE))
+    assert a.beta_rule == 0 and a.l_th == b_.l_th
