@@ -51,6 +51,9 @@ extern "C" {
 #define DISCO_FLAG_PACING 2u     /* delivery buffer: tokens handed over no faster than r_c */
 #define DISCO_FLAG_STOCHASTIC 16u /* Stoch-S / Stoch-D baseline (Sec. 5.1): each request goes to the constrained
                                     endpoint with probability b, else to the other one; no race, no migration */
+#define DISCO_FLAG_BETA_RULE 32u  /* device-constrained phase 2 as in Sec. 4.2, Eq. 1-2: wait 0 for prompts up to
+                                    l_immediate, min(beta l, w_tail) above, beta the smallest whole number of ticks
+                                    per prompt token that keeps the device's expected input-token share within b */
 #define DISCO_MODE_AUTO (0u << 2)               /* Algorithm 1 decides from the costs */
 #define DISCO_MODE_DEVICE_CONSTRAINED (1u << 2) /* force Algorithm 2 */
 #define DISCO_MODE_SERVER_CONSTRAINED (2u << 2) /* force Algorithm 3 */
@@ -101,6 +104,7 @@ typedef struct {
     uint32_t flags;        /* DISCO_FLAG_* | DISCO_MODE_* */
     uint32_t expected_len; /* Eq. 4's remaining length: 0 = the trace's true remainder n - m; else what is left of
                               this expected total output length, max(expected_len - m, 0) */
+    uint32_t l_immediate;  /* DISCO_FLAG_BETA_RULE: prompts up to this length start the device at once (Eq. 1's l_th) */
 } disco_policy_t;
 
 /* Optional per-pair outputs, device memory, each [P][n] with requests
@@ -131,6 +135,9 @@ typedef struct {
     int32_t l_star;               /* Algorithm 2: shorter prompts wait 0, this length waits w_star, longer ones w_tail */
     int32_t B;                    /* Eq. 6 buffer, tokens */
     int64_t w_star, w_tail, tau;  /* ticks (microseconds) */
+    int32_t beta_rule;            /* Eq. 1-2 variant in force (device-constrained groups of DISCO_FLAG_BETA_RULE policies) */
+    int32_t l_immediate;          /* its immediate-start threshold (0 when b <= alpha) */
+    int64_t beta;                 /* its slope, ticks per prompt token */
 } disco_prep_t;
 
 typedef struct disco_ctx disco_ctx_t;

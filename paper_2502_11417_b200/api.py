@@ -44,7 +44,7 @@ class TraceDesc(C.Structure):
 
 class Policy(C.Structure):
     _fields_ = [("budget", C.c_float), ("alpha", C.c_float), ("mig_threshold", C.c_float), ("t_m_s", C.c_float),
-                ("r_c", C.c_float), ("flags", C.c_uint32), ("expected_len", C.c_uint32)]
+                ("r_c", C.c_float), ("flags", C.c_uint32), ("expected_len", C.c_uint32), ("l_immediate", C.c_uint32)]
 
 
 class PairOut(C.Structure):
@@ -69,7 +69,8 @@ class PolicyStats(C.Structure):
 
 class Prep(C.Structure):
     _fields_ = [("device_constrained", C.c_int32), ("l_th", C.c_int32), ("l_star", C.c_int32), ("B", C.c_int32),
-                ("w_star", C.c_int64), ("w_tail", C.c_int64), ("tau", C.c_int64)]
+                ("w_star", C.c_int64), ("w_tail", C.c_int64), ("tau", C.c_int64),
+                ("beta_rule", C.c_int32), ("l_immediate", C.c_int32), ("beta", C.c_int64)]
 
 
 EXPORTS = ["disco_load_trace", "disco_eval_policies", "disco_reduce_stats", "disco_select_policy",
@@ -155,7 +156,7 @@ def policy_array(policies: Sequence[Dict[str, float]]):
     arr = (Policy * len(policies))()
     for k, p in enumerate(policies):
         arr[k] = Policy(p["budget"], p["alpha"], p["mig_threshold"], p["t_m_s"], p["r_c"], p["flags"],
-                        p.get("expected_len", 0))
+                        p.get("expected_len", 0), p.get("l_immediate", 0))
     return arr
 
 

@@ -268,6 +268,7 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
     // ---- policy constants and timeline classes
     std::vector<PolicyConst> pc(P);
     std::vector<ClassConst> classes;
+    bool any_beta = false;                // some policy uses the Eq. 1-2 wait rule
     bool cls_extras_pending = false;      // some policy routes at random or triggers on an expected length
     for (uint32_t p = 0; p < P; ++p) {
         const disco_policy_t& q = pol[p];
@@ -278,8 +279,9 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
         if (!(q.r_c > 0.0f) || !std::isfinite(q.r_c)) return fail(DISCO_EINVAL, "consumption rate must be positive" + at);
         if (!(q.t_m_s >= 0.0f) || !std::isfinite(q.t_m_s)) return fail(DISCO_EINVAL, "migration time must be >= 0" + at);
         const uint32_t mode = (q.flags >> 2) & 3u;
-        if (mode == 3 || (q.flags >> 5)) return fail(DISCO_EINVAL, "unknown flags" + at);
+        if (mode == 3 || (q.flags >> 6)) return fail(DISCO_EINVAL, "unknown flags" + at);
         if (q.expected_len > (1u << 20)) return fail(DISCO_EINVAL, "expected length too large" + at);
+        if (q.l_immediate > (uint32_t)kMaxPrompt) return fail(DISCO_EINVAL, "l_immediate above the longest prompt" + at);
         const int64_t tau = ticks_of_rate(q.r_c), t_m = ticks_of_seconds(q.t_m_s);
         if (tau < 1 || tau >= (1 << 30)) return fail(DISCO_EINVAL, "consumption interval outside 1 .. 2^30 ticks" + at);
         const bool pacing = (q.flags & DISCO_FLAG_PACING) != 0, mig = (q.flags & DISCO_FLAG_MIGRATION) != 0;
@@ -288,10 +290,11 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
         PolicyConst& o = pc[p];
         o.budget = q.budget; o.alpha = q.alpha; o.theta = q.mig_threshold; o.flags = q.flags;
         o.tau = (int32_t)tau; o.B = (int32_t)B; o.mode = (int32_t)mode;
-        o.expected_len = q.expected_len; o.pad = 0;
+        o.expected_len = q.expected_len; o.l_immediate = q.l_immediate;
+        if (q.flags & DISCO_FLAG_BETA_RULE) any_beta = true;
         o.route_all = q.budget >= 1.0f ? 1 : 0;
         o.route_thr = o.route_all ? 0xFFFFFFFFu : (uint32_t)std::floor((double)q.budget * 4294967296.0);
-        if ((q.flags & DISCO_FLAG_STOCHASTIC) || q.expected_len) cls_extras_pending = true;
+        if ((q.flags & (DISCO_FLAG_STOCHASTIC | DISCO_FLAG_BETA_RULE)) || q.expected_len) cls_extras_pending = true;
         int cls = -1;
         for (size_t k = 0; k < classes.size(); ++k)
             if (classes[k].tau == o.tau && classes[k].B == o.B && classes[k].pacing == (int)pacing) { cls = (int)k; break; }
@@ -410,6 +413,11 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
     // ---- Algorithms 1-3 for every (group, policy)
     CU(launch_prep(c->d_pol.as<PolicyConst>(), P, G, c->d_gc.as<GroupConst>(), c->cum_mass.as<int64_t>(),
                    c->cnt, c->sorted.as<int32_t>(), c->grp_off.as<uint32_t>(), c->d_prep.as<Prep>(), st));
+    if (any_beta) {
+        CU(launch_prep_beta(c->d_pol.as<PolicyConst>(), P, G, c->cum_mass.as<int64_t>(), c->cnt, c->sorted.as<int32_t>(),
+                            c->grp_off.as<uint32_t>(), c->d_prep.as<Prep>(), st));
+        g_launches += 1;
+    }
 
     TraceDev tr;
     tr.n = n; tr.n_groups = G; tr.S = c->S.as<int32_t>(); tr.l = c->l.as<uint16_t>(); tr.nout = c->nout.as<uint16_t>();
@@ -525,6 +533,8 @@ int disco_get_prep(disco_ctx_t* c, uint32_t g, uint32_t p, disco_prep_t* out, vo
     CU(cudaStreamSynchronize(st));
     out->device_constrained = pr.device_constrained; out->l_th = pr.l_th; out->l_star = pr.l_star;
     out->B = c->pol[p].B; out->w_star = pr.w_star; out->w_tail = pr.w_tail; out->tau = c->pol[p].tau;
+    out->beta_rule = pr.beta_rule; out->l_immediate = pr.beta_rule ? pr.l_star : 0; out->beta = pr.beta_rule ? pr.w_star : 0;
+    if (pr.beta_rule) { out->l_star = 0; out->w_star = 0; }
     return 0;
 }
 

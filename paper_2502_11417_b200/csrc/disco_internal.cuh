@@ -36,7 +36,7 @@ struct PolicyConst {
     uint32_t expected_len;       // 0 = true remainder in the migration trigger
     uint32_t route_thr;          // stochastic routing: constrained endpoint iff hash < route_thr (or route_all)
     int32_t route_all;
-    int32_t pad;
+    uint32_t l_immediate;        // Eq. 1's immediate-start threshold (beta rule)
 };
 
 // ---- what Algorithms 1-3 produce for one (group, policy) ----
@@ -50,7 +50,7 @@ struct Prep {
     int32_t stochastic;          // random routing instead of Algorithms 2-3
     uint32_t expected_len, route_thr;
     int32_t route_all;
-    int32_t pad;
+    int32_t beta_rule;           // Eq. 1-2 variant: l_star holds the immediate-start threshold, w_star the slope beta
 };
 
 // ---- a timeline class: the parameters a play-out depends on besides the request ----
@@ -128,6 +128,8 @@ int set_error(int code, const char* msg);
 cudaError_t launch_prep(const PolicyConst* pol, uint32_t P, int G, const GroupConst* gc, const int64_t* cum_mass,
                         const uint32_t* cnt, const int32_t* sorted, const uint32_t* grp_off, Prep* prep,
                         cudaStream_t st);
+cudaError_t launch_prep_beta(const PolicyConst* pol, uint32_t P, int G, const int64_t* cum_mass, const uint32_t* cnt,
+                             const int32_t* sorted, const uint32_t* grp_off, Prep* prep, cudaStream_t st);
 cudaError_t launch_timeline(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, bool pacing,
                             const int32_t* knots, uint64_t seed, TimelineRec rec, int32_t* err, uint32_t* todo,
                             uint32_t* todo_count /* zero on entry */, cudaEvent_t mid /* recorded between its two kernels, or null */,

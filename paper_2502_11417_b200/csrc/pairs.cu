@@ -46,6 +46,9 @@ __device__ __forceinline__ PairOut decide(const PairIn& q, const Prep& pr, uint3
             o.dev_only = pr.device_constrained ? constrained : !constrained;
             w = 0xFFFFFFFFu;                                                       // otherwise the device never starts
         }
+        if (pr.beta_rule)                                                          // Eq. 1: min(beta l, w_tail) above l_immediate
+            w = (int32_t)q.l <= pr.l_star ? 0u : (uint32_t)min((unsigned long long)(uint32_t)pr.w_star * q.l,
+                                                               (unsigned long long)(uint32_t)pr.w_tail);
         if (pr.expected_len) saving = q.delta_c * (float)max((int32_t)pr.expected_len - (int32_t)q.m, 0);
     }
     o.started = o.dev_only || q.S > w;                                             // the device starts after the wait

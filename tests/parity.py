@@ -61,6 +61,8 @@ def check_prep(tr, orc, policies, tag=""):
             assert a.tau == b.tau and a.B == min(b.B, 8192), (tag, g, p)
             if a.device_constrained:
                 assert (a.l_star, a.w_star, a.w_tail) == (b.l_star, b.w_star, b.w_tail), (tag, g, p)
+                assert (a.beta_rule, a.l_immediate, a.beta) == (b.beta_rule, b.l_immediate, b.beta), \
+                    (tag, g, p, (a.beta_rule, a.l_immediate, a.beta), (b.beta_rule, b.l_immediate, b.beta))
             else:
                 assert a.l_th == b.l_th, (tag, g, p, a.l_th, b.l_th)
 

@@ -85,6 +85,23 @@ def test_stochastic_baselines_and_expected_length():
         assert gs[0].n_race == 0 and gs[3].n_race == 0
 
 
+def test_linear_wait_rule():
+    # Eq. 1-2: waits min(beta l, w_tail) with an immediate-start threshold, beside Algorithm 2's policies
+    BETA = synth.FLAG_BETA_RULE
+    pols = [synth.policy(b, flags=BETA | f | md, l_immediate=li)
+            for b in (0.0, 0.03, 0.05, 0.2, 0.5, 0.9, 1.0) for li in (0, 40, 4096)
+            for f, md in ((PACE, D_MODE), (MIG | PACE, synth.MODE_AUTO), (MIG, S_MODE))]
+    pols += [synth.policy(b, flags=MIG | PACE | D_MODE) for b in (0.2, 0.9)]
+    for dear in (False, True):
+        w = synth.tiny_workload(41 + dear, 3000, n_servers=2, n_devices=2, max_prompt=600, max_out=200,
+                                device_dearer=dear)
+        full_parity(w, pols, tag=f"beta dear={dear}")
+    # one group at a workload's own length mix, so that the slope search runs over a full length histogram
+    w = synth.make_workload(1, n=20000, n_budgets=4)
+    full_parity(w, [synth.policy(b, flags=BETA | MIG | PACE | D_MODE, l_immediate=li)
+                    for b in (0.1, 0.4, 0.8) for li in (0, 64)], tag="beta workload1")
+
+
 def test_buffer_search_paths():
     # the hand-off search under clamping (generation sometimes slower than consumption), for shallow
     # buffers, buffers deeper than a warp's delivery-time history, and buffers that never fill
@@ -191,7 +208,8 @@ def test_invalid_inputs_are_rejected():
         assert ei.value.code == -1
     t = load()
     for badpol in [synth.policy(1.5), synth.policy(0.5, alpha=0.0), synth.policy(0.5, mig_threshold=-1.0),
-                   synth.policy(0.5, r_c=0.0), synth.policy(0.5, flags=3 << 2), synth.policy(0.5, flags=1 << 5),
+                   synth.policy(0.5, r_c=0.0), synth.policy(0.5, flags=3 << 2), synth.policy(0.5, flags=1 << 6),
+                       synth.policy(0.5, flags=synth.FLAG_BETA_RULE, l_immediate=4097),
                    synth.policy(float("nan"))]:
         with pytest.raises(DiscoError) as ei:
             t.eval_policies([badpol], 0)
