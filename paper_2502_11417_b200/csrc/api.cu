@@ -366,7 +366,17 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
         cls_range.push_back({b, (uint32_t)pol_list.size()});
     }
     const uint32_t tiles = (P + 31) / 32;
-    const uint32_t want_chunks = std::max<uint32_t>(1, 148 / std::min<uint32_t>(tiles, 148));   // one block per SM
+    uint32_t want_chunks = std::max<uint32_t>(1, 148 / std::min<uint32_t>(tiles, 148));   // one block per SM
+    const uint32_t min_chunks = (uint32_t)((N1 + 65279) / 65280);
+    if (min_chunks > want_chunks) {
+        // several waves of blocks: pick the chunk count near the minimum whose last wave is fullest
+        double best = 0.0;
+        for (uint32_t k = min_chunks; k < min_chunks + 148; ++k) {
+            const uint64_t blocks = (uint64_t)k * tiles, waves = (blocks + 147) / 148;
+            const double fill = (double)blocks / (double)(waves * 148);
+            if (fill > best + 1e-9) { best = fill; want_chunks = k; }
+        }
+    }
     uint32_t CH = (uint32_t)((N1 + want_chunks - 1) / want_chunks);
     CH = (CH + 255) / 256 * 256;
     CH = std::min<uint32_t>(std::max<uint32_t>(CH, 256), 65280);     // 16-bit histogram counters per block

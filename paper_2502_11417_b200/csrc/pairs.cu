@@ -62,20 +62,30 @@ __device__ __forceinline__ PairOut decide(const PairIn& q, const Prep& pr, uint3
 
 // ------------------------------------------------------------------------------------------------------
 // Reductions: lane = policy.
+//
+// A pair ends in one of six outcomes, and everything it adds to the sums depends on the request and the
+// outcome only.  The lane that loads a request therefore writes, once, one row of addends per outcome into
+// shared memory; a policy lane decides the outcome and adds the row it selects.
 // ------------------------------------------------------------------------------------------------------
-constexpr int kAccThreads = 512;         // one block per SM: its histograms take about half the shared memory
+constexpr int kAccThreads = 512;         // one block per SM: histograms and staging fill its shared memory
 constexpr int kAccWarps = kAccThreads / 32;
 constexpr int kHWords = 433;            // 866 sixteen-bit counters per policy row; odd word stride
+constexpr int kStageVec = 7;            // uint4 per request in each of the two staging blocks (odd: no bank conflicts)
+
+enum Outcome { O_SERVER_ONLY = 0, O_DEVICE_ONLY = 1, O_RACE_SRV = 2, O_RACE_DEV = 3, O_MIGR_TO_DEV = 4, O_MIGR_TO_SRV = 5 };
 
 // words in front of the staging area: two histograms and the sums, rounded up to 16 bytes
 __host__ __device__ constexpr int acc_stage_offset_words(int PL) { return (2 * PL * kHWords + 2 * PL * kNAcc + 3) / 4 * 4; }
 
-__device__ __forceinline__ void hist16_add(uint32_t* row, int bin) {
-    atomicAdd(&row[bin >> 1], 1u << ((bin & 1) * 16));
+// A histogram increment as one word: byte offset of the counter pair in bits 2..11, the increment (low or
+// high sixteen bits) in bits 0 and 16.
+__device__ __forceinline__ uint32_t hist16_code(int bin) { return ((uint32_t)(bin >> 1) << 2) | ((bin & 1) ? 0x10000u : 1u); }
+__device__ __forceinline__ void hist16_apply(uint32_t* row, uint32_t code) {
+    atomicAdd((uint32_t*)((char*)row + (code & 0xFFCu)), code & 0x10001u);
 }
 
 template <bool EXT>
-__global__ void __launch_bounds__(kAccThreads)
+__global__ void __launch_bounds__(kAccThreads, 1)
 k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __restrict__ ccp,
             const Prep* __restrict__ prep, uint32_t P, const uint32_t* __restrict__ pol_list, uint32_t n_list,
             int PL, const Chunk* __restrict__ chunks, TimelineRec rec, uint32_t k0, unsigned long long* __restrict__ acc,
@@ -104,56 +114,79 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
     const uint32_t tau = (uint32_t)cc.tau;
 
     for (int i = threadIdx.x; i < 2 * PL * kHWords + 2 * PL * kNAcc; i += kAccThreads) smem[i] = 0;   // (staging needs no clearing)
-    __syncthreads();
+    // With no waits in the tile (Algorithm 3, random routing) a TTFT is the request's S or its T_d, whose
+    // histogram increments are staged; otherwise the bin is worked out per pair.
+    const bool waits = __syncthreads_or(act && pr.device_constrained && !pr.stochastic) != 0;
     uint32_t* my_ttft = h_ttft + pol_in_tile * kHWords;
     uint32_t* my_stall = h_stall + pol_in_tile * kHWords;
 
-    uint32_t c_do = 0, c_rc = 0, c_dw = 0, c_mg = 0, a_td = 0, a_ps = 0, a_pd = 0, a_dl = 0, a_tau = 0;
+    uint32_t a_td = 0, a_ps = 0, a_pd = 0, a_dl = 0, a_tau = 0;
+    uint32_t cnt_a = 0, cnt_b = 0;                              // device-only | race << 16,  device won | migrated << 16
     unsigned long long a_tt = 0;
 
-    // Per-request values are worked out once per request by the lane that loaded it and staged in shared
-    // memory; the policy lanes then read them as broadcasts.
-    uint4* stage = (uint4*)(smem + acc_stage_offset_words(PL)) + wib * 32 * 3;     // [warp][32 requests][3 x uint4]
+    // [warp][32 requests][kStageVec]: block A = the request, then the first half of each outcome's row;
+    // block B = the second halves, then the stall increment and what only the extended policies read.
+    uint4* stA = (uint4*)(smem + acc_stage_offset_words(PL)) + wib * 32 * kStageVec;
+    uint4* stB = stA + kAccWarps * 32 * kStageVec;
     // The wait map without mode tests: Algorithm 3 has no waits (l_star beyond every length), Algorithm 2 no
     // device-only prompts (l_th = 0, as the preparation kernel leaves it).
     const int32_t l_th = pr.l_th, l_star = pr.device_constrained ? pr.l_star : 0x7FFFFFFF;
     const uint32_t w_star = (uint32_t)pr.w_star, w_tail = (uint32_t)pr.w_tail;
-    const float theta = pr.theta;
-    const bool mig_on = pr.mig_on != 0;
+    // Which race winner may migrate is a property of the group; a policy without migration never passes.
+    const float theta = (pr.mig_on && candidate != 0) ? pr.theta : __int_as_float(0x7F800000);
+    const bool dev_migrates = candidate == 2;
 
     for (uint32_t b0 = wib * 32u; b0 < ch.len; b0 += kAccWarps * 32u) {
         // ---- 32 requests, one per lane
+        __syncwarp();
         {
             const uint32_t kk = ch.start + min(b0 + lane, ch.len - 1);
             const uint32_t l = tr.l[kk], n = tr.nout[kk], S = (uint32_t)tr.S[kk], m = rec.m[kk];
-            const uint32_t stall = rec.stall[kk];
+            const uint32_t stall = rec.stall[kk], dly = rec.delayed[kk];
             const uint32_t nt0 = kt0 >= 0 ? rec.win[0][(size_t)kk * W0 + kt0] : 0u;
             const uint32_t nt1 = kt1 >= 0 ? rec.win[1][(size_t)kk * W1 + kt1] : 0u;
             uint32_t nt2 = kt2 >= 0 ? rec.win[2][(size_t)kk * W2 + kt2] : 0u;
-            int stall_bin = -1;                                // the token after a hand-off: counted with tau's bin
-            if (stall == tau) ++nt2; else stall_bin = bin_of_ticks(stall);
+            uint32_t stall_code = 0xFFFFFFFFu;                 // the token after a hand-off: counted with tau's bin
+            if (stall == tau) ++nt2; else stall_code = hist16_code(bin_of_ticks(stall));
             // a request may only migrate if its buffer filled (m != 0); fold that into the saving (Eq. 4)
             const float saving = m ? delta_c * (float)(n - m) : -1.0f;
-            __syncwarp();
-            stage[lane * 3 + 0] = make_uint4(l, n, S, kappa * l + c0);
-            stage[lane * 3 + 1] = make_uint4(m, EXT ? routing_draw(k0, tr.orig[kk]) : l + m, __float_as_uint(saving),
-                                             rec.delayed[kk]);
-            stage[lane * 3 + 2] = make_uint4(nt0, nt1, nt2, (uint32_t)stall_bin);
-            __syncwarp();
+            const uint32_t Td = kappa * l + c0, lm = l + m;
+            const uint32_t hS = hist16_code(bin_of_ticks(S)), hT = hist16_code(bin_of_ticks(Td));
+            uint4* a = stA + lane * kStageVec;
+            uint4* b = stB + lane * kStageVec;
+            a[0] = make_uint4(l, S, Td, __float_as_uint(saving));
+            //                      tokens on device, server prefill, device prefill, TBTs in tau's bin
+            a[1 + O_SERVER_ONLY] = make_uint4(0u, l, 0u, nt0);
+            a[1 + O_DEVICE_ONLY] = make_uint4(n, 0u, l, nt1);
+            a[1 + O_RACE_SRV] = make_uint4(0u, l, l, nt0);
+            a[1 + O_RACE_DEV] = make_uint4(n, l, l, nt1);
+            a[1 + O_MIGR_TO_DEV] = make_uint4(n - m, l, l + lm, nt2);
+            a[1 + O_MIGR_TO_SRV] = make_uint4(m, l + lm, l, nt2);
+            //                      delayed tokens, counts, counts, TTFT increment
+            b[O_SERVER_ONLY] = make_uint4(0u, 0u, 0u, hS);
+            b[O_DEVICE_ONLY] = make_uint4(0u, 1u, 0u, hT);
+            b[O_RACE_SRV] = make_uint4(0u, 0x10000u, 0u, hS);
+            b[O_RACE_DEV] = make_uint4(0u, 0x10000u, 1u, hT);
+            b[O_MIGR_TO_DEV] = make_uint4(dly, 0x10000u, 0x10000u, hS);
+            b[O_MIGR_TO_SRV] = make_uint4(dly, 0x10000u, 0x10001u, hT);
+            b[6] = make_uint4(stall_code, EXT ? routing_draw(k0, tr.orig[kk]) : 0u, m, n);
         }
+        __syncwarp();
         const int n_here = (int)min(32u, ch.len - b0);
+#pragma unroll 2
         for (int r0 = 0; r0 < n_here; r0 += slots) {
             const int r = r0 + slot;
-            if (!act || r >= n_here) continue;
-            const uint4 A = stage[r * 3 + 0], Bq = stage[r * 3 + 1], Cq = stage[r * 3 + 2];
-            const uint32_t l = A.x, n = A.y, S = A.z, Td = A.w, m = Bq.x, lm = l + m;
-            bool dev_only, started, dev_wins, race, migr;
+            if (r >= n_here) continue;
+            const uint4 Q = stA[r * kStageVec];
+            const uint32_t l = Q.x, S = Q.y, Td = Q.z;
+            bool dev_only, started, dev_wins, migr;
             uint32_t ttft;
             if (EXT) {
+                const uint4 X = stB[r * kStageVec + 6];
                 PairIn q;
-                q.l = l; q.n = n; q.S = S; q.m = m; q.saving = __uint_as_float(Bq.z); q.u = Bq.y; q.delta_c = delta_c;
+                q.l = l; q.n = X.w; q.S = S; q.m = X.z; q.saving = __uint_as_float(Q.w); q.u = X.y; q.delta_c = delta_c;
                 const PairOut o = decide<true>(q, pr, Td, candidate);
-                dev_only = o.dev_only; started = o.started; dev_wins = o.dev_wins; race = o.race; migr = o.migr; ttft = o.ttft;
+                dev_only = o.dev_only; started = o.started; dev_wins = o.dev_wins; migr = o.migr; ttft = o.ttft;
             } else {
                 // ---- dispatch (Algorithm 2's wait map / Algorithm 3's threshold) and the race
                 dev_only = (int32_t)l < l_th;
@@ -162,20 +195,20 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
                 const uint32_t wTd = w + Td;
                 dev_wins = dev_only || (started && S > wTd);        // a tie goes to the server
                 ttft = dev_only ? Td : min(S, wTd);
-                race = started && !dev_only;
-                migr = mig_on && race && candidate == (dev_wins ? 2 : 1) && __uint_as_float(Bq.z) > theta;
+                migr = started && !dev_only && dev_wins == dev_migrates && __uint_as_float(Q.w) > theta;
             }
-            const uint32_t tok_src = migr ? m : n;
-            c_do += dev_only; c_rc += race; c_dw += race && dev_wins; c_mg += migr;
-            a_td += dev_wins ? tok_src : n - tok_src;
-            a_ps += (dev_only ? 0u : l) + ((migr && dev_wins) ? lm : 0u);
-            a_pd += (started ? l : 0u) + ((migr && !dev_wins) ? lm : 0u);
-            a_dl += migr ? Bq.w : 0u;
+            const int oc = dev_only ? O_DEVICE_ONLY : (!started ? O_SERVER_ONLY : (dev_wins ? O_RACE_DEV : O_RACE_SRV) + (migr ? 2 : 0));
+            const uint4 h1 = stA[r * kStageVec + 1 + oc], h2 = stB[r * kStageVec + oc];
+            a_td += h1.x; a_ps += h1.y; a_pd += h1.z; a_tau += h1.w;
+            a_dl += h2.x; cnt_a += h2.y; cnt_b += h2.z;
             a_tt += ttft;
-            a_tau += migr ? Cq.z : (dev_wins ? Cq.y : Cq.x);
-            hist16_add(my_ttft, bin_of_ticks(ttft));
-            if (migr && (int32_t)Cq.w >= 0) hist16_add(my_stall, (int)Cq.w);
-            if (wide) {                                        // regular TBTs outside the bin of tau
+            if (waits) hist16_apply(my_ttft, hist16_code(bin_of_ticks(ttft)));
+            else hist16_apply(my_ttft, h2.w);
+            if (migr) {
+                const uint32_t sc = stB[r * kStageVec + 6].x;
+                if ((int32_t)sc >= 0) hist16_apply(my_stall, sc);
+            }
+            if (wide && act) {                                 // regular TBTs outside the bin of tau
                 const int c = migr ? 2 : (dev_wins ? 1 : 0);
                 const int W = c == 2 ? W2 : (c == 1 ? W1 : W0), kt = c == 2 ? kt2 : (c == 1 ? kt1 : kt0);
                 const uint32_t* wp = rec.win[c] + (size_t)(ch.start + b0 + r) * W;
@@ -190,8 +223,8 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
     // ---- block totals, then one flush per block
     if (act) {
         unsigned long long* a = s_acc + pol_in_tile * kNAcc;
-        atomicAdd(&a[A_DEVICE_ONLY], (unsigned long long)c_do); atomicAdd(&a[A_RACE], (unsigned long long)c_rc);
-        atomicAdd(&a[A_DEVICE_WON], (unsigned long long)c_dw); atomicAdd(&a[A_MIGR], (unsigned long long)c_mg);
+        atomicAdd(&a[A_DEVICE_ONLY], (unsigned long long)(cnt_a & 0xFFFFu)); atomicAdd(&a[A_RACE], (unsigned long long)(cnt_a >> 16));
+        atomicAdd(&a[A_DEVICE_WON], (unsigned long long)(cnt_b & 0xFFFFu)); atomicAdd(&a[A_MIGR], (unsigned long long)(cnt_b >> 16));
         atomicAdd(&a[A_TOK_DEVICE], (unsigned long long)a_td); atomicAdd(&a[A_PRE_SERVER], (unsigned long long)a_ps);
         atomicAdd(&a[A_PRE_DEVICE], (unsigned long long)a_pd); atomicAdd(&a[A_DELAYED], (unsigned long long)a_dl);
         atomicAdd(&a[A_TTFT_SUM], a_tt); atomicAdd(&a[A_TAU_CNT], (unsigned long long)a_tau);
@@ -219,7 +252,7 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
 }
 
 size_t acc_smem_bytes(int PL) {
-    return sizeof(uint32_t) * acc_stage_offset_words(PL) + (size_t)kAccWarps * 32 * 3 * sizeof(uint4);
+    return sizeof(uint32_t) * acc_stage_offset_words(PL) + (size_t)kAccWarps * 32 * 2 * kStageVec * sizeof(uint4);
 }
 
 // ------------------------------------------------------------------------------------------------------
