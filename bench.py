@@ -63,7 +63,7 @@ class ClockSampler:
     def __init__(self, index):
         import threading
         self.index, self.samples, self.reasons, self.max_mhz = int(index), [], set(), None
-        self._stop = threading.Event()
+        self._stop, self._ready = threading.Event(), threading.Event()
         self._thread = threading.Thread(target=self._run, daemon=True)
         self.error = None
 
@@ -79,13 +79,17 @@ class ClockSampler:
                 for bit, name in self.REASONS.items():
                     if mask & bit:
                         self.reasons.add(name)
+                self._ready.set()
                 if self._stop.wait(0.02):
                     break
         except Exception as e:                      # no NVML: report that rather than invent numbers
             self.error = repr(e)
+            self._ready.set()
 
     def start(self):
+        """Returns once the first sample is in, so that opening NVML stays outside the timed region."""
         self._thread.start()
+        self._ready.wait(timeout=60)
 
     def stop(self):
         self._stop.set()

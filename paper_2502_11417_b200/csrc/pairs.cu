@@ -7,6 +7,8 @@
 //    stalls are block-private in shared memory (16-bit counters, two per word).
 //  * k_pairs_rows -- the optional per-pair arrays.  A lane owns a request and walks the policies, so each
 //    store instruction writes 32 consecutive requests of one policy row.
+#include <type_traits>
+
 #include "disco_internal.cuh"
 
 namespace disco {
@@ -70,6 +72,7 @@ __device__ __forceinline__ PairOut decide(const PairIn& q, const Prep& pr, uint3
 constexpr int kAccThreads = 512;         // one block per SM: histograms and staging fill its shared memory
 constexpr int kAccWarps = kAccThreads / 32;
 constexpr int kHWords = 433;            // 866 sixteen-bit counters per policy row; odd word stride
+constexpr int kIlp = 4;                 // requests a lane works on at a time
 constexpr int kStageVec = 7;            // uint4 per request in each of the two staging blocks (odd: no bank conflicts)
 
 enum Outcome { O_SERVER_ONLY = 0, O_DEVICE_ONLY = 1, O_RACE_SRV = 2, O_RACE_DEV = 3, O_MIGR_TO_DEV = 4, O_MIGR_TO_SRV = 5 };
@@ -135,6 +138,7 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
     // Which race winner may migrate is a property of the group; a policy without migration never passes.
     const float theta = (pr.mig_on && candidate != 0) ? pr.theta : __int_as_float(0x7F800000);
     const bool dev_migrates = candidate == 2;
+    const uint32_t lth16 = (uint32_t)max(l_th, 0) << 4;      // against a staged (l << 4 | outcome at w = 0)
 
     for (uint32_t b0 = wib * 32u; b0 < ch.len; b0 += kAccWarps * 32u) {
         // ---- 32 requests, one per lane
@@ -154,7 +158,15 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
             const uint32_t hS = hist16_code(bin_of_ticks(S)), hT = hist16_code(bin_of_ticks(Td));
             uint4* a = stA + lane * kStageVec;
             uint4* b = stB + lane * kStageVec;
-            a[0] = make_uint4(l, S, Td, __float_as_uint(saving));
+            if (EXT || waits) {
+                a[0] = make_uint4(l, S, Td, __float_as_uint(saving));
+            } else {
+                // no policy of the tile waits: the race at w = 0 is the request's own, and so is whether its
+                // winner is the endpoint that may hand over
+                const int oc0 = S > 0u ? (S > Td ? O_RACE_DEV : O_RACE_SRV) : O_SERVER_ONLY;
+                const bool can = oc0 == (dev_migrates ? O_RACE_DEV : O_RACE_SRV);
+                a[0] = make_uint4(l << 4 | (uint32_t)oc0, __float_as_uint(can ? saving : -1.0f), min(S, Td), Td);
+            }
             //                      tokens on device, server prefill, device prefill, TBTs in tau's bin
             a[1 + O_SERVER_ONLY] = make_uint4(0u, l, 0u, nt0);
             a[1 + O_DEVICE_ONLY] = make_uint4(n, 0u, l, nt1);
@@ -173,51 +185,91 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
         }
         __syncwarp();
         const int n_here = (int)min(32u, ch.len - b0);
-#pragma unroll 2
-        for (int r0 = 0; r0 < n_here; r0 += slots) {
-            const int r = r0 + slot;
-            if (r >= n_here) continue;
-            const uint4 Q = stA[r * kStageVec];
-            const uint32_t l = Q.x, S = Q.y, Td = Q.z;
-            bool dev_only, started, dev_wins, migr;
-            uint32_t ttft;
-            if (EXT) {
-                const uint4 X = stB[r * kStageVec + 6];
-                PairIn q;
-                q.l = l; q.n = X.w; q.S = S; q.m = X.z; q.saving = __uint_as_float(Q.w); q.u = X.y; q.delta_c = delta_c;
-                const PairOut o = decide<true>(q, pr, Td, candidate);
-                dev_only = o.dev_only; started = o.started; dev_wins = o.dev_wins; migr = o.migr; ttft = o.ttft;
-            } else {
-                // ---- dispatch (Algorithm 2's wait map / Algorithm 3's threshold) and the race
-                dev_only = (int32_t)l < l_th;
-                const uint32_t w = (int32_t)l < l_star ? 0u : ((int32_t)l == l_star ? w_star : w_tail);
-                started = dev_only || S > w;                       // the device starts after the wait
-                const uint32_t wTd = w + Td;
-                dev_wins = dev_only || (started && S > wTd);        // a tie goes to the server
-                ttft = dev_only ? Td : min(S, wTd);
-                migr = started && !dev_only && dev_wins == dev_migrates && __uint_as_float(Q.w) > theta;
+        // kIlp requests at a time per lane, phase by phase, so that the shared-memory loads of one do not
+        // queue behind the histogram atomics of another
+        auto pairs_of = [&](auto no_waits, const int (&rr)[kIlp], const bool (&ok)[kIlp]) {
+            constexpr bool kNoWaits = decltype(no_waits)::value;
+            uint4 Q[kIlp];
+            bool dev_wins[kIlp], migr[kIlp];
+            int oc[kIlp];
+            uint32_t ttft[kIlp];
+#pragma unroll
+            for (int k = 0; k < kIlp; ++k) Q[k] = stA[rr[k] * kStageVec];
+#pragma unroll
+            for (int k = 0; k < kIlp; ++k) {
+                if (kNoWaits) {
+                    // ---- Algorithm 3's threshold; the race and the hand-over candidate were settled at staging
+                    const bool dev_only = Q[k].x < lth16;
+                    const int oc0 = (int)(Q[k].x & 15u);
+                    migr[k] = !dev_only && __uint_as_float(Q[k].y) > theta;
+                    dev_wins[k] = dev_only || oc0 == O_RACE_DEV;
+                    ttft[k] = dev_only ? Q[k].w : Q[k].z;
+                    oc[k] = dev_only ? O_DEVICE_ONLY : oc0 + (migr[k] ? 2 : 0);
+                    continue;
+                }
+                const uint32_t l = Q[k].x, S = Q[k].y, Td = Q[k].z;
+                bool dev_only, started;
+                if (EXT) {
+                    const uint4 X = stB[rr[k] * kStageVec + 6];
+                    PairIn q;
+                    q.l = l; q.n = X.w; q.S = S; q.m = X.z; q.saving = __uint_as_float(Q[k].w); q.u = X.y; q.delta_c = delta_c;
+                    const PairOut o = decide<true>(q, pr, Td, candidate);
+                    dev_only = o.dev_only; started = o.started; dev_wins[k] = o.dev_wins; migr[k] = o.migr; ttft[k] = o.ttft;
+                } else {
+                    // ---- dispatch (Algorithm 2's wait map / Algorithm 3's threshold) and the race
+                    dev_only = (int32_t)l < l_th;
+                    const uint32_t w = (int32_t)l < l_star ? 0u : ((int32_t)l == l_star ? w_star : w_tail);
+                    started = dev_only || S > w;                       // the device starts after the wait
+                    const uint32_t wTd = w + Td;
+                    dev_wins[k] = dev_only || (started && S > wTd);    // a tie goes to the server
+                    ttft[k] = dev_only ? Td : min(S, wTd);
+                    migr[k] = started && !dev_only && dev_wins[k] == dev_migrates && __uint_as_float(Q[k].w) > theta;
+                }
+                oc[k] = dev_only ? O_DEVICE_ONLY
+                                 : (!started ? O_SERVER_ONLY : (dev_wins[k] ? O_RACE_DEV : O_RACE_SRV) + (migr[k] ? 2 : 0));
             }
-            const int oc = dev_only ? O_DEVICE_ONLY : (!started ? O_SERVER_ONLY : (dev_wins ? O_RACE_DEV : O_RACE_SRV) + (migr ? 2 : 0));
-            const uint4 h1 = stA[r * kStageVec + 1 + oc], h2 = stB[r * kStageVec + oc];
-            a_td += h1.x; a_ps += h1.y; a_pd += h1.z; a_tau += h1.w;
-            a_dl += h2.x; cnt_a += h2.y; cnt_b += h2.z;
-            a_tt += ttft;
-            if (waits) hist16_apply(my_ttft, hist16_code(bin_of_ticks(ttft)));
-            else hist16_apply(my_ttft, h2.w);
-            if (migr) {
-                const uint32_t sc = stB[r * kStageVec + 6].x;
-                if ((int32_t)sc >= 0) hist16_apply(my_stall, sc);
+            uint4 h1[kIlp], h2[kIlp];
+            uint32_t sc[kIlp];
+#pragma unroll
+            for (int k = 0; k < kIlp; ++k) {
+                h1[k] = stA[rr[k] * kStageVec + 1 + oc[k]];
+                h2[k] = stB[rr[k] * kStageVec + oc[k]];
+                sc[k] = stB[rr[k] * kStageVec + 6].x;
+            }
+#pragma unroll
+            for (int k = 0; k < kIlp; ++k) {
+                if (!ok[k]) continue;
+                a_td += h1[k].x; a_ps += h1[k].y; a_pd += h1[k].z; a_tau += h1[k].w;
+                a_dl += h2[k].x; cnt_a += h2[k].y; cnt_b += h2[k].z;
+                a_tt += ttft[k];
+                hist16_apply(my_ttft, (EXT ? !waits : kNoWaits) ? h2[k].w : hist16_code(bin_of_ticks(ttft[k])));
+                if (migr[k] && (int32_t)sc[k] >= 0) hist16_apply(my_stall, sc[k]);
             }
             if (wide && act) {                                 // regular TBTs outside the bin of tau
-                const int c = migr ? 2 : (dev_wins ? 1 : 0);
-                const int W = c == 2 ? W2 : (c == 1 ? W1 : W0), kt = c == 2 ? kt2 : (c == 1 ? kt1 : kt0);
-                const uint32_t* wp = rec.win[c] + (size_t)(ch.start + b0 + r) * W;
-                unsigned long long* hp = hist_tbt + (size_t)p * kNBins + cc.lo[g][c];
-                for (int j = 0; j < W; ++j) {
-                    const uint32_t v = j == kt ? 0u : wp[j];
-                    if (v) atomicAdd(&hp[j], (unsigned long long)v);
+                for (int k = 0; k < kIlp; ++k) {
+                    if (!ok[k]) continue;
+                    const int c = migr[k] ? 2 : (dev_wins[k] ? 1 : 0);
+                    const int W = c == 2 ? W2 : (c == 1 ? W1 : W0), kt = c == 2 ? kt2 : (c == 1 ? kt1 : kt0);
+                    const uint32_t* wp = rec.win[c] + (size_t)(ch.start + b0 + rr[k]) * W;
+                    unsigned long long* hp = hist_tbt + (size_t)p * kNBins + cc.lo[g][c];
+                    for (int j = 0; j < W; ++j) {
+                        const uint32_t v = j == kt ? 0u : wp[j];
+                        if (v) atomicAdd(&hp[j], (unsigned long long)v);
+                    }
                 }
             }
+        };
+        for (int r0 = 0; r0 < n_here; r0 += kIlp * slots) {
+            int rr[kIlp];
+            bool ok[kIlp];
+#pragma unroll
+            for (int k = 0; k < kIlp; ++k) {
+                const int r = r0 + k * slots + slot;
+                ok[k] = r < n_here;
+                rr[k] = min(r, 31);                             // every staging slot holds a valid request
+            }
+            if (!EXT && !waits) pairs_of(std::true_type{}, rr, ok);
+            else pairs_of(std::false_type{}, rr, ok);
         }
     }
     // ---- block totals, then one flush per block
