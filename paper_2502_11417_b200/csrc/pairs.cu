@@ -72,6 +72,7 @@ __device__ __forceinline__ PairOut decide(const PairIn& q, const Prep& pr, uint3
 constexpr int kAccThreads = 512;         // one block per SM: histograms and staging fill its shared memory
 constexpr int kAccWarps = kAccThreads / 32;
 constexpr int kHWords = 433;            // 866 sixteen-bit counters per policy row; odd word stride
+constexpr int kStageReq = 32;           // requests a warp stages at a time
 constexpr int kIlp = 4;                 // requests a lane works on at a time
 constexpr int kStageVec = 7;            // uint4 per request in each of the two staging blocks (odd: no bank conflicts)
 
@@ -129,8 +130,8 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
 
     // [warp][32 requests][kStageVec]: block A = the request, then the first half of each outcome's row;
     // block B = the second halves, then the stall increment and what only the extended policies read.
-    uint4* stA = (uint4*)(smem + acc_stage_offset_words(PL)) + wib * 32 * kStageVec;
-    uint4* stB = stA + kAccWarps * 32 * kStageVec;
+    uint4* stA = (uint4*)(smem + acc_stage_offset_words(PL)) + wib * kStageReq * kStageVec;
+    uint4* stB = stA + kAccWarps * kStageReq * kStageVec;
     // The wait map without mode tests: Algorithm 3 has no waits (l_star beyond every length), Algorithm 2 no
     // device-only prompts (l_th = 0, as the preparation kernel leaves it).
     const int32_t l_th = pr.l_th, l_star = pr.device_constrained ? pr.l_star : 0x7FFFFFFF;
@@ -140,7 +141,7 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
     const bool dev_migrates = candidate == 2;
     const uint32_t lth16 = (uint32_t)max(l_th, 0) << 4;      // against a staged (l << 4 | outcome at w = 0)
 
-    for (uint32_t b0 = wib * 32u; b0 < ch.len; b0 += kAccWarps * 32u) {
+    for (uint32_t b0 = wib * kStageReq; b0 < ch.len; b0 += kAccWarps * kStageReq) {
         // ---- 32 requests, one per lane
         __syncwarp();
         {
@@ -150,8 +151,8 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
             const uint32_t nt0 = kt0 >= 0 ? rec.win[0][(size_t)kk * W0 + kt0] : 0u;
             const uint32_t nt1 = kt1 >= 0 ? rec.win[1][(size_t)kk * W1 + kt1] : 0u;
             uint32_t nt2 = kt2 >= 0 ? rec.win[2][(size_t)kk * W2 + kt2] : 0u;
-            uint32_t stall_code = 0xFFFFFFFFu;                 // the token after a hand-off: counted with tau's bin
-            if (stall == tau) ++nt2; else stall_code = hist16_code(bin_of_ticks(stall));
+            uint32_t stall_code = 0u;                          // the token after a hand-off: counted with tau's bin,
+            if (stall == tau) ++nt2; else stall_code = hist16_code(bin_of_ticks(stall));   // else an increment of its own
             // a request may only migrate if its buffer filled (m != 0); fold that into the saving (Eq. 4)
             const float saving = m ? delta_c * (float)(n - m) : -1.0f;
             const uint32_t Td = kappa * l + c0, lm = l + m;
@@ -174,21 +175,21 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
             a[1 + O_RACE_DEV] = make_uint4(n, l, l, nt1);
             a[1 + O_MIGR_TO_DEV] = make_uint4(n - m, l, l + lm, nt2);
             a[1 + O_MIGR_TO_SRV] = make_uint4(m, l + lm, l, nt2);
-            //                      delayed tokens, counts, counts, TTFT increment
+            //                      delayed tokens << 17 | stall increment, counts, counts, TTFT increment
             b[O_SERVER_ONLY] = make_uint4(0u, 0u, 0u, hS);
             b[O_DEVICE_ONLY] = make_uint4(0u, 1u, 0u, hT);
             b[O_RACE_SRV] = make_uint4(0u, 0x10000u, 0u, hS);
             b[O_RACE_DEV] = make_uint4(0u, 0x10000u, 1u, hT);
-            b[O_MIGR_TO_DEV] = make_uint4(dly, 0x10000u, 0x10000u, hS);
-            b[O_MIGR_TO_SRV] = make_uint4(dly, 0x10000u, 0x10001u, hT);
-            b[6] = make_uint4(stall_code, EXT ? routing_draw(k0, tr.orig[kk]) : 0u, m, n);
+            b[O_MIGR_TO_DEV] = make_uint4(dly << 17 | stall_code, 0x10000u, 0x10000u, hS);
+            b[O_MIGR_TO_SRV] = make_uint4(dly << 17 | stall_code, 0x10000u, 0x10001u, hT);
+            b[6] = make_uint4(0u, EXT ? routing_draw(k0, tr.orig[kk]) : 0u, m, n);
         }
         __syncwarp();
-        const int n_here = (int)min(32u, ch.len - b0);
+        const int n_here = (int)min((uint32_t)kStageReq, ch.len - b0);
         // kIlp requests at a time per lane, phase by phase, so that the shared-memory loads of one do not
         // queue behind the histogram atomics of another
-        auto pairs_of = [&](auto no_waits, const int (&rr)[kIlp], const bool (&ok)[kIlp]) {
-            constexpr bool kNoWaits = decltype(no_waits)::value;
+        auto pairs_of = [&](auto no_waits, auto all_ok, const int (&rr)[kIlp], const bool (&ok)[kIlp]) {
+            constexpr bool kNoWaits = decltype(no_waits)::value, kAllOk = decltype(all_ok)::value;
             uint4 Q[kIlp];
             bool dev_wins[kIlp], migr[kIlp];
             int oc[kIlp];
@@ -229,25 +230,23 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
                                  : (!started ? O_SERVER_ONLY : (dev_wins[k] ? O_RACE_DEV : O_RACE_SRV) + (migr[k] ? 2 : 0));
             }
             uint4 h1[kIlp], h2[kIlp];
-            uint32_t sc[kIlp];
 #pragma unroll
             for (int k = 0; k < kIlp; ++k) {
                 h1[k] = stA[rr[k] * kStageVec + 1 + oc[k]];
                 h2[k] = stB[rr[k] * kStageVec + oc[k]];
-                sc[k] = stB[rr[k] * kStageVec + 6].x;
             }
 #pragma unroll
             for (int k = 0; k < kIlp; ++k) {
-                if (!ok[k]) continue;
+                if (!kAllOk && !ok[k]) continue;
                 a_td += h1[k].x; a_ps += h1[k].y; a_pd += h1[k].z; a_tau += h1[k].w;
-                a_dl += h2[k].x; cnt_a += h2[k].y; cnt_b += h2[k].z;
+                a_dl += h2[k].x >> 17; cnt_a += h2[k].y; cnt_b += h2[k].z;
                 a_tt += ttft[k];
                 hist16_apply(my_ttft, (EXT ? !waits : kNoWaits) ? h2[k].w : hist16_code(bin_of_ticks(ttft[k])));
-                if (migr[k] && (int32_t)sc[k] >= 0) hist16_apply(my_stall, sc[k]);
+                if (h2[k].x & 0x10001u) hist16_apply(my_stall, h2[k].x);      // only a migrated pair's row carries one
             }
             if (wide && act) {                                 // regular TBTs outside the bin of tau
                 for (int k = 0; k < kIlp; ++k) {
-                    if (!ok[k]) continue;
+                    if (!kAllOk && !ok[k]) continue;
                     const int c = migr[k] ? 2 : (dev_wins[k] ? 1 : 0);
                     const int W = c == 2 ? W2 : (c == 1 ? W1 : W0), kt = c == 2 ? kt2 : (c == 1 ? kt1 : kt0);
                     const uint32_t* wp = rec.win[c] + (size_t)(ch.start + b0 + rr[k]) * W;
@@ -259,6 +258,18 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
                 }
             }
         };
+        if (PL == 32 && n_here == kStageReq) {                  // a full batch for 32 policies: r is warp-uniform
+#pragma unroll 2
+            for (int r0 = 0; r0 < kStageReq; r0 += kIlp) {
+                int rr[kIlp];
+                bool ok[kIlp];
+#pragma unroll
+                for (int k = 0; k < kIlp; ++k) { rr[k] = r0 + k; ok[k] = true; }
+                if (!EXT && !waits) pairs_of(std::true_type{}, std::true_type{}, rr, ok);
+                else pairs_of(std::false_type{}, std::true_type{}, rr, ok);
+            }
+            continue;
+        }
         for (int r0 = 0; r0 < n_here; r0 += kIlp * slots) {
             int rr[kIlp];
             bool ok[kIlp];
@@ -266,10 +277,10 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
             for (int k = 0; k < kIlp; ++k) {
                 const int r = r0 + k * slots + slot;
                 ok[k] = r < n_here;
-                rr[k] = min(r, 31);                             // every staging slot holds a valid request
+                rr[k] = min(r, kStageReq - 1);                  // every staging slot holds a valid request
             }
-            if (!EXT && !waits) pairs_of(std::true_type{}, rr, ok);
-            else pairs_of(std::false_type{}, rr, ok);
+            if (!EXT && !waits) pairs_of(std::true_type{}, std::false_type{}, rr, ok);
+            else pairs_of(std::false_type{}, std::false_type{}, rr, ok);
         }
     }
     // ---- block totals, then one flush per block
@@ -304,7 +315,7 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
 }
 
 size_t acc_smem_bytes(int PL) {
-    return sizeof(uint32_t) * acc_stage_offset_words(PL) + (size_t)kAccWarps * 32 * 2 * kStageVec * sizeof(uint4);
+    return sizeof(uint32_t) * acc_stage_offset_words(PL) + (size_t)kAccWarps * kStageReq * 2 * kStageVec * sizeof(uint4);
 }
 
 // ------------------------------------------------------------------------------------------------------
