@@ -88,6 +88,16 @@ __device__ __forceinline__ void hist16_apply(uint32_t* row, uint32_t code) {
     atomicAdd((uint32_t*)((char*)row + (code & 0xFFCu)), code & 0x10001u);
 }
 
+// One more TTFT of t ticks, t < 2^31 (so its bin is below kNBins): the counter pair and the half come straight
+// from the float's exponent and leading mantissa bits, 32 bins per octave as in bin_of_ticks.
+__device__ __forceinline__ void hist16_add_ticks(uint32_t* row, uint32_t t) {
+    if (t < 32u) { hist16_apply(row, hist16_code((int)t)); return; }
+    const uint32_t fb = __float_as_uint(__uint2float_rz(t));
+    atomicAdd((uint32_t*)((char*)row - 4 * (((127 + 4) << 5) >> 1) + ((fb >> 17) & 0x3FFCu)), 1u << ((fb >> 14) & 16u));
+}
+
+enum TileKind { K_NOWAIT = 0, K_WAIT = 1, K_ANY = 2 };
+
 template <bool EXT>
 __global__ void __launch_bounds__(kAccThreads, 1)
 k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __restrict__ ccp,
@@ -121,6 +131,9 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
     // With no waits in the tile (Algorithm 3, random routing) a TTFT is the request's S or its T_d, whose
     // histogram increments are staged; otherwise the bin is worked out per pair.
     const bool waits = __syncthreads_or(act && pr.device_constrained && !pr.stochastic) != 0;
+    // a tile of Algorithm 2 policies alone has no device-only prompts either
+    const bool all_wait = !EXT && __syncthreads_or(act && !pr.device_constrained) == 0;
+    const int kind = EXT ? K_ANY : (!waits ? K_NOWAIT : (all_wait ? K_WAIT : K_ANY));
     uint32_t* my_ttft = h_ttft + pol_in_tile * kHWords;
     uint32_t* my_stall = h_stall + pol_in_tile * kHWords;
 
@@ -188,8 +201,9 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
         const int n_here = (int)min((uint32_t)kStageReq, ch.len - b0);
         // kIlp requests at a time per lane, phase by phase, so that the shared-memory loads of one do not
         // queue behind the histogram atomics of another
-        auto pairs_of = [&](auto no_waits, auto all_ok, const int (&rr)[kIlp], const bool (&ok)[kIlp]) {
-            constexpr bool kNoWaits = decltype(no_waits)::value, kAllOk = decltype(all_ok)::value;
+        auto pairs_of = [&](auto tile_kind, auto all_ok, const int (&rr)[kIlp], const bool (&ok)[kIlp]) {
+            constexpr int kKind = decltype(tile_kind)::value;
+            constexpr bool kNoWaits = kKind == K_NOWAIT, kAllOk = decltype(all_ok)::value;
             uint4 Q[kIlp];
             bool dev_wins[kIlp], migr[kIlp];
             int oc[kIlp];
@@ -209,6 +223,17 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
                     continue;
                 }
                 const uint32_t l = Q[k].x, S = Q[k].y, Td = Q[k].z;
+                if (kKind == K_WAIT) {
+                    // ---- Algorithm 2's wait map and the race
+                    const uint32_t w = (int32_t)l < l_star ? 0u : ((int32_t)l == l_star ? w_star : w_tail);
+                    const bool started = S > w;                        // the device starts after the wait
+                    const uint32_t wTd = w + Td;
+                    dev_wins[k] = S > wTd;                             // a tie goes to the server
+                    ttft[k] = min(S, wTd);
+                    migr[k] = started && dev_wins[k] == dev_migrates && __uint_as_float(Q[k].w) > theta;
+                    oc[k] = !started ? O_SERVER_ONLY : (dev_wins[k] ? O_RACE_DEV : O_RACE_SRV) + (migr[k] ? 2 : 0);
+                    continue;
+                }
                 bool dev_only, started;
                 if (EXT) {
                     const uint4 X = stB[rr[k] * kStageVec + 6];
@@ -241,7 +266,8 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
                 a_td += h1[k].x; a_ps += h1[k].y; a_pd += h1[k].z; a_tau += h1[k].w;
                 a_dl += h2[k].x >> 17; cnt_a += h2[k].y; cnt_b += h2[k].z;
                 a_tt += ttft[k];
-                hist16_apply(my_ttft, (EXT ? !waits : kNoWaits) ? h2[k].w : hist16_code(bin_of_ticks(ttft[k])));
+                if (EXT ? !waits : kNoWaits) hist16_apply(my_ttft, h2[k].w);
+                else hist16_add_ticks(my_ttft, ttft[k]);
                 if (h2[k].x & 0x10001u) hist16_apply(my_stall, h2[k].x);      // only a migrated pair's row carries one
             }
             if (wide && act) {                                 // regular TBTs outside the bin of tau
@@ -265,8 +291,9 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
                 bool ok[kIlp];
 #pragma unroll
                 for (int k = 0; k < kIlp; ++k) { rr[k] = r0 + k; ok[k] = true; }
-                if (!EXT && !waits) pairs_of(std::true_type{}, std::true_type{}, rr, ok);
-                else pairs_of(std::false_type{}, std::true_type{}, rr, ok);
+                if (kind == K_NOWAIT) pairs_of(std::integral_constant<int, K_NOWAIT>{}, std::true_type{}, rr, ok);
+                else if (kind == K_WAIT) pairs_of(std::integral_constant<int, K_WAIT>{}, std::true_type{}, rr, ok);
+                else pairs_of(std::integral_constant<int, K_ANY>{}, std::true_type{}, rr, ok);
             }
             continue;
         }
@@ -279,8 +306,9 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
                 ok[k] = r < n_here;
                 rr[k] = min(r, kStageReq - 1);                  // every staging slot holds a valid request
             }
-            if (!EXT && !waits) pairs_of(std::true_type{}, std::false_type{}, rr, ok);
-            else pairs_of(std::false_type{}, std::false_type{}, rr, ok);
+            if (kind == K_NOWAIT) pairs_of(std::integral_constant<int, K_NOWAIT>{}, std::false_type{}, rr, ok);
+            else if (kind == K_WAIT) pairs_of(std::integral_constant<int, K_WAIT>{}, std::false_type{}, rr, ok);
+            else pairs_of(std::integral_constant<int, K_ANY>{}, std::false_type{}, rr, ok);
         }
     }
     // ---- block totals, then one flush per block
