@@ -154,16 +154,30 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
     const bool dev_migrates = candidate == 2;
     const uint32_t lth16 = (uint32_t)max(l_th, 0) << 4;      // against a staged (l << 4 | outcome at w = 0)
 
+    // One request per lane, fetched a batch ahead so that the loads fly while the previous batch is evaluated.
+    struct Raw { uint32_t l, n, S, m, dly, stall, nt0, nt1, nt2, orig; };   // as loaded: nothing may consume a load early
+    auto fetch = [&](uint32_t b0) {
+        const uint32_t kk = ch.start + min(b0 + lane, ch.len - 1);
+        Raw q;
+        q.l = tr.l[kk]; q.n = tr.nout[kk]; q.S = (uint32_t)tr.S[kk];
+        q.m = rec.m[kk]; q.dly = rec.delayed[kk]; q.stall = rec.stall[kk];
+        q.nt0 = kt0 >= 0 ? rec.win[0][(size_t)kk * W0 + kt0] : 0u;
+        q.nt1 = kt1 >= 0 ? rec.win[1][(size_t)kk * W1 + kt1] : 0u;
+        q.nt2 = kt2 >= 0 ? rec.win[2][(size_t)kk * W2 + kt2] : 0u;
+        q.orig = EXT ? tr.orig[kk] : 0u;
+        return q;
+    };
+    Raw nx = fetch(min(wib * kStageReq, ch.len - 1));
     for (uint32_t b0 = wib * kStageReq; b0 < ch.len; b0 += kAccWarps * kStageReq) {
         // ---- 32 requests, one per lane
+        const Raw cur = nx;
+        if (b0 + kAccWarps * kStageReq < ch.len) nx = fetch(b0 + kAccWarps * kStageReq);
         __syncwarp();
         {
-            const uint32_t kk = ch.start + min(b0 + lane, ch.len - 1);
-            const uint32_t l = tr.l[kk], n = tr.nout[kk], S = (uint32_t)tr.S[kk], m = rec.m[kk];
-            const uint32_t stall = rec.stall[kk], dly = rec.delayed[kk];
-            const uint32_t nt0 = kt0 >= 0 ? rec.win[0][(size_t)kk * W0 + kt0] : 0u;
-            const uint32_t nt1 = kt1 >= 0 ? rec.win[1][(size_t)kk * W1 + kt1] : 0u;
-            uint32_t nt2 = kt2 >= 0 ? rec.win[2][(size_t)kk * W2 + kt2] : 0u;
+            const uint32_t l = cur.l, n = cur.n, S = cur.S, m = cur.m;
+            const uint32_t stall = cur.stall, dly = cur.dly;
+            const uint32_t nt0 = cur.nt0, nt1 = cur.nt1;
+            uint32_t nt2 = cur.nt2;
             uint32_t stall_code = 0u;                          // the token after a hand-off: counted with tau's bin,
             if (stall == tau) ++nt2; else stall_code = hist16_code(bin_of_ticks(stall));   // else an increment of its own
             // a request may only migrate if its buffer filled (m != 0); fold that into the saving (Eq. 4)
@@ -195,7 +209,7 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
             b[O_RACE_DEV] = make_uint4(0u, 0x10000u, 1u, hT);
             b[O_MIGR_TO_DEV] = make_uint4(dly << 17 | stall_code, 0x10000u, 0x10000u, hS);
             b[O_MIGR_TO_SRV] = make_uint4(dly << 17 | stall_code, 0x10000u, 0x10001u, hT);
-            b[6] = make_uint4(0u, EXT ? routing_draw(k0, tr.orig[kk]) : 0u, m, n);
+            b[6] = make_uint4(0u, EXT ? routing_draw(k0, cur.orig) : 0u, m, n);
         }
         __syncwarp();
         const int n_here = (int)min((uint32_t)kStageReq, ch.len - b0);
