@@ -33,9 +33,16 @@ TRACE_BYTES = 9              # packed request: ticks, prompt, output length, gro
 # counter add 1, hash finaliser 8, two range maps (multiply-high) 2, tail mask 1, two sums and two maxima 4,
 # loop 1.
 PLAYOUT_INSTR_PER_TOKEN = 17
-# Lane-instructions one (request, policy) pair needs in the reduction kernel: wait map and race 12,
-# trigger 4, tokens and prefill 10, ten running sums 10, TTFT bin and histogram update 6.
-PAIR_INSTR = 42
+# Lane-instructions one (request, policy) pair needs in the reduction kernel, by the kind of policy.
+# Algorithm 3 (no waits; the race at w = 0 is staged once per request): request vector load 1, length
+# threshold 1, trigger compare and its conjunction 2, outcome index 2, TTFT select 1, row address 1, two row
+# loads 2, seven 32-bit sums and one 64-bit sum 9, staged histogram increment (two masks, address, atomic) 4,
+# stall increment (test, address, atomic) 3.
+PAIR_INSTR_NOWAIT = 27
+# Algorithm 2 (waits): load 1, wait map 4, start compare 1, w + T_d 1, win compare 1, minimum 1, trigger 3,
+# outcome index 3, row address 1, two row loads 2, sums 9, histogram increment from the float bits (convert,
+# small-value test and branch, offset 2, increment 3, address, atomic) 10, stall increment 3.
+PAIR_INSTR_WAIT = 41
 SM_COUNT, SCHEDULERS, LANES = 148, 4, 32
 # DRAM bytes per launch from the committed ncu capture of the dominant kernel (None until captured for
 # the current kernel; see profiles/).
@@ -273,9 +280,19 @@ def run_ours(args):
                 "peak_source": src,
                 "algorithmic_bytes": bytes_alg}
     elif top == "k_pairs_acc":
-        ach = n * P * PAIR_INSTR / (kms[top] * 1e-3) / 1e12
+        # pairs by kind: a (group, policy) waits when Algorithm 1 made the group device-constrained
+        lane_instr, wait_pairs = 0, 0
+        for g in range(tr.n_groups):
+            n_g = tr.group_size(g)
+            n_wait = sum(1 for p in range(P) if tr.prep(g, p).device_constrained)
+            wait_pairs += n_g * n_wait
+            lane_instr += n_g * (n_wait * PAIR_INSTR_WAIT + (P - n_wait) * PAIR_INSTR_NOWAIT)
+        ach = lane_instr / (kms[top] * 1e-3) / 1e12
         roof = {"kernel": top, "bound": "alu", "achieved": ach, "peak": alu_peak, "unit": "Tinstr/s",
-                "frac": ach / alu_peak, "traffic": None, "peak_source": alu_src, "instr_per_pair": PAIR_INSTR}
+                "frac": ach / alu_peak, "traffic": None, "peak_source": alu_src,
+                "instr_per_pair": {"no_wait": PAIR_INSTR_NOWAIT, "wait": PAIR_INSTR_WAIT,
+                                   "mean": lane_instr / float(n * P)},
+                "pairs_with_waits": wait_pairs}
     else:
         ach = token_steps * PLAYOUT_INSTR_PER_TOKEN / (kms[top] * 1e-3) / 1e12
         roof = {"kernel": top, "bound": "alu", "achieved": ach, "peak": alu_peak, "unit": "Tinstr/s",

@@ -289,6 +289,13 @@ class Trace:
         _check(lib().disco_get_prep(self._h, g, p, C.byref(out), _stream_ptr(stream)))
         return out
 
+    def group_size(self, g: int, stream=None) -> int:
+        """Requests of profile group g in the loaded trace."""
+        ng = lib().disco_get_group_tables(self._h, g, None, None, None, 0, _stream_ptr(stream))
+        if ng < 0:
+            _check(int(ng))
+        return int(ng)
+
     def group_tables(self, g: int, n_sorted: Optional[int] = None, stream=None):
         cnt = np.zeros(4097, dtype=np.int64)
         kn = np.zeros(257, dtype=np.int32)
