@@ -272,18 +272,18 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
     bool cls_extras_pending = false;      // some policy routes at random or triggers on an expected length
     for (uint32_t p = 0; p < P; ++p) {
         const disco_policy_t& q = pol[p];
-        const std::string at = " (policy " + std::to_string(p) + ")";
-        if (!(q.budget >= 0.0f && q.budget <= 1.0f)) return fail(DISCO_EINVAL, "budget outside [0,1]" + at);
-        if (!(q.alpha > 0.0f && q.alpha < 1.0f)) return fail(DISCO_EINVAL, "alpha outside (0,1)" + at);
-        if (!(q.mig_threshold >= 0.0f)) return fail(DISCO_EINVAL, "migration threshold negative or NaN" + at);
-        if (!(q.r_c > 0.0f) || !std::isfinite(q.r_c)) return fail(DISCO_EINVAL, "consumption rate must be positive" + at);
-        if (!(q.t_m_s >= 0.0f) || !std::isfinite(q.t_m_s)) return fail(DISCO_EINVAL, "migration time must be >= 0" + at);
+        auto at = [p] { return " (policy " + std::to_string(p) + ")"; };
+        if (!(q.budget >= 0.0f && q.budget <= 1.0f)) return fail(DISCO_EINVAL, "budget outside [0,1]" + at());
+        if (!(q.alpha > 0.0f && q.alpha < 1.0f)) return fail(DISCO_EINVAL, "alpha outside (0,1)" + at());
+        if (!(q.mig_threshold >= 0.0f)) return fail(DISCO_EINVAL, "migration threshold negative or NaN" + at());
+        if (!(q.r_c > 0.0f) || !std::isfinite(q.r_c)) return fail(DISCO_EINVAL, "consumption rate must be positive" + at());
+        if (!(q.t_m_s >= 0.0f) || !std::isfinite(q.t_m_s)) return fail(DISCO_EINVAL, "migration time must be >= 0" + at());
         const uint32_t mode = (q.flags >> 2) & 3u;
-        if (mode == 3 || (q.flags >> 6)) return fail(DISCO_EINVAL, "unknown flags" + at);
-        if (q.expected_len > (1u << 20)) return fail(DISCO_EINVAL, "expected length too large" + at);
-        if (q.l_immediate > (uint32_t)kMaxPrompt) return fail(DISCO_EINVAL, "l_immediate above the longest prompt" + at);
+        if (mode == 3 || (q.flags >> 6)) return fail(DISCO_EINVAL, "unknown flags" + at());
+        if (q.expected_len > (1u << 20)) return fail(DISCO_EINVAL, "expected length too large" + at());
+        if (q.l_immediate > (uint32_t)kMaxPrompt) return fail(DISCO_EINVAL, "l_immediate above the longest prompt" + at());
         const int64_t tau = ticks_of_rate(q.r_c), t_m = ticks_of_seconds(q.t_m_s);
-        if (tau < 1 || tau >= (1 << 30)) return fail(DISCO_EINVAL, "consumption interval outside 1 .. 2^30 ticks" + at);
+        if (tau < 1 || tau >= (1 << 30)) return fail(DISCO_EINVAL, "consumption interval outside 1 .. 2^30 ticks" + at());
         const bool pacing = (q.flags & DISCO_FLAG_PACING) != 0, mig = (q.flags & DISCO_FLAG_MIGRATION) != 0;
         int64_t B = pacing ? (t_m + tau - 1) / tau : 0;               // Eq. 6, rounded up
         if (B > kMaxOutput) B = kMaxOutput;                            // a buffer no stream can fill
@@ -450,8 +450,13 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
     for (size_t k = 0; k < classes.size(); ++k) {
         const ClassConst* dcc = c->d_classes.as<ClassConst>() + k;
         if (timed) CU(cudaEventRecord(c->ev[0], st));
+        // with pacing on, a stream whose slowest interval T + J is within tau never falls behind its reader
+        bool never_clamps = classes[k].pacing != 0;
+        for (int g = 0; g < G; ++g)
+            never_clamps = never_clamps && (int64_t)c->gc[g].T_srv + c->gc[g].J_srv <= classes[k].tau &&
+                           (int64_t)c->gc[g].T_dev + c->gc[g].J_dev <= classes[k].tau;
         CU(launch_timeline(tr, c->d_gc.as<GroupConst>(), dcc, classes[k].pacing != 0, c->knots.as<int32_t>(), seed, rec,
-                           c->err, c->d_todo.as<uint32_t>(), todo_counts + k, timed ? c->ev[1] : nullptr, st));
+                           c->err, c->d_todo.as<uint32_t>(), todo_counts + k, never_clamps, timed ? c->ev[1] : nullptr, st));
         if (timed) CU(cudaEventRecord(c->ev[2], st));
         CU(launch_pairs(tr, c->d_gc.as<GroupConst>(), dcc, c->d_prep.as<Prep>(), P,
                         c->d_pol_list.as<uint32_t>() + cls_range[k].first, cls_range[k].second - cls_range[k].first,
@@ -459,7 +464,7 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
                         c->d_hist_ttft.as<uint64_t>(), c->d_hist_tbt.as<uint64_t>(), seed, cls_extras_pending,
                         timed ? c->ev[3] : nullptr, st));
         if (timed) CU(cudaEventRecord(c->ev[4], st));
-        g_launches += (n ? (classes[k].pacing ? 2 : 1) : 0) + ((n && !chunks.empty()) ? (out ? 2 : 1) : 0);
+        g_launches += (n ? ((classes[k].pacing && !never_clamps) ? 2 : 1) : 0) + ((n && !chunks.empty()) ? (out ? 2 : 1) : 0);
     }
     c->timing_valid = timed && n != 0;
     c->P = P; c->pol = pc;

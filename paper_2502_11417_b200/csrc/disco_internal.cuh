@@ -132,7 +132,9 @@ cudaError_t launch_prep_beta(const PolicyConst* pol, uint32_t P, int G, const in
                              const int32_t* sorted, const uint32_t* grp_off, Prep* prep, cudaStream_t st);
 cudaError_t launch_timeline(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, bool pacing,
                             const int32_t* knots, uint64_t seed, TimelineRec rec, int32_t* err, uint32_t* todo,
-                            uint32_t* todo_count /* zero on entry */, cudaEvent_t mid /* recorded between its two kernels, or null */,
+                            uint32_t* todo_count /* zero on entry */,
+                            bool never_clamps /* pacing on and tau >= T + J for both endpoints of every group */,
+                            cudaEvent_t mid /* recorded between its two kernels, or null */,
                             cudaStream_t st);
 cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const Prep* prep, uint32_t P,
                          const uint32_t* pol_list, uint32_t n_list, const Chunk* chunks, uint32_t n_chunks,

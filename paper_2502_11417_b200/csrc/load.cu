@@ -177,6 +177,7 @@ __global__ void k_radix_scatter(const uint64_t* __restrict__ keys_in, uint64_t* 
         __syncthreads();
 #pragma unroll
         for (int j = 0; j < kPer; ++j) {
+            uint32_t nxt = 0xFFFFFFFFu;                          // next pass's counter for this key (none: dead lane)
             if (live[j]) {
                 const uint32_t rank = __popc(peers[j] & ((1u << lane) - 1u));
                 const uint32_t pos = wcnt[w][dig[j]] + rank;
@@ -185,10 +186,15 @@ __global__ void k_radix_scatter(const uint64_t* __restrict__ keys_in, uint64_t* 
                     const uint32_t i = base + w * (32 * kPer) + j * 32 + lane;
                     pay_out[pos] = pay_in ? pay_in[i] : i;
                 }
-                if (counts_next)
-                    atomicAdd(&counts_next[((uint32_t)(key[j] >> (shift + 8)) & 255u) * gridDim.x + pos / per_block], 1u);
+                nxt = ((uint32_t)(key[j] >> (shift + 8)) & 255u) * gridDim.x + pos / per_block;
             }
             __syncwarp();
+            if (counts_next) {
+                // lanes bound for the same counter add once: high digits take few values, and one add per key
+                // would queue every key of the trace on a handful of addresses
+                const uint32_t same = __match_any_sync(0xFFFFFFFFu, nxt);
+                if (live[j] && (same & ((1u << lane) - 1u)) == 0) atomicAdd(&counts_next[nxt], (uint32_t)__popc(same));
+            }
             if (live[j] && (peers[j] & ((1u << lane) - 1u)) == 0) wcnt[w][dig[j]] += __popc(peers[j]);
             __syncwarp();
         }

@@ -361,67 +361,100 @@ size_t acc_smem_bytes(int PL) {
 }
 
 // ------------------------------------------------------------------------------------------------------
-// Per-pair arrays: lane = request, eight policies per block column.
+// Per-pair arrays: lane = request, up to 32 policies per block row.
+//
+// What a pair writes besides its TTFT depends on the request and on which of the six outcomes it ends in.
+// Each thread therefore prices its request once per outcome (Eq. 8, token split, TBT mean and maximum of
+// the stream that applies) into a row of shared memory that only it reads; a pair then costs the decision,
+// one 16-byte row load and the nine stores.  A store instruction writes 32 consecutive requests of one
+// policy row.
 // ------------------------------------------------------------------------------------------------------
 constexpr int kRowThreads = 256;
-constexpr int kRowPols = 8;
+constexpr int kRowPols = 32;
+constexpr int kRowVec = 7;              // uint4 per request: six outcome rows and one of padding (odd stride)
 
 template <bool EXT>
 __global__ void __launch_bounds__(kRowThreads)
 k_pairs_rows(TraceDev tr, const GroupConst* __restrict__ gcs, const Prep* __restrict__ prep, uint32_t P,
-             const uint32_t* __restrict__ pol_list, uint32_t n_list, const Chunk* __restrict__ chunks,
-             TimelineRec rec, uint32_t k0, disco_pair_out_t out) {
+             const uint32_t* __restrict__ pol_list, uint32_t n_list, TimelineRec rec, uint32_t k0,
+             disco_pair_out_t out) {
     __shared__ Prep s_prep[kRowPols];
     __shared__ uint32_t s_pol[kRowPols];
-    const Chunk ch = chunks[blockIdx.x];
-    const int g = ch.g;
+    __shared__ uint4 s_rows[kRowThreads * kRowVec];
     const uint32_t first = blockIdx.y * kRowPols;
     const int npol = (int)min((uint32_t)kRowPols, n_list - first);
+    // the block's requests are consecutive in the internal order; most blocks lie inside one group
+    const uint32_t k_lo = blockIdx.x * kRowThreads, k_hi = min(tr.n, k_lo + kRowThreads) - 1;
+    int g_lo = 0, g_hi = 0;
+    while (g_lo + 1 < tr.n_groups && k_lo >= tr.grp_off[g_lo + 1]) ++g_lo;
+    g_hi = g_lo;
+    while (g_hi + 1 < tr.n_groups && k_hi >= tr.grp_off[g_hi + 1]) ++g_hi;
+    const bool one_group = g_lo == g_hi;
     if ((int)threadIdx.x < npol) {
         const uint32_t p = pol_list[first + threadIdx.x];
         s_pol[threadIdx.x] = p;
-        s_prep[threadIdx.x] = prep[(size_t)g * P + p];
+        s_prep[threadIdx.x] = prep[(size_t)g_lo * P + p];
     }
     __syncthreads();
+    const uint32_t k = k_lo + threadIdx.x;
+    if (k >= tr.n) return;
+    int g = g_lo;
+    while (g < g_hi && k >= tr.grp_off[g + 1]) ++g;
     const GroupConst& gc = gcs[g];
-    const uint32_t kappa = (uint32_t)gc.kappa, c0 = (uint32_t)gc.c0;
     const int candidate = gc.candidate;
     const float delta_c = gc.delta_c, cps = gc.cps, cds = gc.cds, lcpd = gc.lcpd, lcdd = gc.lcdd;
     const size_t N = tr.n;
 
-    for (uint32_t r = threadIdx.x; r < ch.len; r += kRowThreads) {
-        const uint32_t k = ch.start + r;
-        PairIn q;
-        q.l = tr.l[k]; q.n = tr.nout[k]; q.S = (uint32_t)tr.S[k]; q.m = rec.m[k];
-        q.saving = delta_c * (float)(q.n - q.m);
-        q.delta_c = delta_c;
-        const uint32_t orig = tr.orig[k];
-        q.u = EXT ? routing_draw(k0, orig) : 0u;
-        const uint32_t Td = kappa * q.l + c0, dly = rec.delayed[k];
-        const uint32_t sum0 = rec.sum[0][k], sum1 = rec.sum[1][k], sum2 = rec.sum[2][k];
-        const uint32_t max0 = rec.max[0][k], max1 = rec.max[1][k], max2 = rec.max[2][k];
+    PairIn q;
+    q.l = tr.l[k]; q.n = tr.nout[k]; q.S = (uint32_t)tr.S[k]; q.m = rec.m[k];
+    q.saving = delta_c * (float)(q.n - q.m);
+    q.delta_c = delta_c;
+    const uint32_t orig = tr.orig[k];
+    q.u = EXT ? routing_draw(k0, orig) : 0u;
+    const uint32_t Td = (uint32_t)gc.kappa * q.l + (uint32_t)gc.c0, dly = rec.delayed[k];
+    uint4* row = s_rows + threadIdx.x * kRowVec;
+    {
         const float inv_cnt = q.n > 1 ? 1e-6f / (float)(q.n - 1) : 0.0f;
+        float mean[3], mx[3];
+#pragma unroll
+        for (int c = 0; c < 3; ++c) { mean[c] = (float)rec.sum[c][k] * inv_cnt; mx[c] = (float)rec.max[c][k] * 1e-6f; }
+        const uint32_t l = q.l, n = q.n, m = q.m, lm = l + m;
+        auto put = [&](int oc, uint32_t pre_srv, uint32_t pre_dev, uint32_t tok_dev, int stream) {
+            const uint32_t tok_srv = n - tok_dev;
+            const float cost = cps * (float)pre_srv + cds * (float)tok_srv + lcpd * (float)pre_dev + lcdd * (float)tok_dev;   // Eq. 8
+            row[oc] = make_uint4(__float_as_uint(cost), tok_srv | tok_dev << 16, __float_as_uint(mean[stream]),
+                                 __float_as_uint(mx[stream]));
+        };
+        put(O_SERVER_ONLY, l, 0u, 0u, 0);
+        put(O_DEVICE_ONLY, 0u, l, n, 1);
+        put(O_RACE_SRV, l, l, 0u, 0);
+        put(O_RACE_DEV, l, l, n, 1);
+        put(O_MIGR_TO_DEV, l, l + lm, n - m, 2);          // the server decoded m tokens, the device re-prefills l + m
+        put(O_MIGR_TO_SRV, l + lm, l, m, 2);
+    }
+    auto pair = [&](const Prep& pr, size_t at) {
+        const PairOut o = decide<EXT>(q, pr, Td, candidate);
+        const int oc = o.dev_only ? O_DEVICE_ONLY
+                                  : (!o.started ? O_SERVER_ONLY : (o.dev_wins ? O_RACE_DEV : O_RACE_SRV) + (o.migr ? 2 : 0));
+        const uint4 r = row[oc];
+        if (out.ttft_s) out.ttft_s[at] = (float)o.ttft * 1e-6f;
+        if (out.tbt_mean_s) out.tbt_mean_s[at] = __uint_as_float(r.z);
+        if (out.tbt_max_s) out.tbt_max_s[at] = __uint_as_float(r.w);
+        if (out.cost) out.cost[at] = __uint_as_float(r.x);
+        if (out.tok_server) out.tok_server[at] = r.y & 0xFFFFu;
+        if (out.tok_device) out.tok_device[at] = r.y >> 16;
+        if (out.mig_at) out.mig_at[at] = o.migr ? q.m : 0u;
+        if (out.delayed) out.delayed[at] = (uint16_t)(o.migr ? dly : 0u);
+        if (out.decision) out.decision[at] = (uint8_t)(o.dev_only ? DISCO_DEVICE_ONLY
+                                                                 : (o.started ? DISCO_RACE : DISCO_SERVER_ONLY));
+    };
+    if (one_group) {
+#pragma unroll 4
+        for (int pi = 0; pi < npol; ++pi) pair(s_prep[pi], (size_t)s_pol[pi] * N + orig);
+    } else {
         for (int pi = 0; pi < npol; ++pi) {
-            const PairOut o = decide<EXT>(q, s_prep[pi], Td, candidate);
-            const uint32_t sum = o.migr ? sum2 : (o.dev_wins ? sum1 : sum0);
-            const uint32_t mx = o.migr ? max2 : (o.dev_wins ? max1 : max0);
-            const uint32_t lm = q.l + q.m;
-            const uint32_t tok_src = o.migr ? q.m : q.n;
-            const uint32_t tok_dev = o.dev_wins ? tok_src : q.n - tok_src, tok_srv = q.n - tok_dev;
-            const uint32_t pre_srv = (o.dev_only ? 0u : q.l) + ((o.migr && o.dev_wins) ? lm : 0u);
-            const uint32_t pre_dev = (o.started ? q.l : 0u) + ((o.migr && !o.dev_wins) ? lm : 0u);
-            const size_t at = (size_t)s_pol[pi] * N + orig;
-            if (out.ttft_s) out.ttft_s[at] = (float)o.ttft * 1e-6f;
-            if (out.tbt_mean_s) out.tbt_mean_s[at] = (float)sum * inv_cnt;
-            if (out.tbt_max_s) out.tbt_max_s[at] = (float)mx * 1e-6f;
-            if (out.cost) out.cost[at] = cps * (float)pre_srv + cds * (float)tok_srv + lcpd * (float)pre_dev +
-                                         lcdd * (float)tok_dev;                        // Eq. 8
-            if (out.tok_server) out.tok_server[at] = tok_srv;
-            if (out.tok_device) out.tok_device[at] = tok_dev;
-            if (out.mig_at) out.mig_at[at] = o.migr ? q.m : 0u;
-            if (out.delayed) out.delayed[at] = (uint16_t)(o.migr ? dly : 0u);
-            if (out.decision) out.decision[at] = (uint8_t)(o.dev_only ? DISCO_DEVICE_ONLY
-                                                                     : (o.started ? DISCO_RACE : DISCO_SERVER_ONLY));
+            const Prep pr = prep[(size_t)g * P + s_pol[pi]];
+            pair(pr, (size_t)s_pol[pi] * N + orig);
         }
     }
 }
@@ -451,8 +484,8 @@ cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassCo
     const bool rows = out.ttft_s || out.tbt_mean_s || out.tbt_max_s || out.cost || out.tok_server || out.tok_device ||
                       out.mig_at || out.delayed || out.decision;
     if (rows) {
-        dim3 grid_r(n_chunks, (n_list + kRowPols - 1) / kRowPols);
-        row_kernel<<<grid_r, kRowThreads, 0, st>>>(tr, gc, prep, P, pol_list, n_list, chunks, rec, k0, out);
+        dim3 grid_r((tr.n + kRowThreads - 1) / kRowThreads, (n_list + kRowPols - 1) / kRowPols);
+        row_kernel<<<grid_r, kRowThreads, 0, st>>>(tr, gc, prep, P, pol_list, n_list, rec, k0, out);
         e = cudaGetLastError();
     }
     return e;

@@ -57,6 +57,10 @@ __device__ __forceinline__ uint32_t walk(uint32_t key, uint32_t j0, int t0, int 
 
 
 // rpw = requests per warp (4, 8, 16 or 32): small traces use small batches so that enough warps are in flight.
+// LEAN: the host has checked that tau >= T + J for both endpoints of every group, so no interval can exceed
+// tau and every request is clamp-free by construction.  Then only the candidate stream's sums are needed to
+// find the hand-off index; the target stream is drawn only for the tokens right after a hand-off that stalls.
+template <bool LEAN>
 __global__ void __launch_bounds__(kFastWarps * 32)
 k_playout_fast(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __restrict__ ccp,
                const int32_t* __restrict__ knots, uint32_t k0, TimelineRec rec, uint32_t* __restrict__ todo,
@@ -132,25 +136,39 @@ k_playout_fast(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst
 
         // ---- every token: hash draw and both endpoints' jitter, ((h * (2J+1)) >> 32)
         const int Lmax = (int)__reduce_max_sync(FULL, L);
-        uint32_t hS = 0, hD = 0, xS = 0, xD = 0;
         uint32_t hin = key + j0 * kHashTok;
+        int32_t s_S = 0, s_D = 0;
+        bool clean = true;
+        if (LEAN) {
+            const uint32_t mul = G.cand == 2 ? G.mulD : G.mulS;    // the stream of the endpoint that may hand over
+            uint32_t hC = 0;
 #pragma unroll 4
-        for (int t = 0; t < Lmax; ++t) {
-            uint32_t h = mix32(hin);
-            hin += kHashTok;
-            h = t < cnt ? h : 0u;
-            const uint32_t x = __umulhi(h, G.mulS), y = __umulhi(h, G.mulD);
-            hS += x; hD += y; xS = max(xS, x); xD = max(xD, y);
+            for (int t = 0; t < Lmax; ++t) {
+                const uint32_t x = __umulhi(mix32(hin), mul);
+                hin += kHashTok;
+                if (t < cnt) hC += x;
+            }
+            s_S = s_D = cnt * (G.cand == 2 ? G.cD_base : G.cS_base) - (int32_t)hC;
+        } else {
+            uint32_t hS = 0, hD = 0, xS = 0, xD = 0;
+#pragma unroll 4
+            for (int t = 0; t < Lmax; ++t) {
+                uint32_t h = mix32(hin);
+                hin += kHashTok;
+                h = t < cnt ? h : 0u;
+                const uint32_t x = __umulhi(h, G.mulS), y = __umulhi(h, G.mulD);
+                hS += x; hD += y; xS = max(xS, x); xD = max(xD, y);
+            }
+            s_S = cnt * G.cS_base - (int32_t)hS; s_D = cnt * G.cD_base - (int32_t)hD;
+            const bool neg = cnt != 0 && ((int32_t)xS > G.cS_base || (int32_t)xD > G.cD_base);   // some c_j < 0
+            clean = (__ballot_sync(FULL, neg) & tmask) == 0;
+            if (nI != 0 && !clean && q == 0) todo[atomicAdd(todo_count, 1u)] = batch0 + r;   // for the general kernel
         }
-        const int32_t s_S = cnt * G.cS_base - (int32_t)hS, s_D = cnt * G.cD_base - (int32_t)hD;
-        const bool neg = cnt != 0 && ((int32_t)xS > G.cS_base || (int32_t)xD > G.cD_base);   // some c_j < 0
-        const bool clean = (__ballot_sync(FULL, neg) & tmask) == 0;
-        if (nI != 0 && !clean && q == 0) todo[atomicAdd(todo_count, 1u)] = batch0 + r;   // for the general kernel
         const bool go = clean && nI != 0;
         // ---- hand-off index on the candidate stream
         const int cand = go ? G.cand : 0;
         const int32_t sC = cand == 1 ? s_S : s_D, sT = cand == 1 ? s_D : s_S;
-        const int32_t inC = team_inclusive_sum(sC, q), inT = team_inclusive_sum(sT, q);
+        const int32_t inC = team_inclusive_sum(sC, q), inT = LEAN ? 0 : team_inclusive_sum(sT, q);
         const uint32_t mulC = cand == 1 ? G.mulS : G.mulD, mulT = cand == 1 ? G.mulD : G.mulS;
         const int32_t cC_base = cand == 1 ? G.cS_base : G.cD_base, cT_base = cand == 1 ? G.cD_base : G.cS_base;
         uint32_t m = 0;
@@ -172,6 +190,7 @@ k_playout_fast(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst
         }
         // ---- stream X
         uint32_t stall = 0, delayed = 0;
+        int32_t need_lean = 0;                                     // LEAN: how late token m+1 is, if it stalls
         if (m) {                                                   // team-uniform
             uint32_t M;
             if (cand == 1) M = (uint32_t)G.kappa * (l + m) + (uint32_t)G.c0;       // device re-prefills prompt + m tokens
@@ -182,7 +201,8 @@ k_playout_fast(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst
             }
             const int32_t v = e_m + (tau - (int32_t)M);            // slot lag of token m+1, negated
             stall = (uint32_t)tau + (uint32_t)max(-v, 0);
-            if (v < 0) {
+            if (LEAN) need_lean = max(-v, 0);
+            if (!LEAN && v < 0) {
                 // tokens m+2.. stay late while the target's prefix sum of c is below `need`
                 const int32_t need = -v;
                 const uint32_t first_idx = m;                      // run-global index (j - 2) of token m+2
@@ -203,6 +223,26 @@ k_playout_fast(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst
                 }
                 delayed = 1u + __reduce_add_sync(tmask, contrib);
             }
+        }
+        if (LEAN) {
+            // tokens m+2.. stay late while the target's prefix sum of c (from token m+2) is below the lag.  The
+            // team draws `lanes` tokens of the target stream a round until the sum gets there (c >= 0: the
+            // late tokens are a prefix).  All 32 lanes run the rounds; teams that are done draw nothing.
+            bool more = need_lean > 0 && m + 2 <= n;
+            uint32_t jb = m + 2, late = 0;
+            int32_t carry = 0;
+            while (__any_sync(FULL, more)) {
+                const uint32_t j = jb + (uint32_t)q;
+                const bool in = more && j <= n;
+                const int32_t c = in ? cT_base - (int32_t)__umulhi(mix32(key + j * kHashTok), mulT) : 0;
+                const int32_t R = carry + team_inclusive_sum(c, q);
+                late += __popc(__ballot_sync(FULL, in && R < need_lean) & tmask);
+                const bool reached = (__ballot_sync(FULL, in && R >= need_lean) & tmask) != 0;
+                carry = __shfl_sync(FULL, R, a + lanes - 1);
+                jb += (uint32_t)lanes;
+                more = more && !reached && jb <= n;
+            }
+            if (need_lean > 0) delayed = 1u + late;
         }
         // ---- hand the results to the lanes that own the four requests' slots
         const uint32_t packed = (nI == 0 || go ? 0x80000000u : 0u) | m | (delayed << 16);
@@ -235,14 +275,15 @@ k_playout_fast(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst
 
 cudaError_t launch_playout_fast(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const int32_t* knots,
                                 uint64_t seed, TimelineRec rec, uint32_t* todo, uint32_t* todo_count,
-                                cudaStream_t st) {
+                                bool never_clamps, cudaStream_t st) {
     if (tr.n == 0) return cudaSuccess;
     // requests per warp: enough warps to fill the GPU (about 48 per SM) before batches grow to 32
     int rpw = 4;
     while (rpw < 32 && (uint64_t)tr.n / (2 * rpw) >= 148u * 48u) rpw *= 2;
     const uint32_t per_block = kFastWarps * (uint32_t)rpw;
-    k_playout_fast<<<(tr.n + per_block - 1) / per_block, kFastWarps * 32, 0, st>>>(tr, gc, cc, knots, seed_key(seed), rec,
-                                                                                    todo, todo_count, rpw);
+    auto* kernel = never_clamps ? k_playout_fast<true> : k_playout_fast<false>;
+    kernel<<<(tr.n + per_block - 1) / per_block, kFastWarps * 32, 0, st>>>(tr, gc, cc, knots, seed_key(seed), rec, todo,
+                                                                            todo_count, rpw);
     return cudaGetLastError();
 }
 
