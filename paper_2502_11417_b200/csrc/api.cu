@@ -346,7 +346,7 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
 #define R(buf, bytes) if ((e = c->buf.reserve(bytes)) != cudaSuccess) return fail_cuda(e, "device allocation for the evaluation")
     R(d_prep, (size_t)G * P * sizeof(Prep));
     const size_t acc_bytes = (size_t)P * G * kNAcc * 8, hist_bytes = (size_t)P * kNBins * 8;
-    const size_t cnt_bytes = (classes.size() * 4 + 15) / 16 * 16;        // one to-do counter per class
+    const size_t cnt_bytes = (classes.size() * 8 + 15) / 16 * 16;        // a to-do counter and a ticket counter per class
     R(d_accum, acc_bytes + 2 * hist_bytes + cnt_bytes);
     R(d_todo, N1 * 4);
     c->d_acc.p = c->d_accum.p; c->d_hist_ttft.p = (char*)c->d_accum.p + acc_bytes;
@@ -456,7 +456,7 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
             never_clamps = never_clamps && (int64_t)c->gc[g].T_srv + c->gc[g].J_srv <= classes[k].tau &&
                            (int64_t)c->gc[g].T_dev + c->gc[g].J_dev <= classes[k].tau;
         CU(launch_timeline(tr, c->d_gc.as<GroupConst>(), dcc, classes[k].pacing != 0, c->knots.as<int32_t>(), seed, rec,
-                           c->err, c->d_todo.as<uint32_t>(), todo_counts + k, never_clamps, timed ? c->ev[1] : nullptr, st));
+                           c->err, c->d_todo.as<uint32_t>(), todo_counts + 2 * k, never_clamps, timed ? c->ev[1] : nullptr, st));
         if (timed) CU(cudaEventRecord(c->ev[2], st));
         CU(launch_pairs(tr, c->d_gc.as<GroupConst>(), dcc, c->d_prep.as<Prep>(), P,
                         c->d_pol_list.as<uint32_t>() + cls_range[k].first, cls_range[k].second - cls_range[k].first,

@@ -132,7 +132,7 @@ cudaError_t launch_prep_beta(const PolicyConst* pol, uint32_t P, int G, const in
                              const int32_t* sorted, const uint32_t* grp_off, Prep* prep, cudaStream_t st);
 cudaError_t launch_timeline(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, bool pacing,
                             const int32_t* knots, uint64_t seed, TimelineRec rec, int32_t* err, uint32_t* todo,
-                            uint32_t* todo_count /* zero on entry */,
+                            uint32_t* todo_count /* two words, zero on entry: length of the list, batch tickets */,
                             bool never_clamps /* pacing on and tau >= T + J for both endpoints of every group */,
                             cudaEvent_t mid /* recorded between its two kernels, or null */,
                             cudaStream_t st);

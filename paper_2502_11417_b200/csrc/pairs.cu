@@ -373,13 +373,34 @@ constexpr int kRowThreads = 256;
 constexpr int kRowPols = 32;
 constexpr int kRowVec = 7;              // uint4 per request: six outcome rows and one of padding (odd stride)
 
-template <bool EXT>
+// What the dispatch of one (group, policy) needs, with the mode tests folded into the thresholds: Algorithm 3
+// has no waits (l_star beyond every length), Algorithm 2 no device-only prompts (l_th = 0, as the preparation
+// kernel leaves it), and a policy or group without migration never passes the trigger (theta = +inf).
+struct __align__(8) RowPol {
+    int32_t l_th, l_star;
+    uint32_t w_star, w_tail;
+    float theta;
+    uint32_t pol;
+};
+
+__device__ __forceinline__ RowPol row_pol(const Prep& pr, int candidate, uint32_t p) {
+    RowPol r;
+    r.l_th = pr.l_th; r.l_star = pr.device_constrained ? pr.l_star : 0x7FFFFFFF;
+    r.w_star = (uint32_t)pr.w_star; r.w_tail = (uint32_t)pr.w_tail;
+    r.theta = (pr.mig_on && candidate != 0) ? pr.theta : __int_as_float(0x7F800000);
+    r.pol = p;
+    return r;
+}
+
+// IDX32: every element index p * N + i fits 32 bits, so a store address is one widening multiply-add.
+template <bool EXT, bool IDX32>
 __global__ void __launch_bounds__(kRowThreads)
 k_pairs_rows(TraceDev tr, const GroupConst* __restrict__ gcs, const Prep* __restrict__ prep, uint32_t P,
              const uint32_t* __restrict__ pol_list, uint32_t n_list, TimelineRec rec, uint32_t k0,
              disco_pair_out_t out) {
-    __shared__ Prep s_prep[kRowPols];
-    __shared__ uint32_t s_pol[kRowPols];
+    using idx_t = typename std::conditional<IDX32, uint32_t, size_t>::type;
+    __shared__ Prep s_prep[EXT ? kRowPols : 1];
+    __shared__ RowPol s_rp[kRowPols];
     __shared__ uint4 s_rows[kRowThreads * kRowVec];
     const uint32_t first = blockIdx.y * kRowPols;
     const int npol = (int)min((uint32_t)kRowPols, n_list - first);
@@ -392,8 +413,9 @@ k_pairs_rows(TraceDev tr, const GroupConst* __restrict__ gcs, const Prep* __rest
     const bool one_group = g_lo == g_hi;
     if ((int)threadIdx.x < npol) {
         const uint32_t p = pol_list[first + threadIdx.x];
-        s_pol[threadIdx.x] = p;
-        s_prep[threadIdx.x] = prep[(size_t)g_lo * P + p];
+        const Prep pr = prep[(size_t)g_lo * P + p];
+        if (EXT) s_prep[threadIdx.x] = pr;
+        s_rp[threadIdx.x] = row_pol(pr, gcs[g_lo].candidate, p);
     }
     __syncthreads();
     const uint32_t k = k_lo + threadIdx.x;
@@ -402,8 +424,9 @@ k_pairs_rows(TraceDev tr, const GroupConst* __restrict__ gcs, const Prep* __rest
     while (g < g_hi && k >= tr.grp_off[g + 1]) ++g;
     const GroupConst& gc = gcs[g];
     const int candidate = gc.candidate;
+    const bool dev_migrates = candidate == 2;
     const float delta_c = gc.delta_c, cps = gc.cps, cds = gc.cds, lcpd = gc.lcpd, lcdd = gc.lcdd;
-    const size_t N = tr.n;
+    const idx_t N = (idx_t)tr.n;
 
     PairIn q;
     q.l = tr.l[k]; q.n = tr.nout[k]; q.S = (uint32_t)tr.S[k]; q.m = rec.m[k];
@@ -412,8 +435,10 @@ k_pairs_rows(TraceDev tr, const GroupConst* __restrict__ gcs, const Prep* __rest
     const uint32_t orig = tr.orig[k];
     q.u = EXT ? routing_draw(k0, orig) : 0u;
     const uint32_t Td = (uint32_t)gc.kappa * q.l + (uint32_t)gc.c0, dly = rec.delayed[k];
-    uint4* row = s_rows + threadIdx.x * kRowVec;
+    const float saving_m = q.m ? q.saving : -1.0f;        // a request migrates only if its buffer filled (m != 0)
+    const uint4* row = s_rows + threadIdx.x * kRowVec;
     {
+        uint4* wrow = s_rows + threadIdx.x * kRowVec;
         const float inv_cnt = q.n > 1 ? 1e-6f / (float)(q.n - 1) : 0.0f;
         float mean[3], mx[3];
 #pragma unroll
@@ -422,8 +447,8 @@ k_pairs_rows(TraceDev tr, const GroupConst* __restrict__ gcs, const Prep* __rest
         auto put = [&](int oc, uint32_t pre_srv, uint32_t pre_dev, uint32_t tok_dev, int stream) {
             const uint32_t tok_srv = n - tok_dev;
             const float cost = cps * (float)pre_srv + cds * (float)tok_srv + lcpd * (float)pre_dev + lcdd * (float)tok_dev;   // Eq. 8
-            row[oc] = make_uint4(__float_as_uint(cost), tok_srv | tok_dev << 16, __float_as_uint(mean[stream]),
-                                 __float_as_uint(mx[stream]));
+            wrow[oc] = make_uint4(__float_as_uint(cost), tok_srv | tok_dev << 16, __float_as_uint(mean[stream]),
+                                  __float_as_uint(mx[stream]));
         };
         put(O_SERVER_ONLY, l, 0u, 0u, 0);
         put(O_DEVICE_ONLY, 0u, l, n, 1);
@@ -432,29 +457,45 @@ k_pairs_rows(TraceDev tr, const GroupConst* __restrict__ gcs, const Prep* __rest
         put(O_MIGR_TO_DEV, l, l + lm, n - m, 2);          // the server decoded m tokens, the device re-prefills l + m
         put(O_MIGR_TO_SRV, l + lm, l, m, 2);
     }
-    auto pair = [&](const Prep& pr, size_t at) {
-        const PairOut o = decide<EXT>(q, pr, Td, candidate);
-        const int oc = o.dev_only ? O_DEVICE_ONLY
-                                  : (!o.started ? O_SERVER_ONLY : (o.dev_wins ? O_RACE_DEV : O_RACE_SRV) + (o.migr ? 2 : 0));
+    auto emit = [&](idx_t at, bool dev_only, bool started, bool dev_wins, bool migr, uint32_t ttft) {
+        const int oc = dev_only ? O_DEVICE_ONLY
+                                : (!started ? O_SERVER_ONLY : (dev_wins ? O_RACE_DEV : O_RACE_SRV) + (migr ? 2 : 0));
         const uint4 r = row[oc];
-        if (out.ttft_s) out.ttft_s[at] = (float)o.ttft * 1e-6f;
+        if (out.ttft_s) out.ttft_s[at] = (float)ttft * 1e-6f;
         if (out.tbt_mean_s) out.tbt_mean_s[at] = __uint_as_float(r.z);
         if (out.tbt_max_s) out.tbt_max_s[at] = __uint_as_float(r.w);
         if (out.cost) out.cost[at] = __uint_as_float(r.x);
         if (out.tok_server) out.tok_server[at] = r.y & 0xFFFFu;
         if (out.tok_device) out.tok_device[at] = r.y >> 16;
-        if (out.mig_at) out.mig_at[at] = o.migr ? q.m : 0u;
-        if (out.delayed) out.delayed[at] = (uint16_t)(o.migr ? dly : 0u);
-        if (out.decision) out.decision[at] = (uint8_t)(o.dev_only ? DISCO_DEVICE_ONLY
-                                                                 : (o.started ? DISCO_RACE : DISCO_SERVER_ONLY));
+        if (out.mig_at) out.mig_at[at] = migr ? q.m : 0u;
+        if (out.delayed) out.delayed[at] = (uint16_t)(migr ? dly : 0u);
+        if (out.decision) out.decision[at] = (uint8_t)(dev_only ? DISCO_DEVICE_ONLY : (started ? DISCO_RACE : DISCO_SERVER_ONLY));
+    };
+    auto pair = [&](const RowPol& rp, const Prep* full) {
+        const idx_t at = (idx_t)rp.pol * N + (idx_t)orig;
+        if (EXT) {
+            const PairOut o = decide<true>(q, *full, Td, candidate);
+            emit(at, o.dev_only, o.started, o.dev_wins, o.migr, o.ttft);
+            return;
+        }
+        // ---- dispatch (Algorithm 2's wait map / Algorithm 3's threshold) and the race
+        const bool dev_only = (int32_t)q.l < rp.l_th;
+        const uint32_t w = (int32_t)q.l < rp.l_star ? 0u : ((int32_t)q.l == rp.l_star ? rp.w_star : rp.w_tail);
+        const bool started = dev_only || q.S > w;               // the device starts after the wait
+        const uint32_t wTd = w + Td;
+        const bool dev_wins = dev_only || (started && q.S > wTd);   // a tie goes to the server
+        const uint32_t ttft = dev_only ? Td : min(q.S, wTd);
+        const bool migr = started && !dev_only && dev_wins == dev_migrates && saving_m > rp.theta;
+        emit(at, dev_only, started, dev_wins, migr, ttft);
     };
     if (one_group) {
 #pragma unroll 4
-        for (int pi = 0; pi < npol; ++pi) pair(s_prep[pi], (size_t)s_pol[pi] * N + orig);
+        for (int pi = 0; pi < npol; ++pi) pair(s_rp[pi], EXT ? &s_prep[pi] : nullptr);
     } else {
         for (int pi = 0; pi < npol; ++pi) {
-            const Prep pr = prep[(size_t)g * P + s_pol[pi]];
-            pair(pr, (size_t)s_pol[pi] * N + orig);
+            const Prep pr = prep[(size_t)g * P + s_rp[pi].pol];
+            const RowPol rp = row_pol(pr, candidate, s_rp[pi].pol);
+            pair(rp, &pr);
         }
     }
 }
@@ -469,7 +510,6 @@ cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassCo
     int PL = 1;
     while (PL < 32 && (uint32_t)PL < n_list) PL <<= 1;
     auto* acc_kernel = extras ? k_pairs_acc<true> : k_pairs_acc<false>;
-    auto* row_kernel = extras ? k_pairs_rows<true> : k_pairs_rows<false>;
     const uint32_t k0 = seed_key(seed);
     cudaError_t e = cudaFuncSetAttribute(acc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)acc_smem_bytes(32));
@@ -484,6 +524,9 @@ cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassCo
     const bool rows = out.ttft_s || out.tbt_mean_s || out.tbt_max_s || out.cost || out.tok_server || out.tok_device ||
                       out.mig_at || out.delayed || out.decision;
     if (rows) {
+        const bool idx32 = (uint64_t)P * tr.n <= 0xFFFFFFFFull;
+        auto* row_kernel = extras ? (idx32 ? k_pairs_rows<true, true> : k_pairs_rows<true, false>)
+                                  : (idx32 ? k_pairs_rows<false, true> : k_pairs_rows<false, false>);
         dim3 grid_r((tr.n + kRowThreads - 1) / kRowThreads, (n_list + kRowPols - 1) / kRowPols);
         row_kernel<<<grid_r, kRowThreads, 0, st>>>(tr, gc, prep, P, pol_list, n_list, rec, k0, out);
         e = cudaGetLastError();

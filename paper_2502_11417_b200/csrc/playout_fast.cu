@@ -1,8 +1,8 @@
 // Decode play-out (Sec. 4.3) for requests whose streams never clamp: both endpoints generate every token
 // no slower than it is consumed (c_j = tau - x_j >= 0 for all j), so delivery is exactly tau-paced.
 //
-// A warp plays four requests at a time and shares its 32 lanes among them in proportion to their token
-// counts (every lane then owns a contiguous run of about the same length, whatever the mix of lengths).
+// A warp plays eight requests at a time and shares its 32 lanes among them by their token counts (every
+// lane then owns a contiguous run of about the same length, whatever the mix of lengths).
 // Every token's hash is drawn and mapped to both endpoints' jitter; the lane keeps the sums and maxima.  If any c_j is negative the request is put on a list for the general kernel (playout.cu).
 // Otherwise:
 //  * streams S and D: every TBT equals tau;
@@ -10,6 +10,8 @@
 //    candidate stream exceeds (B-1) tau; the owning lane re-draws its run up to that token;
 //  * stream X: token m+1 waits for the hand-off latency M; it is `need` = M - e_m - tau late if that is
 //    positive, and each later token of the target stream gains its c_j until the lag is made up.
+#include <algorithm>
+
 #include "disco_internal.cuh"
 
 namespace disco {
@@ -17,7 +19,7 @@ namespace disco {
 namespace {
 
 constexpr uint32_t FULL = 0xFFFFFFFFu;
-constexpr int kPerIter = 4;               // requests a warp plays at a time
+constexpr int kPerIter = 8;               // requests a warp plays at a time
 constexpr int kFastWarps = 8;
 
 struct LaneGroup {                       // constants of a lane's current request group
@@ -56,7 +58,7 @@ __device__ __forceinline__ uint32_t walk(uint32_t key, uint32_t j0, int t0, int 
 }
 
 
-// rpw = requests per warp (4, 8, 16 or 32): small traces use small batches so that enough warps are in flight.
+// rpw = requests per warp (8, 16 or 32): small traces use small batches so that enough warps are in flight.
 // LEAN: the host has checked that tau >= T + J for both endpoints of every group, so no interval can exceed
 // tau and every request is clamp-free by construction.  Then only the candidate stream's sums are needed to
 // find the hand-off index; the target stream is drawn only for the tokens right after a hand-off that stalls.
@@ -64,10 +66,8 @@ template <bool LEAN>
 __global__ void __launch_bounds__(kFastWarps * 32)
 k_playout_fast(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __restrict__ ccp,
                const int32_t* __restrict__ knots, uint32_t k0, TimelineRec rec, uint32_t* __restrict__ todo,
-               uint32_t* __restrict__ todo_count, int rpw) {
-    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
-    const uint32_t batch0 = (blockIdx.x * kFastWarps + wib) * (uint32_t)rpw;
-    if (batch0 >= tr.n) return;
+               uint32_t* __restrict__ todo_count, uint32_t* __restrict__ tickets, int rpw) {
+    const int lane = threadIdx.x & 31;
     const ClassConst& cc = *ccp;
     const int32_t tau = cc.tau;                                   // pacing is on for every launch of this kernel
     const uint32_t B = (uint32_t)cc.B;
@@ -76,198 +76,209 @@ k_playout_fast(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst
     const int W0 = cc.W[0], W1 = cc.W[1], W2 = cc.W[2];
     const bool mig_any = cc.mig_any != 0;
 
-    // ---- one request per lane: inputs
-    const uint32_t kk = batch0 + lane;
-    const bool live = lane < rpw && kk < tr.n;
-    uint32_t n_l = 1, l_l = 1, key_l = 0;
-    int g_l = 0;
-    if (live) {
-        n_l = tr.nout[kk]; l_l = tr.l[kk];
-        key_l = mix32(k0 + tr.orig[kk] * kHashReq);
-        while (g_l + 1 < tr.n_groups && kk >= tr.grp_off[g_l + 1]) ++g_l;
-    }
-    // ---- one request per lane: results (bit 31 of o_md: played here; bits 0-15 m, 16-30 late tokens)
-    uint32_t o_md = 0, o_stall = 0;
-
     LaneGroup G;
     int cur_g = -1;
+    // Batches of rpw requests are handed out by a ticket counter (zero at launch), so a warp that drew short
+    // requests takes more of them and the last batches are spread over the whole GPU.
+    for (;;) {
+        uint32_t ticket = 0;
+        if (lane == 0) ticket = atomicAdd(tickets, 1u);
+        const uint32_t batch0 = __shfl_sync(FULL, ticket, 0) * (uint32_t)rpw;
+        if (batch0 >= tr.n) break;
+        // ---- one request per lane: inputs
+        const uint32_t kk = batch0 + lane;
+        const bool live = lane < rpw && kk < tr.n;
+        uint32_t n_l = 1, l_l = 1, key_l = 0;
+        int g_l = 0;
+        if (live) {
+            n_l = tr.nout[kk]; l_l = tr.l[kk];
+            key_l = mix32(k0 + tr.orig[kk] * kHashReq);
+            while (g_l + 1 < tr.n_groups && kk >= tr.grp_off[g_l + 1]) ++g_l;
+        }
+        // ---- one request per lane: results (bit 31 of o_md: played here; bits 0-15 m, 16-30 late tokens)
+        uint32_t o_md = 0, o_stall = 0;
 
-    for (int it = 0; it < rpw / kPerIter; ++it) {
-        // ---- share the lanes among the four requests in proportion to their intervals (n - 1 each)
-        const int r0 = it * kPerIter;
-        const uint32_t nI0 = __shfl_sync(FULL, n_l, r0) - 1, nI1 = __shfl_sync(FULL, n_l, r0 + 1) - 1;
-        const uint32_t nI2 = __shfl_sync(FULL, n_l, r0 + 2) - 1, nI3 = __shfl_sync(FULL, n_l, r0 + 3) - 1;
-        const uint32_t tot = nI0 + nI1 + nI2 + nI3;
-        int b1 = 0, b2 = 0, b3 = 0;                                // team i owns lanes [b_i, b_{i+1}), b0 = 0, b4 = 32
-        if (tot) {
-            b1 = (int)((32u * nI0 + tot / 2) / tot);
-            b2 = (int)((32u * (nI0 + nI1) + tot / 2) / tot);
-            b3 = (int)((32u * (nI0 + nI1 + nI2) + tot / 2) / tot);
-            b1 = max(b1, (int)(nI0 != 0));                         // a request with tokens gets at least one lane
-            b2 = max(b2, b1 + (int)(nI1 != 0));
-            b3 = max(b3, b2 + (int)(nI2 != 0));
-            b3 = min(b3, 32 - (int)(nI3 != 0));
-            b2 = min(b2, b3 - (int)(nI2 != 0));
-            b1 = min(b1, b2 - (int)(nI1 != 0));
-        }
-        const int team = (lane >= b1) + (lane >= b2) + (lane >= b3);
-        const int a = team == 0 ? 0 : (team == 1 ? b1 : (team == 2 ? b2 : b3));
-        const int a_next = team == 0 ? b1 : (team == 1 ? b2 : (team == 2 ? b3 : 32));
-        const int lanes = a_next - a, q = lane - a;
-        const uint32_t tmask = lanes == 32 ? FULL : (((1u << lanes) - 1u) << a);   // this team's lanes: teams may diverge
-        const int r = r0 + team;
-        const uint32_t n = __shfl_sync(FULL, n_l, r), l = __shfl_sync(FULL, l_l, r);
-        const uint32_t key = __shfl_sync(FULL, key_l, r);
-        const int g = __shfl_sync(FULL, g_l, r);
-        if (g != cur_g) {
-            cur_g = g;
-            const GroupConst& gc = gcs[g];
-            G.mulS = 2u * (uint32_t)gc.J_srv + 1u; G.mulD = 2u * (uint32_t)gc.J_dev + 1u;
-            G.cS_base = tau - (gc.T_srv - gc.J_srv); G.cD_base = tau - (gc.T_dev - gc.J_dev);
-            G.kappa = gc.kappa; G.c0 = gc.c0;
-            G.cand = mig_any ? gc.candidate : 0;
-            G.K = knots + g * kNKnots;
-        }
-        const uint32_t nI = tot ? n - 1 : 0u;                      // inter-token intervals, tokens 2..n
-        const uint32_t L = (nI + (uint32_t)lanes - 1) / (uint32_t)lanes;   // tokens per lane (lanes >= 1 here)
-        const uint32_t lo = (uint32_t)q * L;
-        const int cnt = lo >= nI ? 0 : (int)min(L, nI - lo);
-        const uint32_t j0 = lo + 2;
+        for (int it = 0; it < rpw / kPerIter; ++it) {
+            // ---- share the lanes among the eight requests: one lane for each request that has intervals, the
+            //      other lanes in proportion to the intervals (n - 1 each).  Any split that gives such a request
+            //      a lane is valid; the rounding only moves load.  Every group of eight lanes holds the same
+            //      eight values here, lane s of a group standing for request r0 + s.
+            const int r0 = it * kPerIter, s8 = lane & 7;
+            const uint32_t nI_s = __shfl_sync(FULL, n_l, r0 + s8) - 1;
+            uint32_t inc = nI_s;
+#pragma unroll
+            for (int off = 1; off < 8; off <<= 1) {
+                const uint32_t up = __shfl_up_sync(FULL, inc, off, 8);
+                if (s8 >= off) inc += up;
+            }
+            const uint32_t tot = __shfl_sync(FULL, inc, 7, 8);
+            const uint32_t busy = __ballot_sync(FULL, nI_s != 0) & 0xFFu;          // requests with intervals
+            const float per = __fdividef((float)(32 - __popc(busy)), (float)max(tot, 1u));
+            // first lane of request s: requests with intervals before it, plus its share of the spare lanes
+            const int start_s = __popc(busy & ((1u << s8) - 1u)) + __float2int_rn((float)(inc - nI_s) * per);
+            const bool owner_s = lane < 8 && nI_s != 0;
+            const uint32_t starts = __reduce_or_sync(FULL, owner_s ? 1u << start_s : 0u);   // bit 0 is set unless tot == 0
+            // request of the k-th team (teams in request order), four bits each
+            const uint32_t team_req = __reduce_or_sync(FULL, owner_s ? (uint32_t)s8 << (4 * __popc(busy & ((1u << s8) - 1u))) : 0u);
+            const uint32_t upto = starts & (0xFFFFFFFFu >> (31 - lane));           // team starts at or below this lane
+            const uint32_t after = starts & ~(0xFFFFFFFFu >> (31 - lane));
+            const int a = upto ? 31 - __clz(upto) : 0;
+            const int a_next = after ? __ffs(after) - 1 : 32;
+            const int lanes = a_next - a, q = lane - a;
+            const uint32_t tmask = lanes == 32 ? FULL : (((1u << lanes) - 1u) << a);   // this team's lanes: teams may diverge
+            const int r = r0 + (int)((team_req >> (4 * max(__popc(upto) - 1, 0))) & 7u);
+            const uint32_t n = __shfl_sync(FULL, n_l, r), l = __shfl_sync(FULL, l_l, r);
+            const uint32_t key = __shfl_sync(FULL, key_l, r);
+            const int g = __shfl_sync(FULL, g_l, r);
+            if (g != cur_g) {
+                cur_g = g;
+                const GroupConst& gc = gcs[g];
+                G.mulS = 2u * (uint32_t)gc.J_srv + 1u; G.mulD = 2u * (uint32_t)gc.J_dev + 1u;
+                G.cS_base = tau - (gc.T_srv - gc.J_srv); G.cD_base = tau - (gc.T_dev - gc.J_dev);
+                G.kappa = gc.kappa; G.c0 = gc.c0;
+                G.cand = mig_any ? gc.candidate : 0;
+                G.K = knots + g * kNKnots;
+            }
+            const uint32_t nI = tot ? n - 1 : 0u;                      // inter-token intervals, tokens 2..n
+            // tokens per lane, ceil(nI / lanes) or one more (lanes >= 1 here); all that matters is lanes * L >= nI
+            uint32_t L = __float2uint_ru(__fdividef((float)nI, (float)lanes));
+            if (L * (uint32_t)lanes < nI) ++L;
+            const uint32_t lo = (uint32_t)q * L;
+            const int cnt = lo >= nI ? 0 : (int)min(L, nI - lo);
+            const uint32_t j0 = lo + 2;
 
-        // ---- every token: hash draw and both endpoints' jitter, ((h * (2J+1)) >> 32)
-        const int Lmax = (int)__reduce_max_sync(FULL, L);
-        uint32_t hin = key + j0 * kHashTok;
-        int32_t s_S = 0, s_D = 0;
-        bool clean = true;
-        if (LEAN) {
-            const uint32_t mul = G.cand == 2 ? G.mulD : G.mulS;    // the stream of the endpoint that may hand over
-            uint32_t hC = 0;
-#pragma unroll 4
-            for (int t = 0; t < Lmax; ++t) {
-                const uint32_t x = __umulhi(mix32(hin), mul);
-                hin += kHashTok;
-                if (t < cnt) hC += x;
-            }
-            s_S = s_D = cnt * (G.cand == 2 ? G.cD_base : G.cS_base) - (int32_t)hC;
-        } else {
-            uint32_t hS = 0, hD = 0, xS = 0, xD = 0;
-#pragma unroll 4
-            for (int t = 0; t < Lmax; ++t) {
-                uint32_t h = mix32(hin);
-                hin += kHashTok;
-                h = t < cnt ? h : 0u;
-                const uint32_t x = __umulhi(h, G.mulS), y = __umulhi(h, G.mulD);
-                hS += x; hD += y; xS = max(xS, x); xD = max(xD, y);
-            }
-            s_S = cnt * G.cS_base - (int32_t)hS; s_D = cnt * G.cD_base - (int32_t)hD;
-            const bool neg = cnt != 0 && ((int32_t)xS > G.cS_base || (int32_t)xD > G.cD_base);   // some c_j < 0
-            clean = (__ballot_sync(FULL, neg) & tmask) == 0;
-            if (nI != 0 && !clean && q == 0) todo[atomicAdd(todo_count, 1u)] = batch0 + r;   // for the general kernel
-        }
-        const bool go = clean && nI != 0;
-        // ---- hand-off index on the candidate stream
-        const int cand = go ? G.cand : 0;
-        const int32_t sC = cand == 1 ? s_S : s_D, sT = cand == 1 ? s_D : s_S;
-        const int32_t inC = team_inclusive_sum(sC, q), inT = LEAN ? 0 : team_inclusive_sum(sT, q);
-        const uint32_t mulC = cand == 1 ? G.mulS : G.mulD, mulT = cand == 1 ? G.mulD : G.mulS;
-        const int32_t cC_base = cand == 1 ? G.cS_base : G.cD_base, cT_base = cand == 1 ? G.cD_base : G.cS_base;
-        uint32_t m = 0;
-        int32_t e_m = 0;
-        if (cand && B == 0) m = 1;                                 // nothing to fill: hand off after token 1
-        const uint32_t crossers = __ballot_sync(FULL, cand && B != 0 && inC > thr) & tmask;
-        if (crossers) {                                            // team-uniform from here on
-            const int owner = __ffs(crossers) - 1;                 // first lane whose run takes the sum past thr
-            uint32_t j_found = 0;
-            int32_t run = inC - sC;
-            if (lane == owner) {
-                bool hit;
-                const uint32_t passed = walk(key, j0, 0, cnt, cC_base, mulC, thr, true, run, hit);
-                j_found = j0 + passed;                             // hit is certain: the run's total exceeds thr
-            }
-            j_found = __shfl_sync(tmask, j_found, owner);
-            e_m = __shfl_sync(tmask, run, owner);                  // clean stream: e_m = S_m
-            m = j_found + 1 <= n ? j_found : 0u;                   // the hand-off needs a token left to generate
-        }
-        // ---- stream X
-        uint32_t stall = 0, delayed = 0;
-        int32_t need_lean = 0;                                     // LEAN: how late token m+1 is, if it stalls
-        if (m) {                                                   // team-uniform
-            uint32_t M;
-            if (cand == 1) M = (uint32_t)G.kappa * (l + m) + (uint32_t)G.c0;       // device re-prefills prompt + m tokens
-            else {
-                const uint32_t u = mix32(key);                     // a server TTFT drawn from F by its knots
-                const uint32_t ki = u >> 24, fr = (u >> 8) & 0xFFFFu;
-                M = (uint32_t)(G.K[ki] + (int32_t)(((int64_t)(G.K[ki + 1] - G.K[ki]) * (int64_t)fr) >> 16));
-            }
-            const int32_t v = e_m + (tau - (int32_t)M);            // slot lag of token m+1, negated
-            stall = (uint32_t)tau + (uint32_t)max(-v, 0);
-            if (LEAN) need_lean = max(-v, 0);
-            if (!LEAN && v < 0) {
-                // tokens m+2.. stay late while the target's prefix sum of c is below `need`
-                const int32_t need = -v;
-                const uint32_t first_idx = m;                      // run-global index (j - 2) of token m+2
-                const int qs = (int)min((uint32_t)(lanes - 1), first_idx / L);
-                int32_t runA = 0;
-                uint32_t contrib = 0;
-                bool hitA = false;
-                if (q == qs && first_idx < nI)
-                    contrib = walk(key, j0, (int)(first_idx - lo), cnt, cT_base, mulT, need, false, runA, hitA);
-                runA = __shfl_sync(tmask, runA, a + qs);
-                hitA = __shfl_sync(tmask, (int)hitA, a + qs) != 0;
-                const int32_t inT_qs = __shfl_sync(tmask, inT, a + qs);
-                if (!hitA && q > qs && cnt) {
-                    const int32_t through = runA + (inT - inT_qs);               // target's sum up to this run's end
-                    int32_t before = through - sT;
-                    if (through < need) contrib = (uint32_t)cnt;
-                    else if (before < need) { bool hit; contrib = walk(key, j0, 0, cnt, cT_base, mulT, need, false, before, hit); }
+            // ---- every token: hash draw and both endpoints' jitter, ((h * (2J+1)) >> 32)
+            const int Lmax = (int)__reduce_max_sync(FULL, L);
+            uint32_t hin = key + j0 * kHashTok;
+            int32_t s_S = 0, s_D = 0;
+            bool clean = true;
+            if (LEAN) {
+                const uint32_t mul = G.cand == 2 ? G.mulD : G.mulS;    // the stream of the endpoint that may hand over
+                uint32_t hC = 0;
+    #pragma unroll 4
+                for (int t = 0; t < Lmax; ++t) {
+                    const uint32_t x = __umulhi(mix32(hin), mul);
+                    hin += kHashTok;
+                    if (t < cnt) hC += x;
                 }
-                delayed = 1u + __reduce_add_sync(tmask, contrib);
+                s_S = s_D = cnt * (G.cand == 2 ? G.cD_base : G.cS_base) - (int32_t)hC;
+            } else {
+                uint32_t hS = 0, hD = 0, xS = 0, xD = 0;
+    #pragma unroll 4
+                for (int t = 0; t < Lmax; ++t) {
+                    uint32_t h = mix32(hin);
+                    hin += kHashTok;
+                    h = t < cnt ? h : 0u;
+                    const uint32_t x = __umulhi(h, G.mulS), y = __umulhi(h, G.mulD);
+                    hS += x; hD += y; xS = max(xS, x); xD = max(xD, y);
+                }
+                s_S = cnt * G.cS_base - (int32_t)hS; s_D = cnt * G.cD_base - (int32_t)hD;
+                const bool neg = cnt != 0 && ((int32_t)xS > G.cS_base || (int32_t)xD > G.cD_base);   // some c_j < 0
+                clean = (__ballot_sync(FULL, neg) & tmask) == 0;
+                if (nI != 0 && !clean && q == 0) todo[atomicAdd(todo_count, 1u)] = batch0 + r;   // for the general kernel
+            }
+            const bool go = clean && nI != 0;
+            // ---- hand-off index on the candidate stream
+            const int cand = go ? G.cand : 0;
+            const int32_t sC = cand == 1 ? s_S : s_D, sT = cand == 1 ? s_D : s_S;
+            const int32_t inC = team_inclusive_sum(sC, q), inT = LEAN ? 0 : team_inclusive_sum(sT, q);
+            const uint32_t mulC = cand == 1 ? G.mulS : G.mulD, mulT = cand == 1 ? G.mulD : G.mulS;
+            const int32_t cC_base = cand == 1 ? G.cS_base : G.cD_base, cT_base = cand == 1 ? G.cD_base : G.cS_base;
+            uint32_t m = 0;
+            int32_t e_m = 0;
+            if (cand && B == 0) m = 1;                                 // nothing to fill: hand off after token 1
+            const uint32_t crossers = __ballot_sync(FULL, cand && B != 0 && inC > thr) & tmask;
+            if (crossers) {                                            // team-uniform from here on
+                const int owner = __ffs(crossers) - 1;                 // first lane whose run takes the sum past thr
+                uint32_t j_found = 0;
+                int32_t run = inC - sC;
+                if (lane == owner) {
+                    bool hit;
+                    const uint32_t passed = walk(key, j0, 0, cnt, cC_base, mulC, thr, true, run, hit);
+                    j_found = j0 + passed;                             // hit is certain: the run's total exceeds thr
+                }
+                j_found = __shfl_sync(tmask, j_found, owner);
+                e_m = __shfl_sync(tmask, run, owner);                  // clean stream: e_m = S_m
+                m = j_found + 1 <= n ? j_found : 0u;                   // the hand-off needs a token left to generate
+            }
+            // ---- stream X
+            uint32_t stall = 0, delayed = 0;
+            int32_t need_lean = 0;                                     // LEAN: how late token m+1 is, if it stalls
+            if (m) {                                                   // team-uniform
+                uint32_t M;
+                if (cand == 1) M = (uint32_t)G.kappa * (l + m) + (uint32_t)G.c0;       // device re-prefills prompt + m tokens
+                else {
+                    const uint32_t u = mix32(key);                     // a server TTFT drawn from F by its knots
+                    const uint32_t ki = u >> 24, fr = (u >> 8) & 0xFFFFu;
+                    M = (uint32_t)(G.K[ki] + (int32_t)(((int64_t)(G.K[ki + 1] - G.K[ki]) * (int64_t)fr) >> 16));
+                }
+                const int32_t v = e_m + (tau - (int32_t)M);            // slot lag of token m+1, negated
+                stall = (uint32_t)tau + (uint32_t)max(-v, 0);
+                if (LEAN) need_lean = max(-v, 0);
+                if (!LEAN && v < 0) {
+                    // tokens m+2.. stay late while the target's prefix sum of c is below `need`
+                    const int32_t need = -v;
+                    const uint32_t first_idx = m;                      // run-global index (j - 2) of token m+2
+                    const int qs = (int)min((uint32_t)(lanes - 1), first_idx / L);
+                    int32_t runA = 0;
+                    uint32_t contrib = 0;
+                    bool hitA = false;
+                    if (q == qs && first_idx < nI)
+                        contrib = walk(key, j0, (int)(first_idx - lo), cnt, cT_base, mulT, need, false, runA, hitA);
+                    runA = __shfl_sync(tmask, runA, a + qs);
+                    hitA = __shfl_sync(tmask, (int)hitA, a + qs) != 0;
+                    const int32_t inT_qs = __shfl_sync(tmask, inT, a + qs);
+                    if (!hitA && q > qs && cnt) {
+                        const int32_t through = runA + (inT - inT_qs);               // target's sum up to this run's end
+                        int32_t before = through - sT;
+                        if (through < need) contrib = (uint32_t)cnt;
+                        else if (before < need) { bool hit; contrib = walk(key, j0, 0, cnt, cT_base, mulT, need, false, before, hit); }
+                    }
+                    delayed = 1u + __reduce_add_sync(tmask, contrib);
+                }
+            }
+            if (LEAN) {
+                // tokens m+2.. stay late while the target's prefix sum of c (from token m+2) is below the lag.  The
+                // team draws `lanes` tokens of the target stream a round until the sum gets there (c >= 0: the
+                // late tokens are a prefix).  All 32 lanes run the rounds; teams that are done draw nothing.
+                bool more = need_lean > 0 && m + 2 <= n;
+                uint32_t jb = m + 2, late = 0;
+                int32_t carry = 0;
+                while (__any_sync(FULL, more)) {
+                    const uint32_t j = jb + (uint32_t)q;
+                    const bool in = more && j <= n;
+                    const int32_t c = in ? cT_base - (int32_t)__umulhi(mix32(key + j * kHashTok), mulT) : 0;
+                    const int32_t R = carry + team_inclusive_sum(c, q);
+                    late += __popc(__ballot_sync(FULL, in && R < need_lean) & tmask);
+                    const bool reached = (__ballot_sync(FULL, in && R >= need_lean) & tmask) != 0;
+                    carry = __shfl_sync(FULL, R, a + lanes - 1);
+                    jb += (uint32_t)lanes;
+                    more = more && !reached && jb <= n;
+                }
+                if (need_lean > 0) delayed = 1u + late;
+            }
+            // ---- hand the results to the lanes that own the eight requests' slots
+            const uint32_t packed = (nI == 0 || go ? 0x80000000u : 0u) | m | (delayed << 16);
+            const uint32_t got_md = __shfl_sync(FULL, packed, start_s & 31), got_stall = __shfl_sync(FULL, stall, start_s & 31);
+            if ((lane >> 3) == it) {
+                const bool has_lanes = nI_s != 0;                      // no lanes: a single-token request, all zeros
+                o_md = has_lanes ? got_md : 0x80000000u;
+                o_stall = has_lanes ? got_stall : 0u;
             }
         }
-        if (LEAN) {
-            // tokens m+2.. stay late while the target's prefix sum of c (from token m+2) is below the lag.  The
-            // team draws `lanes` tokens of the target stream a round until the sum gets there (c >= 0: the
-            // late tokens are a prefix).  All 32 lanes run the rounds; teams that are done draw nothing.
-            bool more = need_lean > 0 && m + 2 <= n;
-            uint32_t jb = m + 2, late = 0;
-            int32_t carry = 0;
-            while (__any_sync(FULL, more)) {
-                const uint32_t j = jb + (uint32_t)q;
-                const bool in = more && j <= n;
-                const int32_t c = in ? cT_base - (int32_t)__umulhi(mix32(key + j * kHashTok), mulT) : 0;
-                const int32_t R = carry + team_inclusive_sum(c, q);
-                late += __popc(__ballot_sync(FULL, in && R < need_lean) & tmask);
-                const bool reached = (__ballot_sync(FULL, in && R >= need_lean) & tmask) != 0;
-                carry = __shfl_sync(FULL, R, a + lanes - 1);
-                jb += (uint32_t)lanes;
-                more = more && !reached && jb <= n;
-            }
-            if (need_lean > 0) delayed = 1u + late;
+        __syncwarp();
+        // ---- one request per lane: results out
+        if (live && (o_md >> 31)) {
+            const uint32_t nI = n_l - 1, ut = (uint32_t)tau, m = o_md & 0xFFFFu, dl = (o_md >> 16) & 0x7FFFu;
+            rec.sum[0][kk] = nI * ut; rec.max[0][kk] = nI ? ut : 0u;
+            rec.sum[1][kk] = nI * ut; rec.max[1][kk] = nI ? ut : 0u;
+            rec.sum[2][kk] = m ? (nI - 1) * ut + o_stall : 0u; rec.max[2][kk] = m ? o_stall : 0u;
+            rec.stall[kk] = m ? o_stall : 0u; rec.m[kk] = (uint16_t)m; rec.delayed[kk] = (uint16_t)(m ? dl : 0u);
+            const int kt0 = cc.ktau[g_l][0], kt1 = cc.ktau[g_l][1], kt2 = cc.ktau[g_l][2];
+            for (int i = 0; i < W0; ++i) rec.win[0][(size_t)kk * W0 + i] = i == kt0 ? nI : 0u;
+            for (int i = 0; i < W1; ++i) rec.win[1][(size_t)kk * W1 + i] = i == kt1 ? nI : 0u;
+            for (int i = 0; i < W2; ++i) rec.win[2][(size_t)kk * W2 + i] = (i == kt2 && m) ? nI - 1 : 0u;
         }
-        // ---- hand the results to the lanes that own the four requests' slots
-        const uint32_t packed = (nI == 0 || go ? 0x80000000u : 0u) | m | (delayed << 16);
-        const int slot = lane & 3;                                 // which of the four requests this lane may own
-        const int src = slot == 0 ? 0 : (slot == 1 ? b1 : (slot == 2 ? b2 : b3));
-        const int src_next = slot == 0 ? b1 : (slot == 1 ? b2 : (slot == 2 ? b3 : 32));
-        const uint32_t got_md = __shfl_sync(FULL, packed, src & 31), got_stall = __shfl_sync(FULL, stall, src & 31);
-        if ((lane >> 2) == it) {
-            const bool has_lanes = tot != 0 && src_next > src;     // no lanes: a single-token request, all zeros
-            o_md = has_lanes ? got_md : 0x80000000u;
-            o_stall = has_lanes ? got_stall : 0u;
-        }
-    }
-    __syncwarp();
-    // ---- one request per lane: results out
-    if (live && (o_md >> 31)) {
-        const uint32_t nI = n_l - 1, ut = (uint32_t)tau, m = o_md & 0xFFFFu, dl = (o_md >> 16) & 0x7FFFu;
-        rec.sum[0][kk] = nI * ut; rec.max[0][kk] = nI ? ut : 0u;
-        rec.sum[1][kk] = nI * ut; rec.max[1][kk] = nI ? ut : 0u;
-        rec.sum[2][kk] = m ? (nI - 1) * ut + o_stall : 0u; rec.max[2][kk] = m ? o_stall : 0u;
-        rec.stall[kk] = m ? o_stall : 0u; rec.m[kk] = (uint16_t)m; rec.delayed[kk] = (uint16_t)(m ? dl : 0u);
-        const int kt0 = cc.ktau[g_l][0], kt1 = cc.ktau[g_l][1], kt2 = cc.ktau[g_l][2];
-        for (int i = 0; i < W0; ++i) rec.win[0][(size_t)kk * W0 + i] = i == kt0 ? nI : 0u;
-        for (int i = 0; i < W1; ++i) rec.win[1][(size_t)kk * W1 + i] = i == kt1 ? nI : 0u;
-        for (int i = 0; i < W2; ++i) rec.win[2][(size_t)kk * W2 + i] = (i == kt2 && m) ? nI - 1 : 0u;
     }
 }
 
@@ -277,13 +288,14 @@ cudaError_t launch_playout_fast(const TraceDev& tr, const GroupConst* gc, const 
                                 uint64_t seed, TimelineRec rec, uint32_t* todo, uint32_t* todo_count,
                                 bool never_clamps, cudaStream_t st) {
     if (tr.n == 0) return cudaSuccess;
-    // requests per warp: enough warps to fill the GPU (about 48 per SM) before batches grow to 32
-    int rpw = 4;
-    while (rpw < 32 && (uint64_t)tr.n / (2 * rpw) >= 148u * 48u) rpw *= 2;
+    // requests per ticket: small batches spread the end of the launch evenly; large traces amortise the ticket
+    int rpw = kPerIter;
+    while (rpw < 32 && (uint64_t)tr.n / (2 * rpw) >= 148u * 48u * 4u) rpw *= 2;
     const uint32_t per_block = kFastWarps * (uint32_t)rpw;
     auto* kernel = never_clamps ? k_playout_fast<true> : k_playout_fast<false>;
-    kernel<<<(tr.n + per_block - 1) / per_block, kFastWarps * 32, 0, st>>>(tr, gc, cc, knots, seed_key(seed), rec, todo,
-                                                                            todo_count, rpw);
+    // as many blocks as the GPU holds at once (at most six of these per SM); the ticket counter feeds them
+    const uint32_t blocks = std::min<uint32_t>((tr.n + per_block - 1) / per_block, 148u * 6u);
+    kernel<<<blocks, kFastWarps * 32, 0, st>>>(tr, gc, cc, knots, seed_key(seed), rec, todo, todo_count, todo_count + 1, rpw);
     return cudaGetLastError();
 }
 
