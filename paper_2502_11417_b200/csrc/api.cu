@@ -443,6 +443,9 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
     std::memset(&po, 0, sizeof po);
     if (out) po = *out;
 
+    uint64_t out_tokens = 0;
+    for (int g = 0; g < G; ++g) out_tokens += rb.grp_sum_n[g];
+    const bool long_outputs = out_tokens >= 512ull * n;
     // ---- per timeline class: play every request out, then evaluate the class's policies on the summaries
     g_launches += 1;
     c->timing_valid = false;
@@ -456,7 +459,8 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
             never_clamps = never_clamps && (int64_t)c->gc[g].T_srv + c->gc[g].J_srv <= classes[k].tau &&
                            (int64_t)c->gc[g].T_dev + c->gc[g].J_dev <= classes[k].tau;
         CU(launch_timeline(tr, c->d_gc.as<GroupConst>(), dcc, classes[k].pacing != 0, c->knots.as<int32_t>(), seed, rec,
-                           c->err, c->d_todo.as<uint32_t>(), todo_counts + 2 * k, never_clamps, timed ? c->ev[1] : nullptr, st));
+                           c->err, c->d_todo.as<uint32_t>(), todo_counts + 2 * k, never_clamps, long_outputs,
+                           timed ? c->ev[1] : nullptr, st));
         if (timed) CU(cudaEventRecord(c->ev[2], st));
         CU(launch_pairs(tr, c->d_gc.as<GroupConst>(), dcc, c->d_prep.as<Prep>(), P,
                         c->d_pol_list.as<uint32_t>() + cls_range[k].first, cls_range[k].second - cls_range[k].first,

@@ -134,6 +134,7 @@ cudaError_t launch_timeline(const TraceDev& tr, const GroupConst* gc, const Clas
                             const int32_t* knots, uint64_t seed, TimelineRec rec, int32_t* err, uint32_t* todo,
                             uint32_t* todo_count /* two words, zero on entry: length of the list, batch tickets */,
                             bool never_clamps /* pacing on and tau >= T + J for both endpoints of every group */,
+                            bool long_outputs /* mean output length of 512 tokens or more */,
                             cudaEvent_t mid /* recorded between its two kernels, or null */,
                             cudaStream_t st);
 cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const Prep* prep, uint32_t P,

@@ -509,13 +509,13 @@ k_playout(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __r
 
 cudaError_t launch_playout_fast(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const int32_t* knots,
                                 uint64_t seed, TimelineRec rec, uint32_t* todo, uint32_t* todo_count, bool never_clamps,
-                                cudaStream_t st);
+                                bool long_outputs, cudaStream_t st);
 
 // pacing: with the delivery buffer on, the clamp-free kernel plays every request it can and lists the rest
 // in todo[0 .. *todo_count) (todo_count must be zero on entry); the general kernel then plays the list.
 cudaError_t launch_timeline(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, bool pacing,
                             const int32_t* knots, uint64_t seed, TimelineRec rec, int32_t* err, uint32_t* todo,
-                            uint32_t* todo_count, bool never_clamps, cudaEvent_t mid, cudaStream_t st) {
+                            uint32_t* todo_count, bool never_clamps, bool long_outputs, cudaEvent_t mid, cudaStream_t st) {
     if (tr.n == 0) return cudaSuccess;
     const uint32_t per_block = kWarps * 32;
     if (!pacing) {
@@ -524,7 +524,7 @@ cudaError_t launch_timeline(const TraceDev& tr, const GroupConst* gc, const Clas
         k_playout<<<blocks, kWarps * 32, 0, st>>>(tr, gc, cc, knots, seed_key(seed), rec, err, nullptr, nullptr, tr.n);
         return cudaGetLastError();
     }
-    cudaError_t e = launch_playout_fast(tr, gc, cc, knots, seed, rec, todo, todo_count, never_clamps, st);
+    cudaError_t e = launch_playout_fast(tr, gc, cc, knots, seed, rec, todo, todo_count, never_clamps, long_outputs, st);
     if (e) return e;
     if (mid && (e = cudaEventRecord(mid, st))) return e;
     if (never_clamps) return cudaSuccess;             // no interval can exceed tau: the list stays empty

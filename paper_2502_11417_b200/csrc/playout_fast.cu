@@ -1,7 +1,7 @@
 // Decode play-out (Sec. 4.3) for requests whose streams never clamp: both endpoints generate every token
 // no slower than it is consumed (c_j = tau - x_j >= 0 for all j), so delivery is exactly tau-paced.
 //
-// A warp plays eight requests at a time and shares its 32 lanes among them by their token counts (every
+// A warp plays four or eight requests at a time and shares its 32 lanes among them by their token counts (every
 // lane then owns a contiguous run of about the same length, whatever the mix of lengths).
 // Every token's hash is drawn and mapped to both endpoints' jitter; the lane keeps the sums and maxima.  If any c_j is negative the request is put on a list for the general kernel (playout.cu).
 // Otherwise:
@@ -19,7 +19,6 @@ namespace disco {
 namespace {
 
 constexpr uint32_t FULL = 0xFFFFFFFFu;
-constexpr int kPerIter = 8;               // requests a warp plays at a time
 constexpr int kFastWarps = 8;
 
 struct LaneGroup {                       // constants of a lane's current request group
@@ -62,7 +61,7 @@ __device__ __forceinline__ uint32_t walk(uint32_t key, uint32_t j0, int t0, int 
 // LEAN: the host has checked that tau >= T + J for both endpoints of every group, so no interval can exceed
 // tau and every request is clamp-free by construction.  Then only the candidate stream's sums are needed to
 // find the hand-off index; the target stream is drawn only for the tokens right after a hand-off that stalls.
-template <bool LEAN>
+template <bool LEAN, int PER>
 __global__ void __launch_bounds__(kFastWarps * 32)
 k_playout_fast(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __restrict__ ccp,
                const int32_t* __restrict__ knots, uint32_t k0, TimelineRec rec, uint32_t* __restrict__ todo,
@@ -98,25 +97,25 @@ k_playout_fast(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst
         // ---- one request per lane: results (bit 31 of o_md: played here; bits 0-15 m, 16-30 late tokens)
         uint32_t o_md = 0, o_stall = 0;
 
-        for (int it = 0; it < rpw / kPerIter; ++it) {
-            // ---- share the lanes among the eight requests: one lane for each request that has intervals, the
+        for (int it = 0; it < rpw / PER; ++it) {
+            // ---- share the lanes among the PER requests: one lane for each request that has intervals, the
             //      other lanes in proportion to the intervals (n - 1 each).  Any split that gives such a request
-            //      a lane is valid; the rounding only moves load.  Every group of eight lanes holds the same
-            //      eight values here, lane s of a group standing for request r0 + s.
-            const int r0 = it * kPerIter, s8 = lane & 7;
+            //      a lane is valid; the rounding only moves load.  Every group of PER lanes holds the same
+            //      PER values here, lane s of a group standing for request r0 + s.
+            const int r0 = it * PER, s8 = lane & (PER - 1);
             const uint32_t nI_s = __shfl_sync(FULL, n_l, r0 + s8) - 1;
             uint32_t inc = nI_s;
 #pragma unroll
-            for (int off = 1; off < 8; off <<= 1) {
-                const uint32_t up = __shfl_up_sync(FULL, inc, off, 8);
+            for (int off = 1; off < PER; off <<= 1) {
+                const uint32_t up = __shfl_up_sync(FULL, inc, off, PER);
                 if (s8 >= off) inc += up;
             }
-            const uint32_t tot = __shfl_sync(FULL, inc, 7, 8);
-            const uint32_t busy = __ballot_sync(FULL, nI_s != 0) & 0xFFu;          // requests with intervals
+            const uint32_t tot = __shfl_sync(FULL, inc, PER - 1, PER);
+            const uint32_t busy = __ballot_sync(FULL, nI_s != 0) & ((1u << PER) - 1u);   // requests with intervals
             const float per = __fdividef((float)(32 - __popc(busy)), (float)max(tot, 1u));
             // first lane of request s: requests with intervals before it, plus its share of the spare lanes
             const int start_s = __popc(busy & ((1u << s8) - 1u)) + __float2int_rn((float)(inc - nI_s) * per);
-            const bool owner_s = lane < 8 && nI_s != 0;
+            const bool owner_s = lane < PER && nI_s != 0;
             const uint32_t starts = __reduce_or_sync(FULL, owner_s ? 1u << start_s : 0u);   // bit 0 is set unless tot == 0
             // request of the k-th team (teams in request order), four bits each
             const uint32_t team_req = __reduce_or_sync(FULL, owner_s ? (uint32_t)s8 << (4 * __popc(busy & ((1u << s8) - 1u))) : 0u);
@@ -257,10 +256,10 @@ k_playout_fast(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst
                 }
                 if (need_lean > 0) delayed = 1u + late;
             }
-            // ---- hand the results to the lanes that own the eight requests' slots
+            // ---- hand the results to the lanes that own the requests' slots
             const uint32_t packed = (nI == 0 || go ? 0x80000000u : 0u) | m | (delayed << 16);
             const uint32_t got_md = __shfl_sync(FULL, packed, start_s & 31), got_stall = __shfl_sync(FULL, stall, start_s & 31);
-            if ((lane >> 3) == it) {
+            if (lane / PER == it) {
                 const bool has_lanes = nI_s != 0;                      // no lanes: a single-token request, all zeros
                 o_md = has_lanes ? got_md : 0x80000000u;
                 o_stall = has_lanes ? got_stall : 0u;
@@ -286,13 +285,16 @@ k_playout_fast(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst
 
 cudaError_t launch_playout_fast(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const int32_t* knots,
                                 uint64_t seed, TimelineRec rec, uint32_t* todo, uint32_t* todo_count,
-                                bool never_clamps, cudaStream_t st) {
+                                bool never_clamps, bool long_outputs, cudaStream_t st) {
     if (tr.n == 0) return cudaSuccess;
     // requests per ticket: small batches spread the end of the launch evenly; large traces amortise the ticket
-    int rpw = kPerIter;
+    int rpw = 8;
     while (rpw < 32 && (uint64_t)tr.n / (2 * rpw) >= 148u * 48u * 4u) rpw *= 2;
     const uint32_t per_block = kFastWarps * (uint32_t)rpw;
-    auto* kernel = never_clamps ? k_playout_fast<true> : k_playout_fast<false>;
+    // requests per round: eight halve the cost of a round per request; with long outputs the token loop is
+    // what counts, and four requests split the lanes more evenly
+    auto* kernel = never_clamps ? (long_outputs ? k_playout_fast<true, 4> : k_playout_fast<true, 8>)
+                                : (long_outputs ? k_playout_fast<false, 4> : k_playout_fast<false, 8>);
     // as many blocks as the GPU holds at once (at most six of these per SM); the ticket counter feeds them
     const uint32_t blocks = std::min<uint32_t>((tr.n + per_block - 1) / per_block, 148u * 6u);
     kernel<<<blocks, kFastWarps * 32, 0, st>>>(tr, gc, cc, knots, seed_key(seed), rec, todo, todo_count, todo_count + 1, rpw);
