@@ -65,7 +65,7 @@ template <bool LEAN, int PER>
 __global__ void __launch_bounds__(kFastWarps * 32)
 k_playout_fast(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __restrict__ ccp,
                const int32_t* __restrict__ knots, uint32_t k0, TimelineRec rec, uint32_t* __restrict__ todo,
-               uint32_t* __restrict__ todo_count, uint32_t* __restrict__ tickets, int rpw) {
+               uint32_t* __restrict__ todo_count, uint32_t* __restrict__ tickets, int rpw, uint32_t one) {
     const int lane = threadIdx.x & 31;
     const ClassConst& cc = *ccp;
     const int32_t tau = cc.tau;                                   // pacing is on for every launch of this kernel
@@ -158,7 +158,7 @@ k_playout_fast(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst
                 for (int t = 0; t < Lmax; ++t) {
                     const uint32_t x = __umulhi(mix32(hin), mul);
                     hin += kHashTok;
-                    if (t < cnt) hC += x;
+                    if (t < cnt) hC = x * one + hC;        // `one` = 1: a multiply-add, off the busy integer pipe
                 }
                 s_S = s_D = cnt * (G.cand == 2 ? G.cD_base : G.cS_base) - (int32_t)hC;
             } else {
@@ -297,7 +297,7 @@ cudaError_t launch_playout_fast(const TraceDev& tr, const GroupConst* gc, const 
                                 : (long_outputs ? k_playout_fast<false, 4> : k_playout_fast<false, 8>);
     // as many blocks as the GPU holds at once (at most six of these per SM); the ticket counter feeds them
     const uint32_t blocks = std::min<uint32_t>((tr.n + per_block - 1) / per_block, 148u * 6u);
-    kernel<<<blocks, kFastWarps * 32, 0, st>>>(tr, gc, cc, knots, seed_key(seed), rec, todo, todo_count, todo_count + 1, rpw);
+    kernel<<<blocks, kFastWarps * 32, 0, st>>>(tr, gc, cc, knots, seed_key(seed), rec, todo, todo_count, todo_count + 1, rpw, 1u);
     return cudaGetLastError();
 }
 
