@@ -49,7 +49,7 @@ PAIR_INSTR_WAIT = 41
 SM_COUNT, SCHEDULERS, LANES = 148, 4, 32
 # DRAM bytes per launch from the committed ncu capture of the dominant kernel (None until captured for
 # the current kernel; see profiles/).
-NCU_TRAFFIC_BYTES = {"k_pairs_rows": 145562368, "k_pairs_acc": None, "k_playout_fast": 823040, "k_playout": None}
+NCU_TRAFFIC_BYTES = {"k_pairs_rows": 144974592, "k_pairs_acc": None, "k_playout_fast": 827648, "k_playout": None}
 
 
 def env_rank():

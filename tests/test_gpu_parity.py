@@ -71,6 +71,26 @@ def test_generation_slower_than_consumption():
     full_parity(w, pols, tag="slow-gen")
 
 
+def test_long_outputs_with_and_without_clamping():
+    # mean output above 512 tokens (four requests per warp round); r_c = 5 never clamps, r_c = 30 does for the
+    # phone-class device (10 tok/s), so both forms of the clamp-free kernel and its to-do list run
+    w = synth.make_workload(3, n=1200, n_budgets=3)
+    assert w.output_len.mean() >= 512
+    pols = [synth.policy(b, r_c=rc, t_m_s=tm) for b in (0.3, 1.0) for rc, tm in ((5.0, 1.0), (30.0, 0.3), (5.0, 4.0))]
+    full_parity(w, pols, tag="long-outputs")
+
+
+def test_consumption_interval_equal_to_slowest_token():
+    # tau = T + J exactly for the device (100,000 + 5,000 ticks): intervals of zero slack, never negative
+    w = synth.make_workload(3, n=900, n_budgets=2)
+    pols = [synth.policy(b, r_c=1e6 / 105000.0, t_m_s=tm) for b in (0.5, 1.0) for tm in (0.5, 2.0)]
+    gs, _ = full_parity(w, pols, tag="tau-equals-slowest")
+    tr = Trace.from_workload(w)
+    tr.eval_policies(pols, w.seed)
+    assert tr.prep(0, 0).tau == 105000
+    tr.close()
+
+
 def test_stochastic_baselines_and_expected_length():
     # Stoch-S / Stoch-D routing and the expected-length trigger, mixed with ordinary policies in one call
     STOCH = synth.FLAG_STOCHASTIC
