@@ -121,6 +121,24 @@ inline int host_bin_of_ticks(int64_t t) {
     return (int)(b < kNBins - 1 ? b : kNBins - 1);
 }
 
+#ifdef __CUDACC__
+// Launch that lets the grid be scheduled while its predecessor in the stream is still draining (programmatic
+// stream serialisation).  Every kernel launched this way calls grid_dependency_wait() before it reads or
+// writes global memory; the wait returns once the preceding grids have completed and their writes are visible.
+template <class... KArgs, class... Args>
+inline cudaError_t launch_after(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+#endif
+
 // Records the calling thread's error message (read back by disco_last_error) and returns `code`.
 int set_error(int code, const char* msg);
 

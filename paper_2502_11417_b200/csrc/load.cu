@@ -96,6 +96,7 @@ __global__ void k_radix_hist(const uint64_t* __restrict__ keys, uint32_t n, uint
 __global__ void k_radix_rowscan(uint32_t* __restrict__ counts /* [256][blocks] */, uint32_t blocks,
                                 uint32_t* __restrict__ totals /* [256] */) {
     __shared__ uint32_t part[128];
+    grid_dependency_wait();
     uint32_t* row = counts + (size_t)blockIdx.x * blocks;
     const uint32_t per = (blocks + 127u) / 128u;
     const uint32_t lo = min(blocks, threadIdx.x * per), hi = min(blocks, lo + per);
@@ -122,6 +123,7 @@ __global__ void k_radix_scatter(const uint64_t* __restrict__ keys_in, uint64_t* 
     __shared__ uint32_t run[256];                 // next output slot of each digit for this block
     __shared__ uint32_t wcnt[kRadixWarps][256];   // keys of each digit per warp in the current slab
     const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    grid_dependency_wait();
     {
         // offsets[d][b]: keys of digit d in earlier blocks (k_radix_rowscan); totals[d]: keys of digit d.
         // This block's first slot for digit d = keys of smaller digits + keys of d in earlier blocks.
@@ -226,6 +228,7 @@ __global__ void k_group_mass(const uint32_t* __restrict__ cnt, int64_t* __restri
     __shared__ unsigned long long pm[NT];
     __shared__ uint32_t pc[NT];
     const int g = blockIdx.x;
+    grid_dependency_wait();
     const uint32_t* c = cnt + (size_t)g * L;
     int64_t* out = cum + (size_t)g * (L + 1);
     const int per = (L + NT - 1) / NT;                 // 5
@@ -254,6 +257,7 @@ __global__ void k_group_knots(int G, const uint32_t* __restrict__ ng, const int3
                               const unsigned long long* __restrict__ grp_sum_n, LoadReadback* __restrict__ rb) {
     __shared__ uint32_t off[kMaxGroups + 1];
     const int g = blockIdx.x;
+    grid_dependency_wait();
     if (threadIdx.x == 0) {
         uint32_t r = 0;
         for (int k = 0; k < G; ++k) { off[k] = r; r += ng[k]; }
@@ -338,10 +342,10 @@ cudaError_t run_load(const LoadArgs& a, cudaStream_t st) {
             for (int p = 0; p < passes; ++p) {                  // the scatter also counts the next digit
                 const bool last = p == passes - 1;
                 uint32_t* cur = a.radix_counts + (size_t)p * 256u * blocks;
-                k_radix_rowscan<<<256, 128, 0, st>>>(cur, blocks, totals);
-                k_radix_scatter<<<blocks, kRadixThreads, 0, st>>>(src, dst, nullptr, nullptr, n, per_block, 8 * p, cur,
-                                                                  totals, last ? nullptr : cur + 256u * blocks,
-                                                                  last ? a.sorted : nullptr);
+                if ((e = launch_after(k_radix_rowscan, 256, 128, 0, st, cur, blocks, totals))) return e;
+                if ((e = launch_after(k_radix_scatter, blocks, kRadixThreads, 0, st, src, dst, nullptr, nullptr, n, per_block,
+                                      8 * p, cur, totals, last ? nullptr : cur + 256u * blocks,
+                                      last ? a.sorted : nullptr))) return e;
                 uint64_t* t = src; src = dst; dst = t;
             }
         } else {
@@ -352,9 +356,9 @@ cudaError_t run_load(const LoadArgs& a, cudaStream_t st) {
             k_low_words<<<grid_for(n, 256), 256, 0, st>>>(n, src, a.sorted);
         }
     }
-    k_group_mass<<<G, 1024, 0, st>>>(a.cnt, a.cum_mass, a.ng_exact);
-    k_group_knots<<<G, 256, 0, st>>>(G, a.ng, a.sorted, a.grp_off, a.knots, a.err, a.max_n,
-                                     (const unsigned long long*)a.grp_sum_n, a.readback);
+    if ((e = launch_after(k_group_mass, G, 1024, 0, st, a.cnt, a.cum_mass, a.ng_exact))) return e;
+    if ((e = launch_after(k_group_knots, G, 256, 0, st, G, a.ng, a.sorted, a.grp_off, a.knots, a.err, a.max_n,
+                          (const unsigned long long*)a.grp_sum_n, a.readback))) return e;
     return cudaGetLastError();
 }
 
