@@ -108,6 +108,7 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
     uint32_t* h_ttft = smem;                                  // [PL][kHWords]
     uint32_t* h_stall = smem + PL * kHWords;                  // [PL][kHWords]
     unsigned long long* s_acc = (unsigned long long*)(smem + 2 * PL * kHWords);   // [PL][kNAcc]; 866 words per policy keep it 8-byte aligned
+    grid_dependency_wait();
 
     const Chunk ch = chunks[blockIdx.x];
     const int g = ch.g;
@@ -402,6 +403,7 @@ k_pairs_rows(TraceDev tr, const GroupConst* __restrict__ gcs, const Prep* __rest
     __shared__ Prep s_prep[EXT ? kRowPols : 1];
     __shared__ RowPol s_rp[kRowPols];
     __shared__ uint4 s_rows[kRowThreads * kRowVec];
+    grid_dependency_wait();
     const uint32_t first = blockIdx.y * kRowPols;
     const int npol = (int)min((uint32_t)kRowPols, n_list - first);
     // the block's requests are consecutive in the internal order; most blocks lie inside one group
@@ -515,11 +517,10 @@ cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassCo
                                          (int)acc_smem_bytes(32));
     if (e) return e;
     dim3 grid(n_chunks, (n_list + PL - 1) / PL);
-    acc_kernel<<<grid, kAccThreads, acc_smem_bytes(PL), st>>>(tr, gc, cc, prep, P, pol_list, n_list, PL, chunks, rec, k0,
-                                                               (unsigned long long*)acc,
-                                                               (unsigned long long*)hist_ttft,
-                                                               (unsigned long long*)hist_tbt);
-    if ((e = cudaGetLastError())) return e;
+    if ((e = launch_after(acc_kernel, grid, kAccThreads, acc_smem_bytes(PL), st, tr, gc, cc, prep, P, pol_list, n_list, PL,
+                          chunks, rec, k0, (unsigned long long*)acc, (unsigned long long*)hist_ttft,
+                          (unsigned long long*)hist_tbt)))
+        return e;
     if (mid && (e = cudaEventRecord(mid, st))) return e;
     const bool rows = out.ttft_s || out.tbt_mean_s || out.tbt_max_s || out.cost || out.tok_server || out.tok_device ||
                       out.mig_at || out.delayed || out.decision;
@@ -528,8 +529,7 @@ cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassCo
         auto* row_kernel = extras ? (idx32 ? k_pairs_rows<true, true> : k_pairs_rows<true, false>)
                                   : (idx32 ? k_pairs_rows<false, true> : k_pairs_rows<false, false>);
         dim3 grid_r((tr.n + kRowThreads - 1) / kRowThreads, (n_list + kRowPols - 1) / kRowPols);
-        row_kernel<<<grid_r, kRowThreads, 0, st>>>(tr, gc, prep, P, pol_list, n_list, rec, k0, out);
-        e = cudaGetLastError();
+        e = launch_after(row_kernel, grid_r, kRowThreads, 0, st, tr, gc, prep, P, pol_list, n_list, rec, k0, out);
     }
     return e;
 }

@@ -290,6 +290,7 @@ k_playout(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __r
     __shared__ uint32_t ring_s[kWarps][kRing];
     __shared__ XResult xres_s[kWarps];
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    grid_dependency_wait();
     const uint32_t count = todo_count ? *todo_count : count_imm;
     for (uint32_t batch0 = (blockIdx.x * kWarps + wib) * 32u; batch0 < count; batch0 += gridDim.x * kWarps * 32u) {
     uint32_t* ring = ring_s[wib];
@@ -521,16 +522,16 @@ cudaError_t launch_timeline(const TraceDev& tr, const GroupConst* gc, const Clas
     if (!pacing) {
         if (mid) { cudaError_t e0 = cudaEventRecord(mid, st); if (e0) return e0; }
         const uint32_t blocks = std::min<uint32_t>((tr.n + per_block - 1) / per_block, 148u * 16u);
-        k_playout<<<blocks, kWarps * 32, 0, st>>>(tr, gc, cc, knots, seed_key(seed), rec, err, nullptr, nullptr, tr.n);
-        return cudaGetLastError();
+        return launch_after(k_playout, blocks, kWarps * 32, 0, st, tr, gc, cc, knots, seed_key(seed), rec, err, nullptr,
+                            nullptr, tr.n);
     }
     cudaError_t e = launch_playout_fast(tr, gc, cc, knots, seed, rec, todo, todo_count, never_clamps, long_outputs, st);
     if (e) return e;
     if (mid && (e = cudaEventRecord(mid, st))) return e;
     if (never_clamps) return cudaSuccess;             // no interval can exceed tau: the list stays empty
     const uint32_t blocks = std::min<uint32_t>((tr.n + per_block - 1) / per_block, 148u * 2u);
-    k_playout<<<blocks, kWarps * 32, 0, st>>>(tr, gc, cc, knots, seed_key(seed), rec, err, todo, todo_count, 0u);
-    return cudaGetLastError();
+    return launch_after(k_playout, blocks, kWarps * 32, 0, st, tr, gc, cc, knots, seed_key(seed), rec, err, todo, todo_count,
+                        0u);
 }
 
 }  // namespace disco

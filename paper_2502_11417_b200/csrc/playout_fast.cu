@@ -67,6 +67,7 @@ k_playout_fast(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst
                const int32_t* __restrict__ knots, uint32_t k0, TimelineRec rec, uint32_t* __restrict__ todo,
                uint32_t* __restrict__ todo_count, uint32_t* __restrict__ tickets, int rpw, uint32_t one) {
     const int lane = threadIdx.x & 31;
+    grid_dependency_wait();
     const ClassConst& cc = *ccp;
     const int32_t tau = cc.tau;                                   // pacing is on for every launch of this kernel
     const uint32_t B = (uint32_t)cc.B;
@@ -297,8 +298,8 @@ cudaError_t launch_playout_fast(const TraceDev& tr, const GroupConst* gc, const 
                                 : (long_outputs ? k_playout_fast<false, 4> : k_playout_fast<false, 8>);
     // as many blocks as the GPU holds at once (at most six of these per SM); the ticket counter feeds them
     const uint32_t blocks = std::min<uint32_t>((tr.n + per_block - 1) / per_block, 148u * 6u);
-    kernel<<<blocks, kFastWarps * 32, 0, st>>>(tr, gc, cc, knots, seed_key(seed), rec, todo, todo_count, todo_count + 1, rpw, 1u);
-    return cudaGetLastError();
+    return launch_after(kernel, blocks, kFastWarps * 32, 0, st, tr, gc, cc, knots, seed_key(seed), rec, todo, todo_count,
+                        todo_count + 1, rpw, 1u);
 }
 
 }  // namespace disco

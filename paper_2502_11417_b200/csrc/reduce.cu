@@ -56,6 +56,7 @@ __global__ void k_finalize(uint32_t P, int G, const GroupConst* __restrict__ gc,
                            const unsigned long long* __restrict__ grp_sum_n, const uint32_t* __restrict__ grp_off,
                            disco_policy_stats_t* __restrict__ stats, const int32_t* __restrict__ err) {
     const uint32_t p = blockIdx.x;
+    grid_dependency_wait();
     if (p == 0 && threadIdx.x < 4) ((int32_t*)(stats + P))[threadIdx.x] = err[threadIdx.x];   // error word rides along
     __shared__ unsigned long long tot[kNAcc];
     __shared__ int qb[4];
@@ -153,10 +154,9 @@ __global__ void k_select(const disco_policy_stats_t* __restrict__ stats, uint32_
 cudaError_t launch_finalize(uint32_t P, int G, const GroupConst* gc, const uint64_t* acc, const uint64_t* hist_ttft,
                             const uint64_t* hist_tbt, const uint64_t* grp_sum_n, const uint32_t* grp_off,
                             disco_policy_stats_t* stats, const int32_t* err, cudaStream_t st) {
-    k_finalize<<<P, 32, 0, st>>>(P, G, gc, (const unsigned long long*)acc, (const unsigned long long*)hist_ttft,
-                                 (const unsigned long long*)hist_tbt, (const unsigned long long*)grp_sum_n, grp_off,
-                                 stats, err);
-    return cudaGetLastError();
+    return launch_after(k_finalize, P, 32, 0, st, P, G, gc, (const unsigned long long*)acc,
+                        (const unsigned long long*)hist_ttft, (const unsigned long long*)hist_tbt,
+                        (const unsigned long long*)grp_sum_n, grp_off, stats, err);
 }
 
 cudaError_t launch_select(const disco_policy_stats_t* stats, uint32_t P, double cost_cap, float tbt_slo_s,
