@@ -215,7 +215,7 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     from paper_2502_11417_b200 import synth, Trace
-    from paper_2502_11417_b200.api import policy_array, kernel_launch_count, PolicyStats
+    from paper_2502_11417_b200.api import policy_array, kernel_launch_count, PolicyStats, stats_view
     import ctypes
 
     w = synth.make_workload(args.config, n=args.requests, n_budgets=args.budgets, replica=rank)
@@ -239,11 +239,11 @@ def run_ours(args):
     cap_factor, slo = w.select["cost_cap_factor"], w.select["tbt_slo_s"]
 
     def step(arrays):
-        tr.load_trace(*arrays, w.servers, w.devices)
-        tr.eval_policies(pols, w.seed, out)
-        st = tr.reduce_stats()
-        cap = cap_factor * min(st[p].total_cost for p in range(P))
-        return tr.select_policy(cap, slo)
+        tr.load_trace(*arrays, w.servers, w.devices, stream=stream)
+        tr.eval_policies(pols, w.seed, out, stream=stream)
+        st = tr.reduce_stats(stream=stream)
+        cap = cap_factor * float(stats_view(st)["total_cost"].min())
+        return tr.select_policy(cap, slo, stream=stream)
 
     def timed(arrays, steps, warmup, collect=None):
         for _ in range(warmup):

@@ -127,9 +127,28 @@ def _check(rc: int, allow=()):
 
 
 def _stream_ptr(stream) -> Optional[int]:
-    import torch
-    s = torch.cuda.current_stream() if stream is None else stream
-    return C.c_void_p(s.cuda_stream)
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+_cuda_ok = None
+
+
+def _require_cuda():
+    global _cuda_ok
+    if _cuda_ok is None:
+        import torch
+        _cuda_ok = bool(torch.cuda.is_available())
+    if not _cuda_ok:
+        raise DiscoError(ECUDA, "no CUDA device: libdisco has no CPU path")
+
+
+def stats_view(stats):
+    """The (PolicyStats * P) array returned by reduce_stats as a numpy structured array (no copy), for
+    column-wise reads such as stats_view(st)["total_cost"].min()."""
+    return np.frombuffer(stats, dtype=np.dtype(PolicyStats))
 
 
 def _torch_dtype(name):
@@ -196,8 +215,7 @@ class Trace:
         """Arrays may be numpy arrays / pinned CPU tensors (host memory) or CUDA tensors (device memory),
         all of the same kind.  Reloading reuses the context's device memory."""
         import torch
-        if not torch.cuda.is_available():
-            raise DiscoError(ECUDA, "no CUDA device: libdisco has no CPU path")
+        _require_cuda()
         arrs = [prompt_len, output_len, server_ttft_s, server_profile, device_profile]
         on_dev = isinstance(prompt_len, torch.Tensor) and prompt_len.is_cuda
         want = [("int32", np.int32), ("int32", np.int32), ("float32", np.float32), ("uint8", np.uint8),
