@@ -145,10 +145,16 @@ def _require_cuda():
         raise DiscoError(ECUDA, "no CUDA device: libdisco has no CPU path")
 
 
+_stats_dtype = None
+
+
 def stats_view(stats):
     """The (PolicyStats * P) array returned by reduce_stats as a numpy structured array (no copy), for
     column-wise reads such as stats_view(st)["total_cost"].min()."""
-    return np.frombuffer(stats, dtype=np.dtype(PolicyStats))
+    global _stats_dtype
+    if _stats_dtype is None:
+        _stats_dtype = np.dtype(PolicyStats)
+    return np.frombuffer(stats, dtype=_stats_dtype)
 
 
 def _torch_dtype(name):

@@ -60,6 +60,8 @@ struct disco_ctx {
     int G = 0;
     bool loaded = false;
     std::vector<GroupConst> gc;
+    std::vector<GroupConst> gc_dev;   // what d_gc holds (a reload with the same profiles skips the copy)
+    const void* gc_dev_at = nullptr;
     // trace
     DevBuf in_prompt, in_out, in_ttft, in_sp, in_dp;      // staging of host inputs
     DevBuf keys_a, keys_b, tmp_idx;
@@ -236,8 +238,13 @@ int disco_load_trace(disco_ctx_t** pctx, const disco_trace_desc_t* d, void* stre
     a.ng = c->ng; a.grp_off = c->grp_off.as<uint32_t>(); a.knots = c->knots.as<int32_t>();
     a.grp_sum_n = c->grp_sum_n; a.max_n = c->max_n; a.err = c->err;
     // the profile table is read from pageable memory: this copy returns once it has been staged
-    if ((e = cudaMemcpyAsync(c->d_gc.p, c->gc.data(), c->gc.size() * sizeof(GroupConst), cudaMemcpyHostToDevice, st)) != cudaSuccess)
-        return bail(fail_cuda(e, "profile copy"));
+    const bool same_profiles = c->gc_dev_at == c->d_gc.p && c->gc_dev.size() == c->gc.size() &&
+                               std::memcmp(c->gc_dev.data(), c->gc.data(), c->gc.size() * sizeof(GroupConst)) == 0;
+    if (!same_profiles) {
+        c->gc_dev_at = nullptr;
+        if ((e = cudaMemcpyAsync(c->d_gc.p, c->gc.data(), c->gc.size() * sizeof(GroupConst), cudaMemcpyHostToDevice, st)) != cudaSuccess)
+            return bail(fail_cuda(e, "profile copy"));
+    }
     if ((e = run_load(a, st)) != cudaSuccess) return bail(fail_cuda(e, "trace ingestion kernels"));
     g_launches += load_kernel_launches(n, c->G);
     // read back the few numbers the host needs: error word, group sizes, longest output, largest TTFT per group
@@ -245,6 +252,7 @@ int disco_load_trace(disco_ctx_t** pctx, const disco_trace_desc_t* d, void* stre
     if ((e = cudaMemcpyAsync(rb, c->d_rb.p, sizeof(LoadReadback), cudaMemcpyDeviceToHost, st)) != cudaSuccess)
         return bail(fail_cuda(e, "readback"));
     if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return bail(fail_cuda(e, "trace ingestion"));
+    if (!same_profiles) { c->gc_dev = c->gc; c->gc_dev_at = c->d_gc.p; }      // the copy has landed
     if (rb->err[0]) {
         static const char* what[] = {"", "prompt length outside 1..4096", "output length outside 1..8192",
                                      "server TTFT not finite, not positive or above 2000 s", "profile id out of range"};

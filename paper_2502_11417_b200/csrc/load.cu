@@ -222,13 +222,13 @@ __global__ void k_low_words(uint32_t n, const uint64_t* __restrict__ keys, int32
         out[k] = (int32_t)(uint32_t)keys[k];
 }
 
-// One block per group: cumulative input-token mass cum[L] = sum_{l<L} l*cnt[l], L = 0..4097, and N_g.
-__global__ void k_group_mass(const uint32_t* __restrict__ cnt, int64_t* __restrict__ cum, uint32_t* __restrict__ ng) {
+// One block of 1024 threads per group: cumulative input-token mass cum[L] = sum_{l<L} l*cnt[l], L = 0..4097, and N_g.
+__device__ __forceinline__ void group_mass(const uint32_t* __restrict__ cnt, int64_t* __restrict__ cum,
+                                           uint32_t* __restrict__ ng) {
     constexpr int NT = 1024, L = kMaxPrompt + 1;      // 4097 lengths
     __shared__ unsigned long long pm[NT];
     __shared__ uint32_t pc[NT];
     const int g = blockIdx.x;
-    grid_dependency_wait();
     const uint32_t* c = cnt + (size_t)g * L;
     int64_t* out = cum + (size_t)g * (L + 1);
     const int per = (L + NT - 1) / NT;                 // 5
@@ -250,14 +250,14 @@ __global__ void k_group_mass(const uint32_t* __restrict__ cnt, int64_t* __restri
 }
 
 // Group offsets in the partitioned order, the 257 knots K_g[k] = sorted_g[(k (N_g - 1)) / 256] and the few
-// numbers the host reads back.  One block per group (after k_group_mass has produced the group sizes).
-__global__ void k_group_knots(int G, const uint32_t* __restrict__ ng, const int32_t* __restrict__ sorted,
-                              uint32_t* __restrict__ grp_off, int32_t* __restrict__ knots,
-                              const int32_t* __restrict__ err, const uint32_t* __restrict__ max_n,
-                              const unsigned long long* __restrict__ grp_sum_n, LoadReadback* __restrict__ rb) {
+// numbers the host reads back.  One block per group (ng: the group sizes counted at ingestion).
+__device__ __forceinline__ void group_knots(int G, const uint32_t* __restrict__ ng, const int32_t* __restrict__ sorted,
+                                            uint32_t* __restrict__ grp_off, int32_t* __restrict__ knots,
+                                            const int32_t* __restrict__ err, const uint32_t* __restrict__ max_n,
+                                            const unsigned long long* __restrict__ grp_sum_n,
+                                            LoadReadback* __restrict__ rb) {
     __shared__ uint32_t off[kMaxGroups + 1];
     const int g = blockIdx.x;
-    grid_dependency_wait();
     if (threadIdx.x == 0) {
         uint32_t r = 0;
         for (int k = 0; k < G; ++k) { off[k] = r; r += ng[k]; }
@@ -276,6 +276,17 @@ __global__ void k_group_knots(int G, const uint32_t* __restrict__ ng, const int3
             rb->max_n = *max_n;
         }
     }
+}
+
+// The group tables in one launch: one block of 1024 threads per group.
+__global__ void __launch_bounds__(1024)
+k_group_tables(int G, const uint32_t* __restrict__ cnt, int64_t* __restrict__ cum, uint32_t* __restrict__ ng_exact,
+               const uint32_t* __restrict__ ng, const int32_t* __restrict__ sorted, uint32_t* __restrict__ grp_off,
+               int32_t* __restrict__ knots, const int32_t* __restrict__ err, const uint32_t* __restrict__ max_n,
+               const unsigned long long* __restrict__ grp_sum_n, LoadReadback* __restrict__ rb) {
+    grid_dependency_wait();
+    group_knots(G, ng, sorted, grp_off, knots, err, max_n, grp_sum_n, rb);
+    group_mass(cnt, cum, ng_exact);
 }
 
 int grid_for(uint32_t n, int threads) {
@@ -302,10 +313,10 @@ cudaError_t radix_pass(const uint64_t* kin, uint64_t* kout, const uint32_t* pin,
 }  // namespace
 
 uint32_t load_kernel_launches(uint32_t n, int G) {
-    if (n == 0) return 2;
-    if (G == 1 && n <= (1u << 20)) return 1 + 2 * 4 + 2;     // ingest, (row scan, scatter) x 4, group tables
+    if (n == 0) return 1;
+    if (G == 1 && n <= (1u << 20)) return 1 + 2 * 4 + 1;     // ingest, (row scan, scatter) x 4, group tables
     const uint32_t passes = G > 1 ? 6 : 4;                  // radix passes: partition + 5, or 4
-    return 1 + (G > 1 ? 1 : 0) + 3 * passes + 1 + 2;         // ingest, gather, passes, low words, group tables
+    return 1 + (G > 1 ? 1 : 0) + 3 * passes + 1 + 1;         // ingest, gather, passes, low words, group tables
 }
 
 cudaError_t run_load(const LoadArgs& a, cudaStream_t st) {
@@ -356,9 +367,8 @@ cudaError_t run_load(const LoadArgs& a, cudaStream_t st) {
             k_low_words<<<grid_for(n, 256), 256, 0, st>>>(n, src, a.sorted);
         }
     }
-    if ((e = launch_after(k_group_mass, G, 1024, 0, st, a.cnt, a.cum_mass, a.ng_exact))) return e;
-    if ((e = launch_after(k_group_knots, G, 256, 0, st, G, a.ng, a.sorted, a.grp_off, a.knots, a.err, a.max_n,
-                          (const unsigned long long*)a.grp_sum_n, a.readback))) return e;
+    if ((e = launch_after(k_group_tables, G, 1024, 0, st, G, a.cnt, a.cum_mass, a.ng_exact, a.ng, a.sorted, a.grp_off,
+                          a.knots, a.err, a.max_n, (const unsigned long long*)a.grp_sum_n, a.readback))) return e;
     return cudaGetLastError();
 }
 
