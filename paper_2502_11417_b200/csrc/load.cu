@@ -84,6 +84,7 @@ __global__ void k_radix_hist(const uint64_t* __restrict__ keys, uint32_t n, uint
                              uint32_t* __restrict__ counts /* [256][gridDim.x] */) {
     __shared__ uint32_t h[256];
     h[threadIdx.x] = 0;
+    grid_dependency_wait();
     __syncthreads();
     const uint32_t lo = min(n, blockIdx.x * per_block), hi = min(n, lo + per_block);
     for (uint32_t i = lo + threadIdx.x; i < hi; i += kRadixThreads)
@@ -314,7 +315,7 @@ cudaError_t radix_pass(const uint64_t* kin, uint64_t* kout, const uint32_t* pin,
 
 uint32_t load_kernel_launches(uint32_t n, int G) {
     if (n == 0) return 1;
-    if (G == 1 && n <= (1u << 20)) return 1 + 2 * 4 + 1;     // ingest, (row scan, scatter) x 4, group tables
+    if (G == 1 && n <= (1u << 20)) return 1 + 2 * 4 + 2 + 1;  // ingest, (row scan, scatter) x 4, two histograms, group tables
     const uint32_t passes = G > 1 ? 6 : 4;                  // radix passes: partition + 5, or 4
     return 1 + (G > 1 ? 1 : 0) + 3 * passes + 1 + 1;         // ingest, gather, passes, low words, group tables
 }
@@ -332,7 +333,7 @@ cudaError_t run_load(const LoadArgs& a, cudaStream_t st) {
     const bool small = G == 1 && n <= (1u << 20);      // fused histograms pay off while launches dominate
     // everything that must start at zero lies in one block: cnt, grp_sum_n, grp_n, max_n, err, counts A
     // (zero_bytes covers the tables; the per-pass digit counters of the small path follow them)
-    if ((e = cudaMemsetAsync(a.zero_block, 0, a.zero_bytes + (small ? (size_t)5 * 256u * blocks * 4u : 0u), st))) return e;
+    if ((e = cudaMemsetAsync(a.zero_block, 0, a.zero_bytes + (small ? (size_t)2 * 256u * blocks * 4u : 0u), st))) return e;
     if (n) {
         uint32_t* counts_a = a.radix_counts;                                   // small path: pass p uses slice p
         uint32_t* counts_b = a.radix_counts + (size_t)4 * 256u * kRadixMaxBlocks;  // large path: one scanned buffer
@@ -350,12 +351,17 @@ cudaError_t run_load(const LoadArgs& a, cudaStream_t st) {
         const int passes = G > 1 ? 5 : 4;
         if (small) {
             uint32_t* totals = a.radix_counts + (size_t)5 * 256u * kRadixMaxBlocks;
-            for (int p = 0; p < passes; ++p) {                  // the scatter also counts the next digit
-                const bool last = p == passes - 1;
+            for (int p = 0; p < passes; ++p) {
+                // The first scatter also counts the second pass's digits (the low bytes of the ticks are spread
+                // evenly, so its adds meet little contention).  High bytes take few values: those passes count
+                // with the block-private histogram kernel instead.
+                const bool last = p == passes - 1, fused_next = p == 0;
                 uint32_t* cur = a.radix_counts + (size_t)p * 256u * blocks;
+                if (p >= 2 && (e = launch_after(k_radix_hist, blocks, kRadixThreads, 0, st, (const uint64_t*)src, n, per_block,
+                                                8 * p, cur))) return e;
                 if ((e = launch_after(k_radix_rowscan, 256, 128, 0, st, cur, blocks, totals))) return e;
                 if ((e = launch_after(k_radix_scatter, blocks, kRadixThreads, 0, st, src, dst, nullptr, nullptr, n, per_block,
-                                      8 * p, cur, totals, last ? nullptr : cur + 256u * blocks,
+                                      8 * p, cur, totals, fused_next ? cur + 256u * blocks : nullptr,
                                       last ? a.sorted : nullptr))) return e;
                 uint64_t* t = src; src = dst; dst = t;
             }
