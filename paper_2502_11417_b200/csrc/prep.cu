@@ -18,6 +18,32 @@ __device__ int32_t inverse_cdf(const int32_t* sorted, uint32_t N, double q) {
     return sorted[k];
 }
 
+// Smallest x in [lo, hi) with pred(x), or hi if there is none; pred is false up to some point and true from
+// there on.  Fifteen probes a round instead of one: the probes of a round are independent loads, so the search
+// over the 4098 cumulative masses takes four rounds of memory latency instead of thirteen.
+template <class F>
+__device__ __forceinline__ int first_true(int lo, int hi, F pred) {
+    while (hi - lo > 16) {
+        const int step = (hi - lo + 15) >> 4;
+        bool f[15];
+#pragma unroll
+        for (int k = 0; k < 15; ++k) { const int x = lo + (k + 1) * step; f[k] = x < hi ? pred(x) : true; }
+        int k0 = 15;                                                  // first probe that holds
+#pragma unroll
+        for (int k = 14; k >= 0; --k) if (f[k]) k0 = k;
+        const int nlo = k0 == 0 ? lo : lo + k0 * step + 1;            // the probe before it failed
+        const int nhi = k0 == 15 ? hi : min(hi, lo + (k0 + 1) * step);
+        lo = nlo; hi = nhi;
+    }
+    bool f[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) { const int x = lo + k; f[k] = x < hi ? pred(x) : true; }
+    int k0 = 16;
+#pragma unroll
+    for (int k = 15; k >= 0; --k) if (f[k]) k0 = k;
+    return min(lo + k0, hi);
+}
+
 __global__ void k_prep(const PolicyConst* __restrict__ pol, uint32_t P, int G, const GroupConst* __restrict__ gc,
                        const int64_t* __restrict__ cum_mass, const uint32_t* __restrict__ cnt,
                        const int32_t* __restrict__ sorted, const uint32_t* __restrict__ grp_off,
@@ -46,12 +72,7 @@ __global__ void k_prep(const PolicyConst* __restrict__ pol, uint32_t P, int G, c
     if (!r.device_constrained) {
         // Eq. 3: smallest L with device-only mass sum_{l<L} l cnt[l] >= (1-b) Total
         const double target = __dmul_rn(__dsub_rn(1.0, b), Total);
-        int lo = 0, hi = kMaxPrompt + 1;                              // answer in [0, 4097]
-        while (lo < hi) {
-            const int mid = (lo + hi) >> 1;
-            if ((double)cum[mid] >= target) hi = mid; else lo = mid + 1;
-        }
-        r.l_th = lo;
+        r.l_th = first_true(0, kMaxPrompt + 1, [&](int L) { return (double)cum[L] >= target; });   // in [0, 4097]
     } else {
         // Algorithm 2, phase 1: tail protection
         const double q_tail = __dsub_rn(1.0, fmin(alpha, b));
@@ -66,12 +87,9 @@ __global__ void k_prep(const PolicyConst* __restrict__ pol, uint32_t P, int G, c
         } else {
             // phase 2: A input tokens may start the device at once; shortest prompts first
             const double A = __dmul_rn(__ddiv_rn(__dsub_rn(b, alpha), __dsub_rn(1.0, alpha)), Total);
-            int lo = 0, hi = kMaxPrompt + 1;                          // first length whose cumulative mass exceeds A
-            while (lo < hi) {
-                const int mid = (lo + hi) >> 1;
-                if ((double)cum[mid + 1] > A) hi = mid; else lo = mid + 1;
-            }
-            r.l_star = lo;                                             // 4097 = every class is funded
+            // first length whose cumulative mass exceeds A; 4097 = every class is funded
+            const int lo = first_true(0, kMaxPrompt + 1, [&](int l) { return (double)cum[l + 1] > A; });
+            r.l_star = lo;
             if (lo <= kMaxPrompt) {
                 const double f = __ddiv_rn(__dsub_rn(A, (double)cum[lo]), __dmul_rn((double)lo, (double)c[lo]));
                 r.w_star = inverse_cdf(srt, N, __dmul_rn(__dsub_rn(1.0, alpha), __dsub_rn(1.0, f)));
