@@ -378,7 +378,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=1000)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--config", type=int, default=1, help="workload 0..5 (default: workload 1)")
     ap.add_argument("--requests", type=int, default=None, help="shrink the trace (profiling on a small case)")
     ap.add_argument("--budgets", type=int, default=None, help="shrink the budget axis (profiling on a small case)")

@@ -362,7 +362,7 @@ size_t acc_smem_bytes(int PL) {
 }
 
 // ------------------------------------------------------------------------------------------------------
-// Per-pair arrays: lane = request, up to 32 policies per block row.
+// Per-pair arrays: lane = request, up to 16 policies per block row.
 //
 // What a pair writes besides its TTFT depends on the request and on which of the six outcomes it ends in.
 // Each thread therefore prices its request once per outcome (Eq. 8, token split, TBT mean and maximum of
@@ -371,7 +371,7 @@ size_t acc_smem_bytes(int PL) {
 // policy row.
 // ------------------------------------------------------------------------------------------------------
 constexpr int kRowThreads = 256;
-constexpr int kRowPols = 32;
+constexpr int kRowPols = 16;
 constexpr int kRowVec = 7;              // uint4 per request: six outcome rows and one of padding (odd stride)
 
 // What the dispatch of one (group, policy) needs, with the mode tests folded into the thresholds: Algorithm 3
