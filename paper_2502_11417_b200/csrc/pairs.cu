@@ -326,8 +326,17 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
             else pairs_of(std::integral_constant<int, K_ANY>{}, std::false_type{}, rr, ok);
         }
     }
-    // ---- block totals, then one flush per block
-    if (act) {
+    // ---- block totals, then one flush per block.  With fewer than 32 policies in the tile several lanes of a warp
+    //      hold sums of the same policy: they are added up by shuffles first, so that one lane per policy and warp
+    //      touches the shared totals (with one policy, 512 threads would otherwise queue on ten addresses).
+    for (int off = 16; off >= PL; off >>= 1) {
+        a_td += __shfl_xor_sync(0xFFFFFFFFu, a_td, off); a_ps += __shfl_xor_sync(0xFFFFFFFFu, a_ps, off);
+        a_pd += __shfl_xor_sync(0xFFFFFFFFu, a_pd, off); a_dl += __shfl_xor_sync(0xFFFFFFFFu, a_dl, off);
+        a_tau += __shfl_xor_sync(0xFFFFFFFFu, a_tau, off);
+        cnt_a += __shfl_xor_sync(0xFFFFFFFFu, cnt_a, off); cnt_b += __shfl_xor_sync(0xFFFFFFFFu, cnt_b, off);
+        a_tt += __shfl_xor_sync(0xFFFFFFFFu, a_tt, off);
+    }
+    if (act && lane < PL) {
         unsigned long long* a = s_acc + pol_in_tile * kNAcc;
         atomicAdd(&a[A_DEVICE_ONLY], (unsigned long long)(cnt_a & 0xFFFFu)); atomicAdd(&a[A_RACE], (unsigned long long)(cnt_a >> 16));
         atomicAdd(&a[A_DEVICE_WON], (unsigned long long)(cnt_b & 0xFFFFu)); atomicAdd(&a[A_MIGR], (unsigned long long)(cnt_b >> 16));
