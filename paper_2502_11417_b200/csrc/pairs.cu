@@ -337,12 +337,18 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
         a_tt += __shfl_xor_sync(0xFFFFFFFFu, a_tt, off);
     }
     if (act && lane < PL) {
-        unsigned long long* a = s_acc + pol_in_tile * kNAcc;
-        atomicAdd(&a[A_DEVICE_ONLY], (unsigned long long)(cnt_a & 0xFFFFu)); atomicAdd(&a[A_RACE], (unsigned long long)(cnt_a >> 16));
-        atomicAdd(&a[A_DEVICE_WON], (unsigned long long)(cnt_b & 0xFFFFu)); atomicAdd(&a[A_MIGR], (unsigned long long)(cnt_b >> 16));
-        atomicAdd(&a[A_TOK_DEVICE], (unsigned long long)a_td); atomicAdd(&a[A_PRE_SERVER], (unsigned long long)a_ps);
-        atomicAdd(&a[A_PRE_DEVICE], (unsigned long long)a_pd); atomicAdd(&a[A_DELAYED], (unsigned long long)a_dl);
-        atomicAdd(&a[A_TTFT_SUM], a_tt); atomicAdd(&a[A_TAU_CNT], (unsigned long long)a_tau);
+        // 32-bit adds on the low words (shared memory has no native 64-bit add): every total but the TTFT sum
+        // stays below 2^32 within a block (at most 65,280 requests of at most 12,288 tokens each); the TTFT
+        // sum carries into its high word
+        uint32_t* a = (uint32_t*)(s_acc + pol_in_tile * kNAcc);
+        atomicAdd(&a[2 * A_DEVICE_ONLY], cnt_a & 0xFFFFu); atomicAdd(&a[2 * A_RACE], cnt_a >> 16);
+        atomicAdd(&a[2 * A_DEVICE_WON], cnt_b & 0xFFFFu); atomicAdd(&a[2 * A_MIGR], cnt_b >> 16);
+        atomicAdd(&a[2 * A_TOK_DEVICE], a_td); atomicAdd(&a[2 * A_PRE_SERVER], a_ps);
+        atomicAdd(&a[2 * A_PRE_DEVICE], a_pd); atomicAdd(&a[2 * A_DELAYED], a_dl);
+        atomicAdd(&a[2 * A_TAU_CNT], a_tau);
+        const uint32_t lo = (uint32_t)a_tt, before = atomicAdd(&a[2 * A_TTFT_SUM], lo);
+        const uint32_t hi = (uint32_t)(a_tt >> 32) + (before + lo < before ? 1u : 0u);
+        if (hi) atomicAdd(&a[2 * A_TTFT_SUM + 1], hi);
     }
     __syncthreads();
     const int pols_here = (int)min((uint32_t)PL, n_list - blockIdx.y * PL);
