@@ -297,6 +297,7 @@ def run_ours(args):
     names = ["k_playout_fast", "k_playout", "k_pairs_acc", "k_pairs_rows"]
     kms = {nm: statistics.mean(t[i] for t in ktimes) for i, nm in enumerate(names)}
     token_steps = int((w.output_len - 1).sum())
+    n_classes = len({(float(np.float32(q["r_c"])), float(np.float32(q["t_m_s"])), int(q["flags"]) & 2) for q in w.policies})
     alu_peak = SM_COUNT * SCHEDULERS * LANES * sm_max_mhz * 1e6 / 1e12         # T lane-instructions/s
     alu_src = "148 SMs x 4 schedulers x 32 lanes x %.0f MHz (issue slots)" % sm_max_mhz
     per_token = PLAYOUT_INSTR_PER_TOKEN_LEAN if never_clamps(w) else PLAYOUT_INSTR_PER_TOKEN
@@ -359,6 +360,9 @@ def run_ours(args):
             "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
             "sim_tokens_per_s": toks * args.steps / (total_ms * 1e-3),
+            # token-steps actually played: one play-out per request and timeline class (policies that share the
+            # consumption rate, buffer size and pacing share it), whatever the number of policies
+            "useful_token_steps_per_s": token_steps * n_classes * world * args.steps / (total_ms * 1e-3),
             "config": {"workload": w.name, "requests_per_gpu": n, "policies": P, "pairs_per_step": pairs,
                        "per_pair_outputs": bool(w.materialise), "l2": "flushed between steps (512 MB write)",
                        "kernel_events": "every %d-th timed step (%d samples)" % (KERNEL_EVENT_STRIDE, len(ktimes)),

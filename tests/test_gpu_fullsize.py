@@ -66,3 +66,82 @@ def test_workload4_full_six_groups_policy_subset():
     w = synth.make_workload(4)
     pols = [w.policies[k] for k in (0, 37, 127, 128 + 64, 3 * 128 + 100, 7 * 128 + 127)]
     _check(w, pols, _sampled_ranges(w.n, 6, 40, 4), "workload4")
+
+
+# ---- the whole policy grid with reductions only: the launch configuration of workloads 2 and 4 ---------------
+
+def _oracle_stats_threaded(orc, policies, seed, threads=8):
+    """The oracle over disjoint request ranges on several host threads (its C library releases the GIL); the
+    integer accumulators and histograms merge exactly."""
+    from concurrent.futures import ThreadPoolExecutor
+    from oracle.binding import merge_stats
+    bounds = [orc.n * k // threads for k in range(threads + 1)]
+    with ThreadPoolExecutor(threads) as ex:
+        parts = list(ex.map(lambda k: orc.eval(policies, seed, bounds[k], bounds[k + 1], finish=False)[0],
+                            range(threads)))
+    tot = merge_stats(parts)
+    orc.finish(tot)
+    return tot
+
+
+@pytest.mark.parametrize("cfg,n", [(2, 6000), (4, 9000)])
+def test_whole_policy_grid_against_oracle_on_a_short_trace(cfg, n):
+    # all 1024 policies (32 full policy tiles), no per-pair arrays: every statistic and histogram, and the selection
+    from parity import check_stats
+    w = synth.make_workload(cfg, n=n)
+    assert len(w.policies) == 1024
+    tr = Trace.from_workload(w)
+    tr.eval_policies(w.policies, w.seed)
+    gs = tr.reduce_stats()
+    orc = Oracle.from_workload(w)
+    ostats = _oracle_stats_threaded(orc, w.policies, w.seed)
+    check_stats(gs, ostats, tr.histograms, f"grid-config{cfg}")
+    cheapest = min(s.total_cost for s in ostats)
+    for cap, slo in [(1.25 * cheapest, 0.25), (1.05 * cheapest, 0.25), (1e30, 1e-3)]:
+        assert tr.select_policy(cap, slo) == orc.select(ostats, cap, float(np.float32(slo))), (cfg, cap, slo)
+    tr.close()
+
+
+def _select_by_definition(st, cap, slo):
+    """Sec. 4.1's objective as this library reads it, written out on the host: feasible = cost within the cap and
+    P99 TBT within the objective; best = lowest P99 TTFT bin, then mean TTFT, cost, index; none feasible = cheapest."""
+    feas = [p for p in range(len(st)) if st[p].total_cost <= cap and st[p].p99_tbt_s <= np.float32(slo)]
+    if feas:
+        return 0, min(feas, key=lambda p: (st[p].bin_p99_ttft, st[p].mean_ttft_s, st[p].total_cost, p))
+    return -4, min(range(len(st)), key=lambda p: (st[p].total_cost, p))
+
+
+def test_workload2_full_size_whole_grid_properties():
+    w = synth.make_workload(2)
+    P, N, sum_n = len(w.policies), w.n, int(w.output_len.sum())
+    assert (N, P) == (1_000_000, 1024)
+    tr = Trace.from_workload(w)
+    tr.eval_policies(w.policies, w.seed)
+    st = tr.reduce_stats()
+    nb = 256
+    for p in range(P):
+        s = st[p]
+        assert s.n_requests == N and s.n_intervals == sum_n - N
+        assert s.n_server_only + s.n_device_only + s.n_race == N
+        assert s.tok_server + s.tok_device == sum_n
+        assert s.n_device_won <= s.n_device_started and s.n_migrations <= s.n_race
+    for p in range(0, P, 37):                                              # no histogram update was lost
+        th, bh = tr.histograms(p)
+        assert int(th.sum()) == N and int(bh.sum()) == sum_n - N
+    for t in range(4):                                                     # per threshold: budgets ascending
+        blk = [st[t * nb + k] for k in range(nb)]
+        dev_only = [s.n_device_only for s in blk]
+        assert all(b <= a for a, b in zip(dev_only, dev_only[1:])) and dev_only[0] == N and dev_only[-1] == 0
+        pre_srv = [s.prefill_tok_server for s in blk]
+        assert all(b >= a for a, b in zip(pre_srv, pre_srv[1:]))           # the server's input tokens grow with b
+        share = [s.prefill_tok_server / float(w.prompt_len.sum()) for s in blk]
+        budgets = [w.policies[t * nb + k]["budget"] for k in range(nb)]
+        assert all(sh <= b + 1e-12 for sh, b in zip(share, budgets))       # Eq. 3: the share stays within the budget
+    # a threshold of +inf never migrates; a lower threshold migrates at least as often
+    for k in range(nb):
+        migs = [st[t * nb + k].n_migrations for t in range(4)]
+        assert migs[3] == 0 and all(b <= a for a, b in zip(migs, migs[1:]))
+    cheapest = min(s.total_cost for s in st)
+    for cap, slo in [(1.25 * cheapest, 0.25), (1.02 * cheapest, 0.25), (0.5 * cheapest, 0.25), (1e30, 1e-3)]:
+        assert tr.select_policy(cap, slo) == _select_by_definition(st, cap, slo), (cap, slo)
+    tr.close()
