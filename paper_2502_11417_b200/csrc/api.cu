@@ -474,6 +474,7 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
                         c->d_pol_list.as<uint32_t>() + cls_range[k].first, cls_range[k].second - cls_range[k].first,
                         c->d_chunks.as<Chunk>(), (uint32_t)chunks.size(), rec, po, c->d_acc.as<uint64_t>(),
                         c->d_hist_ttft.as<uint64_t>(), c->d_hist_tbt.as<uint64_t>(), seed, cls_extras_pending,
+                        classes[k].W[0] > 1 || classes[k].W[1] > 1 || classes[k].W[2] > 1,
                         timed ? c->ev[3] : nullptr, st));
         if (timed) CU(cudaEventRecord(c->ev[4], st));
         g_launches += (n ? ((classes[k].pacing && !never_clamps) ? 2 : 1) : 0) + ((n && !chunks.empty()) ? (out ? 2 : 1) : 0);

@@ -159,7 +159,8 @@ cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassCo
                          const uint32_t* pol_list, uint32_t n_list, const Chunk* chunks, uint32_t n_chunks,
                          TimelineRec rec, disco_pair_out_t out, uint64_t* acc, uint64_t* hist_ttft,
                          uint64_t* hist_tbt, uint64_t seed, bool extras /* some policy routes at random or uses an
-                         expected length */, cudaEvent_t mid /* recorded between its two kernels, or null */,
+                         expected length */, bool wide /* some window W of the class spans several bins */,
+                         cudaEvent_t mid /* recorded between its two kernels, or null */,
                          cudaStream_t st);
 cudaError_t launch_finalize(uint32_t P, int G, const GroupConst* gc, const uint64_t* acc, const uint64_t* hist_ttft,
                             const uint64_t* hist_tbt, const uint64_t* grp_sum_n, const uint32_t* grp_off,

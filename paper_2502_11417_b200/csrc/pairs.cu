@@ -98,7 +98,9 @@ __device__ __forceinline__ void hist16_add_ticks(uint32_t* row, uint32_t t) {
 
 enum TileKind { K_NOWAIT = 0, K_WAIT = 1, K_ANY = 2 };
 
-template <bool EXT>
+// WIDE: some stream's regular TBTs span several histogram bins (pacing off, or generation slower than
+// consumption), so a pair also adds its stream's window of bins.
+template <bool EXT, bool WIDE>
 __global__ void __launch_bounds__(kAccThreads, 1)
 k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __restrict__ ccp,
             const Prep* __restrict__ prep, uint32_t P, const uint32_t* __restrict__ pol_list, uint32_t n_list,
@@ -125,7 +127,6 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
     const float delta_c = gc.delta_c;
     const int W0 = cc.W[0], W1 = cc.W[1], W2 = cc.W[2];
     const int kt0 = cc.ktau[g][0], kt1 = cc.ktau[g][1], kt2 = cc.ktau[g][2];
-    const bool wide = W0 > 1 || W1 > 1 || W2 > 1;             // some stream's regular TBTs span several bins
     const uint32_t tau = (uint32_t)cc.tau;
 
     for (int i = threadIdx.x; i < 2 * PL * kHWords + 2 * PL * kNAcc; i += kAccThreads) smem[i] = 0;   // (staging needs no clearing)
@@ -283,9 +284,18 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
                 a_tt += ttft[k];
                 if (EXT ? !waits : kNoWaits) hist16_apply(my_ttft, h2[k].w);
                 else hist16_add_ticks(my_ttft, ttft[k]);
-                if (h2[k].x & 0x10001u) hist16_apply(my_stall, h2[k].x);      // only a migrated pair's row carries one
             }
-            if (wide && act) {                                 // regular TBTs outside the bin of tau
+            // only the row of a pair whose hand-off stalled carries an increment for the stall histogram: one test
+            // for the four pairs, then each
+            uint32_t any_stall = 0;
+#pragma unroll
+            for (int k = 0; k < kIlp; ++k) any_stall |= (kAllOk || ok[k]) ? h2[k].x : 0u;
+            if (any_stall & 0x10001u) {
+#pragma unroll
+                for (int k = 0; k < kIlp; ++k)
+                    if ((kAllOk || ok[k]) && (h2[k].x & 0x10001u)) hist16_apply(my_stall, h2[k].x);
+            }
+            if (WIDE && act) {                                 // regular TBTs outside the bin of tau
                 for (int k = 0; k < kIlp; ++k) {
                     if (!kAllOk && !ok[k]) continue;
                     const int c = migr[k] ? 2 : (dev_wins[k] ? 1 : 0);
@@ -522,11 +532,12 @@ k_pairs_rows(TraceDev tr, const GroupConst* __restrict__ gcs, const Prep* __rest
 cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const Prep* prep, uint32_t P,
                          const uint32_t* pol_list, uint32_t n_list, const Chunk* chunks, uint32_t n_chunks,
                          TimelineRec rec, disco_pair_out_t out, uint64_t* acc, uint64_t* hist_ttft,
-                         uint64_t* hist_tbt, uint64_t seed, bool extras, cudaEvent_t mid, cudaStream_t st) {
+                         uint64_t* hist_tbt, uint64_t seed, bool extras, bool wide, cudaEvent_t mid, cudaStream_t st) {
     if (n_chunks == 0 || n_list == 0) return mid ? cudaEventRecord(mid, st) : cudaSuccess;
     int PL = 1;
     while (PL < 32 && (uint32_t)PL < n_list) PL <<= 1;
-    auto* acc_kernel = extras ? k_pairs_acc<true> : k_pairs_acc<false>;
+    auto* acc_kernel = extras ? (wide ? k_pairs_acc<true, true> : k_pairs_acc<true, false>)
+                              : (wide ? k_pairs_acc<false, true> : k_pairs_acc<false, false>);
     const uint32_t k0 = seed_key(seed);
     cudaError_t e = cudaFuncSetAttribute(acc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)acc_smem_bytes(32));
