@@ -39,13 +39,14 @@ PLAYOUT_INSTR_PER_TOKEN_LEAN = 13
 # Lane-instructions one (request, policy) pair needs in the reduction kernel, by the kind of policy.
 # Algorithm 3 (no waits; the race at w = 0 is staged once per request): request vector load 1, length
 # threshold 1, trigger compare and its conjunction 2, outcome index 2, TTFT select 1, row address 1, two row
-# loads 2, seven 32-bit sums and one 64-bit sum 9, staged histogram increment (two masks, address, atomic) 4,
-# stall increment (test, address, atomic) 3.
-PAIR_INSTR_NOWAIT = 27
+# loads 2, six 32-bit sums (tokens on device, two prefills, TBTs in tau's bin, delayed tokens, the four
+# byte-packed counts) and one 64-bit sum 8, staged histogram increment (address, atomic) 2, stall test shared
+# by four pairs 1.
+PAIR_INSTR_NOWAIT = 21
 # Algorithm 2 (waits): load 1, wait map 4, start compare 1, w + T_d 1, win compare 1, minimum 1, trigger 3,
-# outcome index 3, row address 1, two row loads 2, sums 9, histogram increment from the float bits (convert,
-# small-value test and branch, offset 2, increment 3, address, atomic) 10, stall increment 3.
-PAIR_INSTR_WAIT = 41
+# outcome index 3, row address 1, two row loads 2, sums 8, histogram increment from the float bits (convert,
+# small-value test and branch, offset 2, increment 3, address, atomic) 10, stall test 1.
+PAIR_INSTR_WAIT = 37
 SM_COUNT, SCHEDULERS, LANES = 148, 4, 32
 KERNEL_EVENT_STRIDE = 8      # per-kernel CUDA events are recorded on every 8th timed step
 # DRAM bytes per launch from the committed ncu capture of the dominant kernel (None until captured for

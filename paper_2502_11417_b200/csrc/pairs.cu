@@ -141,6 +141,7 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
 
     uint32_t a_td = 0, a_ps = 0, a_pd = 0, a_dl = 0, a_tau = 0;
     uint32_t cnt_a = 0, cnt_b = 0;                              // device-only | race << 16,  device won | migrated << 16
+    uint32_t cnt8 = 0;                                          // the same four counts, a byte each, within a batch
     unsigned long long a_tt = 0;
 
     // [warp][32 requests][kStageVec]: block A = the request, then the first half of each outcome's row;
@@ -204,13 +205,15 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
             a[1 + O_RACE_DEV] = make_uint4(n, l, l, nt1);
             a[1 + O_MIGR_TO_DEV] = make_uint4(n - m, l, l + lm, nt2);
             a[1 + O_MIGR_TO_SRV] = make_uint4(m, l + lm, l, nt2);
-            //                      delayed tokens << 17 | stall increment, counts, counts, TTFT increment
-            b[O_SERVER_ONLY] = make_uint4(0u, 0u, 0u, hS);
-            b[O_DEVICE_ONLY] = make_uint4(0u, 1u, 0u, hT);
-            b[O_RACE_SRV] = make_uint4(0u, 0x10000u, 0u, hS);
-            b[O_RACE_DEV] = make_uint4(0u, 0x10000u, 1u, hT);
-            b[O_MIGR_TO_DEV] = make_uint4(dly << 17 | stall_code, 0x10000u, 0x10000u, hS);
-            b[O_MIGR_TO_SRV] = make_uint4(dly << 17 | stall_code, 0x10000u, 0x10001u, hT);
+            //                      delayed tokens << 17 | stall increment, counts (a byte each: device only, race,
+            //                      device won, migrated), TTFT counter pair's byte offset, TTFT increment
+            const uint32_t oS = hS & 0xFFCu, iS = hS & 0x10001u, oT = hT & 0xFFCu, iT = hT & 0x10001u;
+            b[O_SERVER_ONLY] = make_uint4(0u, 0x00000000u, oS, iS);
+            b[O_DEVICE_ONLY] = make_uint4(0u, 0x00000001u, oT, iT);
+            b[O_RACE_SRV] = make_uint4(0u, 0x00000100u, oS, iS);
+            b[O_RACE_DEV] = make_uint4(0u, 0x00010100u, oT, iT);
+            b[O_MIGR_TO_DEV] = make_uint4(dly << 17 | stall_code, 0x01000100u, oS, iS);
+            b[O_MIGR_TO_SRV] = make_uint4(dly << 17 | stall_code, 0x01010100u, oT, iT);
             b[6] = make_uint4(0u, EXT ? routing_draw(k0, cur.orig) : 0u, m, n);
         }
         __syncwarp();
@@ -280,9 +283,9 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
             for (int k = 0; k < kIlp; ++k) {
                 if (!kAllOk && !ok[k]) continue;
                 a_td += h1[k].x; a_ps += h1[k].y; a_pd += h1[k].z; a_tau += h1[k].w;
-                a_dl += h2[k].x >> 17; cnt_a += h2[k].y; cnt_b += h2[k].z;
+                a_dl += h2[k].x >> 17; cnt8 += h2[k].y;
                 a_tt += ttft[k];
-                if (EXT ? !waits : kNoWaits) hist16_apply(my_ttft, h2[k].w);
+                if (EXT ? !waits : kNoWaits) atomicAdd((uint32_t*)((char*)my_ttft + h2[k].z), h2[k].w);
                 else hist16_add_ticks(my_ttft, ttft[k]);
             }
             // only the row of a pair whose hand-off stalled carries an increment for the stall histogram: one test
@@ -320,6 +323,7 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
                 else if (kind == K_WAIT) pairs_of(std::integral_constant<int, K_WAIT>{}, std::true_type{}, rr, ok);
                 else pairs_of(std::integral_constant<int, K_ANY>{}, std::true_type{}, rr, ok);
             }
+            cnt_a += __byte_perm(cnt8, 0u, 0x4140); cnt_b += __byte_perm(cnt8, 0u, 0x4342); cnt8 = 0;   // at most 32 a batch
             continue;
         }
         for (int r0 = 0; r0 < n_here; r0 += kIlp * slots) {
@@ -335,6 +339,7 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
             else if (kind == K_WAIT) pairs_of(std::integral_constant<int, K_WAIT>{}, std::false_type{}, rr, ok);
             else pairs_of(std::integral_constant<int, K_ANY>{}, std::false_type{}, rr, ok);
         }
+        cnt_a += __byte_perm(cnt8, 0u, 0x4140); cnt_b += __byte_perm(cnt8, 0u, 0x4342); cnt8 = 0;
     }
     // ---- block totals, then one flush per block.  With fewer than 32 policies in the tile several lanes of a warp
     //      hold sums of the same policy: they are added up by shuffles first, so that one lane per policy and warp
