@@ -232,7 +232,7 @@ int disco_load_trace(disco_ctx_t** pctx, const disco_trace_desc_t* d, void* stre
     }
     a.keys_a = c->keys_a.as<uint64_t>(); a.keys_b = c->keys_b.as<uint64_t>(); a.tmp_idx = c->tmp_idx.as<uint32_t>();
     a.radix_counts = c->radix_counts; a.zero_block = c->zero.p; a.zero_bytes = c->zero_bytes;
-    a.ng_exact = c->ng_exact.as<uint32_t>(); a.readback = c->d_rb.as<LoadReadback>();
+    a.ng_exact = c->ng_exact.as<uint32_t>(); a.readback = c->rb;     // pinned host memory, written by the last kernel
     a.S = c->S.as<int32_t>(); a.l = c->l.as<uint16_t>(); a.nout = c->nout.as<uint16_t>(); a.orig = c->orig.as<uint32_t>();
     a.sorted = c->sorted.as<int32_t>(); a.cnt = c->cnt; a.cum_mass = c->cum_mass.as<int64_t>();
     a.ng = c->ng; a.grp_off = c->grp_off.as<uint32_t>(); a.knots = c->knots.as<int32_t>();
@@ -247,10 +247,8 @@ int disco_load_trace(disco_ctx_t** pctx, const disco_trace_desc_t* d, void* stre
     }
     if ((e = run_load(a, st)) != cudaSuccess) return bail(fail_cuda(e, "trace ingestion kernels"));
     g_launches += load_kernel_launches(n, c->G);
-    // read back the few numbers the host needs: error word, group sizes, longest output, largest TTFT per group
+    // the few numbers the host needs (error word, group sizes, longest output, largest TTFT per group) are in rb
     HostReadback* rb = c->rb;
-    if ((e = cudaMemcpyAsync(rb, c->d_rb.p, sizeof(LoadReadback), cudaMemcpyDeviceToHost, st)) != cudaSuccess)
-        return bail(fail_cuda(e, "readback"));
     if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return bail(fail_cuda(e, "trace ingestion"));
     if (!same_profiles) { c->gc_dev = c->gc; c->gc_dev_at = c->d_gc.p; }      // the copy has landed
     if (rb->err[0]) {
@@ -489,10 +487,7 @@ int disco_reduce_stats(disco_ctx_t* c, disco_policy_stats_t* stats, void* stream
     if (!c || !stats) return fail(DISCO_EINVAL, "null argument");
     if (!c->evaluated) return fail(DISCO_EINVAL, "no evaluation to reduce");
     cudaStream_t st = (cudaStream_t)stream;
-    CU(launch_finalize(c->P, c->G, c->d_gc.as<GroupConst>(), c->d_acc.as<uint64_t>(), c->d_hist_ttft.as<uint64_t>(),
-                       c->d_hist_tbt.as<uint64_t>(), c->grp_sum_n, c->grp_off.as<uint32_t>(),
-                       c->d_stats.as<disco_policy_stats_t>(), c->err, st));
-    // statistics and the error word come back in one copy through pinned memory
+    // statistics and the error word land in pinned host memory straight from the kernel
     const size_t bytes = c->P * sizeof(disco_policy_stats_t) + 16;
     if (bytes > c->stats_host_cap) {
         if (c->stats_host) cudaFreeHost(c->stats_host);
@@ -500,7 +495,9 @@ int disco_reduce_stats(disco_ctx_t* c, disco_policy_stats_t* stats, void* stream
         CU(cudaMallocHost(&c->stats_host, bytes));
         c->stats_host_cap = bytes;
     }
-    CU(cudaMemcpyAsync(c->stats_host, c->d_stats.p, bytes, cudaMemcpyDeviceToHost, st));
+    CU(launch_finalize(c->P, c->G, c->d_gc.as<GroupConst>(), c->d_acc.as<uint64_t>(), c->d_hist_ttft.as<uint64_t>(),
+                       c->d_hist_tbt.as<uint64_t>(), c->grp_sum_n, c->grp_off.as<uint32_t>(),
+                       c->d_stats.as<disco_policy_stats_t>(), (disco_policy_stats_t*)c->stats_host, c->err, st));
     CU(cudaStreamSynchronize(st));
     std::memcpy(stats, c->stats_host, c->P * sizeof(disco_policy_stats_t));
     std::memcpy(c->rb->err, (char*)c->stats_host + c->P * sizeof(disco_policy_stats_t), 16);
@@ -519,8 +516,7 @@ int disco_select_policy(disco_ctx_t* c, double cost_cap, float tbt_slo_s, int32_
     cudaStream_t st = (cudaStream_t)stream;
     if (!c->sel_host) CU(cudaMallocHost((void**)&c->sel_host, 8));
     g_launches += 1;
-    CU(launch_select(c->d_stats.as<disco_policy_stats_t>(), c->P, cost_cap, tbt_slo_s, c->d_select.as<int32_t>(), st));
-    CU(cudaMemcpyAsync(c->sel_host, c->d_select.p, 8, cudaMemcpyDeviceToHost, st));
+    CU(launch_select(c->d_stats.as<disco_policy_stats_t>(), c->P, cost_cap, tbt_slo_s, c->sel_host, st));   // writes the pinned pair
     CU(cudaStreamSynchronize(st));
     *best = c->sel_host[1];
     if (c->sel_host[0] != 0) return fail(DISCO_EINFEASIBLE, "no policy meets the cost cap and the TBT objective");

@@ -164,8 +164,10 @@ cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassCo
                          cudaStream_t st);
 cudaError_t launch_finalize(uint32_t P, int G, const GroupConst* gc, const uint64_t* acc, const uint64_t* hist_ttft,
                             const uint64_t* hist_tbt, const uint64_t* grp_sum_n, const uint32_t* grp_off,
-                            disco_policy_stats_t* stats /* [P] + 16 bytes */, const int32_t* err, cudaStream_t st);
+                            disco_policy_stats_t* stats /* [P] + 16 bytes */,
+                            disco_policy_stats_t* stats_host /* pinned host mirror of the same size, written by the kernel */,
+                            const int32_t* err, cudaStream_t st);
 cudaError_t launch_select(const disco_policy_stats_t* stats, uint32_t P, double cost_cap, float tbt_slo_s,
-                          int32_t* result /* [2]: status, index */, cudaStream_t st);
+                          int32_t* result /* [2]: status, index; may be pinned host memory */, cudaStream_t st);
 
 }  // namespace disco

@@ -54,10 +54,15 @@ __global__ void k_finalize(uint32_t P, int G, const GroupConst* __restrict__ gc,
                            const unsigned long long* __restrict__ acc, const unsigned long long* __restrict__ hist_ttft,
                            const unsigned long long* __restrict__ hist_tbt,
                            const unsigned long long* __restrict__ grp_sum_n, const uint32_t* __restrict__ grp_off,
-                           disco_policy_stats_t* __restrict__ stats, const int32_t* __restrict__ err) {
+                           disco_policy_stats_t* __restrict__ stats, disco_policy_stats_t* __restrict__ stats_host,
+                           const int32_t* __restrict__ err) {
+    // stats_host: the caller's pinned mirror, written straight from here (no copy operation behind the kernel)
     const uint32_t p = blockIdx.x;
     grid_dependency_wait();
-    if (p == 0 && threadIdx.x < 4) ((int32_t*)(stats + P))[threadIdx.x] = err[threadIdx.x];   // error word rides along
+    if (p == 0 && threadIdx.x < 4) {                                                           // error word rides along
+        ((int32_t*)(stats + P))[threadIdx.x] = err[threadIdx.x];
+        ((int32_t*)(stats_host + P))[threadIdx.x] = err[threadIdx.x];
+    }
     __shared__ unsigned long long tot[kNAcc];
     __shared__ int qb[4];
     const unsigned long long N = grp_off[G];
@@ -106,6 +111,7 @@ __global__ void k_finalize(uint32_t P, int G, const GroupConst* __restrict__ gc,
     s.prefill_tok_server = tot[A_PRE_SERVER]; s.prefill_tok_device = tot[A_PRE_DEVICE];
     s.delayed_tokens = tot[A_DELAYED];
     stats[p] = s;
+    stats_host[p] = s;
 }
 
 // Lexicographic objective of the selection: (tail TTFT bin, mean TTFT, cost, index), feasible policies only.
@@ -153,10 +159,11 @@ __global__ void k_select(const disco_policy_stats_t* __restrict__ stats, uint32_
 
 cudaError_t launch_finalize(uint32_t P, int G, const GroupConst* gc, const uint64_t* acc, const uint64_t* hist_ttft,
                             const uint64_t* hist_tbt, const uint64_t* grp_sum_n, const uint32_t* grp_off,
-                            disco_policy_stats_t* stats, const int32_t* err, cudaStream_t st) {
+                            disco_policy_stats_t* stats, disco_policy_stats_t* stats_host, const int32_t* err,
+                            cudaStream_t st) {
     return launch_after(k_finalize, P, 32, 0, st, P, G, gc, (const unsigned long long*)acc,
                         (const unsigned long long*)hist_ttft, (const unsigned long long*)hist_tbt,
-                        (const unsigned long long*)grp_sum_n, grp_off, stats, err);
+                        (const unsigned long long*)grp_sum_n, grp_off, stats, stats_host, err);
 }
 
 cudaError_t launch_select(const disco_policy_stats_t* stats, uint32_t P, double cost_cap, float tbt_slo_s,
