@@ -76,6 +76,33 @@ __global__ void k_ingest(uint32_t n, const int32_t* __restrict__ prompt, const i
     if (threadIdx.x == 0 && s_max) atomicMax(max_n, s_max);
 }
 
+// Inclusive prefix sum over the threads of a block (blockDim.x a multiple of 32, at most 1024): shuffles inside
+// the warps, one pass over the warp totals, two barriers.  `wtot` is shared scratch of 32 entries; every thread
+// of the block must call.  Returns this thread's inclusive sum; *total receives the block's sum.
+template <class T>
+__device__ __forceinline__ T block_inclusive_scan(T v, T* wtot, T* total) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const T up = __shfl_up_sync(0xFFFFFFFFu, v, off);
+        if (lane >= off) v += up;
+    }
+    if (lane == 31) wtot[w] = v;
+    __syncthreads();
+    if (w == 0) {
+        T t = lane < nw ? wtot[lane] : T(0);
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const T up = __shfl_up_sync(0xFFFFFFFFu, t, off);
+            if (lane >= off) t += up;
+        }
+        wtot[lane] = t;                                   // inclusive over the warps
+    }
+    __syncthreads();
+    if (total) *total = wtot[nw - 1];
+    return w ? v + wtot[w - 1] : v;
+}
+
 // ---- one stable LSD radix pass over 64-bit keys (8-bit digit), optional 32-bit payload -------------------
 constexpr int kRadixThreads = 256;
 constexpr int kRadixWarps = kRadixThreads / 32;
@@ -96,24 +123,17 @@ __global__ void k_radix_hist(const uint64_t* __restrict__ keys, uint32_t n, uint
 // One block per digit: exclusive scan of the digit's per-block counts, in place, and the digit's total.
 __global__ void k_radix_rowscan(uint32_t* __restrict__ counts /* [256][blocks] */, uint32_t blocks,
                                 uint32_t* __restrict__ totals /* [256] */) {
-    __shared__ uint32_t part[128];
+    __shared__ uint32_t wtot[32];
     grid_dependency_wait();
     uint32_t* row = counts + (size_t)blockIdx.x * blocks;
     const uint32_t per = (blocks + 127u) / 128u;
     const uint32_t lo = min(blocks, threadIdx.x * per), hi = min(blocks, lo + per);
     uint32_t s = 0;
     for (uint32_t i = lo; i < hi; ++i) s += row[i];
-    part[threadIdx.x] = s;
-    __syncthreads();
-    for (int off = 1; off < 128; off <<= 1) {
-        const uint32_t v = (int)threadIdx.x >= off ? part[threadIdx.x - off] : 0u;
-        __syncthreads();
-        part[threadIdx.x] += v;
-        __syncthreads();
-    }
-    uint32_t run = part[threadIdx.x] - s;
+    uint32_t total;
+    uint32_t run = block_inclusive_scan(s, wtot, &total) - s;
     for (uint32_t i = lo; i < hi; ++i) { const uint32_t c = row[i]; row[i] = run; run += c; }
-    if (threadIdx.x == 127) totals[blockIdx.x] = part[127];
+    if (threadIdx.x == 0) totals[blockIdx.x] = total;
 }
 
 __global__ void k_radix_scatter(const uint64_t* __restrict__ keys_in, uint64_t* __restrict__ keys_out,
@@ -128,17 +148,10 @@ __global__ void k_radix_scatter(const uint64_t* __restrict__ keys_in, uint64_t* 
     {
         // offsets[d][b]: keys of digit d in earlier blocks (k_radix_rowscan); totals[d]: keys of digit d.
         // This block's first slot for digit d = keys of smaller digits + keys of d in earlier blocks.
-        uint32_t* tot = wcnt[0];
-        const uint32_t total = totals[threadIdx.x];
-        tot[threadIdx.x] = total;
-        __syncthreads();
-        for (int off = 1; off < 256; off <<= 1) {
-            const uint32_t v = (int)threadIdx.x >= off ? tot[threadIdx.x - off] : 0u;
-            __syncthreads();
-            tot[threadIdx.x] += v;
-            __syncthreads();
-        }
-        run[threadIdx.x] = tot[threadIdx.x] - total + offsets[threadIdx.x * gridDim.x + blockIdx.x];
+        uint32_t* wtot = wcnt[0];                                    // scratch of the scan (32 words)
+        const uint32_t total = totals[threadIdx.x], before = offsets[threadIdx.x * gridDim.x + blockIdx.x];
+        const uint32_t incl = block_inclusive_scan(total, wtot, (uint32_t*)nullptr);
+        run[threadIdx.x] = incl - total + before;
         __syncthreads();
     }
     const uint32_t lo = min(n, blockIdx.x * per_block), hi = min(n, lo + per_block);
@@ -227,8 +240,8 @@ __global__ void k_low_words(uint32_t n, const uint64_t* __restrict__ keys, int32
 __device__ __forceinline__ void group_mass(const uint32_t* __restrict__ cnt, int64_t* __restrict__ cum,
                                            uint32_t* __restrict__ ng) {
     constexpr int NT = 1024, L = kMaxPrompt + 1;      // 4097 lengths
-    __shared__ unsigned long long pm[NT];
-    __shared__ uint32_t pc[NT];
+    __shared__ unsigned long long wm[32];
+    __shared__ uint32_t wc[32];
     const int g = blockIdx.x;
     const uint32_t* c = cnt + (size_t)g * L;
     int64_t* out = cum + (size_t)g * (L + 1);
@@ -236,18 +249,11 @@ __device__ __forceinline__ void group_mass(const uint32_t* __restrict__ cnt, int
     const int lo = min(L, (int)threadIdx.x * per), hi = min(L, lo + per);
     unsigned long long m = 0; uint32_t k = 0;
     for (int l = lo; l < hi; ++l) { m += (unsigned long long)l * c[l]; k += c[l]; }
-    pm[threadIdx.x] = m; pc[threadIdx.x] = k;
-    __syncthreads();
-    for (int off = 1; off < NT; off <<= 1) {
-        unsigned long long vm = 0; uint32_t vc = 0;
-        if ((int)threadIdx.x >= off) { vm = pm[threadIdx.x - off]; vc = pc[threadIdx.x - off]; }
-        __syncthreads();
-        pm[threadIdx.x] += vm; pc[threadIdx.x] += vc;
-        __syncthreads();
-    }
-    unsigned long long run = pm[threadIdx.x] - m;
+    unsigned long long m_total; uint32_t k_total;
+    unsigned long long run = block_inclusive_scan(m, wm, &m_total) - m;
+    block_inclusive_scan(k, wc, &k_total);
     for (int l = lo; l < hi; ++l) { out[l] = (int64_t)run; run += (unsigned long long)l * c[l]; }
-    if (threadIdx.x == NT - 1) { out[L] = (int64_t)pm[NT - 1]; ng[g] = pc[NT - 1]; }
+    if (threadIdx.x == 0) { out[L] = (int64_t)m_total; ng[g] = k_total; }
 }
 
 // Group offsets in the partitioned order, the 257 knots K_g[k] = sorted_g[(k (N_g - 1)) / 256] and the few
