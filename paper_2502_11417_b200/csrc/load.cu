@@ -24,13 +24,13 @@ __global__ void k_ingest(uint32_t n, const int32_t* __restrict__ prompt, const i
     // counts0: first radix digit counted per sort block (small traces; large ones use the histogram kernel)
     __shared__ unsigned long long s_sum[kMaxGroups];
     __shared__ uint32_t s_cnt[kMaxGroups];
-    __shared__ uint32_t s_max;
+    __shared__ uint32_t s_max, s_max_ticks;         // longest output, largest TTFT ticks (max_n[0], max_n[1])
     __shared__ uint32_t s_len[kMaxPrompt + 1];       // length histogram of this block (single-group traces)
     const int G = (int)(ns * nd);
     const bool one = G == 1;
     for (int g = threadIdx.x; g < G; g += blockDim.x) { s_sum[g] = 0; s_cnt[g] = 0; }
     if (one) for (int i = threadIdx.x; i <= kMaxPrompt; i += blockDim.x) s_len[i] = 0;
-    if (threadIdx.x == 0) s_max = 0;
+    if (threadIdx.x == 0) { s_max = 0; s_max_ticks = 0; }
     __syncthreads();
     const uint32_t stride = gridDim.x * blockDim.x;
     for (uint32_t i0 = blockIdx.x * blockDim.x; i0 < n; i0 += stride) {       // whole warps iterate together
@@ -62,18 +62,21 @@ __global__ void k_ingest(uint32_t n, const int32_t* __restrict__ prompt, const i
             const uint32_t so = __reduce_add_sync(0xFFFFFFFFu, ok ? (uint32_t)o : 0u);
             const uint32_t mo = __reduce_max_sync(0xFFFFFFFFu, ok ? (uint32_t)o : 0u);
             const uint32_t co = __popc(__ballot_sync(0xFFFFFFFFu, ok));
+            const uint32_t mt = __reduce_max_sync(0xFFFFFFFFu, ok ? (uint32_t)S : 0u);
             if ((threadIdx.x & 31) == 0 && co) {
                 atomicAdd(&s_sum[0], (unsigned long long)so); atomicAdd(&s_cnt[0], co); atomicMax(&s_max, mo);
+                atomicMax(&s_max_ticks, mt);
             }
         } else if (ok) {
             atomicAdd(&s_sum[g], (unsigned long long)o); atomicAdd(&s_cnt[g], 1u); atomicMax(&s_max, (uint32_t)o);
+            atomicMax(&s_max_ticks, (uint32_t)S);
         }
     }
     __syncthreads();
     for (int g = threadIdx.x; g < G; g += blockDim.x)
         if (s_cnt[g]) { atomicAdd(&grp_sum_n[g], s_sum[g]); atomicAdd(&grp_n[g], s_cnt[g]); }
     if (one) for (int i = threadIdx.x; i <= kMaxPrompt; i += blockDim.x) if (s_len[i]) atomicAdd(&cnt[i], s_len[i]);
-    if (threadIdx.x == 0 && s_max) atomicMax(max_n, s_max);
+    if (threadIdx.x == 0 && s_max) { atomicMax(max_n, s_max); atomicMax(max_n + 1, s_max_ticks); }
 }
 
 // Inclusive prefix sum over the threads of a block (blockDim.x a multiple of 32, at most 1024): shuffles inside
@@ -108,10 +111,14 @@ constexpr int kRadixThreads = 256;
 constexpr int kRadixWarps = kRadixThreads / 32;
 
 __global__ void k_radix_hist(const uint64_t* __restrict__ keys, uint32_t n, uint32_t per_block, int shift,
-                             uint32_t* __restrict__ counts /* [256][gridDim.x] */) {
+                             uint32_t* __restrict__ counts /* [256][gridDim.x] */,
+                             const uint32_t* __restrict__ max_key = nullptr, uint32_t skip_below = 0) {
+    // max_key, skip_below: the pass is not needed (every key has this digit zero, the order is final) when the
+    // largest key is below skip_below; the kernels of such a pass return at once
     __shared__ uint32_t h[256];
     h[threadIdx.x] = 0;
     grid_dependency_wait();
+    if (max_key && *max_key < skip_below) return;
     __syncthreads();
     const uint32_t lo = min(n, blockIdx.x * per_block), hi = min(n, lo + per_block);
     for (uint32_t i = lo + threadIdx.x; i < hi; i += kRadixThreads)
@@ -122,9 +129,11 @@ __global__ void k_radix_hist(const uint64_t* __restrict__ keys, uint32_t n, uint
 
 // One block per digit: exclusive scan of the digit's per-block counts, in place, and the digit's total.
 __global__ void k_radix_rowscan(uint32_t* __restrict__ counts /* [256][blocks] */, uint32_t blocks,
-                                uint32_t* __restrict__ totals /* [256] */) {
+                                uint32_t* __restrict__ totals /* [256] */,
+                                const uint32_t* __restrict__ max_key = nullptr, uint32_t skip_below = 0) {
     __shared__ uint32_t wtot[32];
     grid_dependency_wait();
+    if (max_key && *max_key < skip_below) return;
     uint32_t* row = counts + (size_t)blockIdx.x * blocks;
     const uint32_t per = (blocks + 127u) / 128u;
     const uint32_t lo = min(blocks, threadIdx.x * per), hi = min(blocks, lo + per);
@@ -140,11 +149,17 @@ __global__ void k_radix_scatter(const uint64_t* __restrict__ keys_in, uint64_t* 
                                 const uint32_t* __restrict__ pay_in, uint32_t* __restrict__ pay_out, uint32_t n,
                                 uint32_t per_block, int shift, const uint32_t* __restrict__ offsets,
                                 const uint32_t* __restrict__ totals, uint32_t* __restrict__ counts_next = nullptr,
-                                int32_t* __restrict__ low_out = nullptr) {
+                                int32_t* __restrict__ low_out = nullptr,
+                                const uint32_t* __restrict__ max_key = nullptr, uint32_t skip_below = 0,
+                                int32_t* __restrict__ low_out_if_last = nullptr, uint32_t last_below = 0) {
+    // low_out: the last pass writes the low words (the sorted ticks) instead of the keys.  low_out_if_last: this
+    // pass writes them as well when the largest key is below last_below (the later passes then skip themselves).
     __shared__ uint32_t run[256];                 // next output slot of each digit for this block
     __shared__ uint32_t wcnt[kRadixWarps][256];   // keys of each digit per warp in the current slab
     const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
     grid_dependency_wait();
+    if (max_key && *max_key < skip_below) return;
+    if (low_out_if_last && *max_key >= last_below) low_out_if_last = nullptr;
     {
         // offsets[d][b]: keys of digit d in earlier blocks (k_radix_rowscan); totals[d]: keys of digit d.
         // This block's first slot for digit d = keys of smaller digits + keys of d in earlier blocks.
@@ -198,6 +213,7 @@ __global__ void k_radix_scatter(const uint64_t* __restrict__ keys_in, uint64_t* 
                 const uint32_t rank = __popc(peers[j] & ((1u << lane) - 1u));
                 const uint32_t pos = wcnt[w][dig[j]] + rank;
                 if (low_out) low_out[pos] = (int32_t)(uint32_t)key[j]; else keys_out[pos] = key[j];
+                if (low_out_if_last) low_out_if_last[pos] = (int32_t)(uint32_t)key[j];
                 if (pay_out) {
                     const uint32_t i = base + w * (32 * kPer) + j * 32 + lane;
                     pay_out[pos] = pay_in ? pay_in[i] : i;
@@ -363,12 +379,17 @@ cudaError_t run_load(const LoadArgs& a, cudaStream_t st) {
                 // with the block-private histogram kernel instead.
                 const bool last = p == passes - 1, fused_next = p == 0;
                 uint32_t* cur = a.radix_counts + (size_t)p * 256u * blocks;
+                // Ticks below 2^24 (16.7 s) leave the fourth byte zero: the third pass then also writes the sorted
+                // ticks and the kernels of the fourth return at once (a.max_n[1]: the largest tick, from ingestion).
+                const uint32_t* max_key = a.max_n + 1;
+                const uint32_t skip_below = p == 3 ? (1u << 24) : 0u;
                 if (p >= 2 && (e = launch_after(k_radix_hist, blocks, kRadixThreads, 0, st, (const uint64_t*)src, n, per_block,
-                                                8 * p, cur))) return e;
-                if ((e = launch_after(k_radix_rowscan, 256, 128, 0, st, cur, blocks, totals))) return e;
+                                                8 * p, cur, max_key, skip_below))) return e;
+                if ((e = launch_after(k_radix_rowscan, 256, 128, 0, st, cur, blocks, totals, max_key, skip_below))) return e;
                 if ((e = launch_after(k_radix_scatter, blocks, kRadixThreads, 0, st, src, dst, nullptr, nullptr, n, per_block,
                                       8 * p, cur, totals, fused_next ? cur + 256u * blocks : nullptr,
-                                      last ? a.sorted : nullptr))) return e;
+                                      last ? a.sorted : nullptr, max_key, skip_below,
+                                      p == 2 ? a.sorted : nullptr, 1u << 24))) return e;
                 uint64_t* t = src; src = dst; dst = t;
             }
         } else {

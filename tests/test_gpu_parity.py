@@ -91,6 +91,18 @@ def test_consumption_interval_equal_to_slowest_token():
     tr.close()
 
 
+@pytest.mark.parametrize("top_s", [16.70, 16.80, 1500.0])
+def test_sorted_ticks_around_the_fourth_radix_byte(top_s):
+    # one-group traces whose largest TTFT lies just below 2^24 ticks (the fourth radix pass skips itself), just
+    # above it and far above it: the sorted sample, the knots and everything derived from them
+    w = synth.make_workload(1, n=6000, n_budgets=5)
+    w.server_ttft_s[::97] *= np.float32(7.0)
+    w.server_ttft_s[5] = np.float32(top_s)
+    assert float(w.server_ttft_s.max()) == float(np.float32(top_s))
+    full_parity(w, [synth.policy(b, flags=MIG | PACE | D_MODE) for b in (0.02, 0.3, 0.8)] + w.policies,
+                tag=f"radix-top-{top_s}")
+
+
 def test_stochastic_baselines_and_expected_length():
     # Stoch-S / Stoch-D routing and the expected-length trigger, mixed with ordinary policies in one call
     STOCH = synth.FLAG_STOCHASTIC
