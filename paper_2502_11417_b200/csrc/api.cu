@@ -66,7 +66,7 @@ struct disco_ctx {
     DevBuf in_prompt, in_out, in_ttft, in_sp, in_dp;      // staging of host inputs
     DevBuf keys_a, keys_b, tmp_idx;
     DevBuf S, l, nout, orig, sorted;
-    DevBuf zero, cum_mass, ng_exact, grp_off, knots, d_rb, d_gc;   // `zero`: every table a load must clear, contiguous
+    DevBuf zero, cum_mass, ng_exact, grp_off, knots, d_gc;   // `zero`: every table a load must clear, contiguous
     uint32_t *cnt = nullptr, *ng = nullptr, *max_n = nullptr, *radix_counts = nullptr;
     uint64_t* grp_sum_n = nullptr;
     int32_t* err = nullptr;
@@ -76,7 +76,7 @@ struct disco_ctx {
     uint32_t P = 0;
     bool evaluated = false, reduced = false;
     std::vector<PolicyConst> pol;
-    DevBuf d_prep, d_accum, d_stats, d_tables, d_select, d_todo;
+    DevBuf d_prep, d_accum, d_stats, d_tables, d_todo;
     struct View { void* p = nullptr; template <class T> T* as() const { return (T*)p; } };
     View d_acc, d_hist_ttft, d_hist_tbt;               // three regions of d_accum (cleared by one memset)
     View d_pol, d_classes, d_pol_list, d_chunks;       // four regions of d_tables (filled by one copy)
@@ -94,7 +94,7 @@ struct disco_ctx {
 
     ~disco_ctx() {
         DevBuf* all[] = {&in_prompt, &in_out, &in_ttft, &in_sp, &in_dp, &keys_a, &keys_b, &tmp_idx,
-                         &S, &l, &nout, &orig, &sorted, &zero, &cum_mass, &ng_exact, &grp_off, &knots, &d_rb, &d_gc, &d_prep, &d_accum, &d_stats, &d_tables, &d_select, &d_todo};
+                         &S, &l, &nout, &orig, &sorted, &zero, &cum_mass, &ng_exact, &grp_off, &knots, &d_gc, &d_prep, &d_accum, &d_stats, &d_tables, &d_todo};
         for (DevBuf* b : all) b->release();
         for (auto& b : rec_u32) b.release();
         for (auto& b : rec_u16) b.release();
@@ -174,7 +174,7 @@ cudaError_t reserve_trace(disco_ctx* c, uint32_t n, bool host_inputs, bool has_s
     c->zero_bytes = head;
     R(cum_mass, (size_t)G * (kMaxPrompt + 2) * 8); R(ng_exact, kMaxGroups * 4);
     R(grp_off, (kMaxGroups + 1) * 4); R(knots, (size_t)G * kNKnots * 4);
-    R(d_rb, sizeof(LoadReadback)); R(d_gc, (size_t)G * sizeof(GroupConst));
+    R(d_gc, (size_t)G * sizeof(GroupConst));
 #undef R
     return cudaSuccess;
 }
@@ -357,7 +357,7 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
     R(d_todo, N1 * 4);
     c->d_acc.p = c->d_accum.p; c->d_hist_ttft.p = (char*)c->d_accum.p + acc_bytes;
     c->d_hist_tbt.p = (char*)c->d_accum.p + acc_bytes + hist_bytes;
-    R(d_stats, P * sizeof(disco_policy_stats_t) + 16); R(d_select, 8);
+    R(d_stats, P * sizeof(disco_policy_stats_t) + 16);
     for (int k = 0; k < 7; ++k) R(rec_u32[k], N1 * 4);
     for (int k = 0; k < 2; ++k) R(rec_u16[k], N1 * 2);
     for (int k = 0; k < 3; ++k) R(rec_win[k], N1 * wmax[k] * 4);
