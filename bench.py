@@ -283,7 +283,7 @@ def run_ours(args):
     l0 = kernel_launch_count()
     # the first 75 or so steps of a fresh process run about 10 % slower (clocks and caches settling): at least
     # MIN_WARMUP untimed steps are run, whatever --warmup says; `warmup_run` in the output says how many
-    warm = max(args.warmup, MIN_WARMUP)
+    warm = max(args.warmup, args.min_warmup)
     timed(dev, 0, warm)
     l_warm = kernel_launch_count()
     sampler.start()
@@ -391,6 +391,8 @@ def main():
     ap.add_argument("--config", type=int, default=1, help="workload 0..5 (default: workload 1)")
     ap.add_argument("--requests", type=int, default=None, help="shrink the trace (profiling on a small case)")
     ap.add_argument("--budgets", type=int, default=None, help="shrink the budget axis (profiling on a small case)")
+    ap.add_argument("--min-warmup", type=int, default=MIN_WARMUP,
+                    help="untimed steps run at the least, whatever --warmup says (profiling runs pass a small number)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--oracle-seconds", type=float, default=15.0, help="CPU time of the oracle baseline sample")
     ap.add_argument("--oracle-step-seconds", type=float, default=3.0, help="--impl reference: CPU time per step")
