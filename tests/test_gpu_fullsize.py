@@ -145,3 +145,24 @@ def test_workload2_full_size_whole_grid_properties():
     for cap, slo in [(1.25 * cheapest, 0.25), (1.02 * cheapest, 0.25), (0.5 * cheapest, 0.25), (1e30, 1e-3)]:
         assert tr.select_policy(cap, slo) == _select_by_definition(st, cap, slo), (cap, slo)
     tr.close()
+
+
+def test_pair_arrays_beyond_2_32_elements():
+    # 4.3 M requests x 1024 policies = 4.4e9 pairs: element indices no longer fit 32 bits, so the row writer runs
+    # with 64-bit indices.  Its rows must equal those of two half-grid runs, whose indices do fit.
+    import torch
+    w = synth.make_workload(2, n=4_300_000)
+    P = len(w.policies)
+    assert P * w.n > 2 ** 32 and (P // 2) * w.n < 2 ** 32
+    tr = Trace.from_workload(w)
+    full = tr.alloc_pair_outputs(P, fields=["decision"])
+    tr.eval_policies(w.policies, w.seed, full)
+    tr.reduce_stats()
+    half = tr.alloc_pair_outputs(P // 2, fields=["decision"])
+    for lo in (0, P // 2):
+        tr.eval_policies(w.policies[lo:lo + P // 2], w.seed, half)
+        tr.reduce_stats()
+        assert torch.equal(full["decision"][lo:lo + P // 2], half["decision"]), lo
+    # and the rows are not trivially constant: budgets 0 and 1 decide differently
+    assert int(full["decision"][0].max()) == 1 and int(full["decision"][255].min()) != 1
+    tr.close()
