@@ -91,7 +91,11 @@ typedef struct {
     uint32_t n_servers;               /* >= 1; n_servers * n_devices <= 64 */
     const disco_device_profile_t* devices;  /* host, [n_devices] */
     uint32_t n_devices;
-    uint32_t arrays_on_device;        /* 0: the five [n] arrays are host memory; 1: device memory */
+    uint32_t arrays_on_device;        /* 0: the five [n] arrays are host memory; 1: device memory.  Host arrays that
+                                         are all page-locked (cudaHostAlloc, cudaHostRegister) are read by the
+                                         ingestion kernel in place when the trace has one profile group; otherwise
+                                         they are copied to the device first.  Either way they may be reused as soon
+                                         as disco_load_trace returns. */
 } disco_trace_desc_t;
 
 /* One policy setting (Algorithm 1 inputs b, alpha; Eq. 4 overhead; Eq. 6 t_m, r_c). */

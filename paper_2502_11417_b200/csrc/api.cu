@@ -206,8 +206,24 @@ int disco_load_trace(disco_ctx_t** pctx, const disco_trace_desc_t* d, void* stre
     c->loaded = c->evaluated = c->reduced = false;
     c->n = (uint32_t)d->n; c->ns = d->n_servers; c->nd = d->n_devices; c->G = (int)gc.size(); c->gc = gc;
     const uint32_t n = c->n;
-    const bool host_in = d->arrays_on_device == 0;
+    bool host_in = d->arrays_on_device == 0;
     cudaError_t e;
+    // Host arrays that are page-locked and mapped (cudaHostAlloc, cudaHostRegister, a pinned tensor) are read by
+    // the ingestion kernel in place when the trace has one profile group (every element is then read exactly
+    // once): no staging copies.  Pageable arrays, or traces with several groups, are copied first.
+    const void* in_place[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+    bool zero_copy = host_in && n != 0 && gc.size() == 1;
+    if (zero_copy) {
+        const void* host[5] = {d->prompt_len, d->output_len, d->server_ttft_s, d->server_profile, d->device_profile};
+        for (int k = 0; k < 5 && zero_copy; ++k) {
+            if (!host[k]) continue;
+            cudaPointerAttributes attr;
+            if (cudaPointerGetAttributes(&attr, host[k]) != cudaSuccess) { cudaGetLastError(); zero_copy = false; break; }
+            if (attr.type != cudaMemoryTypeHost || !attr.devicePointer) zero_copy = false;
+            else in_place[k] = attr.devicePointer;
+        }
+    }
+    if (zero_copy) host_in = false;
     if (!c->rb && (e = cudaMallocHost((void**)&c->rb, sizeof(HostReadback))) != cudaSuccess)
         return bail(fail_cuda(e, "cudaMallocHost"));
     if ((e = reserve_trace(c, n, host_in, d->server_profile != nullptr, d->device_profile != nullptr)) != cudaSuccess)
@@ -226,6 +242,9 @@ int disco_load_trace(disco_ctx_t** pctx, const disco_trace_desc_t* d, void* stre
         a.prompt = c->in_prompt.as<int32_t>(); a.outlen = c->in_out.as<int32_t>(); a.ttft = c->in_ttft.as<float>();
         a.sp = d->server_profile ? c->in_sp.as<uint8_t>() : nullptr;
         a.dp = d->device_profile ? c->in_dp.as<uint8_t>() : nullptr;
+    } else if (zero_copy) {
+        a.prompt = (const int32_t*)in_place[0]; a.outlen = (const int32_t*)in_place[1]; a.ttft = (const float*)in_place[2];
+        a.sp = (const uint8_t*)in_place[3]; a.dp = (const uint8_t*)in_place[4];
     } else {
         a.prompt = d->prompt_len; a.outlen = d->output_len; a.ttft = d->server_ttft_s;
         a.sp = d->server_profile; a.dp = d->device_profile;

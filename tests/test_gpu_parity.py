@@ -206,6 +206,29 @@ def test_device_resident_inputs_match_host_inputs():
         assert bytes(sa[p]) == bytes(sb[p])
 
 
+def test_pinned_host_inputs_read_in_place_match_pageable_ones():
+    # one profile group: page-locked host arrays are read by the ingestion kernel in place, pageable ones are
+    # copied first; both must give the same tables and statistics (and the oracle's)
+    import torch
+    from parity import check_tables
+    from oracle import Oracle
+    w = synth.make_workload(1, n=30011, n_budgets=7)
+    w.server_profile = None; w.device_profile = None          # optional arrays left out
+    a = Trace.from_workload(w)
+    a.eval_policies(w.policies, 9)
+    sa = a.reduce_stats()
+    pinned = [torch.from_numpy(x).pin_memory() for x in (w.prompt_len, w.output_len, w.server_ttft_s)]
+    b = Trace().load_trace(*pinned, None, None, w.servers, w.devices)
+    check_tables(b, Oracle.from_workload(w), "pinned")
+    b.eval_policies(w.policies, 9)
+    sb = b.reduce_stats()
+    for p in range(len(w.policies)):
+        assert bytes(sa[p]) == bytes(sb[p])
+    pinned[0][17] = 0                                          # validation still sees the in-place arrays
+    with pytest.raises(DiscoError):
+        Trace().load_trace(*pinned, None, None, w.servers, w.devices)
+
+
 def test_non_default_stream_and_partial_outputs():
     import torch
     w = synth.make_workload(1, n=3000, n_budgets=4)
