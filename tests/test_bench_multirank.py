@@ -50,3 +50,19 @@ def test_replica_zero_is_the_reference_trace():
     assert (a.prompt_len == b.prompt_len).all() and (a.server_ttft_s == b.server_ttft_s).all()
     c = synth.make_workload(1, n=300, replica=3)
     assert not np.array_equal(a.output_len, c.output_len)
+
+
+def test_never_clamps_follows_the_tick_arithmetic():
+    """bench.never_clamps decides which algorithmic instruction count the play-out is held against: true iff
+    every policy paces delivery and tau >= T + J for every endpoint, in microsecond ticks."""
+    import bench
+    from paper_2502_11417_b200 import synth
+    for cfg in range(6):
+        assert bench.never_clamps(synth.make_workload(cfg, n=64))
+    w = synth.make_workload(3, n=64, n_budgets=2)                      # phone-class device: T = 100,000, J = 5,000
+    w.policies = [synth.policy(0.5, r_c=1e6 / 105000.0)]
+    assert bench.never_clamps(w)                                       # tau = T + J exactly
+    w.policies = [synth.policy(0.5, r_c=1e6 / 104999.0)]
+    assert not bench.never_clamps(w)
+    w.policies = [synth.policy(0.5, flags=synth.FLAG_MIGRATION)]       # pacing off
+    assert not bench.never_clamps(w)
