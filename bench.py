@@ -52,7 +52,7 @@ MIN_WARMUP = 100             # untimed steps before either timed region, at the 
 KERNEL_EVENT_STRIDE = 8      # per-kernel CUDA events are recorded on every 8th timed step
 # DRAM bytes per launch from the committed ncu capture of the dominant kernel (None until captured for
 # the current kernel; see profiles/).
-NCU_TRAFFIC_BYTES = {"k_pairs_rows": 149264896, "k_pairs_acc": None, "k_playout_fast": 827904, "k_playout": None}
+NCU_TRAFFIC_BYTES = {"k_pairs_rows": 148985344, "k_pairs_acc": None, "k_playout_fast": 828160, "k_playout": None}
 
 
 def env_rank():
