@@ -381,6 +381,9 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
     for (int k = 0; k < 2; ++k) R(rec_u16[k], N1 * 2);
     for (int k = 0; k < 3; ++k) R(rec_win[k], N1 * wmax[k] * 4);
 
+    // the accumulators are cleared while the host lays out the chunks and tables below
+    CU(cudaMemsetAsync(c->d_accum.p, 0, acc_bytes + 2 * hist_bytes + cnt_bytes, st));
+
     // ---- policies grouped by class; request chunks (one group each) sized so that chunks x policy tiles
     //      fill the GPU about once
     std::vector<uint32_t> pol_list;
@@ -442,7 +445,6 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
     CU(cudaMemcpyAsync(dt, sp, off, cudaMemcpyHostToDevice, st));
     CU(cudaEventRecord(c->stage_free, st));
 
-    CU(cudaMemsetAsync(c->d_accum.p, 0, acc_bytes + 2 * hist_bytes + cnt_bytes, st));
     uint32_t* todo_counts = (uint32_t*)((char*)c->d_accum.p + acc_bytes + 2 * hist_bytes);
 
     // ---- Algorithms 1-3 for every (group, policy)
