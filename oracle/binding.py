@@ -86,7 +86,9 @@ _lib = None
 def lib() -> C.CDLL:
     global _lib
     if _lib is None:
-        L = C.CDLL(build_oracle())
+        # DISCO_ORACLE_LIB: a library built elsewhere from a deliberately broken copy of the source (the mutation
+        # check of the pins, tests/oracle_mutants.py); never set in ordinary runs
+        L = C.CDLL(os.environ.get("DISCO_ORACLE_LIB") or build_oracle())
         L.orc_mix.restype = C.c_uint32; L.orc_mix.argtypes = [C.c_uint32]
         L.orc_hash.restype = C.c_uint32; L.orc_hash.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32]
         L.orc_jitter.restype = C.c_int64; L.orc_jitter.argtypes = [C.c_uint32, C.c_int64]

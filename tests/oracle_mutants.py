@@ -1,0 +1,93 @@
+"""Mutation check of the oracle's pins: plants one plausible mistake at a time in a COPY of the oracle's source
+(a wrong comparison, index, sign, shift or a swapped endpoint), builds it, and runs the CPU pin tests against the
+broken library.  A pin set that bites fails for every mutant.  Nothing here touches the CUDA path.
+
+    python tests/oracle_mutants.py            # all mutants; prints the survivors, exit status 1 if there are any
+    python tests/oracle_mutants.py 3 7        # only these
+"""
+import os
+import subprocess
+import sys
+import tempfile
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+SRC = os.path.join(ROOT, "oracle", "disco_oracle.cpp")
+
+# (what the mistake is, exact text in the source, replacement)
+MUTANTS = [
+    ("hash: first shift 16 -> 15", "    x ^= x >> 16; x *= MUL1;", "    x ^= x >> 15; x *= MUL1;"),
+    ("hash: multipliers swapped", "    x ^= x >> 15; x *= MUL2;", "    x ^= x >> 15; x *= MUL1;"),
+    ("Eq. 3: >= becomes >", "if ((double)mass >= target) break;", "if ((double)mass > target) break;"),
+    ("inverse CDF: rank off by one", "std::ceil(q * (double)G.N) - 1.0;", "std::ceil(q * (double)G.N);"),
+    ("race: device starts on a tie", "R->device_started = S > w;", "R->device_started = S >= w;"),
+    ("race: tie goes to the device", "R->winner_device = !(S <= w + Td);", "R->winner_device = !(S < w + Td);"),
+    ("race: wait dropped from the device's TTFT", "R->ttft = std::min(S, w + Td);", "R->ttft = std::min(S, Td);"),
+    ("jitter amplitude of the other endpoint", "const int64_t J = R->winner_device ? dv.J : sv.J;",
+     "const int64_t J = R->winner_device ? sv.J : dv.J;"),
+    ("pacing: max becomes the generation time",
+     "for (int32_t j = 2; j <= n; ++j) d[j] = pacing ? std::max(g[j], d[j - 1] + tau) : g[j];",
+     "for (int32_t j = 2; j <= n; ++j) d[j] = pacing ? std::max(g[j], d[j - 1]) : g[j];"),
+    ("buffer test: index off by one", "if (d[j - pr.B + 1] > g[j]) { m = j; break; }",
+     "if (d[j - pr.B] > g[j]) { m = j; break; }"),
+    ("buffer test: > becomes >=", "if (d[j - pr.B + 1] > g[j]) { m = j; break; }",
+     "if (d[j - pr.B + 1] >= g[j]) { m = j; break; }"),
+    ("trigger: > becomes >=", "if (saving > pol.mig_threshold) {", "if (saving >= pol.mig_threshold) {"),
+    ("hand-off latency: generated tokens not re-prefilled", "M = dv.kappa * (int64_t)(l + m) + dv.c0;",
+     "M = dv.kappa * (int64_t)(l) + dv.c0;"),
+    ("knot interpolation: fraction shift", "(int64_t)fr) >> 16);", "(int64_t)fr) >> 15);"),
+    ("target stream keeps the source's interval", "Tt = dv.T; Jt = dv.J;", "Tt = sv.T; Jt = dv.J;"),
+    ("delayed tokens: slot origin off by one", "if (g[j] > d[m] + (int64_t)(j - m) * tau) ++R->delayed;",
+     "if (g[j] > d[m] + (int64_t)(j - m - 1) * tau) ++R->delayed;"),
+    ("tokens: endpoints swapped", "R->tok_server = R->winner_device ? tgt : src;",
+     "R->tok_server = R->winner_device ? src : tgt;"),
+    ("prefill billing: loser's prefill not billed", "R->pre_device = R->device_started ? l : 0;",
+     "R->pre_device = (R->device_started && R->winner_device) ? l : 0;"),
+    ("Algorithm 2: tail quantile uses max instead of min", "const double q_tail = 1.0 - std::min(alpha, b);",
+     "const double q_tail = 1.0 - std::max(alpha, b);"),
+    ("Algorithm 2: budget not normalised by 1 - alpha", "const double A = ((b - alpha) / (1.0 - alpha)) * (double)G.Total;",
+     "const double A = (b - alpha) * (double)G.Total;"),
+    ("Algorithm 2: class funded on a strict comparison", "if ((double)with_l <= A) { funded = with_l; continue; }",
+     "if ((double)with_l < A) { funded = with_l; continue; }"),
+    ("Algorithm 2: w* from f instead of 1 - f", "out->w_star = inverse_cdf(G, (1.0 - alpha) * (1.0 - f));",
+     "out->w_star = inverse_cdf(G, (1.0 - alpha) * f);"),
+    ("Eq. 5: candidate endpoints swapped", "out->candidate_winner = (sv.cd > dcd) ? 1 : (dcd > sv.cd) ? 2 : 0;",
+     "out->candidate_winner = (sv.cd > dcd) ? 2 : (dcd > sv.cd) ? 1 : 0;"),
+    ("bins: octave offset", "int64_t b = 32 * (int64_t)(e - 4) + ((t >> (e - 5)) & 31);",
+     "int64_t b = 32 * (int64_t)(e - 5) + ((t >> (e - 5)) & 31);"),
+    ("quantile: rank reached on a strict comparison", "acc += hist[b]; if (acc >= rank) return b; }",
+     "acc += hist[b]; if (acc > rank) return b; }"),
+    ("cost: exchange rate dropped",
+     "+ dv.lambda * (dv.cp * (double)R->pre_device + dv.cd * (double)R->tok_device);",
+     "+ (dv.cp * (double)R->pre_device + dv.cd * (double)R->tok_device);"),
+]
+
+
+def run(ids=None, verbose=True):
+    src = open(SRC).read()
+    survivors = []
+    with tempfile.TemporaryDirectory() as tmp:
+        for k, (what, old, new) in enumerate(MUTANTS):
+            if ids and k not in ids:
+                continue
+            if src.count(old) != 1:
+                raise SystemExit("mutant %d: its text occurs %d times in the source" % (k, src.count(old)))
+            cpp, so = os.path.join(tmp, "m%d.cpp" % k), os.path.join(tmp, "m%d.so" % k)
+            with open(cpp, "w") as f:
+                f.write(src.replace(old, new))
+            subprocess.check_call(["g++", "-std=c++17", "-O2", "-ffp-contract=off", "-fPIC", "-shared", "-w",
+                                   "-I", os.path.dirname(SRC), "-o", so, cpp])
+            env = dict(os.environ, DISCO_ORACLE_LIB=so)
+            r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(ROOT, "tests"), "-x", "-q", "-m", "not gpu",
+                                "-k", "oracle and not mutant", "-p", "no:cacheprovider"],
+                               env=env, cwd=ROOT, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)
+            killed = r.returncode != 0
+            if verbose:
+                print("%2d %-55s %s" % (k, what, "killed" if killed else "SURVIVED"))
+            if not killed:
+                survivors.append((k, what))
+    return survivors
+
+
+if __name__ == "__main__":
+    left = run([int(a) for a in sys.argv[1:]] or None)
+    sys.exit(1 if left else 0)

@@ -206,6 +206,14 @@ def test_device_resident_inputs_match_host_inputs():
         assert bytes(sa[p]) == bytes(sb[p])
 
 
+def test_quantile_rank_reached_at_a_bin_boundary():
+    # four requests alone in their TTFT bins: the nearest rank of P50 falls exactly on the end of a bin
+    tr = constructed([50, 60, 70, 80], [3, 4, 5, 6], np.array([0.008, 0.001, 0.004, 0.002], dtype=np.float32))
+    w = synth.Workload(name="rank", seed=1, materialise=True, policies=[], **tr)
+    gs, _ = full_parity(w, [synth.policy(0.0, flags=PACE | D_MODE), synth.policy(1.0, flags=PACE | S_MODE)], tag="rank")
+    assert gs[0].n_server_only == 4
+
+
 def test_pinned_host_inputs_read_in_place_match_pageable_ones():
     # one profile group: page-locked host arrays are read by the ingestion kernel in place, pageable ones are
     # copied first; both must give the same tables and statistics (and the oracle's)

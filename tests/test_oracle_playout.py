@@ -194,6 +194,7 @@ def test_migration_to_server_draws_from_the_ttft_distribution():
 
 def test_tokens_and_cost_eq8():
     w = synth.tiny_workload(4, 300, n_servers=2, n_devices=2, max_prompt=300, max_out=120)
+    w.devices[0]["lam"], w.devices[1]["lam"] = 0.5, 3.0        # Eq. 8's exchange rate, not one
     o = oracle_of(vars(w))
     pols = [synth.policy(b, flags=f) for b in (0.0, 0.3, 1.0) for f in (S_MODE | MIG | PACE, D_MODE | MIG | PACE, PACE)]
     st, out = o.eval(pols, 4, pairs=True)
@@ -211,7 +212,8 @@ def test_tokens_and_cost_eq8():
         to_srv = (mig > 0) & ~to_dev
         pre_d = pre_d + np.where(to_dev, l + mig, 0)
         pre_s = pre_s + np.where(to_srv, l + mig, 0)
-        want = cps * pre_s + cds * out["tok_server"][p] + (cpd * pre_d + cdd * out["tok_device"][p])
+        lam = np.array([d["lam"] for d in w.devices], np.float32)[w.device_profile].astype(np.float64)
+        want = cps * pre_s + cds * out["tok_server"][p] + lam * (cpd * pre_d + cdd * out["tok_device"][p])
         assert np.allclose(out["cost"][p], want, rtol=1e-12)
         assert st[p].prefill_tok_server == int(pre_s.sum()) and st[p].prefill_tok_device == int(pre_d.sum())
         assert abs(st[p].total_cost - want.sum()) < 1e-9 * want.sum()

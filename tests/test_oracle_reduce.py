@@ -45,6 +45,22 @@ def test_histogram_totals_and_exact_quantiles():
     assert st[1].exact_p99_tbt_s < 0.2
 
 
+def test_nearest_rank_at_a_bin_boundary():
+    # four requests, each alone in its TTFT bin, all served by the server (device-constrained, b = 0): rank
+    # ceil(0.5 * 4) = 2 is reached exactly at the end of the second bin, ceil(0.95 * 4) = ceil(0.99 * 4) = 4 at the last
+    from helpers import constructed
+    ttft = np.array([0.008, 0.001, 0.004, 0.002], dtype=np.float32)
+    tr = constructed([50, 60, 70, 80], [3, 4, 5, 6], ttft)
+    o = oracle_of(tr)
+    st, _ = o.eval([synth.policy(0.0, flags=synth.FLAG_PACING | synth.MODE_DEVICE_CONSTRAINED)], 1)
+    s = st[0]
+    assert s.n_server_only == 4
+    assert (s.bin_p50_ttft, s.bin_p95_ttft, s.bin_p99_ttft) == (L.orc_bin(2000), L.orc_bin(8000), L.orc_bin(8000))
+    assert s.p50_ttft_s == L.orc_bin_lower_edge(L.orc_bin(2000)) * 1e-6
+    # pooled TBTs: 3 + 4 + 5 + 2 = 14 intervals of exactly tau = 200,000 ticks
+    assert s.n_intervals == 14 and s.bin_p99_tbt == L.orc_bin(200000)
+
+
 def test_range_split_merges_exactly():
     w = synth.make_workload(1, n=2000)
     o = oracle_of(vars(w))
