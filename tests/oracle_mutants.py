@@ -56,6 +56,30 @@ MUTANTS = [
      "int64_t b = 32 * (int64_t)(e - 5) + ((t >> (e - 5)) & 31);"),
     ("quantile: rank reached on a strict comparison", "acc += hist[b]; if (acc >= rank) return b; }",
      "acc += hist[b]; if (acc > rank) return b; }"),
+    ("jitter: range 2J instead of 2J + 1", "(uint64_t)(2 * J + 1)) >> 32) - J;", "(uint64_t)(2 * J)) >> 32) - J;"),
+    ("ticks: truncated instead of rounded", "int64_t ticks_of_seconds(float s) { return llrint((double)s * 1e6); }",
+     "int64_t ticks_of_seconds(float s) { return (int64_t)((double)s * 1e6); }"),
+    ("device TTFT: intercept dropped", "const int64_t Td = dv.kappa * (int64_t)l + dv.c0;",
+     "const int64_t Td = dv.kappa * (int64_t)l;"),
+    ("Algorithm 3: threshold inclusive", "if (l < pr.l_th) device_only = true;", "if (l <= pr.l_th) device_only = true;"),
+    ("Algorithm 2: wait map, l* class gets the tail wait",
+     "else w = (l < pr.l_star) ? 0 : (l == pr.l_star) ? pr.w_star : pr.w_tail;",
+     "else w = (l < pr.l_star) ? 0 : pr.w_tail;"),
+    ("Eq. 1: immediate-start threshold exclusive", "if (pr.beta_rule) w = l <= pr.l_immediate ? 0 :",
+     "if (pr.beta_rule) w = l < pr.l_immediate ? 0 :"),
+    ("stochastic routing: endpoints swapped", "const bool to_device = pr.device_constrained ? constrained : !constrained;",
+     "const bool to_device = pr.device_constrained ? !constrained : constrained;"),
+    ("expected length: tokens already generated not subtracted",
+     "std::max<int32_t>((int32_t)pol.expected_len - m, 0) : n - m;",
+     "std::max<int32_t>((int32_t)pol.expected_len, 0) : n - m;"),
+    ("pooled TBTs: first interval left out", "for (int32_t j = 2; j <= n; ++j) {\n                const int64_t tbt = d[j] - d[j - 1];",
+     "for (int32_t j = 3; j <= n; ++j) {\n                const int64_t tbt = d[j] - d[j - 1];"),
+    ("device wins counted for device-only requests too", "st.n_device_won += (R.decision == ORC_RACE && R.winner_device);",
+     "st.n_device_won += R.winner_device;"),
+    ("selection: mean TTFT before the tail", "if (x.p99_ttft_s != y.p99_ttft_s) { if (x.p99_ttft_s < y.p99_ttft_s) b = (int32_t)p; continue; }\n        if (x.mean_ttft_s != y.mean_ttft_s) { if (x.mean_ttft_s < y.mean_ttft_s) b = (int32_t)p; continue; }",
+     "if (x.mean_ttft_s != y.mean_ttft_s) { if (x.mean_ttft_s < y.mean_ttft_s) b = (int32_t)p; continue; }\n        if (x.p99_ttft_s != y.p99_ttft_s) { if (x.p99_ttft_s < y.p99_ttft_s) b = (int32_t)p; continue; }"),
+    ("selection: TBT objective ignored", "if (!(st[p].total_cost <= cost_cap) || !(st[p].p99_tbt_s <= tbt_slo_s)) continue;",
+     "if (!(st[p].total_cost <= cost_cap)) continue;"),
     ("cost: exchange rate dropped",
      "+ dv.lambda * (dv.cp * (double)R->pre_device + dv.cd * (double)R->tok_device);",
      "+ (dv.cp * (double)R->pre_device + dv.cd * (double)R->tok_device);"),

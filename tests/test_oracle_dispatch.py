@@ -137,6 +137,34 @@ def test_algorithm2_funding_identity_and_monotone_waits():
             assert 0 <= pr.w_star <= pr.w_tail
 
 
+def test_algorithm2_wait_map_as_played():
+    # three length classes of 200 requests: every request must wait W[l] (0 below l*, w* in the partly funded class,
+    # w_tail above), i.e. the device starts exactly when the server's first token comes later than that
+    from helpers import constructed
+    rng = np.random.default_rng(12)
+    lens = np.repeat([64, 128, 256], 200)
+    ttft = rng.lognormal(-1.0, 0.6, size=600).astype(np.float32)
+    tr = constructed(lens, rng.integers(2, 40, size=600), ttft,
+                     devices=[synth.device(500.0, 20.0, c_prefill=5e-3, c_decode=5e-3)])
+    o = oracle_of(tr)
+    ticks = np.rint(ttft.astype(np.float64) * 1e6).astype(np.int64)
+    partly = 0
+    for b in (0.1, 0.3, 0.5, 0.7, 0.9):
+        pol = synth.policy(b, flags=synth.FLAG_PACING)
+        pr = o.prep(pol)
+        assert pr.device_constrained and pr.l_star in (64, 128, 256)
+        wait = np.where(lens < pr.l_star, 0, np.where(lens == pr.l_star, pr.w_star, pr.w_tail))
+        st, out = o.eval([pol], 0, pairs=True)
+        started = out["decision"][0] == RACE
+        assert (started == (ticks > wait)).all() and not (out["decision"][0] == 1).any()
+        in_class = lens == pr.l_star
+        if 0 < pr.w_star < pr.w_tail and started[in_class].any() and (~started[in_class]).any():
+            partly += 1
+            # with the tail wait instead of w*, fewer of this class would have started
+            assert (ticks[in_class] > pr.w_star).sum() > (ticks[in_class] > pr.w_tail).sum()
+    assert partly >= 3
+
+
 def test_algorithm2_realised_device_share_tracks_budget():
     # E[I_d(l) l] <= b E[l] (Sec. 4.2): statistical, since the wait is set from the trace's own TTFT quantiles
     w = synth.make_workload(1, n=40000)
