@@ -1,6 +1,8 @@
 """Mutation check of the oracle's pins: plants one plausible mistake at a time in a COPY of the oracle's source
 (a wrong comparison, index, sign, shift or a swapped endpoint), builds it, and runs the CPU pin tests against the
 broken library.  A pin set that bites fails for every mutant.  Nothing here touches the CUDA path.
+Left out because no input can tell them from the original: starting the hand-off search at j = B + 1 (at j = B the
+test reads d_1 = 0 > g_B, never true) and running it up to j = n (the saving on zero remaining tokens is zero).
 
     python tests/oracle_mutants.py            # all mutants; prints the survivors, exit status 1 if there are any
     python tests/oracle_mutants.py 3 7        # only these
@@ -80,6 +82,22 @@ MUTANTS = [
      "if (x.mean_ttft_s != y.mean_ttft_s) { if (x.mean_ttft_s < y.mean_ttft_s) b = (int32_t)p; continue; }\n        if (x.p99_ttft_s != y.p99_ttft_s) { if (x.p99_ttft_s < y.p99_ttft_s) b = (int32_t)p; continue; }"),
     ("selection: TBT objective ignored", "if (!(st[p].total_cost <= cost_cap) || !(st[p].p99_tbt_s <= tbt_slo_s)) continue;",
      "if (!(st[p].total_cost <= cost_cap)) continue;"),
+    ("hash: request and token constants swapped", "    return mix(k0 + i * C_REQ);", "    return mix(k0 + i * C_TOK);"),
+    ("Eq. 6: buffer size rounded down", "std::min<int64_t>((o->t_m + o->tau - 1) / o->tau, 1 << 30) : 0;",
+     "std::min<int64_t>(o->t_m / o->tau, 1 << 30) : 0;"),
+    ("Algorithm 1: max of the device costs", "bool device_constrained = std::min(dcp, dcd) > std::max(sv.cp, sv.cd);",
+     "bool device_constrained = std::max(dcp, dcd) > std::max(sv.cp, sv.cd);"),
+    ("Algorithm 1: exchange rate left out", "const double dcp = dv.lambda * dv.cp, dcd = dv.lambda * dv.cd;",
+     "const double dcp = dv.cp, dcd = dv.lambda * dv.cd;"),
+    ("knots: k N / 256 instead of k (N - 1) / 256", "G.sorted[(size_t)(((int64_t)k * (G.N - 1)) / 256)] : 0;",
+     "G.sorted[(size_t)std::min<int64_t>(((int64_t)k * G.N) / 256, G.N - 1)] : 0;"),
+    ("device-only requests billed a server prefill",
+     "R->decision = ORC_DEVICE_ONLY; R->server_dispatched = false; R->device_started = true;",
+     "R->decision = ORC_DEVICE_ONLY; R->server_dispatched = true; R->device_started = true;"),
+    ("hand-off search runs one token short", "for (int32_t j = pr.B; j <= n - 1; ++j) {", "for (int32_t j = pr.B; j < n - 1; ++j) {"),
+    ("migration of the cheaper winner", "const bool winner_dearer = R->winner_device ? (pr.candidate_winner == 2) : (pr.candidate_winner == 1);",
+     "const bool winner_dearer = R->winner_device ? (pr.candidate_winner == 1) : (pr.candidate_winner == 2);"),
+    ("stochastic routing: draw compared with b 2^31", "(double)u < std::floor(b * 4294967296.0);", "(double)u < std::floor(b * 2147483648.0);"),
     ("cost: exchange rate dropped",
      "+ dv.lambda * (dv.cp * (double)R->pre_device + dv.cd * (double)R->tok_device);",
      "+ (dv.cp * (double)R->pre_device + dv.cd * (double)R->tok_device);"),

@@ -206,6 +206,16 @@ def test_device_resident_inputs_match_host_inputs():
         assert bytes(sa[p]) == bytes(sb[p])
 
 
+def test_handoff_with_one_token_left():
+    # jitter-free streams that fill a buffer of five at token 6: outputs of 5 to 9 tokens, so that the hand-off
+    # falls on the last token that still leaves one to generate, or no longer fits
+    tr = constructed([100] * 5 + [400] * 5, [5, 6, 7, 8, 9] * 2, [1e-6] * 10, devices=[synth.device(200.0, 10.0)])
+    w = synth.Workload(name="last-token", seed=3, materialise=True, policies=[], **tr)
+    gs, _ = full_parity(w, [synth.policy(1.0, t_m_s=1.0, r_c=5.0, flags=MIG | PACE | S_MODE),
+                            synth.policy(1.0, t_m_s=0.0, r_c=5.0, flags=MIG | PACE | S_MODE)], tag="last-token")
+    assert gs[0].n_migrations == 6 and gs[1].n_migrations == 10
+
+
 def test_quantile_rank_reached_at_a_bin_boundary():
     # four requests alone in their TTFT bins: the nearest rank of P50 falls exactly on the end of a bin
     tr = constructed([50, 60, 70, 80], [3, 4, 5, 6], np.array([0.008, 0.001, 0.004, 0.002], dtype=np.float32))

@@ -86,6 +86,20 @@ def test_buffer_migration_worked_example():
         assert abs(out["tbt_max_s"][0, 0] - int(tbt_max) * 1e-6) < 1e-12
 
 
+def test_handoff_at_the_last_token_that_leaves_one_to_generate():
+    # the worked example's stream fills its buffer of 5 at token 6: an output of 7 tokens still hands over (one
+    # token is left for the device), an output of 6 tokens does not (nothing would remain)
+    dev = [synth.device(200.0, 10.0)]
+    pol = synth.policy(1.0, t_m_s=1.0, r_c=5.0, flags=S_MODE | MIG | PACE)
+    for n, want_m in ((8, 6), (7, 6), (6, 0), (5, 0)):
+        o = oracle_of(constructed([100], [n], [1e-6], devices=dev))
+        r = o.play(pol, 0, 0)
+        assert r["decision"] == RACE and not r["winner_is_device"]
+        assert r["mig_at"] == want_m, (n, r["mig_at"])
+        st, out = o.eval([pol], 0, pairs=True)
+        assert out["tok_server"][0, 0] == (want_m or n) and out["tok_device"][0, 0] == n - (want_m or n)
+
+
 @pytest.mark.parametrize("T,tau,t_m,T_tgt,kappa,l,n", [
     (30000, 200000, 1_000_000, 100000, 5000, 100, 50), (30000, 200000, 1_000_000, 100000, 5000, 400, 50),
     (30000, 200000, 1_000_000, 100000, 5000, 400, 12), (50000, 100000, 700_000, 20000, 2000, 300, 80),
