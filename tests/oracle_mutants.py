@@ -98,6 +98,24 @@ MUTANTS = [
     ("migration of the cheaper winner", "const bool winner_dearer = R->winner_device ? (pr.candidate_winner == 2) : (pr.candidate_winner == 1);",
      "const bool winner_dearer = R->winner_device ? (pr.candidate_winner == 1) : (pr.candidate_winner == 2);"),
     ("stochastic routing: draw compared with b 2^31", "(double)u < std::floor(b * 4294967296.0);", "(double)u < std::floor(b * 2147483648.0);"),
+    ("hash: high seed word ignored", "    uint32_t k0 = mix(lo ^ C_SEED) ^ hi;", "    uint32_t k0 = mix(lo ^ C_SEED);"),
+    ("per-request mean TBT over n instead of n - 1", "((double)(d[n] - d[1]) * 1e-6) / (double)(n - 1) : 0.0;",
+     "((double)(d[n] - d[1]) * 1e-6) / (double)(n) : 0.0;"),
+    ("device starts counted for winners only", "st.n_device_started += R.device_started;",
+     "st.n_device_started += (R.device_started && R.winner_device);"),
+    ("P95 computed at 0.90", "const double qs[3] = {0.50, 0.95, 0.99};", "const double qs[3] = {0.50, 0.90, 0.99};"),
+    ("P99 TBT over the requests instead of the intervals", "uint64_t r = (uint64_t)quantile_rank(0.99, st.n_intervals);",
+     "uint64_t r = (uint64_t)quantile_rank(0.99, st.n_requests);"),
+    ("quantile value: upper instead of lower bin edge", "*vals[k] = (double)bin_edge(*bins[k]) * 1e-6;",
+     "*vals[k] = (double)bin_edge(*bins[k] + 1) * 1e-6;"),
+    ("Eq. 1: wait not capped by the tail wait", "w = l <= pr.l_immediate ? 0 : std::min(pr.beta * (int64_t)l, pr.w_tail);",
+     "w = l <= pr.l_immediate ? 0 : pr.beta * (int64_t)l;"),
+    ("Eq. 2: slope search accepts one step too early", "if ((double)started_tokens(mid) <= limit) hi = mid; else lo = mid + 1;",
+     "if ((double)started_tokens(mid) <= limit) hi = mid; else lo = mid;\n            if (hi - lo == 1) { lo = hi - 1; break; }"),
+    ("migrated stream: late tokens counted on delivery times", "if (g[j] > d[m] + (int64_t)(j - m) * tau) ++R->delayed;",
+     "if (d[j] > d[m] + (int64_t)(j - m) * tau) ++R->delayed;"),
+    ("selection without a feasible policy: first instead of cheapest", "if (st[p].total_cost < st[c].total_cost) c = (int32_t)p;",
+     "if (false && st[p].total_cost < st[c].total_cost) c = (int32_t)p;"),
     ("cost: exchange rate dropped",
      "+ dv.lambda * (dv.cp * (double)R->pre_device + dv.cd * (double)R->tok_device);",
      "+ (dv.cp * (double)R->pre_device + dv.cd * (double)R->tok_device);"),

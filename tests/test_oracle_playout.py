@@ -86,6 +86,21 @@ def test_buffer_migration_worked_example():
         assert abs(out["tbt_max_s"][0, 0] - int(tbt_max) * 1e-6) < 1e-12
 
 
+def test_per_request_tbt_mean_and_max_at_constant_rate():
+    # no jitter, no migration: paced delivery at tau = 200,000 ticks gives every interval tau (Table 3's constant
+    # TBT); unpaced delivery gives the winner's generation interval.  The mean is over the n - 1 intervals.
+    tr = constructed([100, 100, 3000, 3000], [2, 9, 2, 33], [1e-6, 1e-6, 10.0, 10.0])   # the server wins the short prompts' race, the device (6 s) the long ones'
+    o = oracle_of(tr)
+    for flags, want in ((PACE | S_MODE, (0.2, 0.2, 0.2, 0.2)), (S_MODE, (0.03, 0.03, 0.05, 0.05))):
+        _, out = o.eval([synth.policy(1.0, flags=flags)], 0, pairs=True)
+        assert list(out["decision"][0]) == [RACE] * 4
+        assert np.allclose(out["tbt_mean_s"][0], want, rtol=0, atol=1e-12)
+        assert np.allclose(out["tbt_max_s"][0], want, rtol=0, atol=1e-12)
+    one = oracle_of(constructed([100], [1], [1e-6]))
+    _, out = one.eval([synth.policy(1.0, flags=PACE | S_MODE)], 0, pairs=True)
+    assert out["tbt_mean_s"][0, 0] == 0.0 and out["tbt_max_s"][0, 0] == 0.0      # a single token has no interval
+
+
 def test_handoff_at_the_last_token_that_leaves_one_to_generate():
     # the worked example's stream fills its buffer of 5 at token 6: an output of 7 tokens still hands over (one
     # token is left for the device), an output of 6 tokens does not (nothing would remain)
