@@ -6,6 +6,9 @@ test reads d_1 = 0 > g_B, never true) and running it up to j = n (the saving on 
 
     python tests/oracle_mutants.py            # all mutants; prints the survivors, exit status 1 if there are any
     python tests/oracle_mutants.py 3 7        # only these
+    python tests/oracle_mutants.py --gpu 3 7  # on a GPU machine: the parity tests (tests/test_gpu_parity.py) against the
+                                              # broken oracle instead of the pins; they must fail too, which shows
+                                              # that they would catch the same mistake made on the CUDA side
 """
 import os
 import subprocess
@@ -122,7 +125,7 @@ MUTANTS = [
 ]
 
 
-def run(ids=None, verbose=True):
+def run(ids=None, verbose=True, gpu=False):
     src = open(SRC).read()
     survivors = []
     with tempfile.TemporaryDirectory() as tmp:
@@ -137,8 +140,9 @@ def run(ids=None, verbose=True):
             subprocess.check_call(["g++", "-std=c++17", "-O2", "-ffp-contract=off", "-fPIC", "-shared", "-w",
                                    "-I", os.path.dirname(SRC), "-o", so, cpp])
             env = dict(os.environ, DISCO_ORACLE_LIB=so)
-            r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(ROOT, "tests"), "-x", "-q", "-m", "not gpu",
-                                "-k", "oracle and not mutant", "-p", "no:cacheprovider"],
+            select = ["-m", "gpu", os.path.join(ROOT, "tests", "test_gpu_parity.py")] if gpu else \
+                     ["-m", "not gpu", "-k", "oracle and not mutant", os.path.join(ROOT, "tests")]
+            r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider"] + select,
                                env=env, cwd=ROOT, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)
             killed = r.returncode != 0
             if verbose:
@@ -149,5 +153,6 @@ def run(ids=None, verbose=True):
 
 
 if __name__ == "__main__":
-    left = run([int(a) for a in sys.argv[1:]] or None)
+    args = [a for a in sys.argv[1:] if a != "--gpu"]
+    left = run([int(a) for a in args] or None, gpu="--gpu" in sys.argv[1:])
     sys.exit(1 if left else 0)

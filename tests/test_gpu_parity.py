@@ -206,6 +206,53 @@ def test_device_resident_inputs_match_host_inputs():
         assert bytes(sa[p]) == bytes(sb[p])
 
 
+def test_buffer_test_on_an_exact_tie():
+    # jitter-free server at T = tau / 2 with a buffer of three: d_3 = g_5 exactly, so the strict test hands over at 6
+    srv = [synth.server(tbt_s=0.050)]
+    tr = constructed([100] * 4, [5, 6, 7, 20], [1e-6] * 4, servers=srv, devices=[synth.device(200.0, 10.0)])
+    w = synth.Workload(name="tie", seed=2, materialise=True, policies=[], **tr)
+    pol = synth.policy(1.0, t_m_s=0.3, r_c=10.0, flags=MIG | PACE | S_MODE)
+    gs, _ = full_parity(w, [pol], tag="buffer-tie")
+    tr2 = Trace.from_workload(w)
+    out = tr2.alloc_pair_outputs(1, fields=["mig_at"])
+    tr2.eval_policies([pol], w.seed, out)
+    assert out["mig_at"][0].tolist() == [0, 0, 6, 6]
+    tr2.close()
+
+
+def test_selection_prefers_the_tail_over_the_mean():
+    # two policies whose order by P99 TTFT is the reverse of their order by mean TTFT
+    w = synth.make_workload(1, n=4000, n_budgets=3)
+    pols = [synth.policy(0.6, flags=PACE | S_MODE), synth.policy(0.4, flags=PACE | D_MODE)]
+    gs, _ = full_parity(w, pols, tag="tail-vs-mean")
+    assert gs[0].bin_p99_ttft < gs[1].bin_p99_ttft and gs[0].mean_ttft_s > gs[1].mean_ttft_s
+    tr = Trace.from_workload(w)
+    tr.eval_policies(pols, w.seed)
+    tr.reduce_stats()
+    assert tr.select_policy(1e30, 10.0) == (0, 0)
+    tr.close()
+
+
+def test_algorithm1_on_unequal_device_costs_and_exchange_rate():
+    # automatic mode: min(lambda c_d) against max(c_s).  Device A: prefill cheap, decode dear -> server-constrained
+    # (a max over the device costs would say otherwise); device B: cheap per unit but lambda = 3 -> device-constrained
+    devs = [synth.device(500.0, 20.0, c_prefill=0.5e-3, c_decode=3e-3, lam=1.0),
+            synth.device(500.0, 20.0, c_prefill=0.4e-3, c_decode=0.4e-3, lam=3.0)]
+    w = synth.tiny_workload(8, 1500, n_servers=1, n_devices=2, max_prompt=400, max_out=120)
+    w.devices = devs
+    pols = [synth.policy(b, flags=MIG | PACE | synth.MODE_AUTO) for b in (0.2, 0.7)]
+    full_parity(w, pols, tag="alg1-costs")
+    tr = Trace.from_workload(w)
+    tr.eval_policies(pols, w.seed)
+    assert not tr.prep(0, 0).device_constrained and tr.prep(1, 0).device_constrained
+    tr.close()
+
+
+def test_seed_above_32_bits():
+    w = synth.make_workload(1, n=3000, n_budgets=4)
+    full_parity(w, seed=0x123456789ABCDEF0, tag="seed-hi")
+
+
 def test_handoff_with_one_token_left():
     # jitter-free streams that fill a buffer of five at token 6: outputs of 5 to 9 tokens, so that the hand-off
     # falls on the last token that still leaves one to generate, or no longer fits
