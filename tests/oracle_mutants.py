@@ -119,6 +119,19 @@ MUTANTS = [
      "if (d[j] > d[m] + (int64_t)(j - m) * tau) ++R->delayed;"),
     ("selection without a feasible policy: first instead of cheapest", "if (st[p].total_cost < st[c].total_cost) c = (int32_t)p;",
      "if (false && st[p].total_cost < st[c].total_cost) c = (int32_t)p;"),
+    ("bins: linear region one too short", "    if (t < 32) return (int32_t)t;", "    if (t < 31) return (int32_t)t;"),
+    ("bins: mantissa bits taken one place off", "+ ((t >> (e - 5)) & 31);", "+ ((t >> (e - 4)) & 31);"),
+    ("groups: server and device index swapped", "const ServerTicks& sv = tr.srv[grp / tr.dev.size()];",
+     "const ServerTicks& sv = tr.srv[grp % tr.srv.size()];"),
+    ("Algorithm 2: b = alpha treated as above alpha", "    if (b <= alpha) {                 /* every length keeps the maximum wait */",
+     "    if (b < alpha) {                 /* every length keeps the maximum wait */"),
+    ("knot draw: index from the low byte", "const uint32_t k = u >> 24, fr = (u >> 8) & 0xFFFFu;",
+     "const uint32_t k = u & 0xFFu, fr = (u >> 8) & 0xFFFFu;"),
+    ("migration latency draw uses the token-1 hash", "const uint32_t u = token_hash(key, 0);\n                    const uint32_t k = u >> 24",
+     "const uint32_t u = token_hash(key, 1);\n                    const uint32_t k = u >> 24"),
+    ("target stream: first token not delayed by the hand-off", "g[m + 1] = g[m] + M;", "g[m + 1] = g[m] + Tt;"),
+    ("server-constrained race keeps a wait", "if (l < pr.l_th) device_only = true;           /* Algorithm 3: short prompts stay on the device */",
+     "if (l < pr.l_th) device_only = true; else w = 1000;"),
     ("cost: exchange rate dropped",
      "+ dv.lambda * (dv.cp * (double)R->pre_device + dv.cd * (double)R->tok_device);",
      "+ (dv.cp * (double)R->pre_device + dv.cd * (double)R->tok_device);"),

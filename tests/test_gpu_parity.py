@@ -248,6 +248,43 @@ def test_algorithm1_on_unequal_device_costs_and_exchange_rate():
     tr.close()
 
 
+def test_profile_ids_with_unequal_numbers_of_servers_and_devices():
+    # 2 server x 3 device profiles with distinct intervals and device TTFTs (group = server id * 3 + device id)
+    srv = [synth.server(tbt_s=0.030, jitter=0.2), synth.server(tbt_s=0.045, jitter=0.1)]
+    dev = [synth.device(500.0, 20.0, jitter=0.05), synth.device(250.0, 10.0, jitter=0.05, ttft_intercept_s=0.02),
+           synth.device(1000.0, 40.0, jitter=0.1, c_prefill=5e-3, c_decode=5e-3)]
+    rng = np.random.default_rng(5)
+    n = 2400
+    tr = constructed(rng.integers(1, 600, size=n), rng.integers(1, 200, size=n), rng.lognormal(-1.0, 0.8, size=n),
+                     servers=srv, devices=dev, sprof=rng.integers(0, 2, size=n), dprof=rng.integers(0, 3, size=n))
+    w = synth.Workload(name="2x3", seed=6, materialise=True, policies=[], **tr)
+    gs, _ = full_parity(w, [synth.policy(b, mig_threshold=th) for b in (0.1, 0.5, 0.9) for th in (0.0, 0.05)], tag="2x3")
+    assert any(s.n_migrations for s in gs)
+
+
+def test_bins_around_the_end_of_the_linear_region():
+    # TTFTs and inter-token intervals of 29 to 34 ticks: bins 0..31 hold one tick each, the octaves start at 32
+    srv = [synth.server(tbt_s=31e-6), synth.server(tbt_s=32e-6)]
+    ttft = np.array([29e-6, 30e-6, 31e-6, 32e-6, 33e-6, 34e-6] * 2, np.float32)
+    tr = constructed([50] * 12, [4] * 12, ttft, servers=srv, sprof=[0] * 6 + [1] * 6)
+    w = synth.Workload(name="bins", seed=1, materialise=True, policies=[], **tr)
+    gs, _ = full_parity(w, [synth.policy(0.0, flags=D_MODE), synth.policy(0.0, flags=PACE | D_MODE, r_c=1e6 / 31.0)],
+                        tag="bins-31-32")
+    assert gs[0].n_server_only == 12
+
+
+def test_budget_equal_to_the_tail_ratio():
+    # b = alpha exactly: Algorithm 2 stays in its tail-only branch (every length waits w_tail)
+    w = synth.make_workload(1, n=3000, n_budgets=2)
+    pols = [synth.policy(b, alpha=a, flags=MIG | PACE | D_MODE) for b, a in ((0.05, 0.05), (0.3, 0.3), (0.30000001, 0.3),
+                                                                            (0.31, 0.3))]
+    full_parity(w, pols, tag="b-equals-alpha")
+    tr = Trace.from_workload(w)
+    tr.eval_policies(pols, w.seed)
+    assert tr.prep(0, 0).l_star == 0 and tr.prep(0, 1).l_star == 0 and tr.prep(0, 3).l_star > 0
+    tr.close()
+
+
 def test_seed_above_32_bits():
     w = synth.make_workload(1, n=3000, n_budgets=4)
     full_parity(w, seed=0x123456789ABCDEF0, tag="seed-hi")

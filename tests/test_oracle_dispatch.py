@@ -178,6 +178,25 @@ def test_algorithm2_realised_device_share_tracks_budget():
         assert abs(share - b) < 0.02, (b, share)
 
 
+def test_profile_ids_select_their_own_endpoints():
+    # 2 server x 3 device profiles, no jitter, no pacing: a request's device TTFT and its inter-token interval are
+    # those of the profiles it names (group = server id * number of devices + device id)
+    srv = [synth.server(tbt_s=0.030), synth.server(tbt_s=0.045)]
+    dev = [synth.device(500.0, 20.0), synth.device(250.0, 10.0, ttft_intercept_s=0.02), synth.device(1000.0, 40.0)]
+    sp = np.array([0, 0, 0, 1, 1, 1] * 2, np.uint8)
+    dp = np.array([0, 1, 2, 0, 1, 2] * 2, np.uint8)
+    ttft = np.array([1e-6] * 6 + [100.0] * 6, np.float32)              # the server wins the first six races, the device the others
+    tr = constructed([100] * 12, [11] * 12, ttft, servers=srv, devices=dev, sprof=sp, dprof=dp)
+    o = oracle_of(tr)
+    _, out = o.eval([synth.policy(1.0, flags=synth.MODE_SERVER_CONSTRAINED)], 0, pairs=True)
+    kappa, c0 = np.array([2000, 4000, 1000]), np.array([0, 20000, 0])
+    T_srv, T_dev = np.array([30000, 45000]), np.array([50000, 100000, 25000])
+    assert (out["decision"][0] == RACE).all()
+    assert np.allclose(out["ttft_s"][0][6:], (kappa[dp[6:]] * 100 + c0[dp[6:]]) * 1e-6, rtol=0, atol=1e-12)
+    assert np.allclose(out["tbt_mean_s"][0][:6], T_srv[sp[:6]] * 1e-6, rtol=0, atol=1e-12)
+    assert np.allclose(out["tbt_mean_s"][0][6:], T_dev[dp[6:]] * 1e-6, rtol=0, atol=1e-12)
+
+
 def test_race_rule_and_tie():
     # device: 2000 ticks per prompt token + 10000 intercept; prompt 45 -> Td = 100000 ticks
     dev = [synth.device(500.0, 20.0, ttft_intercept_s=0.01)]
