@@ -132,6 +132,16 @@ MUTANTS = [
     ("target stream: first token not delayed by the hand-off", "g[m + 1] = g[m] + M;", "g[m + 1] = g[m] + Tt;"),
     ("server-constrained race keeps a wait", "if (l < pr.l_th) device_only = true;           /* Algorithm 3: short prompts stay on the device */",
      "if (l < pr.l_th) device_only = true; else w = 1000;"),
+    ("no buffer: hand-off after the second token", "        if (pr.B == 0) {\n            m = 1;", "        if (pr.B == 0) {\n            m = 2;"),
+    ("unpaced migrated stream delivered at the paced times", "                    d[j] = pacing ? std::max(g[j], d[j - 1] + tau) : g[j];",
+     "                    d[j] = std::max(g[j], d[j - 1] + tau);"),
+    ("late tokens counted without pacing too", "                if (pacing)\n                    for (int32_t j = m + 1; j <= n; ++j)",
+     "                if (true)\n                    for (int32_t j = m + 1; j <= n; ++j)"),
+    ("single-token outputs may hand over", "if (mig_on && R->decision == ORC_RACE && winner_dearer && n >= 2) {",
+     "if (mig_on && R->decision == ORC_RACE && winner_dearer && n >= 1) {"),
+    ("intervals counted as n instead of n - 1", "st.n_intervals += (uint64_t)(n - 1);", "st.n_intervals += (uint64_t)n;"),
+    ("device-only requests may migrate", "if (mig_on && R->decision == ORC_RACE && winner_dearer && n >= 2) {",
+     "if (mig_on && R->decision != ORC_SERVER_ONLY && winner_dearer && n >= 2) {"),
     ("cost: exchange rate dropped",
      "+ dv.lambda * (dv.cp * (double)R->pre_device + dv.cd * (double)R->tok_device);",
      "+ (dv.cp * (double)R->pre_device + dv.cd * (double)R->tok_device);"),

@@ -285,6 +285,17 @@ def test_budget_equal_to_the_tail_ratio():
     tr.close()
 
 
+def test_single_token_outputs_never_hand_over():
+    # an output of one token leaves nothing to migrate, whatever the trigger says (expected length 128, no buffer)
+    for dear in (False, True):
+        w = synth.tiny_workload(23 + dear, 1200, n_servers=2, n_devices=2, max_prompt=300, max_out=30, device_dearer=dear)
+        w.output_len[::3] = 1
+        pols = [synth.policy(b, flags=f | md, expected_len=E, t_m_s=tm) for b in (0.3, 1.0) for f in (MIG, MIG | PACE)
+                for md in (S_MODE, D_MODE) for E in (0, 128) for tm in (0.0, 1.0)]
+        gs, _ = full_parity(w, pols, tag=f"single-token dear={dear}")
+        assert any(s.n_migrations for s in gs)
+
+
 def test_seed_above_32_bits():
     w = synth.make_workload(1, n=3000, n_budgets=4)
     full_parity(w, seed=0x123456789ABCDEF0, tag="seed-hi")

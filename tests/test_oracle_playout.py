@@ -101,6 +101,31 @@ def test_per_request_tbt_mean_and_max_at_constant_rate():
     assert out["tbt_mean_s"][0, 0] == 0.0 and out["tbt_max_s"][0, 0] == 0.0      # a single token has no interval
 
 
+def test_migration_invariants_over_modes_and_flags():
+    # only a raced request with at least two tokens may hand over; without pacing there is no slot to be late for
+    # and delivery is generation, before and after a hand-off
+    for dear in (False, True):
+        w = synth.tiny_workload(23 + dear, 400, n_servers=2, n_devices=2, max_prompt=300, max_out=30, device_dearer=dear)
+        w.output_len[::7] = 1
+        o = oracle_of(vars(w))
+        pols = [synth.policy(b, flags=f | md, expected_len=E, t_m_s=tm)
+                for b in (0.0, 0.5, 1.0) for f in (MIG, MIG | PACE) for md in (S_MODE, D_MODE) for E in (0, 128)
+                for tm in (0.0, 1.0)]
+        st, out = o.eval(pols, 5, pairs=True)
+        some = 0
+        for p, pol in enumerate(pols):
+            mig = out["mig_at"][p] > 0
+            some += int(mig.sum())
+            assert (out["decision"][p][mig] == RACE).all()
+            assert not mig[w.output_len == 1].any()
+            if not pol["flags"] & PACE:
+                assert (out["delayed"][p] == 0).all() and st[p].delayed_tokens == 0
+                for i in np.flatnonzero(mig)[:5]:
+                    r = o.play(pol, 5, int(i))
+                    assert r["mig_at"] == 1 and list(r["d"][1:]) == list(r["g"][1:])
+        assert some > 100
+
+
 def test_handoff_at_the_last_token_that_leaves_one_to_generate():
     # the worked example's stream fills its buffer of 5 at token 6: an output of 7 tokens still hands over (one
     # token is left for the device), an output of 6 tokens does not (nothing would remain)
