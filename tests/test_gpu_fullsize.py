@@ -166,3 +166,22 @@ def test_pair_arrays_beyond_2_32_elements():
     # and the rows are not trivially constant: budgets 0 and 1 decide differently
     assert int(full["decision"][0].max()) == 1 and int(full["decision"][255].min()) != 1
     tr.close()
+
+
+@pytest.mark.parametrize("cfg,policy_step", [(3, 1), (4, 16)])
+def test_aggregates_on_262144_requests(cfg, policy_step):
+    # traces of 2^18 requests with the shape of workloads 3 and 4 (many chunks, several waves of blocks, six groups
+    # for workload 4): tables, every statistic and histogram against the oracle run on host threads
+    from parity import check_stats, check_tables
+    w = synth.make_workload(cfg, n=1 << 18)
+    pols = w.policies[::policy_step]
+    tr = Trace.from_workload(w)
+    orc = Oracle.from_workload(w)
+    check_tables(tr, orc, f"sub-config{cfg}")
+    tr.eval_policies(pols, w.seed)
+    gs = tr.reduce_stats()
+    ostats = _oracle_stats_threaded(orc, pols, w.seed, threads=16)
+    check_stats(gs, ostats, tr.histograms, f"sub-config{cfg}")
+    cheapest = min(s.total_cost for s in ostats)
+    assert tr.select_policy(1.25 * cheapest, 0.25) == orc.select(ostats, 1.25 * cheapest, float(np.float32(0.25)))
+    tr.close()
