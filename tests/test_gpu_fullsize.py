@@ -23,6 +23,8 @@ def _check(w, policies, ranges, tag):
     tr.eval_policies(policies, w.seed, out)
     gs = tr.reduce_stats()
     orc = Oracle.from_workload(w)
+    from parity import check_tables
+    check_tables(tr, orc, tag)             # length histograms, sorted TTFT ticks and knots at full size
     host = {f: out[f].cpu().numpy() for f in out}
     for i0, i1 in ranges:
         _, oout = orc.eval(policies, w.seed, i0, i1, pairs=True, finish=False)
