@@ -96,6 +96,11 @@ typedef struct {
                                          ingestion kernel in place when the trace has one profile group; otherwise
                                          they are copied to the device first.  Either way they may be reused as soon
                                          as disco_load_trace returns. */
+    uint64_t first_index;             /* index, in the whole trace, of request 0 of these arrays: 0 unless the arrays
+                                         are a contiguous range (a shard) of a larger trace.  The per-token jitter hash
+                                         is keyed by the request's index in the whole trace, so a shard loaded with its
+                                         first_index draws what the whole trace would draw for its rows;
+                                         first_index + n <= 2^32.  Per-pair output columns stay local (0 .. n-1). */
 } disco_trace_desc_t;
 
 /* One policy setting (Algorithm 1 inputs b, alpha; Eq. 4 overhead; Eq. 6 t_m, r_c). */
@@ -167,12 +172,19 @@ int disco_eval_policies(disco_ctx_t* ctx, const disco_policy_t* pol, uint32_t P,
  * P records to host memory `stats`.  Synchronises `stream`. */
 int disco_reduce_stats(disco_ctx_t* ctx, disco_policy_stats_t* stats, void* stream);
 
-/* Picks, among the policies of the last reduction whose total cost is within
- * cost_cap and whose P99 TBT is within tbt_slo_s, the one with the smallest
- * P99 TTFT (then mean TTFT, then cost, then index) -- the objectives of
- * Sec. 4.1.  *best (host) receives its index.  If none is feasible, returns
- * DISCO_EINFEASIBLE and *best is the cheapest policy.  Synchronises. */
-int disco_select_policy(disco_ctx_t* ctx, double cost_cap, float tbt_slo_s, int32_t* best, void* stream);
+/* Picks, among P statistics records (host memory; those of disco_reduce_stats,
+ * or records the caller merged itself), the policy whose total cost is within
+ * cost_cap and whose P99 TBT is within tbt_slo_s that has the smallest P99 TTFT
+ * (by histogram bin; then mean TTFT, then cost, then index) -- the objectives
+ * of Sec. 4.1.  *best (host) receives its index.  If none is feasible, returns
+ * DISCO_EINFEASIBLE and *best is the cheapest policy.  Runs on the host: the
+ * records are already there, so no launch and no synchronisation. */
+int disco_select_policy(const disco_policy_stats_t* stats, uint32_t P, double cost_cap, float tbt_slo_s,
+                        int32_t* best);
+
+/* The same selection by a kernel over the records the last disco_reduce_stats
+ * left in the context's device memory.  Synchronises `stream`. */
+int disco_select_policy_device(disco_ctx_t* ctx, double cost_cap, float tbt_slo_s, int32_t* best, void* stream);
 
 /* Copies policy p's TTFT and pooled TBT histograms (host, DISCO_NBINS each; either may be NULL). */
 int disco_get_histograms(disco_ctx_t* ctx, uint32_t p, uint64_t* ttft_hist, uint64_t* tbt_hist, void* stream);
@@ -182,10 +194,38 @@ int disco_get_prep(disco_ctx_t* ctx, uint32_t g, uint32_t p, disco_prep_t* out, 
 
 /* Copies group g's tables to host memory (any may be NULL): requests per prompt
  * length cnt[DISCO_MAX_PROMPT+1], the 257 equally spaced order statistics of F,
- * and up to `n_sorted` of the smallest sorted TTFT ticks.  Returns the group's
- * request count, or a negative status. */
+ * and up to `n_sorted` of the smallest sorted TTFT ticks.  Returns the number of
+ * requests behind the group's tables (the group's own requests, or what
+ * disco_set_group_tables gave), or a negative status. */
 int64_t disco_get_group_tables(disco_ctx_t* ctx, uint32_t g, int64_t* cnt, int32_t* knots,
                                int32_t* sorted_ticks, uint64_t n_sorted, void* stream);
+
+/* ---- Evaluating one trace in several contexts (request-range shards, e.g. one per GPU) -------------------
+ * Requests are independent given the tables of Algorithm 1 (p(l) and F per group), and every per-policy
+ * accumulator is an integer sum over requests.  A shard is loaded with its first_index; it is then given
+ * the tables of the WHOLE trace with disco_set_group_tables (its own tables, from disco_get_group_tables,
+ * summed / merged with the other shards' by the caller), evaluated, and its accumulators exported; the
+ * element-wise sum of all shards' accumulator words, imported into any one context, is reduced by
+ * disco_reduce_stats to exactly the records one context holding the whole trace produces. */
+
+/* Replaces the tables Algorithms 1-3 read by the caller's: cnt[G][DISCO_MAX_PROMPT+1] requests per prompt
+ * length (host memory) and, group after group, the server-TTFT ticks behind F: n_ticks[g] (host) of them for
+ * group g, in any order within the group, `ticks` in host or device memory (for instance the shards' sorted
+ * ticks one after the other).  The library sorts them per group and rebuilds the cumulative token mass
+ * (Eq. 3) and the 257 knots of F.  The context keeps its own requests.  DISCO_EINVAL if a group's length
+ * counts do not add up to n_ticks[g] or a tick is negative (the context must then be reloaded).  Lasts until
+ * the next disco_load_trace.  Synchronises `stream`. */
+int disco_set_group_tables(disco_ctx_t* ctx, const int64_t* cnt, const int32_t* ticks, const uint64_t* n_ticks,
+                           void* stream);
+
+/* The accumulators of the last evaluation as additive 64-bit words: per (policy, group) counters, the
+ * TTFT and pooled TBT histograms per policy, and per group the output tokens and requests they cover.
+ * disco_accumulator_words gives their number (0 before an evaluation); export copies them to `words`,
+ * import overwrites the context's with `words` (host or device memory; for example the sum over shards).
+ * Both synchronise `stream`.  disco_reduce_stats then works on what was imported. */
+uint64_t disco_accumulator_words(disco_ctx_t* ctx);
+int disco_export_accumulators(disco_ctx_t* ctx, uint64_t* words, void* stream);
+int disco_import_accumulators(disco_ctx_t* ctx, const uint64_t* words, void* stream);
 
 /* Measurement aids.  disco_set_timing(ctx, 1) makes each evaluation record CUDA events on its stream around
  * its four main kernels; after disco_reduce_stats, disco_get_timing fills ms4[0..3] with the device
@@ -195,6 +235,14 @@ int64_t disco_get_group_tables(disco_ctx_t* ctx, uint32_t g, int64_t* cnt, int32
 int disco_set_timing(disco_ctx_t* ctx, int on);
 int disco_get_timing(disco_ctx_t* ctx, float* ms4);
 uint64_t disco_kernel_launch_count(void);
+
+/* Measures what the GPU sustains on the integer instruction mix of the token loop (Sec. 4.3 play-out: per
+ * token one counter add, the hash finaliser's three shift-xor pairs and two multiplies, one multiply-high
+ * range map, one compare and one multiply-add into the sum = 13 lane-instructions) with every SM full of
+ * independent lanes and nothing else to do: the ceiling the play-out's roofline fraction is quoted against.
+ * Runs for a few milliseconds on `stream` and synchronises it.  lane_instr_per_s receives token-steps per
+ * second x 13; token_steps_per_s (may be NULL) the token-steps per second themselves. */
+int disco_measure_alu_peak(double* lane_instr_per_s, double* token_steps_per_s, void* stream);
 
 /* Sorting without allocating.  (The paper has no counterpart to this call; it exists for the sake of
  * callers, not of the method.)

@@ -113,6 +113,9 @@ def lib() -> C.CDLL:
         L.orc_eval.restype = C.c_int
         L.orc_eval.argtypes = [C.c_void_p, C.c_void_p, C.c_uint32, C.c_uint64, C.c_uint64, C.c_uint64,
                                C.c_void_p, C.c_void_p, C.c_int]
+        L.orc_eval_cols.restype = C.c_int
+        L.orc_eval_cols.argtypes = [C.c_void_p, C.c_void_p, C.c_uint32, C.c_uint64, C.c_uint64, C.c_uint64,
+                                    C.c_void_p, C.c_uint64, C.c_uint64, C.c_void_p, C.c_int]
         L.orc_finish.argtypes = [C.c_void_p, C.c_uint32]
         L.orc_select.restype = C.c_int
         L.orc_select.argtypes = [C.c_void_p, C.c_uint32, C.c_double, C.c_double, C.c_void_p]
@@ -237,6 +240,25 @@ class Oracle:
         if finish:
             self.L.orc_finish(C.cast(stats, C.c_void_p), P)
         return stats, out
+
+    def eval_columns(self, policies: Sequence[Dict[str, float]], seed: int, ranges):
+        """Per-pair results of the requests in `ranges` (a list of (i0, i1)) only: a dict of arrays [P, K], K the
+        total length of the ranges, columns in the order of the ranges.  Memory is O(P K), whatever the trace's
+        size."""
+        P = len(policies)
+        K = sum(i1 - i0 for i0, i1 in ranges)
+        arr = _policies(policies)
+        out = {name: np.zeros((P, K), dtype=dt) for name, dt in _PAIR_FIELDS}
+        stats = (OracleStats * P)()
+        col = 0
+        for i0, i1 in ranges:
+            po = pair_out_struct(*[out[name].ctypes.data + col * out[name].itemsize for name, _ in _PAIR_FIELDS])
+            rc = self.L.orc_eval_cols(self.h, C.cast(arr, C.c_void_p), P, seed, i0, i1, C.byref(po), K, i0,
+                                      C.cast(stats, C.c_void_p), 0)
+            if rc != 0:
+                raise ValueError(self.L.orc_last_error().decode())
+            col += i1 - i0
+        return out
 
     def finish(self, stats):
         self.L.orc_finish(C.cast(stats, C.c_void_p), len(stats))

@@ -464,7 +464,14 @@ int orc_play(const orc_trace_t* t, const orc_policy_t* pol, uint64_t seed, uint6
 
 int orc_eval(const orc_trace_t* t, const orc_policy_t* pols, uint32_t P, uint64_t seed, uint64_t i0, uint64_t i1,
              const orc_pair_out_t* out, orc_stats_t* stats, int want_exact) {
+    return orc_eval_cols(t, pols, P, seed, i0, i1, out, t ? t->n : 0, 0, stats, want_exact);
+}
+
+int orc_eval_cols(const orc_trace_t* t, const orc_policy_t* pols, uint32_t P, uint64_t seed, uint64_t i0, uint64_t i1,
+                  const orc_pair_out_t* out, uint64_t out_stride, uint64_t out_first, orc_stats_t* stats,
+                  int want_exact) {
     if (!t || !pols || !stats || i0 > i1 || i1 > t->n) return fail("bad argument");
+    if (out && (out_first > i0 || i1 - out_first > out_stride)) return fail("per-pair columns do not cover the range");
     const orc_trace& tr = *t;
     std::vector<int64_t> g(ORC_MAX_OUTPUT + 2), d(ORC_MAX_OUTPUT + 2);
     std::vector<orc_prep_t> prep(tr.groups.size());
@@ -502,7 +509,7 @@ int orc_eval(const orc_trace_t* t, const orc_policy_t* pols, uint32_t P, uint64_
             st.prefill_tok_server += (uint64_t)R.pre_server; st.prefill_tok_device += (uint64_t)R.pre_device;
             st.delayed_tokens += (uint64_t)R.delayed;
             if (out) {
-                const size_t o = (size_t)p * tr.n + i;
+                const size_t o = (size_t)p * out_stride + (size_t)(i - out_first);   /* row p, column of request i */
                 if (out->ttft_s) out->ttft_s[o] = ttft_s;
                 if (out->tbt_mean_s) out->tbt_mean_s[o] = tbt_mean_s;
                 if (out->tbt_max_s) out->tbt_max_s[o] = (double)tbt_max * 1e-6;

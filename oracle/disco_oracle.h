@@ -109,6 +109,11 @@ int orc_play(const orc_trace_t*, const orc_policy_t* pol, uint64_t seed, uint64_
  * out may be NULL.  want_exact != 0 also sorts this call's TTFTs and TBTs. */
 int orc_eval(const orc_trace_t*, const orc_policy_t* pol, uint32_t P, uint64_t seed,
              uint64_t i0, uint64_t i1, const orc_pair_out_t* out, orc_stats_t* stats, int want_exact);
+/* The same with compact per-pair arrays: row p holds out_stride entries, request i goes to column
+ * i - out_first (orc_eval: out_stride = n, out_first = 0). */
+int orc_eval_cols(const orc_trace_t*, const orc_policy_t* pol, uint32_t P, uint64_t seed,
+                  uint64_t i0, uint64_t i1, const orc_pair_out_t* out, uint64_t out_stride, uint64_t out_first,
+                  orc_stats_t* stats, int want_exact);
 void orc_finish(orc_stats_t* stats, uint32_t P);
 
 int orc_select(const orc_stats_t* stats, uint32_t P, double cost_cap, double tbt_slo_s, int32_t* best);

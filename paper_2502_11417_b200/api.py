@@ -39,7 +39,7 @@ class TraceDesc(C.Structure):
     _fields_ = [("n", C.c_uint64), ("prompt_len", C.c_void_p), ("output_len", C.c_void_p),
                 ("server_ttft_s", C.c_void_p), ("server_profile", C.c_void_p), ("device_profile", C.c_void_p),
                 ("servers", C.c_void_p), ("n_servers", C.c_uint32), ("devices", C.c_void_p),
-                ("n_devices", C.c_uint32), ("arrays_on_device", C.c_uint32)]
+                ("n_devices", C.c_uint32), ("arrays_on_device", C.c_uint32), ("first_index", C.c_uint64)]
 
 
 class Policy(C.Structure):
@@ -75,7 +75,10 @@ class Prep(C.Structure):
 
 EXPORTS = ["disco_load_trace", "disco_eval_policies", "disco_reduce_stats", "disco_select_policy",
            "disco_get_histograms", "disco_get_prep", "disco_get_group_tables", "disco_free_trace",
-           "disco_last_error", "disco_set_timing", "disco_get_timing", "disco_kernel_launch_count", "disco_sort_ttft_ticks_noalloc"]
+           "disco_last_error", "disco_set_timing", "disco_get_timing", "disco_kernel_launch_count",
+           "disco_sort_ttft_ticks_noalloc", "disco_select_policy_device", "disco_set_group_tables",
+           "disco_accumulator_words", "disco_export_accumulators", "disco_import_accumulators",
+           "disco_measure_alu_peak"]
 
 PAIR_FIELDS = [("ttft_s", "float32"), ("tbt_mean_s", "float32"), ("tbt_max_s", "float32"), ("cost", "float32"),
                ("tok_server", "uint32"), ("tok_device", "uint32"), ("mig_at", "uint32"), ("delayed", "uint16"),
@@ -99,7 +102,15 @@ def lib() -> C.CDLL:
         L.disco_eval_policies.restype = C.c_int; L.disco_eval_policies.argtypes = [vp, vp, u32, u64, vp, vp]
         L.disco_reduce_stats.restype = C.c_int; L.disco_reduce_stats.argtypes = [vp, vp, vp]
         L.disco_select_policy.restype = C.c_int
-        L.disco_select_policy.argtypes = [vp, C.c_double, C.c_float, C.POINTER(C.c_int32), vp]
+        L.disco_select_policy.argtypes = [vp, u32, C.c_double, C.c_float, C.POINTER(C.c_int32)]
+        L.disco_select_policy_device.restype = C.c_int
+        L.disco_select_policy_device.argtypes = [vp, C.c_double, C.c_float, C.POINTER(C.c_int32), vp]
+        L.disco_set_group_tables.restype = C.c_int; L.disco_set_group_tables.argtypes = [vp, vp, vp, vp, vp]
+        L.disco_accumulator_words.restype = u64; L.disco_accumulator_words.argtypes = [vp]
+        L.disco_export_accumulators.restype = C.c_int; L.disco_export_accumulators.argtypes = [vp, vp, vp]
+        L.disco_import_accumulators.restype = C.c_int; L.disco_import_accumulators.argtypes = [vp, vp, vp]
+        L.disco_measure_alu_peak.restype = C.c_int
+        L.disco_measure_alu_peak.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_double), vp]
         L.disco_get_histograms.restype = C.c_int; L.disco_get_histograms.argtypes = [vp, u32, vp, vp, vp]
         L.disco_get_prep.restype = C.c_int; L.disco_get_prep.argtypes = [vp, u32, u32, vp, vp]
         L.disco_get_group_tables.restype = C.c_int64
@@ -185,6 +196,24 @@ def policy_array(policies: Sequence[Dict[str, float]]):
     return arr
 
 
+def select_policy(stats, cost_cap: float, tbt_slo_s: float):
+    """disco_select_policy over a (PolicyStats * P) array in host memory (the records of reduce_stats, or
+    merged ones).  Returns (status, index): status 0, or EINFEASIBLE with the cheapest policy's index."""
+    best = C.c_int32(-1)
+    rc = _check(lib().disco_select_policy(C.cast(stats, C.c_void_p), len(stats), cost_cap, tbt_slo_s, C.byref(best)),
+                allow=(EINFEASIBLE,))
+    return rc, best.value
+
+
+def measure_alu_peak(stream=None):
+    """disco_measure_alu_peak: (lane-instructions/s, token-steps/s) the GPU sustains on the token loop's
+    instruction mix."""
+    _require_cuda()
+    a, b = C.c_double(0.0), C.c_double(0.0)
+    _check(lib().disco_measure_alu_peak(C.byref(a), C.byref(b), _stream_ptr(stream)))
+    return a.value, b.value
+
+
 NOALLOC_MAX_N = 262144
 
 
@@ -217,9 +246,10 @@ class Trace:
 
     # -- disco_load_trace ---------------------------------------------------------------------------------
     def load_trace(self, prompt_len, output_len, server_ttft_s, server_profile, device_profile, servers, devices,
-                   stream=None):
+                   stream=None, first_index: int = 0):
         """Arrays may be numpy arrays / pinned CPU tensors (host memory) or CUDA tensors (device memory),
-        all of the same kind.  Reloading reuses the context's device memory."""
+        all of the same kind.  Reloading reuses the context's device memory.  first_index: position of these
+        arrays' first request in the whole trace when they are a shard of it."""
         import torch
         _require_cuda()
         arrs = [prompt_len, output_len, server_ttft_s, server_profile, device_profile]
@@ -248,7 +278,7 @@ class Trace:
         n = int(len(prompt_len))
         sv, dv = server_array(servers), device_array(devices)
         desc = TraceDesc(n, ptrs[0], ptrs[1], ptrs[2], ptrs[3], ptrs[4], C.cast(sv, C.c_void_p), len(servers),
-                         C.cast(dv, C.c_void_p), len(devices), 1 if on_dev else 0)
+                         C.cast(dv, C.c_void_p), len(devices), 1 if on_dev else 0, int(first_index))
         _check(lib().disco_load_trace(C.byref(self._h), C.byref(desc), _stream_ptr(stream)))
         self.n = n
         self.n_groups = len(servers) * len(devices)
@@ -295,11 +325,61 @@ class Trace:
 
     # -- disco_select_policy -------------------------------------------------------------------------------
     def select_policy(self, cost_cap: float, tbt_slo_s: float, stream=None):
-        """Returns (status, index): status 0, or EINFEASIBLE with the cheapest policy's index."""
+        """disco_select_policy_device: the selection by a kernel over the records of the last reduce_stats.
+        Returns (status, index): status 0, or EINFEASIBLE with the cheapest policy's index."""
         best = C.c_int32(-1)
-        rc = _check(lib().disco_select_policy(self._h, cost_cap, tbt_slo_s, C.byref(best), _stream_ptr(stream)),
-                    allow=(EINFEASIBLE,))
+        rc = _check(lib().disco_select_policy_device(self._h, cost_cap, tbt_slo_s, C.byref(best),
+                                                     _stream_ptr(stream)), allow=(EINFEASIBLE,))
         return rc, best.value
+
+    # -- shards of one trace ---------------------------------------------------------------------------------
+    def set_group_tables(self, cnt, ticks, n_ticks, stream=None):
+        """disco_set_group_tables: cnt int64 [G, 4097] and n_ticks uint64 [G] as numpy arrays; ticks int32, the
+        groups one after the other in any order within a group, a numpy array or a CUDA tensor."""
+        cnt = np.ascontiguousarray(cnt, dtype=np.int64)
+        ns = np.ascontiguousarray(n_ticks, dtype=np.uint64)
+        if isinstance(ticks, np.ndarray):
+            ticks = np.ascontiguousarray(ticks, dtype=np.int32)
+            ptr, size = ticks.ctypes.data, ticks.size
+        else:
+            if ticks.dtype != _torch_dtype("int32") or not ticks.is_contiguous():
+                raise TypeError("ticks must be a contiguous int32 tensor")
+            ptr, size = ticks.data_ptr(), ticks.numel()
+        if cnt.shape != (self.n_groups, 4097) or ns.shape != (self.n_groups,) or size != int(ns.sum()):
+            raise ValueError("cnt must be [G, 4097], n_ticks [G], ticks of their total length")
+        _check(lib().disco_set_group_tables(self._h, cnt.ctypes.data, ptr if size else None, ns.ctypes.data,
+                                            _stream_ptr(stream)))
+        return self
+
+    def accumulator_words(self) -> int:
+        return int(lib().disco_accumulator_words(self._h))
+
+    def export_accumulators(self, out=None, stream=None):
+        """The additive accumulator words of the last evaluation: a numpy uint64 array (host), or written into
+        `out`, a CUDA int64 / numpy uint64 buffer of accumulator_words() elements."""
+        k = self.accumulator_words()
+        if out is None:
+            out = np.zeros(k, dtype=np.uint64)
+        if isinstance(out, np.ndarray):
+            ptr, size, width = out.ctypes.data, out.size, out.dtype.itemsize
+        else:
+            ptr, size, width = out.data_ptr(), out.numel(), out.element_size()
+        if size != k or width != 8:
+            raise ValueError("accumulator buffer must hold accumulator_words() 64-bit words")
+        _check(lib().disco_export_accumulators(self._h, ptr, _stream_ptr(stream)))
+        return out
+
+    def import_accumulators(self, words, stream=None):
+        k = self.accumulator_words()
+        if isinstance(words, np.ndarray):
+            words = np.ascontiguousarray(words, dtype=np.uint64)
+            ptr, size = words.ctypes.data, words.size
+        else:
+            ptr, size = words.data_ptr(), words.numel()
+        if size != k:
+            raise ValueError("accumulator buffer must hold accumulator_words() 64-bit words")
+        _check(lib().disco_import_accumulators(self._h, ptr, _stream_ptr(stream)))
+        return self
 
     # -- inspection ----------------------------------------------------------------------------------------
     def histograms(self, p: int, stream=None):

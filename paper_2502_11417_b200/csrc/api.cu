@@ -67,6 +67,17 @@ struct disco_ctx {
     DevBuf keys_a, keys_b, tmp_idx;
     DevBuf S, l, nout, orig, sorted;
     DevBuf zero, cum_mass, ng_exact, grp_off, knots, d_gc;   // `zero`: every table a load must clear, contiguous
+    DevBuf fin_totals;                 // [2G] u64: output tokens and requests per group that the accumulators cover
+    uint64_t first_index = 0;          // index of request 0 in the whole trace (hash key base)
+    int sms = 0;                       // multiprocessors of the context's device
+    // F as Algorithms 1-3 read it: the trace's own sorted ticks, or a whole trace's given by the caller
+    DevBuf F_sorted_imp, F_off_imp;
+    const int32_t* F_sorted = nullptr;
+    const uint32_t* F_off = nullptr;
+    bool tables_imported = false;
+    std::vector<uint64_t> F_n;         // requests per group behind F (the group's own count unless imported)
+    bool fin_imported = false;         // fin_totals holds a caller's merged totals, not this trace's
+    std::vector<uint64_t> fin_own;     // this trace's totals, to put back before the next evaluation
     uint32_t *cnt = nullptr, *ng = nullptr, *max_n = nullptr, *radix_counts = nullptr;
     uint64_t* grp_sum_n = nullptr;
     int32_t* err = nullptr;
@@ -94,7 +105,8 @@ struct disco_ctx {
 
     ~disco_ctx() {
         DevBuf* all[] = {&in_prompt, &in_out, &in_ttft, &in_sp, &in_dp, &keys_a, &keys_b, &tmp_idx,
-                         &S, &l, &nout, &orig, &sorted, &zero, &cum_mass, &ng_exact, &grp_off, &knots, &d_gc, &d_prep, &d_accum, &d_stats, &d_tables, &d_todo};
+                         &S, &l, &nout, &orig, &sorted, &zero, &cum_mass, &ng_exact, &grp_off, &knots, &d_gc, &d_prep, &d_accum, &d_stats, &d_tables, &d_todo,
+                         &fin_totals, &F_sorted_imp, &F_off_imp};
         for (DevBuf* b : all) b->release();
         for (auto& b : rec_u32) b.release();
         for (auto& b : rec_u16) b.release();
@@ -175,6 +187,7 @@ cudaError_t reserve_trace(disco_ctx* c, uint32_t n, bool host_inputs, bool has_s
     R(cum_mass, (size_t)G * (kMaxPrompt + 2) * 8); R(ng_exact, kMaxGroups * 4);
     R(grp_off, (kMaxGroups + 1) * 4); R(knots, (size_t)G * kNKnots * 4);
     R(d_gc, (size_t)G * sizeof(GroupConst));
+    R(fin_totals, (size_t)2 * kMaxGroups * 8);
 #undef R
     return cudaSuccess;
 }
@@ -192,6 +205,7 @@ int disco_load_trace(disco_ctx_t** pctx, const disco_trace_desc_t* d, void* stre
     if (d->n >= (1ull << 31)) return fail(DISCO_EINVAL, "too many requests");
     if (d->n && (!d->prompt_len || !d->output_len || !d->server_ttft_s)) return fail(DISCO_EINVAL, "null trace array");
     if (d->arrays_on_device > 1) return fail(DISCO_EINVAL, "arrays_on_device must be 0 or 1");
+    if (d->first_index + d->n > (1ull << 32)) return fail(DISCO_EINVAL, "first_index + n exceeds 2^32");
     std::vector<GroupConst> gc;
     if (int rc = check_profiles(d, &gc)) return rc;
     cudaStream_t st = (cudaStream_t)stream;
@@ -205,6 +219,15 @@ int disco_load_trace(disco_ctx_t** pctx, const disco_trace_desc_t* d, void* stre
     auto bail = [&](int rc) { if (fresh) delete c; else c->loaded = false; return rc; };
     c->loaded = c->evaluated = c->reduced = false;
     c->n = (uint32_t)d->n; c->ns = d->n_servers; c->nd = d->n_devices; c->G = (int)gc.size(); c->gc = gc;
+    c->first_index = d->first_index;
+    c->tables_imported = false;
+    c->fin_imported = false;
+    if (!c->sms) {
+        int dev = 0;
+        cudaError_t e0 = cudaGetDevice(&dev);
+        if (e0 == cudaSuccess) e0 = cudaDeviceGetAttribute(&c->sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e0 != cudaSuccess || c->sms < 1) return bail(fail_cuda(e0, "multiprocessor count of the current device"));
+    }
     const uint32_t n = c->n;
     bool host_in = d->arrays_on_device == 0;
     cudaError_t e;
@@ -256,6 +279,7 @@ int disco_load_trace(disco_ctx_t** pctx, const disco_trace_desc_t* d, void* stre
     a.sorted = c->sorted.as<int32_t>(); a.cnt = c->cnt; a.cum_mass = c->cum_mass.as<int64_t>();
     a.ng = c->ng; a.grp_off = c->grp_off.as<uint32_t>(); a.knots = c->knots.as<int32_t>();
     a.grp_sum_n = c->grp_sum_n; a.max_n = c->max_n; a.err = c->err;
+    a.fin_totals = c->fin_totals.as<uint64_t>(); a.sms = c->sms;
     // the profile table is read from pageable memory: this copy returns once it has been staged
     const bool same_profiles = c->gc_dev_at == c->d_gc.p && c->gc_dev.size() == c->gc.size() &&
                                std::memcmp(c->gc_dev.data(), c->gc.data(), c->gc.size() * sizeof(GroupConst)) == 0;
@@ -275,6 +299,8 @@ int disco_load_trace(disco_ctx_t** pctx, const disco_trace_desc_t* d, void* stre
                                      "server TTFT not finite, not positive or above 2000 s", "profile id out of range"};
         return bail(fail(DISCO_EINVAL, std::string(what[rb->err[0]]) + " at request " + std::to_string(rb->err[1])));
     }
+    c->F_sorted = c->sorted.as<int32_t>(); c->F_off = c->grp_off.as<uint32_t>();
+    c->F_n.assign(rb->ng, rb->ng + c->G);
     c->loaded = true;
     *pctx = c;
     return 0;
@@ -381,6 +407,12 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
     for (int k = 0; k < 2; ++k) R(rec_u16[k], N1 * 2);
     for (int k = 0; k < 3; ++k) R(rec_win[k], N1 * wmax[k] * 4);
 
+    if (c->fin_imported) {            // an import replaced the totals the final reductions refer to: back to the trace's own
+        c->fin_own.assign((size_t)2 * G, 0);
+        for (int g = 0; g < G; ++g) { c->fin_own[g] = rb.grp_sum_n[g]; c->fin_own[G + g] = rb.ng[g]; }
+        CU(cudaMemcpyAsync(c->fin_totals.p, c->fin_own.data(), c->fin_own.size() * 8, cudaMemcpyHostToDevice, st));
+        c->fin_imported = false;
+    }
     // the accumulators are cleared while the host lays out the chunks and tables below
     CU(cudaMemsetAsync(c->d_accum.p, 0, acc_bytes + 2 * hist_bytes + cnt_bytes, st));
 
@@ -394,14 +426,15 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
         cls_range.push_back({b, (uint32_t)pol_list.size()});
     }
     const uint32_t tiles = (P + 31) / 32;
-    uint32_t want_chunks = std::max<uint32_t>(1, 148 / std::min<uint32_t>(tiles, 148));   // one block per SM
+    const uint32_t sms = (uint32_t)c->sms;
+    uint32_t want_chunks = std::max<uint32_t>(1, sms / std::min<uint32_t>(tiles, sms));   // one block per SM
     const uint32_t min_chunks = (uint32_t)((N1 + 65279) / 65280);
     if (min_chunks > want_chunks) {
         // several waves of blocks: pick the chunk count near the minimum whose last wave is fullest
         double best = 0.0;
-        for (uint32_t k = min_chunks; k < min_chunks + 148; ++k) {
-            const uint64_t blocks = (uint64_t)k * tiles, waves = (blocks + 147) / 148;
-            const double fill = (double)blocks / (double)(waves * 148);
+        for (uint32_t k = min_chunks; k < min_chunks + sms; ++k) {
+            const uint64_t blocks = (uint64_t)k * tiles, waves = (blocks + sms - 1) / sms;
+            const double fill = (double)blocks / (double)(waves * sms);
             if (fill > best + 1e-9) { best = fill; want_chunks = k; }
         }
     }
@@ -449,10 +482,10 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
 
     // ---- Algorithms 1-3 for every (group, policy)
     CU(launch_prep(c->d_pol.as<PolicyConst>(), P, G, c->d_gc.as<GroupConst>(), c->cum_mass.as<int64_t>(),
-                   c->cnt, c->sorted.as<int32_t>(), c->grp_off.as<uint32_t>(), c->d_prep.as<Prep>(), st));
+                   c->cnt, c->F_sorted, c->F_off, c->d_prep.as<Prep>(), st));
     if (any_beta) {
-        CU(launch_prep_beta(c->d_pol.as<PolicyConst>(), P, G, c->cum_mass.as<int64_t>(), c->cnt, c->sorted.as<int32_t>(),
-                            c->grp_off.as<uint32_t>(), c->d_prep.as<Prep>(), st));
+        CU(launch_prep_beta(c->d_pol.as<PolicyConst>(), P, G, c->cum_mass.as<int64_t>(), c->cnt, c->F_sorted,
+                            c->F_off, c->d_prep.as<Prep>(), st));
         g_launches += 1;
     }
 
@@ -473,6 +506,8 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
     uint64_t out_tokens = 0;
     for (int g = 0; g < G; ++g) out_tokens += rb.grp_sum_n[g];
     const bool long_outputs = out_tokens >= 512ull * n;
+    // the hash is keyed by the request's index in the whole trace: key = mix(k0 + (first_index + i) * C_REQ)
+    const uint32_t k0 = seed_key(seed) + (uint32_t)c->first_index * kHashReq;
     // ---- per timeline class: play every request out, then evaluate the class's policies on the summaries
     g_launches += 1;
     c->timing_valid = false;
@@ -485,14 +520,14 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
         for (int g = 0; g < G; ++g)
             never_clamps = never_clamps && (int64_t)c->gc[g].T_srv + c->gc[g].J_srv <= classes[k].tau &&
                            (int64_t)c->gc[g].T_dev + c->gc[g].J_dev <= classes[k].tau;
-        CU(launch_timeline(tr, c->d_gc.as<GroupConst>(), dcc, classes[k].pacing != 0, c->knots.as<int32_t>(), seed, rec,
+        CU(launch_timeline(tr, c->d_gc.as<GroupConst>(), dcc, classes[k].pacing != 0, c->knots.as<int32_t>(), k0, rec,
                            c->err, c->d_todo.as<uint32_t>(), todo_counts + 2 * k, never_clamps, long_outputs,
-                           timed ? c->ev[1] : nullptr, st));
+                           timed ? c->ev[1] : nullptr, c->sms, st));
         if (timed) CU(cudaEventRecord(c->ev[2], st));
         CU(launch_pairs(tr, c->d_gc.as<GroupConst>(), dcc, c->d_prep.as<Prep>(), P,
                         c->d_pol_list.as<uint32_t>() + cls_range[k].first, cls_range[k].second - cls_range[k].first,
                         c->d_chunks.as<Chunk>(), (uint32_t)chunks.size(), rec, po, c->d_acc.as<uint64_t>(),
-                        c->d_hist_ttft.as<uint64_t>(), c->d_hist_tbt.as<uint64_t>(), seed, cls_extras_pending,
+                        c->d_hist_ttft.as<uint64_t>(), c->d_hist_tbt.as<uint64_t>(), k0, cls_extras_pending,
                         classes[k].W[0] > 1 || classes[k].W[1] > 1 || classes[k].W[2] > 1,
                         timed ? c->ev[3] : nullptr, st));
         if (timed) CU(cudaEventRecord(c->ev[4], st));
@@ -517,7 +552,7 @@ int disco_reduce_stats(disco_ctx_t* c, disco_policy_stats_t* stats, void* stream
         c->stats_host_cap = bytes;
     }
     CU(launch_finalize(c->P, c->G, c->d_gc.as<GroupConst>(), c->d_acc.as<uint64_t>(), c->d_hist_ttft.as<uint64_t>(),
-                       c->d_hist_tbt.as<uint64_t>(), c->grp_sum_n, c->grp_off.as<uint32_t>(),
+                       c->d_hist_tbt.as<uint64_t>(), c->fin_totals.as<uint64_t>(),
                        c->d_stats.as<disco_policy_stats_t>(), (disco_policy_stats_t*)c->stats_host, c->err, st));
     CU(cudaStreamSynchronize(st));
     std::memcpy(stats, c->stats_host, c->P * sizeof(disco_policy_stats_t));
@@ -531,7 +566,40 @@ int disco_reduce_stats(disco_ctx_t* c, disco_policy_stats_t* stats, void* stream
     return 0;
 }
 
-int disco_select_policy(disco_ctx_t* c, double cost_cap, float tbt_slo_s, int32_t* best, void* stream) {
+int disco_select_policy(const disco_policy_stats_t* stats, uint32_t P, double cost_cap, float tbt_slo_s,
+                        int32_t* best) {
+    if (!stats || !best || P == 0) return fail(DISCO_EINVAL, "null argument or P = 0");
+    if (P > (1u << 19)) return fail(DISCO_EINVAL, "too many policies");
+    // lexicographic objective: feasible first; then (P99 TTFT bin, mean TTFT, cost, index); none feasible: cheapest
+    const double slo = (double)tbt_slo_s;
+    int64_t pick = -1;
+    bool pick_ok = false;
+    for (uint32_t p = 0; p < P; ++p) {
+        const disco_policy_stats_t& s = stats[p];
+        if (s.bin_p99_tbt < 0 || s.bin_p99_tbt >= kNBins || s.bin_p99_ttft < 0 || s.bin_p99_ttft >= kNBins)
+            return fail(DISCO_EINVAL, "histogram bin out of range (policy " + std::to_string(p) + ")");
+        const bool ok = s.total_cost <= cost_cap && (double)host_bin_edge_ticks(s.bin_p99_tbt) * 1e-6 <= slo;
+        bool take;
+        if (pick < 0) take = true;
+        else if (ok != pick_ok) take = ok;
+        else {
+            const disco_policy_stats_t& b = stats[pick];
+            if (ok) {
+                if (s.bin_p99_ttft != b.bin_p99_ttft) take = s.bin_p99_ttft < b.bin_p99_ttft;
+                else if (s.mean_ttft_s != b.mean_ttft_s) take = s.mean_ttft_s < b.mean_ttft_s;
+                else take = s.total_cost < b.total_cost;
+            } else {
+                take = s.total_cost < b.total_cost;
+            }
+        }
+        if (take) { pick = p; pick_ok = ok; }
+    }
+    *best = (int32_t)pick;
+    if (!pick_ok) return fail(DISCO_EINFEASIBLE, "no policy meets the cost cap and the TBT objective");
+    return 0;
+}
+
+int disco_select_policy_device(disco_ctx_t* c, double cost_cap, float tbt_slo_s, int32_t* best, void* stream) {
     if (!c || !best) return fail(DISCO_EINVAL, "null argument");
     if (!c->reduced) return fail(DISCO_EINVAL, "reduce the statistics before selecting");
     cudaStream_t st = (cudaStream_t)stream;
@@ -587,7 +655,10 @@ int64_t disco_get_group_tables(disco_ctx_t* c, uint32_t g, int64_t* cnt, int32_t
                                uint64_t n_sorted, void* stream) {
     if (!c || !c->loaded || g >= (uint32_t)c->G) return fail(DISCO_EINVAL, "bad argument");
     cudaStream_t st = (cudaStream_t)stream;
-    const uint32_t ng = c->rb->ng[g], off = c->rb->grp_off[g];
+    // the tables Algorithms 1-3 read: the trace's own, or the whole trace's a caller has set
+    const uint64_t ng = c->F_n[g];
+    uint64_t off = c->rb->grp_off[g];
+    if (c->tables_imported) { off = 0; for (uint32_t k = 0; k < g; ++k) off += c->F_n[k]; }
     if (cnt) {
         std::vector<uint32_t> tmp(kMaxPrompt + 1);
         CU(cudaMemcpyAsync(tmp.data(), c->cnt + (size_t)g * (kMaxPrompt + 1), tmp.size() * 4, cudaMemcpyDeviceToHost, st));
@@ -596,9 +667,113 @@ int64_t disco_get_group_tables(disco_ctx_t* c, uint32_t g, int64_t* cnt, int32_t
     }
     if (knots) CU(cudaMemcpyAsync(knots, c->knots.as<int32_t>() + (size_t)g * kNKnots, kNKnots * 4, cudaMemcpyDeviceToHost, st));
     const uint64_t k = std::min<uint64_t>(n_sorted, ng);
-    if (sorted_ticks && k) CU(cudaMemcpyAsync(sorted_ticks, c->sorted.as<int32_t>() + off, k * 4, cudaMemcpyDeviceToHost, st));
+    if (sorted_ticks && k) CU(cudaMemcpyAsync(sorted_ticks, c->F_sorted + off, k * 4, cudaMemcpyDeviceToHost, st));
     CU(cudaStreamSynchronize(st));
     return (int64_t)ng;
+}
+
+int disco_set_group_tables(disco_ctx_t* c, const int64_t* cnt, const int32_t* ticks, const uint64_t* n_ticks,
+                           void* stream) {
+    if (!c || !cnt || !n_ticks) return fail(DISCO_EINVAL, "null argument");
+    if (!c->loaded) return fail(DISCO_EINVAL, "no trace loaded");
+    cudaStream_t st = (cudaStream_t)stream;
+    const int G = c->G;
+    const size_t L = kMaxPrompt + 1;
+    uint64_t total = 0;
+    std::vector<uint32_t> off(G + 1, 0), cnt32((size_t)G * L);
+    for (int g = 0; g < G; ++g) {
+        uint64_t by_length = 0;
+        for (size_t l = 0; l < L; ++l) {
+            const int64_t v = cnt[(size_t)g * L + l];
+            if (v < 0 || v > 0xFFFFFFFFll || (l == 0 && v != 0))
+                return fail(DISCO_EINVAL, "length count negative, above 2^32 - 1 or at length 0 (group " + std::to_string(g) + ")");
+            by_length += (uint64_t)v;
+            cnt32[(size_t)g * L + l] = (uint32_t)v;
+        }
+        if (by_length != n_ticks[g])
+            return fail(DISCO_EINVAL, "length counts do not add up to the number of TTFT ticks (group " + std::to_string(g) + ")");
+        total += n_ticks[g];
+        if (total > 0xFFFFFFFFull) return fail(DISCO_EINVAL, "more than 2^32 - 1 requests behind the tables");
+        off[g + 1] = (uint32_t)total;
+    }
+    if (total && !ticks) return fail(DISCO_EINVAL, "null argument");
+    cudaError_t e;
+    const size_t T1 = (size_t)std::max<uint64_t>(total, 1);
+    // the sort's scratch: the key buffers of the load (free between loads), grown if the whole trace is larger
+    if ((e = c->F_sorted_imp.reserve(T1 * 4)) != cudaSuccess || (e = c->F_off_imp.reserve((size_t)(kMaxGroups + 1) * 4)) != cudaSuccess ||
+        (e = c->keys_a.reserve(T1 * 8)) != cudaSuccess || (e = c->keys_b.reserve(T1 * 8)) != cudaSuccess ||
+        (e = c->tmp_idx.reserve(T1 * 4)) != cudaSuccess)
+        return fail_cuda(e, "device allocation for the tables");
+    CU(cudaMemsetAsync(c->err, 0, 16, st));
+    if (total) CU(cudaMemcpyAsync(c->tmp_idx.p, ticks, (size_t)total * 4, cudaMemcpyDefault, st));
+    CU(cudaMemcpyAsync(c->F_off_imp.p, off.data(), (size_t)(G + 1) * 4, cudaMemcpyHostToDevice, st));
+    CU(cudaMemcpyAsync(c->cnt, cnt32.data(), cnt32.size() * 4, cudaMemcpyHostToDevice, st));
+    uint32_t* counts = c->radix_counts + (size_t)4 * 256u * kRadixMaxBlocks;
+    CU(sort_grouped_ticks(c->tmp_idx.as<int32_t>(), c->F_off_imp.as<uint32_t>(), G, (uint32_t)total, c->keys_a.as<uint64_t>(),
+                          c->keys_b.as<uint64_t>(), counts, c->err, c->F_sorted_imp.as<int32_t>(), c->sms, st));
+    CU(launch_tables_imported(G, c->cnt, c->cum_mass.as<int64_t>(), c->ng_exact.as<uint32_t>(),
+                              c->F_sorted_imp.as<int32_t>(), c->F_off_imp.as<uint32_t>(), c->knots.as<int32_t>(), st));
+    if (total) g_launches += 2 + 3 * (G > 1 ? 5 : 4);
+    g_launches += 1;
+    // error word and each group's largest tick (the largest hand-off latency a draw from F can give)
+    int32_t err_host[4] = {0, 0, 0, 0};
+    std::vector<int32_t> top(G, 0);
+    CU(cudaMemcpyAsync(err_host, c->err, 16, cudaMemcpyDeviceToHost, st));
+    for (int g = 0; g < G; ++g)
+        if (n_ticks[g]) CU(cudaMemcpyAsync(&top[g], c->F_sorted_imp.as<int32_t>() + off[g + 1] - 1, 4, cudaMemcpyDeviceToHost, st));
+    CU(cudaStreamSynchronize(st));          // the host vectors above are read by the copies until here
+    c->evaluated = c->reduced = false;
+    if (err_host[0]) {
+        c->loaded = false;                  // the length counts have been overwritten: the context must be reloaded
+        return fail(DISCO_EINVAL, "negative TTFT tick at position " + std::to_string(err_host[1]) + "; reload the trace");
+    }
+    c->F_sorted = c->F_sorted_imp.as<int32_t>(); c->F_off = c->F_off_imp.as<uint32_t>();
+    c->tables_imported = true;
+    for (int g = 0; g < G; ++g) { c->F_n[g] = n_ticks[g]; c->rb->knot_max[g] = top[g]; }
+    return 0;
+}
+
+uint64_t disco_accumulator_words(disco_ctx_t* c) {
+    if (!c || !c->evaluated) return 0;
+    return (uint64_t)c->P * c->G * kNAcc + 2ull * c->P * kNBins + 2ull * c->G;
+}
+
+int disco_export_accumulators(disco_ctx_t* c, uint64_t* words, void* stream) {
+    if (!c || !words) return fail(DISCO_EINVAL, "null argument");
+    if (!c->evaluated) return fail(DISCO_EINVAL, "no evaluation to export");
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t head = (size_t)c->P * c->G * kNAcc + 2 * (size_t)c->P * kNBins;      // one block of d_accum
+    CU(cudaMemcpyAsync(words, c->d_accum.p, head * 8, cudaMemcpyDefault, st));
+    CU(cudaMemcpyAsync(words + head, c->fin_totals.p, (size_t)2 * c->G * 8, cudaMemcpyDefault, st));
+    CU(cudaStreamSynchronize(st));
+    return 0;
+}
+
+int disco_import_accumulators(disco_ctx_t* c, const uint64_t* words, void* stream) {
+    if (!c || !words) return fail(DISCO_EINVAL, "null argument");
+    if (!c->evaluated) return fail(DISCO_EINVAL, "evaluate the policies first: the accumulators take their shape from it");
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t head = (size_t)c->P * c->G * kNAcc + 2 * (size_t)c->P * kNBins;
+    CU(cudaMemcpyAsync(c->d_accum.p, words, head * 8, cudaMemcpyDefault, st));
+    CU(cudaMemcpyAsync(c->fin_totals.p, words + head, (size_t)2 * c->G * 8, cudaMemcpyDefault, st));
+    CU(cudaStreamSynchronize(st));
+    c->reduced = false;
+    c->timing_valid = false;
+    c->fin_imported = true;
+    return 0;
+}
+
+int disco_measure_alu_peak(double* lane_instr_per_s, double* token_steps_per_s, void* stream) {
+    if (!lane_instr_per_s) return fail(DISCO_EINVAL, "null argument");
+    int dev = 0, sms = 0;
+    CU(cudaGetDevice(&dev));
+    CU(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    double rate = 0.0;
+    CU(run_alu_peak(sms, &rate, (cudaStream_t)stream));
+    g_launches += 3;
+    *lane_instr_per_s = rate * 13.0;
+    if (token_steps_per_s) *token_steps_per_s = rate;
+    return 0;
 }
 
 }  // extern "C"

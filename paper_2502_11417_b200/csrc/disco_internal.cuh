@@ -121,6 +121,11 @@ inline int host_bin_of_ticks(int64_t t) {
     return (int)(b < kNBins - 1 ? b : kNBins - 1);
 }
 
+// Lower edge of a bin, ticks.
+inline int64_t host_bin_edge_ticks(int b) {
+    return b < 32 ? (int64_t)b : (int64_t)(32 + (b & 31)) << ((b >> 5) - 1);
+}
+
 #ifdef __CUDACC__
 // Launch that lets the grid be scheduled while its predecessor in the stream is still draining (programmatic
 // stream serialisation).  Every kernel launched this way calls grid_dependency_wait() before it reads or
@@ -149,25 +154,37 @@ cudaError_t launch_prep(const PolicyConst* pol, uint32_t P, int G, const GroupCo
 cudaError_t launch_prep_beta(const PolicyConst* pol, uint32_t P, int G, const int64_t* cum_mass, const uint32_t* cnt,
                              const int32_t* sorted, const uint32_t* grp_off, Prep* prep, cudaStream_t st);
 cudaError_t launch_timeline(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, bool pacing,
-                            const int32_t* knots, uint64_t seed, TimelineRec rec, int32_t* err, uint32_t* todo,
+                            const int32_t* knots, uint32_t k0 /* hash key base: seed_key(seed) + first_index * kHashReq */,
+                            TimelineRec rec, int32_t* err, uint32_t* todo,
                             uint32_t* todo_count /* two words, zero on entry: length of the list, batch tickets */,
                             bool never_clamps /* pacing on and tau >= T + J for both endpoints of every group */,
                             bool long_outputs /* mean output length of 512 tokens or more */,
                             cudaEvent_t mid /* recorded between its two kernels, or null */,
-                            cudaStream_t st);
+                            int sms /* multiprocessors of the device */, cudaStream_t st);
 cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const Prep* prep, uint32_t P,
                          const uint32_t* pol_list, uint32_t n_list, const Chunk* chunks, uint32_t n_chunks,
                          TimelineRec rec, disco_pair_out_t out, uint64_t* acc, uint64_t* hist_ttft,
-                         uint64_t* hist_tbt, uint64_t seed, bool extras /* some policy routes at random or uses an
+                         uint64_t* hist_tbt, uint32_t k0, bool extras /* some policy routes at random or uses an
                          expected length */, bool wide /* some window W of the class spans several bins */,
                          cudaEvent_t mid /* recorded between its two kernels, or null */,
                          cudaStream_t st);
 cudaError_t launch_finalize(uint32_t P, int G, const GroupConst* gc, const uint64_t* acc, const uint64_t* hist_ttft,
-                            const uint64_t* hist_tbt, const uint64_t* grp_sum_n, const uint32_t* grp_off,
+                            const uint64_t* hist_tbt,
+                            const uint64_t* fin_totals /* [2G]: output tokens per group, then requests per group */,
                             disco_policy_stats_t* stats /* [P] + 16 bytes */,
                             disco_policy_stats_t* stats_host /* pinned host mirror of the same size, written by the kernel */,
                             const int32_t* err, cudaStream_t st);
 cudaError_t launch_select(const disco_policy_stats_t* stats, uint32_t P, double cost_cap, float tbt_slo_s,
                           int32_t* result /* [2]: status, index; may be pinned host memory */, cudaStream_t st);
+// Cumulative token mass and knots from tables given by the caller (F_off[g] .. F_off[g+1] delimit group g's ticks).
+cudaError_t launch_tables_imported(int G, const uint32_t* cnt, int64_t* cum_mass, uint32_t* ng_exact,
+                                   const int32_t* F_sorted, const uint32_t* F_off, int32_t* knots, cudaStream_t st);
+// Sorts ticks stored group after group (off[g] .. off[g+1], device memory) ascending within each group into `out`;
+// keys_a / keys_b: scratch of `total` 64-bit words each, counts: 256 * 1024 + 256 words; err[0..1]: set to (3, index) on
+// a negative tick.  Launches 2 + 3 * (G > 1 ? 5 : 4) kernels.
+cudaError_t sort_grouped_ticks(const int32_t* ticks, const uint32_t* off, int G, uint32_t total, uint64_t* keys_a,
+                               uint64_t* keys_b, uint32_t* counts, int32_t* err, int32_t* out, int sms, cudaStream_t st);
+// Times the token loop's instruction mix on every multiprocessor; *token_steps_per_s receives the rate.
+cudaError_t run_alu_peak(int sms, double* token_steps_per_s, cudaStream_t st);
 
 }  // namespace disco

@@ -278,6 +278,7 @@ __device__ __forceinline__ void group_knots(int G, const uint32_t* __restrict__ 
                                             uint32_t* __restrict__ grp_off, int32_t* __restrict__ knots,
                                             const int32_t* __restrict__ err, const uint32_t* __restrict__ max_n,
                                             const unsigned long long* __restrict__ grp_sum_n,
+                                            unsigned long long* __restrict__ fin_totals,
                                             LoadReadback* __restrict__ rb) {
     __shared__ uint32_t off[kMaxGroups + 1];
     const int g = blockIdx.x;
@@ -293,6 +294,7 @@ __device__ __forceinline__ void group_knots(int G, const uint32_t* __restrict__ 
     if (threadIdx.x == 0) {
         rb->knot_max[g] = N ? sorted[off[g] + N - 1] : 0;
         rb->ng[g] = N; rb->grp_sum_n[g] = grp_sum_n[g];
+        fin_totals[g] = grp_sum_n[g]; fin_totals[G + g] = N;      // what the final reductions' totals refer to
         if (g == 0) {
             for (int k = 0; k <= G; ++k) { grp_off[k] = off[k]; rb->grp_off[k] = off[k]; }
             for (int k = 0; k < 4; ++k) rb->err[k] = err[k];
@@ -306,16 +308,29 @@ __global__ void __launch_bounds__(1024)
 k_group_tables(int G, const uint32_t* __restrict__ cnt, int64_t* __restrict__ cum, uint32_t* __restrict__ ng_exact,
                const uint32_t* __restrict__ ng, const int32_t* __restrict__ sorted, uint32_t* __restrict__ grp_off,
                int32_t* __restrict__ knots, const int32_t* __restrict__ err, const uint32_t* __restrict__ max_n,
-               const unsigned long long* __restrict__ grp_sum_n, LoadReadback* __restrict__ rb) {
+               const unsigned long long* __restrict__ grp_sum_n, unsigned long long* __restrict__ fin_totals,
+               LoadReadback* __restrict__ rb) {
     grid_dependency_wait();
-    group_knots(G, ng, sorted, grp_off, knots, err, max_n, grp_sum_n, rb);
+    group_knots(G, ng, sorted, grp_off, knots, err, max_n, grp_sum_n, fin_totals, rb);
     group_mass(cnt, cum, ng_exact);
 }
 
-int grid_for(uint32_t n, int threads) {
+// The same tables from a length histogram and a sorted sample given by the caller (a whole trace's, of which
+// the context holds a shard): one block of 1024 threads per group.
+__global__ void __launch_bounds__(1024)
+k_tables_imported(const uint32_t* __restrict__ cnt, int64_t* __restrict__ cum, uint32_t* __restrict__ ng_exact,
+                  const int32_t* __restrict__ F_sorted, const uint32_t* __restrict__ F_off, int32_t* __restrict__ knots) {
+    const int g = blockIdx.x;
+    const uint32_t off = F_off[g], N = F_off[g + 1] - off;
+    for (int k = threadIdx.x; k < kNKnots; k += blockDim.x)
+        knots[g * kNKnots + k] = N ? F_sorted[off + (uint32_t)(((uint64_t)k * (N - 1)) / 256u)] : 0;
+    group_mass(cnt, cum, ng_exact);
+}
+
+int grid_for(uint32_t n, int threads, int sms) {
     long long b = ((long long)n + threads - 1) / threads;
     if (b < 1) b = 1;
-    if (b > 148 * 16) b = 148 * 16;
+    if (b > (long long)sms * 16) b = (long long)sms * 16;
     return (int)b;
 }
 
@@ -359,14 +374,14 @@ cudaError_t run_load(const LoadArgs& a, cudaStream_t st) {
     if (n) {
         uint32_t* counts_a = a.radix_counts;                                   // small path: pass p uses slice p
         uint32_t* counts_b = a.radix_counts + (size_t)4 * 256u * kRadixMaxBlocks;  // large path: one scanned buffer
-        k_ingest<<<std::min(grid_for(n, 4 * kIngestThreads), 296), kIngestThreads, 0, st>>>(
+        k_ingest<<<std::min(grid_for(n, 4 * kIngestThreads, a.sms), 2 * a.sms), kIngestThreads, 0, st>>>(
             n, a.prompt, a.outlen, a.ttft, a.sp, a.dp, a.ns, a.nd, a.keys_a, a.cnt,
             (unsigned long long*)a.grp_sum_n, a.ng, a.max_n, a.err,
             G == 1 ? a.S : nullptr, a.l, a.nout, a.orig, small ? counts_a : nullptr, per_block, blocks);
         if (G > 1) {
             // internal request order: stable partition by group
             if ((e = radix_pass(a.keys_a, a.keys_b, nullptr, a.tmp_idx, n, 32, counts_b, st))) return e;
-            k_gather<<<grid_for(n, 256), 256, 0, st>>>(n, a.tmp_idx, a.keys_a, a.prompt, a.outlen, a.S, a.l, a.nout, a.orig);
+            k_gather<<<grid_for(n, 256, a.sms), 256, 0, st>>>(n, a.tmp_idx, a.keys_a, a.prompt, a.outlen, a.S, a.l, a.nout, a.orig);
         }
         // sort (group, ticks): four byte passes over the ticks, one over the group id
         uint64_t *src = a.keys_a, *dst = a.keys_b;
@@ -397,11 +412,48 @@ cudaError_t run_load(const LoadArgs& a, cudaStream_t st) {
                 if ((e = radix_pass(src, dst, nullptr, nullptr, n, 8 * p, counts_b, st))) return e;
                 uint64_t* t = src; src = dst; dst = t;
             }
-            k_low_words<<<grid_for(n, 256), 256, 0, st>>>(n, src, a.sorted);
+            k_low_words<<<grid_for(n, 256, a.sms), 256, 0, st>>>(n, src, a.sorted);
         }
     }
     if ((e = launch_after(k_group_tables, G, 1024, 0, st, G, a.cnt, a.cum_mass, a.ng_exact, a.ng, a.sorted, a.grp_off,
-                          a.knots, a.err, a.max_n, (const unsigned long long*)a.grp_sum_n, a.readback))) return e;
+                          a.knots, a.err, a.max_n, (const unsigned long long*)a.grp_sum_n,
+                          (unsigned long long*)a.fin_totals, a.readback))) return e;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_tables_imported(int G, const uint32_t* cnt, int64_t* cum_mass, uint32_t* ng_exact,
+                                   const int32_t* F_sorted, const uint32_t* F_off, int32_t* knots, cudaStream_t st) {
+    k_tables_imported<<<G, 1024, 0, st>>>(cnt, cum_mass, ng_exact, F_sorted, F_off, knots);
+    return cudaGetLastError();
+}
+
+namespace {
+// Sort keys (group << 32 | ticks) for ticks stored group after group; a negative tick sets the error word.
+__global__ void k_keys_of_grouped_ticks(uint32_t total, const int32_t* __restrict__ ticks, const uint32_t* __restrict__ off,
+                                        int G, uint64_t* __restrict__ keys, int32_t* __restrict__ err) {
+    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+        int g = 0;
+        while (g + 1 < G && i >= off[g + 1]) ++g;
+        const int32_t t = ticks[i];
+        if (t < 0 && atomicCAS(&err[0], 0, 3) == 0) err[1] = (int32_t)i;
+        keys[i] = ((uint64_t)(uint32_t)g << 32) | (uint32_t)max(t, 0);
+    }
+}
+}  // namespace
+
+cudaError_t sort_grouped_ticks(const int32_t* ticks, const uint32_t* off, int G, uint32_t total, uint64_t* keys_a,
+                               uint64_t* keys_b, uint32_t* counts, int32_t* err, int32_t* out, int sms, cudaStream_t st) {
+    if (total == 0) return cudaSuccess;
+    cudaError_t e;
+    k_keys_of_grouped_ticks<<<grid_for(total, 256, sms), 256, 0, st>>>(total, ticks, off, G, keys_a, err);
+    if ((e = cudaGetLastError())) return e;
+    uint64_t *src = keys_a, *dst = keys_b;
+    const int passes = G > 1 ? 5 : 4;                   // the ticks' four bytes, then the group id
+    for (int p = 0; p < passes; ++p) {
+        if ((e = radix_pass(src, dst, nullptr, nullptr, total, 8 * p, counts, st))) return e;
+        uint64_t* t = src; src = dst; dst = t;
+    }
+    k_low_words<<<grid_for(total, 256, sms), 256, 0, st>>>(total, src, out);
     return cudaGetLastError();
 }
 
@@ -439,6 +491,7 @@ __global__ void k_ttft_keys(uint32_t n, const float* __restrict__ ttft, uint64_t
 
 std::mutex g_na_mutex;
 unsigned char* g_na_base[64] = {};        // device address of the scratch array, per device ordinal
+int g_na_sms[64] = {};                    // multiprocessors, per device ordinal
 
 }  // namespace
 }  // namespace disco
@@ -457,14 +510,20 @@ extern "C" int disco_sort_ttft_ticks_noalloc(const float* server_ttft_s, uint32_
     if (e != cudaSuccess) return set_error(DISCO_ECUDA, cudaGetErrorString(e));
     if (dev < 0 || dev >= 64) return set_error(DISCO_EINVAL, "device ordinal above 63");
     unsigned char* base;
+    int sms;
     {
         // In host code the array's name is only a handle; its address on the current device has to be asked for.
         std::lock_guard<std::mutex> lock(g_na_mutex);
         if (!g_na_base[dev]) {
+            int count = 0;
+            if ((e = cudaDeviceGetAttribute(&count, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess || count < 1)
+                return set_error(DISCO_ECUDA, "cannot read the multiprocessor count of the current device");
             e = cudaGetSymbolAddress((void**)&g_na_base[dev], g_noalloc_scratch);
             if (e != cudaSuccess) { g_na_base[dev] = nullptr; return set_error(DISCO_ECUDA, cudaGetErrorString(e)); }
+            g_na_sms[dev] = count;
         }
         base = g_na_base[dev];
+        sms = g_na_sms[dev];
     }
     uint64_t* keys_a = (uint64_t*)base;
     uint64_t* keys_b = (uint64_t*)(base + kNaKeysBytes);
@@ -473,18 +532,24 @@ extern "C" int disco_sort_ttft_ticks_noalloc(const float* server_ttft_s, uint32_
     // the array still holds the previous call's data: the error word must start at zero; keys and counters
     // are fully rewritten for the first n entries before they are read
     if ((e = cudaMemsetAsync(err, 0, 16, st)) != cudaSuccess) return set_error(DISCO_ECUDA, cudaGetErrorString(e));
-    k_ttft_keys<<<grid_for(n, 256), 256, 0, st>>>(n, server_ttft_s, keys_a, err);
+    // Once a kernel has been queued the shared array is in use: every way out below, failures included, first
+    // waits for the stream, so that a caller who retries cannot overlap kernels still writing the array.
+    auto fail_after_launch = [&](cudaError_t err_code) {
+        cudaStreamSynchronize(st);
+        return set_error(DISCO_ECUDA, cudaGetErrorString(err_code));
+    };
+    k_ttft_keys<<<grid_for(n, 256, sms), 256, 0, st>>>(n, server_ttft_s, keys_a, err);
+    if ((e = cudaGetLastError()) != cudaSuccess) return fail_after_launch(e);
     uint64_t *src = keys_a, *dst = keys_b;
     for (int p = 0; p < 4; ++p) {
-        if ((e = radix_pass(src, dst, nullptr, nullptr, n, 8 * p, counts, st)) != cudaSuccess)
-            return set_error(DISCO_ECUDA, cudaGetErrorString(e));
+        if ((e = radix_pass(src, dst, nullptr, nullptr, n, 8 * p, counts, st)) != cudaSuccess) return fail_after_launch(e);
         uint64_t* t = src; src = dst; dst = t;
     }
-    k_low_words<<<grid_for(n, 256), 256, 0, st>>>(n, src, sorted_ticks);
+    k_low_words<<<grid_for(n, 256, sms), 256, 0, st>>>(n, src, sorted_ticks);
+    if ((e = cudaGetLastError()) != cudaSuccess) return fail_after_launch(e);
     int32_t h_err[2] = {0, 0};
-    if ((e = cudaMemcpyAsync(h_err, err, sizeof h_err, cudaMemcpyDeviceToHost, st)) != cudaSuccess ||
-        (e = cudaStreamSynchronize(st)) != cudaSuccess)
-        return set_error(DISCO_ECUDA, cudaGetErrorString(e));
+    if ((e = cudaMemcpyAsync(h_err, err, sizeof h_err, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return fail_after_launch(e);
+    if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return set_error(DISCO_ECUDA, cudaGetErrorString(e));
     if (h_err[0]) return set_error(DISCO_EINVAL, "server TTFT not finite, not positive or above 2000 s");
     return 0;
 }

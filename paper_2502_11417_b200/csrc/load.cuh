@@ -39,6 +39,8 @@ struct LoadArgs {
     uint64_t* grp_sum_n;                  // [kMaxGroups] output tokens per group
     uint32_t* max_n;                      // longest output
     int32_t* err;                         // [4]: code, request index, window flag
+    uint64_t* fin_totals;                 // [2G]: output tokens per group, then requests per group
+    int sms;                              // multiprocessors of the device (grid sizing)
 };
 
 cudaError_t run_load(const LoadArgs& a, cudaStream_t st);

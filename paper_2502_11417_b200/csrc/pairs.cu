@@ -48,7 +48,7 @@ __device__ __forceinline__ PairOut decide(const PairIn& q, const Prep& pr, uint3
             o.dev_only = pr.device_constrained ? constrained : !constrained;
             w = 0xFFFFFFFFu;                                                       // otherwise the device never starts
         }
-        if (pr.beta_rule)                                                          // Eq. 1: min(beta l, w_tail) above l_immediate
+        else if (pr.beta_rule)                                                     // Eq. 1: min(beta l, w_tail) above l_immediate
             w = (int32_t)q.l <= pr.l_star ? 0u : (uint32_t)min((unsigned long long)(uint32_t)pr.w_star * q.l,
                                                                (unsigned long long)(uint32_t)pr.w_tail);
         if (pr.expected_len) saving = q.delta_c * (float)max((int32_t)pr.expected_len - (int32_t)q.m, 0);
@@ -537,13 +537,12 @@ k_pairs_rows(TraceDev tr, const GroupConst* __restrict__ gcs, const Prep* __rest
 cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const Prep* prep, uint32_t P,
                          const uint32_t* pol_list, uint32_t n_list, const Chunk* chunks, uint32_t n_chunks,
                          TimelineRec rec, disco_pair_out_t out, uint64_t* acc, uint64_t* hist_ttft,
-                         uint64_t* hist_tbt, uint64_t seed, bool extras, bool wide, cudaEvent_t mid, cudaStream_t st) {
+                         uint64_t* hist_tbt, uint32_t k0, bool extras, bool wide, cudaEvent_t mid, cudaStream_t st) {
     if (n_chunks == 0 || n_list == 0) return mid ? cudaEventRecord(mid, st) : cudaSuccess;
     int PL = 1;
     while (PL < 32 && (uint32_t)PL < n_list) PL <<= 1;
     auto* acc_kernel = extras ? (wide ? k_pairs_acc<true, true> : k_pairs_acc<true, false>)
                               : (wide ? k_pairs_acc<false, true> : k_pairs_acc<false, false>);
-    const uint32_t k0 = seed_key(seed);
     cudaError_t e = cudaFuncSetAttribute(acc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)acc_smem_bytes(32));
     if (e) return e;

@@ -509,28 +509,29 @@ k_playout(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __r
 }  // namespace
 
 cudaError_t launch_playout_fast(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const int32_t* knots,
-                                uint64_t seed, TimelineRec rec, uint32_t* todo, uint32_t* todo_count, bool never_clamps,
-                                bool long_outputs, cudaStream_t st);
+                                uint32_t k0, TimelineRec rec, uint32_t* todo, uint32_t* todo_count, bool never_clamps,
+                                bool long_outputs, int sms, cudaStream_t st);
 
 // pacing: with the delivery buffer on, the clamp-free kernel plays every request it can and lists the rest
 // in todo[0 .. *todo_count) (todo_count must be zero on entry); the general kernel then plays the list.
 cudaError_t launch_timeline(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, bool pacing,
-                            const int32_t* knots, uint64_t seed, TimelineRec rec, int32_t* err, uint32_t* todo,
-                            uint32_t* todo_count, bool never_clamps, bool long_outputs, cudaEvent_t mid, cudaStream_t st) {
+                            const int32_t* knots, uint32_t k0, TimelineRec rec, int32_t* err, uint32_t* todo,
+                            uint32_t* todo_count, bool never_clamps, bool long_outputs, cudaEvent_t mid, int sms,
+                            cudaStream_t st) {
     if (tr.n == 0) return cudaSuccess;
     const uint32_t per_block = kWarps * 32;
     if (!pacing) {
         if (mid) { cudaError_t e0 = cudaEventRecord(mid, st); if (e0) return e0; }
-        const uint32_t blocks = std::min<uint32_t>((tr.n + per_block - 1) / per_block, 148u * 16u);
-        return launch_after(k_playout, blocks, kWarps * 32, 0, st, tr, gc, cc, knots, seed_key(seed), rec, err, nullptr,
+        const uint32_t blocks = std::min<uint32_t>((tr.n + per_block - 1) / per_block, (uint32_t)sms * 16u);
+        return launch_after(k_playout, blocks, kWarps * 32, 0, st, tr, gc, cc, knots, k0, rec, err, nullptr,
                             nullptr, tr.n);
     }
-    cudaError_t e = launch_playout_fast(tr, gc, cc, knots, seed, rec, todo, todo_count, never_clamps, long_outputs, st);
+    cudaError_t e = launch_playout_fast(tr, gc, cc, knots, k0, rec, todo, todo_count, never_clamps, long_outputs, sms, st);
     if (e) return e;
     if (mid && (e = cudaEventRecord(mid, st))) return e;
     if (never_clamps) return cudaSuccess;             // no interval can exceed tau: the list stays empty
-    const uint32_t blocks = std::min<uint32_t>((tr.n + per_block - 1) / per_block, 148u * 2u);
-    return launch_after(k_playout, blocks, kWarps * 32, 0, st, tr, gc, cc, knots, seed_key(seed), rec, err, todo, todo_count,
+    const uint32_t blocks = std::min<uint32_t>((tr.n + per_block - 1) / per_block, (uint32_t)sms * 2u);
+    return launch_after(k_playout, blocks, kWarps * 32, 0, st, tr, gc, cc, knots, k0, rec, err, todo, todo_count,
                         0u);
 }
 

@@ -285,20 +285,20 @@ k_playout_fast(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst
 }  // namespace
 
 cudaError_t launch_playout_fast(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const int32_t* knots,
-                                uint64_t seed, TimelineRec rec, uint32_t* todo, uint32_t* todo_count,
-                                bool never_clamps, bool long_outputs, cudaStream_t st) {
+                                uint32_t k0, TimelineRec rec, uint32_t* todo, uint32_t* todo_count,
+                                bool never_clamps, bool long_outputs, int sms, cudaStream_t st) {
     if (tr.n == 0) return cudaSuccess;
     // requests per ticket: small batches spread the end of the launch evenly; large traces amortise the ticket
     int rpw = 8;
-    while (rpw < 32 && (uint64_t)tr.n / (2 * rpw) >= 148u * 48u * 4u) rpw *= 2;
+    while (rpw < 32 && (uint64_t)tr.n / (2 * rpw) >= (uint64_t)sms * 48u * 4u) rpw *= 2;
     const uint32_t per_block = kFastWarps * (uint32_t)rpw;
     // requests per round: eight halve the cost of a round per request; with long outputs the token loop is
     // what counts, and four requests split the lanes more evenly
     auto* kernel = never_clamps ? (long_outputs ? k_playout_fast<true, 4> : k_playout_fast<true, 8>)
                                 : (long_outputs ? k_playout_fast<false, 4> : k_playout_fast<false, 8>);
     // as many blocks as the GPU holds at once (at most six of these per SM); the ticket counter feeds them
-    const uint32_t blocks = std::min<uint32_t>((tr.n + per_block - 1) / per_block, 148u * 6u);
-    return launch_after(kernel, blocks, kFastWarps * 32, 0, st, tr, gc, cc, knots, seed_key(seed), rec, todo, todo_count,
+    const uint32_t blocks = std::min<uint32_t>((tr.n + per_block - 1) / per_block, (uint32_t)sms * 6u);
+    return launch_after(kernel, blocks, kFastWarps * 32, 0, st, tr, gc, cc, knots, k0, rec, todo, todo_count,
                         todo_count + 1, rpw, 1u);
 }
 

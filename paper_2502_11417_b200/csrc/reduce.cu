@@ -53,7 +53,7 @@ __device__ void warp_quantile_bins(const unsigned long long* hist, unsigned long
 __global__ void k_finalize(uint32_t P, int G, const GroupConst* __restrict__ gc,
                            const unsigned long long* __restrict__ acc, const unsigned long long* __restrict__ hist_ttft,
                            const unsigned long long* __restrict__ hist_tbt,
-                           const unsigned long long* __restrict__ grp_sum_n, const uint32_t* __restrict__ grp_off,
+                           const unsigned long long* __restrict__ fin_totals,
                            disco_policy_stats_t* __restrict__ stats, disco_policy_stats_t* __restrict__ stats_host,
                            const int32_t* __restrict__ err) {
     // stats_host: the caller's pinned mirror, written straight from here (no copy operation behind the kernel)
@@ -65,7 +65,11 @@ __global__ void k_finalize(uint32_t P, int G, const GroupConst* __restrict__ gc,
     }
     __shared__ unsigned long long tot[kNAcc];
     __shared__ int qb[4];
-    const unsigned long long N = grp_off[G];
+    // fin_totals: output tokens and requests per group behind the accumulators (this trace's, or what a caller
+    // merged from several shards)
+    const unsigned long long* grp_sum_n = fin_totals;
+    unsigned long long N = 0;
+    for (int g = 0; g < G; ++g) N += fin_totals[G + g];
     if (threadIdx.x < kNAcc) {
         unsigned long long s = 0;
         for (int g = 0; g < G; ++g) s += acc[((size_t)p * G + g) * kNAcc + threadIdx.x];
@@ -158,12 +162,12 @@ __global__ void k_select(const disco_policy_stats_t* __restrict__ stats, uint32_
 }  // namespace
 
 cudaError_t launch_finalize(uint32_t P, int G, const GroupConst* gc, const uint64_t* acc, const uint64_t* hist_ttft,
-                            const uint64_t* hist_tbt, const uint64_t* grp_sum_n, const uint32_t* grp_off,
+                            const uint64_t* hist_tbt, const uint64_t* fin_totals,
                             disco_policy_stats_t* stats, disco_policy_stats_t* stats_host, const int32_t* err,
                             cudaStream_t st) {
     return launch_after(k_finalize, P, 32, 0, st, P, G, gc, (const unsigned long long*)acc,
                         (const unsigned long long*)hist_ttft, (const unsigned long long*)hist_tbt,
-                        (const unsigned long long*)grp_sum_n, grp_off, stats, stats_host, err);
+                        (const unsigned long long*)fin_totals, stats, stats_host, err);
 }
 
 cudaError_t launch_select(const disco_policy_stats_t* stats, uint32_t P, double cost_cap, float tbt_slo_s,

@@ -1,5 +1,8 @@
 """Full-size workloads, in the launch configuration the benchmark times: sampled pairs against the oracle
-(request ranges it can play one by one) and properties that hold at any size (needs a GPU)."""
+(request ranges it can play one by one), whole-grid statistics against the oracle run on the host's threads,
+and properties that hold at any size (needs a GPU)."""
+import os
+
 import numpy as np
 import pytest
 
@@ -26,12 +29,12 @@ def _check(w, policies, ranges, tag):
     from parity import check_tables
     check_tables(tr, orc, tag)             # length histograms, sorted TTFT ticks and knots at full size
     host = {f: out[f].cpu().numpy() for f in out}
-    for i0, i1 in ranges:
-        _, oout = orc.eval(policies, w.seed, i0, i1, pairs=True, finish=False)
-        for f in EXACT_PAIR:
-            assert (host[f][:, i0:i1] == oout[f][:, i0:i1]).all(), (tag, f, i0)
-        for f in FLOAT_PAIR:
-            assert rel_close(host[f][:, i0:i1], oout[f][:, i0:i1], REL_TOL).all(), (tag, f, i0)
+    oout = orc.eval_columns(policies, w.seed, ranges)
+    cols = np.concatenate([np.arange(i0, i1) for i0, i1 in ranges])
+    for f in EXACT_PAIR:
+        assert (host[f][:, cols] == oout[f]).all(), (tag, f)
+    for f in FLOAT_PAIR:
+        assert rel_close(host[f][:, cols], oout[f], REL_TOL).all(), (tag, f)
     # properties at full size
     sum_n, N = int(w.output_len.sum()), w.n
     for p in range(P):
@@ -72,11 +75,12 @@ def test_workload4_full_six_groups_policy_subset():
 
 # ---- the whole policy grid with reductions only: the launch configuration of workloads 2 and 4 ---------------
 
-def _oracle_stats_threaded(orc, policies, seed, threads=8):
+def _oracle_stats_threaded(orc, policies, seed, threads=None):
     """The oracle over disjoint request ranges on several host threads (its C library releases the GIL); the
     integer accumulators and histograms merge exactly."""
     from concurrent.futures import ThreadPoolExecutor
     from oracle.binding import merge_stats
+    threads = threads or max(1, os.cpu_count() or 1)
     bounds = [orc.n * k // threads for k in range(threads + 1)]
     with ThreadPoolExecutor(threads) as ex:
         parts = list(ex.map(lambda k: orc.eval(policies, seed, bounds[k], bounds[k + 1], finish=False)[0],
@@ -149,14 +153,69 @@ def test_workload2_full_size_whole_grid_properties():
     tr.close()
 
 
+def test_workload2_full_size_against_the_oracle():
+    # 10^6 requests x 1024 policies: every counter, both histograms of every policy and the selection against the
+    # oracle (about 2e11 token-steps of it, on all host threads), then every field of the pairs of each 64th
+    # request under policies that span all four thresholds
+    from parity import check_stats
+    w = synth.make_workload(2)
+    P, N = len(w.policies), w.n
+    assert (N, P) == (1_000_000, 1024)
+    tr = Trace.from_workload(w)
+    tr.eval_policies(w.policies, w.seed)
+    gs = tr.reduce_stats()
+    orc = Oracle.from_workload(w)
+    ostats = _oracle_stats_threaded(orc, w.policies, w.seed)
+    check_stats(gs, ostats, tr.histograms, "config2-full")
+    cheapest = min(s.total_cost for s in ostats)
+    from paper_2502_11417_b200.api import select_policy
+    for cap, slo in [(1.25 * cheapest, 0.25), (1.02 * cheapest, 0.25), (0.5 * cheapest, 0.25), (1e30, 1e-3)]:
+        want = orc.select(ostats, cap, float(np.float32(slo)))
+        assert tr.select_policy(cap, slo) == want and select_policy(gs, cap, slo) == want, (cap, slo)
+    sub = [t * 256 + k for t in range(4) for k in (0, 37, 100, 128, 200, 255)]
+    pols = [w.policies[p] for p in sub]
+    out = tr.alloc_pair_outputs(len(pols))
+    tr.eval_policies(pols, w.seed, out)
+    tr.reduce_stats()
+    cols = np.arange(0, N, 64)
+    oout = orc.eval_columns(pols, w.seed, [(int(i), int(i) + 1) for i in cols])
+    for f in EXACT_PAIR:
+        assert (out[f][:, ::64].cpu().numpy() == oout[f]).all(), f
+    for f in FLOAT_PAIR:
+        assert rel_close(out[f][:, ::64].cpu().numpy(), oout[f], REL_TOL).all(), f
+    assert (oout["mig_at"] > 0).any() and (oout["decision"] == 1).any() and (oout["decision"] == 2).any()
+    tr.close()
+
+
 def test_pair_arrays_beyond_2_32_elements():
     # 4.3 M requests x 1024 policies = 4.4e9 pairs: element indices no longer fit 32 bits, so the row writer runs
-    # with 64-bit indices.  Its rows must equal those of two half-grid runs, whose indices do fit.
+    # with 64-bit indices.  Its rows must equal those of two half-grid runs, whose indices do fit ...
     import torch
     w = synth.make_workload(2, n=4_300_000)
     P = len(w.policies)
     assert P * w.n > 2 ** 32 and (P // 2) * w.n < 2 ** 32
     tr = Trace.from_workload(w)
+    # ... and the oracle's, every field, on sampled request ranges under all 1024 policies (the arrays are
+    # written a few fields at a time: all nine at once would take 136 GB)
+    orc = Oracle.from_workload(w)
+    ranges = _sampled_ranges(w.n, 6, 24, 12)
+    cols = np.concatenate([np.arange(i0, i1) for i0, i1 in ranges])
+    oout = orc.eval_columns(w.policies, w.seed, ranges)
+    for fields in (["ttft_s", "decision"], ["tbt_mean_s", "delayed"], ["tbt_max_s"], ["cost"], ["tok_server"],
+                   ["tok_device"], ["mig_at"]):
+        part = tr.alloc_pair_outputs(P, fields=fields)
+        tr.eval_policies(w.policies, w.seed, part)
+        tr.reduce_stats()
+        for f in fields:
+            got = torch.stack([part[f][:, i0:i1] for i0, i1 in ranges], 0).permute(1, 0, 2).reshape(P, -1).cpu().numpy()
+            assert got.shape == oout[f].shape
+            if f in EXACT_PAIR:
+                assert (got == oout[f]).all(), f
+            else:
+                assert rel_close(got, oout[f], REL_TOL).all(), f
+        del part
+        torch.cuda.empty_cache()
+    assert (oout["mig_at"] > 0).any()
     full = tr.alloc_pair_outputs(P, fields=["decision"])
     tr.eval_policies(w.policies, w.seed, full)
     tr.reduce_stats()
@@ -170,10 +229,11 @@ def test_pair_arrays_beyond_2_32_elements():
     tr.close()
 
 
-@pytest.mark.parametrize("cfg,policy_step", [(3, 1), (4, 16)])
+@pytest.mark.parametrize("cfg,policy_step", [(3, 1), (4, 1)])
 def test_aggregates_on_262144_requests(cfg, policy_step):
-    # traces of 2^18 requests with the shape of workloads 3 and 4 (many chunks, several waves of blocks, six groups
-    # for workload 4): tables, every statistic and histogram against the oracle run on host threads
+    # traces of 2^18 requests with the shape of workloads 3 and 4 under ALL their policies (many chunks, several
+    # waves of blocks, six groups and 32 full policy tiles for workload 4): tables, every statistic and histogram
+    # against the oracle run on host threads
     from parity import check_stats, check_tables
     w = synth.make_workload(cfg, n=1 << 18)
     pols = w.policies[::policy_step]
@@ -182,7 +242,7 @@ def test_aggregates_on_262144_requests(cfg, policy_step):
     check_tables(tr, orc, f"sub-config{cfg}")
     tr.eval_policies(pols, w.seed)
     gs = tr.reduce_stats()
-    ostats = _oracle_stats_threaded(orc, pols, w.seed, threads=16)
+    ostats = _oracle_stats_threaded(orc, pols, w.seed)
     check_stats(gs, ostats, tr.histograms, f"sub-config{cfg}")
     cheapest = min(s.total_cost for s in ostats)
     assert tr.select_policy(1.25 * cheapest, 0.25) == orc.select(ostats, 1.25 * cheapest, float(np.float32(0.25)))

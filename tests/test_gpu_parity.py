@@ -110,11 +110,19 @@ def test_stochastic_baselines_and_expected_length():
             for md in (S_MODE, D_MODE, synth.MODE_AUTO)]
     pols += [synth.policy(b, mig_threshold=th, expected_len=E) for b in (0.4, 1.0) for th in (0.0, 0.02)
              for E in (0, 5, 64, 128, 4096)]
+    # random routing takes precedence over the Eq. 1-2 wait rule: one endpoint, no race
+    both = [synth.policy(b, flags=STOCH | synth.FLAG_BETA_RULE | MIG | PACE | md, l_immediate=li)
+            for b in (0.3, 0.77) for md in (D_MODE, synth.MODE_AUTO) for li in (0, 50)]
+    first_both = len(pols)
+    pols += both
     for dear in (False, True):
         w = synth.tiny_workload(31 + dear, 3000, n_servers=2, n_devices=2, max_prompt=600, max_out=200,
                                 device_dearer=dear)
         gs, _ = full_parity(w, pols, tag=f"next dear={dear}")
         assert gs[0].n_race == 0 and gs[3].n_race == 0
+        assert all(gs[first_both + k].n_race == 0 and gs[first_both + k].n_migrations == 0 for k in range(len(both)))
+        # a tile of such policies alone (staged histogram increments in the reduction kernel)
+        full_parity(w, both, tag=f"stoch+beta dear={dear}")
 
 
 def test_linear_wait_rule():
