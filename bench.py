@@ -2,21 +2,25 @@
 """Throughput of the DiSCo policy-evaluation path on B200: request-policy evaluations per second.
 
 One step = one pass of the whole path over one synthetic workload: trace ingestion (ticks, p(l), sorted
-F), Algorithms 1-3 for every policy, token-by-token play-out, per-pair evaluation with the per-pair
-arrays written (workloads 0 and 1), per-policy reductions and policy selection.
+F), Algorithms 1-3 for every policy, token-by-token play-out, per-pair evaluation (with the per-pair
+arrays written for workloads 0 and 1), per-policy reductions and policy selection.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference] [--sharded]
 
-`value` is measured with the trace arrays already resident in HBM; `e2e` goes through the same calls with
-pinned host arrays (host->device copies and the statistics read-back inside the timed region).  With
-N > 1 (torchrun) every rank evaluates an independent trace of the same shape (weak scaling, no
-collective on the data path).  `--impl reference` times the CPU oracle on the host cores instead.
+The line's `value` is workload `--config` (default 4: 16 M requests x 1024 policies, six profile groups,
+nothing materialised) with the trace arrays already resident in HBM; `e2e` goes through the same calls
+with pinned host arrays (host->device copies and the statistics read-back inside the timed region).  At
+one GPU the line also carries `per_config`: the same measurements for every workload 0-5, taken in the
+same process.  With N > 1 (torchrun) every rank evaluates an independent trace of the same shape (weak
+scaling, no collective on the data path); `--sharded` instead splits ONE trace into request ranges, one
+per rank (strong scaling: the ranks exchange the tables of Algorithm 1 and add up their accumulators).
+`--impl reference` times the CPU oracle on the host cores instead.
 """
 import argparse
 import json
+import math
 import os
 import statistics
-import subprocess
 import sys
 import time
 
@@ -47,12 +51,16 @@ PAIR_INSTR_NOWAIT = 21
 # outcome index 3, row address 1, two row loads 2, sums 8, histogram increment from the float bits (convert,
 # small-value test and branch, offset 2, increment 3, address, atomic) 10, stall test 1.
 PAIR_INSTR_WAIT = 37
-SM_COUNT, SCHEDULERS, LANES = 148, 4, 32
-MIN_WARMUP = 100             # untimed steps before either timed region, at the least
-KERNEL_EVENT_STRIDE = 8      # per-kernel CUDA events are recorded on every 8th timed step
-# DRAM bytes per launch from the committed ncu capture of the dominant kernel (None until captured for
-# the current kernel; see profiles/).
-NCU_TRAFFIC_BYTES = {"k_pairs_rows": 148985344, "k_pairs_acc": None, "k_playout_fast": 828160, "k_playout": None}
+SCHEDULERS, LANES = 4, 32    # warp schedulers per multiprocessor, lanes per warp
+MIN_WARMUP_SECONDS = 0.5     # untimed steps run until this much device time has passed (and at least --warmup)
+MAX_WARMUP_STEPS = 200
+# From the committed ncu captures (profiles/): DRAM bytes per launch of the bench's own launch shape, and the
+# lane-slots the hardware executed per unit of work beside the algorithmic counts above.  None: not captured
+# for the current kernel.
+NCU_TRAFFIC_BYTES = {("k_pairs_rows", 1): 148985344, ("k_playout_fast", 1): 828160}
+NCU_EXECUTED_PER_UNIT = {}
+HEADLINE_CONFIG = 4
+ALL_CONFIGS = (0, 1, 2, 3, 4, 5)
 
 
 def env_rank():
@@ -149,6 +157,38 @@ def whole_job_rate(units_per_rank, world, steps, total_ms):
     return units_per_rank * world * steps / (total_ms * 1e-3)
 
 
+def shard_bounds(n, world):
+    """Contiguous request ranges, one per rank: rank r holds [bounds[r], bounds[r+1])."""
+    return [n * r // world for r in range(world + 1)]
+
+
+def exchange_group_tables(cnt, sorted_by_group, dist, device):
+    """Whole-trace tables from the ranks' own: the length histograms add up (one all-reduce); every rank's
+    sorted ticks of a group are gathered (padded to the longest run) and laid out group after group.  Returns
+    (cnt int64 [G, 4097] on the host, ticks int32 tensor, n_ticks uint64 [G]); the ticks of a group are the
+    ranks' sorted runs one after the other, which is what disco_set_group_tables takes.
+    cnt: numpy int64 [G, 4097]; sorted_by_group: list of G int32 tensors on `device`."""
+    import torch
+    world = dist.get_world_size()
+    G = len(sorted_by_group)
+    c = torch.from_numpy(np.ascontiguousarray(cnt, dtype=np.int64)).to(device)
+    dist.all_reduce(c, op=dist.ReduceOp.SUM)
+    mine = torch.tensor([int(s.numel()) for s in sorted_by_group], dtype=torch.int64, device=device)
+    sizes = [torch.empty_like(mine) for _ in range(world)]
+    dist.all_gather(sizes, mine)
+    sizes = torch.stack(sizes).cpu().numpy()                               # [world, G]
+    longest = int(sizes.max()) if sizes.size else 0
+    pieces = []
+    for g in range(G):
+        pad = torch.zeros(max(longest, 1), dtype=torch.int32, device=device)
+        pad[:sorted_by_group[g].numel()] = sorted_by_group[g]
+        got = [torch.empty_like(pad) for _ in range(world)]
+        dist.all_gather(got, pad)
+        pieces += [got[r][:int(sizes[r, g])] for r in range(world)]
+    ticks = torch.cat(pieces) if pieces else torch.empty(0, dtype=torch.int32, device=device)
+    return c.cpu().numpy(), ticks.contiguous(), sizes.sum(axis=0).astype(np.uint64)
+
+
 def oracle_sample_run(w, n_req, threads):
     """Times the oracle, as it stands, on the first n_req requests under every policy of w, one thread per
     contiguous request range.  Returns seconds."""
@@ -156,6 +196,7 @@ def oracle_sample_run(w, n_req, threads):
     from oracle import Oracle
     orc = oracle_sample_run.cache.get(id(w))
     if orc is None:
+        oracle_sample_run.cache.clear()
         orc = Oracle.from_workload(w)
         oracle_sample_run.cache[id(w)] = orc
     threads = max(1, min(threads, n_req))
@@ -174,9 +215,22 @@ oracle_sample_run.cache = {}
 
 
 def size_oracle_sample(w, threads, seconds):
-    probe = min(w.n, max(threads * 64, 2048))
+    probe = min(w.n, max(threads * 4, 64))
     t = oracle_sample_run(w, probe, threads)
-    return int(min(w.n, max(probe, probe * seconds / max(t, 1e-4))))
+    if t < 0.05 and probe < w.n:                    # too short to extrapolate from: probe once more, larger
+        probe = min(w.n, probe * 16)
+        t = oracle_sample_run(w, probe, threads)
+    return int(min(w.n, max(threads, probe * seconds / max(t, 1e-4))))
+
+
+def cpu_baseline_of(w, seconds):
+    cores = os.cpu_count() or 1
+    n_req = size_oracle_sample(w, cores, seconds)
+    t = oracle_sample_run(w, n_req, cores)
+    P = w.n_policies
+    return {"value": n_req * P / t, "unit": UNIT, "cores": min(cores, n_req), "kind": "oracle",
+            "sample": "first %d of %d requests x all %d policies, %.1f s" % (n_req, w.n, P, t),
+            "token_steps_per_s": int((w.output_len[:n_req] - 1).sum()) * P / t}
 
 
 def run_reference(args):
@@ -191,7 +245,7 @@ def run_reference(args):
         oracle_sample_run(w, n_req, cores)
     times = [oracle_sample_run(w, n_req, cores) for _ in range(args.steps)]
     pairs = n_req * w.n_policies
-    toks = int(w.output_len[:n_req].sum()) * w.n_policies
+    toks = int((w.output_len[:n_req] - 1).sum()) * w.n_policies
     total = sum(times)
     value = pairs * args.steps / total
     sample = "first %d of %d requests x all %d policies per step" % (n_req, w.n, w.n_policies)
@@ -207,6 +261,216 @@ def run_reference(args):
     return 0
 
 
+class Bench:
+    """The measurements of one workload on this rank's GPU."""
+
+    def __init__(self, args, dist, rank, world, flush, peaks, alu_measured):
+        self.args, self.dist, self.rank, self.world = args, dist, rank, world
+        self.flush, self.peaks, self.alu_measured = flush, peaks, alu_measured
+
+    def run(self, cfg, steps, warmup, oracle_seconds, sampler=None, sharded=False):
+        import ctypes
+        import torch
+        from paper_2502_11417_b200 import synth, Trace
+        from paper_2502_11417_b200.api import (policy_array, kernel_launch_count, PolicyStats, stats_view,
+                                               select_policy)
+        args, dist, world, flush = self.args, self.dist, self.world, self.flush
+        stream = torch.cuda.current_stream()
+        if sharded:
+            whole = synth.make_workload(cfg, n=args.requests, n_budgets=args.budgets)
+            b = shard_bounds(whole.n, world)
+            lo, hi = b[self.rank], b[self.rank + 1]
+            w = whole
+        else:
+            w = synth.make_workload(cfg, n=args.requests, n_budgets=args.budgets, replica=self.rank)
+            lo, hi = 0, w.n
+        P, n = w.n_policies, hi - lo
+        G = len(w.servers) * len(w.devices)
+        pols = policy_array(w.policies)
+        cols = (w.prompt_len, w.output_len, w.server_ttft_s, w.server_profile, w.device_profile)
+        host = [torch.from_numpy(np.ascontiguousarray(x[lo:hi])).pin_memory() for x in cols]
+        dev = [x.cuda() for x in host]
+        h2d = sum(x.numel() * x.element_size() for x in host) + P * ctypes.sizeof(pols[0])
+        d2h = P * ctypes.sizeof(PolicyStats) + 8
+        tr = Trace()
+        tr.n = n
+        out = None
+        if w.materialise:
+            tr.load_trace(*dev, w.servers, w.devices, first_index=lo)
+            out = tr.alloc_pair_outputs(P)
+        cap_factor, slo = w.select["cost_cap_factor"], w.select["tbt_slo_s"]
+        words = None
+
+        def step(arrays):
+            nonlocal words
+            tr.load_trace(*arrays, w.servers, w.devices, stream=stream, first_index=lo)
+            if sharded:
+                # exchange 1: every rank needs the whole trace's p(l) and F before Algorithms 1-3 run
+                cnt = np.stack([tr.group_tables(g, n_sorted=0)[0] for g in range(G)])
+                mine = [tr.sorted_ticks_device(g) for g in range(G)]
+                tcnt, ticks, n_ticks = exchange_group_tables(cnt, mine, dist, "cuda")
+                tr.set_group_tables(tcnt, ticks, n_ticks, stream=stream)
+            tr.eval_policies(pols, w.seed, out, stream=stream)
+            if sharded:
+                # exchange 2: the accumulators are integer sums over requests
+                if words is None:
+                    words = torch.empty(tr.accumulator_words(), dtype=torch.int64, device="cuda")
+                tr.export_accumulators(words, stream=stream)
+                dist.all_reduce(words, op=dist.ReduceOp.SUM)
+                tr.import_accumulators(words, stream=stream)
+            st = tr.reduce_stats(stream=stream)
+            cap = cap_factor * float(stats_view(st)["total_cost"].min())
+            return select_policy(st, cap, slo)
+
+        def run_steps(arrays, k, collect=None):
+            """k steps, each between its own pair of events, L2 flushed before each; returns the summed device
+            milliseconds of this rank (the flush is outside the events)."""
+            evs = []
+            for _ in range(k):
+                flush.zero_()
+                if collect is not None:
+                    tr.set_timing(True)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                step(arrays)
+                e1.record(stream)
+                evs.append((e0, e1))
+                if collect is not None:
+                    collect.append(tr.timing())
+            torch.cuda.synchronize()
+            return sum(a.elapsed_time(b) for a, b in evs)
+
+        def warm_up(arrays):
+            """At least `warmup` steps and MIN_WARMUP_SECONDS of device time (the first steps of a fresh process
+            run slower: clocks and caches settle); the same count on every rank."""
+            done, ms = 0, 0.0
+            while done < MAX_WARMUP_STEPS and (done < warmup or ms < 1e3 * MIN_WARMUP_SECONDS):
+                k = max(1, min(warmup - done, 8)) if done < warmup else 4
+                ms += run_steps(arrays, k)
+                done += k
+                if dist is not None:                 # all ranks stop together
+                    t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+                    dist.all_reduce(t, op=dist.ReduceOp.MIN)
+                    ms = float(t.item())
+            return done
+
+        def timed(arrays):
+            torch.cuda.synchronize()
+            if dist is not None:
+                dist.barrier()
+            tr.set_timing(False)
+            ms = run_steps(arrays, steps)
+            if dist is not None:
+                dist.barrier()
+            return max_over_ranks(ms, dist, "cuda")
+
+        warm_dev = warm_up(dev)
+        l0 = kernel_launch_count()
+        if sampler is not None:
+            sampler.start()
+        total_ms = timed(dev)
+        clocks = sampler.stop() if sampler is not None else None
+        launches = kernel_launch_count() - l0
+        # per-kernel durations: a pass of its own (the library's events around its big kernels keep neighbouring
+        # launches from overlapping, which would slow the timed steps), one sample per step
+        ktimes = []
+        run_steps(dev, max(steps, 5), ktimes)
+        tr.set_timing(False)
+        warm_host = warm_up(host)
+        e2e_ms = timed(host)
+
+        units = (w.n if sharded else n * world) * P                      # pairs of the whole job per step
+        value = units * steps / (total_ms * 1e-3)
+        e2e_value = units * steps / (e2e_ms * 1e-3)
+        token_steps = int((w.output_len[lo:hi] - 1).sum())
+        n_classes = len({(float(np.float32(q["r_c"])), float(np.float32(q["t_m_s"])), int(q["flags"]) & 2)
+                         for q in w.policies})
+        job_token_steps = (int((w.output_len - 1).sum()) if sharded else token_steps * world) * n_classes
+
+        # ---- rooflines of the timed kernels
+        hbm_gbs, sm_max_mhz, src = self.peaks
+        sms = torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count
+        names = ["k_playout_fast", "k_playout", "k_pairs_acc", "k_pairs_rows"]
+        kms = {nm: statistics.mean(t[i] for t in ktimes) for i, nm in enumerate(names)}
+        alu_peak = sms * SCHEDULERS * LANES * sm_max_mhz * 1e6 / 1e12         # T lane-instructions/s
+        alu_src = "%d SMs x %d schedulers x %d lanes x %.0f MHz (issue slots)" % (sms, SCHEDULERS, LANES, sm_max_mhz)
+        alu_meas = self.alu_measured / 1e12 if self.alu_measured else None
+        per_token = PLAYOUT_INSTR_PER_TOKEN_LEAN if never_clamps(w) else PLAYOUT_INSTR_PER_TOKEN
+        full_size = not args.requests and not args.budgets
+
+        def alu_roof(name, lane_instr, ms, **extra):
+            ach = lane_instr / (ms * 1e-3) / 1e12
+            r = {"kernel": name, "bound": "alu", "achieved": ach, "peak": alu_peak, "unit": "Tinstr/s",
+                 "frac": ach / alu_peak, "traffic": NCU_TRAFFIC_BYTES.get((name, cfg)) if full_size else None,
+                 "peak_source": alu_src,
+                 # what the GPU sustains on the token loop's own instruction mix with every SM full
+                 # (disco_measure_alu_peak, measured in this run)
+                 "peak_measured": alu_meas, "frac_of_measured": ach / alu_meas if alu_meas else None,
+                 "executed_lane_slots_per_unit": NCU_EXECUTED_PER_UNIT.get((name, cfg)),
+                 "ms_per_launch": ms}
+            r.update(extra)
+            return r
+
+        def roof_of(name):
+            ms = kms[name]
+            if ms <= 0.0:
+                return None
+            if name == "k_pairs_rows":
+                if not w.materialise:
+                    return None
+                bytes_alg = n * P * PAIR_OUT_BYTES + n * TRACE_BYTES
+                ach = bytes_alg / (ms * 1e-3) / 1e9
+                return {"kernel": name, "bound": "hbm", "achieved": ach, "peak": hbm_gbs, "unit": "GB/s",
+                        "frac": ach / hbm_gbs, "traffic": NCU_TRAFFIC_BYTES.get((name, cfg)) if full_size else None,
+                        "peak_source": src, "algorithmic_bytes": bytes_alg, "ms_per_launch": ms}
+            if name == "k_pairs_acc":
+                # pairs by kind: a (group, policy) waits when Algorithm 1 made the group device-constrained
+                lane_instr, wait_pairs = 0, 0
+                for g in range(tr.n_groups):
+                    n_g = tr.group_size(g)
+                    n_wait = sum(1 for p in range(P) if tr.prep(g, p).device_constrained)
+                    wait_pairs += n_g * n_wait
+                    lane_instr += n_g * (n_wait * PAIR_INSTR_WAIT + (P - n_wait) * PAIR_INSTR_NOWAIT)
+                return alu_roof(name, lane_instr, ms,
+                                instr_per_pair={"no_wait": PAIR_INSTR_NOWAIT, "wait": PAIR_INSTR_WAIT,
+                                                "mean": lane_instr / float(max(n * P, 1))},
+                                pairs_with_waits=wait_pairs)
+            if name == "k_playout_fast":
+                return alu_roof(name, token_steps * per_token * n_classes, ms, token_steps=token_steps * n_classes,
+                                instr_per_token_step=per_token)
+            return None                       # k_playout: only the requests the clamp-free kernel listed
+
+        roofs = [r for r in (roof_of(nm) for nm in names) if r is not None]
+        roof = None
+        if roofs:
+            roof = dict(max(roofs, key=lambda r: r["ms_per_launch"]))
+            roof["all_kernels"] = [{k: r.get(k) for k in ("kernel", "bound", "achieved", "peak", "unit", "frac",
+                                                          "frac_of_measured", "ms_per_launch")} for r in roofs]
+            roof["kernels_ms"] = kms
+            roof["kernel_event_samples"] = len(ktimes)
+        cpu = None
+        if self.rank == 0 and world == 1 and oracle_seconds > 0:
+            cpu = cpu_baseline_of(w, oracle_seconds)
+        tr.close()
+        res = {"value": value, "ms_per_step": total_ms / steps, "steps": steps, "warmup": warm_dev,
+               # token-steps actually played per second: one play-out per request and timeline class (policies
+               # that share the consumption rate, buffer size and pacing share it), whatever the number of policies
+               "sim_tokens_per_s": job_token_steps * steps / (total_ms * 1e-3),
+               # tokens of all (request, policy) pairs covered per second: each played token counted once for
+               # every policy that shares its play-out
+               "pair_tokens_per_s": job_token_steps / n_classes * P * steps / (total_ms * 1e-3),
+               "config": {"workload": w.name, "requests_per_gpu": n, "policies": P, "groups": G,
+                          "pairs_per_step": units, "per_pair_outputs": bool(w.materialise),
+                          "l2": "flushed between steps (512 MB write)", "seed": w.seed,
+                          "select": "cost cap %.2f x cheapest policy, P99 TBT <= %.2f s" % (cap_factor, slo)},
+               "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                       "ms_per_step": e2e_ms / steps, "warmup": warm_host},
+               "gpu_launches": launches, "roofline": roof, "cpu_baseline": cpu}
+        if clocks is not None:
+            res["clocks"] = clocks
+        return res
+
+
 def run_ours(args):
     import torch
     rank, local_rank, world = env_rank()
@@ -217,168 +481,60 @@ def run_ours(args):
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-    from paper_2502_11417_b200 import synth, Trace
-    from paper_2502_11417_b200.api import policy_array, kernel_launch_count, PolicyStats, stats_view
-    import ctypes
+    if args.sharded and world == 1:
+        import torch.distributed as dist
+        if not dist.is_initialized():
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+            os.environ.setdefault("MASTER_PORT", str(29400 + os.getpid() % 500))
+            dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", local_rank))
+    from paper_2502_11417_b200.api import measure_alu_peak
 
-    w = synth.make_workload(args.config, n=args.requests, n_budgets=args.budgets, replica=rank)
-    P, n = w.n_policies, w.n
-    pols = policy_array(w.policies)
-    host = [torch.from_numpy(x).pin_memory() for x in (w.prompt_len, w.output_len, w.server_ttft_s,
-                                                       w.server_profile, w.device_profile)]
-    dev = [x.cuda() for x in host]
-    h2d = sum(x.numel() * x.element_size() for x in host) + P * ctypes.sizeof(pols[0])
-    d2h = P * ctypes.sizeof(PolicyStats) + 8
-    tr = Trace()
-    tr.n = n
-    out = None
-    if w.materialise:
-        tr.load_trace(*dev, w.servers, w.devices)
-        out = tr.alloc_pair_outputs(P)
     flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")       # larger than the 126 MB L2
-    stream = torch.cuda.current_stream()
-    tr.load_trace(*dev, w.servers, w.devices)
-    cap_factor, slo = w.select["cost_cap_factor"], w.select["tbt_slo_s"]
-
-    def step(arrays):
-        tr.load_trace(*arrays, w.servers, w.devices, stream=stream)
-        tr.eval_policies(pols, w.seed, out, stream=stream)
-        st = tr.reduce_stats(stream=stream)
-        cap = cap_factor * float(stats_view(st)["total_cost"].min())
-        return tr.select_policy(cap, slo, stream=stream)
-
-    def timed(arrays, steps, warmup, collect=None):
-        for _ in range(warmup):
-            step(arrays)
-        torch.cuda.synchronize()
-        if dist is not None:
-            dist.barrier()
-        evs = []
-        for i in range(steps):
-            flush.zero_()
-            # the library's own events around its four big kernels cost about 45 us a step at workload 1 (they
-            # keep neighbouring launches from overlapping), so they are recorded on every KERNEL_EVENT_STRIDE-th
-            # timed step only
-            sample = collect is not None and i % KERNEL_EVENT_STRIDE == 0
-            tr.set_timing(sample)
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(stream)
-            step(arrays)
-            e1.record(stream)
-            evs.append((e0, e1))
-            if sample:
-                collect.append(tr.timing())
-        torch.cuda.synchronize()
-        if dist is not None:
-            dist.barrier()
-        return max_over_ranks(sum(a.elapsed_time(b) for a, b in evs), dist, "cuda")
-
     vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
     try:
         phys = int(vis.split(",")[local_rank]) if vis else local_rank
     except ValueError:
         phys = local_rank
-    sampler = ClockSampler(phys)
-    ktimes = []
-    l0 = kernel_launch_count()
-    # the first 75 or so steps of a fresh process run about 10 % slower (clocks and caches settling): at least
-    # MIN_WARMUP untimed steps are run, whatever --warmup says; `warmup_run` in the output says how many
-    warm = max(args.warmup, args.min_warmup)
-    timed(dev, 0, warm)
-    l_warm = kernel_launch_count()
-    sampler.start()
-    total_ms = timed(dev, args.steps, 0, ktimes)
-    clocks = sampler.stop()
-    launches = kernel_launch_count() - l_warm
-    e2e_ms = timed(host, args.steps, warm)
-
-    pairs = n * P * world
-    toks = int(w.output_len.sum()) * P * world          # approximate for N > 1: replicas have like shapes
-    value = whole_job_rate(n * P, world, args.steps, total_ms)
-    e2e_value = whole_job_rate(n * P, world, args.steps, e2e_ms)
-
-    # ---- roofline of the dominant kernel of a step
-    hbm_gbs, sm_max_mhz, src = measured_peaks()
-    names = ["k_playout_fast", "k_playout", "k_pairs_acc", "k_pairs_rows"]
-    kms = {nm: statistics.mean(t[i] for t in ktimes) for i, nm in enumerate(names)}
-    token_steps = int((w.output_len - 1).sum())
-    n_classes = len({(float(np.float32(q["r_c"])), float(np.float32(q["t_m_s"])), int(q["flags"]) & 2) for q in w.policies})
-    alu_peak = SM_COUNT * SCHEDULERS * LANES * sm_max_mhz * 1e6 / 1e12         # T lane-instructions/s
-    alu_src = "148 SMs x 4 schedulers x 32 lanes x %.0f MHz (issue slots)" % sm_max_mhz
-    per_token = PLAYOUT_INSTR_PER_TOKEN_LEAN if never_clamps(w) else PLAYOUT_INSTR_PER_TOKEN
-
-    def roof_of(name):
-        ms = kms[name]
-        if ms <= 0.0:
-            return None
-        if name == "k_pairs_rows":
-            if not w.materialise:
-                return None
-            bytes_alg = n * P * PAIR_OUT_BYTES + n * TRACE_BYTES
-            ach = bytes_alg / (ms * 1e-3) / 1e9
-            return {"kernel": name, "bound": "hbm", "achieved": ach, "peak": hbm_gbs, "unit": "GB/s",
-                    "frac": ach / hbm_gbs,
-                    "traffic": NCU_TRAFFIC_BYTES[name] if args.config == 1 and not args.requests else None,
-                    "peak_source": src, "algorithmic_bytes": bytes_alg, "ms_per_launch": ms}
-        if name == "k_pairs_acc":
-            # pairs by kind: a (group, policy) waits when Algorithm 1 made the group device-constrained
-            lane_instr, wait_pairs = 0, 0
-            for g in range(tr.n_groups):
-                n_g = tr.group_size(g)
-                n_wait = sum(1 for p in range(P) if tr.prep(g, p).device_constrained)
-                wait_pairs += n_g * n_wait
-                lane_instr += n_g * (n_wait * PAIR_INSTR_WAIT + (P - n_wait) * PAIR_INSTR_NOWAIT)
-            ach = lane_instr / (ms * 1e-3) / 1e12
-            return {"kernel": name, "bound": "alu", "achieved": ach, "peak": alu_peak, "unit": "Tinstr/s",
-                    "frac": ach / alu_peak, "traffic": None, "peak_source": alu_src,
-                    "instr_per_pair": {"no_wait": PAIR_INSTR_NOWAIT, "wait": PAIR_INSTR_WAIT,
-                                       "mean": lane_instr / float(n * P)},
-                    "pairs_with_waits": wait_pairs, "ms_per_launch": ms}
-        if name == "k_playout_fast":
-            ach = token_steps * per_token / (ms * 1e-3) / 1e12
-            return {"kernel": name, "bound": "alu", "achieved": ach, "peak": alu_peak, "unit": "Tinstr/s",
-                    "frac": ach / alu_peak,
-                    "traffic": NCU_TRAFFIC_BYTES[name] if args.config == 1 and not args.requests else None,
-                    "peak_source": alu_src, "token_steps": token_steps, "instr_per_token_step": per_token,
-                    "ms_per_launch": ms}
-        return None                       # k_playout: only the requests the clamp-free kernel listed
-
-    roofs = [r for r in (roof_of(nm) for nm in names) if r is not None]
-    roof = dict(max(roofs, key=lambda r: r["ms_per_launch"]))
-    roof["all_kernels"] = [{k: r[k] for k in ("kernel", "bound", "achieved", "peak", "unit", "frac", "ms_per_launch")}
-                           for r in roofs]
-    roof["kernels_ms"] = kms
-
-    if rank != 0:
-        if dist is not None:
-            dist.destroy_process_group()
-        return 0
-    cpu = None
-    if world == 1 and args.oracle_seconds > 0:
-        cores = os.cpu_count() or 1
-        n_req = size_oracle_sample(w, cores, args.oracle_seconds)
-        t = oracle_sample_run(w, n_req, cores)
-        cpu = {"value": n_req * P / t, "unit": UNIT, "cores": min(cores, n_req), "kind": "oracle",
-               "sample": "first %d of %d requests x all %d policies, %.1f s" % (n_req, n, P, t),
-               "sim_tokens_per_s": int(w.output_len[:n_req].sum()) * P / t}
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "warmup_run": warm, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
-            "sim_tokens_per_s": toks * args.steps / (total_ms * 1e-3),
-            # token-steps actually played: one play-out per request and timeline class (policies that share the
-            # consumption rate, buffer size and pacing share it), whatever the number of policies
-            "useful_token_steps_per_s": token_steps * n_classes * world * args.steps / (total_ms * 1e-3),
-            "config": {"workload": w.name, "requests_per_gpu": n, "policies": P, "pairs_per_step": pairs,
-                       "per_pair_outputs": bool(w.materialise), "l2": "flushed between steps (512 MB write)",
-                       "kernel_events": "every %d-th timed step (%d samples)" % (KERNEL_EVENT_STRIDE, len(ktimes)),
-                       "seed": w.seed},
-            "clocks": clocks,
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "ms_per_step": e2e_ms / args.steps},
-            "gpu_launches": launches,
-            "roofline": roof, "cpu_baseline": cpu}
-    print(json.dumps(line))
-    if dist is not None:
+    measure_alu_peak()                                                     # first call: module load, clocks
+    alu = statistics.median(measure_alu_peak()[0] for _ in range(3))
+    b = Bench(args, dist, rank, world, flush, measured_peaks(), alu)
+    main = b.run(args.config, args.steps, args.warmup, args.oracle_seconds if world == 1 else 0.0,
+                 sampler=ClockSampler(phys), sharded=args.sharded)
+    per_config = None
+    if world == 1 and not args.sharded and not args.no_per_config and not args.requests and not args.budgets:
+        per_config = []
+        for cfg in ALL_CONFIGS:
+            if cfg == args.config:
+                r = main
+            else:
+                # enough steps for a stable mean, bounded in time (a workload-3 step takes about 3 ms, a
+                # workload-2 step under 2 ms, the others well under 1 ms)
+                r = b.run(cfg, max(args.steps, 20), args.warmup, min(args.oracle_seconds, 3.0))
+            keep = {k: r[k] for k in ("value", "ms_per_step", "steps", "warmup", "sim_tokens_per_s",
+                                      "pair_tokens_per_s", "gpu_launches", "cpu_baseline")}
+            keep["workload"] = r["config"]["workload"]
+            keep["requests"], keep["policies"] = r["config"]["requests_per_gpu"], r["config"]["policies"]
+            keep["e2e"] = {k: r["e2e"][k] for k in ("value", "ms_per_step")}
+            keep["roofline"] = None if r["roofline"] is None else {
+                "kernel": r["roofline"]["kernel"], "bound": r["roofline"]["bound"], "frac": r["roofline"]["frac"],
+                "frac_of_measured": r["roofline"].get("frac_of_measured"), "all_kernels": r["roofline"]["all_kernels"]}
+            per_config.append(keep)
+    if rank == 0:
+        line = {"metric": METRIC, "value": main["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": main["warmup"], "warmup_requested": args.warmup, "ms_per_step": main["ms_per_step"],
+                "higher_is_better": True, "scaling": "strong" if args.sharded else "weak", "vs_baseline": None,
+                "dtype": "int32", "data": "synthetic", "sim_tokens_per_s": main["sim_tokens_per_s"],
+                "pair_tokens_per_s": main["pair_tokens_per_s"], "config": main["config"], "clocks": main["clocks"],
+                "e2e": main["e2e"], "gpu_launches": main["gpu_launches"], "roofline": main["roofline"],
+                "cpu_baseline": main["cpu_baseline"],
+                "alu_peak_measured": {"lane_instr_per_s": alu, "how": "disco_measure_alu_peak: the token loop's "
+                                      "13-instruction mix on every SM, median of 3"}}
+        if args.sharded:
+            line["config"]["split"] = "one trace in %d request ranges; tables all-gathered, accumulators all-reduced" % world
+        if per_config is not None:
+            line["per_config"] = per_config
+        print(json.dumps(line))
+    if dist is not None and dist.is_initialized():
         dist.destroy_process_group()
     return 0
 
@@ -386,13 +542,14 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
-    ap.add_argument("--warmup", type=int, default=50)
-    ap.add_argument("--config", type=int, default=1, help="workload 0..5 (default: workload 1)")
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=HEADLINE_CONFIG, help="workload 0..5 (default: workload 4)")
     ap.add_argument("--requests", type=int, default=None, help="shrink the trace (profiling on a small case)")
     ap.add_argument("--budgets", type=int, default=None, help="shrink the budget axis (profiling on a small case)")
-    ap.add_argument("--min-warmup", type=int, default=MIN_WARMUP,
-                    help="untimed steps run at the least, whatever --warmup says (profiling runs pass a small number)")
+    ap.add_argument("--no-per-config", action="store_true", help="skip the other workloads' measurements")
+    ap.add_argument("--sharded", action="store_true",
+                    help="N > 1: split one trace into request ranges instead of running N independent traces")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--oracle-seconds", type=float, default=15.0, help="CPU time of the oracle baseline sample")
     ap.add_argument("--oracle-step-seconds", type=float, default=3.0, help="--impl reference: CPU time per step")

@@ -192,9 +192,10 @@ int disco_get_histograms(disco_ctx_t* ctx, uint32_t p, uint64_t* ttft_hist, uint
 /* Copies what Algorithms 1-3 produced for group g = server_profile * n_devices + device_profile, policy p. */
 int disco_get_prep(disco_ctx_t* ctx, uint32_t g, uint32_t p, disco_prep_t* out, void* stream);
 
-/* Copies group g's tables to host memory (any may be NULL): requests per prompt
- * length cnt[DISCO_MAX_PROMPT+1], the 257 equally spaced order statistics of F,
- * and up to `n_sorted` of the smallest sorted TTFT ticks.  Returns the number of
+/* Copies group g's tables out (any may be NULL): requests per prompt length
+ * cnt[DISCO_MAX_PROMPT+1] (host memory), the 257 equally spaced order statistics
+ * of F and up to `n_sorted` of the smallest sorted TTFT ticks (host or device
+ * memory, each).  Synchronises `stream`.  Returns the number of
  * requests behind the group's tables (the group's own requests, or what
  * disco_set_group_tables gave), or a negative status. */
 int64_t disco_get_group_tables(disco_ctx_t* ctx, uint32_t g, int64_t* cnt, int32_t* knots,

@@ -414,6 +414,19 @@ class Trace:
             _check(int(rc))
         return cnt, kn, srt[:k]
 
+    def sorted_ticks_device(self, g: int, stream=None):
+        """Group g's ascending server-TTFT ticks as a CUDA int32 tensor (a device-to-device copy)."""
+        import torch
+        ng = lib().disco_get_group_tables(self._h, g, None, None, None, 0, _stream_ptr(stream))
+        if ng < 0:
+            _check(int(ng))
+        out = torch.empty(int(ng), dtype=torch.int32, device="cuda")
+        if ng:
+            rc = lib().disco_get_group_tables(self._h, g, None, None, out.data_ptr(), int(ng), _stream_ptr(stream))
+            if rc < 0:
+                _check(int(rc))
+        return out
+
     def set_timing(self, on: bool = True):
         _check(lib().disco_set_timing(self._h, int(on)))
 

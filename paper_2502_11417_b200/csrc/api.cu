@@ -665,9 +665,9 @@ int64_t disco_get_group_tables(disco_ctx_t* c, uint32_t g, int64_t* cnt, int32_t
         CU(cudaStreamSynchronize(st));
         for (size_t i = 0; i < tmp.size(); ++i) cnt[i] = tmp[i];
     }
-    if (knots) CU(cudaMemcpyAsync(knots, c->knots.as<int32_t>() + (size_t)g * kNKnots, kNKnots * 4, cudaMemcpyDeviceToHost, st));
+    if (knots) CU(cudaMemcpyAsync(knots, c->knots.as<int32_t>() + (size_t)g * kNKnots, kNKnots * 4, cudaMemcpyDefault, st));
     const uint64_t k = std::min<uint64_t>(n_sorted, ng);
-    if (sorted_ticks && k) CU(cudaMemcpyAsync(sorted_ticks, c->F_sorted + off, k * 4, cudaMemcpyDeviceToHost, st));
+    if (sorted_ticks && k) CU(cudaMemcpyAsync(sorted_ticks, c->F_sorted + off, k * 4, cudaMemcpyDefault, st));
     CU(cudaStreamSynchronize(st));
     return (int64_t)ng;
 }

@@ -44,6 +44,59 @@ def test_max_over_ranks_and_independent_traces():
     assert bench.max_over_ranks(7.0, None, "cpu") == 7.0
 
 
+def _shard_rank_main(rank, world, port, q):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import bench
+    from oracle import Oracle
+    from paper_2502_11417_b200 import synth
+    w = synth.make_workload(4, n=3001, n_budgets=2)                    # every rank holds a range of ONE trace
+    b = bench.shard_bounds(w.n, world)
+    lo, hi = b[rank], b[rank + 1]
+    part = Oracle(w.prompt_len[lo:hi], w.output_len[lo:hi], w.server_ttft_s[lo:hi], w.server_profile[lo:hi],
+                  w.device_profile[lo:hi], w.servers, w.devices)
+    G = part.n_groups
+    tabs = [part.group_tables(g) for g in range(G)]
+    cnt = np.stack([t[0] for t in tabs])
+    mine = [torch.from_numpy(t[1].astype(np.int32)) for t in tabs]
+    tcnt, ticks, n_ticks = bench.exchange_group_tables(cnt, mine, dist, "cpu")
+    words = torch.arange(10, dtype=torch.int64) * (rank + 1)           # accumulators add up: one all-reduce
+    dist.all_reduce(words, op=dist.ReduceOp.SUM)
+    q.put((rank, lo, hi, tcnt, ticks.numpy(), n_ticks, words.numpy()))
+    dist.destroy_process_group()
+
+
+def test_request_range_shards_exchange_whole_trace_tables():
+    """Two CPU ranks hold halves of one trace; after the exchange each has the length histogram and, group by
+    group, the TTFT ticks of the whole trace (checked against the oracle's tables of the whole trace)."""
+    from oracle import Oracle
+    from paper_2502_11417_b200 import synth
+    world, port = 2, 30500 + os.getpid() % 1000
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_shard_rank_main, args=(r, world, port, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    got = sorted((q.get(timeout=120) for _ in range(world)), key=lambda t: t[0])
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    w = synth.make_workload(4, n=3001, n_budgets=2)
+    whole = Oracle.from_workload(w)
+    assert [(g[1], g[2]) for g in got] == [(0, 1500), (1500, 3001)]    # contiguous, disjoint, covering
+    for _, _, _, tcnt, ticks, n_ticks, words in got:
+        off = 0
+        for g in range(whole.n_groups):
+            cnt, srt, _ = whole.group_tables(g)
+            assert (tcnt[g] == cnt).all() and int(n_ticks[g]) == len(srt)
+            assert (np.sort(ticks[off:off + len(srt)]) == srt).all()   # the group's ticks, the ranks' runs in turn
+            off += len(srt)
+        assert off == len(ticks) == w.n
+        assert (words == np.arange(10) * 3).all()
+    import bench
+    assert bench.shard_bounds(10, 4) == [0, 2, 5, 7, 10]
+
+
 def test_replica_zero_is_the_reference_trace():
     from paper_2502_11417_b200 import synth
     a, b = synth.make_workload(1, n=300), synth.make_workload(1, n=300, replica=0)
