@@ -215,11 +215,15 @@ oracle_sample_run.cache = {}
 
 
 def size_oracle_sample(w, threads, seconds):
+    """Number of leading requests the oracle takes about `seconds` for on `threads` threads: probes grow until
+    one took at least a fifth of the target (short runs are dominated by the per-call policy preparation and do
+    not extrapolate), then scale linearly."""
     probe = min(w.n, max(threads * 4, 64))
-    t = oracle_sample_run(w, probe, threads)
-    if t < 0.05 and probe < w.n:                    # too short to extrapolate from: probe once more, larger
-        probe = min(w.n, probe * 16)
+    while True:
         t = oracle_sample_run(w, probe, threads)
+        if probe >= w.n or t >= 0.2 * seconds:
+            break
+        probe = int(min(w.n, max(2 * probe, probe * 0.5 * seconds / max(t, 1e-3))))
     return int(min(w.n, max(threads, probe * seconds / max(t, 1e-4))))
 
 
@@ -344,7 +348,7 @@ class Bench:
             """At least `warmup` steps and MIN_WARMUP_SECONDS of device time (the first steps of a fresh process
             run slower: clocks and caches settle); the same count on every rank."""
             done, ms = 0, 0.0
-            while done < MAX_WARMUP_STEPS and (done < warmup or ms < 1e3 * MIN_WARMUP_SECONDS):
+            while done < MAX_WARMUP_STEPS and (done < warmup or ms < 1e3 * args.min_warmup_seconds):
                 k = max(1, min(warmup - done, 8)) if done < warmup else 4
                 ms += run_steps(arrays, k)
                 done += k
@@ -548,6 +552,8 @@ def main():
     ap.add_argument("--requests", type=int, default=None, help="shrink the trace (profiling on a small case)")
     ap.add_argument("--budgets", type=int, default=None, help="shrink the budget axis (profiling on a small case)")
     ap.add_argument("--no-per-config", action="store_true", help="skip the other workloads' measurements")
+    ap.add_argument("--min-warmup-seconds", type=float, default=MIN_WARMUP_SECONDS,
+                    help="untimed steps go on until this much device time has passed (profiling runs pass 0)")
     ap.add_argument("--sharded", action="store_true",
                     help="N > 1: split one trace into request ranges instead of running N independent traces")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

@@ -237,6 +237,11 @@ int disco_set_timing(disco_ctx_t* ctx, int on);
 int disco_get_timing(disco_ctx_t* ctx, float* ms4);
 uint64_t disco_kernel_launch_count(void);
 
+/* How the last evaluation's pairs were evaluated (host counts3[3]): pairs of requests that end the same way under
+ * every policy of a 32-policy tile and were settled once for the tile; pairs evaluated one by one; requests
+ * settled, counted once per tile.  The first two add up to requests x policies.  Synchronises `stream`. */
+int disco_get_work_counts(disco_ctx_t* ctx, uint64_t* counts3, void* stream);
+
 /* Measures what the GPU sustains on the integer instruction mix of the token loop (Sec. 4.3 play-out: per
  * token one counter add, the hash finaliser's three shift-xor pairs and two multiplies, one multiply-high
  * range map, one compare and one multiply-add into the sum = 13 lane-instructions) with every SM full of

@@ -78,7 +78,7 @@ EXPORTS = ["disco_load_trace", "disco_eval_policies", "disco_reduce_stats", "dis
            "disco_last_error", "disco_set_timing", "disco_get_timing", "disco_kernel_launch_count",
            "disco_sort_ttft_ticks_noalloc", "disco_select_policy_device", "disco_set_group_tables",
            "disco_accumulator_words", "disco_export_accumulators", "disco_import_accumulators",
-           "disco_measure_alu_peak"]
+           "disco_measure_alu_peak", "disco_get_work_counts"]
 
 PAIR_FIELDS = [("ttft_s", "float32"), ("tbt_mean_s", "float32"), ("tbt_max_s", "float32"), ("cost", "float32"),
                ("tok_server", "uint32"), ("tok_device", "uint32"), ("mig_at", "uint32"), ("delayed", "uint16"),
@@ -109,6 +109,7 @@ def lib() -> C.CDLL:
         L.disco_accumulator_words.restype = u64; L.disco_accumulator_words.argtypes = [vp]
         L.disco_export_accumulators.restype = C.c_int; L.disco_export_accumulators.argtypes = [vp, vp, vp]
         L.disco_import_accumulators.restype = C.c_int; L.disco_import_accumulators.argtypes = [vp, vp, vp]
+        L.disco_get_work_counts.restype = C.c_int; L.disco_get_work_counts.argtypes = [vp, vp, vp]
         L.disco_measure_alu_peak.restype = C.c_int
         L.disco_measure_alu_peak.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_double), vp]
         L.disco_get_histograms.restype = C.c_int; L.disco_get_histograms.argtypes = [vp, u32, vp, vp, vp]
@@ -436,6 +437,13 @@ class Trace:
         ms = (C.c_float * 4)()
         _check(lib().disco_get_timing(self._h, ms))
         return tuple(ms)
+
+    def work_counts(self, stream=None):
+        """(pairs settled per policy tile, pairs evaluated one by one, requests settled per tile) of the last
+        evaluation."""
+        w = (C.c_uint64 * 3)()
+        _check(lib().disco_get_work_counts(self._h, w, _stream_ptr(stream)))
+        return tuple(int(x) for x in w)
 
     def close(self):
         if self._h:

@@ -89,7 +89,7 @@ struct disco_ctx {
     std::vector<PolicyConst> pol;
     DevBuf d_prep, d_accum, d_stats, d_tables, d_todo;
     struct View { void* p = nullptr; template <class T> T* as() const { return (T*)p; } };
-    View d_acc, d_hist_ttft, d_hist_tbt;               // three regions of d_accum (cleared by one memset)
+    View d_acc, d_hist_ttft, d_hist_tbt, d_work;       // regions of d_accum (cleared by one memset)
     View d_pol, d_classes, d_pol_list, d_chunks;       // four regions of d_tables (filled by one copy)
     DevBuf rec_u32[7], rec_u16[2], rec_win[3];
     void* stage = nullptr;       // pinned staging for the small host->device tables
@@ -397,7 +397,8 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
 #define R(buf, bytes) if ((e = c->buf.reserve(bytes)) != cudaSuccess) return fail_cuda(e, "device allocation for the evaluation")
     R(d_prep, (size_t)G * P * sizeof(Prep));
     const size_t acc_bytes = (size_t)P * G * kNAcc * 8, hist_bytes = (size_t)P * kNBins * 8;
-    const size_t cnt_bytes = (classes.size() * 8 + 15) / 16 * 16;        // a to-do counter and a ticket counter per class
+    // a to-do counter and a ticket counter per class, then the work counters of the pair kernel (four words)
+    const size_t cls_cnt_bytes = (classes.size() * 8 + 15) / 16 * 16, cnt_bytes = cls_cnt_bytes + 32;
     R(d_accum, acc_bytes + 2 * hist_bytes + cnt_bytes);
     R(d_todo, N1 * 4);
     c->d_acc.p = c->d_accum.p; c->d_hist_ttft.p = (char*)c->d_accum.p + acc_bytes;
@@ -479,6 +480,7 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
     CU(cudaEventRecord(c->stage_free, st));
 
     uint32_t* todo_counts = (uint32_t*)((char*)c->d_accum.p + acc_bytes + 2 * hist_bytes);
+    c->d_work.p = (char*)c->d_accum.p + acc_bytes + 2 * hist_bytes + cls_cnt_bytes;
 
     // ---- Algorithms 1-3 for every (group, policy)
     CU(launch_prep(c->d_pol.as<PolicyConst>(), P, G, c->d_gc.as<GroupConst>(), c->cum_mass.as<int64_t>(),
@@ -527,7 +529,8 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
         CU(launch_pairs(tr, c->d_gc.as<GroupConst>(), dcc, c->d_prep.as<Prep>(), P,
                         c->d_pol_list.as<uint32_t>() + cls_range[k].first, cls_range[k].second - cls_range[k].first,
                         c->d_chunks.as<Chunk>(), (uint32_t)chunks.size(), rec, po, c->d_acc.as<uint64_t>(),
-                        c->d_hist_ttft.as<uint64_t>(), c->d_hist_tbt.as<uint64_t>(), k0, cls_extras_pending,
+                        c->d_hist_ttft.as<uint64_t>(), c->d_hist_tbt.as<uint64_t>(), c->d_work.as<uint64_t>(), k0,
+                        cls_extras_pending,
                         classes[k].W[0] > 1 || classes[k].W[1] > 1 || classes[k].W[2] > 1,
                         timed ? c->ev[3] : nullptr, st));
         if (timed) CU(cudaEventRecord(c->ev[4], st));
@@ -626,6 +629,15 @@ int disco_get_timing(disco_ctx_t* c, float* ms4) {
     if (!c || !ms4) return fail(DISCO_EINVAL, "null argument");
     if (!c->timing_valid || !c->reduced) return fail(DISCO_EINVAL, "no timed evaluation has been reduced");
     for (int k = 0; k < 4; ++k) ms4[k] = c->ms[k];
+    return 0;
+}
+
+int disco_get_work_counts(disco_ctx_t* c, uint64_t* counts3, void* stream) {
+    if (!c || !counts3) return fail(DISCO_EINVAL, "null argument");
+    if (!c->evaluated) return fail(DISCO_EINVAL, "no evaluation");
+    cudaStream_t st = (cudaStream_t)stream;
+    CU(cudaMemcpyAsync(counts3, c->d_work.p, 24, cudaMemcpyDeviceToHost, st));
+    CU(cudaStreamSynchronize(st));
     return 0;
 }
 
@@ -758,7 +770,6 @@ int disco_import_accumulators(disco_ctx_t* c, const uint64_t* words, void* strea
     CU(cudaMemcpyAsync(c->fin_totals.p, words + head, (size_t)2 * c->G * 8, cudaMemcpyDefault, st));
     CU(cudaStreamSynchronize(st));
     c->reduced = false;
-    c->timing_valid = false;
     c->fin_imported = true;
     return 0;
 }

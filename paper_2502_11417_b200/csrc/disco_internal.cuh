@@ -164,7 +164,10 @@ cudaError_t launch_timeline(const TraceDev& tr, const GroupConst* gc, const Clas
 cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const Prep* prep, uint32_t P,
                          const uint32_t* pol_list, uint32_t n_list, const Chunk* chunks, uint32_t n_chunks,
                          TimelineRec rec, disco_pair_out_t out, uint64_t* acc, uint64_t* hist_ttft,
-                         uint64_t* hist_tbt, uint32_t k0, bool extras /* some policy routes at random or uses an
+                         uint64_t* hist_tbt,
+                         uint64_t* work /* [3], added to: pairs settled for a whole policy tile at once, pairs evaluated
+                         one by one, requests settled per tile */,
+                         uint32_t k0, bool extras /* some policy routes at random or uses an
                          expected length */, bool wide /* some window W of the class spans several bins */,
                          cudaEvent_t mid /* recorded between its two kernels, or null */,
                          cudaStream_t st);
