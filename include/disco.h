@@ -237,10 +237,11 @@ int disco_set_timing(disco_ctx_t* ctx, int on);
 int disco_get_timing(disco_ctx_t* ctx, float* ms4);
 uint64_t disco_kernel_launch_count(void);
 
-/* How the last evaluation's pairs were evaluated (host counts3[3]): pairs of requests that end the same way under
- * every policy of a 32-policy tile and were settled once for the tile; pairs evaluated one by one; requests
- * settled, counted once per tile.  The first two add up to requests x policies.  Synchronises `stream`. */
-int disco_get_work_counts(disco_ctx_t* ctx, uint64_t* counts3, void* stream);
+/* How the last evaluation's pairs were reduced (host counts4[4]): pairs settled zone by zone (a request against
+ * the runs of neighbouring policies of a 32-policy tile that dispatch it alike); pairs evaluated one by one;
+ * requests settled zone by zone, counted once per tile; those of them that needed corrections below a run
+ * boundary.  The first two add up to requests x policies.  Synchronises `stream`. */
+int disco_get_work_counts(disco_ctx_t* ctx, uint64_t* counts4, void* stream);
 
 /* Measures what the GPU sustains on the integer instruction mix of the token loop (Sec. 4.3 play-out: per
  * token one counter add, the hash finaliser's three shift-xor pairs and two multiplies, one multiply-high

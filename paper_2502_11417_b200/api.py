@@ -439,9 +439,9 @@ class Trace:
         return tuple(ms)
 
     def work_counts(self, stream=None):
-        """(pairs settled per policy tile, pairs evaluated one by one, requests settled per tile) of the last
-        evaluation."""
-        w = (C.c_uint64 * 3)()
+        """(pairs settled zone by zone, pairs evaluated one by one, requests settled per tile, those with
+        corrections) of the last evaluation."""
+        w = (C.c_uint64 * 4)()
         _check(lib().disco_get_work_counts(self._h, w, _stream_ptr(stream)))
         return tuple(int(x) for x in w)
 

@@ -87,7 +87,7 @@ struct disco_ctx {
     uint32_t P = 0;
     bool evaluated = false, reduced = false;
     std::vector<PolicyConst> pol;
-    DevBuf d_prep, d_accum, d_stats, d_tables, d_todo;
+    DevBuf d_prep, d_accum, d_stats, d_tables, d_todo, d_left;
     struct View { void* p = nullptr; template <class T> T* as() const { return (T*)p; } };
     View d_acc, d_hist_ttft, d_hist_tbt, d_work;       // regions of d_accum (cleared by one memset)
     View d_pol, d_classes, d_pol_list, d_chunks;       // four regions of d_tables (filled by one copy)
@@ -106,7 +106,7 @@ struct disco_ctx {
     ~disco_ctx() {
         DevBuf* all[] = {&in_prompt, &in_out, &in_ttft, &in_sp, &in_dp, &keys_a, &keys_b, &tmp_idx,
                          &S, &l, &nout, &orig, &sorted, &zero, &cum_mass, &ng_exact, &grp_off, &knots, &d_gc, &d_prep, &d_accum, &d_stats, &d_tables, &d_todo,
-                         &fin_totals, &F_sorted_imp, &F_off_imp};
+                         &fin_totals, &F_sorted_imp, &F_off_imp, &d_left};
         for (DevBuf* b : all) b->release();
         for (auto& b : rec_u32) b.release();
         for (auto& b : rec_u16) b.release();
@@ -427,26 +427,35 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
         cls_range.push_back({b, (uint32_t)pol_list.size()});
     }
     const uint32_t tiles = (P + 31) / 32;
+    // a lane of the zone kernel counts its requests in bytes: at most 255 requests a lane, 512 lanes a block
+    const uint32_t kMaxChunk = 130560;
     const uint32_t sms = (uint32_t)c->sms;
     uint32_t want_chunks = std::max<uint32_t>(1, sms / std::min<uint32_t>(tiles, sms));   // one block per SM
-    const uint32_t min_chunks = (uint32_t)((N1 + 65279) / 65280);
+    const uint32_t min_chunks = (uint32_t)((N1 + kMaxChunk - 1) / kMaxChunk);
     if (min_chunks > want_chunks) {
-        // several waves of blocks: pick the chunk count near the minimum whose last wave is fullest
+        // several waves of blocks: the fewest chunks whose last wave is nearly full (long chunks spread a block's
+        // set-up and flush over more requests), else the count near the minimum whose last wave is fullest
         double best = 0.0;
         for (uint32_t k = min_chunks; k < min_chunks + sms; ++k) {
             const uint64_t blocks = (uint64_t)k * tiles, waves = (blocks + sms - 1) / sms;
             const double fill = (double)blocks / (double)(waves * sms);
             if (fill > best + 1e-9) { best = fill; want_chunks = k; }
+            if (fill >= 0.94) break;
         }
     }
     uint32_t CH = (uint32_t)((N1 + want_chunks - 1) / want_chunks);
     CH = (CH + 255) / 256 * 256;
-    CH = std::min<uint32_t>(std::max<uint32_t>(CH, 256), 65280);     // 16-bit histogram counters per block
+    CH = std::min<uint32_t>(std::max<uint32_t>(CH, 256), kMaxChunk);
     std::vector<Chunk> chunks;
     for (int g = 0; g < G; ++g)
         for (uint32_t s = rb.grp_off[g]; s < rb.grp_off[g + 1]; s += CH)
             chunks.push_back({s, std::min(CH, rb.grp_off[g + 1] - s), g, 0});
 #undef R
+
+    // scratch of the pair kernels: a bit per (request, policy tile), a counter per (chunk, policy tile)
+    const size_t left_mask_words = (size_t)N1 * ((tiles + 31) / 32);
+    if ((e = c->d_left.reserve((left_mask_words + chunks.size() * (size_t)tiles + 4) * 4)) != cudaSuccess)
+        return fail_cuda(e, "device allocation for the evaluation");
 
     // ---- small tables to the device through pinned staging
     const size_t need = P * sizeof(PolicyConst) + classes.size() * sizeof(ClassConst) + P * 4 +
@@ -529,12 +538,14 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
         CU(launch_pairs(tr, c->d_gc.as<GroupConst>(), dcc, c->d_prep.as<Prep>(), P,
                         c->d_pol_list.as<uint32_t>() + cls_range[k].first, cls_range[k].second - cls_range[k].first,
                         c->d_chunks.as<Chunk>(), (uint32_t)chunks.size(), rec, po, c->d_acc.as<uint64_t>(),
-                        c->d_hist_ttft.as<uint64_t>(), c->d_hist_tbt.as<uint64_t>(), c->d_work.as<uint64_t>(), k0,
-                        cls_extras_pending,
-                        classes[k].W[0] > 1 || classes[k].W[1] > 1 || classes[k].W[2] > 1,
+                        c->d_hist_ttft.as<uint64_t>(), c->d_hist_tbt.as<uint64_t>(), c->d_left.as<uint32_t>(),
+                        c->d_left.as<uint32_t>() + left_mask_words, c->d_work.as<uint64_t>(), k0, cls_extras_pending,
+                        !classes[k].pacing || classes[k].W[0] > 1 || classes[k].W[1] > 1 || classes[k].W[2] > 1,
                         timed ? c->ev[3] : nullptr, st));
         if (timed) CU(cudaEventRecord(c->ev[4], st));
-        g_launches += (n ? ((classes[k].pacing && !never_clamps) ? 2 : 1) : 0) + ((n && !chunks.empty()) ? (out ? 2 : 1) : 0);
+        const bool wide_k = !classes[k].pacing || classes[k].W[0] > 1 || classes[k].W[1] > 1 || classes[k].W[2] > 1;
+        g_launches += (n ? ((classes[k].pacing && !never_clamps) ? 2 : 1) : 0) +
+                      ((n && !chunks.empty()) ? (out ? 2 : 1) + (wide_k ? 0 : 1) : 0);
     }
     c->timing_valid = timed && n != 0;
     c->P = P; c->pol = pc;
@@ -632,11 +643,11 @@ int disco_get_timing(disco_ctx_t* c, float* ms4) {
     return 0;
 }
 
-int disco_get_work_counts(disco_ctx_t* c, uint64_t* counts3, void* stream) {
-    if (!c || !counts3) return fail(DISCO_EINVAL, "null argument");
+int disco_get_work_counts(disco_ctx_t* c, uint64_t* counts4, void* stream) {
+    if (!c || !counts4) return fail(DISCO_EINVAL, "null argument");
     if (!c->evaluated) return fail(DISCO_EINVAL, "no evaluation");
     cudaStream_t st = (cudaStream_t)stream;
-    CU(cudaMemcpyAsync(counts3, c->d_work.p, 24, cudaMemcpyDeviceToHost, st));
+    CU(cudaMemcpyAsync(counts4, c->d_work.p, 32, cudaMemcpyDeviceToHost, st));
     CU(cudaStreamSynchronize(st));
     return 0;
 }

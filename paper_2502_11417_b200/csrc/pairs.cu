@@ -9,7 +9,7 @@
 //    store instruction writes 32 consecutive requests of one policy row.
 #include <type_traits>
 
-#include "disco_internal.cuh"
+#include "tile.cuh"
 
 namespace disco {
 
@@ -69,42 +69,18 @@ __device__ __forceinline__ PairOut decide(const PairIn& q, const Prep& pr, uint3
 // outcome only.  The lane that loads a request therefore writes, once, one row of addends per outcome into
 // shared memory; a policy lane decides the outcome and adds the row it selects.
 //
-// Most requests do not need that.  The policies of a tile differ in a few thresholds only (Algorithm 3's
-// l_th, Algorithm 2's l*, w* and w_tail, Eq. 4's overhead), so a request whose prompt length, server TTFT and
-// projected saving lie on one side of ALL of the tile's thresholds ends in the same outcome, with the same TTFT,
-// under every policy of the tile.  The lane that loaded such a request settles it alone: it adds the outcome's
-// addends to sums and histograms that the whole tile shares, which are added to each policy's when the block
-// flushes.  Only the requests that fall between the tile's thresholds are staged and evaluated pair by pair.
+// Tiles whose policies can be evaluated zone by zone (tile.cuh, zones.cu) have been through that kernel first:
+// this one then takes only the requests it flagged for the tile in the bit mask, packed to the front of the
+// staging area, and returns at once where nothing was flagged.
 // ------------------------------------------------------------------------------------------------------
 constexpr int kAccThreads = 512;         // one block per SM: histograms and staging fill its shared memory
 constexpr int kAccWarps = kAccThreads / 32;
-constexpr int kHWords = 433;            // 866 sixteen-bit counters per policy row; odd word stride
 constexpr int kStageReq = 32;           // requests a warp stages at a time
 constexpr int kIlp = 4;                 // requests a lane works on at a time
 constexpr int kStageVec = 7;            // uint4 per request in each of the two staging blocks (odd: no bank conflicts)
 
-enum Outcome { O_SERVER_ONLY = 0, O_DEVICE_ONLY = 1, O_RACE_SRV = 2, O_RACE_DEV = 3, O_MIGR_TO_DEV = 4, O_MIGR_TO_SRV = 5 };
-
-// words in front of the staging area: per-policy histograms and sums, two work counters (requests settled for the
-// whole tile, requests evaluated pair by pair), the tile's shared histograms; rounded up to 16 bytes
-__host__ __device__ constexpr int acc_stage_offset_words(int PL) {
-    return (2 * PL * kHWords + 2 * PL * kNAcc + 2 + 2 * kHWords + 3) / 4 * 4;
-}
-
-// A histogram increment as one word: byte offset of the counter pair in bits 2..11, the increment (low or
-// high sixteen bits) in bits 0 and 16.
-__device__ __forceinline__ uint32_t hist16_code(int bin) { return ((uint32_t)(bin >> 1) << 2) | ((bin & 1) ? 0x10000u : 1u); }
-__device__ __forceinline__ void hist16_apply(uint32_t* row, uint32_t code) {
-    atomicAdd((uint32_t*)((char*)row + (code & 0xFFCu)), code & 0x10001u);
-}
-
-// One more TTFT of t ticks, t < 2^31 (so its bin is below kNBins): the counter pair and the half come straight
-// from the float's exponent and leading mantissa bits, 32 bins per octave as in bin_of_ticks.
-__device__ __forceinline__ void hist16_add_ticks(uint32_t* row, uint32_t t) {
-    if (t < 32u) { hist16_apply(row, hist16_code((int)t)); return; }
-    const uint32_t fb = __float_as_uint(__uint2float_rz(t));
-    atomicAdd((uint32_t*)((char*)row - 4 * (((127 + 4) << 5) >> 1) + ((fb >> 17) & 0x3FFCu)), 1u << ((fb >> 14) & 16u));
-}
+// words in front of the staging area: two histograms and the sums, rounded up to 16 bytes
+__host__ __device__ constexpr int acc_stage_offset_words(int PL) { return (2 * PL * kHWords + 2 * PL * kNAcc + 3) / 4 * 4; }
 
 enum TileKind { K_NOWAIT = 0, K_WAIT = 1, K_ANY = 2 };
 
@@ -116,20 +92,18 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
             const Prep* __restrict__ prep, uint32_t P, const uint32_t* __restrict__ pol_list, uint32_t n_list,
             int PL, const Chunk* __restrict__ chunks, uint32_t n_tiles, TimelineRec rec, uint32_t k0,
             unsigned long long* __restrict__ acc, unsigned long long* __restrict__ hist_ttft,
-            unsigned long long* __restrict__ hist_tbt, unsigned long long* __restrict__ work) {
+            unsigned long long* __restrict__ hist_tbt, const uint32_t* __restrict__ left_mask,
+            const uint32_t* __restrict__ left_count, unsigned long long* __restrict__ work) {
     extern __shared__ uint32_t smem[];
     uint32_t* h_ttft = smem;                                  // [PL][kHWords]
     uint32_t* h_stall = smem + PL * kHWords;                  // [PL][kHWords]
     unsigned long long* s_acc = (unsigned long long*)(smem + 2 * PL * kHWords);   // [PL][kNAcc]; 866 words per policy keep it 8-byte aligned
-    uint32_t* s_work = (uint32_t*)(s_acc + PL * kNAcc);       // [2] requests settled for the tile, requests staged
-    uint32_t* hc_ttft = s_work + 2;                           // [kHWords] TTFTs of the requests settled for the whole tile
-    uint32_t* hc_stall = hc_ttft + kHWords;                   // [kHWords] their hand-off stalls
     grid_dependency_wait();
 
     // consecutive blocks take the policy tiles of one request chunk, so that the chunk is read from HBM once and
     // from L2 by the other tiles
-    const uint32_t tile = blockIdx.x % n_tiles;
-    const Chunk ch = chunks[blockIdx.x / n_tiles];
+    const uint32_t tile = blockIdx.x % n_tiles, chunk_id = blockIdx.x / n_tiles;
+    const Chunk ch = chunks[chunk_id];
     const int g = ch.g;
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     const int pol_in_tile = lane % PL, slot = lane / PL, slots = 32 / PL;
@@ -137,6 +111,11 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
     const bool act = pol_idx < n_list;
     const uint32_t p = pol_list[act ? pol_idx : 0];
     const Prep pr = prep[(size_t)g * P + p];
+    const int pols_here = (int)min((uint32_t)PL, n_list - tile * PL);
+    // a tile that went through the zone kernel: only the requests it flagged are left (block-uniform)
+    const bool flagged_only = left_mask != nullptr && tile_by_zones(pr, act, lane, pols_here);
+    if (flagged_only && left_count[(size_t)chunk_id * n_tiles + tile] == 0u) return;
+    const uint32_t mask_words = left_words_per_request(n_tiles), mask_bit = 1u << (tile & 31u);
     const GroupConst& gc = gcs[g];
     const ClassConst& cc = *ccp;
     const uint32_t kappa = (uint32_t)gc.kappa, c0 = (uint32_t)gc.c0;
@@ -146,7 +125,6 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
     const int kt0 = cc.ktau[g][0], kt1 = cc.ktau[g][1], kt2 = cc.ktau[g][2];
     const uint32_t tau = (uint32_t)cc.tau;
 
-    for (int i = threadIdx.x; i < acc_stage_offset_words(PL); i += kAccThreads) smem[i] = 0;   // (staging needs no clearing)
     // With no waits in the tile (Algorithm 3, random routing) a TTFT is the request's S or its T_d, whose
     // histogram increments are staged; otherwise the bin is worked out per pair.
     const bool waits = __syncthreads_or(act && pr.device_constrained && !pr.stochastic) != 0;
@@ -156,9 +134,19 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
     uint32_t* my_ttft = h_ttft + pol_in_tile * kHWords;
     uint32_t* my_stall = h_stall + pol_in_tile * kHWords;
 
+    // The block-private histogram counters are 16 bits wide: at most 65,280 requests are evaluated between two
+    // flushes.  A longer chunk (one that the zone kernel left more than that of, or took nothing of) goes in passes.
+    const uint32_t to_do = flagged_only ? left_count[(size_t)chunk_id * n_tiles + tile] : ch.len;
+    const uint32_t pass_len = to_do <= 65280u ? ch.len : 65280u;
+    for (uint32_t r_lo = 0; r_lo < ch.len; r_lo += pass_len) {
+    const uint32_t r_hi = min(ch.len, r_lo + pass_len);
+    for (int i = threadIdx.x; i < 2 * PL * kHWords + 2 * PL * kNAcc; i += kAccThreads) smem[i] = 0;   // (staging needs no clearing)
+    __syncthreads();
+
     uint32_t a_td = 0, a_ps = 0, a_pd = 0, a_dl = 0, a_tau = 0;
     uint32_t cnt_a = 0, cnt_b = 0;                              // device-only | race << 16,  device won | migrated << 16
     uint32_t cnt8 = 0;                                          // the same four counts, a byte each, within a batch
+    uint32_t staged = 0;                                        // requests this warp evaluated pair by pair
     unsigned long long a_tt = 0;
 
     // [warp][32 requests][kStageVec]: block A = the request, then the first half of each outcome's row;
@@ -174,25 +162,10 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
     const bool dev_migrates = candidate == 2;
     const uint32_t lth16 = (uint32_t)max(l_th, 0) << 4;      // against a staged (l << 4 | outcome at w = 0)
 
-    // ---- what the tile's policies have in common (block-uniform): the ranges of their thresholds.  A request
-    //      outside every range ends the same way under all of them.
-    const bool uni_ok = !EXT && !WIDE && kind != K_ANY;
-    const uint32_t pmask = __ballot_sync(0xFFFFFFFFu, act);       // lanes that hold a policy (every warp the same)
-    const int32_t key_lo = kind == K_WAIT ? pr.l_star : pr.l_th;  // Algorithm 2's l*, Algorithm 3's l_th
-    const int32_t len_min = __reduce_min_sync(0xFFFFFFFFu, act ? key_lo : 0x7FFFFFFF);
-    const int32_t len_max = __reduce_max_sync(0xFFFFFFFFu, act ? key_lo : (int32_t)0x80000000);
-    const uint32_t wt_min = __reduce_min_sync(0xFFFFFFFFu, act ? w_tail : 0xFFFFFFFFu);
-    const uint32_t wt_max = __reduce_max_sync(0xFFFFFFFFu, act ? w_tail : 0u);
-    // thresholds are non-negative floats or +inf: their bit patterns order like the values
-    const float th_min = __uint_as_float(__reduce_min_sync(0xFFFFFFFFu, act ? __float_as_uint(theta) : 0x7F800000u));
-    const float th_max = __uint_as_float(__reduce_max_sync(0xFFFFFFFFu, act ? __float_as_uint(theta) : 0u));
-    const int race_that_migrates = dev_migrates ? O_RACE_DEV : O_RACE_SRV;
-    (void)pmask;
-
     // One request per lane, fetched a batch ahead so that the loads fly while the previous batch is evaluated.
     struct Raw { uint32_t l, n, S, m, dly, stall, nt0, nt1, nt2, orig; };   // as loaded: nothing may consume a load early
-    auto fetch = [&](uint32_t b0) {
-        const uint32_t kk = ch.start + min(b0 + lane, ch.len - 1);
+    auto fetch = [&](uint32_t at) {                              // the request at position `at` of the chunk
+        const uint32_t kk = ch.start + min(at, r_hi - 1);
         Raw q;
         q.l = tr.l[kk]; q.n = tr.nout[kk]; q.S = (uint32_t)tr.S[kk];
         q.m = rec.m[kk]; q.dly = rec.delayed[kk]; q.stall = rec.stall[kk];
@@ -202,90 +175,22 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
         q.orig = EXT ? tr.orig[kk] : 0u;
         return q;
     };
-    Raw nx = fetch(min(wib * kStageReq, ch.len - 1));
-    for (uint32_t b0 = wib * kStageReq; b0 < ch.len; b0 += kAccWarps * kStageReq) {
-        // ---- 32 requests, one per lane
-        const Raw cur = nx;
-        if (b0 + kAccWarps * kStageReq < ch.len) nx = fetch(b0 + kAccWarps * kStageReq);
-        __syncwarp();
-        const bool valid = b0 + lane < ch.len;
-        const uint32_t l = cur.l, n = cur.n, S = cur.S, m = cur.m;
-        const uint32_t stall = cur.stall, dly = cur.dly;
-        const uint32_t nt0 = cur.nt0, nt1 = cur.nt1;
-        uint32_t nt2 = cur.nt2;
-        uint32_t stall_code = 0u;                          // the token after a hand-off: counted with tau's bin,
-        if (stall == tau) ++nt2; else stall_code = hist16_code(bin_of_ticks(stall));   // else an increment of its own
-        // a request may only migrate if its buffer filled (m != 0); fold that into the saving (Eq. 4)
-        const float saving = m ? delta_c * (float)(n - m) : -1.0f;
-        const uint32_t Td = kappa * l + c0, lm = l + m;
-
-        // ---- does the request end the same way under every policy of the tile?
-        bool uni = false;
-        int oc = O_SERVER_ONLY;
-        uint32_t ttft_u = S;
-        if (uni_ok) {
-            int base = -1;                                 // the race outcome before the migration trigger, if settled
-            if (kind == K_NOWAIT) {
-                if ((int32_t)l < len_min) { uni = true; oc = O_DEVICE_ONLY; ttft_u = Td; }   // below every l_th
-                else if ((int32_t)l >= len_max) {                                           // at or above every l_th: race at w = 0
-                    base = S > 0u ? (S > Td ? O_RACE_DEV : O_RACE_SRV) : O_SERVER_ONLY;
-                    ttft_u = min(S, Td);
-                }
-            } else if ((int32_t)l < len_min) {             // shorter than every l*: wait 0
-                base = S > 0u ? (S > Td ? O_RACE_DEV : O_RACE_SRV) : O_SERVER_ONLY;
-                ttft_u = min(S, Td);
-            } else if ((int32_t)l > len_max) {             // longer than every l*: each policy waits its w_tail
-                if (S <= wt_min) base = O_SERVER_ONLY;                         // the server answers within every wait
-                else if (S > wt_max) {                                         // the device starts under every policy
-                    if (S <= wt_min + Td) base = O_RACE_SRV;                   // ... and loses under every policy
-                    else if (wt_min == wt_max) { base = O_RACE_DEV; ttft_u = wt_min + Td; }
-                }
-            }
-            if (base >= 0) {
-                if (base != race_that_migrates || !(saving > th_min)) { uni = true; oc = base; }      // no policy hands over
-                else if (saving > th_max) { uni = true; oc = base + 2; }                            // every policy does
-            }
-        }
-        const bool settle = valid && uni;
-        {
-            // ---- the lane settles its request for the whole tile
-            const bool migr = oc >= O_MIGR_TO_DEV, dev_wins = (oc & 1) != 0, race = oc >= O_RACE_SRV;
-            const uint32_t u_td = !settle ? 0u : (migr ? (dev_wins ? m : n - m) : (dev_wins ? n : 0u));
-            const uint32_t u_ps = !settle || oc == O_DEVICE_ONLY ? 0u : l + ((migr && dev_wins) ? lm : 0u);
-            const uint32_t u_pd = !settle || oc == O_SERVER_ONLY ? 0u : l + ((migr && !dev_wins) ? lm : 0u);
-            const uint32_t u_tau = !settle ? 0u : (migr ? nt2 : (dev_wins ? nt1 : nt0));
-            const uint32_t u_dl = settle && migr ? dly : 0u;
-            const uint32_t u_cnt = !settle ? 0u : ((oc == O_DEVICE_ONLY ? 1u : 0u) | (race ? 0x100u : 0u) |
-                                                   (race && dev_wins ? 0x10000u : 0u) | (migr ? 0x1000000u : 0u));
-            const uint32_t u_tt = settle ? ttft_u : 0u;
-            const uint32_t settled = __ballot_sync(0xFFFFFFFFu, settle);
-            if (settled) {                                 // warp-uniform
-                if (settle) {
-                    hist16_add_ticks(hc_ttft, ttft_u);
-                    if (migr && stall_code) hist16_apply(hc_stall, stall_code);
-                }
-                const uint32_t r_td = __reduce_add_sync(0xFFFFFFFFu, u_td), r_ps = __reduce_add_sync(0xFFFFFFFFu, u_ps);
-                const uint32_t r_pd = __reduce_add_sync(0xFFFFFFFFu, u_pd), r_tau = __reduce_add_sync(0xFFFFFFFFu, u_tau);
-                const uint32_t r_dl = __reduce_add_sync(0xFFFFFFFFu, u_dl), r_cnt = __reduce_add_sync(0xFFFFFFFFu, u_cnt);
-                const uint32_t r_lo = __reduce_add_sync(0xFFFFFFFFu, u_tt & 0xFFFFu), r_hi = __reduce_add_sync(0xFFFFFFFFu, u_tt >> 16);
-                // Every policy of the tile gets these sums, so each policy lane adds them to its own (with fewer than
-                // 32 policies a policy has several lanes, whose sums are added up at the end: one of them takes it).
-                // At most 32 requests: the byte-packed counts cannot carry into each other.
-                if (slot == 0) {
-                    a_td += r_td; a_ps += r_ps; a_pd += r_pd; a_tau += r_tau; a_dl += r_dl;
-                    cnt_a += __byte_perm(r_cnt, 0u, 0x4140); cnt_b += __byte_perm(r_cnt, 0u, 0x4342);
-                    a_tt += ((unsigned long long)r_hi << 16) + r_lo;
-                }
-                if (lane == 0) atomicAdd(&s_work[0], (uint32_t)__popc(settled));
-            }
-        }
-        // ---- the other requests are staged, packed to the front, and evaluated pair by pair
-        const uint32_t mixed = __ballot_sync(0xFFFFFFFFu, valid && !uni);
-        if (mixed == 0u) continue;
-        const int n_here = __popc(mixed);
-        if (lane == 0) atomicAdd(&s_work[1], (uint32_t)n_here);
-        if (valid && !uni) {
-            const int at = __popc(mixed & ((1u << lane) - 1u));
+    // Stages the requests of the lanes in `taken`, packed to the front of the staging area, and evaluates them under
+    // the tile's policies.  b0: chunk position of lane 0's request when the lanes hold a batch in order.
+    auto run_batch = [&](const Raw& cur, uint32_t taken, uint32_t b0) {
+        const int n_here = __popc(taken);
+        staged += (uint32_t)n_here;
+        if ((taken >> lane) & 1u) {
+            const int at = __popc(taken & ((1u << lane) - 1u));
+            const uint32_t l = cur.l, n = cur.n, S = cur.S, m = cur.m;
+            const uint32_t stall = cur.stall, dly = cur.dly;
+            const uint32_t nt0 = cur.nt0, nt1 = cur.nt1;
+            uint32_t nt2 = cur.nt2;
+            uint32_t stall_code = 0u;                          // the token after a hand-off: counted with tau's bin,
+            if (stall == tau) ++nt2; else stall_code = hist16_code(bin_of_ticks(stall));   // else an increment of its own
+            // a request may only migrate if its buffer filled (m != 0); fold that into the saving (Eq. 4)
+            const float saving = m ? delta_c * (float)(n - m) : -1.0f;
+            const uint32_t Td = kappa * l + c0, lm = l + m;
             const uint32_t hS = hist16_code(bin_of_ticks(S)), hT = hist16_code(bin_of_ticks(Td));
             uint4* a = stA + at * kStageVec;
             uint4* b = stB + at * kStageVec;
@@ -402,6 +307,7 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
                     if (!kAllOk && !ok[k]) continue;
                     const int c = migr[k] ? 2 : (dev_wins[k] ? 1 : 0);
                     const int W = c == 2 ? W2 : (c == 1 ? W1 : W0), kt = c == 2 ? kt2 : (c == 1 ? kt1 : kt0);
+                    // (no bit mask with wide windows: the staged requests are the batch's first ones, in order)
                     const uint32_t* wp = rec.win[c] + (size_t)(ch.start + b0 + rr[k]) * W;
                     unsigned long long* hp = hist_tbt + (size_t)p * kNBins + cc.lo[g][c];
                     for (int j = 0; j < W; ++j) {
@@ -438,6 +344,43 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
             else pairs_of(std::integral_constant<int, K_ANY>{}, std::false_type{}, rr, ok);
         }
         cnt_a += __byte_perm(cnt8, 0u, 0x4140); cnt_b += __byte_perm(cnt8, 0u, 0x4342); cnt8 = 0;
+    };
+    if (!flagged_only) {
+        // ---- every request of the range: one per lane, fetched a batch ahead so that the loads fly while the
+        //      previous batch is evaluated
+        Raw nx = fetch(r_lo + wib * kStageReq + lane);
+        for (uint32_t b0 = r_lo + wib * kStageReq; b0 < r_hi; b0 += kAccWarps * kStageReq) {
+            const Raw cur = nx;
+            if (b0 + kAccWarps * kStageReq < r_hi) nx = fetch(b0 + kAccWarps * kStageReq + lane);
+            __syncwarp();
+            run_batch(cur, __ballot_sync(0xFFFFFFFFu, b0 + lane < r_hi), b0);
+        }
+    } else {
+        // ---- only the requests the zone kernel flagged for this tile: the warp reads the flags of 32 requests at a
+        //      time and collects the flagged ones, one per lane, until it holds (nearly) a full batch
+        uint32_t held = 0;                                       // chunk position of the request this lane holds
+        int n_held = 0;                                          // warp-uniform
+        auto work_off = [&]() {
+            const Raw d = fetch(held);                           // (lanes beyond n_held fetch a valid request and drop it)
+            __syncwarp();
+            run_batch(d, n_held == 32 ? 0xFFFFFFFFu : (1u << n_held) - 1u, 0u);
+            n_held = 0;
+        };
+        uint32_t nf = left_mask[(size_t)(ch.start + min(r_lo + wib * kStageReq + lane, r_hi - 1)) * mask_words + (tile >> 5)];
+        for (uint32_t b0 = r_lo + wib * kStageReq; b0 < r_hi; b0 += kAccWarps * kStageReq) {
+            const uint32_t flags = nf;
+            if (b0 + kAccWarps * kStageReq < r_hi)
+                nf = left_mask[(size_t)(ch.start + min(b0 + kAccWarps * kStageReq + lane, r_hi - 1)) * mask_words + (tile >> 5)];
+            const uint32_t taken = __ballot_sync(0xFFFFFFFFu, b0 + lane < r_hi && (flags & mask_bit) != 0u);
+            if (taken == 0u) continue;
+            const int n_new = __popc(taken);
+            if (n_held + n_new > 32) work_off();
+            const int want = lane - n_held;                      // lane n_held + j takes the j-th flagged request
+            if (want >= 0 && want < n_new) held = b0 + __fns(taken, 0, want + 1);
+            n_held += n_new;
+            if (n_held >= 28) work_off();
+        }
+        if (n_held > 0) work_off();
     }
     // ---- block totals, then one flush per block.  With fewer than 32 policies in the tile several lanes of a warp
     //      hold sums of the same policy: they are added up by shuffles first, so that one lane per policy and warp
@@ -463,26 +406,17 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
         const uint32_t hi = (uint32_t)(a_tt >> 32) + (before + lo < before ? 1u : 0u);
         if (hi) atomicAdd(&a[2 * A_TTFT_SUM + 1], hi);
     }
+    if (work && lane == 0 && staged) atomicAdd(&work[1], (unsigned long long)staged * pols_here);   // pairs evaluated one by one
     __syncthreads();
-    // every policy of the tile also gets the histograms of the requests settled for the whole tile
-    const int pols_here = (int)min((uint32_t)PL, n_list - tile * PL);
     const int bin_tau = bin_of_ticks(tau);
     for (int i = threadIdx.x; i < pols_here * kHWords; i += kAccThreads) {
         const int pi = i / kHWords, wd = i - pi * kHWords;
         const size_t o = (size_t)pol_list[tile * PL + pi] * kNBins + 2 * wd;
         const uint32_t a = h_ttft[pi * kHWords + wd], b = h_stall[pi * kHWords + wd];
-        const uint32_t ca = hc_ttft[wd], cb = hc_stall[wd];
-        const uint32_t a0 = (a & 0xFFFFu) + (ca & 0xFFFFu), a1 = (a >> 16) + (ca >> 16);
-        const uint32_t b0 = (b & 0xFFFFu) + (cb & 0xFFFFu), b1 = (b >> 16) + (cb >> 16);
-        if (a0) atomicAdd(&hist_ttft[o], (unsigned long long)a0);
-        if (a1) atomicAdd(&hist_ttft[o + 1], (unsigned long long)a1);
-        if (b0) atomicAdd(&hist_tbt[o], (unsigned long long)b0);
-        if (b1) atomicAdd(&hist_tbt[o + 1], (unsigned long long)b1);
-    }
-    if (threadIdx.x == 0 && work) {
-        atomicAdd(&work[0], (unsigned long long)s_work[0] * pols_here);             // pairs settled tile-wide
-        atomicAdd(&work[1], (unsigned long long)s_work[1] * pols_here);             // pairs evaluated one by one
-        atomicAdd(&work[2], (unsigned long long)s_work[0]);                         // requests settled, per tile
+        if (a & 0xFFFFu) atomicAdd(&hist_ttft[o], (unsigned long long)(a & 0xFFFFu));
+        if (a >> 16) atomicAdd(&hist_ttft[o + 1], (unsigned long long)(a >> 16));
+        if (b & 0xFFFFu) atomicAdd(&hist_tbt[o], (unsigned long long)(b & 0xFFFFu));
+        if (b >> 16) atomicAdd(&hist_tbt[o + 1], (unsigned long long)(b >> 16));
     }
     for (int i = threadIdx.x; i < pols_here * kNAcc; i += kAccThreads) {
         const int pi = i / kNAcc, s = i - pi * kNAcc;
@@ -492,6 +426,8 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
         if (s == A_TAU_CNT) atomicAdd(&hist_tbt[(size_t)pp * kNBins + bin_tau], v);   // TBTs equal to tau
         else atomicAdd(&acc[((size_t)pp * tr.n_groups + g) * kNAcc + s], v);
     }
+    __syncthreads();
+    }   // next pass
 }
 
 size_t acc_smem_bytes(int PL) {
@@ -644,8 +580,8 @@ k_pairs_rows(TraceDev tr, const GroupConst* __restrict__ gcs, const Prep* __rest
 cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const Prep* prep, uint32_t P,
                          const uint32_t* pol_list, uint32_t n_list, const Chunk* chunks, uint32_t n_chunks,
                          TimelineRec rec, disco_pair_out_t out, uint64_t* acc, uint64_t* hist_ttft,
-                         uint64_t* hist_tbt, uint64_t* work, uint32_t k0, bool extras, bool wide, cudaEvent_t mid,
-                         cudaStream_t st) {
+                         uint64_t* hist_tbt, uint32_t* left_mask, uint32_t* left_count, uint64_t* work, uint32_t k0,
+                         bool extras, bool wide, cudaEvent_t mid, cudaStream_t st) {
     if (n_chunks == 0 || n_list == 0) return mid ? cudaEventRecord(mid, st) : cudaSuccess;
     int PL = 1;
     while (PL < 32 && (uint32_t)PL < n_list) PL <<= 1;
@@ -656,9 +592,20 @@ cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassCo
     if (e) return e;
     const uint32_t n_tiles = (n_list + PL - 1) / PL;
     if ((uint64_t)n_chunks * n_tiles > 0x7FFFFFFFull) return cudaErrorInvalidConfiguration;
+    // zone by zone first (tiles it cannot take return at once), then pair by pair what is left
+    const bool zones = !wide && left_mask != nullptr;
+    if (zones) {
+        const size_t mask_bytes = (size_t)tr.n * left_words_per_request(n_tiles) * 4;
+        if ((e = cudaMemsetAsync(left_mask, 0, mask_bytes, st))) return e;
+        if ((e = launch_pairs_zones(tr, gc, cc, prep, P, pol_list, n_list, PL, chunks, n_chunks, rec, acc, hist_ttft,
+                                    hist_tbt, left_mask, left_count, work, st)))
+            return e;
+    }
     if ((e = launch_after(acc_kernel, dim3(n_chunks * n_tiles), kAccThreads, acc_smem_bytes(PL), st, tr, gc, cc, prep, P,
                           pol_list, n_list, PL, chunks, n_tiles, rec, k0, (unsigned long long*)acc,
-                          (unsigned long long*)hist_ttft, (unsigned long long*)hist_tbt, (unsigned long long*)work)))
+                          (unsigned long long*)hist_ttft, (unsigned long long*)hist_tbt,
+                          (const uint32_t*)(zones ? left_mask : nullptr), (const uint32_t*)left_count,
+                          (unsigned long long*)work)))
         return e;
     if (mid && (e = cudaEventRecord(mid, st))) return e;
     const bool rows = out.ttft_s || out.tbt_mean_s || out.tbt_max_s || out.cost || out.tok_server || out.tok_device ||
