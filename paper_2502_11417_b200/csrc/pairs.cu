@@ -366,19 +366,27 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
             run_batch(d, n_held == 32 ? 0xFFFFFFFFu : (1u << n_held) - 1u, 0u);
             n_held = 0;
         };
-        uint32_t nf = left_mask[(size_t)(ch.start + min(r_lo + wib * kStageReq + lane, r_hi - 1)) * mask_words + (tile >> 5)];
-        for (uint32_t b0 = r_lo + wib * kStageReq; b0 < r_hi; b0 += kAccWarps * kStageReq) {
-            const uint32_t flags = nf;
-            if (b0 + kAccWarps * kStageReq < r_hi)
-                nf = left_mask[(size_t)(ch.start + min(b0 + kAccWarps * kStageReq + lane, r_hi - 1)) * mask_words + (tile >> 5)];
-            const uint32_t taken = __ballot_sync(0xFFFFFFFFu, b0 + lane < r_hi && (flags & mask_bit) != 0u);
-            if (taken == 0u) continue;
-            const int n_new = __popc(taken);
-            if (n_held + n_new > 32) work_off();
-            const int want = lane - n_held;                      // lane n_held + j takes the j-th flagged request
-            if (want >= 0 && want < n_new) held = b0 + __fns(taken, 0, want + 1);
-            n_held += n_new;
-            if (n_held >= 28) work_off();
+        constexpr int kScan = 4;                                 // flag words a lane has in flight
+        constexpr uint32_t kStride = kAccWarps * kStageReq;
+        auto flags_at = [&](uint32_t at) {
+            return at < r_hi ? left_mask[(size_t)(ch.start + at) * mask_words + (tile >> 5)] & mask_bit : 0u;
+        };
+        for (uint32_t c0 = r_lo + wib * kStageReq; c0 < r_hi; c0 += kScan * kStride) {
+            const uint32_t f0 = flags_at(c0 + lane), f1 = flags_at(c0 + kStride + lane);
+            const uint32_t f2 = flags_at(c0 + 2 * kStride + lane), f3 = flags_at(c0 + 3 * kStride + lane);
+            static_assert(kScan == 4, "four flag words are loaded by name");
+#pragma unroll 1
+            for (int j = 0; j < kScan; ++j) {                    // (not unrolled: the batch evaluation is long code)
+                const uint32_t b0 = c0 + j * kStride;
+                const uint32_t taken = __ballot_sync(0xFFFFFFFFu, (j == 0 ? f0 : j == 1 ? f1 : j == 2 ? f2 : f3) != 0u);
+                if (taken == 0u) continue;
+                const int n_new = __popc(taken);
+                if (n_held + n_new > 32) work_off();
+                const int want = lane - n_held;                  // lane n_held + j takes the j-th flagged request
+                if (want >= 0 && want < n_new) held = b0 + __fns(taken, 0, want + 1);
+                n_held += n_new;
+                if (n_held >= 28) work_off();
+            }
         }
         if (n_held > 0) work_off();
     }

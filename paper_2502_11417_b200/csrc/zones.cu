@@ -31,8 +31,10 @@ constexpr int kZThreads = 1024;
 static_assert(kZThreads == 1024, "the flush assigns its work to threads 0 .. 1023 by index");
 constexpr int kZWarps = kZThreads / 32;
 constexpr int kZRows = 33;              // difference rows: row q is carried to the policies below q, q = 1 .. 32
-constexpr uint32_t kZPass = 32640;      // requests between two flushes of a block
-constexpr uint32_t kZMaxItems = 16000;  // queued requests between two flushes: a 16-bit count moves by at most 2 each
+// Requests between two flushes of a block.  A signed 16-bit count of the difference rows moves by at most one per
+// queued request under Algorithm 3 (one boundary) and by at most two under Algorithm 2 (a boundary and a policy of
+// its own at the same row), and every request of a pass may be queued.
+constexpr uint32_t kZPass = 32640, kZPassWaits = 16320;
 constexpr int kZQueue = 64;             // queue slots per warp
 enum ZSum { Z_TD = 0, Z_PS, Z_PD, Z_TAU, Z_DL, Z_CNT_A, Z_CNT_B, Z_TT_LO, Z_TT_HI, kZSums };
 constexpr int kZSumStride = 12;
@@ -50,6 +52,7 @@ struct ZoneSmem {
     uint32_t queue[kZWarps][kZQueue];   // requests (chunk-relative) that await their corrections
     int32_t key[32];                    // the policies' length thresholds, in tile order
     uint32_t w_star[32];                // Algorithm 2: the wait of the length class l*
+    uint32_t w_tail[32];                // ... and of the longer prompts
     float theta[32];                    // Eq. 4's overhead (+inf: the policy never hands over)
     uint32_t pol[32];                   // the policies' indices in the caller's list
     uint8_t tab1[kLenTab], tab2[kLenTab];
@@ -87,6 +90,7 @@ struct TileCtx {
     float delta_c, th_min, th_max;
     int npol, race_that_migrates, W0, W1, W2, kt0, kt1, kt2;
     bool may_migrate;
+    bool wt_ordered;                    // the policies' w_tail do not increase along the tile
 };
 
 template <bool LEAN>
@@ -137,17 +141,26 @@ __device__ __forceinline__ bool tail_outcome(const TileCtx& c, const Req& q, uin
     return t >= 0;
 }
 
-// The run of Algorithm 2 policies that wait their w_tail.  Returns false if the policies disagree.
-__device__ __forceinline__ bool head_outcome_waits(const TileCtx& c, const Req& q, uint32_t Td, float saving, int& oc,
-                                                   uint32_t& tt) {
-    int base = -1;
+// The run of Algorithm 2 policies [0, k1) that wait their w_tail.  On success the policies [j, k1) end in
+// (oc, tt) and the policies [0, j), whose longer waits cover the server's TTFT, in O_SERVER_ONLY with the same
+// TTFT (j = 0: none).  Returns false if the run cannot be expressed that way.
+__device__ __forceinline__ bool head_outcome_waits(const TileCtx& c, const ZoneSmem& sm, const Req& q, uint32_t Td,
+                                                   float saving, int k1, int& oc, uint32_t& tt, int& j) {
+    int base;
     tt = q.S;
+    j = 0;
     if (q.S <= c.wt_min) base = O_SERVER_ONLY;                                 // the server answers within every wait
-    else if (q.S > c.wt_max) {                                                 // the device starts under every policy
-        if (q.S <= c.wt_min + Td) base = O_RACE_SRV;                           // ... and loses under every policy
-        else if (c.wt_min == c.wt_max) { base = O_RACE_DEV; tt = c.wt_min + Td; }
-    }
-    if (base < 0) return false;
+    else if (q.S <= c.wt_min + Td) {                                           // whoever starts the device loses the race
+        base = O_RACE_SRV;
+        if (q.S <= c.wt_max) {                                                 // some waits cover S: those policies first
+            if (!c.wt_ordered) return false;
+            int lo = 0, hi = k1;
+            while (lo < hi) { const int mid = (lo + hi) >> 1; if (sm.w_tail[mid] >= q.S) lo = mid + 1; else hi = mid; }
+            j = lo;
+            if (j == k1) { base = O_SERVER_ONLY; j = 0; }                      // every wait of the run covers S
+        }
+    } else if (c.wt_min == c.wt_max) { base = O_RACE_DEV; tt = c.wt_min + Td; }   // the device wins under every policy
+    else return false;
     const int t = trigger_all(c, base, saving);
     oc = base + 2 * t;
     return t >= 0;
@@ -188,14 +201,14 @@ __device__ __forceinline__ void drain_queue(ZoneSmem& sm, const TileCtx& c, cons
         const uint32_t Td = c.kappa * q.l + c.c0;
         const float saving = saving_of(c, q);
         const int k1 = sm.tab1[q.l], k2 = WAITS ? sm.tab2[q.l] : k1;
-        int oc_b, oc_h = O_DEVICE_ONLY;
+        int oc_b, oc_h = O_DEVICE_ONLY, j = 0;
         uint32_t tt_b, tt_h = Td;
         tail_outcome(c, q, Td, saving, oc_b, tt_b);              // (every run was settled when the request was queued)
-        if (k1 > 0) {
-            if (WAITS) head_outcome_waits(c, q, Td, saving, oc_h, tt_h);
-            enter_difference(sm, k1, 1u, q, stall_code, oc_h, tt_h, oc_b, tt_b);
-        }
-        if (WAITS) {
+        if (WAITS && k1 > 0) head_outcome_waits(c, sm, q, Td, saving, k1, oc_h, tt_h, j);
+        if (k2 >= c.npol) { oc_b = oc_h; tt_b = tt_h; }          // every policy is in the first run: it is the common part
+        else if (k1 > 0) enter_difference(sm, k1, 1u, q, stall_code, oc_h, tt_h, oc_b, tt_b);
+        if (j > 0) enter_difference(sm, j, 1u, q, stall_code, O_SERVER_ONLY, q.S, oc_h, tt_h);
+        if (WAITS && k2 < c.npol) {
             for (int p = k1; p < k2; ++p) {                      // policies whose l* is this length: their own wait
                 const uint32_t w = sm.w_star[p];
                 int oc = O_SERVER_ONLY;
@@ -246,11 +259,13 @@ __device__ __forceinline__ void zone_pass(ZoneSmem& sm, const TileCtx& c, uint32
         if (k2 < npol) {
             ok = tail_outcome(c, q, Td, saving, oc_all, tt_all);
             later = k2 > 0;                                      // a first run, or policies with l* = l
-            if (WAITS && k1 > 0) { int oc; uint32_t tt; ok = head_outcome_waits(c, q, Td, saving, oc, tt) && ok; }
+            if (WAITS && k1 > 0) { int oc, j; uint32_t tt; ok = head_outcome_waits(c, sm, q, Td, saving, k1, oc, tt, j) && ok; }
         } else if (k1 < npol) {
             ok = false;                                          // l* = l for the last policies and nobody waits 0
         } else if (WAITS) {
-            ok = head_outcome_waits(c, q, Td, saving, oc_all, tt_all);       // every policy waits its w_tail
+            int j;                                               // every policy waits its w_tail
+            ok = head_outcome_waits(c, sm, q, Td, saving, k1, oc_all, tt_all, j);
+            later = j > 0;
         }
         ok = ok && valid;
         // a place in the block's budget of corrections
@@ -259,7 +274,7 @@ __device__ __forceinline__ void zone_pass(ZoneSmem& sm, const TileCtx& c, uint32
             uint32_t place = 0;
             if (lane == 0) place = atomicAdd(&sm.n_items, (uint32_t)__popc(wants));
             place = __shfl_sync(0xFFFFFFFFu, place, 0) + __popc(wants & ((1u << lane) - 1u));
-            if (later && place >= kZMaxItems) ok = false;        // the difference rows are full: the pair kernel's
+            if (later && place >= kZPass) ok = false;            // (cannot happen: a pass is no longer than the budget)
         }
         if (valid && !ok) {
             atomicOr(&left_mask[(size_t)(c.ch->start + i) * words + (tile >> 5)], left_bit);
@@ -351,10 +366,15 @@ k_pairs_zones(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst*
     c.wt_min = __reduce_min_sync(0xFFFFFFFFu, act ? (uint32_t)pr.w_tail : 0xFFFFFFFFu);
     c.wt_max = __reduce_max_sync(0xFFFFFFFFu, act ? (uint32_t)pr.w_tail : 0u);
     c.may_migrate = c.th_min != __int_as_float(0x7F800000);      // some policy of the tile can hand over
+    {
+        const uint32_t next = __shfl_down_sync(0xFFFFFFFFu, (uint32_t)pr.w_tail, 1);
+        c.wt_ordered = __all_sync(0xFFFFFFFFu, lane + 1 >= npol || (uint32_t)pr.w_tail >= next) != 0;
+    }
 
     if (wib == 0 && lane < npol) {
         sm.key[lane] = waits ? pr.l_star : pr.l_th;
         sm.w_star[lane] = (uint32_t)pr.w_star;
+        sm.w_tail[lane] = (uint32_t)pr.w_tail;
         sm.theta[lane] = theta;
         sm.pol[lane] = pol_list[pol_idx];
     }
@@ -378,8 +398,9 @@ k_pairs_zones(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst*
     const int bin_tau = bin_of_ticks(c.tau);
     uint32_t left_total = 0, items_total = 0;
 
-    for (uint32_t r_lo = 0; r_lo < ch.len; r_lo += kZPass) {
-        const uint32_t r_hi = min(ch.len, r_lo + kZPass);
+    const uint32_t pass_len = waits ? kZPassWaits : kZPass;
+    for (uint32_t r_lo = 0; r_lo < ch.len; r_lo += pass_len) {
+        const uint32_t r_hi = min(ch.len, r_lo + pass_len);
         for (int i = threadIdx.x; i < (int)(offsetof(ZoneSmem, queue) / 4); i += kZThreads) ((uint32_t*)zsmem_raw)[i] = 0;
         __syncthreads();
         if (waits) {
@@ -391,7 +412,7 @@ k_pairs_zones(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst*
         }
         __syncthreads();
         left_total += sm.n_left;
-        items_total += min(sm.n_items, kZMaxItems);
+        items_total += sm.n_items;
         // ---- flush: policy p gets the common part plus the difference rows above it (rows q > p)
         //      (two threads a histogram word: one for the upper half of the policies, one for the lower half)
         if ((threadIdx.x & 511) < kHWords) {
