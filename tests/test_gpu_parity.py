@@ -399,3 +399,52 @@ def test_invalid_inputs_are_rejected():
     with pytest.raises(DiscoError) as ei:
         t2.eval_policies([synth.policy(0.5, r_c=2.0)], 0)
     assert ei.value.code == -1
+
+
+def _work(w, pols):
+    tr = Trace.from_workload(w)
+    tr.eval_policies(pols, w.seed)
+    tr.reduce_stats()
+    counts = tr.work_counts()
+    tr.close()
+    return counts
+
+
+def test_zone_by_zone_reduction_and_what_it_leaves_to_the_pair_kernel():
+    # ascending budgets: a tile's policies are ordered, so requests are settled against runs of policies; what the
+    # runs cannot express goes pair by pair.  Every variant must give the oracle's numbers.
+    for dear in (False, True):                     # Algorithm 3 tiles, Algorithm 2 tiles
+        w = synth.tiny_workload(51 + dear, 6000, n_servers=2, n_devices=1, max_prompt=900, max_out=160, device_dearer=dear)
+        grid = synth.budget_grid(40)
+        # one overhead per tile: nothing but the odd request is left over
+        plain = [synth.policy(b, mig_threshold=0.004) for b in grid]
+        full_parity(w, plain, tag=f"zones plain dear={dear}")
+        zone, left, _, corr = _work(w, plain)
+        assert zone > 0.9 * w.n * len(plain) and corr > 0
+        # overheads that alternate inside a tile: requests whose saving lies between them are left to the pair kernel
+        mixed = [synth.policy(b, mig_threshold=(0.0, 0.05, synth.INF)[k % 3]) for k, b in enumerate(grid)]
+        full_parity(w, mixed, tag=f"zones mixed overheads dear={dear}")
+        zone, left, _, _ = _work(w, mixed)
+        assert zone > 0 and left > 0
+        # many budgets at or below the tail ratio (each its own w_tail), and budgets that repeat (equal thresholds)
+        low = [synth.policy(b, alpha=0.3) for b in sorted(list(synth.budget_grid(24)) + [0.1, 0.1, 0.5, 0.5, 0.5])]
+        full_parity(w, low, tag=f"zones low budgets dear={dear}")
+        # descending budgets: the thresholds are not ordered, the whole tile goes pair by pair
+        down = plain[::-1]
+        full_parity(w, down, tag=f"zones descending dear={dear}")
+        zone, left, _, _ = _work(w, down)
+        assert left > 0.5 * w.n * len(down)
+        # pacing off: no zone kernel at all
+        nopace = [synth.policy(b, flags=MIG) for b in grid]
+        full_parity(w, nopace, tag=f"zones pacing off dear={dear}")
+        assert _work(w, nopace)[0] == 0
+
+
+def test_more_than_32_policy_tiles_use_several_flag_words():
+    # 1100 policies = 35 tiles: two flag words per request; overheads alternate so that requests are flagged in
+    # tiles of both words
+    w = synth.tiny_workload(61, 1500, n_servers=1, n_devices=2, max_prompt=700, max_out=120, device_dearer=True)
+    pols = [synth.policy(b, mig_threshold=(0.0, 0.03)[k % 2]) for k, b in enumerate(synth.budget_grid(1100))]
+    full_parity(w, pols, select=False, tag="35 tiles")
+    zone, left, _, _ = _work(w, pols)
+    assert zone > 0 and left > 0
