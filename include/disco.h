@@ -93,9 +93,11 @@ typedef struct {
     uint32_t n_devices;
     uint32_t arrays_on_device;        /* 0: the five [n] arrays are host memory; 1: device memory.  Host arrays that
                                          are all page-locked (cudaHostAlloc, cudaHostRegister) are read by the
-                                         ingestion kernel in place when the trace has one profile group; otherwise
-                                         they are copied to the device first.  Either way they may be reused as soon
-                                         as disco_load_trace returns. */
+                                         ingestion kernel in place; pageable ones are copied to the device first.
+                                         Either way they may be reused as soon as disco_load_trace returns.
+                                         2: host memory that is always copied first, by the copy engine: the transfer
+                                         then leaves the multiprocessors free, so that it can run beside the kernels
+                                         of another context (a second worker evaluating the previous trace). */
     uint64_t first_index;             /* index, in the whole trace, of request 0 of these arrays: 0 unless the arrays
                                          are a contiguous range (a shard) of a larger trace.  The per-token jitter hash
                                          is keyed by the request's index in the whole trace, so a shard loaded with its
@@ -242,6 +244,14 @@ uint64_t disco_kernel_launch_count(void);
  * requests settled zone by zone, counted once per tile; those of them that needed corrections below a run
  * boundary.  The first two add up to requests x policies.  Synchronises `stream`. */
 int disco_get_work_counts(disco_ctx_t* ctx, uint64_t* counts4, void* stream);
+
+/* Checked build.  Compiled with -DDISCO_DEBUG the library checks every index its kernels derive (request, policy,
+ * group, chunk, knot, histogram bin, window and staging slot, table entry) against its bound before the access; an
+ * index out of range is recorded and the access skipped -- nothing traps -- and the next call that synchronises
+ * returns DISCO_ECUDA with the kernel's name and the index in disco_last_error().  disco_debug_selftest shows that
+ * the checks are live: it has a kernel offer an out-of-range index (the access is never made) and returns the
+ * DISCO_ECUDA that follows; in an ordinary build it returns DISCO_EINVAL. */
+int disco_debug_selftest(void* stream);
 
 /* Measures what the GPU sustains on the integer instruction mix of the token loop (Sec. 4.3 play-out: per
  * token one counter add, the hash finaliser's three shift-xor pairs and two multiplies, one multiply-high

@@ -87,8 +87,12 @@ def lib() -> C.CDLL:
     global _lib
     if _lib is None:
         # DISCO_ORACLE_LIB: a library built elsewhere from a deliberately broken copy of the source (the mutation
-        # check of the pins, tests/oracle_mutants.py); never set in ordinary runs
-        L = C.CDLL(os.environ.get("DISCO_ORACLE_LIB") or build_oracle())
+        # check of the pins, tests/oracle_mutants.py).  It is honoured only together with the marker that script
+        # sets, so that a stray variable cannot swap the checker under an ordinary test run.
+        swapped = os.environ.get("DISCO_ORACLE_LIB")
+        if swapped and os.environ.get("DISCO_ORACLE_MUTATION_CHECK") != "1":
+            raise RuntimeError("DISCO_ORACLE_LIB is set outside the mutation check (tests/oracle_mutants.py)")
+        L = C.CDLL(swapped or build_oracle())
         L.orc_mix.restype = C.c_uint32; L.orc_mix.argtypes = [C.c_uint32]
         L.orc_hash.restype = C.c_uint32; L.orc_hash.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32]
         L.orc_jitter.restype = C.c_int64; L.orc_jitter.argtypes = [C.c_uint32, C.c_int64]

@@ -78,7 +78,7 @@ EXPORTS = ["disco_load_trace", "disco_eval_policies", "disco_reduce_stats", "dis
            "disco_last_error", "disco_set_timing", "disco_get_timing", "disco_kernel_launch_count",
            "disco_sort_ttft_ticks_noalloc", "disco_select_policy_device", "disco_set_group_tables",
            "disco_accumulator_words", "disco_export_accumulators", "disco_import_accumulators",
-           "disco_measure_alu_peak", "disco_get_work_counts"]
+           "disco_measure_alu_peak", "disco_get_work_counts", "disco_debug_selftest"]
 
 PAIR_FIELDS = [("ttft_s", "float32"), ("tbt_mean_s", "float32"), ("tbt_max_s", "float32"), ("cost", "float32"),
                ("tok_server", "uint32"), ("tok_device", "uint32"), ("mig_at", "uint32"), ("delayed", "uint16"),
@@ -92,10 +92,11 @@ def library_path() -> str:
 
 
 def lib() -> C.CDLL:
-    """Loads libdisco.so (building it first if the sources are newer).  Raises if it cannot be had."""
+    """Loads libdisco.so (building it first if the sources are newer).  Raises if it cannot be had.  With
+    DISCO_CHECKED_BUILD=1 in the environment the index-checking variant (-DDISCO_DEBUG) is built and loaded instead."""
     global _lib
     if _lib is None:
-        path = _build.build()
+        path = _build.build(checked=os.environ.get("DISCO_CHECKED_BUILD") == "1")
         L = C.CDLL(path)
         vp, u32, u64 = C.c_void_p, C.c_uint32, C.c_uint64
         L.disco_load_trace.restype = C.c_int; L.disco_load_trace.argtypes = [C.POINTER(vp), vp, vp]
@@ -110,6 +111,7 @@ def lib() -> C.CDLL:
         L.disco_export_accumulators.restype = C.c_int; L.disco_export_accumulators.argtypes = [vp, vp, vp]
         L.disco_import_accumulators.restype = C.c_int; L.disco_import_accumulators.argtypes = [vp, vp, vp]
         L.disco_get_work_counts.restype = C.c_int; L.disco_get_work_counts.argtypes = [vp, vp, vp]
+        L.disco_debug_selftest.restype = C.c_int; L.disco_debug_selftest.argtypes = [vp]
         L.disco_measure_alu_peak.restype = C.c_int
         L.disco_measure_alu_peak.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_double), vp]
         L.disco_get_histograms.restype = C.c_int; L.disco_get_histograms.argtypes = [vp, u32, vp, vp, vp]
@@ -247,10 +249,11 @@ class Trace:
 
     # -- disco_load_trace ---------------------------------------------------------------------------------
     def load_trace(self, prompt_len, output_len, server_ttft_s, server_profile, device_profile, servers, devices,
-                   stream=None, first_index: int = 0):
+                   stream=None, first_index: int = 0, staged_copy: bool = False):
         """Arrays may be numpy arrays / pinned CPU tensors (host memory) or CUDA tensors (device memory),
         all of the same kind.  Reloading reuses the context's device memory.  first_index: position of these
-        arrays' first request in the whole trace when they are a shard of it."""
+        arrays' first request in the whole trace when they are a shard of it.  staged_copy: host arrays are copied
+        by the copy engine even when they are page-locked (instead of being read in place by the ingestion kernel)."""
         import torch
         _require_cuda()
         arrs = [prompt_len, output_len, server_ttft_s, server_profile, device_profile]
@@ -279,7 +282,8 @@ class Trace:
         n = int(len(prompt_len))
         sv, dv = server_array(servers), device_array(devices)
         desc = TraceDesc(n, ptrs[0], ptrs[1], ptrs[2], ptrs[3], ptrs[4], C.cast(sv, C.c_void_p), len(servers),
-                         C.cast(dv, C.c_void_p), len(devices), 1 if on_dev else 0, int(first_index))
+                         C.cast(dv, C.c_void_p), len(devices), 1 if on_dev else (2 if staged_copy else 0),
+                         int(first_index))
         _check(lib().disco_load_trace(C.byref(self._h), C.byref(desc), _stream_ptr(stream)))
         self.n = n
         self.n_groups = len(servers) * len(devices)

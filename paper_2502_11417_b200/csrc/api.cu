@@ -53,7 +53,40 @@ using HostReadback = LoadReadback;   // pinned host mirror of the load's read-ba
 
 namespace disco {
 int set_error(int code, const char* msg) { return fail(code, msg); }
+
+#ifdef DISCO_DEBUG
+namespace {
+std::vector<cudaError_t (*)(int32_t*)>& dbg_readers() { static std::vector<cudaError_t (*)(int32_t*)> v; return v; }
+}  // namespace
+void dbg_register(cudaError_t (*reader)(int32_t*)) { dbg_readers().push_back(reader); }
+#endif
 }  // namespace disco
+
+namespace {
+// Checked build: after a call has synchronised, asks every translation unit for an index its kernels refused.
+// Returns 0, or DISCO_ECUDA with the kernel and the index in the error string.
+int debug_check() {
+#ifdef DISCO_DEBUG
+    static const char* kernels[DBG_K_COUNT] = {"", "k_ingest", "radix sort", "k_gather", "group tables", "k_prep",
+                                               "k_playout_fast", "k_playout", "k_pairs_acc", "k_pairs_zones", "k_pairs_rows",
+                                               "k_finalize", "k_select", "self-test"};
+    static const char* whats[DBG_WHAT_COUNT] = {"", "request", "policy", "group", "chunk", "knot", "histogram bin",
+                                                "window slot", "staging slot", "table entry", "counter", "element"};
+    for (auto reader : disco::dbg_readers()) {
+        int32_t w[4] = {0, 0, 0, 0};
+        const cudaError_t e = reader(w);
+        if (e != cudaSuccess) return fail_cuda(e, "reading the checked build's record");
+        if (w[0]) {
+            const char* k = w[0] > 0 && w[0] < DBG_K_COUNT ? kernels[w[0]] : "?";
+            const char* t = w[1] > 0 && w[1] < DBG_WHAT_COUNT ? whats[w[1]] : "?";
+            return fail(DISCO_ECUDA, std::string("checked build: ") + k + " refused " + t + " index " + std::to_string(w[2]) +
+                                         " (bound " + std::to_string(w[3]) + ")");
+        }
+    }
+#endif
+    return 0;
+}
+}  // namespace
 
 struct disco_ctx {
     uint32_t n = 0, ns = 0, nd = 0;
@@ -64,7 +97,7 @@ struct disco_ctx {
     const void* gc_dev_at = nullptr;
     // trace
     DevBuf in_prompt, in_out, in_ttft, in_sp, in_dp;      // staging of host inputs
-    DevBuf keys_a, keys_b, tmp_idx;
+    DevBuf keys_a, keys_b, tmp_idx, tmp_ln;
     DevBuf S, l, nout, orig, sorted;
     DevBuf zero, cum_mass, ng_exact, grp_off, knots, d_gc;   // `zero`: every table a load must clear, contiguous
     DevBuf fin_totals;                 // [2G] u64: output tokens and requests per group that the accumulators cover
@@ -104,7 +137,7 @@ struct disco_ctx {
     bool timing_valid = false;
 
     ~disco_ctx() {
-        DevBuf* all[] = {&in_prompt, &in_out, &in_ttft, &in_sp, &in_dp, &keys_a, &keys_b, &tmp_idx,
+        DevBuf* all[] = {&in_prompt, &in_out, &in_ttft, &in_sp, &in_dp, &keys_a, &keys_b, &tmp_idx, &tmp_ln,
                          &S, &l, &nout, &orig, &sorted, &zero, &cum_mass, &ng_exact, &grp_off, &knots, &d_gc, &d_prep, &d_accum, &d_stats, &d_tables, &d_todo,
                          &fin_totals, &F_sorted_imp, &F_off_imp, &d_left};
         for (DevBuf* b : all) b->release();
@@ -172,6 +205,7 @@ cudaError_t reserve_trace(disco_ctx* c, uint32_t n, bool host_inputs, bool has_s
         if (has_dp) R(in_dp, N);
     }
     R(keys_a, N * 8); R(keys_b, N * 8); R(tmp_idx, N * 4);
+    if (G > 1) R(tmp_ln, N * 4);
     R(S, N * 4); R(l, N * 2); R(nout, N * 2); R(orig, N * 4); R(sorted, N * 4);
     // one block for everything a load clears: cnt | grp_sum_n | ng | max_n | err | first radix counter buffer,
     // followed by the second counter buffer
@@ -194,6 +228,10 @@ cudaError_t reserve_trace(disco_ctx* c, uint32_t n, bool host_inputs, bool has_s
 
 }  // namespace
 
+namespace disco {
+int check_debug_record() { return debug_check(); }
+}  // namespace disco
+
 extern "C" {
 
 const char* disco_last_error(void) { return g_err.c_str(); }
@@ -204,7 +242,7 @@ int disco_load_trace(disco_ctx_t** pctx, const disco_trace_desc_t* d, void* stre
     if (!pctx || !d) return fail(DISCO_EINVAL, "null argument");
     if (d->n >= (1ull << 31)) return fail(DISCO_EINVAL, "too many requests");
     if (d->n && (!d->prompt_len || !d->output_len || !d->server_ttft_s)) return fail(DISCO_EINVAL, "null trace array");
-    if (d->arrays_on_device > 1) return fail(DISCO_EINVAL, "arrays_on_device must be 0 or 1");
+    if (d->arrays_on_device > 2) return fail(DISCO_EINVAL, "arrays_on_device must be 0, 1 or 2");
     if (d->first_index + d->n > (1ull << 32)) return fail(DISCO_EINVAL, "first_index + n exceeds 2^32");
     std::vector<GroupConst> gc;
     if (int rc = check_profiles(d, &gc)) return rc;
@@ -229,13 +267,13 @@ int disco_load_trace(disco_ctx_t** pctx, const disco_trace_desc_t* d, void* stre
         if (e0 != cudaSuccess || c->sms < 1) return bail(fail_cuda(e0, "multiprocessor count of the current device"));
     }
     const uint32_t n = c->n;
-    bool host_in = d->arrays_on_device == 0;
+    bool host_in = d->arrays_on_device != 1;
     cudaError_t e;
     // Host arrays that are page-locked and mapped (cudaHostAlloc, cudaHostRegister, a pinned tensor) are read by
-    // the ingestion kernel in place when the trace has one profile group (every element is then read exactly
-    // once): no staging copies.  Pageable arrays, or traces with several groups, are copied first.
+    // the ingestion kernel in place (it reads every element exactly once): no staging copies.  Pageable arrays are
+    // copied first.
     const void* in_place[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
-    bool zero_copy = host_in && n != 0 && gc.size() == 1;
+    bool zero_copy = host_in && n != 0 && d->arrays_on_device == 0;
     if (zero_copy) {
         const void* host[5] = {d->prompt_len, d->output_len, d->server_ttft_s, d->server_profile, d->device_profile};
         for (int k = 0; k < 5 && zero_copy; ++k) {
@@ -273,6 +311,7 @@ int disco_load_trace(disco_ctx_t** pctx, const disco_trace_desc_t* d, void* stre
         a.sp = d->server_profile; a.dp = d->device_profile;
     }
     a.keys_a = c->keys_a.as<uint64_t>(); a.keys_b = c->keys_b.as<uint64_t>(); a.tmp_idx = c->tmp_idx.as<uint32_t>();
+    a.l_tmp = c->tmp_ln.as<uint16_t>(); a.n_tmp = c->tmp_ln.as<uint16_t>() + (n ? n : 1);
     a.radix_counts = c->radix_counts; a.zero_block = c->zero.p; a.zero_bytes = c->zero_bytes;
     a.ng_exact = c->ng_exact.as<uint32_t>(); a.readback = c->rb;     // pinned host memory, written by the last kernel
     a.S = c->S.as<int32_t>(); a.l = c->l.as<uint16_t>(); a.nout = c->nout.as<uint16_t>(); a.orig = c->orig.as<uint32_t>();
@@ -293,6 +332,7 @@ int disco_load_trace(disco_ctx_t** pctx, const disco_trace_desc_t* d, void* stre
     // the few numbers the host needs (error word, group sizes, longest output, largest TTFT per group) are in rb
     HostReadback* rb = c->rb;
     if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return bail(fail_cuda(e, "trace ingestion"));
+    if (int rc = debug_check()) return bail(rc);
     if (!same_profiles) { c->gc_dev = c->gc; c->gc_dev_at = c->d_gc.p; }      // the copy has landed
     if (rb->err[0]) {
         static const char* what[] = {"", "prompt length outside 1..4096", "output length outside 1..8192",
@@ -424,6 +464,18 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
     for (size_t k = 0; k < classes.size(); ++k) {
         const uint32_t b = (uint32_t)pol_list.size();
         for (uint32_t p = 0; p < P; ++p) if (pc[p].cls == (int)k) pol_list.push_back(p);
+        // Within a class the policies are taken in an order that puts like policies side by side with their budgets
+        // ascending, whatever order the caller gave them in: along such a run Algorithm 3's l_th does not increase
+        // and Algorithm 2's l* does not decrease, which is what the zone-by-zone reduction needs of a tile.
+        std::stable_sort(pol_list.begin() + b, pol_list.end(), [&](uint32_t x, uint32_t y) {
+            const PolicyConst &a = pc[x], &c2 = pc[y];
+            if (a.flags != c2.flags) return a.flags < c2.flags;
+            if (a.expected_len != c2.expected_len) return a.expected_len < c2.expected_len;
+            if (a.l_immediate != c2.l_immediate) return a.l_immediate < c2.l_immediate;
+            if (a.alpha != c2.alpha) return a.alpha < c2.alpha;
+            if (a.theta != c2.theta) return a.theta < c2.theta;
+            return a.budget < c2.budget;
+        });
         cls_range.push_back({b, (uint32_t)pol_list.size()});
     }
     const uint32_t tiles = (P + 31) / 32;
@@ -569,6 +621,7 @@ int disco_reduce_stats(disco_ctx_t* c, disco_policy_stats_t* stats, void* stream
                        c->d_hist_tbt.as<uint64_t>(), c->fin_totals.as<uint64_t>(),
                        c->d_stats.as<disco_policy_stats_t>(), (disco_policy_stats_t*)c->stats_host, c->err, st));
     CU(cudaStreamSynchronize(st));
+    if (int rc = debug_check()) return rc;
     std::memcpy(stats, c->stats_host, c->P * sizeof(disco_policy_stats_t));
     std::memcpy(c->rb->err, (char*)c->stats_host + c->P * sizeof(disco_policy_stats_t), 16);
     g_launches += 1;
@@ -621,6 +674,7 @@ int disco_select_policy_device(disco_ctx_t* c, double cost_cap, float tbt_slo_s,
     g_launches += 1;
     CU(launch_select(c->d_stats.as<disco_policy_stats_t>(), c->P, cost_cap, tbt_slo_s, c->sel_host, st));   // writes the pinned pair
     CU(cudaStreamSynchronize(st));
+    if (int rc = debug_check()) return rc;
     *best = c->sel_host[1];
     if (c->sel_host[0] != 0) return fail(DISCO_EINFEASIBLE, "no policy meets the cost cap and the TBT objective");
     return 0;
@@ -745,6 +799,7 @@ int disco_set_group_tables(disco_ctx_t* c, const int64_t* cnt, const int32_t* ti
     for (int g = 0; g < G; ++g)
         if (n_ticks[g]) CU(cudaMemcpyAsync(&top[g], c->F_sorted_imp.as<int32_t>() + off[g + 1] - 1, 4, cudaMemcpyDeviceToHost, st));
     CU(cudaStreamSynchronize(st));          // the host vectors above are read by the copies until here
+    if (int rc = debug_check()) { c->loaded = false; return rc; }
     c->evaluated = c->reduced = false;
     if (err_host[0]) {
         c->loaded = false;                  // the length counts have been overwritten: the context must be reloaded
@@ -783,6 +838,19 @@ int disco_import_accumulators(disco_ctx_t* c, const uint64_t* words, void* strea
     c->reduced = false;
     c->fin_imported = true;
     return 0;
+}
+
+int disco_debug_selftest(void* stream) {
+#ifdef DISCO_DEBUG
+    // a kernel offers an index beyond its bound to the check: the access is skipped, the record comes back as an error
+    CU(run_debug_selftest((cudaStream_t)stream));
+    CU(cudaStreamSynchronize((cudaStream_t)stream));
+    g_launches += 1;
+    return debug_check();
+#else
+    (void)stream;
+    return fail(DISCO_EINVAL, "not a checked build (compile with -DDISCO_DEBUG)");
+#endif
 }
 
 int disco_measure_alu_peak(double* lane_instr_per_s, double* token_steps_per_s, void* stream) {

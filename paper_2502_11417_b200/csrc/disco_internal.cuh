@@ -147,6 +147,48 @@ __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepco
 // Records the calling thread's error message (read back by disco_last_error) and returns `code`.
 int set_error(int code, const char* msg);
 
+// ---- checked build (-DDISCO_DEBUG) -----------------------------------------------------------------------
+// Every index a kernel derives from data or from its launch geometry -- request, policy, group, chunk, knot,
+// histogram bin, window slot, staging slot, table entry -- goes through DBG_OK(index, bound, kernel, what) before
+// the access.  An index outside [0, bound) is recorded (first one wins) and the access is skipped: nothing traps,
+// the context stays usable, and the next call that synchronises returns DISCO_ECUDA naming kernel and index.
+// In the ordinary build DBG_OK is the constant true and the checks vanish.
+enum DbgKernel { DBG_K_INGEST = 1, DBG_K_RADIX, DBG_K_GATHER, DBG_K_TABLES, DBG_K_PREP, DBG_K_PLAYOUT_FAST, DBG_K_PLAYOUT,
+                 DBG_K_PAIRS_ACC, DBG_K_PAIRS_ZONES, DBG_K_PAIRS_ROWS, DBG_K_FINALIZE, DBG_K_SELECT, DBG_K_SELFTEST,
+                 DBG_K_COUNT };
+enum DbgWhat { DBG_REQUEST = 1, DBG_POLICY, DBG_GROUP, DBG_CHUNK, DBG_KNOT, DBG_BIN, DBG_WINDOW, DBG_SLOT, DBG_TABLE,
+               DBG_COUNTER, DBG_ELEMENT, DBG_WHAT_COUNT };
+#ifdef DISCO_DEBUG
+#ifdef __CUDACC__
+static __device__ int32_t dbg_word[4];          // one per translation unit: kernel, what, index, bound
+__device__ __forceinline__ bool dbg_in(long long i, long long n, int kernel, int what) {
+    if (i >= 0 && i < n) return true;
+    if (atomicCAS(&dbg_word[0], 0, kernel) == 0) {
+        dbg_word[1] = what;
+        dbg_word[2] = (int32_t)(i < -2147483647LL ? -2147483647LL : (i > 2147483647LL ? 2147483647LL : i));
+        dbg_word[3] = (int32_t)(n > 2147483647LL ? 2147483647LL : n);
+    }
+    return false;
+}
+#define DBG_OK(i, n, kernel, what) (::disco::dbg_in((long long)(i), (long long)(n), (kernel), (what)))
+// Reads (and clears) this translation unit's record; registered with the host side once per unit that has kernels.
+void dbg_register(cudaError_t (*reader)(int32_t*));
+struct DbgRegistrar { explicit DbgRegistrar(cudaError_t (*r)(int32_t*)) { dbg_register(r); } };
+#define DBG_TRANSLATION_UNIT()                                                                         \
+    namespace {                                                                                        \
+    cudaError_t dbg_read_unit(int32_t* out) {                                                          \
+        cudaError_t e = cudaMemcpyFromSymbol(out, ::disco::dbg_word, 16);                              \
+        if (e == cudaSuccess && out[0]) { const int32_t z[4] = {0, 0, 0, 0}; e = cudaMemcpyToSymbol(::disco::dbg_word, z, 16); } \
+        return e;                                                                                      \
+    }                                                                                                  \
+    ::disco::DbgRegistrar dbg_registrar_unit(dbg_read_unit);                                           \
+    }
+#endif
+#else
+#define DBG_OK(i, n, kernel, what) true
+#define DBG_TRANSLATION_UNIT()
+#endif
+
 // ---- launch wrappers (defined in the kernel translation units) -------------------------------------------
 cudaError_t launch_prep(const PolicyConst* pol, uint32_t P, int G, const GroupConst* gc, const int64_t* cum_mass,
                         const uint32_t* cnt, const int32_t* sorted, const uint32_t* grp_off, Prep* prep,
@@ -195,6 +237,13 @@ cudaError_t launch_tables_imported(int G, const uint32_t* cnt, int64_t* cum_mass
 // a negative tick.  Launches 2 + 3 * (G > 1 ? 5 : 4) kernels.
 cudaError_t sort_grouped_ticks(const int32_t* ticks, const uint32_t* off, int G, uint32_t total, uint64_t* keys_a,
                                uint64_t* keys_b, uint32_t* counts, int32_t* err, int32_t* out, int sms, cudaStream_t st);
+// Checked build: 0, or DISCO_ECUDA (error string set) if a kernel refused an index since the last call.  Always 0 in
+// an ordinary build.  To be called after the stream has been synchronised.
+int check_debug_record();
+#ifdef DISCO_DEBUG
+// Launches a kernel whose only access uses an index beyond its bound (refused by the check, never made).
+cudaError_t run_debug_selftest(cudaStream_t st);
+#endif
 // Times the token loop's instruction mix on every multiprocessor; *token_steps_per_s receives the rate.
 cudaError_t run_alu_peak(int sms, double* token_steps_per_s, cudaStream_t st);
 

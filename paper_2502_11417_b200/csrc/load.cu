@@ -20,7 +20,8 @@ __global__ void k_ingest(uint32_t n, const int32_t* __restrict__ prompt, const i
                          int32_t* __restrict__ S_out, uint16_t* __restrict__ l_out, uint16_t* __restrict__ n_out,
                          uint32_t* __restrict__ orig_out, uint32_t* __restrict__ counts0, uint32_t per_block0,
                          uint32_t blocks0) {
-    // S_out..orig_out: single-group traces keep the caller's order, so the internal arrays are written here;
+    // S_out, orig_out: single-group traces keep the caller's order, so the internal arrays are written here (l_out,
+    // n_out are then the internal arrays too; otherwise packed copies in the caller's order for the gather);
     // counts0: first radix digit counted per sort block (small traces; large ones use the histogram kernel)
     __shared__ unsigned long long s_sum[kMaxGroups];
     __shared__ uint32_t s_cnt[kMaxGroups];
@@ -52,11 +53,13 @@ __global__ void k_ingest(uint32_t n, const int32_t* __restrict__ prompt, const i
         // ticks = nearest integer (ties to even) of the fp64 product, as a host llrint would give
         const long long S = __double2ll_rn(__dmul_rn((double)t, 1e6));
         const uint32_t g = ok ? s * nd + d : 0u;
-        if (ok) {
+        if (ok && DBG_OK(g, G, DBG_K_INGEST, DBG_GROUP) && DBG_OK(l, kMaxPrompt + 1, DBG_K_INGEST, DBG_TABLE)) {
             keys[i] = ((uint64_t)g << 32) | (uint32_t)S;
             if (one) atomicAdd(&s_len[l], 1u); else atomicAdd(&cnt[g * (kMaxPrompt + 1) + l], 1u);
-            if (S_out) { S_out[i] = (int32_t)S; l_out[i] = (uint16_t)l; n_out[i] = (uint16_t)o; orig_out[i] = i; }
-            if (counts0) atomicAdd(&counts0[((uint32_t)S & 255u) * blocks0 + i / per_block0], 1u);
+            if (S_out) { S_out[i] = (int32_t)S; orig_out[i] = i; }
+            l_out[i] = (uint16_t)l; n_out[i] = (uint16_t)o;
+            if (counts0 && DBG_OK(i / per_block0, blocks0, DBG_K_INGEST, DBG_COUNTER))
+                atomicAdd(&counts0[((uint32_t)S & 255u) * blocks0 + i / per_block0], 1u);
         }
         if (one) {                                             // one group: sums by warp reduction
             const uint32_t so = __reduce_add_sync(0xFFFFFFFFu, ok ? (uint32_t)o : 0u);
@@ -212,13 +215,16 @@ __global__ void k_radix_scatter(const uint64_t* __restrict__ keys_in, uint64_t* 
             if (live[j]) {
                 const uint32_t rank = __popc(peers[j] & ((1u << lane) - 1u));
                 const uint32_t pos = wcnt[w][dig[j]] + rank;
-                if (low_out) low_out[pos] = (int32_t)(uint32_t)key[j]; else keys_out[pos] = key[j];
-                if (low_out_if_last) low_out_if_last[pos] = (int32_t)(uint32_t)key[j];
-                if (pay_out) {
-                    const uint32_t i = base + w * (32 * kPer) + j * 32 + lane;
-                    pay_out[pos] = pay_in ? pay_in[i] : i;
+                if (DBG_OK(pos, n, DBG_K_RADIX, DBG_ELEMENT)) {
+                    if (low_out) low_out[pos] = (int32_t)(uint32_t)key[j]; else keys_out[pos] = key[j];
+                    if (low_out_if_last) low_out_if_last[pos] = (int32_t)(uint32_t)key[j];
+                    if (pay_out) {
+                        const uint32_t i = base + w * (32 * kPer) + j * 32 + lane;
+                        pay_out[pos] = pay_in ? pay_in[i] : i;
+                    }
                 }
-                nxt = ((uint32_t)(key[j] >> (shift + 8)) & 255u) * gridDim.x + pos / per_block;
+                if (DBG_OK(pos / per_block, gridDim.x, DBG_K_RADIX, DBG_COUNTER))
+                    nxt = ((uint32_t)(key[j] >> (shift + 8)) & 255u) * gridDim.x + pos / per_block;
             }
             __syncwarp();
             if (counts_next) {
@@ -235,14 +241,15 @@ __global__ void k_radix_scatter(const uint64_t* __restrict__ keys_in, uint64_t* 
 }
 
 __global__ void k_gather(uint32_t n, const uint32_t* __restrict__ orig_in, const uint64_t* __restrict__ keys,
-                         const int32_t* __restrict__ prompt, const int32_t* __restrict__ outlen,
+                         const uint16_t* __restrict__ prompt, const uint16_t* __restrict__ outlen,
                          int32_t* __restrict__ S, uint16_t* __restrict__ l, uint16_t* __restrict__ nout,
                          uint32_t* __restrict__ orig) {
     for (uint32_t k = blockIdx.x * blockDim.x + threadIdx.x; k < n; k += gridDim.x * blockDim.x) {
         const uint32_t i = orig_in ? orig_in[k] : k;
+        if (!DBG_OK(i, n, DBG_K_GATHER, DBG_REQUEST)) continue;
         S[k] = (int32_t)(uint32_t)keys[i];
-        l[k] = (uint16_t)prompt[i];
-        nout[k] = (uint16_t)outlen[i];
+        l[k] = prompt[i];
+        nout[k] = outlen[i];
         orig[k] = i;
     }
 }
@@ -289,8 +296,10 @@ __device__ __forceinline__ void group_knots(int G, const uint32_t* __restrict__ 
     }
     __syncthreads();
     const uint32_t N = off[g + 1] - off[g];
-    for (int k = threadIdx.x; k < kNKnots; k += blockDim.x)
-        knots[g * kNKnots + k] = N ? sorted[off[g] + (uint32_t)(((uint64_t)k * (N - 1)) / 256u)] : 0;
+    for (int k = threadIdx.x; k < kNKnots; k += blockDim.x) {
+        const uint32_t at = N ? (uint32_t)(((uint64_t)k * (N - 1)) / 256u) : 0u;
+        knots[g * kNKnots + k] = (N && DBG_OK(at, N, DBG_K_TABLES, DBG_ELEMENT)) ? sorted[off[g] + at] : 0;
+    }
     if (threadIdx.x == 0) {
         rb->knot_max[g] = N ? sorted[off[g] + N - 1] : 0;
         rb->ng[g] = N; rb->grp_sum_n[g] = grp_sum_n[g];
@@ -322,8 +331,10 @@ k_tables_imported(const uint32_t* __restrict__ cnt, int64_t* __restrict__ cum, u
                   const int32_t* __restrict__ F_sorted, const uint32_t* __restrict__ F_off, int32_t* __restrict__ knots) {
     const int g = blockIdx.x;
     const uint32_t off = F_off[g], N = F_off[g + 1] - off;
-    for (int k = threadIdx.x; k < kNKnots; k += blockDim.x)
-        knots[g * kNKnots + k] = N ? F_sorted[off + (uint32_t)(((uint64_t)k * (N - 1)) / 256u)] : 0;
+    for (int k = threadIdx.x; k < kNKnots; k += blockDim.x) {
+        const uint32_t at = N ? (uint32_t)(((uint64_t)k * (N - 1)) / 256u) : 0u;
+        knots[g * kNKnots + k] = (N && DBG_OK(at, N, DBG_K_TABLES, DBG_ELEMENT)) ? F_sorted[off + at] : 0;
+    }
     group_mass(cnt, cum, ng_exact);
 }
 
@@ -349,6 +360,8 @@ cudaError_t radix_pass(const uint64_t* kin, uint64_t* kout, const uint32_t* pin,
 }
 
 }  // namespace
+
+DBG_TRANSLATION_UNIT()
 
 uint32_t load_kernel_launches(uint32_t n, int G) {
     if (n == 0) return 1;
@@ -377,11 +390,12 @@ cudaError_t run_load(const LoadArgs& a, cudaStream_t st) {
         k_ingest<<<std::min(grid_for(n, 4 * kIngestThreads, a.sms), 2 * a.sms), kIngestThreads, 0, st>>>(
             n, a.prompt, a.outlen, a.ttft, a.sp, a.dp, a.ns, a.nd, a.keys_a, a.cnt,
             (unsigned long long*)a.grp_sum_n, a.ng, a.max_n, a.err,
-            G == 1 ? a.S : nullptr, a.l, a.nout, a.orig, small ? counts_a : nullptr, per_block, blocks);
+            G == 1 ? a.S : nullptr, G == 1 ? a.l : a.l_tmp, G == 1 ? a.nout : a.n_tmp, a.orig,
+            small ? counts_a : nullptr, per_block, blocks);
         if (G > 1) {
             // internal request order: stable partition by group
             if ((e = radix_pass(a.keys_a, a.keys_b, nullptr, a.tmp_idx, n, 32, counts_b, st))) return e;
-            k_gather<<<grid_for(n, 256, a.sms), 256, 0, st>>>(n, a.tmp_idx, a.keys_a, a.prompt, a.outlen, a.S, a.l, a.nout, a.orig);
+            k_gather<<<grid_for(n, 256, a.sms), 256, 0, st>>>(n, a.tmp_idx, a.keys_a, a.l_tmp, a.n_tmp, a.S, a.l, a.nout, a.orig);
         }
         // sort (group, ticks): four byte passes over the ticks, one over the group id
         uint64_t *src = a.keys_a, *dst = a.keys_b;
@@ -550,6 +564,7 @@ extern "C" int disco_sort_ttft_ticks_noalloc(const float* server_ttft_s, uint32_
     int32_t h_err[2] = {0, 0};
     if ((e = cudaMemcpyAsync(h_err, err, sizeof h_err, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return fail_after_launch(e);
     if ((e = cudaStreamSynchronize(st)) != cudaSuccess) return set_error(DISCO_ECUDA, cudaGetErrorString(e));
+    if (int rc = check_debug_record()) return rc;
     if (h_err[0]) return set_error(DISCO_EINVAL, "server TTFT not finite, not positive or above 2000 s");
     return 0;
 }

@@ -25,6 +25,7 @@ struct LoadArgs {
     // scratch
     uint64_t *keys_a, *keys_b;            // [n] (group << 32 | ticks)
     uint32_t* tmp_idx;                    // [n]
+    uint16_t *l_tmp, *n_tmp;              // [n] each: lengths in the caller's order (traces with several groups)
     uint32_t* radix_counts;               // [5][256 * kRadixMaxBlocks], directly after zero_block's tables
     void* zero_block; size_t zero_bytes;  // cnt, grp_sum_n, ng, max_n, err, contiguous
     uint32_t* ng_exact;                   // [G] group sizes recounted from the length histogram

@@ -110,6 +110,9 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
     const uint32_t pol_idx = tile * PL + pol_in_tile;
     const bool act = pol_idx < n_list;
     const uint32_t p = pol_list[act ? pol_idx : 0];
+    if (!DBG_OK(p, P, DBG_K_PAIRS_ACC, DBG_POLICY) || !DBG_OK(g, tr.n_groups, DBG_K_PAIRS_ACC, DBG_GROUP) ||
+        (ch.len && !DBG_OK((unsigned long long)ch.start + ch.len - 1, tr.n, DBG_K_PAIRS_ACC, DBG_REQUEST)))
+        return;
     const Prep pr = prep[(size_t)g * P + p];
     const int pols_here = (int)min((uint32_t)PL, n_list - tile * PL);
     // a tile that went through the zone kernel: only the requests it flagged are left (block-uniform)
@@ -180,7 +183,7 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
     auto run_batch = [&](const Raw& cur, uint32_t taken, uint32_t b0) {
         const int n_here = __popc(taken);
         staged += (uint32_t)n_here;
-        if ((taken >> lane) & 1u) {
+        if (((taken >> lane) & 1u) && DBG_OK(__popc(taken & ((1u << lane) - 1u)), kStageReq, DBG_K_PAIRS_ACC, DBG_SLOT)) {
             const int at = __popc(taken & ((1u << lane) - 1u));
             const uint32_t l = cur.l, n = cur.n, S = cur.S, m = cur.m;
             const uint32_t stall = cur.stall, dly = cur.dly;
@@ -290,7 +293,7 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
                 a_dl += h2[k].x >> 17; cnt8 += h2[k].y;
                 a_tt += ttft[k];
                 if (EXT ? !waits : kNoWaits) atomicAdd((uint32_t*)((char*)my_ttft + h2[k].z), h2[k].w);
-                else hist16_add_ticks(my_ttft, ttft[k]);
+                else if (DBG_OK(bin_of_ticks(ttft[k]), kNBins, DBG_K_PAIRS_ACC, DBG_BIN)) hist16_add_ticks(my_ttft, ttft[k]);
             }
             // only the row of a pair whose hand-off stalled carries an increment for the stall histogram: one test
             // for the four pairs, then each
@@ -312,7 +315,7 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
                     unsigned long long* hp = hist_tbt + (size_t)p * kNBins + cc.lo[g][c];
                     for (int j = 0; j < W; ++j) {
                         const uint32_t v = j == kt ? 0u : wp[j];
-                        if (v) atomicAdd(&hp[j], (unsigned long long)v);
+                        if (v && DBG_OK(cc.lo[g][c] + j, kNBins, DBG_K_PAIRS_ACC, DBG_BIN)) atomicAdd(&hp[j], (unsigned long long)v);
                     }
                 }
             }
@@ -338,6 +341,7 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
                 const int r = r0 + k * slots + slot;
                 ok[k] = r < n_here;
                 rr[k] = min(r, n_here - 1);                     // a slot that was staged in this batch
+                if (!DBG_OK(rr[k], kStageReq, DBG_K_PAIRS_ACC, DBG_SLOT)) { rr[k] = 0; ok[k] = false; }
             }
             if (kind == K_NOWAIT) pairs_of(std::integral_constant<int, K_NOWAIT>{}, std::false_type{}, rr, ok);
             else if (kind == K_WAIT) pairs_of(std::integral_constant<int, K_WAIT>{}, std::false_type{}, rr, ok);
@@ -556,6 +560,7 @@ k_pairs_rows(TraceDev tr, const GroupConst* __restrict__ gcs, const Prep* __rest
     };
     auto pair = [&](const RowPol& rp, const Prep* full) {
         const idx_t at = (idx_t)rp.pol * N + (idx_t)orig;
+        if (!DBG_OK(rp.pol, P, DBG_K_PAIRS_ROWS, DBG_POLICY) || !DBG_OK(orig, tr.n, DBG_K_PAIRS_ROWS, DBG_REQUEST)) return;
         if (EXT) {
             const PairOut o = decide<true>(q, *full, Td, candidate);
             emit(at, o.dev_only, o.started, o.dev_wins, o.migr, o.ttft);
@@ -584,6 +589,8 @@ k_pairs_rows(TraceDev tr, const GroupConst* __restrict__ gcs, const Prep* __rest
 }
 
 }  // namespace
+
+DBG_TRANSLATION_UNIT()
 
 cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const Prep* prep, uint32_t P,
                          const uint32_t* pol_list, uint32_t n_list, const Chunk* chunks, uint32_t n_chunks,

@@ -33,7 +33,25 @@ k_alu_peak(uint32_t k0, uint32_t mul, int tokens, int cnt, uint32_t one, uint32_
     if (hC == 0xFFFFFFFFu) out[id & 31u] = hC;      // keeps the loop alive; practically never taken
 }
 
+#ifdef DISCO_DEBUG
+__global__ void k_debug_selftest(uint32_t* __restrict__ out, int bound) {
+    const int i = bound + 2 + (int)threadIdx.x;                  // beyond the bound on purpose
+    if (DBG_OK(i, bound, DBG_K_SELFTEST, DBG_ELEMENT)) out[i] = 1u;   // refused: the store never happens
+}
+#endif
+
 }  // namespace
+
+#ifdef DISCO_DEBUG
+DBG_TRANSLATION_UNIT()
+cudaError_t run_debug_selftest(cudaStream_t st) {
+    uint32_t* d_sink = nullptr;
+    cudaError_t e = cudaGetSymbolAddress((void**)&d_sink, sink);
+    if (e) return e;
+    k_debug_selftest<<<1, 32, 0, st>>>(d_sink, 32);
+    return cudaGetLastError();
+}
+#endif
 
 cudaError_t run_alu_peak(int sms, double* token_steps_per_s, cudaStream_t st) {
     uint32_t* d_sink = nullptr;

@@ -58,7 +58,7 @@ struct GroupClass {                      // constants of the request's group und
 
 __device__ __forceinline__ void count_slow(uint32_t tbt, uint32_t* win, int lo, int W, int32_t* err) {
     const int b = bin_of_ticks(tbt) - lo;
-    if (b >= 0 && b < W) atomicAdd(&win[b], 1u); else atomicExch(&err[2], 1);
+    if (b >= 0 && b < W && DBG_OK(b, W, DBG_K_PLAYOUT, DBG_WINDOW)) atomicAdd(&win[b], 1u); else atomicExch(&err[2], 1);
 }
 
 __device__ __forceinline__ int32_t warp_inclusive_sum(int32_t v, int lane) {
@@ -190,6 +190,7 @@ __device__ __forceinline__ uint32_t handoff_latency(const GroupClass& G, uint32_
     if (G.cand == 1) return (uint32_t)G.kappa * (l + m) + (uint32_t)G.c0;   // device re-prefills prompt + m tokens
     const uint32_t u = mix32(key);                                          // a server TTFT drawn from F by its knots
     const uint32_t kk = u >> 24, fr = (u >> 8) & 0xFFFFu;
+    if (!DBG_OK(kk + 1, kNKnots, DBG_K_PLAYOUT, DBG_KNOT)) return 0u;
     return (uint32_t)(G.K[kk] + (int32_t)(((int64_t)(G.K[kk + 1] - G.K[kk]) * (int64_t)fr) >> 16));
 }
 
@@ -303,8 +304,9 @@ k_playout(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __r
     const int32_t thr = thr64 > INT_MAX ? INT_MAX : (int32_t)thr64;
 
     // ---- one request per lane: inputs
-    const bool live = batch0 + lane < count;
+    bool live = batch0 + lane < count;
     const uint32_t kk = !live ? 0u : (todo ? todo[batch0 + lane] : batch0 + lane);
+    if (live && !DBG_OK(kk, tr.n, DBG_K_PLAYOUT, DBG_REQUEST)) live = false;
     uint32_t n_l = 1, l_l = 1, key_l = 0;
     int g_l = 0;
     if (live) {
@@ -331,7 +333,7 @@ k_playout(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __r
         const uint32_t key = __shfl_sync(FULL, key_l, r);
         const int g = __shfl_sync(FULL, g_l, r);
         const uint32_t k = __shfl_sync(FULL, kk, r);
-        if (g != cur_g) {
+        if (g != cur_g && DBG_OK(g, tr.n_groups, DBG_K_PLAYOUT, DBG_GROUP)) {
             cur_g = g;
             const GroupConst& gc = gcs[g];
             G.mulS = 2u * (uint32_t)gc.J_srv + 1u; G.mulD = 2u * (uint32_t)gc.J_dev + 1u;
@@ -507,6 +509,8 @@ k_playout(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __r
 }
 
 }  // namespace
+
+DBG_TRANSLATION_UNIT()
 
 cudaError_t launch_playout_fast(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const int32_t* knots,
                                 uint32_t k0, TimelineRec rec, uint32_t* todo, uint32_t* todo_count, bool never_clamps,

@@ -130,7 +130,7 @@ k_playout_fast(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst
             const uint32_t n = __shfl_sync(FULL, n_l, r), l = __shfl_sync(FULL, l_l, r);
             const uint32_t key = __shfl_sync(FULL, key_l, r);
             const int g = __shfl_sync(FULL, g_l, r);
-            if (g != cur_g) {
+            if (g != cur_g && DBG_OK(g, tr.n_groups, DBG_K_PLAYOUT_FAST, DBG_GROUP)) {
                 cur_g = g;
                 const GroupConst& gc = gcs[g];
                 G.mulS = 2u * (uint32_t)gc.J_srv + 1u; G.mulD = 2u * (uint32_t)gc.J_dev + 1u;
@@ -175,7 +175,10 @@ k_playout_fast(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst
                 s_S = cnt * G.cS_base - (int32_t)hS; s_D = cnt * G.cD_base - (int32_t)hD;
                 const bool neg = cnt != 0 && ((int32_t)xS > G.cS_base || (int32_t)xD > G.cD_base);   // some c_j < 0
                 clean = (__ballot_sync(FULL, neg) & tmask) == 0;
-                if (nI != 0 && !clean && q == 0) todo[atomicAdd(todo_count, 1u)] = batch0 + r;   // for the general kernel
+                if (nI != 0 && !clean && q == 0) {                     // for the general kernel
+                    const uint32_t at = atomicAdd(todo_count, 1u);
+                    if (DBG_OK(at, tr.n, DBG_K_PLAYOUT_FAST, DBG_REQUEST)) todo[at] = batch0 + r;
+                }
             }
             const bool go = clean && nI != 0;
             // ---- hand-off index on the candidate stream
@@ -210,7 +213,9 @@ k_playout_fast(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst
                 else {
                     const uint32_t u = mix32(key);                     // a server TTFT drawn from F by its knots
                     const uint32_t ki = u >> 24, fr = (u >> 8) & 0xFFFFu;
-                    M = (uint32_t)(G.K[ki] + (int32_t)(((int64_t)(G.K[ki + 1] - G.K[ki]) * (int64_t)fr) >> 16));
+                    M = 0;
+                    if (DBG_OK(ki + 1, kNKnots, DBG_K_PLAYOUT_FAST, DBG_KNOT))
+                        M = (uint32_t)(G.K[ki] + (int32_t)(((int64_t)(G.K[ki + 1] - G.K[ki]) * (int64_t)fr) >> 16));
                 }
                 const int32_t v = e_m + (tau - (int32_t)M);            // slot lag of token m+1, negated
                 stall = (uint32_t)tau + (uint32_t)max(-v, 0);
@@ -268,7 +273,8 @@ k_playout_fast(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst
         }
         __syncwarp();
         // ---- one request per lane: results out
-        if (live && (o_md >> 31)) {
+        if (live && (o_md >> 31) && DBG_OK(kk, tr.n, DBG_K_PLAYOUT_FAST, DBG_REQUEST) &&
+            DBG_OK(g_l, kMaxGroups, DBG_K_PLAYOUT_FAST, DBG_GROUP)) {
             const uint32_t nI = n_l - 1, ut = (uint32_t)tau, m = o_md & 0xFFFFu, dl = (o_md >> 16) & 0x7FFFu;
             rec.sum[0][kk] = nI * ut; rec.max[0][kk] = nI ? ut : 0u;
             rec.sum[1][kk] = nI * ut; rec.max[1][kk] = nI ? ut : 0u;
@@ -283,6 +289,8 @@ k_playout_fast(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst
 }
 
 }  // namespace
+
+DBG_TRANSLATION_UNIT()
 
 cudaError_t launch_playout_fast(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const int32_t* knots,
                                 uint32_t k0, TimelineRec rec, uint32_t* todo, uint32_t* todo_count,

@@ -15,7 +15,7 @@ __device__ int32_t inverse_cdf(const int32_t* sorted, uint32_t N, double q) {
     long long k = (long long)r;
     if (k < 0) k = 0;
     if (k > (long long)N - 1) k = (long long)N - 1;
-    return sorted[k];
+    return DBG_OK(k, N, DBG_K_PREP, DBG_ELEMENT) ? sorted[k] : 0;
 }
 
 // Smallest x in [lo, hi) with pred(x), or hi if there is none; pred is false up to some point and true from
@@ -52,6 +52,7 @@ __global__ void k_prep(const PolicyConst* __restrict__ pol, uint32_t P, int G, c
     if (idx >= P * (uint32_t)G) return;
     const int g = (int)(idx / P);
     const uint32_t p = idx % P;
+    if (!DBG_OK(g, G, DBG_K_PREP, DBG_GROUP)) return;
     const PolicyConst pc = pol[p];
     const int64_t* cum = cum_mass + (size_t)g * (kMaxPrompt + 2);     // cum[L] = sum_{l<L} l*cnt[l]
     const uint32_t* c = cnt + (size_t)g * (kMaxPrompt + 1);
@@ -72,7 +73,8 @@ __global__ void k_prep(const PolicyConst* __restrict__ pol, uint32_t P, int G, c
     if (!r.device_constrained) {
         // Eq. 3: smallest L with device-only mass sum_{l<L} l cnt[l] >= (1-b) Total
         const double target = __dmul_rn(__dsub_rn(1.0, b), Total);
-        r.l_th = first_true(0, kMaxPrompt + 1, [&](int L) { return (double)cum[L] >= target; });   // in [0, 4097]
+        r.l_th = first_true(0, kMaxPrompt + 1, [&](int L) {                                         // in [0, 4097]
+            return DBG_OK(L, kMaxPrompt + 2, DBG_K_PREP, DBG_TABLE) ? (double)cum[L] >= target : true; });
     } else {
         // Algorithm 2, phase 1: tail protection
         const double q_tail = __dsub_rn(1.0, fmin(alpha, b));
@@ -88,9 +90,10 @@ __global__ void k_prep(const PolicyConst* __restrict__ pol, uint32_t P, int G, c
             // phase 2: A input tokens may start the device at once; shortest prompts first
             const double A = __dmul_rn(__ddiv_rn(__dsub_rn(b, alpha), __dsub_rn(1.0, alpha)), Total);
             // first length whose cumulative mass exceeds A; 4097 = every class is funded
-            const int lo = first_true(0, kMaxPrompt + 1, [&](int l) { return (double)cum[l + 1] > A; });
+            const int lo = first_true(0, kMaxPrompt + 1, [&](int l) {
+                return DBG_OK(l + 1, kMaxPrompt + 2, DBG_K_PREP, DBG_TABLE) ? (double)cum[l + 1] > A : true; });
             r.l_star = lo;
-            if (lo <= kMaxPrompt) {
+            if (lo <= kMaxPrompt && DBG_OK(lo, kMaxPrompt + 1, DBG_K_PREP, DBG_TABLE)) {
                 const double f = __ddiv_rn(__dsub_rn(A, (double)cum[lo]), __dmul_rn((double)lo, (double)c[lo]));
                 r.w_star = inverse_cdf(srt, N, __dmul_rn(__dsub_rn(1.0, alpha), __dsub_rn(1.0, f)));
             }
@@ -128,7 +131,11 @@ k_prep_beta(const PolicyConst* __restrict__ pol, uint32_t P, const int64_t* __re
             if (k == 0) continue;
             const long long w = l <= l_imm ? 0 : min(beta * (long long)l, w_tail);
             uint32_t lo = 0, hi = N;                                  // requests with S <= w
-            while (lo < hi) { const uint32_t mid = (lo + hi) >> 1; if ((long long)srt[mid] <= w) lo = mid + 1; else hi = mid; }
+            while (lo < hi) {
+                const uint32_t mid = (lo + hi) >> 1;
+                if (!DBG_OK(mid, N, DBG_K_PREP, DBG_ELEMENT)) break;
+                if ((long long)srt[mid] <= w) lo = mid + 1; else hi = mid;
+            }
             acc += (long long)l * (long long)k * (long long)(N - lo);
         }
 #pragma unroll
@@ -153,6 +160,8 @@ k_prep_beta(const PolicyConst* __restrict__ pol, uint32_t P, const int64_t* __re
 }
 
 }  // namespace
+
+DBG_TRANSLATION_UNIT()
 
 cudaError_t launch_prep(const PolicyConst* pol, uint32_t P, int G, const GroupConst* gc, const int64_t* cum_mass,
                         const uint32_t* cnt, const int32_t* sorted, const uint32_t* grp_off, Prep* prep,

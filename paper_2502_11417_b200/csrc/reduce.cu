@@ -44,6 +44,7 @@ __device__ void warp_quantile_bins(const unsigned long long* hist, unsigned long
             }
             const unsigned owner = __ballot_sync(0xFFFFFFFFu, found >= 0);
             bin = owner ? __shfl_sync(0xFFFFFFFFu, found, __ffs(owner) - 1) : kNBins - 1;
+            if (!DBG_OK(bin, kNBins, DBG_K_FINALIZE, DBG_BIN)) bin = kNBins - 1;
         }
         out[k] = bin;
     }
@@ -160,6 +161,8 @@ __global__ void k_select(const disco_policy_stats_t* __restrict__ stats, uint32_
 }
 
 }  // namespace
+
+DBG_TRANSLATION_UNIT()
 
 cudaError_t launch_finalize(uint32_t P, int G, const GroupConst* gc, const uint64_t* acc, const uint64_t* hist_ttft,
                             const uint64_t* hist_tbt, const uint64_t* fin_totals,

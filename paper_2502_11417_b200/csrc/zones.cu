@@ -169,6 +169,7 @@ __device__ __forceinline__ bool head_outcome_waits(const TileCtx& c, const ZoneS
 // Enters (outcome oc, TTFT tt) minus (outcome oc_b, TTFT tt_b) of request q at difference row `row`, times sign.
 __device__ __forceinline__ void enter_difference(ZoneSmem& sm, int row, uint32_t sign, const Req& q, uint32_t stall_code,
                                                  int oc, uint32_t tt, int oc_b, uint32_t tt_b) {
+    if (!DBG_OK(row, kZRows, DBG_K_PAIRS_ZONES, DBG_SLOT)) return;
     const Addends h = addends_of(oc, q), a = addends_of(oc_b, q);
     uint32_t* r = sm.e_sum[row];
     atomicAdd(&r[Z_TD], sign * (h.td - a.td));
@@ -195,8 +196,9 @@ __device__ __forceinline__ void enter_difference(ZoneSmem& sm, int row, uint32_t
 template <bool WAITS, bool LEAN>
 __device__ __forceinline__ void drain_queue(ZoneSmem& sm, const TileCtx& c, const uint32_t* queue, int count) {
     const int lane = threadIdx.x & 31;
-    if (lane < count) {
+    if (lane < count && DBG_OK(lane, kZQueue, DBG_K_PAIRS_ZONES, DBG_SLOT)) {
         Req q = load_request<LEAN>(c, queue[lane]);
+        if (!DBG_OK(q.l, kMaxPrompt + 1, DBG_K_PAIRS_ZONES, DBG_TABLE)) q.l = 0;
         const uint32_t stall_code = finish_request<LEAN>(c, q);
         const uint32_t Td = c.kappa * q.l + c.c0;
         const float saving = saving_of(c, q);
@@ -248,7 +250,8 @@ __device__ __forceinline__ void zone_pass(ZoneSmem& sm, const TileCtx& c, uint32
         const uint32_t i = i0 + lane;
         Req q = nx;
         if (i0 + kZThreads < r_hi) nx = load_request<LEAN>(c, i + kZThreads);
-        const bool valid = i < r_hi;
+        bool valid = i < r_hi;
+        if (!DBG_OK(q.l, kMaxPrompt + 1, DBG_K_PAIRS_ZONES, DBG_TABLE)) { q.l = 0; valid = false; }
         const uint32_t Td = c.kappa * q.l + c.c0;
         const int k1 = sm.tab1[q.l], k2 = WAITS ? sm.tab2[q.l] : k1;
         const float saving = saving_of(c, q);
@@ -285,13 +288,14 @@ __device__ __forceinline__ void zone_pass(ZoneSmem& sm, const TileCtx& c, uint32
             const uint32_t stall_code = finish_request<LEAN>(c, q);
             const Addends a = addends_of(oc_all, q);
             c_td += a.td; c_ps += a.ps; c_pd += a.pd; c_tau += a.tau; c_dl += a.dl; c_cnt += a.cnt; c_tt += tt_all;
-            atomicAdd(&sm.c_ttft[bin_of_ticks(tt_all)], 1u);
+            if (DBG_OK(bin_of_ticks(tt_all), kNBins, DBG_K_PAIRS_ZONES, DBG_BIN)) atomicAdd(&sm.c_ttft[bin_of_ticks(tt_all)], 1u);
             if (oc_all >= O_MIGR_TO_DEV && stall_code != 0u) atomicAdd(&sm.c_stall[bin_of_ticks(q.stall)], 1u);
         }
         // ---- queue the requests that need corrections; a full warp of them is worked off at once
         const uint32_t enq = __ballot_sync(0xFFFFFFFFu, ok && later);
         if (enq) {
-            if (ok && later) queue[queued + __popc(enq & ((1u << lane) - 1u))] = i;
+            if (ok && later && DBG_OK(queued + __popc(enq & ((1u << lane) - 1u)), kZQueue, DBG_K_PAIRS_ZONES, DBG_SLOT))
+                queue[queued + __popc(enq & ((1u << lane) - 1u))] = i;
             queued += __popc(enq);
             __syncwarp();
             if (queued >= 32) {
@@ -348,6 +352,9 @@ k_pairs_zones(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst*
     const bool act = pol_idx < n_list;
     const Prep pr = prep[(size_t)g * P + pol_list[act ? pol_idx : 0]];
     if (!tile_by_zones(pr, act, lane, npol)) return;              // block-uniform: the pair kernel takes the tile
+    if (!DBG_OK(g, tr.n_groups, DBG_K_PAIRS_ZONES, DBG_GROUP) ||
+        (ch.len && !DBG_OK((unsigned long long)ch.start + ch.len - 1, tr.n, DBG_K_PAIRS_ZONES, DBG_REQUEST)))
+        return;
     const GroupConst& gc = gcs[g];
     const ClassConst& cc = *ccp;
     const bool waits = pr.device_constrained != 0;                // Algorithm 2 (true) or Algorithm 3 (every lane alike)
@@ -376,7 +383,7 @@ k_pairs_zones(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst*
         sm.w_star[lane] = (uint32_t)pr.w_star;
         sm.w_tail[lane] = (uint32_t)pr.w_tail;
         sm.theta[lane] = theta;
-        sm.pol[lane] = pol_list[pol_idx];
+        sm.pol[lane] = DBG_OK(pol_list[pol_idx], P, DBG_K_PAIRS_ZONES, DBG_POLICY) ? pol_list[pol_idx] : 0u;
     }
     __syncthreads();
     // tables over the prompt length: how many of the tile's (ordered) thresholds lie on which side of it
@@ -473,6 +480,8 @@ k_pairs_zones(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst*
 }
 
 }  // namespace
+
+DBG_TRANSLATION_UNIT()
 
 cudaError_t launch_pairs_zones(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const Prep* prep,
                                uint32_t P, const uint32_t* pol_list, uint32_t n_list, int PL, const Chunk* chunks,

@@ -162,7 +162,7 @@ def run(ids=None, verbose=True, gpu=False):
                 f.write(src.replace(old, new))
             subprocess.check_call(["g++", "-std=c++17", "-O2", "-ffp-contract=off", "-fPIC", "-shared", "-w",
                                    "-I", os.path.dirname(SRC), "-o", so, cpp])
-            env = dict(os.environ, DISCO_ORACLE_LIB=so)
+            env = dict(os.environ, DISCO_ORACLE_LIB=so, DISCO_ORACLE_MUTATION_CHECK="1")
             select = ["-m", "gpu", os.path.join(ROOT, "tests", "test_gpu_parity.py")] if gpu else \
                      ["-m", "not gpu", "-k", "oracle and not mutant", os.path.join(ROOT, "tests")]
             r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider"] + select,

@@ -429,11 +429,15 @@ def test_zone_by_zone_reduction_and_what_it_leaves_to_the_pair_kernel():
         # many budgets at or below the tail ratio (each its own w_tail), and budgets that repeat (equal thresholds)
         low = [synth.policy(b, alpha=0.3) for b in sorted(list(synth.budget_grid(24)) + [0.1, 0.1, 0.5, 0.5, 0.5])]
         full_parity(w, low, tag=f"zones low budgets dear={dear}")
-        # descending budgets: the thresholds are not ordered, the whole tile goes pair by pair
-        down = plain[::-1]
-        full_parity(w, down, tag=f"zones descending dear={dear}")
-        zone, left, _, _ = _work(w, down)
-        assert left > 0.5 * w.n * len(down)
+        # the caller's order does not matter: the library lines like policies up by budget itself
+        rng = np.random.default_rng(7)
+        shuffled = [plain[k] for k in rng.permutation(len(plain))]
+        full_parity(w, shuffled, tag=f"zones shuffled dear={dear}")
+        assert _work(w, shuffled)[0] > 0.9 * w.n * len(plain)
+        # random routing has no ordered thresholds: such tiles go pair by pair
+        stoch = [synth.policy(b, flags=synth.FLAG_STOCHASTIC | PACE) for b in grid]
+        full_parity(w, stoch, tag=f"zones none dear={dear}")
+        assert _work(w, stoch)[0] == 0
         # pacing off: no zone kernel at all
         nopace = [synth.policy(b, flags=MIG) for b in grid]
         full_parity(w, nopace, tag=f"zones pacing off dear={dear}")
