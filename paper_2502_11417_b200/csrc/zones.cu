@@ -31,10 +31,11 @@ constexpr int kZThreads = 1024;
 static_assert(kZThreads == 1024, "the flush assigns its work to threads 0 .. 1023 by index");
 constexpr int kZWarps = kZThreads / 32;
 constexpr int kZRows = 33;              // difference rows: row q is carried to the policies below q, q = 1 .. 32
-// Requests between two flushes of a block.  A signed 16-bit count of the difference rows moves by at most one per
-// queued request under Algorithm 3 (one boundary) and by at most two under Algorithm 2 (a boundary and a policy of
-// its own at the same row), and every request of a pass may be queued.
-constexpr uint32_t kZPass = 32640, kZPassWaits = 16320;
+// Requests a block may queue for corrections between two flushes.  A signed 16-bit count of the difference rows
+// moves by at most one per queued request under Algorithm 3 (one boundary) and by at most two under Algorithm 2 (a
+// boundary and a policy of its own at the same row).
+constexpr uint32_t kZItems = 32640, kZItemsWaits = 16320;
+constexpr uint32_t kZStretch = 8160;     // requests between two looks at that budget
 constexpr int kZQueue = 64;             // queue slots per warp
 enum ZSum { Z_TD = 0, Z_PS, Z_PD, Z_TAU, Z_DL, Z_CNT_A, Z_CNT_B, Z_TT_LO, Z_TT_HI, kZSums };
 constexpr int kZSumStride = 12;
@@ -229,22 +230,94 @@ __device__ __forceinline__ void drain_queue(ZoneSmem& sm, const TileCtx& c, cons
     __syncwarp();
 }
 
+// Where a block's results go.
+struct FlushTo {
+    unsigned long long *acc, *hist_ttft, *hist_tbt;
+    int n_groups, g, bin_tau;
+};
+
+// Adds what the block holds to the policies' global sums and histograms.  All threads call; the shared tables must
+// be complete (barrier before) and may be cleared after the next barrier.
+__device__ __forceinline__ void flush_tile(ZoneSmem& sm, int npol, const FlushTo& to) {
+    unsigned long long* acc = to.acc; unsigned long long* hist_ttft = to.hist_ttft; unsigned long long* hist_tbt = to.hist_tbt;
+    const int g = to.g, bin_tau = to.bin_tau;
+    // policy p gets the common part plus the difference rows above it (rows q > p); two threads a histogram word:
+    // one for the upper half of the policies, one for the lower half
+    if ((threadIdx.x & 511) < kHWords) {
+        const int wd = threadIdx.x & 511;
+        const int half = npol > 16 ? 16 : 0;                                        // policies [half, npol) | [0, half)
+        const bool upper = threadIdx.x < 512;
+        int32_t t0 = (int32_t)sm.c_ttft[2 * wd], t1 = (int32_t)sm.c_ttft[2 * wd + 1];
+        int32_t s0 = (int32_t)sm.c_stall[2 * wd], s1 = (int32_t)sm.c_stall[2 * wd + 1];
+        for (int p = npol - 1; p >= (upper ? half : 0); --p) {
+            const uint32_t et = sm.e_ttft[p + 1][wd], es = sm.e_stall[p + 1][wd];   // row p + 1: for policies up to p
+            t0 += packed_lo(et); t1 += packed_hi(et); s0 += packed_lo(es); s1 += packed_hi(es);
+            if (!upper && p >= half) continue;                                      // (the other thread's policies)
+            const size_t o = (size_t)sm.pol[p] * kNBins + 2 * wd;
+            if (t0) atomicAdd(&hist_ttft[o], (unsigned long long)t0);
+            if (t1) atomicAdd(&hist_ttft[o + 1], (unsigned long long)t1);
+            if (s0) atomicAdd(&hist_tbt[o], (unsigned long long)s0);
+            if (s1) atomicAdd(&hist_tbt[o + 1], (unsigned long long)s1);
+        }
+    }
+    if (threadIdx.x >= 512 && threadIdx.x < 512 + 32 * kZSums) {                 // a thread per (field, policy)
+        const int f = (threadIdx.x - 512) >> 5, p = threadIdx.x & 31;
+        const bool is_packed = f == Z_CNT_A || f == Z_CNT_B;                    // two counts in the word
+        long long lo = is_packed ? (long long)(sm.c_sum[f] & 0xFFFFFFFFull) : (long long)sm.c_sum[f];
+        long long hi = is_packed ? (long long)(sm.c_sum[f] >> 32) : 0;
+        for (int q = p + 1; q <= npol; ++q) {                                   // the rows above the policy
+            const uint32_t e = sm.e_sum[q][f];
+            if (is_packed) { lo += packed_lo(e); hi += packed_hi(e); } else lo += (int32_t)e;
+        }
+        if (p < npol) {
+            const uint32_t pp = sm.pol[p];
+            unsigned long long* a = acc + ((size_t)pp * to.n_groups + g) * kNAcc;
+            // (the two halves of the TTFT sum may be negative on their own: the 64-bit adds wrap to the right total)
+            switch (f) {
+                case Z_TD: if (lo) atomicAdd(&a[A_TOK_DEVICE], (unsigned long long)lo); break;
+                case Z_PS: if (lo) atomicAdd(&a[A_PRE_SERVER], (unsigned long long)lo); break;
+                case Z_PD: if (lo) atomicAdd(&a[A_PRE_DEVICE], (unsigned long long)lo); break;
+                case Z_TAU: if (lo) atomicAdd(&hist_tbt[(size_t)pp * kNBins + bin_tau], (unsigned long long)lo); break;
+                case Z_DL: if (lo) atomicAdd(&a[A_DELAYED], (unsigned long long)lo); break;
+                case Z_CNT_A: if (lo) atomicAdd(&a[A_DEVICE_ONLY], (unsigned long long)lo);
+                              if (hi) atomicAdd(&a[A_RACE], (unsigned long long)hi); break;
+                case Z_CNT_B: if (lo) atomicAdd(&a[A_DEVICE_WON], (unsigned long long)lo);
+                              if (hi) atomicAdd(&a[A_MIGR], (unsigned long long)hi); break;
+                case Z_TT_LO: if (lo) atomicAdd(&a[A_TTFT_SUM], (unsigned long long)lo); break;
+                default: if (lo) atomicAdd(&a[A_TTFT_SUM], (unsigned long long)lo << 16); break;   // Z_TT_HI
+            }
+        }
+    }
+}
+
 // WAITS: the tile's policies are Algorithm 2's (wait map); otherwise Algorithm 3's (length threshold).
 // LEAN: pacing is on and each stream's regular intervals fall in one histogram bin (tau's).
+//
+// The chunk is worked through in stretches of kZStretch requests.  The shared tables are flushed (and cleared) when
+// the requests queued for corrections since the last flush, plus a stretch that could all be queued, would no longer
+// fit the signed 16-bit counts of the difference rows -- and at the end of the chunk.
 template <bool WAITS, bool LEAN>
-__device__ __forceinline__ void zone_pass(ZoneSmem& sm, const TileCtx& c, uint32_t r_lo, uint32_t r_hi, uint32_t tile,
-                                          uint32_t n_tiles, uint32_t* __restrict__ left_mask) {
+__device__ __forceinline__ void zone_chunk(ZoneSmem& sm, const TileCtx& c, uint32_t tile, uint32_t n_tiles,
+                                           uint32_t* __restrict__ left_mask, const FlushTo& out, uint32_t& left_total,
+                                           uint32_t& items_total) {
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     const int npol = c.npol;
     uint32_t* queue = sm.queue[wib];
     int queued = 0;                                              // warp-uniform, below 32 between iterations
-    // what every policy of the tile gets from this lane's requests (a lane sees at most 64 of them in a pass)
+    // what every policy of the tile gets from this lane's requests since the last flush (a lane sees at most 128 of
+    // a chunk's requests: its byte counts cannot overflow)
     uint32_t c_td = 0, c_ps = 0, c_pd = 0, c_tau = 0, c_dl = 0, c_cnt = 0;
     unsigned long long c_tt = 0;
-    uint32_t n_left = 0;
+    uint32_t n_left = 0, n_queued = 0;
     const uint32_t words = left_words_per_request(n_tiles);
     const uint32_t left_bit = 1u << (tile & 31u);
+    const uint32_t budget = WAITS ? kZItemsWaits : kZItems;
+    const uint32_t len = c.ch->len;
 
+    for (int i = threadIdx.x; i < (int)(offsetof(ZoneSmem, queue) / 4); i += kZThreads) ((uint32_t*)&sm)[i] = 0;
+    __syncthreads();
+    for (uint32_t r_lo = 0; r_lo < len; r_lo += kZStretch) {
+    const uint32_t r_hi = min(len, r_lo + kZStretch);
     Req nx = load_request<LEAN>(c, r_lo + threadIdx.x);
     for (uint32_t i0 = r_lo + wib * 32u; i0 < r_hi; i0 += kZThreads) {      // a warp's lanes iterate together
         const uint32_t i = i0 + lane;
@@ -271,14 +344,6 @@ __device__ __forceinline__ void zone_pass(ZoneSmem& sm, const TileCtx& c, uint32
             later = j > 0;
         }
         ok = ok && valid;
-        // a place in the block's budget of corrections
-        const uint32_t wants = __ballot_sync(0xFFFFFFFFu, ok && later);
-        if (wants) {
-            uint32_t place = 0;
-            if (lane == 0) place = atomicAdd(&sm.n_items, (uint32_t)__popc(wants));
-            place = __shfl_sync(0xFFFFFFFFu, place, 0) + __popc(wants & ((1u << lane) - 1u));
-            if (later && place >= kZPass) ok = false;            // (cannot happen: a pass is no longer than the budget)
-        }
         if (valid && !ok) {
             atomicOr(&left_mask[(size_t)(c.ch->start + i) * words + (tile >> 5)], left_bit);
             ++n_left;
@@ -297,6 +362,7 @@ __device__ __forceinline__ void zone_pass(ZoneSmem& sm, const TileCtx& c, uint32
             if (ok && later && DBG_OK(queued + __popc(enq & ((1u << lane) - 1u)), kZQueue, DBG_K_PAIRS_ZONES, DBG_SLOT))
                 queue[queued + __popc(enq & ((1u << lane) - 1u))] = i;
             queued += __popc(enq);
+            n_queued += (uint32_t)__popc(enq);
             __syncwarp();
             if (queued >= 32) {
                 drain_queue<WAITS, LEAN>(sm, c, queue, 32);
@@ -308,27 +374,43 @@ __device__ __forceinline__ void zone_pass(ZoneSmem& sm, const TileCtx& c, uint32
             }
         }
     }
-    if (queued > 0) drain_queue<WAITS, LEAN>(sm, c, queue, queued);
-    // ---- block totals of what every policy gets
-    uint32_t c_ca = cnt_pair_a(c_cnt), c_cb = cnt_pair_b(c_cnt);   // a lane's byte counts stay below 256
+    // ---- end of a stretch: flush now, or go on with the tables as they are?
+    if (lane == 0 && n_queued) { atomicAdd(&sm.n_items, n_queued); }
+    n_queued = 0;
+    __syncthreads();
+    const bool flush_now = r_hi == len || sm.n_items + kZStretch > budget;      // block-uniform
+    if (flush_now) {
+        if (queued > 0) { drain_queue<WAITS, LEAN>(sm, c, queue, queued); queued = 0; }
+        // block totals of what every policy gets
+        uint32_t c_ca = cnt_pair_a(c_cnt), c_cb = cnt_pair_b(c_cnt);   // a lane's byte counts stay below 256
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        c_td += __shfl_xor_sync(0xFFFFFFFFu, c_td, off); c_ps += __shfl_xor_sync(0xFFFFFFFFu, c_ps, off);
-        c_pd += __shfl_xor_sync(0xFFFFFFFFu, c_pd, off); c_tau += __shfl_xor_sync(0xFFFFFFFFu, c_tau, off);
-        c_dl += __shfl_xor_sync(0xFFFFFFFFu, c_dl, off); c_ca += __shfl_xor_sync(0xFFFFFFFFu, c_ca, off);
-        c_cb += __shfl_xor_sync(0xFFFFFFFFu, c_cb, off); c_tt += __shfl_xor_sync(0xFFFFFFFFu, c_tt, off);
-        n_left += __shfl_xor_sync(0xFFFFFFFFu, n_left, off);
+        for (int off = 16; off > 0; off >>= 1) {
+            c_td += __shfl_xor_sync(0xFFFFFFFFu, c_td, off); c_ps += __shfl_xor_sync(0xFFFFFFFFu, c_ps, off);
+            c_pd += __shfl_xor_sync(0xFFFFFFFFu, c_pd, off); c_tau += __shfl_xor_sync(0xFFFFFFFFu, c_tau, off);
+            c_dl += __shfl_xor_sync(0xFFFFFFFFu, c_dl, off); c_ca += __shfl_xor_sync(0xFFFFFFFFu, c_ca, off);
+            c_cb += __shfl_xor_sync(0xFFFFFFFFu, c_cb, off); c_tt += __shfl_xor_sync(0xFFFFFFFFu, c_tt, off);
+            n_left += __shfl_xor_sync(0xFFFFFFFFu, n_left, off);
+        }
+        if (lane == 0) {
+            // a warp adds once per flush: the 64-bit adds (compare-and-swap loops in shared memory) do not queue up
+            atomicAdd(&sm.c_sum[Z_TD], (unsigned long long)c_td); atomicAdd(&sm.c_sum[Z_PS], (unsigned long long)c_ps);
+            atomicAdd(&sm.c_sum[Z_PD], (unsigned long long)c_pd); atomicAdd(&sm.c_sum[Z_TAU], (unsigned long long)c_tau);
+            atomicAdd(&sm.c_sum[Z_DL], (unsigned long long)c_dl);
+            atomicAdd(&sm.c_sum[Z_CNT_A], (unsigned long long)(c_ca & 0xFFFFu) | ((unsigned long long)(c_ca >> 16) << 32));
+            atomicAdd(&sm.c_sum[Z_CNT_B], (unsigned long long)(c_cb & 0xFFFFu) | ((unsigned long long)(c_cb >> 16) << 32));
+            atomicAdd(&sm.c_sum[Z_TT_LO], c_tt);
+            atomicAdd(&sm.n_left, n_left);
+        }
+        c_td = c_ps = c_pd = c_tau = c_dl = c_cnt = 0; c_tt = 0; n_left = 0;
+        __syncthreads();
+        left_total += sm.n_left;
+        items_total += sm.n_items;
+        flush_tile(sm, npol, out);
+        __syncthreads();
+        for (int i = threadIdx.x; i < (int)(offsetof(ZoneSmem, queue) / 4); i += kZThreads) ((uint32_t*)&sm)[i] = 0;
+        __syncthreads();
     }
-    if (lane == 0) {
-        // sixteen warps, once each: the 64-bit adds (compare-and-swap loops in shared memory) do not queue up
-        atomicAdd(&sm.c_sum[Z_TD], (unsigned long long)c_td); atomicAdd(&sm.c_sum[Z_PS], (unsigned long long)c_ps);
-        atomicAdd(&sm.c_sum[Z_PD], (unsigned long long)c_pd); atomicAdd(&sm.c_sum[Z_TAU], (unsigned long long)c_tau);
-        atomicAdd(&sm.c_sum[Z_DL], (unsigned long long)c_dl);
-        atomicAdd(&sm.c_sum[Z_CNT_A], (unsigned long long)(c_ca & 0xFFFFu) | ((unsigned long long)(c_ca >> 16) << 32));
-        atomicAdd(&sm.c_sum[Z_CNT_B], (unsigned long long)(c_cb & 0xFFFFu) | ((unsigned long long)(c_cb >> 16) << 32));
-        atomicAdd(&sm.c_sum[Z_TT_LO], c_tt);
-        atomicAdd(&sm.n_left, n_left);
-    }
+    }   // next stretch
 }
 
 __global__ void __launch_bounds__(kZThreads, 1)
@@ -402,72 +484,17 @@ k_pairs_zones(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst*
     }
     // with pacing on and one histogram bin per stream, every regular interval of a stream lies in that bin (tau's)
     const bool lean = cc.pacing != 0 && cc.W[0] == 1 && cc.W[1] == 1 && cc.W[2] == 1;
-    const int bin_tau = bin_of_ticks(c.tau);
     uint32_t left_total = 0, items_total = 0;
 
-    const uint32_t pass_len = waits ? kZPassWaits : kZPass;
-    for (uint32_t r_lo = 0; r_lo < ch.len; r_lo += pass_len) {
-        const uint32_t r_hi = min(ch.len, r_lo + pass_len);
-        for (int i = threadIdx.x; i < (int)(offsetof(ZoneSmem, queue) / 4); i += kZThreads) ((uint32_t*)zsmem_raw)[i] = 0;
-        __syncthreads();
-        if (waits) {
-            if (lean) zone_pass<true, true>(sm, c, r_lo, r_hi, tile, n_tiles, left_mask);
-            else zone_pass<true, false>(sm, c, r_lo, r_hi, tile, n_tiles, left_mask);
-        } else {
-            if (lean) zone_pass<false, true>(sm, c, r_lo, r_hi, tile, n_tiles, left_mask);
-            else zone_pass<false, false>(sm, c, r_lo, r_hi, tile, n_tiles, left_mask);
-        }
-        __syncthreads();
-        left_total += sm.n_left;
-        items_total += sm.n_items;
-        // ---- flush: policy p gets the common part plus the difference rows above it (rows q > p)
-        //      (two threads a histogram word: one for the upper half of the policies, one for the lower half)
-        if ((threadIdx.x & 511) < kHWords) {
-            const int wd = threadIdx.x & 511;
-            const int half = npol > 16 ? 16 : 0;                                        // policies [half, npol) | [0, half)
-            const bool upper = threadIdx.x < 512;
-            int32_t t0 = (int32_t)sm.c_ttft[2 * wd], t1 = (int32_t)sm.c_ttft[2 * wd + 1];
-            int32_t s0 = (int32_t)sm.c_stall[2 * wd], s1 = (int32_t)sm.c_stall[2 * wd + 1];
-            for (int p = npol - 1; p >= (upper ? half : 0); --p) {
-                const uint32_t et = sm.e_ttft[p + 1][wd], es = sm.e_stall[p + 1][wd];   // row p + 1: for policies up to p
-                t0 += packed_lo(et); t1 += packed_hi(et); s0 += packed_lo(es); s1 += packed_hi(es);
-                if (!upper && p >= half) continue;                                      // (the other thread's policies)
-                const size_t o = (size_t)sm.pol[p] * kNBins + 2 * wd;
-                if (t0) atomicAdd(&hist_ttft[o], (unsigned long long)t0);
-                if (t1) atomicAdd(&hist_ttft[o + 1], (unsigned long long)t1);
-                if (s0) atomicAdd(&hist_tbt[o], (unsigned long long)s0);
-                if (s1) atomicAdd(&hist_tbt[o + 1], (unsigned long long)s1);
-            }
-        }
-        if (threadIdx.x >= 512 && threadIdx.x < 512 + 32 * kZSums) {                 // a thread per (field, policy)
-            const int f = (threadIdx.x - 512) >> 5, p = threadIdx.x & 31;
-            const bool is_packed = f == Z_CNT_A || f == Z_CNT_B;                    // two counts in the word
-            long long lo = is_packed ? (long long)(sm.c_sum[f] & 0xFFFFFFFFull) : (long long)sm.c_sum[f];
-            long long hi = is_packed ? (long long)(sm.c_sum[f] >> 32) : 0;
-            for (int q = p + 1; q <= npol; ++q) {                                   // the rows above the policy
-                const uint32_t e = sm.e_sum[q][f];
-                if (is_packed) { lo += packed_lo(e); hi += packed_hi(e); } else lo += (int32_t)e;
-            }
-            if (p < npol) {
-                const uint32_t pp = sm.pol[p];
-                unsigned long long* a = acc + ((size_t)pp * tr.n_groups + g) * kNAcc;
-                // (the two halves of the TTFT sum may be negative on their own: the 64-bit adds wrap to the right total)
-                switch (f) {
-                    case Z_TD: if (lo) atomicAdd(&a[A_TOK_DEVICE], (unsigned long long)lo); break;
-                    case Z_PS: if (lo) atomicAdd(&a[A_PRE_SERVER], (unsigned long long)lo); break;
-                    case Z_PD: if (lo) atomicAdd(&a[A_PRE_DEVICE], (unsigned long long)lo); break;
-                    case Z_TAU: if (lo) atomicAdd(&hist_tbt[(size_t)pp * kNBins + bin_tau], (unsigned long long)lo); break;
-                    case Z_DL: if (lo) atomicAdd(&a[A_DELAYED], (unsigned long long)lo); break;
-                    case Z_CNT_A: if (lo) atomicAdd(&a[A_DEVICE_ONLY], (unsigned long long)lo);
-                                  if (hi) atomicAdd(&a[A_RACE], (unsigned long long)hi); break;
-                    case Z_CNT_B: if (lo) atomicAdd(&a[A_DEVICE_WON], (unsigned long long)lo);
-                                  if (hi) atomicAdd(&a[A_MIGR], (unsigned long long)hi); break;
-                    case Z_TT_LO: if (lo) atomicAdd(&a[A_TTFT_SUM], (unsigned long long)lo); break;
-                    default: if (lo) atomicAdd(&a[A_TTFT_SUM], (unsigned long long)lo << 16); break;   // Z_TT_HI
-                }
-            }
-        }
-        __syncthreads();
+    FlushTo out;
+    out.acc = acc; out.hist_ttft = hist_ttft; out.hist_tbt = hist_tbt; out.n_groups = tr.n_groups; out.g = g;
+    out.bin_tau = bin_of_ticks(c.tau);
+    if (waits) {
+        if (lean) zone_chunk<true, true>(sm, c, tile, n_tiles, left_mask, out, left_total, items_total);
+        else zone_chunk<true, false>(sm, c, tile, n_tiles, left_mask, out, left_total, items_total);
+    } else {
+        if (lean) zone_chunk<false, true>(sm, c, tile, n_tiles, left_mask, out, left_total, items_total);
+        else zone_chunk<false, false>(sm, c, tile, n_tiles, left_mask, out, left_total, items_total);
     }
     if (threadIdx.x == 0) {
         left_count[(size_t)chunk_id * n_tiles + tile] = left_total;
