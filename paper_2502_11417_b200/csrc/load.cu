@@ -19,18 +19,20 @@ __global__ void k_ingest(uint32_t n, const int32_t* __restrict__ prompt, const i
                          uint32_t* __restrict__ grp_n, uint32_t* __restrict__ max_n, int32_t* __restrict__ err,
                          int32_t* __restrict__ S_out, uint16_t* __restrict__ l_out, uint16_t* __restrict__ n_out,
                          uint32_t* __restrict__ orig_out, uint32_t* __restrict__ counts0, uint32_t per_block0,
-                         uint32_t blocks0) {
+                         uint32_t blocks0, int hist_groups) {
     // S_out, orig_out: single-group traces keep the caller's order, so the internal arrays are written here (l_out,
     // n_out are then the internal arrays too; otherwise packed copies in the caller's order for the gather);
     // counts0: first radix digit counted per sort block (small traces; large ones use the histogram kernel)
     __shared__ unsigned long long s_sum[kMaxGroups];
     __shared__ uint32_t s_cnt[kMaxGroups];
     __shared__ uint32_t s_max, s_max_ticks;         // longest output, largest TTFT ticks (max_n[0], max_n[1])
-    __shared__ uint32_t s_len[kMaxPrompt + 1];       // length histogram of this block (single-group traces)
+    // hist_groups: groups whose length histograms this block keeps in shared memory (all of them, or none when they
+    // do not fit: then the counts go to global memory one by one)
+    extern __shared__ uint32_t s_len[];              // [hist_groups][kMaxPrompt + 1]
     const int G = (int)(ns * nd);
     const bool one = G == 1;
     for (int g = threadIdx.x; g < G; g += blockDim.x) { s_sum[g] = 0; s_cnt[g] = 0; }
-    if (one) for (int i = threadIdx.x; i <= kMaxPrompt; i += blockDim.x) s_len[i] = 0;
+    for (int i = threadIdx.x; i < hist_groups * (kMaxPrompt + 1); i += blockDim.x) s_len[i] = 0;
     if (threadIdx.x == 0) { s_max = 0; s_max_ticks = 0; }
     __syncthreads();
     const uint32_t stride = gridDim.x * blockDim.x;
@@ -55,7 +57,7 @@ __global__ void k_ingest(uint32_t n, const int32_t* __restrict__ prompt, const i
         const uint32_t g = ok ? s * nd + d : 0u;
         if (ok && DBG_OK(g, G, DBG_K_INGEST, DBG_GROUP) && DBG_OK(l, kMaxPrompt + 1, DBG_K_INGEST, DBG_TABLE)) {
             keys[i] = ((uint64_t)g << 32) | (uint32_t)S;
-            if (one) atomicAdd(&s_len[l], 1u); else atomicAdd(&cnt[g * (kMaxPrompt + 1) + l], 1u);
+            if (hist_groups) atomicAdd(&s_len[g * (kMaxPrompt + 1) + l], 1u); else atomicAdd(&cnt[g * (kMaxPrompt + 1) + l], 1u);
             if (S_out) { S_out[i] = (int32_t)S; orig_out[i] = i; }
             l_out[i] = (uint16_t)l; n_out[i] = (uint16_t)o;
             if (counts0 && DBG_OK(i / per_block0, blocks0, DBG_K_INGEST, DBG_COUNTER))
@@ -70,15 +72,28 @@ __global__ void k_ingest(uint32_t n, const int32_t* __restrict__ prompt, const i
                 atomicAdd(&s_sum[0], (unsigned long long)so); atomicAdd(&s_cnt[0], co); atomicMax(&s_max, mo);
                 atomicMax(&s_max_ticks, mt);
             }
-        } else if (ok) {
-            atomicAdd(&s_sum[g], (unsigned long long)o); atomicAdd(&s_cnt[g], 1u); atomicMax(&s_max, (uint32_t)o);
-            atomicMax(&s_max_ticks, (uint32_t)S);
+        } else {
+            // several groups: the lanes of each group present in the warp add up among themselves, one lane adds
+            const uint32_t mo = __reduce_max_sync(0xFFFFFFFFu, ok ? (uint32_t)o : 0u);
+            const uint32_t mt = __reduce_max_sync(0xFFFFFFFFu, ok ? (uint32_t)S : 0u);
+            uint32_t rest = __ballot_sync(0xFFFFFFFFu, ok);
+            const int lane = threadIdx.x & 31;
+            if (lane == 0 && rest) { atomicMax(&s_max, mo); atomicMax(&s_max_ticks, mt); }
+            while (rest) {
+                const int first = __ffs(rest) - 1;
+                const uint32_t g1 = __shfl_sync(0xFFFFFFFFu, g, first);
+                const bool mine = ok && g == g1;
+                const uint32_t same = __ballot_sync(0xFFFFFFFFu, mine);
+                const uint32_t so = __reduce_add_sync(0xFFFFFFFFu, mine ? (uint32_t)o : 0u);
+                if (lane == first) { atomicAdd(&s_sum[g1], (unsigned long long)so); atomicAdd(&s_cnt[g1], (uint32_t)__popc(same)); }
+                rest &= ~same;
+            }
         }
     }
     __syncthreads();
     for (int g = threadIdx.x; g < G; g += blockDim.x)
         if (s_cnt[g]) { atomicAdd(&grp_sum_n[g], s_sum[g]); atomicAdd(&grp_n[g], s_cnt[g]); }
-    if (one) for (int i = threadIdx.x; i <= kMaxPrompt; i += blockDim.x) if (s_len[i]) atomicAdd(&cnt[i], s_len[i]);
+    for (int i = threadIdx.x; i < hist_groups * (kMaxPrompt + 1); i += blockDim.x) if (s_len[i]) atomicAdd(&cnt[i], s_len[i]);
     if (threadIdx.x == 0 && s_max) { atomicMax(max_n, s_max); atomicMax(max_n + 1, s_max_ticks); }
 }
 
@@ -387,11 +402,15 @@ cudaError_t run_load(const LoadArgs& a, cudaStream_t st) {
     if (n) {
         uint32_t* counts_a = a.radix_counts;                                   // small path: pass p uses slice p
         uint32_t* counts_b = a.radix_counts + (size_t)4 * 256u * kRadixMaxBlocks;  // large path: one scanned buffer
-        k_ingest<<<std::min(grid_for(n, 4 * kIngestThreads, a.sms), 2 * a.sms), kIngestThreads, 0, st>>>(
+        // block-private length histograms while they fit two blocks to a multiprocessor (up to six groups)
+        const int hist_groups = (size_t)G * (kMaxPrompt + 1) * 4 <= 100 * 1024 ? G : 0;
+        const size_t hist_bytes = (size_t)hist_groups * (kMaxPrompt + 1) * 4;
+        if ((e = cudaFuncSetAttribute(k_ingest, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024))) return e;
+        k_ingest<<<std::min(grid_for(n, 4 * kIngestThreads, a.sms), 2 * a.sms), kIngestThreads, hist_bytes, st>>>(
             n, a.prompt, a.outlen, a.ttft, a.sp, a.dp, a.ns, a.nd, a.keys_a, a.cnt,
             (unsigned long long*)a.grp_sum_n, a.ng, a.max_n, a.err,
             G == 1 ? a.S : nullptr, G == 1 ? a.l : a.l_tmp, G == 1 ? a.nout : a.n_tmp, a.orig,
-            small ? counts_a : nullptr, per_block, blocks);
+            small ? counts_a : nullptr, per_block, blocks, hist_groups);
         if (G > 1) {
             // internal request order: stable partition by group
             if ((e = radix_pass(a.keys_a, a.keys_b, nullptr, a.tmp_idx, n, 32, counts_b, st))) return e;
