@@ -350,6 +350,31 @@ def test_pinned_host_inputs_read_in_place_match_pageable_ones():
         Trace().load_trace(*pinned, None, None, w.servers, w.devices)
 
 
+def test_pinned_host_inputs_of_several_groups_and_staged_copies():
+    # six groups: page-locked arrays are read in place as well (packed copies of the lengths feed the partition);
+    # arrays_on_device = 2 copies them with the copy engine instead.  All three routes give identical records.
+    import torch
+    from parity import check_tables
+    from oracle import Oracle
+    w = synth.make_workload(4, n=25013, n_budgets=3)
+    cols = (w.prompt_len, w.output_len, w.server_ttft_s, w.server_profile, w.device_profile)
+    a = Trace.from_workload(w)                                  # pageable numpy arrays: copied
+    a.eval_policies(w.policies, 9)
+    sa = a.reduce_stats()
+    pinned = [torch.from_numpy(x).pin_memory() for x in cols]
+    for staged in (False, True):
+        b = Trace().load_trace(*pinned, w.servers, w.devices, staged_copy=staged)
+        check_tables(b, Oracle.from_workload(w), f"pinned staged={staged}")
+        b.eval_policies(w.policies, 9)
+        sb = b.reduce_stats()
+        for p in range(len(w.policies)):
+            assert bytes(sa[p]) == bytes(sb[p]), (staged, p)
+        b.close()
+    pinned[3][11] = 7                                          # validation still sees the in-place arrays
+    with pytest.raises(DiscoError):
+        Trace().load_trace(*pinned, w.servers, w.devices)
+
+
 def test_non_default_stream_and_partial_outputs():
     import torch
     w = synth.make_workload(1, n=3000, n_budgets=4)
