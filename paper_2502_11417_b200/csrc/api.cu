@@ -11,6 +11,7 @@
 
 #include "disco_internal.cuh"
 #include "load.cuh"
+#include "tile.cuh"
 
 using namespace disco;
 
@@ -506,7 +507,10 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
 
     // scratch of the pair kernels: a bit per (request, policy tile), a counter per (chunk, policy tile)
     const size_t left_mask_words = (size_t)N1 * ((tiles + 31) / 32);
-    if ((e = c->d_left.reserve((left_mask_words + chunks.size() * (size_t)tiles + 4) * 4)) != cudaSuccess)
+    // ... and, while that stays below 1 GB, a short list of flagged requests per (chunk, tile)
+    const size_t left_cells = chunks.size() * (size_t)tiles;
+    const size_t left_list_words = left_cells * kLeftList * 4 <= (1ull << 30) ? left_cells * kLeftList : 0;
+    if ((e = c->d_left.reserve((left_mask_words + left_cells + left_list_words + 4) * 4)) != cudaSuccess)
         return fail_cuda(e, "device allocation for the evaluation");
 
     // ---- small tables to the device through pinned staging
@@ -591,7 +595,9 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
                         c->d_pol_list.as<uint32_t>() + cls_range[k].first, cls_range[k].second - cls_range[k].first,
                         c->d_chunks.as<Chunk>(), (uint32_t)chunks.size(), rec, po, c->d_acc.as<uint64_t>(),
                         c->d_hist_ttft.as<uint64_t>(), c->d_hist_tbt.as<uint64_t>(), c->d_left.as<uint32_t>(),
-                        c->d_left.as<uint32_t>() + left_mask_words, c->d_work.as<uint64_t>(), k0, cls_extras_pending,
+                        c->d_left.as<uint32_t>() + left_mask_words,
+                        left_list_words ? c->d_left.as<uint32_t>() + left_mask_words + left_cells : nullptr,
+                        c->d_work.as<uint64_t>(), k0, cls_extras_pending,
                         !classes[k].pacing || classes[k].W[0] > 1 || classes[k].W[1] > 1 || classes[k].W[2] > 1,
                         timed ? c->ev[3] : nullptr, st));
         if (timed) CU(cudaEventRecord(c->ev[4], st));

@@ -210,6 +210,7 @@ cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassCo
                          uint32_t* left_mask /* [n][ceil(tiles / 32)] scratch for the requests the zone kernel leaves to
                          the pair kernel, or null: every pair is evaluated one by one */,
                          uint32_t* left_count /* [n_chunks][tiles] scratch */,
+                         uint32_t* left_lists /* [n_chunks][tiles][kLeftList] scratch, or null */,
                          uint64_t* work /* [3], added to: pairs settled zone by zone, pairs evaluated one by one,
                          requests settled per tile */,
                          uint32_t k0, bool extras /* some policy routes at random or uses an
@@ -219,8 +220,8 @@ cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassCo
 cudaError_t launch_pairs_zones(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const Prep* prep,
                                uint32_t P, const uint32_t* pol_list, uint32_t n_list, int PL, const Chunk* chunks,
                                uint32_t n_chunks, TimelineRec rec, uint64_t* acc, uint64_t* hist_ttft,
-                               uint64_t* hist_tbt, uint32_t* left_mask, uint32_t* left_count, uint64_t* work,
-                               cudaStream_t st);
+                               uint64_t* hist_tbt, uint32_t* left_mask, uint32_t* left_count, uint32_t* left_lists,
+                               uint64_t* work, cudaStream_t st);
 cudaError_t launch_finalize(uint32_t P, int G, const GroupConst* gc, const uint64_t* acc, const uint64_t* hist_ttft,
                             const uint64_t* hist_tbt,
                             const uint64_t* fin_totals /* [2G]: output tokens per group, then requests per group */,

@@ -93,7 +93,8 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
             int PL, const Chunk* __restrict__ chunks, uint32_t n_tiles, TimelineRec rec, uint32_t k0,
             unsigned long long* __restrict__ acc, unsigned long long* __restrict__ hist_ttft,
             unsigned long long* __restrict__ hist_tbt, const uint32_t* __restrict__ left_mask,
-            const uint32_t* __restrict__ left_count, unsigned long long* __restrict__ work) {
+            const uint32_t* __restrict__ left_count, const uint32_t* __restrict__ left_lists,
+            unsigned long long* __restrict__ work) {
     extern __shared__ uint32_t smem[];
     uint32_t* h_ttft = smem;                                  // [PL][kHWords]
     uint32_t* h_stall = smem + PL * kHWords;                  // [PL][kHWords]
@@ -370,6 +371,15 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
             run_batch(d, n_held == 32 ? 0xFFFFFFFFu : (1u << n_held) - 1u, 0u);
             n_held = 0;
         };
+        if (left_lists && to_do <= kLeftList) {
+            // few enough to be listed by position: no scan
+            const uint32_t* list = left_lists + ((size_t)chunk_id * n_tiles + tile) * kLeftList;
+            for (uint32_t k0l = wib * 32u; k0l < to_do; k0l += kAccWarps * 32u) {
+                n_held = (int)min(32u, to_do - k0l);
+                if (lane < n_held) held = list[k0l + lane];
+                work_off();
+            }
+        } else {
         constexpr int kScan = 4;                                 // flag words a lane has in flight
         constexpr uint32_t kStride = kAccWarps * kStageReq;
         auto flags_at = [&](uint32_t at) {
@@ -393,6 +403,7 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
             }
         }
         if (n_held > 0) work_off();
+        }
     }
     // ---- block totals, then one flush per block.  With fewer than 32 policies in the tile several lanes of a warp
     //      hold sums of the same policy: they are added up by shuffles first, so that one lane per policy and warp
@@ -595,7 +606,8 @@ DBG_TRANSLATION_UNIT()
 cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const Prep* prep, uint32_t P,
                          const uint32_t* pol_list, uint32_t n_list, const Chunk* chunks, uint32_t n_chunks,
                          TimelineRec rec, disco_pair_out_t out, uint64_t* acc, uint64_t* hist_ttft,
-                         uint64_t* hist_tbt, uint32_t* left_mask, uint32_t* left_count, uint64_t* work, uint32_t k0,
+                         uint64_t* hist_tbt, uint32_t* left_mask, uint32_t* left_count, uint32_t* left_lists,
+                         uint64_t* work, uint32_t k0,
                          bool extras, bool wide, cudaEvent_t mid, cudaStream_t st) {
     if (n_chunks == 0 || n_list == 0) return mid ? cudaEventRecord(mid, st) : cudaSuccess;
     int PL = 1;
@@ -613,14 +625,14 @@ cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassCo
         const size_t mask_bytes = (size_t)tr.n * left_words_per_request(n_tiles) * 4;
         if ((e = cudaMemsetAsync(left_mask, 0, mask_bytes, st))) return e;
         if ((e = launch_pairs_zones(tr, gc, cc, prep, P, pol_list, n_list, PL, chunks, n_chunks, rec, acc, hist_ttft,
-                                    hist_tbt, left_mask, left_count, work, st)))
+                                    hist_tbt, left_mask, left_count, left_lists, work, st)))
             return e;
     }
     if ((e = launch_after(acc_kernel, dim3(n_chunks * n_tiles), kAccThreads, acc_smem_bytes(PL), st, tr, gc, cc, prep, P,
                           pol_list, n_list, PL, chunks, n_tiles, rec, k0, (unsigned long long*)acc,
                           (unsigned long long*)hist_ttft, (unsigned long long*)hist_tbt,
                           (const uint32_t*)(zones ? left_mask : nullptr), (const uint32_t*)left_count,
-                          (unsigned long long*)work)))
+                          (const uint32_t*)left_lists, (unsigned long long*)work)))
         return e;
     if (mid && (e = cudaEventRecord(mid, st))) return e;
     const bool rows = out.ttft_s || out.tbt_mean_s || out.tbt_max_s || out.cost || out.tok_server || out.tok_device ||

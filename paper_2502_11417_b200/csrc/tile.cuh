@@ -54,5 +54,8 @@ __device__ __forceinline__ bool tile_by_zones(const Prep& pr, bool act, int lane
 // Requests a zone-by-zone kernel could not settle for a tile are flagged in a bit mask: word
 // request * words_per_request + tile / 32, bit tile % 32.
 __host__ __device__ __forceinline__ uint32_t left_words_per_request(uint32_t n_tiles) { return (n_tiles + 31u) / 32u; }
+// The first kLeftList of them per (chunk, tile) are also listed by chunk position, so that the pair kernel need not
+// scan the flags of a chunk for a handful of requests.
+constexpr uint32_t kLeftList = 2048;
 
 }  // namespace disco

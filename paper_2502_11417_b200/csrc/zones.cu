@@ -49,7 +49,8 @@ struct ZoneSmem {
     uint32_t e_sum[kZRows][kZSumStride];   // difference rows of the sums (wrap-around 32-bit words)
     unsigned long long c_sum[kZSums];
     uint32_t n_left, n_items;
-    // ---- not cleared between passes
+    // ---- not cleared between flushes
+    uint32_t n_listed;                  // requests left to the pair kernel so far (their list positions)
     uint32_t queue[kZWarps][kZQueue];   // requests (chunk-relative) that await their corrections
     int32_t key[32];                    // the policies' length thresholds, in tile order
     uint32_t w_star[32];                // Algorithm 2: the wait of the length class l*
@@ -298,8 +299,8 @@ __device__ __forceinline__ void flush_tile(ZoneSmem& sm, int npol, const FlushTo
 // fit the signed 16-bit counts of the difference rows -- and at the end of the chunk.
 template <bool WAITS, bool LEAN>
 __device__ __forceinline__ void zone_chunk(ZoneSmem& sm, const TileCtx& c, uint32_t tile, uint32_t n_tiles,
-                                           uint32_t* __restrict__ left_mask, const FlushTo& out, uint32_t& left_total,
-                                           uint32_t& items_total) {
+                                           uint32_t* __restrict__ left_mask, uint32_t* __restrict__ left_list,
+                                           const FlushTo& out, uint32_t& left_total, uint32_t& items_total) {
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     const int npol = c.npol;
     uint32_t* queue = sm.queue[wib];
@@ -347,6 +348,7 @@ __device__ __forceinline__ void zone_chunk(ZoneSmem& sm, const TileCtx& c, uint3
         if (valid && !ok) {
             atomicOr(&left_mask[(size_t)(c.ch->start + i) * words + (tile >> 5)], left_bit);
             ++n_left;
+            if (left_list) { const uint32_t at = atomicAdd(&sm.n_listed, 1u); if (at < kLeftList) left_list[at] = i; }
         }
         // ---- every policy of the tile gets the outcome of the last run
         if (ok) {
@@ -419,7 +421,8 @@ k_pairs_zones(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst*
               int PL, const Chunk* __restrict__ chunks, uint32_t n_tiles, TimelineRec rec,
               unsigned long long* __restrict__ acc, unsigned long long* __restrict__ hist_ttft,
               unsigned long long* __restrict__ hist_tbt, uint32_t* __restrict__ left_mask,
-              uint32_t* __restrict__ left_count, unsigned long long* __restrict__ work) {
+              uint32_t* __restrict__ left_count, uint32_t* __restrict__ left_lists,
+              unsigned long long* __restrict__ work) {
     extern __shared__ __align__(16) unsigned char zsmem_raw[];
     ZoneSmem& sm = *reinterpret_cast<ZoneSmem*>(zsmem_raw);
     grid_dependency_wait();
@@ -460,6 +463,8 @@ k_pairs_zones(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst*
         c.wt_ordered = __all_sync(0xFFFFFFFFu, lane + 1 >= npol || (uint32_t)pr.w_tail >= next) != 0;
     }
 
+    if (threadIdx.x == 0) sm.n_listed = 0;
+    uint32_t* left_list = left_lists ? left_lists + ((size_t)chunk_id * n_tiles + tile) * kLeftList : nullptr;
     if (wib == 0 && lane < npol) {
         sm.key[lane] = waits ? pr.l_star : pr.l_th;
         sm.w_star[lane] = (uint32_t)pr.w_star;
@@ -490,11 +495,11 @@ k_pairs_zones(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst*
     out.acc = acc; out.hist_ttft = hist_ttft; out.hist_tbt = hist_tbt; out.n_groups = tr.n_groups; out.g = g;
     out.bin_tau = bin_of_ticks(c.tau);
     if (waits) {
-        if (lean) zone_chunk<true, true>(sm, c, tile, n_tiles, left_mask, out, left_total, items_total);
-        else zone_chunk<true, false>(sm, c, tile, n_tiles, left_mask, out, left_total, items_total);
+        if (lean) zone_chunk<true, true>(sm, c, tile, n_tiles, left_mask, left_list, out, left_total, items_total);
+        else zone_chunk<true, false>(sm, c, tile, n_tiles, left_mask, left_list, out, left_total, items_total);
     } else {
-        if (lean) zone_chunk<false, true>(sm, c, tile, n_tiles, left_mask, out, left_total, items_total);
-        else zone_chunk<false, false>(sm, c, tile, n_tiles, left_mask, out, left_total, items_total);
+        if (lean) zone_chunk<false, true>(sm, c, tile, n_tiles, left_mask, left_list, out, left_total, items_total);
+        else zone_chunk<false, false>(sm, c, tile, n_tiles, left_mask, left_list, out, left_total, items_total);
     }
     if (threadIdx.x == 0) {
         left_count[(size_t)chunk_id * n_tiles + tile] = left_total;
@@ -513,15 +518,15 @@ DBG_TRANSLATION_UNIT()
 cudaError_t launch_pairs_zones(const TraceDev& tr, const GroupConst* gc, const ClassConst* cc, const Prep* prep,
                                uint32_t P, const uint32_t* pol_list, uint32_t n_list, int PL, const Chunk* chunks,
                                uint32_t n_chunks, TimelineRec rec, uint64_t* acc, uint64_t* hist_ttft,
-                               uint64_t* hist_tbt, uint32_t* left_mask, uint32_t* left_count, uint64_t* work,
-                               cudaStream_t st) {
+                               uint64_t* hist_tbt, uint32_t* left_mask, uint32_t* left_count, uint32_t* left_lists,
+                               uint64_t* work, cudaStream_t st) {
     const uint32_t n_tiles = (n_list + PL - 1) / PL;
     if ((uint64_t)n_chunks * n_tiles > 0x7FFFFFFFull) return cudaErrorInvalidConfiguration;
     cudaError_t e = cudaFuncSetAttribute(k_pairs_zones, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ZoneSmem));
     if (e) return e;
     return launch_after(k_pairs_zones, dim3(n_chunks * n_tiles), kZThreads, sizeof(ZoneSmem), st, tr, gc, cc, prep, P,
                         pol_list, n_list, PL, chunks, n_tiles, rec, (unsigned long long*)acc,
-                        (unsigned long long*)hist_ttft, (unsigned long long*)hist_tbt, left_mask, left_count,
+                        (unsigned long long*)hist_ttft, (unsigned long long*)hist_tbt, left_mask, left_count, left_lists,
                         (unsigned long long*)work);
 }
 
