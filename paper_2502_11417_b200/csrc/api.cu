@@ -98,7 +98,7 @@ struct disco_ctx {
     const void* gc_dev_at = nullptr;
     // trace
     DevBuf in_prompt, in_out, in_ttft, in_sp, in_dp;      // staging of host inputs
-    DevBuf keys_a, keys_b, tmp_idx, tmp_ln;
+    DevBuf keys_a, keys_b, tmp_idx, tmp_ln, cursors, inv;
     DevBuf S, l, nout, orig, sorted;
     DevBuf zero, cum_mass, ng_exact, grp_off, knots, d_gc;   // `zero`: every table a load must clear, contiguous
     DevBuf fin_totals;                 // [2G] u64: output tokens and requests per group that the accumulators cover
@@ -138,7 +138,7 @@ struct disco_ctx {
     bool timing_valid = false;
 
     ~disco_ctx() {
-        DevBuf* all[] = {&in_prompt, &in_out, &in_ttft, &in_sp, &in_dp, &keys_a, &keys_b, &tmp_idx, &tmp_ln,
+        DevBuf* all[] = {&in_prompt, &in_out, &in_ttft, &in_sp, &in_dp, &keys_a, &keys_b, &tmp_idx, &tmp_ln, &cursors, &inv,
                          &S, &l, &nout, &orig, &sorted, &zero, &cum_mass, &ng_exact, &grp_off, &knots, &d_gc, &d_prep, &d_accum, &d_stats, &d_tables, &d_todo,
                          &fin_totals, &F_sorted_imp, &F_off_imp, &d_left};
         for (DevBuf* b : all) b->release();
@@ -205,8 +205,8 @@ cudaError_t reserve_trace(disco_ctx* c, uint32_t n, bool host_inputs, bool has_s
         if (has_sp) R(in_sp, N);
         if (has_dp) R(in_dp, N);
     }
-    R(keys_a, N * 8); R(keys_b, N * 8); R(tmp_idx, N * 4);
-    if (G > 1) R(tmp_ln, N * 4);
+    R(keys_a, N * 8); R(keys_b, N * 8);
+    R(tmp_ln, N * 4); R(cursors, (size_t)G * (kMaxPrompt + 1) * 4); R(inv, N * 4);
     R(S, N * 4); R(l, N * 2); R(nout, N * 2); R(orig, N * 4); R(sorted, N * 4);
     // one block for everything a load clears: cnt | grp_sum_n | ng | max_n | err | first radix counter buffer,
     // followed by the second counter buffer
@@ -311,7 +311,7 @@ int disco_load_trace(disco_ctx_t** pctx, const disco_trace_desc_t* d, void* stre
         a.prompt = d->prompt_len; a.outlen = d->output_len; a.ttft = d->server_ttft_s;
         a.sp = d->server_profile; a.dp = d->device_profile;
     }
-    a.keys_a = c->keys_a.as<uint64_t>(); a.keys_b = c->keys_b.as<uint64_t>(); a.tmp_idx = c->tmp_idx.as<uint32_t>();
+    a.keys_a = c->keys_a.as<uint64_t>(); a.keys_b = c->keys_b.as<uint64_t>(); a.cursors = c->cursors.as<uint32_t>(); a.inv = c->inv.as<uint32_t>();
     a.l_tmp = c->tmp_ln.as<uint16_t>(); a.n_tmp = c->tmp_ln.as<uint16_t>() + (n ? n : 1);
     a.radix_counts = c->radix_counts; a.zero_block = c->zero.p; a.zero_bytes = c->zero_bytes;
     a.ng_exact = c->ng_exact.as<uint32_t>(); a.readback = c->rb;     // pinned host memory, written by the last kernel
@@ -480,17 +480,19 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
         cls_range.push_back({b, (uint32_t)pol_list.size()});
     }
     const uint32_t tiles = (P + 31) / 32;
-    // a lane of the zone kernel counts its requests in bytes: at most 255 requests a lane, 512 lanes a block
+    // the zone kernel runs a block per (chunk, family of four policy tiles); a lane of it counts its requests in
+    // bytes: at most 127 requests a lane, 1024 lanes a block
     const uint32_t kMaxChunk = 130560;
     const uint32_t sms = (uint32_t)c->sms;
-    uint32_t want_chunks = std::max<uint32_t>(1, sms / std::min<uint32_t>(tiles, sms));   // one block per SM
+    const uint32_t fams = (tiles + 3) / 4;
+    uint32_t want_chunks = std::max<uint32_t>(1, sms / std::min<uint32_t>(fams, sms));   // one block per SM
     const uint32_t min_chunks = (uint32_t)((N1 + kMaxChunk - 1) / kMaxChunk);
     if (min_chunks > want_chunks) {
         // several waves of blocks: the fewest chunks whose last wave is nearly full (long chunks spread a block's
         // set-up and flush over more requests), else the count near the minimum whose last wave is fullest
         double best = 0.0;
         for (uint32_t k = min_chunks; k < min_chunks + sms; ++k) {
-            const uint64_t blocks = (uint64_t)k * tiles, waves = (blocks + sms - 1) / sms;
+            const uint64_t blocks = (uint64_t)k * fams, waves = (blocks + sms - 1) / sms;
             const double fill = (double)blocks / (double)(waves * sms);
             if (fill > best + 1e-9) { best = fill; want_chunks = k; }
             if (fill >= 0.94) break;
@@ -558,7 +560,7 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
 
     TraceDev tr;
     tr.n = n; tr.n_groups = G; tr.S = c->S.as<int32_t>(); tr.l = c->l.as<uint16_t>(); tr.nout = c->nout.as<uint16_t>();
-    tr.orig = c->orig.as<uint32_t>(); tr.grp_off = c->grp_off.as<uint32_t>();
+    tr.orig = c->orig.as<uint32_t>(); tr.inv = c->inv.as<uint32_t>(); tr.len_end = c->cursors.as<uint32_t>(); tr.grp_off = c->grp_off.as<uint32_t>();
     TimelineRec rec;
     for (int k = 0; k < 3; ++k) {
         rec.sum[k] = c->rec_u32[2 * k].as<uint32_t>(); rec.max[k] = c->rec_u32[2 * k + 1].as<uint32_t>();
@@ -597,7 +599,7 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
                         c->d_hist_ttft.as<uint64_t>(), c->d_hist_tbt.as<uint64_t>(), c->d_left.as<uint32_t>(),
                         c->d_left.as<uint32_t>() + left_mask_words,
                         left_list_words ? c->d_left.as<uint32_t>() + left_mask_words + left_cells : nullptr,
-                        c->d_work.as<uint64_t>(), k0, cls_extras_pending,
+                        sms, c->d_work.as<uint64_t>(), k0, cls_extras_pending,
                         !classes[k].pacing || classes[k].W[0] > 1 || classes[k].W[1] > 1 || classes[k].W[2] > 1,
                         timed ? c->ev[3] : nullptr, st));
         if (timed) CU(cudaEventRecord(c->ev[4], st));

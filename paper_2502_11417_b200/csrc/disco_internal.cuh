@@ -76,9 +76,11 @@ struct TimelineRec {
 struct TraceDev {
     uint32_t n;
     int32_t n_groups;
-    const int32_t* S;            // server TTFT ticks, internal order (requests partitioned by group)
+    const int32_t* S;            // server TTFT ticks, internal order: by group, inside a group by prompt length
     const uint16_t *l, *nout;
     const uint32_t* orig;        // caller's index of each request
+    const uint32_t* inv;         // place of each of the caller's requests in the internal order
+    const uint32_t* len_end;     // [G][4097]: where the group's requests of each prompt length end (the next length starts)
     const uint32_t* grp_off;     // [G+1]
 };
 
@@ -211,8 +213,9 @@ cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassCo
                          the pair kernel, or null: every pair is evaluated one by one */,
                          uint32_t* left_count /* [n_chunks][tiles] scratch */,
                          uint32_t* left_lists /* [n_chunks][tiles][kLeftList] scratch, or null */,
-                         uint64_t* work /* [3], added to: pairs settled zone by zone, pairs evaluated one by one,
-                         requests settled per tile */,
+                         uint32_t zone_blocks /* blocks the zone kernel may run: one per multiprocessor */,
+                         uint64_t* work /* [4], added to: pairs settled zone by zone, pairs evaluated one by one,
+                         requests settled per policy family, sweeps over segments of a chunk */,
                          uint32_t k0, bool extras /* some policy routes at random or uses an
                          expected length */, bool wide /* some window W of the class spans several bins */,
                          cudaEvent_t mid /* recorded between its two kernels, or null */,
@@ -221,7 +224,7 @@ cudaError_t launch_pairs_zones(const TraceDev& tr, const GroupConst* gc, const C
                                uint32_t P, const uint32_t* pol_list, uint32_t n_list, int PL, const Chunk* chunks,
                                uint32_t n_chunks, TimelineRec rec, uint64_t* acc, uint64_t* hist_ttft,
                                uint64_t* hist_tbt, uint32_t* left_mask, uint32_t* left_count, uint32_t* left_lists,
-                               uint64_t* work, cudaStream_t st);
+                               uint32_t max_blocks, uint64_t* work, cudaStream_t st);
 cudaError_t launch_finalize(uint32_t P, int G, const GroupConst* gc, const uint64_t* acc, const uint64_t* hist_ttft,
                             const uint64_t* hist_tbt,
                             const uint64_t* fin_totals /* [2G]: output tokens per group, then requests per group */,

@@ -1,5 +1,5 @@
 // Trace ingestion on the device: tick conversion and validation, per-group prompt-length histogram,
-// stable partition of the requests by group, radix sort of the server-TTFT ticks (the empirical F of
+// internal request order (by group, then by prompt length), radix sort of the server-TTFT ticks (the empirical F of
 // Algorithm 1), cumulative input-token mass (Eq. 3) and the quantile knots of F.
 #include "load.cuh"
 
@@ -17,11 +17,10 @@ __global__ void k_ingest(uint32_t n, const int32_t* __restrict__ prompt, const i
                          const uint8_t* __restrict__ dp, uint32_t ns, uint32_t nd, uint64_t* __restrict__ keys,
                          uint32_t* __restrict__ cnt, unsigned long long* __restrict__ grp_sum_n,
                          uint32_t* __restrict__ grp_n, uint32_t* __restrict__ max_n, int32_t* __restrict__ err,
-                         int32_t* __restrict__ S_out, uint16_t* __restrict__ l_out, uint16_t* __restrict__ n_out,
-                         uint32_t* __restrict__ orig_out, uint32_t* __restrict__ counts0, uint32_t per_block0,
+                         uint16_t* __restrict__ l_out, uint16_t* __restrict__ n_out,
+                         uint32_t* __restrict__ counts0, uint32_t per_block0,
                          uint32_t blocks0, int hist_groups) {
-    // S_out, orig_out: single-group traces keep the caller's order, so the internal arrays are written here (l_out,
-    // n_out are then the internal arrays too; otherwise packed copies in the caller's order for the gather);
+    // l_out, n_out: packed copies of the lengths in the caller's order, for the scatter into the internal order;
     // counts0: first radix digit counted per sort block (small traces; large ones use the histogram kernel)
     __shared__ unsigned long long s_sum[kMaxGroups];
     __shared__ uint32_t s_cnt[kMaxGroups];
@@ -58,7 +57,6 @@ __global__ void k_ingest(uint32_t n, const int32_t* __restrict__ prompt, const i
         if (ok && DBG_OK(g, G, DBG_K_INGEST, DBG_GROUP) && DBG_OK(l, kMaxPrompt + 1, DBG_K_INGEST, DBG_TABLE)) {
             keys[i] = ((uint64_t)g << 32) | (uint32_t)S;
             if (hist_groups) atomicAdd(&s_len[g * (kMaxPrompt + 1) + l], 1u); else atomicAdd(&cnt[g * (kMaxPrompt + 1) + l], 1u);
-            if (S_out) { S_out[i] = (int32_t)S; orig_out[i] = i; }
             l_out[i] = (uint16_t)l; n_out[i] = (uint16_t)o;
             if (counts0 && DBG_OK(i / per_block0, blocks0, DBG_K_INGEST, DBG_COUNTER))
                 atomicAdd(&counts0[((uint32_t)S & 255u) * blocks0 + i / per_block0], 1u);
@@ -255,17 +253,54 @@ __global__ void k_radix_scatter(const uint64_t* __restrict__ keys_in, uint64_t* 
     }
 }
 
-__global__ void k_gather(uint32_t n, const uint32_t* __restrict__ orig_in, const uint64_t* __restrict__ keys,
-                         const uint16_t* __restrict__ prompt, const uint16_t* __restrict__ outlen,
-                         int32_t* __restrict__ S, uint16_t* __restrict__ l, uint16_t* __restrict__ nout,
-                         uint32_t* __restrict__ orig) {
-    for (uint32_t k = blockIdx.x * blockDim.x + threadIdx.x; k < n; k += gridDim.x * blockDim.x) {
-        const uint32_t i = orig_in ? orig_in[k] : k;
-        if (!DBG_OK(i, n, DBG_K_GATHER, DBG_REQUEST)) continue;
-        S[k] = (int32_t)(uint32_t)keys[i];
-        l[k] = prompt[i];
-        nout[k] = outlen[i];
-        orig[k] = i;
+// Where the requests of each (group, prompt length) start in the internal order: the groups one after another,
+// inside a group the prompt lengths ascending.  One block of 1024 threads per group.
+__global__ void __launch_bounds__(1024)
+k_length_cursors(const uint32_t* __restrict__ cnt, const uint32_t* __restrict__ ng, uint32_t* __restrict__ cursor) {
+    constexpr int NT = 1024, L = kMaxPrompt + 1;
+    __shared__ uint32_t wc[32];
+    const int g = blockIdx.x;
+    uint32_t base = 0;
+    for (int h = 0; h < g; ++h) base += ng[h];
+    const int per = (L + NT - 1) / NT;
+    const int lo = min(L, (int)threadIdx.x * per), hi = min(L, lo + per);
+    uint32_t k = 0;
+    for (int l = lo; l < hi; ++l) k += cnt[(size_t)g * L + l];
+    uint32_t run = base + block_inclusive_scan(k, wc, (uint32_t*)nullptr) - k;
+    for (int l = lo; l < hi; ++l) { cursor[(size_t)g * L + l] = run; run += cnt[(size_t)g * L + l]; }
+}
+
+// The internal request order: each request takes the next free place of its (group, prompt length).  Requests of
+// one group and length keep no particular order among themselves (nothing downstream depends on it: orig and inv
+// map between the two orders).  The lanes of a warp that share a bucket take their places with one add.
+__global__ void k_scatter_by_length(uint32_t n, int G, const uint64_t* __restrict__ keys,
+                                    const uint16_t* __restrict__ prompt, const uint16_t* __restrict__ outlen,
+                                    const int32_t* __restrict__ err, uint32_t* __restrict__ cursor,
+                                    int32_t* __restrict__ S, uint16_t* __restrict__ l, uint16_t* __restrict__ nout,
+                                    uint32_t* __restrict__ orig, uint32_t* __restrict__ inv) {
+    if (err[0] != 0) return;                          // a rejected trace: its lengths were not all written
+    const int lane = threadIdx.x & 31;
+    const uint32_t stride = gridDim.x * blockDim.x;
+    for (uint32_t i0 = blockIdx.x * blockDim.x; i0 < n; i0 += stride) {       // whole warps iterate together
+        const uint32_t i = i0 + threadIdx.x;
+        bool in = i < n;
+        const uint64_t key = in ? keys[i] : 0ull;
+        const uint32_t g = (uint32_t)(key >> 32), len = in ? prompt[i] : 0u;
+        in = in && DBG_OK(g, G, DBG_K_GATHER, DBG_GROUP) && DBG_OK(len, kMaxPrompt + 1, DBG_K_GATHER, DBG_TABLE);
+        const uint32_t live = __ballot_sync(0xFFFFFFFFu, in);
+        if (!in) continue;
+        const uint32_t bucket = g * (uint32_t)(kMaxPrompt + 1) + len;
+        const uint32_t peers = __match_any_sync(live, bucket);
+        const int leader = __ffs(peers) - 1;
+        uint32_t at = 0;
+        if (lane == leader) at = atomicAdd(&cursor[bucket], (uint32_t)__popc(peers));
+        at = __shfl_sync(peers, at, leader) + (uint32_t)__popc(peers & ((1u << lane) - 1u));
+        if (!DBG_OK(at, n, DBG_K_GATHER, DBG_REQUEST)) continue;
+        S[at] = (int32_t)(uint32_t)key;
+        l[at] = (uint16_t)len;
+        nout[at] = outlen[i];
+        orig[at] = i;
+        inv[i] = at;
     }
 }
 
@@ -380,9 +415,10 @@ DBG_TRANSLATION_UNIT()
 
 uint32_t load_kernel_launches(uint32_t n, int G) {
     if (n == 0) return 1;
-    if (G == 1 && n <= (1u << 20)) return 1 + 2 * 4 + 2 + 1;  // ingest, (row scan, scatter) x 4, two histograms, group tables
-    const uint32_t passes = G > 1 ? 6 : 4;                  // radix passes: partition + 5, or 4
-    return 1 + (G > 1 ? 1 : 0) + 3 * passes + 1 + 1;         // ingest, gather, passes, low words, group tables
+    // ingest, cursors, scatter by length; (row scan, scatter) x 4, two histograms; group tables
+    if (G == 1 && n <= (1u << 20)) return 3 + 2 * 4 + 2 + 1;
+    const uint32_t passes = G > 1 ? 5 : 4;                  // radix passes over (group, ticks)
+    return 3 + 3 * passes + 1 + 1;                          // ..., passes, low words, group tables
 }
 
 cudaError_t run_load(const LoadArgs& a, cudaStream_t st) {
@@ -409,13 +445,11 @@ cudaError_t run_load(const LoadArgs& a, cudaStream_t st) {
         k_ingest<<<std::min(grid_for(n, 4 * kIngestThreads, a.sms), 2 * a.sms), kIngestThreads, hist_bytes, st>>>(
             n, a.prompt, a.outlen, a.ttft, a.sp, a.dp, a.ns, a.nd, a.keys_a, a.cnt,
             (unsigned long long*)a.grp_sum_n, a.ng, a.max_n, a.err,
-            G == 1 ? a.S : nullptr, G == 1 ? a.l : a.l_tmp, G == 1 ? a.nout : a.n_tmp, a.orig,
-            small ? counts_a : nullptr, per_block, blocks, hist_groups);
-        if (G > 1) {
-            // internal request order: stable partition by group
-            if ((e = radix_pass(a.keys_a, a.keys_b, nullptr, a.tmp_idx, n, 32, counts_b, st))) return e;
-            k_gather<<<grid_for(n, 256, a.sms), 256, 0, st>>>(n, a.tmp_idx, a.keys_a, a.l_tmp, a.n_tmp, a.S, a.l, a.nout, a.orig);
-        }
+            a.l_tmp, a.n_tmp, small ? counts_a : nullptr, per_block, blocks, hist_groups);
+        // internal request order: by group, then by prompt length
+        k_length_cursors<<<G, 1024, 0, st>>>(a.cnt, a.ng, a.cursors);
+        k_scatter_by_length<<<grid_for(n, 256, a.sms), 256, 0, st>>>(n, G, a.keys_a, a.l_tmp, a.n_tmp, a.err, a.cursors,
+                                                                     a.S, a.l, a.nout, a.orig, a.inv);
         // sort (group, ticks): four byte passes over the ticks, one over the group id
         uint64_t *src = a.keys_a, *dst = a.keys_b;
         const int passes = G > 1 ? 5 : 4;

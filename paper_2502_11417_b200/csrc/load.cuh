@@ -24,14 +24,15 @@ struct LoadArgs {
     const uint8_t *sp, *dp;               // may be null
     // scratch
     uint64_t *keys_a, *keys_b;            // [n] (group << 32 | ticks)
-    uint32_t* tmp_idx;                    // [n]
-    uint16_t *l_tmp, *n_tmp;              // [n] each: lengths in the caller's order (traces with several groups)
+    uint16_t *l_tmp, *n_tmp;              // [n] each: lengths in the caller's order
+    uint32_t* cursors;                    // [G][4097]: next free place of each (group, prompt length)
     uint32_t* radix_counts;               // [5][256 * kRadixMaxBlocks], directly after zero_block's tables
     void* zero_block; size_t zero_bytes;  // cnt, grp_sum_n, ng, max_n, err, contiguous
     uint32_t* ng_exact;                   // [G] group sizes recounted from the length histogram
     LoadReadback* readback;               // device copy of what the host reads back
     // outputs
-    int32_t* S; uint16_t *l, *nout; uint32_t* orig;   // internal (group-partitioned) order, [n]
+    int32_t* S; uint16_t *l, *nout; uint32_t* orig;   // internal order (by group, then by prompt length), [n]
+    uint32_t* inv;                        // [n]: place of each of the caller's requests in the internal order
     int32_t* sorted;                      // [n] ticks ascending within each group
     uint32_t* cnt;                        // [G][4097] requests per prompt length
     int64_t* cum_mass;                    // [G][4098]

@@ -117,7 +117,7 @@ k_pairs_acc(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* _
     const Prep pr = prep[(size_t)g * P + p];
     const int pols_here = (int)min((uint32_t)PL, n_list - tile * PL);
     // a tile that went through the zone kernel: only the requests it flagged are left (block-uniform)
-    const bool flagged_only = left_mask != nullptr && tile_by_zones(pr, act, lane, pols_here);
+    const bool flagged_only = left_mask != nullptr && left_count[(size_t)chunk_id * n_tiles + tile] != kNotByZones;
     if (flagged_only && left_count[(size_t)chunk_id * n_tiles + tile] == 0u) return;
     const uint32_t mask_words = left_words_per_request(n_tiles), mask_bit = 1u << (tile & 31u);
     const GroupConst& gc = gcs[g];
@@ -516,8 +516,14 @@ k_pairs_rows(TraceDev tr, const GroupConst* __restrict__ gcs, const Prep* __rest
         s_rp[threadIdx.x] = row_pol(pr, gcs[g_lo].candidate, p);
     }
     __syncthreads();
-    const uint32_t k = k_lo + threadIdx.x;
+    uint32_t k = k_lo + threadIdx.x;
     if (k >= tr.n) return;
+    // one group: a thread per request in the caller's order, so that the rows are written side by side (the reads
+    // are scattered instead, once per request); several groups: the block's policies depend on the group, a thread
+    // per request in the internal order
+    uint32_t orig = k;
+    if (tr.n_groups == 1) k = tr.inv[k]; else orig = tr.orig[k];
+    if (!DBG_OK(k, tr.n, DBG_K_PAIRS_ROWS, DBG_REQUEST)) return;
     int g = g_lo;
     while (g < g_hi && k >= tr.grp_off[g + 1]) ++g;
     const GroupConst& gc = gcs[g];
@@ -530,7 +536,6 @@ k_pairs_rows(TraceDev tr, const GroupConst* __restrict__ gcs, const Prep* __rest
     q.l = tr.l[k]; q.n = tr.nout[k]; q.S = (uint32_t)tr.S[k]; q.m = rec.m[k];
     q.saving = delta_c * (float)(q.n - q.m);
     q.delta_c = delta_c;
-    const uint32_t orig = tr.orig[k];
     q.u = EXT ? routing_draw(k0, orig) : 0u;
     const uint32_t Td = (uint32_t)gc.kappa * q.l + (uint32_t)gc.c0, dly = rec.delayed[k];
     const float saving_m = q.m ? q.saving : -1.0f;        // a request migrates only if its buffer filled (m != 0)
@@ -607,7 +612,7 @@ cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassCo
                          const uint32_t* pol_list, uint32_t n_list, const Chunk* chunks, uint32_t n_chunks,
                          TimelineRec rec, disco_pair_out_t out, uint64_t* acc, uint64_t* hist_ttft,
                          uint64_t* hist_tbt, uint32_t* left_mask, uint32_t* left_count, uint32_t* left_lists,
-                         uint64_t* work, uint32_t k0,
+                         uint32_t zone_blocks, uint64_t* work, uint32_t k0,
                          bool extras, bool wide, cudaEvent_t mid, cudaStream_t st) {
     if (n_chunks == 0 || n_list == 0) return mid ? cudaEventRecord(mid, st) : cudaSuccess;
     int PL = 1;
@@ -625,7 +630,7 @@ cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassCo
         const size_t mask_bytes = (size_t)tr.n * left_words_per_request(n_tiles) * 4;
         if ((e = cudaMemsetAsync(left_mask, 0, mask_bytes, st))) return e;
         if ((e = launch_pairs_zones(tr, gc, cc, prep, P, pol_list, n_list, PL, chunks, n_chunks, rec, acc, hist_ttft,
-                                    hist_tbt, left_mask, left_count, left_lists, work, st)))
+                                    hist_tbt, left_mask, left_count, left_lists, zone_blocks, work, st)))
             return e;
     }
     if ((e = launch_after(acc_kernel, dim3(n_chunks * n_tiles), kAccThreads, acc_smem_bytes(PL), st, tr, gc, cc, prep, P,

@@ -1,6 +1,6 @@
 // What the two reduction kernels over (request, policy) pairs share: the six outcomes of a pair, the 16-bit
-// block-private histogram counters, and the test that tells whether a tile of policies can be evaluated zone by
-// zone (zones.cu) or must be evaluated pair by pair (pairs.cu).
+// block-private histogram counters, and how the zone-by-zone kernel (zones.cu) tells the pair-by-pair kernel
+// (pairs.cu) what it left over.
 #pragma once
 
 #include "disco_internal.cuh"
@@ -36,26 +36,13 @@ __device__ __forceinline__ void hist16_add_ticks(uint32_t* row, uint32_t t) {
 __device__ __forceinline__ int32_t packed_lo(uint32_t w) { return (int32_t)(int16_t)(w & 0xFFFFu); }
 __device__ __forceinline__ int32_t packed_hi(uint32_t w) { return (int32_t)(w - (uint32_t)packed_lo(w)) >> 16; }
 
-// The policies of a tile, one per lane (lane % PL; with PL < 32 the lanes repeat them), seen by all 32 lanes.
-// A tile is evaluated zone by zone when its policies are plain Algorithm 2 or plain Algorithm 3 policies of one
-// kind (no random routing, no Eq. 1-2 wait rule, one expected length for Eq. 4) and their length thresholds are
-// ordered along the tile -- Algorithm 3's l_th not increasing, Algorithm 2's l* not decreasing, as they are along
-// an ascending budget axis.  Then the policies under which a request is dispatched alike are neighbours.
-__device__ __forceinline__ bool tile_by_zones(const Prep& pr, bool act, int lane, int npol) {
-    const uint32_t E0 = __shfl_sync(0xFFFFFFFFu, pr.expected_len, 0);
-    const int dc0 = __shfl_sync(0xFFFFFFFFu, pr.device_constrained, 0);
-    bool ok = !act || (!pr.stochastic && !pr.beta_rule && pr.expected_len == E0 && pr.device_constrained == dc0);
-    const int32_t key = dc0 ? pr.l_star : pr.l_th;
-    const int32_t next = __shfl_down_sync(0xFFFFFFFFu, key, 1);
-    if (lane + 1 < npol) ok = ok && (dc0 ? key <= next : key >= next);
-    return __all_sync(0xFFFFFFFFu, ok) != 0;
-}
-
 // Requests a zone-by-zone kernel could not settle for a tile are flagged in a bit mask: word
 // request * words_per_request + tile / 32, bit tile % 32.
 __host__ __device__ __forceinline__ uint32_t left_words_per_request(uint32_t n_tiles) { return (n_tiles + 31u) / 32u; }
 // The first kLeftList of them per (chunk, tile) are also listed by chunk position, so that the pair kernel need not
 // scan the flags of a chunk for a handful of requests.
 constexpr uint32_t kLeftList = 2048;
+// The count of a (chunk, tile) whose policies the zone-by-zone kernel could not take at all.
+constexpr uint32_t kNotByZones = 0xFFFFFFFFu;
 
 }  // namespace disco
