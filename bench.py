@@ -51,14 +51,13 @@ PAIR_INSTR_NOWAIT = 21
 # outcome index 3, row address 1, two row loads 2, sums 8, histogram increment from the float bits (convert,
 # small-value test and branch, offset 2, increment 3, address, atomic) 10, stall test 1.
 PAIR_INSTR_WAIT = 37
-# Lane-instructions the zone-by-zone reduction needs per request and policy tile: request loads 6, device TTFT 1,
-# run boundaries from the length tables 2, projected saving 4, race at wait 0 (two compares, select, minimum) 4,
-# trigger against the tile's range 3, outcome select 2, the outcome's addends 14, eight sums 9, histogram bin and
-# increment 6, loop 1.  A request with a run below the boundary (or policies whose l* is its length) also enters a
-# correction: reload 6, the run's outcome 8, addends of both outcomes 28, nine differences and their adds 18, two
-# histogram increments 12.
-ZONE_INSTR_PER_REQUEST_TILE = 52
-ZONE_INSTR_PER_CORRECTION = 72
+# Lane-instructions the zone-by-zone reduction needs per request and policy FAMILY (up to 128 policies along a
+# budget axis, whatever their number): request loads 6, device TTFT 1, projected saving 4, race at wait 0 (two
+# compares, select, minimum) 4, trigger against the family's range 3, outcome select 2, the common outcome's
+# addends 14, its ten sums 11, histogram bin and increment 6; the first run's outcome 8, its addends 14, ten
+# differences to the common outcome 20, histogram bin and increment 6; loop 1.  The extra sweeps over requests
+# whose prompt length is some policy's l* are not counted.
+ZONE_INSTR_PER_REQUEST_FAMILY = 100
 SCHEDULERS, LANES = 4, 32    # warp schedulers per multiprocessor, lanes per warp
 MIN_WARMUP_SECONDS = 0.5     # untimed steps run until this much device time has passed (and at least --warmup)
 MAX_WARMUP_STEPS = 200
@@ -67,7 +66,7 @@ MAX_WARMUP_STEPS = 200
 # for the current kernel.
 NCU_TRAFFIC_BYTES = {("k_pairs_rows", 1): 149923840, ("k_playout_fast", 1): 827904}
 # issued lane-slots per token-step (play-out; the workload-3 figure is of a 200,000-request capture of its shape) and
-# per request and policy tile (zone kernel, workload 2 at full size)
+# per request and policy family (zone kernel, workload 2 at full size)
 NCU_EXECUTED_PER_UNIT = {("k_playout_fast", 1): 31.9, ("k_playout_fast", 3): 21.8, ("k_pairs_zones+k_pairs_acc", 2): 222.0}
 HEADLINE_CONFIG = 4
 ALL_CONFIGS = (0, 1, 2, 3, 4, 5)
@@ -491,22 +490,21 @@ class Bench:
                         "peak_source": src, "algorithmic_bytes": bytes_alg, "ms_per_launch": ms}
             if name == "k_pairs_acc":
                 # the two reduction kernels together (their events bracket both): requests settled zone by zone per
-                # policy tile, corrections among them, and the pairs left to the pair-by-pair kernel, by kind (a
-                # (group, policy) waits when Algorithm 1 made the group device-constrained)
-                zone_pairs, left_pairs, settled, corrections = tr.work_counts()
+                # policy family, and the pairs left to the pair-by-pair kernel, by kind (a (group, policy) waits
+                # when Algorithm 1 made the group device-constrained)
+                zone_pairs, left_pairs, settled, sweeps = tr.work_counts()
                 wait_pairs = 0
                 for g in range(tr.n_groups):
                     n_g = tr.group_size(g)
                     wait_pairs += n_g * sum(1 for p in range(P) if tr.prep(g, p).device_constrained)
                 wait_share = wait_pairs / float(max(n * P, 1))
                 per_left_pair = wait_share * PAIR_INSTR_WAIT + (1.0 - wait_share) * PAIR_INSTR_NOWAIT
-                lane_instr = (settled * ZONE_INSTR_PER_REQUEST_TILE + corrections * ZONE_INSTR_PER_CORRECTION +
-                              left_pairs * per_left_pair)
+                lane_instr = settled * ZONE_INSTR_PER_REQUEST_FAMILY + left_pairs * per_left_pair
                 return alu_roof("k_pairs_zones+k_pairs_acc", lane_instr, ms,
                                 work={"pairs_by_zones": zone_pairs, "pairs_one_by_one": left_pairs,
-                                      "requests_settled_per_tile": settled, "corrections": corrections},
-                                instr={"per_request_tile": ZONE_INSTR_PER_REQUEST_TILE,
-                                       "per_correction": ZONE_INSTR_PER_CORRECTION, "per_pair_one_by_one": per_left_pair},
+                                      "requests_settled_per_family": settled, "segment_sweeps": sweeps},
+                                instr={"per_request_family": ZONE_INSTR_PER_REQUEST_FAMILY,
+                                       "per_pair_one_by_one": per_left_pair},
                                 instr_per_pair_mean=lane_instr / float(max(n * P, 1)))
             if name == "k_playout_fast":
                 return alu_roof(name, token_steps * per_token * n_classes, ms, token_steps=token_steps * n_classes,

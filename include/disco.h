@@ -240,9 +240,9 @@ int disco_get_timing(disco_ctx_t* ctx, float* ms4);
 uint64_t disco_kernel_launch_count(void);
 
 /* How the last evaluation's pairs were reduced (host counts4[4]): pairs settled zone by zone (a request against
- * the runs of neighbouring policies of a 32-policy tile that dispatch it alike); pairs evaluated one by one;
- * requests settled zone by zone, counted once per tile; those of them that needed corrections below a run
- * boundary.  The first two add up to requests x policies.  Synchronises `stream`. */
+ * the runs of neighbouring policies of a family of up to 128 policies that dispatch it alike); pairs evaluated
+ * one by one; requests settled zone by zone, counted once per policy family; sweeps the zone kernel's blocks made
+ * over segments of their request chunks.  The first two add up to requests x policies.  Synchronises `stream`. */
 int disco_get_work_counts(disco_ctx_t* ctx, uint64_t* counts4, void* stream);
 
 /* Checked build.  Compiled with -DDISCO_DEBUG the library checks every index its kernels derive (request, policy,

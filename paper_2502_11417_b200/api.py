@@ -443,8 +443,8 @@ class Trace:
         return tuple(ms)
 
     def work_counts(self, stream=None):
-        """(pairs settled zone by zone, pairs evaluated one by one, requests settled per tile, those with
-        corrections) of the last evaluation."""
+        """(pairs settled zone by zone, pairs evaluated one by one, requests settled per policy family, sweeps
+        over chunk segments) of the last evaluation."""
         w = (C.c_uint64 * 4)()
         _check(lib().disco_get_work_counts(self._h, w, _stream_ptr(stream)))
         return tuple(int(x) for x in w)

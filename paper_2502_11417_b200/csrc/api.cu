@@ -98,7 +98,7 @@ struct disco_ctx {
     const void* gc_dev_at = nullptr;
     // trace
     DevBuf in_prompt, in_out, in_ttft, in_sp, in_dp;      // staging of host inputs
-    DevBuf keys_a, keys_b, tmp_idx, tmp_ln, cursors, inv;
+    DevBuf keys_a, keys_b, tmp_idx, tmp_ln, cursors, inv, placed;
     DevBuf S, l, nout, orig, sorted;
     DevBuf zero, cum_mass, ng_exact, grp_off, knots, d_gc;   // `zero`: every table a load must clear, contiguous
     DevBuf fin_totals;                 // [2G] u64: output tokens and requests per group that the accumulators cover
@@ -138,7 +138,7 @@ struct disco_ctx {
     bool timing_valid = false;
 
     ~disco_ctx() {
-        DevBuf* all[] = {&in_prompt, &in_out, &in_ttft, &in_sp, &in_dp, &keys_a, &keys_b, &tmp_idx, &tmp_ln, &cursors, &inv,
+        DevBuf* all[] = {&in_prompt, &in_out, &in_ttft, &in_sp, &in_dp, &keys_a, &keys_b, &tmp_idx, &tmp_ln, &cursors, &inv, &placed,
                          &S, &l, &nout, &orig, &sorted, &zero, &cum_mass, &ng_exact, &grp_off, &knots, &d_gc, &d_prep, &d_accum, &d_stats, &d_tables, &d_todo,
                          &fin_totals, &F_sorted_imp, &F_off_imp, &d_left};
         for (DevBuf* b : all) b->release();
@@ -206,7 +206,7 @@ cudaError_t reserve_trace(disco_ctx* c, uint32_t n, bool host_inputs, bool has_s
         if (has_dp) R(in_dp, N);
     }
     R(keys_a, N * 8); R(keys_b, N * 8);
-    R(tmp_ln, N * 4); R(cursors, (size_t)G * (kMaxPrompt + 1) * 4); R(inv, N * 4);
+    R(tmp_ln, N * 4); R(cursors, (size_t)G * (kMaxPrompt + 1) * 4); R(inv, N * 4); R(placed, N * 16);
     R(S, N * 4); R(l, N * 2); R(nout, N * 2); R(orig, N * 4); R(sorted, N * 4);
     // one block for everything a load clears: cnt | grp_sum_n | ng | max_n | err | first radix counter buffer,
     // followed by the second counter buffer
@@ -311,7 +311,7 @@ int disco_load_trace(disco_ctx_t** pctx, const disco_trace_desc_t* d, void* stre
         a.prompt = d->prompt_len; a.outlen = d->output_len; a.ttft = d->server_ttft_s;
         a.sp = d->server_profile; a.dp = d->device_profile;
     }
-    a.keys_a = c->keys_a.as<uint64_t>(); a.keys_b = c->keys_b.as<uint64_t>(); a.cursors = c->cursors.as<uint32_t>(); a.inv = c->inv.as<uint32_t>();
+    a.keys_a = c->keys_a.as<uint64_t>(); a.keys_b = c->keys_b.as<uint64_t>(); a.cursors = c->cursors.as<uint32_t>(); a.inv = c->inv.as<uint32_t>(); a.placed = c->placed.as<uint4>();
     a.l_tmp = c->tmp_ln.as<uint16_t>(); a.n_tmp = c->tmp_ln.as<uint16_t>() + (n ? n : 1);
     a.radix_counts = c->radix_counts; a.zero_block = c->zero.p; a.zero_bytes = c->zero_bytes;
     a.ng_exact = c->ng_exact.as<uint32_t>(); a.readback = c->rb;     // pinned host memory, written by the last kernel
@@ -438,8 +438,10 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
 #define R(buf, bytes) if ((e = c->buf.reserve(bytes)) != cudaSuccess) return fail_cuda(e, "device allocation for the evaluation")
     R(d_prep, (size_t)G * P * sizeof(Prep));
     const size_t acc_bytes = (size_t)P * G * kNAcc * 8, hist_bytes = (size_t)P * kNBins * 8;
-    // a to-do counter and a ticket counter per class, then the work counters of the pair kernel (four words)
-    const size_t cls_cnt_bytes = (classes.size() * 8 + 15) / 16 * 16, cnt_bytes = cls_cnt_bytes + 32;
+    // a to-do counter and a ticket counter per class, the work counters of the pair kernels (four words), and a
+    // ticket counter per class for the zone kernel
+    const size_t cls_cnt_bytes = (classes.size() * 8 + 15) / 16 * 16;
+    const size_t cnt_bytes = cls_cnt_bytes + 32 + (classes.size() * 4 + 15) / 16 * 16;
     R(d_accum, acc_bytes + 2 * hist_bytes + cnt_bytes);
     R(d_todo, N1 * 4);
     c->d_acc.p = c->d_accum.p; c->d_hist_ttft.p = (char*)c->d_accum.p + acc_bytes;
@@ -599,7 +601,7 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
                         c->d_hist_ttft.as<uint64_t>(), c->d_hist_tbt.as<uint64_t>(), c->d_left.as<uint32_t>(),
                         c->d_left.as<uint32_t>() + left_mask_words,
                         left_list_words ? c->d_left.as<uint32_t>() + left_mask_words + left_cells : nullptr,
-                        sms, c->d_work.as<uint64_t>(), k0, cls_extras_pending,
+                        sms, (uint32_t*)(c->d_work.as<uint64_t>() + 4) + k, c->d_work.as<uint64_t>(), k0, cls_extras_pending,
                         !classes[k].pacing || classes[k].W[0] > 1 || classes[k].W[1] > 1 || classes[k].W[2] > 1,
                         timed ? c->ev[3] : nullptr, st));
         if (timed) CU(cudaEventRecord(c->ev[4], st));

@@ -214,6 +214,7 @@ cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassCo
                          uint32_t* left_count /* [n_chunks][tiles] scratch */,
                          uint32_t* left_lists /* [n_chunks][tiles][kLeftList] scratch, or null */,
                          uint32_t zone_blocks /* blocks the zone kernel may run: one per multiprocessor */,
+                         uint32_t* zone_ticket /* one word, zero: the zone kernel's blocks draw their work from it */,
                          uint64_t* work /* [4], added to: pairs settled zone by zone, pairs evaluated one by one,
                          requests settled per policy family, sweeps over segments of a chunk */,
                          uint32_t k0, bool extras /* some policy routes at random or uses an
@@ -224,7 +225,7 @@ cudaError_t launch_pairs_zones(const TraceDev& tr, const GroupConst* gc, const C
                                uint32_t P, const uint32_t* pol_list, uint32_t n_list, int PL, const Chunk* chunks,
                                uint32_t n_chunks, TimelineRec rec, uint64_t* acc, uint64_t* hist_ttft,
                                uint64_t* hist_tbt, uint32_t* left_mask, uint32_t* left_count, uint32_t* left_lists,
-                               uint32_t max_blocks, uint64_t* work, cudaStream_t st);
+                               uint32_t max_blocks, uint32_t* ticket, uint64_t* work, cudaStream_t st);
 cudaError_t launch_finalize(uint32_t P, int G, const GroupConst* gc, const uint64_t* acc, const uint64_t* hist_ttft,
                             const uint64_t* hist_tbt,
                             const uint64_t* fin_totals /* [2G]: output tokens per group, then requests per group */,

@@ -272,12 +272,13 @@ k_length_cursors(const uint32_t* __restrict__ cnt, const uint32_t* __restrict__ 
 
 // The internal request order: each request takes the next free place of its (group, prompt length).  Requests of
 // one group and length keep no particular order among themselves (nothing downstream depends on it: orig and inv
-// map between the two orders).  The lanes of a warp that share a bucket take their places with one add.
+// map between the two orders).  The lanes of a warp that share a bucket take their places with one add.  A
+// request goes to its place as one 16-byte record (ticks, lengths, caller's index): one scattered store instead
+// of four; k_unpack_requests then writes the arrays side by side.
 __global__ void k_scatter_by_length(uint32_t n, int G, const uint64_t* __restrict__ keys,
                                     const uint16_t* __restrict__ prompt, const uint16_t* __restrict__ outlen,
                                     const int32_t* __restrict__ err, uint32_t* __restrict__ cursor,
-                                    int32_t* __restrict__ S, uint16_t* __restrict__ l, uint16_t* __restrict__ nout,
-                                    uint32_t* __restrict__ orig, uint32_t* __restrict__ inv) {
+                                    uint4* __restrict__ placed, uint32_t* __restrict__ inv) {
     if (err[0] != 0) return;                          // a rejected trace: its lengths were not all written
     const int lane = threadIdx.x & 31;
     const uint32_t stride = gridDim.x * blockDim.x;
@@ -296,11 +297,21 @@ __global__ void k_scatter_by_length(uint32_t n, int G, const uint64_t* __restric
         if (lane == leader) at = atomicAdd(&cursor[bucket], (uint32_t)__popc(peers));
         at = __shfl_sync(peers, at, leader) + (uint32_t)__popc(peers & ((1u << lane) - 1u));
         if (!DBG_OK(at, n, DBG_K_GATHER, DBG_REQUEST)) continue;
-        S[at] = (int32_t)(uint32_t)key;
-        l[at] = (uint16_t)len;
-        nout[at] = outlen[i];
-        orig[at] = i;
+        placed[at] = make_uint4((uint32_t)key, len | ((uint32_t)outlen[i] << 16), i, 0u);
         inv[i] = at;
+    }
+}
+
+__global__ void k_unpack_requests(uint32_t n, const uint4* __restrict__ placed, const int32_t* __restrict__ err,
+                                  int32_t* __restrict__ S, uint16_t* __restrict__ l, uint16_t* __restrict__ nout,
+                                  uint32_t* __restrict__ orig) {
+    if (err[0] != 0) return;
+    for (uint32_t k = blockIdx.x * blockDim.x + threadIdx.x; k < n; k += gridDim.x * blockDim.x) {
+        const uint4 r = placed[k];
+        S[k] = (int32_t)r.x;
+        l[k] = (uint16_t)(r.y & 0xFFFFu);
+        nout[k] = (uint16_t)(r.y >> 16);
+        orig[k] = r.z;
     }
 }
 
@@ -415,10 +426,10 @@ DBG_TRANSLATION_UNIT()
 
 uint32_t load_kernel_launches(uint32_t n, int G) {
     if (n == 0) return 1;
-    // ingest, cursors, scatter by length; (row scan, scatter) x 4, two histograms; group tables
-    if (G == 1 && n <= (1u << 20)) return 3 + 2 * 4 + 2 + 1;
+    // ingest, cursors, scatter by length, unpack; (row scan, scatter) x 4, two histograms; group tables
+    if (G == 1 && n <= (1u << 20)) return 4 + 2 * 4 + 2 + 1;
     const uint32_t passes = G > 1 ? 5 : 4;                  // radix passes over (group, ticks)
-    return 3 + 3 * passes + 1 + 1;                          // ..., passes, low words, group tables
+    return 4 + 3 * passes + 1 + 1;                          // ..., passes, low words, group tables
 }
 
 cudaError_t run_load(const LoadArgs& a, cudaStream_t st) {
@@ -449,7 +460,8 @@ cudaError_t run_load(const LoadArgs& a, cudaStream_t st) {
         // internal request order: by group, then by prompt length
         k_length_cursors<<<G, 1024, 0, st>>>(a.cnt, a.ng, a.cursors);
         k_scatter_by_length<<<grid_for(n, 256, a.sms), 256, 0, st>>>(n, G, a.keys_a, a.l_tmp, a.n_tmp, a.err, a.cursors,
-                                                                     a.S, a.l, a.nout, a.orig, a.inv);
+                                                                     a.placed, a.inv);
+        k_unpack_requests<<<grid_for(n, 256, a.sms), 256, 0, st>>>(n, a.placed, a.err, a.S, a.l, a.nout, a.orig);
         // sort (group, ticks): four byte passes over the ticks, one over the group id
         uint64_t *src = a.keys_a, *dst = a.keys_b;
         const int passes = G > 1 ? 5 : 4;

@@ -26,6 +26,7 @@ struct LoadArgs {
     uint64_t *keys_a, *keys_b;            // [n] (group << 32 | ticks)
     uint16_t *l_tmp, *n_tmp;              // [n] each: lengths in the caller's order
     uint32_t* cursors;                    // [G][4097]: next free place of each (group, prompt length)
+    uint4* placed;                        // [n]: the requests in the internal order, one record each
     uint32_t* radix_counts;               // [5][256 * kRadixMaxBlocks], directly after zero_block's tables
     void* zero_block; size_t zero_bytes;  // cnt, grp_sum_n, ng, max_n, err, contiguous
     uint32_t* ng_exact;                   // [G] group sizes recounted from the length histogram

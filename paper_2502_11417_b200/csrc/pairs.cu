@@ -612,7 +612,7 @@ cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassCo
                          const uint32_t* pol_list, uint32_t n_list, const Chunk* chunks, uint32_t n_chunks,
                          TimelineRec rec, disco_pair_out_t out, uint64_t* acc, uint64_t* hist_ttft,
                          uint64_t* hist_tbt, uint32_t* left_mask, uint32_t* left_count, uint32_t* left_lists,
-                         uint32_t zone_blocks, uint64_t* work, uint32_t k0,
+                         uint32_t zone_blocks, uint32_t* zone_ticket, uint64_t* work, uint32_t k0,
                          bool extras, bool wide, cudaEvent_t mid, cudaStream_t st) {
     if (n_chunks == 0 || n_list == 0) return mid ? cudaEventRecord(mid, st) : cudaSuccess;
     int PL = 1;
@@ -630,7 +630,7 @@ cudaError_t launch_pairs(const TraceDev& tr, const GroupConst* gc, const ClassCo
         const size_t mask_bytes = (size_t)tr.n * left_words_per_request(n_tiles) * 4;
         if ((e = cudaMemsetAsync(left_mask, 0, mask_bytes, st))) return e;
         if ((e = launch_pairs_zones(tr, gc, cc, prep, P, pol_list, n_list, PL, chunks, n_chunks, rec, acc, hist_ttft,
-                                    hist_tbt, left_mask, left_count, left_lists, zone_blocks, work, st)))
+                                    hist_tbt, left_mask, left_count, left_lists, zone_blocks, zone_ticket, work, st)))
             return e;
     }
     if ((e = launch_after(acc_kernel, dim3(n_chunks * n_tiles), kAccThreads, acc_smem_bytes(PL), st, tr, gc, cc, prep, P,

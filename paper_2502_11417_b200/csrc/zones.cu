@@ -28,17 +28,24 @@ namespace disco {
 
 namespace {
 
-constexpr int kZThreads = 1024;
+#ifndef DISCO_ZONE_THREADS
+#define DISCO_ZONE_THREADS 1024
+#endif
+#ifndef DISCO_ZONE_BLOCKS_PER_SM
+#define DISCO_ZONE_BLOCKS_PER_SM 1
+#endif
+constexpr int kZThreads = DISCO_ZONE_THREADS;
+constexpr int kZBlocksPerSm = DISCO_ZONE_BLOCKS_PER_SM;
 constexpr int kZWarps = kZThreads / 32;
 constexpr int kFamTiles = 4;            // tiles of 32 policies a family may span
 constexpr int kFamPol = 32 * kFamTiles;
 constexpr int kSumRows = kFamPol + 1;   // difference rows of the sums: row q is carried to the policies below q
 constexpr int kCoarseRows = kFamTiles + 1;   // ... of the histograms: row t is carried to every policy of the tiles below t
 constexpr int kMaxSeg = 2 * kFamPol + 2;
+constexpr int kJRows = 33;              // rows a single request may enter a difference at: within the first tile
 enum ZSum { Z_TD = 0, Z_PS, Z_PD, Z_TAU, Z_DL, Z_DO, Z_RACE, Z_DW, Z_MIGR, Z_TT, kZSums };
 constexpr int kLenTab = kMaxPrompt + 8; // bytes per table over the prompt lengths 0 .. 4096
-static_assert(kZThreads >= kNBins + kZSums, "a segment's histograms and sums are entered by one thread per bin or field");
-static_assert(kZThreads >= kMaxSeg && kZWarps >= kZSums, "one thread per candidate segment, one warp per field");
+static_assert(kZWarps >= kZSums, "the sums go out one warp per field");
 
 struct Seg { uint32_t pa, pb; int32_t k1, k2; };       // requests [pa, pb) of the chunk share (k1, k2)
 
@@ -50,7 +57,8 @@ struct ZoneSmem {
     long long e_sum[kSumRows][kZSums];                  // difference rows of the sums
     long long c_sum[kZSums];                            // what every policy gets
     long long part[kZWarps][kZSums];                    // the warps' shares of a segment's difference
-    uint32_t n_left, n_listed, n_seg, n_pass;
+    int32_t j_sum[kJRows][kZSums];                      // differences entered request by request during a sweep, rows 1 .. 32
+    uint32_t n_left, n_apart, n_listed, n_listed0, n_seg, ticket;
     uint32_t red[4];                                    // smallest / largest overhead (float bits), smallest / largest w_tail
     Seg seg[kMaxSeg];
     int32_t key[kFamPol];                               // the policies' length thresholds, in list order
@@ -106,6 +114,7 @@ struct TileCtx {
     int npol, race_that_migrates;
     bool may_migrate;
     bool wt_ordered;                    // the policies' w_tail do not increase along the family
+    bool tile0_apart;                   // more than one tile, and only the first tile's w_tail differ from wt_min
 };
 
 // With every stream delivered at the pace tau the TBTs in tau's bin are all n - 1 intervals (n - 2 beside a
@@ -150,11 +159,16 @@ __device__ __forceinline__ bool tail_outcome(const TileCtx& c, const Req& q, uin
 // The run of Algorithm 2 policies [0, k1) that wait their w_tail.  On success the policies [j, k1) end in
 // (oc, tt) and the policies [0, j), whose longer waits cover the server's TTFT, in O_SERVER_ONLY with the same
 // TTFT (j = 0: none).  Returns false if the run cannot be expressed that way.
+//
+// apart: in a family of several tiles whose first tile alone has waits above wt_min, the device wins under the
+// policies of the other tiles at wt_min + T_d while the first tile's policies each end their own way: the outcome
+// then holds for the tiles after the first, and the request is left to the pair kernel for the first tile only.
 __device__ __forceinline__ bool head_outcome_waits(const TileCtx& c, const ZoneSmem& sm, const Req& q, uint32_t Td,
-                                                   float saving, int k1, int& oc, uint32_t& tt, int& j) {
+                                                   float saving, int k1, int& oc, uint32_t& tt, int& j, bool& apart) {
     int base;
     tt = q.S;
     j = 0;
+    apart = false;
     if (q.S <= c.wt_min) base = O_SERVER_ONLY;                                 // the server answers within every wait
     else if (q.S <= c.wt_min + Td) {                                           // whoever starts the device loses the race
         base = O_RACE_SRV;
@@ -165,8 +179,10 @@ __device__ __forceinline__ bool head_outcome_waits(const TileCtx& c, const ZoneS
             j = lo;
             if (j == k1) { base = O_SERVER_ONLY; j = 0; }                      // every wait of the run covers S
         }
-    } else if (c.wt_min == c.wt_max) { base = O_RACE_DEV; tt = c.wt_min + Td; }   // the device wins under every policy
-    else return false;
+    } else if (c.wt_min == c.wt_max || c.tile0_apart) {                        // the device wins under every policy
+        base = O_RACE_DEV; tt = c.wt_min + Td;                                 // (of the tiles after the first)
+        apart = c.wt_min != c.wt_max;
+    } else return false;
     const int t = trigger_all(c, base, saving);
     oc = base + 2 * t;
     return t >= 0;
@@ -181,9 +197,21 @@ __device__ __forceinline__ void hist_add(uint32_t* hist, bool on, int bin) {
     if ((peers & ((1u << (threadIdx.x & 31)) - 1u)) == 0u) atomicAdd(&hist[bin], (uint32_t)__popc(peers));
 }
 
+// One request's difference into a row of 32-bit sums (the TTFT sum is not entered: the caller sees to it).  A
+// segment's rows are added to the 64-bit ones when the segment is entered; a sum stays below 2^31 over a chunk.
+__device__ __forceinline__ void enter_small(int32_t* row, const Sums& e) {
+#pragma unroll
+    for (int f = 0; f < kZSums; ++f) {
+        if (f == Z_TT) continue;
+        const int v = (int)field_of(e, f);
+        if (v) atomicAdd(&row[f], v);
+    }
+}
+
 // What a request comes to under the policies of its segment.
 struct Verdict {
     bool ok;                            // the runs express it
+    bool apart;                         // ... except for the policies of the family's first tile
     int oc_c, oc_h, j;                  // outcome every policy gets; outcome of the first run [j, k1); covered waits [0, j)
     uint32_t tt_c, tt_h;
 };
@@ -195,14 +223,15 @@ template <bool WAITS>
 __device__ __forceinline__ Verdict judge(const TileCtx& c, const ZoneSmem& sm, const Req& q, uint32_t Td, float saving,
                                          int k1, int k2) {
     Verdict v;
-    v.oc_c = O_DEVICE_ONLY; v.oc_h = O_DEVICE_ONLY; v.j = 0; v.tt_c = Td; v.tt_h = Td; v.ok = true;
+    v.oc_c = O_DEVICE_ONLY; v.oc_h = O_DEVICE_ONLY; v.j = 0; v.tt_c = Td; v.tt_h = Td; v.ok = true; v.apart = false;
     if (k2 < c.npol) {
         v.ok = tail_outcome(c, q, Td, saving, v.oc_c, v.tt_c);
-        if (WAITS && k1 > 0) v.ok = head_outcome_waits(c, sm, q, Td, saving, k1, v.oc_h, v.tt_h, v.j) && v.ok;
+        if (WAITS && k1 > 0) v.ok = head_outcome_waits(c, sm, q, Td, saving, k1, v.oc_h, v.tt_h, v.j, v.apart) && v.ok;
     } else if (WAITS) {
-        v.ok = head_outcome_waits(c, sm, q, Td, saving, k1, v.oc_c, v.tt_c, v.j);
+        v.ok = head_outcome_waits(c, sm, q, Td, saving, k1, v.oc_c, v.tt_c, v.j, v.apart);
         v.oc_h = v.oc_c; v.tt_h = v.tt_c;
     }
+    v.apart = v.apart && v.ok;
     return v;
 }
 
@@ -218,8 +247,8 @@ struct FlushTo {
 // policy gets is returned, its histograms go to h_*.
 template <bool WAITS>
 __device__ __forceinline__ Sums sweep(ZoneSmem& sm, const TileCtx& c, const Seg& s, int point, Sums& every, uint32_t& n_left,
-                                      uint32_t tile0, int n_fam, uint32_t n_tiles, uint32_t* __restrict__ left_mask,
-                                      uint32_t* __restrict__ left_list, const FlushTo& out) {
+                                      uint32_t& n_apart, uint32_t tile0, int n_fam, uint32_t n_tiles,
+                                      uint32_t* __restrict__ left_mask, uint32_t* __restrict__ left_list, const FlushTo& out) {
     const int lane = threadIdx.x & 31;
     const int k1 = s.k1, k2 = s.k2;
     const bool first_run = k2 < c.npol && k1 > 0;                // a first run that differs from what every policy gets
@@ -239,47 +268,65 @@ __device__ __forceinline__ Sums sweep(ZoneSmem& sm, const TileCtx& c, const Seg&
         const float saving = saving_of(c, q);
         const Verdict v = judge<WAITS>(c, sm, q, Td, saving, k1, k2);
         const bool ok = v.ok && valid;
+        const bool apart = v.apart && valid;                     // left to the pair kernel for the first tile alone
         if (point < 0) {
-            if (valid && !ok) {
-                atomicOr(&left_mask[(size_t)(c.ch->start + i) * words + (tile0 >> 5)], left_bits);
-                ++n_left;
+            if (valid && (!ok || apart)) {
+                // left to the pair kernel: for every tile of the family, or for the first one alone
+                atomicOr(&left_mask[(size_t)(c.ch->start + i) * words + (tile0 >> 5)], ok ? 1u << (tile0 & 31u) : left_bits);
+                if (ok) ++n_apart; else ++n_left;
                 if (left_list) {
-                    const uint32_t at = atomicAdd(&sm.n_listed, 1u);
-                    if (at < kLeftList) for (int t = 0; t < n_fam; ++t) left_list[(size_t)t * kLeftList + at] = i;
+                    const uint32_t at0 = atomicAdd(&sm.n_listed0, 1u);
+                    if (at0 < kLeftList) left_list[at0] = i;
+                    if (!ok && n_fam > 1) {
+                        const uint32_t at = atomicAdd(&sm.n_listed, 1u);
+                        if (at < kLeftList) for (int t = 1; t < n_fam; ++t) left_list[(size_t)t * kLeftList + at] = i;
+                    }
                 }
             }
             if (ok) add_outcome(every, 1, v.oc_c, q, v.tt_c);
             hist_add(sm.g_ttft, ok, bin_of_ticks(v.tt_c));
-            hist_add(sm.g_stall, ok && v.oc_c >= O_MIGR_TO_DEV && stall_bin, bin_of_ticks(q.stall));
+            if (c.may_migrate) hist_add(sm.g_stall, ok && v.oc_c >= O_MIGR_TO_DEV && stall_bin, bin_of_ticks(q.stall));
+            // (a request left for the first tile alone, whose first run lies inside that tile: no first run to enter)
+            const bool runs = ok && !(WAITS && apart && k1 < 32);
             if (first_run) {
-                if (ok) { add_outcome(d, 1, v.oc_h, q, v.tt_h); add_outcome(d, -1, v.oc_c, q, v.tt_c); }
-                hist_add(sm.h_ttft, ok, bin_of_ticks(v.tt_h));
-                hist_add(sm.h_stall, ok && v.oc_h >= O_MIGR_TO_DEV && stall_bin, bin_of_ticks(q.stall));
+                if (runs) { add_outcome(d, 1, v.oc_h, q, v.tt_h); add_outcome(d, -1, v.oc_c, q, v.tt_c); }
+                // (h_* minus g_* is entered for the segment: a request without a first run joins both)
+                hist_add(sm.h_ttft, ok, bin_of_ticks(runs ? v.tt_h : v.tt_c));
+                if (c.may_migrate) hist_add(sm.h_stall, ok && (runs ? v.oc_h : v.oc_c) >= O_MIGR_TO_DEV && stall_bin, bin_of_ticks(q.stall));
+            }
+            if (WAITS && c.tile0_apart) {
+                // ---- the first tile gets nothing from the family for such a request (the pair kernel evaluates it there):
+                //      what its policies would get is taken back at row 32, the row carried to the first tile
+                if (__ballot_sync(0xFFFFFFFFu, apart)) {
+                    const bool head = first_run && k1 >= 32;             // they would get the first run's outcome, else the common one
+                    const int oc_x = head ? v.oc_h : v.oc_c;
+                    const uint32_t tt_x = head ? v.tt_h : v.tt_c;
+                    long long tt_back = 0;
+                    if (apart) {
+                        Sums e;
+                        clear(e);
+                        add_outcome(e, -1, oc_x, q, tt_x);
+                        enter_small(sm.j_sum[32], e);
+                        tt_back = e.tt;
+                        if (DBG_OK(bin_of_ticks(tt_x), kNBins, DBG_K_PAIRS_ZONES, DBG_BIN)) atomicSub(&sm.k_ttft[1][bin_of_ticks(tt_x)], 1);
+                        if (oc_x >= O_MIGR_TO_DEV && stall_bin) atomicSub(&sm.k_stall[1][bin_of_ticks(q.stall)], 1);
+                    }
+#pragma unroll
+                    for (int off = 16; off > 0; off >>= 1) tt_back += __shfl_xor_sync(0xFFFFFFFFu, tt_back, off);
+                    if (lane == 0) atomicAdd((unsigned long long*)&sm.e_sum[32][Z_TT], (unsigned long long)tt_back);
+                }
             }
             if (WAITS && c.wt_min != c.wt_max) {
                 // ---- waits that cover the server's TTFT: the policies [0, j) end in O_SERVER_ONLY instead of the first
                 //      run's outcome (a race the server wins, with the same TTFT).  The lanes that share j add up.
-                const bool has_j = ok && v.j > 0;
-                uint32_t rest = __ballot_sync(0xFFFFFFFFu, has_j);
-                if (rest) {
+                const bool has_j = ok && v.j > 0 && DBG_OK(v.j, kJRows, DBG_K_PAIRS_ZONES, DBG_SLOT);
+                if (has_j) {
                     Sums e;
                     clear(e);
-                    if (has_j) { add_outcome(e, 1, O_SERVER_ONLY, q, q.S); add_outcome(e, -1, v.oc_h, q, v.tt_h); }
-                    while (rest) {
-                        const int first = __ffs(rest) - 1;
-                        const int jj = __shfl_sync(0xFFFFFFFFu, v.j, first);
-                        const bool mine = has_j && v.j == jj;
-                        rest &= ~__ballot_sync(0xFFFFFFFFu, mine);
-                        if (!DBG_OK(jj, kSumRows, DBG_K_PAIRS_ZONES, DBG_SLOT)) continue;
-#pragma unroll
-                        for (int f = 0; f < kZSums; ++f) {
-                            const long long mv = mine ? field_of(e, f) : 0;
-                            const int lo = __reduce_add_sync(0xFFFFFFFFu, (int)mv);      // (Z_TT: the two TTFTs are equal)
-                            if (lane == first && lo) atomicAdd((unsigned long long*)&sm.e_sum[jj][f], (unsigned long long)(long long)lo);
-                        }
-                    }
+                    add_outcome(e, 1, O_SERVER_ONLY, q, q.S); add_outcome(e, -1, v.oc_h, q, v.tt_h);   // (the two TTFTs are equal)
+                    enter_small(sm.j_sum[v.j], e);
                     // a hand-off stall the first run would have had: those policies lose it
-                    if (has_j && v.oc_h >= O_MIGR_TO_DEV && stall_bin)
+                    if (v.oc_h >= O_MIGR_TO_DEV && stall_bin)
                         for (int p = 0; p < v.j; ++p)
                             atomicAdd(&out.hist_tbt[(size_t)sm.pol[p] * kNBins + bin_of_ticks(q.stall)], ~0ull);
                 }
@@ -294,9 +341,11 @@ __device__ __forceinline__ Sums sweep(ZoneSmem& sm, const TileCtx& c, const Seg&
                 oc = q.S > w + Td ? O_RACE_DEV : O_RACE_SRV;     // a tie goes to the server
                 if (oc == c.race_that_migrates && saving > sm.theta[point]) oc += 2;
             }
-            if (ok) { add_outcome(d, 1, oc, q, tt); add_outcome(d, -1, v.oc_c, q, v.tt_c); }
-            hist_add(sm.h_ttft, ok, bin_of_ticks(tt));
-            hist_add(sm.h_stall, ok && oc >= O_MIGR_TO_DEV && stall_bin, bin_of_ticks(q.stall));
+            const bool mine = ok && !(apart && point < 32);    // (the pair kernel has the first tile of such a request)
+            if (mine) { add_outcome(d, 1, oc, q, tt); add_outcome(d, -1, v.oc_c, q, v.tt_c); }
+            // (h_* minus g_* is entered for the policy: a request that is not its own joins both)
+            hist_add(sm.h_ttft, ok, bin_of_ticks(mine ? tt : v.tt_c));
+            if (c.may_migrate) hist_add(sm.h_stall, ok && (mine ? oc : v.oc_c) >= O_MIGR_TO_DEV && stall_bin, bin_of_ticks(q.stall));
         }
     }
     return d;
@@ -323,7 +372,7 @@ __device__ __forceinline__ void share_out(ZoneSmem& sm, const Sums& s) {
 // histograms of the policies of row's own tile.  alone >= 0: for that policy alone.  With add_every, g_* joins what
 // every policy gets.  Clears h_* and, with clear_g, g_*.  All threads call; barrier after.
 __device__ __forceinline__ void enter_segment(ZoneSmem& sm, int row, int alone, bool add_every, bool clear_g, const FlushTo& out) {
-    const int b = threadIdx.x;
+    for (int b = threadIdx.x; b < kNBins + kZSums + kJRows * kZSums; b += kZThreads) {
     if (b < kNBins) {
         const int32_t gt = (int32_t)sm.g_ttft[b], gs = (int32_t)sm.g_stall[b];
         const int32_t dt = (int32_t)sm.h_ttft[b] - gt, ds = (int32_t)sm.h_stall[b] - gs;
@@ -345,12 +394,22 @@ __device__ __forceinline__ void enter_segment(ZoneSmem& sm, int row, int alone, 
         }
         sm.h_ttft[b] = 0; sm.h_stall[b] = 0;
         if (clear_g) { sm.g_ttft[b] = 0; sm.g_stall[b] = 0; }
-    } else if (b < kNBins + kZSums && (row > 0 || alone >= 0)) {
-        const int f = b - kNBins;
-        long long v = 0;
-        for (int w = 0; w < kZWarps; ++w) v += sm.part[w][f];
-        if (row > 0) sm.e_sum[row][f] += v;
-        else { sm.e_sum[alone + 1][f] += v; if (alone > 0) sm.e_sum[alone][f] -= v; }   // (row 0 is carried to nobody)
+    } else if (b < kNBins + kZSums) {
+        if (row > 0 || alone >= 0) {
+            const int f = b - kNBins;
+            long long v = 0;
+            for (int w = 0; w < kZWarps; ++w) v += sm.part[w][f];
+            // (atomic: the threads below may add to the same row)
+            unsigned long long* e = (unsigned long long*)&sm.e_sum[row > 0 ? row : alone + 1][f];
+            atomicAdd(e, (unsigned long long)v);
+            if (row <= 0 && alone > 0) atomicAdd((unsigned long long*)&sm.e_sum[alone][f], 0ull - (unsigned long long)v);   // (row 0 is carried to nobody)
+        }
+    } else {
+        // what single requests entered during the sweep
+        const int k = b - kNBins - kZSums, r = k / kZSums, f = k % kZSums;
+        const int32_t v = sm.j_sum[r][f];
+        if (v) { atomicAdd((unsigned long long*)&sm.e_sum[r][f], (unsigned long long)(long long)v); sm.j_sum[r][f] = 0; }
+    }
     }
 }
 
@@ -391,22 +450,22 @@ __device__ __forceinline__ void flush_sums(const ZoneSmem& sm, int npol, const F
 // Adds to the global histograms of every policy what the chunk gave all of them plus the coarse rows above the
 // policy's tile.  All threads call (barrier before).
 __device__ __forceinline__ void flush_hist(const ZoneSmem& sm, int n_fam, int npol, const FlushTo& to) {
-    const int b = threadIdx.x;
-    if (b >= kNBins) return;
-    int32_t t = sm.c_ttft[b], s = sm.c_stall[b];
-    for (int tile = n_fam - 1; tile >= 0; --tile) {
-        if (tile + 1 < kCoarseRows && tile + 1 <= n_fam) { t += sm.k_ttft[tile + 1][b]; s += sm.k_stall[tile + 1][b]; }
-        if ((t | s) == 0) continue;
-        for (int p = 32 * tile; p < min(npol, 32 * tile + 32); ++p) {
-            const size_t o = (size_t)sm.pol[p] * kNBins + b;
-            if (t) atomicAdd(&to.hist_ttft[o], (unsigned long long)(long long)t);
-            if (s) atomicAdd(&to.hist_tbt[o], (unsigned long long)(long long)s);
+    for (int b = threadIdx.x; b < kNBins; b += kZThreads) {
+        int32_t t = sm.c_ttft[b], s = sm.c_stall[b];
+        for (int tile = n_fam - 1; tile >= 0; --tile) {
+            if (tile + 1 < kCoarseRows) { t += sm.k_ttft[tile + 1][b]; s += sm.k_stall[tile + 1][b]; }
+            if ((t | s) == 0) continue;
+            for (int p = 32 * tile; p < min(npol, 32 * tile + 32); ++p) {
+                const size_t o = (size_t)sm.pol[p] * kNBins + b;
+                if (t) atomicAdd(&to.hist_ttft[o], (unsigned long long)(long long)t);
+                if (s) atomicAdd(&to.hist_tbt[o], (unsigned long long)(long long)s);
+            }
         }
     }
 }
 
 // What a family's evaluation of a chunk reports.
-struct FamTotals { uint32_t left, passes; };
+struct FamTotals { uint32_t left, apart, passes; };   // apart: left for the first tile alone
 
 // One chunk under one family of n_fam tiles starting at tile0 (the shared tables of the family are set up).
 // WAITS: the policies are Algorithm 2's (wait map); otherwise Algorithm 3's (length threshold).
@@ -424,9 +483,8 @@ __device__ __forceinline__ FamTotals zone_family(ZoneSmem& sm, const TileCtx& c,
     // ---- the segments: stretches of prompt lengths between two thresholds, and (Algorithm 2) the thresholds
     //      themselves; a thread per candidate looks up where its lengths lie in the chunk
     {
-        const int q = threadIdx.x;
-        const int n_cand = WAITS ? 2 * npol + 1 : npol + 1;
-        if (q < n_cand && len) {
+        const int n_cand = len ? (WAITS ? 2 * npol + 1 : npol + 1) : 0;
+        for (int q = threadIdx.x; q < n_cand; q += kZThreads) {
             auto cl = [](int x) { return min(max(x, 0), kMaxPrompt + 1); };
             int la, lb;
             bool any = true;
@@ -461,7 +519,7 @@ __device__ __forceinline__ FamTotals zone_family(ZoneSmem& sm, const TileCtx& c,
 
     Sums every;
     clear(every);
-    uint32_t n_left = 0, passes = 0;
+    uint32_t n_left = 0, n_apart = 0, passes = 0;
     const int n_seg = (int)min(sm.n_seg, (uint32_t)kMaxSeg);
     for (int si = 0; si < n_seg; ++si) {
         const Seg s = sm.seg[si];
@@ -474,13 +532,14 @@ __device__ __forceinline__ FamTotals zone_family(ZoneSmem& sm, const TileCtx& c,
                          ((1u << n_fam) - 1u) << (tile0 & 31u));
                 ++n_left;
                 if (left_list) {
-                    const uint32_t at = atomicAdd(&sm.n_listed, 1u);
-                    if (at < kLeftList) for (int t = 0; t < n_fam; ++t) left_list[(size_t)t * kLeftList + at] = i;
+                    const uint32_t at0 = atomicAdd(&sm.n_listed0, 1u), at = n_fam > 1 ? atomicAdd(&sm.n_listed, 1u) : 0u;
+                    if (at0 < kLeftList) left_list[at0] = i;
+                    if (at < kLeftList) for (int t = 1; t < n_fam; ++t) left_list[(size_t)t * kLeftList + at] = i;
                 }
             }
             continue;
         }
-        const Sums d = sweep<WAITS>(sm, c, s, -1, every, n_left, tile0, n_fam, n_tiles, left_mask, left_list, out);
+        const Sums d = sweep<WAITS>(sm, c, s, -1, every, n_left, n_apart, tile0, n_fam, n_tiles, left_mask, left_list, out);
         const bool first_run = s.k2 < npol && s.k1 > 0;
         if (first_run) share_out(sm, d);
         __syncthreads();
@@ -489,7 +548,7 @@ __device__ __forceinline__ FamTotals zone_family(ZoneSmem& sm, const TileCtx& c,
         ++passes;
         if (WAITS && points) {
             for (int p = s.k1; p < s.k2; ++p) {
-                const Sums dp = sweep<WAITS>(sm, c, s, p, every, n_left, tile0, n_fam, n_tiles, left_mask, left_list, out);
+                const Sums dp = sweep<WAITS>(sm, c, s, p, every, n_left, n_apart, tile0, n_fam, n_tiles, left_mask, left_list, out);
                 share_out(sm, dp);
                 __syncthreads();
                 enter_segment(sm, 0, p, false, p + 1 == s.k2, out);
@@ -501,7 +560,8 @@ __device__ __forceinline__ FamTotals zone_family(ZoneSmem& sm, const TileCtx& c,
     // ---- the chunk is done: what every policy gets, then everything goes out
     share_out(sm, every);
     n_left = __reduce_add_sync(0xFFFFFFFFu, n_left);
-    if ((threadIdx.x & 31) == 0 && n_left) atomicAdd(&sm.n_left, n_left);
+    n_apart = __reduce_add_sync(0xFFFFFFFFu, n_apart);
+    if ((threadIdx.x & 31) == 0 && (n_left | n_apart)) { atomicAdd(&sm.n_left, n_left); atomicAdd(&sm.n_apart, n_apart); }
     __syncthreads();
     if (threadIdx.x < kZSums) {
         long long v = 0;
@@ -513,6 +573,7 @@ __device__ __forceinline__ FamTotals zone_family(ZoneSmem& sm, const TileCtx& c,
     flush_hist(sm, n_fam, npol, out);
     FamTotals tot;
     tot.left = sm.n_left;
+    tot.apart = sm.n_apart;
     tot.passes = passes;
     __syncthreads();
     return tot;
@@ -522,8 +583,8 @@ __device__ __forceinline__ FamTotals zone_family(ZoneSmem& sm, const TileCtx& c,
 // evaluated as one family: plain Algorithm 2 or plain Algorithm 3 policies of one kind (no random routing, no
 // Eq. 1-2 wait rule, one expected length for Eq. 4) whose length thresholds are ordered along the list --
 // Algorithm 3's l_th not increasing, Algorithm 2's l* not decreasing, as they are along an ascending budget axis.
-// A family of more than one tile of Algorithm 2 policies must also share one w_tail: then its first run never
-// splits by wait.  All threads call.
+// In a family of more than one tile of Algorithm 2 policies, only the first tile's waits w_tail may differ from the
+// smallest one (as they do along a budget axis: the lowest budgets wait longest).  All threads call.
 __device__ __forceinline__ bool family_setup(ZoneSmem& sm, TileCtx& c, const Prep* __restrict__ prep, uint32_t P, int g,
                                              const GroupConst& gc, const uint32_t* __restrict__ pol_list, uint32_t first,
                                              int npol, bool& waits) {
@@ -563,18 +624,21 @@ __device__ __forceinline__ bool family_setup(ZoneSmem& sm, TileCtx& c, const Pre
     c.th_min = __uint_as_float(sm.red[0]); c.th_max = __uint_as_float(sm.red[1]);
     c.wt_min = sm.red[2]; c.wt_max = sm.red[3];
     c.may_migrate = c.th_min != __int_as_float(0x7F800000);          // some policy of the family can hand over
-    if (npol > 32 && waits && c.wt_min != c.wt_max) ok = false;
+    // several tiles of Algorithm 2 policies: beyond the first tile the waits w_tail must all be the smallest one
+    const bool rest_alike = __syncthreads_and(p < 32 || p >= npol || sm.w_tail[p] == c.wt_min) != 0;
+    c.tile0_apart = npol > 32 && waits && c.wt_min != c.wt_max;
+    if (c.tile0_apart && !(rest_alike && c.wt_ordered)) ok = false;
     return ok;
 }
 
-__global__ void __launch_bounds__(kZThreads, 1)
+__global__ void __launch_bounds__(kZThreads, kZBlocksPerSm)
 k_pairs_zones(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst* __restrict__ ccp,
               const Prep* __restrict__ prep, uint32_t P, const uint32_t* __restrict__ pol_list, uint32_t n_list,
               int PL, const Chunk* __restrict__ chunks, uint32_t n_chunks, uint32_t n_tiles, TimelineRec rec,
               unsigned long long* __restrict__ acc, unsigned long long* __restrict__ hist_ttft,
               unsigned long long* __restrict__ hist_tbt, uint32_t* __restrict__ left_mask,
               uint32_t* __restrict__ left_count, uint32_t* __restrict__ left_lists,
-              unsigned long long* __restrict__ work) {
+              uint32_t* __restrict__ ticket, unsigned long long* __restrict__ work) {
     extern __shared__ __align__(16) unsigned char zsmem_raw[];
     ZoneSmem& sm = *reinterpret_cast<ZoneSmem*>(zsmem_raw);
     grid_dependency_wait();
@@ -583,7 +647,13 @@ k_pairs_zones(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst*
     const bool lean = cc.pacing != 0 && cc.W[0] == 1 && cc.W[1] == 1 && cc.W[2] == 1;
     const uint32_t n_fams = (n_tiles + kFamTiles - 1) / kFamTiles;
 
-    for (uint32_t item = blockIdx.x; item < n_chunks * n_fams; item += gridDim.x) {
+    // the blocks draw (chunk, family) items from a counter (zero at launch): items differ in cost
+    for (;;) {
+        __syncthreads();
+        if (threadIdx.x == 0) sm.ticket = atomicAdd(ticket, 1u);
+        __syncthreads();
+        const uint32_t item = sm.ticket;
+        if (item >= n_chunks * n_fams) break;
         const uint32_t fam = item % n_fams, chunk_id = item / n_fams;
         const Chunk ch = chunks[chunk_id];
         const int g = ch.g;
@@ -633,9 +703,9 @@ k_pairs_zones(TraceDev tr, const GroupConst* __restrict__ gcs, const ClassConst*
             const FamTotals tot = waits ? zone_family<true>(sm, c, tile0, n_fam, n_tiles, chunk_id, tr.len_end, left_mask, left_lists, out)
                                         : zone_family<false>(sm, c, tile0, n_fam, n_tiles, chunk_id, tr.len_end, left_mask, left_lists, out);
             if (threadIdx.x == 0) {
-                for (int t = 0; t < n_fam; ++t) left_count[(size_t)chunk_id * n_tiles + tile0 + t] = tot.left;
+                for (int t = 0; t < n_fam; ++t) left_count[(size_t)chunk_id * n_tiles + tile0 + t] = tot.left + (t ? 0u : tot.apart);
                 if (work) {
-                    atomicAdd(&work[0], (unsigned long long)(ch.len - tot.left) * npol);   // pairs settled zone by zone
+                    atomicAdd(&work[0], (unsigned long long)(ch.len - tot.left) * npol - (unsigned long long)tot.apart * 32u);   // pairs settled zone by zone
                     atomicAdd(&work[2], (unsigned long long)(ch.len - tot.left));          // requests settled, per family
                     atomicAdd(&work[3], (unsigned long long)tot.passes);                   // sweeps over segments
                 }
@@ -653,17 +723,17 @@ cudaError_t launch_pairs_zones(const TraceDev& tr, const GroupConst* gc, const C
                                uint32_t P, const uint32_t* pol_list, uint32_t n_list, int PL, const Chunk* chunks,
                                uint32_t n_chunks, TimelineRec rec, uint64_t* acc, uint64_t* hist_ttft,
                                uint64_t* hist_tbt, uint32_t* left_mask, uint32_t* left_count, uint32_t* left_lists,
-                               uint32_t max_blocks, uint64_t* work, cudaStream_t st) {
+                               uint32_t max_blocks, uint32_t* ticket, uint64_t* work, cudaStream_t st) {
     const uint32_t n_tiles = (n_list + PL - 1) / PL;
     const uint32_t n_fams = (n_tiles + kFamTiles - 1) / kFamTiles;
     if ((uint64_t)n_chunks * n_tiles > 0x7FFFFFFFull) return cudaErrorInvalidConfiguration;
     cudaError_t e = cudaFuncSetAttribute(k_pairs_zones, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(ZoneSmem));
     if (e) return e;
-    const uint32_t blocks = (uint32_t)std::min<uint64_t>((uint64_t)n_chunks * n_fams, max_blocks);
+    const uint32_t blocks = (uint32_t)std::min<uint64_t>((uint64_t)n_chunks * n_fams, (uint64_t)max_blocks * kZBlocksPerSm);
     return launch_after(k_pairs_zones, dim3(blocks), kZThreads, sizeof(ZoneSmem), st, tr, gc, cc, prep, P,
                         pol_list, n_list, PL, chunks, n_chunks, n_tiles, rec, (unsigned long long*)acc,
                         (unsigned long long*)hist_ttft, (unsigned long long*)hist_tbt, left_mask, left_count, left_lists,
-                        (unsigned long long*)work);
+                        ticket, (unsigned long long*)work);
 }
 
 }  // namespace disco
