@@ -188,13 +188,24 @@ __device__ __forceinline__ bool head_outcome_waits(const TileCtx& c, const ZoneS
     return t >= 0;
 }
 
-// One more count in a block-private histogram; the lanes of the warp that meet in a bin add once.
+// One more count in a block-private histogram, for counts that tend to meet in one bin (requests of one prompt
+// length share the device's TTFT): if all the warp's counts fall in one bin, one lane adds them.
 __device__ __forceinline__ void hist_add(uint32_t* hist, bool on, int bin) {
     on = on && DBG_OK(bin, kNBins, DBG_K_PAIRS_ZONES, DBG_BIN);
     const uint32_t live = __ballot_sync(0xFFFFFFFFu, on);
-    if (!on) return;
-    const uint32_t peers = __match_any_sync(live, bin);
-    if ((peers & ((1u << (threadIdx.x & 31)) - 1u)) == 0u) atomicAdd(&hist[bin], (uint32_t)__popc(peers));
+    if (live == 0u) return;
+    const int leader = __ffs(live) - 1;
+    const int bin0 = __shfl_sync(0xFFFFFFFFu, bin, leader);
+    if (__all_sync(0xFFFFFFFFu, !on || bin == bin0)) {
+        if ((int)(threadIdx.x & 31) == leader) atomicAdd(&hist[bin0], (uint32_t)__popc(live));
+    } else if (on) {
+        atomicAdd(&hist[bin], 1u);
+    }
+}
+
+// The same for counts that are rare or spread over many bins: every lane adds for itself.
+__device__ __forceinline__ void hist_add_each(uint32_t* hist, bool on, int bin) {
+    if (on && DBG_OK(bin, kNBins, DBG_K_PAIRS_ZONES, DBG_BIN)) atomicAdd(&hist[bin], 1u);
 }
 
 // One request's difference into a row of 32-bit sums (the TTFT sum is not entered: the caller sees to it).  A
@@ -284,15 +295,15 @@ __device__ __forceinline__ Sums sweep(ZoneSmem& sm, const TileCtx& c, const Seg&
                 }
             }
             if (ok) add_outcome(every, 1, v.oc_c, q, v.tt_c);
-            hist_add(sm.g_ttft, ok, bin_of_ticks(v.tt_c));
-            if (c.may_migrate) hist_add(sm.g_stall, ok && v.oc_c >= O_MIGR_TO_DEV && stall_bin, bin_of_ticks(q.stall));
+            hist_add_each(sm.g_ttft, ok, bin_of_ticks(v.tt_c));
+            if (c.may_migrate) hist_add_each(sm.g_stall, ok && v.oc_c >= O_MIGR_TO_DEV && stall_bin, bin_of_ticks(q.stall));
             // (a request left for the first tile alone, whose first run lies inside that tile: no first run to enter)
             const bool runs = ok && !(WAITS && apart && k1 < 32);
             if (first_run) {
                 if (runs) { add_outcome(d, 1, v.oc_h, q, v.tt_h); add_outcome(d, -1, v.oc_c, q, v.tt_c); }
                 // (h_* minus g_* is entered for the segment: a request without a first run joins both)
                 hist_add(sm.h_ttft, ok, bin_of_ticks(runs ? v.tt_h : v.tt_c));
-                if (c.may_migrate) hist_add(sm.h_stall, ok && (runs ? v.oc_h : v.oc_c) >= O_MIGR_TO_DEV && stall_bin, bin_of_ticks(q.stall));
+                if (c.may_migrate) hist_add_each(sm.h_stall, ok && (runs ? v.oc_h : v.oc_c) >= O_MIGR_TO_DEV && stall_bin, bin_of_ticks(q.stall));
             }
             if (WAITS && c.tile0_apart) {
                 // ---- the first tile gets nothing from the family for such a request (the pair kernel evaluates it there):
@@ -345,7 +356,7 @@ __device__ __forceinline__ Sums sweep(ZoneSmem& sm, const TileCtx& c, const Seg&
             if (mine) { add_outcome(d, 1, oc, q, tt); add_outcome(d, -1, v.oc_c, q, v.tt_c); }
             // (h_* minus g_* is entered for the policy: a request that is not its own joins both)
             hist_add(sm.h_ttft, ok, bin_of_ticks(mine ? tt : v.tt_c));
-            if (c.may_migrate) hist_add(sm.h_stall, ok && (mine ? oc : v.oc_c) >= O_MIGR_TO_DEV && stall_bin, bin_of_ticks(q.stall));
+            if (c.may_migrate) hist_add_each(sm.h_stall, ok && (mine ? oc : v.oc_c) >= O_MIGR_TO_DEV && stall_bin, bin_of_ticks(q.stall));
         }
     }
     return d;
