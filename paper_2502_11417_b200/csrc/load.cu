@@ -302,6 +302,49 @@ __global__ void k_scatter_by_length(uint32_t n, int G, const uint64_t* __restric
     }
 }
 
+// The same for traces whose length histograms fit in shared memory (up to six groups).  A block takes slices of
+// kSliceRequests requests: it counts the slice's requests per bucket in shared memory, reserves each bucket's places
+// with ONE add to the global cursor, and hands the places out from shared memory.  A popular bucket's cursor then
+// sees one add per slice instead of one per warp (adds to one address are served one after another).
+constexpr uint32_t kSliceRequests = 16384;
+constexpr int kSliceThreads = 1024;
+
+__global__ void __launch_bounds__(kSliceThreads)
+k_scatter_by_length_slices(uint32_t n, int G, const uint64_t* __restrict__ keys,
+                           const uint16_t* __restrict__ prompt, const uint16_t* __restrict__ outlen,
+                           const int32_t* __restrict__ err, uint32_t* __restrict__ cursor,
+                           uint4* __restrict__ placed, uint32_t* __restrict__ inv) {
+    extern __shared__ uint32_t s_at[];               // [G][kMaxPrompt + 1]: counts, then next free places
+    if (err[0] != 0) return;                         // a rejected trace: its lengths were not all written
+    const uint32_t buckets = (uint32_t)G * (uint32_t)(kMaxPrompt + 1);
+    for (uint32_t lo = blockIdx.x * kSliceRequests; lo < n; lo += gridDim.x * kSliceRequests) {
+        const uint32_t hi = min(n, lo + kSliceRequests);
+        for (uint32_t b = threadIdx.x; b < buckets; b += kSliceThreads) s_at[b] = 0;
+        __syncthreads();
+        for (uint32_t i = lo + threadIdx.x; i < hi; i += kSliceThreads) {
+            const uint32_t g = (uint32_t)(keys[i] >> 32), len = prompt[i];
+            if (DBG_OK(g, G, DBG_K_GATHER, DBG_GROUP) && DBG_OK(len, kMaxPrompt + 1, DBG_K_GATHER, DBG_TABLE))
+                atomicAdd(&s_at[g * (uint32_t)(kMaxPrompt + 1) + len], 1u);
+        }
+        __syncthreads();
+        for (uint32_t b = threadIdx.x; b < buckets; b += kSliceThreads) {
+            const uint32_t c = s_at[b];
+            if (c) s_at[b] = atomicAdd(&cursor[b], c);
+        }
+        __syncthreads();
+        for (uint32_t i = lo + threadIdx.x; i < hi; i += kSliceThreads) {
+            const uint64_t key = keys[i];
+            const uint32_t g = (uint32_t)(key >> 32), len = prompt[i];
+            if (!DBG_OK(g, G, DBG_K_GATHER, DBG_GROUP) || !DBG_OK(len, kMaxPrompt + 1, DBG_K_GATHER, DBG_TABLE)) continue;
+            const uint32_t at = atomicAdd(&s_at[g * (uint32_t)(kMaxPrompt + 1) + len], 1u);
+            if (!DBG_OK(at, n, DBG_K_GATHER, DBG_REQUEST)) continue;
+            placed[at] = make_uint4((uint32_t)key, len | ((uint32_t)outlen[i] << 16), i, 0u);
+            inv[i] = at;
+        }
+        __syncthreads();
+    }
+}
+
 __global__ void k_unpack_requests(uint32_t n, const uint4* __restrict__ placed, const int32_t* __restrict__ err,
                                   int32_t* __restrict__ S, uint16_t* __restrict__ l, uint16_t* __restrict__ nout,
                                   uint32_t* __restrict__ orig) {
@@ -459,8 +502,16 @@ cudaError_t run_load(const LoadArgs& a, cudaStream_t st) {
             a.l_tmp, a.n_tmp, small ? counts_a : nullptr, per_block, blocks, hist_groups);
         // internal request order: by group, then by prompt length
         k_length_cursors<<<G, 1024, 0, st>>>(a.cnt, a.ng, a.cursors);
-        k_scatter_by_length<<<grid_for(n, 256, a.sms), 256, 0, st>>>(n, G, a.keys_a, a.l_tmp, a.n_tmp, a.err, a.cursors,
-                                                                     a.placed, a.inv);
+        const size_t cursor_bytes = (size_t)G * (kMaxPrompt + 1) * 4;
+        if (cursor_bytes <= 100 * 1024) {
+            if ((e = cudaFuncSetAttribute(k_scatter_by_length_slices, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024))) return e;
+            const uint32_t slices = (n + kSliceRequests - 1) / kSliceRequests;
+            k_scatter_by_length_slices<<<std::min<uint32_t>(slices, 2u * (uint32_t)a.sms), kSliceThreads, cursor_bytes, st>>>(
+                n, G, a.keys_a, a.l_tmp, a.n_tmp, a.err, a.cursors, a.placed, a.inv);
+        } else {
+            k_scatter_by_length<<<grid_for(n, 256, a.sms), 256, 0, st>>>(n, G, a.keys_a, a.l_tmp, a.n_tmp, a.err, a.cursors,
+                                                                         a.placed, a.inv);
+        }
         k_unpack_requests<<<grid_for(n, 256, a.sms), 256, 0, st>>>(n, a.placed, a.err, a.S, a.l, a.nout, a.orig);
         // sort (group, ticks): four byte passes over the ticks, one over the group id
         uint64_t *src = a.keys_a, *dst = a.keys_b;
