@@ -482,12 +482,14 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
         cls_range.push_back({b, (uint32_t)pol_list.size()});
     }
     const uint32_t tiles = (P + 31) / 32;
-    // the zone kernel runs a block per (chunk, family of four policy tiles); a lane of it counts its requests in
-    // bytes: at most 127 requests a lane, 1024 lanes a block
+    // the zone kernel's blocks take (chunk, family of four policy tiles) items; the pair kernel works a chunk in
+    // passes of at most 65,280 requests
     const uint32_t kMaxChunk = 130560;
     const uint32_t sms = (uint32_t)c->sms;
     const uint32_t fams = (tiles + 3) / 4;
-    uint32_t want_chunks = std::max<uint32_t>(1, sms / std::min<uint32_t>(fams, sms));   // one block per SM
+    // about two items a block (the blocks draw them from a counter, so uneven items even out), chunks of 2,048
+    // requests or more
+    uint32_t want_chunks = std::max<uint32_t>(1, (2 * sms + fams - 1) / fams);
     const uint32_t min_chunks = (uint32_t)((N1 + kMaxChunk - 1) / kMaxChunk);
     if (min_chunks > want_chunks) {
         // several waves of blocks: the fewest chunks whose last wave is nearly full (long chunks spread a block's
@@ -502,7 +504,7 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
     }
     uint32_t CH = (uint32_t)((N1 + want_chunks - 1) / want_chunks);
     CH = (CH + 255) / 256 * 256;
-    CH = std::min<uint32_t>(std::max<uint32_t>(CH, 256), kMaxChunk);
+    CH = std::min<uint32_t>(std::max<uint32_t>(CH, 2048), kMaxChunk);
     std::vector<Chunk> chunks;
     for (int g = 0; g < G; ++g)
         for (uint32_t s = rb.grp_off[g]; s < rb.grp_off[g + 1]; s += CH)

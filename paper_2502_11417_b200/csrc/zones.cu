@@ -267,13 +267,10 @@ __device__ __forceinline__ Sums sweep(ZoneSmem& sm, const TileCtx& c, const Seg&
     const uint32_t left_bits = ((1u << n_fam) - 1u) << (tile0 & 31u);       // (a family does not straddle a mask word)
     Sums d;
     clear(d);
-    bool nx_stall;
-    Req nx = load_request(c, s.pa + threadIdx.x, nx_stall);
     for (uint32_t i0 = s.pa + (threadIdx.x & ~31u); i0 < s.pb; i0 += kZThreads) {      // a warp's lanes iterate together
         const uint32_t i = i0 + lane;
-        Req q = nx;
-        const bool stall_bin = nx_stall;
-        if (i0 + kZThreads < s.pb) nx = load_request(c, i + kZThreads, nx_stall);
+        bool stall_bin;
+        const Req q = load_request(c, i, stall_bin);
         const bool valid = i < s.pb;
         const uint32_t Td = c.kappa * q.l + c.c0;
         const float saving = saving_of(c, q);
