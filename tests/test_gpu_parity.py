@@ -477,3 +477,38 @@ def test_more_than_32_policy_tiles_use_several_flag_words():
     full_parity(w, pols, select=False, tag="35 tiles")
     zone, left, _, _ = _work(w, pols)
     assert zone > 0 and left > 0
+
+
+def test_one_prompt_length_and_lengths_at_the_ends():
+    # every request in one bucket of the internal order: a chunk is one segment (or a threshold's own), and all
+    # lanes of a warp meet in one row and one histogram bin
+    grid = synth.budget_grid(70)                   # three policy tiles: a family of several tiles
+    for dear in (False, True):
+        w = synth.tiny_workload(71 + dear, 5000, n_servers=1, n_devices=1, max_prompt=900, max_out=120, device_dearer=dear)
+        w.prompt_len[:] = 300
+        full_parity(w, [synth.policy(b, mig_threshold=0.004) for b in grid], tag=f"one length dear={dear}")
+        # only the shortest and the longest prompt there is
+        w.prompt_len[:] = np.where(np.arange(w.n) % 3 == 0, 1, 4096).astype(np.int32)
+        full_parity(w, [synth.policy(b, mig_threshold=0.004) for b in grid], tag=f"lengths 1 and 4096 dear={dear}")
+
+
+def test_more_groups_than_fit_the_scatter_in_shared_memory():
+    # 3 x 3 = 9 groups: the internal request order is built with one add per warp and bucket to the global cursors
+    # (the length histograms of more than six groups do not fit the slice-wise kernel's shared memory)
+    w = synth.tiny_workload(73, 9000, n_servers=3, n_devices=3, max_prompt=600, max_out=100)
+    full_parity(w, [synth.policy(b, mig_threshold=0.01) for b in synth.budget_grid(40)], tag="nine groups")
+    zone, left, _, _ = _work(w, [synth.policy(b, mig_threshold=0.01) for b in synth.budget_grid(40)])
+    assert zone + left == w.n * 40
+
+
+def test_family_whose_first_tile_alone_has_longer_waits():
+    # Algorithm 2 along 128 ascending budgets: the lowest budgets wait longest (w_tail falls until it settles), so a
+    # family of four tiles stays whole and requests under which the device wins after such a wait are left to the
+    # pair kernel for the first tile only
+    w = synth.tiny_workload(74, 20000, n_servers=1, n_devices=1, max_prompt=2000, max_out=200, device_dearer=True)
+    pols = [synth.policy(b, mig_threshold=th) for th in (0.0, synth.INF) for b in synth.budget_grid(128)]
+    full_parity(w, pols, select=False, tag="four-tile families with waits")
+    zone, left, settled, _ = _work(w, pols)
+    assert zone + left == w.n * len(pols)
+    assert left < 0.1 * zone
+    assert settled <= 2 * w.n                      # one sweep per request and family, not per tile
