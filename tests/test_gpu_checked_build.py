@@ -14,7 +14,8 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 CASES = ("test_config0_full or test_config1_shape or test_config3_shape or test_config4_shape or test_config5_shape "
          "or test_edge_cases or test_empty_trace or test_flag_and_mode_matrix or test_buffer_search_paths "
          "or test_stochastic_baselines or test_linear_wait_rule or test_zone_by_zone or test_more_than_32_policy_tiles "
-         "or test_mixed_timeline_classes or test_generation_slower or test_sorted_ticks_around")
+         "or test_mixed_timeline_classes or test_generation_slower or test_sorted_ticks_around "
+         "or test_one_prompt_length or test_more_groups_than_fit or test_family_whose_first_tile")
 
 
 def _run(args):
