@@ -10,7 +10,7 @@ namespace disco {
 
 namespace {
 
-constexpr int kIngestThreads = 256;
+constexpr int kIngestThreads = 1024;
 
 __global__ void k_ingest(uint32_t n, const int32_t* __restrict__ prompt, const int32_t* __restrict__ outlen,
                          const float* __restrict__ ttft, const uint8_t* __restrict__ sp,
