@@ -68,7 +68,7 @@ namespace {
 // Returns 0, or DISCO_ECUDA with the kernel and the index in the error string.
 int debug_check() {
 #ifdef DISCO_DEBUG
-    static const char* kernels[DBG_K_COUNT] = {"", "k_ingest", "radix sort", "k_gather", "group tables", "k_prep",
+    static const char* kernels[DBG_K_COUNT] = {"", "k_ingest", "radix sort", "k_scatter_by_length", "group tables", "k_prep",
                                                "k_playout_fast", "k_playout", "k_pairs_acc", "k_pairs_zones", "k_pairs_rows",
                                                "k_finalize", "k_select", "self-test"};
     static const char* whats[DBG_WHAT_COUNT] = {"", "request", "policy", "group", "chunk", "knot", "histogram bin",
