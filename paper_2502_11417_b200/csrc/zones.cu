@@ -220,7 +220,7 @@ __device__ __forceinline__ void enter_small(int32_t* row, const Sums& e) {
 }
 
 // What a request comes to under the policies of its segment.
-struct Verdict {
+struct Fate {
     bool ok;                            // the runs express it
     bool apart;                         // ... except for the policies of the family's first tile
     int oc_c, oc_h, j;                  // outcome every policy gets; outcome of the first run [j, k1); covered waits [0, j)
@@ -231,9 +231,9 @@ struct Verdict {
 // any) differs from it; with k1 = k2 = npol every policy is in the first run, whose outcome then is what every
 // policy gets.
 template <bool WAITS>
-__device__ __forceinline__ Verdict judge(const TileCtx& c, const ZoneSmem& sm, const Req& q, uint32_t Td, float saving,
+__device__ __forceinline__ Fate fate_of(const TileCtx& c, const ZoneSmem& sm, const Req& q, uint32_t Td, float saving,
                                          int k1, int k2) {
-    Verdict v;
+    Fate v;
     v.oc_c = O_DEVICE_ONLY; v.oc_h = O_DEVICE_ONLY; v.j = 0; v.tt_c = Td; v.tt_h = Td; v.ok = true; v.apart = false;
     if (k2 < c.npol) {
         v.ok = tail_outcome(c, q, Td, saving, v.oc_c, v.tt_c);
@@ -274,7 +274,7 @@ __device__ __forceinline__ Sums sweep(ZoneSmem& sm, const TileCtx& c, const Seg&
         const bool valid = i < s.pb;
         const uint32_t Td = c.kappa * q.l + c.c0;
         const float saving = saving_of(c, q);
-        const Verdict v = judge<WAITS>(c, sm, q, Td, saving, k1, k2);
+        const Fate v = fate_of<WAITS>(c, sm, q, Td, saving, k1, k2);
         const bool ok = v.ok && valid;
         const bool apart = v.apart && valid;                     // left to the pair kernel for the first tile alone
         if (point < 0) {
