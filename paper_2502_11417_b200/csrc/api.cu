@@ -484,7 +484,7 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
     const uint32_t tiles = (P + 31) / 32;
     // the zone kernel's blocks take (chunk, family of four policy tiles) items; the pair kernel works a chunk in
     // passes of at most 65,280 requests
-    const uint32_t kMaxChunk = 130560;
+    const uint32_t kMaxChunk = 65280;
     const uint32_t sms = (uint32_t)c->sms;
     const uint32_t fams = (tiles + 3) / 4;
     // about two items a block (the blocks draw them from a counter, so uneven items even out), chunks of 2,048
@@ -505,10 +505,18 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
     uint32_t CH = (uint32_t)((N1 + want_chunks - 1) / want_chunks);
     CH = (CH + 255) / 256 * 256;
     CH = std::min<uint32_t>(std::max<uint32_t>(CH, 2048), kMaxChunk);
+    // the groups' chunks take turns in the list: groups differ in what a chunk costs (Algorithm 2 sweeps more), and
+    // the blocks draw their work in list order, so the last items drawn should not all be of the dear kind
     std::vector<Chunk> chunks;
-    for (int g = 0; g < G; ++g)
-        for (uint32_t s = rb.grp_off[g]; s < rb.grp_off[g + 1]; s += CH)
-            chunks.push_back({s, std::min(CH, rb.grp_off[g + 1] - s), g, 0});
+    for (uint32_t turn = 0, added = 1; added; ++turn) {
+        added = 0;
+        for (int g = 0; g < G; ++g) {
+            const uint64_t s = (uint64_t)rb.grp_off[g] + (uint64_t)turn * CH;
+            if (s >= rb.grp_off[g + 1]) continue;
+            chunks.push_back({(uint32_t)s, std::min(CH, rb.grp_off[g + 1] - (uint32_t)s), g, 0});
+            ++added;
+        }
+    }
 #undef R
 
     // scratch of the pair kernels: a bit per (request, policy tile), a counter per (chunk, policy tile)
