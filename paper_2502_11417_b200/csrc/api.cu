@@ -505,18 +505,16 @@ int disco_eval_policies(disco_ctx_t* c, const disco_policy_t* pol, uint32_t P, u
     uint32_t CH = (uint32_t)((N1 + want_chunks - 1) / want_chunks);
     CH = (CH + 255) / 256 * 256;
     CH = std::min<uint32_t>(std::max<uint32_t>(CH, 2048), kMaxChunk);
-    // the groups' chunks take turns in the list: groups differ in what a chunk costs (Algorithm 2 sweeps more), and
-    // the blocks draw their work in list order, so the last items drawn should not all be of the dear kind
+    // the chunks of the groups that Algorithm 1 finds device-constrained come first: Algorithm 2's wait map costs the
+    // zone kernel more sweeps per chunk, and its blocks draw their work in list order, so the items drawn last (when
+    // some blocks already idle) should be the cheap ones
     std::vector<Chunk> chunks;
-    for (uint32_t turn = 0, added = 1; added; ++turn) {
-        added = 0;
+    for (int dear = 1; dear >= 0; --dear)
         for (int g = 0; g < G; ++g) {
-            const uint64_t s = (uint64_t)rb.grp_off[g] + (uint64_t)turn * CH;
-            if (s >= rb.grp_off[g + 1]) continue;
-            chunks.push_back({(uint32_t)s, std::min(CH, rb.grp_off[g + 1] - (uint32_t)s), g, 0});
-            ++added;
+            if ((c->gc[g].auto_device_constrained != 0) != (dear != 0)) continue;
+            for (uint32_t s = rb.grp_off[g]; s < rb.grp_off[g + 1]; s += CH)
+                chunks.push_back({s, std::min(CH, rb.grp_off[g + 1] - s), g, 0});
         }
-    }
 #undef R
 
     // scratch of the pair kernels: a bit per (request, policy tile), a counter per (chunk, policy tile)
