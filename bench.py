@@ -65,9 +65,11 @@ MAX_WARMUP_STEPS = 200
 # lane-slots the hardware executed per unit of work beside the algorithmic counts above.  None: not captured
 # for the current kernel.
 NCU_TRAFFIC_BYTES = {("k_pairs_rows", 1): 145709568, ("k_playout_fast", 1): 827904}
-# issued lane-slots per token-step (play-out; the workload-3 figure is of a 200,000-request capture of its shape) and
+# issued lane-slots per token-step (play-out; the workload-3 figure is of a 200,000-request capture of its shape, the
+# workload-4 figure of a 4,000,000-request one) and
 # per request and policy family (zone kernel, workload 2 at full size)
-NCU_EXECUTED_PER_UNIT = {("k_playout_fast", 1): 31.9, ("k_playout_fast", 3): 21.8, ("k_pairs_zones+k_pairs_acc", 2): 269.0}
+NCU_EXECUTED_PER_UNIT = {("k_playout_fast", 1): 31.9, ("k_playout_fast", 3): 21.8, ("k_playout_fast", 4): 28.2,
+                         ("k_pairs_zones+k_pairs_acc", 2): 269.0}
 HEADLINE_CONFIG = 4
 ALL_CONFIGS = (0, 1, 2, 3, 4, 5)
 
