@@ -299,7 +299,10 @@ __device__ __forceinline__ Sums sweep(ZoneSmem& sm, const TileCtx& c, const Seg&
             if (first_run) {
                 if (runs) { add_outcome(d, 1, v.oc_h, q, v.tt_h); add_outcome(d, -1, v.oc_c, q, v.tt_c); }
                 // (h_* minus g_* is entered for the segment: a request without a first run joins both)
-                hist_add(sm.h_ttft, ok, bin_of_ticks(runs ? v.tt_h : v.tt_c));
+                // (Algorithm 3: the first run's TTFT is the device's, one bin for a prompt length; Algorithm 2: mostly
+                // the server's own, spread over the bins)
+                if (WAITS) hist_add_each(sm.h_ttft, ok, bin_of_ticks(runs ? v.tt_h : v.tt_c));
+                else hist_add(sm.h_ttft, ok, bin_of_ticks(runs ? v.tt_h : v.tt_c));
                 if (c.may_migrate) hist_add_each(sm.h_stall, ok && (runs ? v.oc_h : v.oc_c) >= O_MIGR_TO_DEV && stall_bin, bin_of_ticks(q.stall));
             }
             if (WAITS && c.tile0_apart) {
@@ -352,7 +355,7 @@ __device__ __forceinline__ Sums sweep(ZoneSmem& sm, const TileCtx& c, const Seg&
             const bool mine = ok && !(apart && point < 32);    // (the pair kernel has the first tile of such a request)
             if (mine) { add_outcome(d, 1, oc, q, tt); add_outcome(d, -1, v.oc_c, q, v.tt_c); }
             // (h_* minus g_* is entered for the policy: a request that is not its own joins both)
-            hist_add(sm.h_ttft, ok, bin_of_ticks(mine ? tt : v.tt_c));
+            hist_add_each(sm.h_ttft, ok, bin_of_ticks(mine ? tt : v.tt_c));
             if (c.may_migrate) hist_add_each(sm.h_stall, ok && (mine ? oc : v.oc_c) >= O_MIGR_TO_DEV && stall_bin, bin_of_ticks(q.stall));
         }
     }
