@@ -267,6 +267,7 @@ __device__ __forceinline__ Sums sweep(ZoneSmem& sm, const TileCtx& c, const Seg&
     const uint32_t left_bits = ((1u << n_fam) - 1u) << (tile0 & 31u);       // (a family does not straddle a mask word)
     Sums d;
     clear(d);
+    long long tt_back = 0;                                       // TTFTs taken back at row 32 (requests left for the first tile alone)
     for (uint32_t i0 = s.pa + (threadIdx.x & ~31u); i0 < s.pb; i0 += kZThreads) {      // a warp's lanes iterate together
         const uint32_t i = i0 + lane;
         bool stall_bin;
@@ -312,19 +313,15 @@ __device__ __forceinline__ Sums sweep(ZoneSmem& sm, const TileCtx& c, const Seg&
                     const bool head = first_run && k1 >= 32;             // they would get the first run's outcome, else the common one
                     const int oc_x = head ? v.oc_h : v.oc_c;
                     const uint32_t tt_x = head ? v.tt_h : v.tt_c;
-                    long long tt_back = 0;
                     if (apart) {
                         Sums e;
                         clear(e);
                         add_outcome(e, -1, oc_x, q, tt_x);
                         enter_small(sm.j_sum[32], e);
-                        tt_back = e.tt;
+                        tt_back += e.tt;                                 // (entered once, when the sweep is over)
                         if (DBG_OK(bin_of_ticks(tt_x), kNBins, DBG_K_PAIRS_ZONES, DBG_BIN)) atomicSub(&sm.k_ttft[1][bin_of_ticks(tt_x)], 1);
                         if (oc_x >= O_MIGR_TO_DEV && stall_bin) atomicSub(&sm.k_stall[1][bin_of_ticks(q.stall)], 1);
                     }
-#pragma unroll
-                    for (int off = 16; off > 0; off >>= 1) tt_back += __shfl_xor_sync(0xFFFFFFFFu, tt_back, off);
-                    if (lane == 0) atomicAdd((unsigned long long*)&sm.e_sum[32][Z_TT], (unsigned long long)tt_back);
                 }
             }
             if (WAITS && c.wt_min != c.wt_max) {
@@ -358,6 +355,11 @@ __device__ __forceinline__ Sums sweep(ZoneSmem& sm, const TileCtx& c, const Seg&
             hist_add_each(sm.h_ttft, ok, bin_of_ticks(mine ? tt : v.tt_c));
             if (c.may_migrate) hist_add_each(sm.h_stall, ok && (mine ? oc : v.oc_c) >= O_MIGR_TO_DEV && stall_bin, bin_of_ticks(q.stall));
         }
+    }
+    if (WAITS && c.tile0_apart && point < 0) {
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) tt_back += __shfl_xor_sync(0xFFFFFFFFu, tt_back, off);
+        if (lane == 0 && tt_back) atomicAdd((unsigned long long*)&sm.e_sum[32][Z_TT], (unsigned long long)tt_back);
     }
     return d;
 }
